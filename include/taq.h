@@ -1,0 +1,195 @@
+/*
+ * taq.h - C ABI of the B200 (sm_100a) Trigger-Aware Quantization (TAQ) cross-attention library.
+ *
+ * The library computes one UNet cross-attention layer under TAQ (paper Sec. III-B): the projections run on
+ * packed low-bit weights; key/value rows of ordinary text tokens are int8 and the attention probabilities of
+ * ordinary tokens are uint8, while the rows and probability columns of the checkpoint's trigger tokens stay
+ * fp16 (Eq. 2 and Eq. 3).  Where the paper leaves the quantizer open the reading is: symmetric, dynamic,
+ * round-to-nearest-even, one scale per row (a row = the d_head elements of one token in one head) for
+ * Q/K/V, one scale per output channel (W8) or per group of 128 fan-in elements (W4) for weights, and the
+ * fixed range [0,1] with step 1/255 for probabilities.
+ *
+ * Conventions for every entry point
+ *   - Pointers named *_dev are DEVICE pointers owned by the caller; descriptors (the structs below) are HOST
+ *     pointers.  The library allocates and frees no device memory and keeps no reference to any buffer after
+ *     the call returns (the work itself runs asynchronously on `stream`).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls only enqueue work;
+ *     none synchronises except taq_poll_device_status.
+ *   - Every tensor pointer must be 16-byte aligned.  Tensors are dense, row-major, innermost index last.
+ *   - The return value is a taq_status; no exception, abort or device trap crosses the ABI.  All shape, size
+ *     and alignment checks happen on the host before anything is launched; taq_last_error() gives a message
+ *     for the last failing call of the calling thread.  Non-finite inputs give unspecified (but non-trapping)
+ *     results.  Identical inputs give bit-identical outputs.
+ */
+#ifndef TAQ_H_
+#define TAQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    TAQ_OK = 0,
+    TAQ_ERR_INVALID_ARG = 1,      /* null pointer, bad enum value, bad bit-width */
+    TAQ_ERR_SHAPE = 2,            /* a dimension is outside what the kernels support */
+    TAQ_ERR_ALIGNMENT = 3,        /* a pointer is not 16-byte aligned */
+    TAQ_ERR_BUFFER_TOO_SMALL = 4, /* packed / kv / workspace buffer smaller than the *_bytes() query says */
+    TAQ_ERR_UNSUPPORTED = 5,
+    TAQ_ERR_CUDA = 6,             /* a CUDA runtime call failed; message in taq_last_error() */
+    TAQ_ERR_TIMEOUT = 7           /* a bounded device-side wait gave up (see taq_poll_device_status) */
+} taq_status;
+
+/* Static strings; never NULL. */
+const char* taq_status_string(taq_status s);
+const char* taq_last_error(void);
+int taq_version(void);
+
+/* --------------------------------------------------------------------------------------------------------
+ * Weights (step "pack": per-output-channel symmetric round-to-nearest; bit-widths as in Table 1's W column,
+ * extended to 4 bits for the 4-8x memory claim of Sec. I).
+ *
+ * bits = 8: codes in [-127,127], one fp32 scale per output channel (group must be 0).
+ * bits = 4: codes in [-7,7], one fp32 scale per `group` consecutive fan-in elements of a channel (group = 0
+ *           means the whole row; otherwise a multiple of 32, typically 128; the last group may be shorter).
+ *   scale = absmax / qmax (fp32 division), code = clamp(rint(w / scale)) (fp32 division, ties to even);
+ *   an all-zero group has scale 0 and codes 0.
+ * Packed blob (relocatable, offsets from its start; every section 128-byte aligned):
+ *   [0,64)  header: u32 magic 'TAQW', version, n_out, k_in, bits, group, n_groups, has_bias; u64 off_codes,
+ *           off_scales, off_bias, total_bytes
+ *   codes   bits=8: int8 [n_out][k_in];  bits=4: u8 [n_out][k_in/2], fan-in element 2i in the low nibble and
+ *           2i+1 in the high nibble, each nibble = code + 8
+ *   scales  fp32 [n_out][n_groups]
+ *   bias    fp32 [n_out] (zeros when no bias was given)
+ * Restrictions: n_out >= 1, k_in a multiple of 8.
+ * -------------------------------------------------------------------------------------------------------- */
+typedef struct {
+    int32_t n_out;   /* output channels (rows of W) */
+    int32_t k_in;    /* fan-in (columns of W) */
+    int32_t bits;    /* 4 or 8 */
+    int32_t group;   /* 0 or the group length along fan-in */
+} taq_weight_desc;
+
+size_t taq_packed_weight_bytes(const taq_weight_desc* desc);   /* 0 if desc is invalid */
+
+/* W_dev: fp32 [n_out][k_in].  bias_dev: fp32 [n_out] or NULL.  packed_dev: >= taq_packed_weight_bytes(). */
+taq_status taq_pack_weights(const taq_weight_desc* desc, const float* W_dev, const float* bias_dev,
+                            void* packed_dev, size_t packed_bytes, void* stream);
+
+/* Test hook: expands a blob into int8 codes [n_out][k_in] and fp32 scales [n_out][n_groups]. */
+taq_status taq_unpack_weights(const taq_weight_desc* desc, const void* packed_dev, int8_t* codes_dev,
+                              float* scales_dev, void* stream);
+
+/* Stand-alone activation quantizer Q_a of Eq. 2: x fp32 [rows][cols] -> int8 codes [rows][cols] and fp32
+ * scales [rows]; qmax in [1,127].  Bit-exact with the definition above on identical fp32 inputs. */
+taq_status taq_quantize_rows(const float* x_dev, int64_t rows, int32_t cols, int32_t qmax,
+                             int8_t* codes_dev, float* scales_dev, void* stream);
+
+/* --------------------------------------------------------------------------------------------------------
+ * Layer description.  Notation of Sec. III-B: B sequences, N query (image) tokens, C = H * d channels,
+ * T text tokens of width Dc.
+ * -------------------------------------------------------------------------------------------------------- */
+typedef struct {
+    int32_t batch;        /* B */
+    int32_t n_query;      /* N */
+    int32_t channels;     /* C, a multiple of heads and of 8 */
+    int32_t heads;        /* H; d = C / H must be a multiple of 8, at most 256 */
+    int32_t n_ctx;        /* T <= 128 */
+    int32_t ctx_dim;      /* Dc, a multiple of 8 */
+    int32_t w_bits;       /* 4 or 8: format of all four packed projections of the layer */
+    int32_t w_group;      /* 0 or group length */
+    int32_t q_bits;       /* 8: Q~ = Q_a(Q) (Eq. 2, third line); 0: Q stays fp16 */
+    int32_t kv_bits;      /* 8 */
+    int32_t p_bits;       /* 8 */
+    int32_t max_trigger;  /* capacity of fp16 trigger rows per sequence, 0..n_ctx */
+} taq_layer_desc;
+
+/* Mixed-precision K~/V~ of Eq. 2, one block per sequence, blocks back to back.  Offsets inside a block: */
+typedef struct {
+    size_t block_bytes;
+    size_t off_k_codes;    /* int8 [H][T][d]   (rows of trigger tokens hold zeros) */
+    size_t off_v_codes;    /* int8 [H][T][d] */
+    size_t off_k_scales;   /* fp32 [H][T]      (0 for trigger rows) */
+    size_t off_v_scales;   /* fp32 [H][T] */
+    size_t off_k_trigger;  /* fp16 [max_trigger][H][d], slot order = increasing token position */
+    size_t off_v_trigger;  /* fp16 [max_trigger][H][d] */
+    size_t off_trig_slot;  /* int32 [128]: slot of token j, or -1 if j is an ordinary token */
+} taq_kv_layout;
+
+taq_status taq_kv_layout_of(const taq_layer_desc* desc, taq_kv_layout* out);
+size_t taq_kv_bytes(const taq_layer_desc* desc);               /* batch * block_bytes; 0 if invalid */
+
+/* Steps "K/V projection" and "TAQ K/V quantize" (Sec. III-B first paragraph; Eq. 2 lines 1-2):
+ * K = ctx Wk^T, V = ctx Wv^T per head; rows with trig_mask = 1 are stored as fp16, all others as int8 codes
+ * with one scale per (sequence, head, token).  Done once per prompt: K/V do not depend on the image tokens.
+ *   ctx_f16_dev  fp16 [B][T][Dc];  Wk_packed/Wv_packed: blobs of shape [C][Dc] in the layer's weight format
+ *   trig_mask_dev u8 [B][T], 1 = trigger token (M_KV; the same for every head and channel)
+ *   kv_packed_dev >= taq_kv_bytes().
+ * A sequence with more than max_trigger trigger tokens raises the device status word (TAQ_ERR_SHAPE). */
+taq_status taq_kv_project(const taq_layer_desc* desc, const void* ctx_f16_dev, const void* Wk_packed_dev,
+                          const void* Wv_packed_dev, const uint8_t* trig_mask_dev, void* kv_packed_dev,
+                          size_t kv_bytes, void* stream);
+
+/* Dequant-GEMM on packed weights (the to_q / to_out projections; "quantizing all remaining ... pathways",
+ * Sec. III-B last paragraph): y = x W^T (+ bias), W^ = fp16(code * scale) as the matrix operand, fp32
+ * accumulation.
+ *   x_f16_dev fp16 [rows][k_in]
+ *   out_kind TAQ_OUT_F16: y fp16 [rows][n_out], bias added.  TAQ_OUT_F32: y fp32, bias added.
+ *   TAQ_OUT_INT8_HEAD_ROWS: the Q~ = Q_a(Q) epilogue - y int8 [rows][n_out], scales_dev fp32 [rows][heads],
+ *   one scale per row of n_out/heads elements; bias is ignored. */
+typedef enum { TAQ_OUT_F16 = 0, TAQ_OUT_F32 = 1, TAQ_OUT_INT8_HEAD_ROWS = 2 } taq_out_kind;
+
+taq_status taq_quantized_linear(const taq_weight_desc* desc, const void* x_f16_dev, int64_t rows,
+                                const void* W_packed_dev, void* y_dev, int32_t out_kind, int32_t heads,
+                                float* scales_dev, void* stream);
+
+/* Fused attention core: A = softmax(Q~ K~^T / sqrt(d)) per head, Eq. 3 (probabilities of ordinary tokens
+ * -> uint8 codes / 255, columns of trigger tokens kept in fp16), O = A^ V~, heads concatenated.  Scores and
+ * probabilities never reach global memory.
+ *   q_dev        q_bits = 8: int8 [B][N][C] with q_scales_dev fp32 [B][N][H];  q_bits = 0: fp16 [B][N][C]
+ *   kv_packed_dev as written by taq_kv_project;  trig_mask_dev u8 [B][T] (M_A: same positions)
+ *   o_f16_dev    fp16 [B][N][C] */
+taq_status taq_cross_attention(const taq_layer_desc* desc, const void* q_dev, const float* q_scales_dev,
+                               const void* kv_packed_dev, const uint8_t* trig_mask_dev, void* o_f16_dev,
+                               void* stream);
+
+/* One denoising-step pass of the layer, K~/V~ already projected: to_q (+ Q_a), attention, to_out (+ bias).
+ *   x_f16_dev fp16 [B][N][C] -> y_f16_dev fp16 [B][N][C];  Wq/Wout blobs of shape [C][C]
+ *   workspace_dev >= taq_workspace_bytes(desc, 1), 128-byte aligned; contents are scratch. */
+size_t taq_workspace_bytes(const taq_layer_desc* desc, int32_t n_requests);
+taq_status taq_layer_forward(const taq_layer_desc* desc, const void* x_f16_dev, const void* Wq_packed_dev,
+                             const void* Wout_packed_dev, const void* kv_packed_dev,
+                             const uint8_t* trig_mask_dev, void* y_f16_dev, void* workspace_dev,
+                             size_t workspace_bytes, void* stream);
+
+/* Batched serving (Sec. I: many personalized checkpoints served concurrently): request r is one sequence
+ * (desc->batch must be 1) whose activations are slice r of x/y [n_requests][N][C] and which carries its own
+ * checkpoint's packed weights, its own K~/V~ block and its own trigger mask.  `reqs_dev` is a DEVICE array of
+ * n_requests entries of device pointers. */
+typedef struct {
+    const void* Wq;             /* packed [C][C] */
+    const void* Wout;           /* packed [C][C] */
+    const void* kv;             /* one K~/V~ block */
+    const uint8_t* trig_mask;   /* u8 [T] */
+} taq_request;
+
+taq_status taq_layer_forward_batched(const taq_layer_desc* desc, const taq_request* reqs_dev, int32_t n_requests,
+                                     const void* x_f16_dev, void* y_f16_dev, void* workspace_dev,
+                                     size_t workspace_bytes, void* stream);
+
+/* Batched admission: K~/V~ for n_requests prompts, each with its own Wk/Wv and mask.  `reqs_dev[r].Wq` and
+ * `.Wout` are read as Wk and Wv here; `.kv` is the output block; ctx fp16 [n_requests][T][Dc]. */
+taq_status taq_kv_project_batched(const taq_layer_desc* desc, const taq_request* reqs_dev, int32_t n_requests,
+                                  const void* ctx_f16_dev, void* stream);
+
+/* Device status word: kernels never trap; a bounded wait that runs out or a capacity violation records a code
+ * and the block that saw it.  This call synchronises `stream`, returns that code (TAQ_OK if none) and clears
+ * it.  block_id_out may be NULL. */
+taq_status taq_poll_device_status(void* stream, int32_t* block_id_out);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TAQ_H_ */

@@ -1,0 +1,250 @@
+"""ctypes binding of ``libtaq.so``: the same entry points as ``include/taq.h``, taking torch CUDA tensors.
+
+Only argument marshalling happens here (pointers, sizes, the current CUDA stream); every step of the TAQ
+cross-attention path runs in the library's kernels.  There is no CPU path: a missing library raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libtaq.so")
+
+TAQ_OK = 0
+TAQ_ERR_INVALID_ARG, TAQ_ERR_SHAPE, TAQ_ERR_ALIGNMENT, TAQ_ERR_BUFFER_TOO_SMALL = 1, 2, 3, 4
+TAQ_ERR_UNSUPPORTED, TAQ_ERR_CUDA, TAQ_ERR_TIMEOUT = 5, 6, 7
+TAQ_OUT_F16, TAQ_OUT_F32, TAQ_OUT_INT8_HEAD_ROWS = 0, 1, 2
+
+EXPORTS = [
+    "taq_status_string", "taq_last_error", "taq_version", "taq_packed_weight_bytes", "taq_pack_weights",
+    "taq_unpack_weights", "taq_quantize_rows", "taq_kv_layout_of", "taq_kv_bytes", "taq_kv_project",
+    "taq_quantized_linear", "taq_cross_attention", "taq_workspace_bytes", "taq_layer_forward",
+    "taq_layer_forward_batched", "taq_kv_project_batched", "taq_poll_device_status",
+]
+
+
+class TaqError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"taq status {status}: {message}")
+        self.status = status
+
+
+class WeightDesc(C.Structure):
+    _fields_ = [("n_out", C.c_int32), ("k_in", C.c_int32), ("bits", C.c_int32), ("group", C.c_int32)]
+
+
+class LayerDesc(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("batch", "n_query", "channels", "heads", "n_ctx", "ctx_dim", "w_bits",
+                                          "w_group", "q_bits", "kv_bits", "p_bits", "max_trigger")]
+
+    @property
+    def d_head(self) -> int:
+        return self.channels // self.heads
+
+
+class KvLayout(C.Structure):
+    _fields_ = [(n, C.c_size_t) for n in ("block_bytes", "off_k_codes", "off_v_codes", "off_k_scales", "off_v_scales",
+                                           "off_k_trigger", "off_v_trigger", "off_trig_slot")]
+
+
+class Request(C.Structure):
+    _fields_ = [("Wq", C.c_void_p), ("Wout", C.c_void_p), ("kv", C.c_void_p), ("trig_mask", C.c_void_p)]
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Loads the shared library on first use.  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2603_22943_b200.build` "
+                               "(there is no fallback path)")
+        L = C.CDLL(LIB_PATH)
+        vp, sz, i32, i64 = C.c_void_p, C.c_size_t, C.c_int32, C.c_int64
+        L.taq_status_string.restype = C.c_char_p
+        L.taq_status_string.argtypes = [C.c_int]
+        L.taq_last_error.restype = C.c_char_p
+        L.taq_last_error.argtypes = []
+        L.taq_version.restype = C.c_int
+        L.taq_packed_weight_bytes.restype = sz
+        L.taq_packed_weight_bytes.argtypes = [C.POINTER(WeightDesc)]
+        L.taq_pack_weights.argtypes = [C.POINTER(WeightDesc), vp, vp, vp, sz, vp]
+        L.taq_unpack_weights.argtypes = [C.POINTER(WeightDesc), vp, vp, vp, vp]
+        L.taq_quantize_rows.argtypes = [vp, i64, i32, i32, vp, vp, vp]
+        L.taq_kv_layout_of.argtypes = [C.POINTER(LayerDesc), C.POINTER(KvLayout)]
+        L.taq_kv_bytes.restype = sz
+        L.taq_kv_bytes.argtypes = [C.POINTER(LayerDesc)]
+        L.taq_kv_project.argtypes = [C.POINTER(LayerDesc), vp, vp, vp, vp, vp, sz, vp]
+        L.taq_quantized_linear.argtypes = [C.POINTER(WeightDesc), vp, i64, vp, vp, i32, i32, vp, vp]
+        L.taq_cross_attention.argtypes = [C.POINTER(LayerDesc), vp, vp, vp, vp, vp, vp]
+        L.taq_workspace_bytes.restype = sz
+        L.taq_workspace_bytes.argtypes = [C.POINTER(LayerDesc), i32]
+        L.taq_layer_forward.argtypes = [C.POINTER(LayerDesc), vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.taq_layer_forward_batched.argtypes = [C.POINTER(LayerDesc), vp, i32, vp, vp, vp, sz, vp]
+        L.taq_kv_project_batched.argtypes = [C.POINTER(LayerDesc), vp, i32, vp, vp]
+        L.taq_poll_device_status.argtypes = [vp, C.POINTER(i32)]
+        for name in EXPORTS:
+            f = getattr(L, name)
+            if f.restype is C.c_int and name not in ("taq_version",):
+                f.restype = C.c_int
+        _lib = L
+    return _lib
+
+
+def _check(status: int) -> None:
+    if status != TAQ_OK:
+        raise TaqError(status, lib().taq_last_error().decode())
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise TypeError("device tensor expected")
+    if not t.is_contiguous():
+        raise TypeError("contiguous tensor expected")
+    return t.data_ptr()
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def weight_desc(n_out: int, k_in: int, bits: int, group: int) -> WeightDesc:
+    return WeightDesc(n_out, k_in, bits, group)
+
+
+def layer_desc(batch, n_query, channels, heads, n_ctx, ctx_dim, w_bits, w_group, q_bits=8, kv_bits=8, p_bits=8,
+               max_trigger=8) -> LayerDesc:
+    return LayerDesc(batch, n_query, channels, heads, n_ctx, ctx_dim, w_bits, w_group, q_bits, kv_bits, p_bits, max_trigger)
+
+
+# ------------------------------------------------------------------------------------------------
+# Entry points (same names as the C ABI)
+# ------------------------------------------------------------------------------------------------
+
+def taq_packed_weight_bytes(desc: WeightDesc) -> int:
+    return lib().taq_packed_weight_bytes(C.byref(desc))
+
+
+def taq_pack_weights(desc: WeightDesc, W: torch.Tensor, bias: Optional[torch.Tensor] = None,
+                     packed: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """W fp32 [n_out,k_in] -> packed blob (uint8 tensor)."""
+    nbytes = taq_packed_weight_bytes(desc)
+    if packed is None:
+        if nbytes == 0:
+            _check(lib().taq_pack_weights(C.byref(desc), _ptr(W), _ptr(bias), None, 0, _stream(stream)))
+        packed = torch.zeros(nbytes, dtype=torch.uint8, device=W.device)
+    _check(lib().taq_pack_weights(C.byref(desc), _ptr(W), _ptr(bias), _ptr(packed), packed.numel(), _stream(stream)))
+    return packed
+
+
+def taq_unpack_weights(desc: WeightDesc, packed: torch.Tensor, stream=None):
+    g = desc.k_in if desc.group == 0 else desc.group
+    n_groups = (desc.k_in + g - 1) // g
+    codes = torch.empty((desc.n_out, desc.k_in), dtype=torch.int8, device=packed.device)
+    scales = torch.empty((desc.n_out, n_groups), dtype=torch.float32, device=packed.device)
+    _check(lib().taq_unpack_weights(C.byref(desc), _ptr(packed), _ptr(codes), _ptr(scales), _stream(stream)))
+    return codes, scales
+
+
+def taq_quantize_rows(x: torch.Tensor, qmax: int = 127, stream=None):
+    """x fp32 [rows, cols] -> (int8 codes, fp32 scales)."""
+    rows, cols = x.shape
+    codes = torch.empty((rows, cols), dtype=torch.int8, device=x.device)
+    scales = torch.empty((rows,), dtype=torch.float32, device=x.device)
+    _check(lib().taq_quantize_rows(_ptr(x), rows, cols, qmax, _ptr(codes), _ptr(scales), _stream(stream)))
+    return codes, scales
+
+
+def taq_kv_layout_of(desc: LayerDesc) -> KvLayout:
+    out = KvLayout()
+    _check(lib().taq_kv_layout_of(C.byref(desc), C.byref(out)))
+    return out
+
+
+def taq_kv_bytes(desc: LayerDesc) -> int:
+    return lib().taq_kv_bytes(C.byref(desc))
+
+
+def taq_kv_project(desc: LayerDesc, ctx: torch.Tensor, Wk_packed: torch.Tensor, Wv_packed: torch.Tensor,
+                   trig_mask: torch.Tensor, kv: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    if kv is None:
+        kv = torch.zeros(max(taq_kv_bytes(desc), 16), dtype=torch.uint8, device=ctx.device)
+    _check(lib().taq_kv_project(C.byref(desc), _ptr(ctx), _ptr(Wk_packed), _ptr(Wv_packed), _ptr(trig_mask), _ptr(kv),
+                                kv.numel(), _stream(stream)))
+    return kv
+
+
+def taq_quantized_linear(desc: WeightDesc, x: torch.Tensor, W_packed: torch.Tensor, out_kind: int = TAQ_OUT_F16,
+                         heads: int = 1, y: Optional[torch.Tensor] = None, scales: Optional[torch.Tensor] = None, stream=None):
+    rows = x.numel() // desc.k_in
+    if y is None:
+        dt = {TAQ_OUT_F16: torch.float16, TAQ_OUT_F32: torch.float32, TAQ_OUT_INT8_HEAD_ROWS: torch.int8}[out_kind]
+        y = torch.empty((rows, desc.n_out), dtype=dt, device=x.device)
+    if out_kind == TAQ_OUT_INT8_HEAD_ROWS and scales is None:
+        scales = torch.empty((rows, heads), dtype=torch.float32, device=x.device)
+    _check(lib().taq_quantized_linear(C.byref(desc), _ptr(x), rows, _ptr(W_packed), _ptr(y), out_kind, heads, _ptr(scales), _stream(stream)))
+    return (y, scales) if out_kind == TAQ_OUT_INT8_HEAD_ROWS else y
+
+
+def taq_cross_attention(desc: LayerDesc, q: torch.Tensor, q_scales: Optional[torch.Tensor], kv: torch.Tensor,
+                        trig_mask: torch.Tensor, o: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    if o is None:
+        o = torch.empty((desc.batch, desc.n_query, desc.channels), dtype=torch.float16, device=kv.device)
+    _check(lib().taq_cross_attention(C.byref(desc), _ptr(q), _ptr(q_scales), _ptr(kv), _ptr(trig_mask), _ptr(o), _stream(stream)))
+    return o
+
+
+def taq_workspace_bytes(desc: LayerDesc, n_requests: int = 1) -> int:
+    return lib().taq_workspace_bytes(C.byref(desc), n_requests)
+
+
+def taq_layer_forward(desc: LayerDesc, x: torch.Tensor, Wq_packed: torch.Tensor, Wout_packed: torch.Tensor, kv: torch.Tensor,
+                      trig_mask: torch.Tensor, y: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                      stream=None) -> torch.Tensor:
+    if y is None:
+        y = torch.empty((desc.batch, desc.n_query, desc.channels), dtype=torch.float16, device=x.device)
+    if workspace is None:
+        workspace = torch.empty(max(taq_workspace_bytes(desc, 1), 128), dtype=torch.uint8, device=x.device)
+    _check(lib().taq_layer_forward(C.byref(desc), _ptr(x), _ptr(Wq_packed), _ptr(Wout_packed), _ptr(kv), _ptr(trig_mask), _ptr(y),
+                                   _ptr(workspace), workspace.numel(), _stream(stream)))
+    return y
+
+
+def make_request_table(entries: Sequence[Sequence[torch.Tensor]], device) -> torch.Tensor:
+    """Device array of taq_request from (Wq, Wout, kv, mask) tensor tuples (4 pointers per entry)."""
+    flat = []
+    for e in entries:
+        flat.extend(int(t.data_ptr()) for t in e)
+    return torch.tensor(flat, dtype=torch.int64).to(device)
+
+
+def taq_layer_forward_batched(desc: LayerDesc, reqs: torch.Tensor, n_requests: int, x: torch.Tensor,
+                              y: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    if y is None:
+        y = torch.empty((n_requests, desc.n_query, desc.channels), dtype=torch.float16, device=x.device)
+    if workspace is None:
+        workspace = torch.empty(max(taq_workspace_bytes(desc, n_requests), 128), dtype=torch.uint8, device=x.device)
+    _check(lib().taq_layer_forward_batched(C.byref(desc), _ptr(reqs), n_requests, _ptr(x), _ptr(y), _ptr(workspace),
+                                           workspace.numel(), _stream(stream)))
+    return y
+
+
+def taq_kv_project_batched(desc: LayerDesc, reqs: torch.Tensor, n_requests: int, ctx: torch.Tensor, stream=None) -> None:
+    _check(lib().taq_kv_project_batched(C.byref(desc), _ptr(reqs), n_requests, _ptr(ctx), _stream(stream)))
+
+
+def taq_poll_device_status(stream=None) -> int:
+    """Synchronises the stream; raises TaqError if a kernel recorded a device-side error."""
+    blk = C.c_int32(-1)
+    _check(lib().taq_poll_device_status(_stream(stream), C.byref(blk)))
+    return TAQ_OK

@@ -1,0 +1,389 @@
+// C ABI of the TAQ library: host-side validation and kernel dispatch.  Nothing here allocates device memory.
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+
+#include "taq_common.cuh"
+#include "taq_sm100.cuh"
+
+namespace taq {
+
+__device__ int g_status_word[2];   // {code, block id}; raised by kernels, read by taq_poll_device_status
+
+static thread_local char tl_error[512] = "";
+
+static taq_status fail(taq_status s, const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(tl_error, sizeof(tl_error), fmt, ap);
+    va_end(ap);
+    return s;
+}
+
+static taq_status cuda_fail(cudaError_t e, const char* what) {
+    return fail(TAQ_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Address of the status word on the current device (looked up once per device).
+static taq_status status_ptr(int** out) {
+    static int* cache[64] = {nullptr};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+    if (dev < 0 || dev >= 64) return fail(TAQ_ERR_UNSUPPORTED, "device ordinal %d out of range", dev);
+    if (!cache[dev]) {
+        void* p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_status_word);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaGetSymbolAddress(status word)");
+        cache[dev] = static_cast<int*>(p);
+    }
+    *out = cache[dev];
+    return TAQ_OK;
+}
+
+static taq_status check_weight_desc(const taq_weight_desc* d) {
+    if (!d) return fail(TAQ_ERR_INVALID_ARG, "weight descriptor is NULL");
+    if (d->bits != 4 && d->bits != 8) return fail(TAQ_ERR_INVALID_ARG, "bits must be 4 or 8, got %d", d->bits);
+    if (d->n_out < 1 || d->k_in < 8 || d->k_in % 8) return fail(TAQ_ERR_SHAPE, "n_out >= 1 and k_in a positive multiple of 8 required (n_out=%d k_in=%d)", d->n_out, d->k_in);
+    if (d->group < 0 || (d->group && d->group % 32)) return fail(TAQ_ERR_SHAPE, "group must be 0 or a multiple of 32, got %d", d->group);
+    if (d->bits == 8 && d->group != 0) return fail(TAQ_ERR_UNSUPPORTED, "8-bit weights take one scale per output channel (group = 0)");
+    if ((long long)d->n_out * d->k_in > (1LL << 40)) return fail(TAQ_ERR_SHAPE, "matrix too large");
+    return TAQ_OK;
+}
+
+static taq_status check_layer_desc(const taq_layer_desc* d) {
+    if (!d) return fail(TAQ_ERR_INVALID_ARG, "layer descriptor is NULL");
+    if (d->batch < 0 || d->n_query < 0) return fail(TAQ_ERR_SHAPE, "negative batch or n_query");
+    if (d->heads < 1 || d->channels < 8 || d->channels % d->heads) return fail(TAQ_ERR_SHAPE, "channels (%d) must be a positive multiple of heads (%d)", d->channels, d->heads);
+    const int dh = d->channels / d->heads;
+    if (dh % 8 || dh > kMaxHeadDim) return fail(TAQ_ERR_SHAPE, "head width %d must be a multiple of 8, at most %d", dh, kMaxHeadDim);
+    if (d->n_ctx < 1 || d->n_ctx > kMaxCtx) return fail(TAQ_ERR_SHAPE, "n_ctx must be in [1,%d], got %d", kMaxCtx, d->n_ctx);
+    if (d->ctx_dim < 8 || d->ctx_dim % 8) return fail(TAQ_ERR_SHAPE, "ctx_dim must be a positive multiple of 8, got %d", d->ctx_dim);
+    if (d->w_bits != 4 && d->w_bits != 8) return fail(TAQ_ERR_INVALID_ARG, "w_bits must be 4 or 8, got %d", d->w_bits);
+    if (d->q_bits != 0 && d->q_bits != 8) return fail(TAQ_ERR_INVALID_ARG, "q_bits must be 0 or 8, got %d", d->q_bits);
+    if (d->kv_bits != 8) return fail(TAQ_ERR_UNSUPPORTED, "kv_bits must be 8, got %d", d->kv_bits);
+    if (d->p_bits != 8) return fail(TAQ_ERR_UNSUPPORTED, "p_bits must be 8, got %d", d->p_bits);
+    if (d->max_trigger < 0 || d->max_trigger > d->n_ctx) return fail(TAQ_ERR_SHAPE, "max_trigger must be in [0,n_ctx], got %d", d->max_trigger);
+    if ((long long)d->batch * d->n_query > (1LL << 31) - 1) return fail(TAQ_ERR_SHAPE, "batch * n_query too large");
+    taq_weight_desc w{d->channels, d->channels, d->w_bits, d->w_group};
+    return check_weight_desc(&w);
+}
+
+#define TAQ_REQUIRE_PTR(p)                                                              \
+    do {                                                                                \
+        if (!(p)) return fail(TAQ_ERR_INVALID_ARG, #p " is NULL");                      \
+        if (!aligned16(p)) return fail(TAQ_ERR_ALIGNMENT, #p " is not 16-byte aligned"); \
+    } while (0)
+
+// Workspace of taq_layer_forward: Q~ (int8 or fp16), its scales, O (fp16); each section 128-byte aligned.
+struct Workspace { size_t off_q, off_qs, off_o, total; };
+static Workspace workspace_layout(const taq_layer_desc* d, int n_requests) {
+    const size_t rows = (size_t)d->batch * d->n_query * n_requests;
+    Workspace w;
+    w.off_q = 0;
+    w.off_qs = align_up(rows * d->channels * (d->q_bits == 8 ? 1 : 2), 128);
+    w.off_o = w.off_qs + align_up(rows * d->heads * sizeof(float), 128);
+    w.total = w.off_o + align_up(rows * d->channels * sizeof(__half), 128);
+    return w;
+}
+
+static taq_status run_linear(const LinearArgs& a, int n_z, cudaStream_t st) {
+    cudaError_t e;
+    if (sm100_linear_supported(a)) e = launch_linear_sm100(a, n_z, st);
+    else e = launch_linear_simt(a, n_z, st);
+    return e == cudaSuccess ? TAQ_OK : cuda_fail(e, "dequant-GEMM launch");
+}
+
+static taq_status run_attention(const AttnArgs& a, int n_z, cudaStream_t st) {
+    cudaError_t e;
+    if (sm100_attention_supported(a)) e = launch_attention_sm100(a, n_z, st);
+    else e = launch_attention_simt(a, n_z, st);
+    return e == cudaSuccess ? TAQ_OK : cuda_fail(e, "attention launch");
+}
+
+}  // namespace taq
+
+using namespace taq;
+
+extern "C" {
+
+const char* taq_status_string(taq_status s) {
+    switch (s) {
+        case TAQ_OK: return "ok";
+        case TAQ_ERR_INVALID_ARG: return "invalid argument";
+        case TAQ_ERR_SHAPE: return "unsupported shape";
+        case TAQ_ERR_ALIGNMENT: return "misaligned pointer";
+        case TAQ_ERR_BUFFER_TOO_SMALL: return "buffer too small";
+        case TAQ_ERR_UNSUPPORTED: return "unsupported";
+        case TAQ_ERR_CUDA: return "CUDA error";
+        case TAQ_ERR_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+const char* taq_last_error(void) { return tl_error; }
+int taq_version(void) { return 1; }
+
+size_t taq_packed_weight_bytes(const taq_weight_desc* d) {
+    if (check_weight_desc(d) != TAQ_OK) return 0;
+    return weight_layout(d->n_out, d->k_in, d->bits, d->group).total;
+}
+
+taq_status taq_pack_weights(const taq_weight_desc* d, const float* W_dev, const float* bias_dev, void* packed_dev,
+                            size_t packed_bytes, void* stream) {
+    taq_status s = check_weight_desc(d);
+    if (s != TAQ_OK) return s;
+    TAQ_REQUIRE_PTR(W_dev);
+    TAQ_REQUIRE_PTR(packed_dev);
+    if (bias_dev && !aligned16(bias_dev)) return fail(TAQ_ERR_ALIGNMENT, "bias_dev is not 16-byte aligned");
+    const size_t need = taq_packed_weight_bytes(d);
+    if (packed_bytes < need) return fail(TAQ_ERR_BUFFER_TOO_SMALL, "packed buffer has %zu bytes, %zu needed", packed_bytes, need);
+    cudaError_t e = launch_pack_weights(*d, W_dev, bias_dev, packed_dev, (cudaStream_t)stream);
+    return e == cudaSuccess ? TAQ_OK : cuda_fail(e, "pack_weights launch");
+}
+
+taq_status taq_unpack_weights(const taq_weight_desc* d, const void* packed_dev, int8_t* codes_dev, float* scales_dev, void* stream) {
+    taq_status s = check_weight_desc(d);
+    if (s != TAQ_OK) return s;
+    TAQ_REQUIRE_PTR(packed_dev);
+    TAQ_REQUIRE_PTR(codes_dev);
+    TAQ_REQUIRE_PTR(scales_dev);
+    cudaError_t e = launch_unpack_weights(*d, packed_dev, codes_dev, scales_dev, (cudaStream_t)stream);
+    return e == cudaSuccess ? TAQ_OK : cuda_fail(e, "unpack_weights launch");
+}
+
+taq_status taq_quantize_rows(const float* x_dev, int64_t rows, int32_t cols, int32_t qmax, int8_t* codes_dev, float* scales_dev, void* stream) {
+    if (rows < 0 || cols < 1) return fail(TAQ_ERR_SHAPE, "rows >= 0 and cols >= 1 required (rows=%lld cols=%d)", (long long)rows, cols);
+    if (qmax < 1 || qmax > 127) return fail(TAQ_ERR_INVALID_ARG, "qmax must be in [1,127], got %d", qmax);
+    if (rows == 0) return TAQ_OK;
+    TAQ_REQUIRE_PTR(x_dev);
+    TAQ_REQUIRE_PTR(codes_dev);
+    TAQ_REQUIRE_PTR(scales_dev);
+    cudaError_t e = launch_quantize_rows(x_dev, rows, cols, qmax, codes_dev, scales_dev, (cudaStream_t)stream);
+    return e == cudaSuccess ? TAQ_OK : cuda_fail(e, "quantize_rows launch");
+}
+
+taq_status taq_kv_layout_of(const taq_layer_desc* d, taq_kv_layout* out) {
+    taq_status s = check_layer_desc(d);
+    if (s != TAQ_OK) return s;
+    if (!out) return fail(TAQ_ERR_INVALID_ARG, "out is NULL");
+    *out = kv_layout(d->heads, d->n_ctx, d->channels / d->heads, d->max_trigger);
+    return TAQ_OK;
+}
+
+size_t taq_kv_bytes(const taq_layer_desc* d) {
+    if (check_layer_desc(d) != TAQ_OK) return 0;
+    return kv_layout(d->heads, d->n_ctx, d->channels / d->heads, d->max_trigger).block_bytes * (size_t)d->batch;
+}
+
+static taq_status kv_project_impl(const taq_layer_desc* d, const taq_request* reqs, int n_z, const void* ctx, const void* Wk,
+                                  const void* Wv, const uint8_t* mask, void* kv, cudaStream_t st) {
+    int* status = nullptr;
+    taq_status s = status_ptr(&status);
+    if (s != TAQ_OK) return s;
+    LinearArgs a{};
+    a.x = (const __half*)ctx;
+    a.reqs = reqs;
+    a.y = kv;
+    a.mask = mask;
+    a.rows = (long long)d->batch * d->n_ctx;
+    a.n_out = d->channels; a.k_in = d->ctx_dim; a.bits = d->w_bits; a.group = d->w_group;
+    a.heads = d->heads; a.n_ctx = d->n_ctx; a.max_trigger = d->max_trigger;
+    a.epi = EPI_KV;
+    a.status = status;
+    for (int which = 0; which < 2; ++which) {
+        a.w = which ? Wv : Wk;
+        a.which = which;
+        a.kv_which = which;
+        s = run_linear(a, n_z, st);
+        if (s != TAQ_OK) return s;
+    }
+    return TAQ_OK;
+}
+
+taq_status taq_kv_project(const taq_layer_desc* d, const void* ctx_f16_dev, const void* Wk_packed_dev, const void* Wv_packed_dev,
+                          const uint8_t* trig_mask_dev, void* kv_packed_dev, size_t kv_bytes, void* stream) {
+    taq_status s = check_layer_desc(d);
+    if (s != TAQ_OK) return s;
+    if (d->batch == 0) return TAQ_OK;
+    TAQ_REQUIRE_PTR(ctx_f16_dev);
+    TAQ_REQUIRE_PTR(Wk_packed_dev);
+    TAQ_REQUIRE_PTR(Wv_packed_dev);
+    TAQ_REQUIRE_PTR(kv_packed_dev);
+    if (!trig_mask_dev) return fail(TAQ_ERR_INVALID_ARG, "trig_mask_dev is NULL");
+    const size_t need = taq_kv_bytes(d);
+    if (kv_bytes < need) return fail(TAQ_ERR_BUFFER_TOO_SMALL, "kv buffer has %zu bytes, %zu needed", kv_bytes, need);
+    return kv_project_impl(d, nullptr, 1, ctx_f16_dev, Wk_packed_dev, Wv_packed_dev, trig_mask_dev, kv_packed_dev, (cudaStream_t)stream);
+}
+
+taq_status taq_kv_project_batched(const taq_layer_desc* d, const taq_request* reqs_dev, int32_t n_requests, const void* ctx_f16_dev, void* stream) {
+    taq_status s = check_layer_desc(d);
+    if (s != TAQ_OK) return s;
+    if (d->batch != 1) return fail(TAQ_ERR_SHAPE, "batched calls take one sequence per request (desc->batch must be 1)");
+    if (n_requests < 0 || n_requests > 65535) return fail(TAQ_ERR_SHAPE, "n_requests must be in [0,65535]");
+    if (n_requests == 0) return TAQ_OK;
+    TAQ_REQUIRE_PTR(reqs_dev);
+    TAQ_REQUIRE_PTR(ctx_f16_dev);
+    return kv_project_impl(d, reqs_dev, n_requests, ctx_f16_dev, nullptr, nullptr, nullptr, nullptr, (cudaStream_t)stream);
+}
+
+taq_status taq_quantized_linear(const taq_weight_desc* d, const void* x_f16_dev, int64_t rows, const void* W_packed_dev, void* y_dev,
+                                int32_t out_kind, int32_t heads, float* scales_dev, void* stream) {
+    taq_status s = check_weight_desc(d);
+    if (s != TAQ_OK) return s;
+    if (rows < 0 || rows > (1LL << 31) - 1) return fail(TAQ_ERR_SHAPE, "rows out of range");
+    if (out_kind != TAQ_OUT_F16 && out_kind != TAQ_OUT_F32 && out_kind != TAQ_OUT_INT8_HEAD_ROWS) return fail(TAQ_ERR_INVALID_ARG, "unknown out_kind %d", out_kind);
+    if (d->n_out % 8) return fail(TAQ_ERR_SHAPE, "n_out must be a multiple of 8 for a dequant-GEMM, got %d", d->n_out);
+    if (out_kind == TAQ_OUT_INT8_HEAD_ROWS) {
+        if (heads < 1 || d->n_out % heads) return fail(TAQ_ERR_SHAPE, "n_out (%d) must be a multiple of heads (%d)", d->n_out, heads);
+        const int dh = d->n_out / heads;
+        if (dh % 8 || dh > kMaxHeadDim) return fail(TAQ_ERR_SHAPE, "head width %d must be a multiple of 8, at most %d", dh, kMaxHeadDim);
+        if (heads > 65535) return fail(TAQ_ERR_SHAPE, "too many heads");
+    }
+    if (rows == 0) return TAQ_OK;
+    TAQ_REQUIRE_PTR(x_f16_dev);
+    TAQ_REQUIRE_PTR(W_packed_dev);
+    TAQ_REQUIRE_PTR(y_dev);
+    if (out_kind == TAQ_OUT_INT8_HEAD_ROWS) TAQ_REQUIRE_PTR(scales_dev);
+    int* status = nullptr;
+    s = status_ptr(&status);
+    if (s != TAQ_OK) return s;
+    LinearArgs a{};
+    a.x = (const __half*)x_f16_dev;
+    a.w = W_packed_dev;
+    a.y = y_dev;
+    a.scales = scales_dev;
+    a.rows = rows;
+    a.n_out = d->n_out; a.k_in = d->k_in; a.bits = d->bits; a.group = d->group;
+    a.heads = out_kind == TAQ_OUT_INT8_HEAD_ROWS ? heads : 1;
+    a.epi = out_kind == TAQ_OUT_F16 ? EPI_F16 : out_kind == TAQ_OUT_F32 ? EPI_F32 : EPI_Q8_HEAD;
+    a.status = status;
+    return run_linear(a, 1, (cudaStream_t)stream);
+}
+
+static AttnArgs attn_args(const taq_layer_desc* d, int* status) {
+    AttnArgs a{};
+    a.batch = d->batch; a.n_query = d->n_query; a.channels = d->channels; a.heads = d->heads; a.n_ctx = d->n_ctx;
+    a.max_trigger = d->max_trigger; a.q_bits = d->q_bits; a.p_bits = d->p_bits;
+    a.status = status;
+    return a;
+}
+
+taq_status taq_cross_attention(const taq_layer_desc* d, const void* q_dev, const float* q_scales_dev, const void* kv_packed_dev,
+                               const uint8_t* trig_mask_dev, void* o_f16_dev, void* stream) {
+    taq_status s = check_layer_desc(d);
+    if (s != TAQ_OK) return s;
+    if (d->batch > 65535) return fail(TAQ_ERR_SHAPE, "batch must be at most 65535");
+    if (d->batch == 0 || d->n_query == 0) return TAQ_OK;
+    TAQ_REQUIRE_PTR(q_dev);
+    if (d->q_bits == 8) TAQ_REQUIRE_PTR(q_scales_dev);
+    TAQ_REQUIRE_PTR(kv_packed_dev);
+    TAQ_REQUIRE_PTR(o_f16_dev);
+    if (!trig_mask_dev) return fail(TAQ_ERR_INVALID_ARG, "trig_mask_dev is NULL");
+    int* status = nullptr;
+    s = status_ptr(&status);
+    if (s != TAQ_OK) return s;
+    AttnArgs a = attn_args(d, status);
+    a.q = q_dev; a.q_scales = q_scales_dev; a.kv = kv_packed_dev; a.mask = trig_mask_dev; a.o = (__half*)o_f16_dev;
+    return run_attention(a, d->batch, (cudaStream_t)stream);
+}
+
+size_t taq_workspace_bytes(const taq_layer_desc* d, int32_t n_requests) {
+    if (check_layer_desc(d) != TAQ_OK || n_requests < 1) return 0;
+    return workspace_layout(d, n_requests).total;
+}
+
+static taq_status layer_forward_impl(const taq_layer_desc* d, const taq_request* reqs, int n_req, const void* x, const void* Wq,
+                                     const void* Wout, const void* kv, const uint8_t* mask, void* y, void* ws, cudaStream_t st) {
+    int* status = nullptr;
+    taq_status s = status_ptr(&status);
+    if (s != TAQ_OK) return s;
+    const Workspace W = workspace_layout(d, n_req);
+    uint8_t* wsb = (uint8_t*)ws;
+    const long long rows_per_z = (long long)d->batch * d->n_query;   // weights are shared by the whole batch
+
+    LinearArgs q{};                                                     // to_q (+ Q~ = Q_a(Q))
+    q.x = (const __half*)x; q.w = Wq; q.reqs = reqs; q.which = 0;
+    q.y = wsb + W.off_q; q.scales = (float*)(wsb + W.off_qs);
+    q.rows = rows_per_z; q.n_out = d->channels; q.k_in = d->channels; q.bits = d->w_bits; q.group = d->w_group;
+    q.heads = d->q_bits == 8 ? d->heads : 1;
+    q.epi = d->q_bits == 8 ? EPI_Q8_HEAD : EPI_F16;
+    q.status = status;
+    s = run_linear(q, n_req, st);
+    if (s != TAQ_OK) return s;
+
+    AttnArgs at = attn_args(d, status);                                 // softmax(Q~K~^T/sqrt(d)), Eq. 3, P.V
+    at.q = wsb + W.off_q; at.q_scales = (const float*)(wsb + W.off_qs); at.kv = kv; at.mask = mask; at.reqs = reqs;
+    at.o = (__half*)(wsb + W.off_o);
+    s = run_attention(at, reqs ? n_req : d->batch, st);
+    if (s != TAQ_OK) return s;
+
+    LinearArgs o{};                                                     // to_out (+ bias)
+    o.x = (const __half*)(wsb + W.off_o); o.w = Wout; o.reqs = reqs; o.which = 1;
+    o.y = y;
+    o.rows = rows_per_z; o.n_out = d->channels; o.k_in = d->channels; o.bits = d->w_bits; o.group = d->w_group;
+    o.heads = 1; o.epi = EPI_F16; o.status = status;
+    return run_linear(o, n_req, st);
+}
+
+taq_status taq_layer_forward(const taq_layer_desc* d, const void* x_f16_dev, const void* Wq_packed_dev, const void* Wout_packed_dev,
+                             const void* kv_packed_dev, const uint8_t* trig_mask_dev, void* y_f16_dev, void* workspace_dev,
+                             size_t workspace_bytes, void* stream) {
+    taq_status s = check_layer_desc(d);
+    if (s != TAQ_OK) return s;
+    if (d->batch > 65535) return fail(TAQ_ERR_SHAPE, "batch must be at most 65535");
+    if (d->batch == 0 || d->n_query == 0) return TAQ_OK;
+    TAQ_REQUIRE_PTR(x_f16_dev);
+    TAQ_REQUIRE_PTR(Wq_packed_dev);
+    TAQ_REQUIRE_PTR(Wout_packed_dev);
+    TAQ_REQUIRE_PTR(kv_packed_dev);
+    TAQ_REQUIRE_PTR(y_f16_dev);
+    TAQ_REQUIRE_PTR(workspace_dev);
+    if (!trig_mask_dev) return fail(TAQ_ERR_INVALID_ARG, "trig_mask_dev is NULL");
+    if (reinterpret_cast<uintptr_t>(workspace_dev) & 127u) return fail(TAQ_ERR_ALIGNMENT, "workspace_dev is not 128-byte aligned");
+    const size_t need = taq_workspace_bytes(d, 1);
+    if (workspace_bytes < need) return fail(TAQ_ERR_BUFFER_TOO_SMALL, "workspace has %zu bytes, %zu needed", workspace_bytes, need);
+    return layer_forward_impl(d, nullptr, 1, x_f16_dev, Wq_packed_dev, Wout_packed_dev, kv_packed_dev, trig_mask_dev, y_f16_dev,
+                              workspace_dev, (cudaStream_t)stream);
+}
+
+taq_status taq_layer_forward_batched(const taq_layer_desc* d, const taq_request* reqs_dev, int32_t n_requests, const void* x_f16_dev,
+                                     void* y_f16_dev, void* workspace_dev, size_t workspace_bytes, void* stream) {
+    taq_status s = check_layer_desc(d);
+    if (s != TAQ_OK) return s;
+    if (d->batch != 1) return fail(TAQ_ERR_SHAPE, "batched calls take one sequence per request (desc->batch must be 1)");
+    if (n_requests < 0 || n_requests > 65535) return fail(TAQ_ERR_SHAPE, "n_requests must be in [0,65535]");
+    if (n_requests == 0 || d->n_query == 0) return TAQ_OK;
+    TAQ_REQUIRE_PTR(reqs_dev);
+    TAQ_REQUIRE_PTR(x_f16_dev);
+    TAQ_REQUIRE_PTR(y_f16_dev);
+    TAQ_REQUIRE_PTR(workspace_dev);
+    if (reinterpret_cast<uintptr_t>(workspace_dev) & 127u) return fail(TAQ_ERR_ALIGNMENT, "workspace_dev is not 128-byte aligned");
+    const size_t need = taq_workspace_bytes(d, n_requests);
+    if (workspace_bytes < need) return fail(TAQ_ERR_BUFFER_TOO_SMALL, "workspace has %zu bytes, %zu needed", workspace_bytes, need);
+    return layer_forward_impl(d, reqs_dev, n_requests, x_f16_dev, nullptr, nullptr, nullptr, nullptr, y_f16_dev, workspace_dev, (cudaStream_t)stream);
+}
+
+taq_status taq_poll_device_status(void* stream, int32_t* block_id_out) {
+    int* status = nullptr;
+    taq_status s = status_ptr(&status);
+    if (s != TAQ_OK) return s;
+    cudaStream_t st = (cudaStream_t)stream;
+    int host[2] = {0, 0};
+    cudaError_t e = cudaMemcpyAsync(host, status, sizeof(host), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(e, "reading the device status word");
+    if (host[0] != 0) {
+        e = cudaMemsetAsync(status, 0, sizeof(host), st);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+        if (e != cudaSuccess) return cuda_fail(e, "clearing the device status word");
+        if (block_id_out) *block_id_out = host[1];
+        return fail((taq_status)host[0], "a kernel raised device status %d (%s) in block %d", host[0], taq_status_string((taq_status)host[0]), host[1]);
+    }
+    if (block_id_out) *block_id_out = -1;
+    return TAQ_OK;
+}
+
+}  // extern "C"

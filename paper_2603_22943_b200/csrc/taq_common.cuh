@@ -1,0 +1,132 @@
+// Shared device/host definitions of the TAQ library: packed-blob header, K~/V~ block layout, status word.
+#pragma once
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "taq.h"
+
+namespace taq {
+
+constexpr uint32_t kWeightMagic = 0x57514154u;  // "TAQW" little-endian
+constexpr int kMaxCtx = 128;                    // T <= 128
+constexpr int kMaxHeadDim = 256;
+
+// First 64 bytes of a packed weight blob (layout documented in taq.h).
+struct PackedHeader {
+    uint32_t magic, version, n_out, k_in, bits, group, n_groups, has_bias;
+    uint64_t off_codes, off_scales, off_bias, total_bytes;
+};
+static_assert(sizeof(PackedHeader) == 64, "header is 64 bytes");
+
+__host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct WeightLayout {
+    int n_groups;
+    int group_len;          // effective group length (k_in when group == 0)
+    size_t row_bytes;       // bytes of codes per output channel
+    size_t off_codes, off_scales, off_bias, total;
+};
+
+__host__ __device__ inline WeightLayout weight_layout(int n_out, int k_in, int bits, int group) {
+    WeightLayout L;
+    L.group_len = group == 0 ? k_in : group;
+    L.n_groups = (k_in + L.group_len - 1) / L.group_len;
+    L.row_bytes = bits == 8 ? (size_t)k_in : (size_t)k_in / 2;
+    L.off_codes = 128;
+    L.off_scales = align_up(L.off_codes + L.row_bytes * n_out, 128);
+    L.off_bias = align_up(L.off_scales + sizeof(float) * (size_t)n_out * L.n_groups, 128);
+    L.total = align_up(L.off_bias + sizeof(float) * (size_t)n_out, 128);
+    return L;
+}
+
+// K~/V~ block of one sequence (layout documented in taq.h).
+__host__ __device__ inline taq_kv_layout kv_layout(int heads, int n_ctx, int d, int max_trigger) {
+    taq_kv_layout L;
+    size_t codes = align_up((size_t)heads * n_ctx * d, 128);
+    size_t scales = align_up(sizeof(float) * (size_t)heads * n_ctx, 128);
+    size_t trig = align_up(sizeof(__half) * (size_t)max_trigger * heads * d, 128);
+    L.off_k_codes = 0;
+    L.off_v_codes = codes;
+    L.off_k_scales = 2 * codes;
+    L.off_v_scales = 2 * codes + scales;
+    L.off_k_trigger = 2 * codes + 2 * scales;
+    L.off_v_trigger = L.off_k_trigger + trig;
+    L.off_trig_slot = L.off_v_trigger + trig;
+    L.block_bytes = L.off_trig_slot + sizeof(int32_t) * kMaxCtx;
+    return L;
+}
+
+// Device status word: {code, block id}.  First writer wins.
+__device__ inline void raise_status(int* status, int code) {
+    if (atomicCAS(&status[0], 0, code) == 0) {
+        status[1] = (int)(blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z));
+    }
+}
+
+// The symmetric quantizer in IEEE binary32: scale = absmax / qmax, code = clamp(rint(x / scale)).
+__device__ inline float quant_scale(float absmax, float qmax) { return __fdiv_rn(absmax, qmax); }
+__device__ inline int quant_code(float x, float scale, int qmax) {
+    if (scale == 0.f) return 0;
+    float r = rintf(__fdiv_rn(x, scale));
+    r = fminf(fmaxf(r, (float)-qmax), (float)qmax);
+    return (int)r;
+}
+
+// Matrix operand of a packed weight: fp16(float(code) * scale), returned as float.
+__device__ inline float dequant_w16(int code, float scale) {
+    return __half2float(__float2half_rn(__fmul_rn((float)code, scale)));
+}
+
+__device__ inline int load_code(const uint8_t* codes, size_t row_bytes, int bits, int n, int k) {
+    if (bits == 8) return (int)((const int8_t*)codes)[(size_t)n * row_bytes + k];
+    uint8_t byte = codes[(size_t)n * row_bytes + (k >> 1)];
+    return (int)((k & 1) ? (byte >> 4) : (byte & 0xF)) - 8;
+}
+
+// ------------------------------------------------------------------------------------------------------
+// Kernel launch arguments shared between translation units.
+// ------------------------------------------------------------------------------------------------------
+enum Epilogue : int { EPI_F16 = 0, EPI_F32 = 1, EPI_Q8_HEAD = 2, EPI_KV = 3 };
+
+// One dequant-GEMM problem family: y = x W^T.  With `reqs` set, grid.z indexes requests and the weight blob
+// (and, for EPI_KV, the output block and mask) come from the request table.
+struct LinearArgs {
+    const __half* x;            // [z][rows][k_in]
+    const void* w;              // packed blob (single problem)
+    const taq_request* reqs;    // nullable
+    int which;                  // 0: reqs[z].Wq, 1: reqs[z].Wout
+    void* y;                    // F16/F32/int8 [z][rows][n_out]; for EPI_KV: kv blocks (single problem)
+    float* scales;              // EPI_Q8_HEAD: [z][rows][heads]
+    const uint8_t* mask;        // EPI_KV: [batch][T] (single problem)
+    long long rows;             // rows per z
+    int n_out, k_in, bits, group;
+    int heads;                  // EPI_Q8_HEAD / EPI_KV
+    int n_ctx, max_trigger;     // EPI_KV: rows = batch * n_ctx
+    int kv_which;               // EPI_KV: 0 = K, 1 = V
+    int epi;
+    int* status;
+};
+
+struct AttnArgs {
+    const void* q;              // int8 or fp16 [z][B][N][C]
+    const float* q_scales;      // [z][B][N][H] (q_bits = 8)
+    const void* kv;             // blocks [B] (single problem)
+    const uint8_t* mask;        // [B][T]
+    const taq_request* reqs;    // nullable; then B = 1 per request
+    __half* o;                  // [z][B][N][C]
+    int batch, n_query, channels, heads, n_ctx, max_trigger;
+    int q_bits, p_bits;
+    int* status;
+};
+
+cudaError_t launch_linear_simt(const LinearArgs& a, int n_z, cudaStream_t stream);
+cudaError_t launch_attention_simt(const AttnArgs& a, int n_z, cudaStream_t stream);
+cudaError_t launch_quantize_rows(const float* x, long long rows, int cols, int qmax, int8_t* codes, float* scales,
+                                 cudaStream_t stream);
+cudaError_t launch_pack_weights(const taq_weight_desc& d, const float* W, const float* bias, void* packed,
+                                cudaStream_t stream);
+cudaError_t launch_unpack_weights(const taq_weight_desc& d, const void* packed, int8_t* codes, float* scales,
+                                  cudaStream_t stream);
+
+}  // namespace taq

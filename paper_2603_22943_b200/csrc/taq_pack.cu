@@ -1,0 +1,130 @@
+// Stand-alone quantizers: activation rows (Q_a of Eq. 2) and weight packing (W8 / W4 per output channel).
+// Integer codes are compared bit for bit with the CPU definition, so every floating-point step here is an
+// explicit IEEE binary32 operation (__fdiv_rn, rintf); nothing may be contracted or approximated.
+#include "taq_common.cuh"
+
+namespace taq {
+
+__device__ inline float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+
+// One warp per row.  Memory-bound: the row is read twice (absmax, then codes); the second read hits L1/L2.
+__global__ void __launch_bounds__(256) quantize_rows_kernel(const float* __restrict__ x, long long rows, int cols, int qmax,
+                                                            int8_t* __restrict__ codes, float* __restrict__ scales) {
+    const int lane = threadIdx.x & 31;
+    const long long warps_total = (long long)gridDim.x * (blockDim.x >> 5);
+    for (long long r = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); r < rows; r += warps_total) {
+        const float* xr = x + r * cols;
+        float a = 0.f;
+        if ((cols & 3) == 0) {
+            const float4* x4 = reinterpret_cast<const float4*>(xr);
+            for (int i = lane; i < cols / 4; i += 32) {
+                float4 v = x4[i];
+                a = fmaxf(a, fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w))));
+            }
+        } else {
+            for (int i = lane; i < cols; i += 32) a = fmaxf(a, fabsf(xr[i]));
+        }
+        a = warp_max(a);
+        const float s = quant_scale(a, (float)qmax);
+        if (lane == 0) scales[r] = s;
+        int8_t* cr = codes + r * cols;
+        if ((cols & 3) == 0) {
+            const float4* x4 = reinterpret_cast<const float4*>(xr);
+            char4* c4 = reinterpret_cast<char4*>(cr);
+            for (int i = lane; i < cols / 4; i += 32) {
+                float4 v = x4[i];
+                c4[i] = make_char4((signed char)quant_code(v.x, s, qmax), (signed char)quant_code(v.y, s, qmax),
+                                   (signed char)quant_code(v.z, s, qmax), (signed char)quant_code(v.w, s, qmax));
+            }
+        } else {
+            for (int i = lane; i < cols; i += 32) cr[i] = (int8_t)quant_code(xr[i], s, qmax);
+        }
+    }
+}
+
+cudaError_t launch_quantize_rows(const float* x, long long rows, int cols, int qmax, int8_t* codes, float* scales,
+                                 cudaStream_t stream) {
+    if (rows == 0) return cudaSuccess;
+    long long blocks = (rows + 7) / 8;
+    if (blocks > 148LL * 32) blocks = 148LL * 32;   // grid-stride beyond 32 resident waves
+    quantize_rows_kernel<<<(unsigned)blocks, 256, 0, stream>>>(x, rows, cols, qmax, codes, scales);
+    return cudaGetLastError();
+}
+
+// One warp per (output channel, group).
+__global__ void __launch_bounds__(256) pack_weights_kernel(const float* __restrict__ W, const float* __restrict__ bias, uint8_t* __restrict__ blob,
+                                                           int n_out, int k_in, int bits, int group) {
+    const WeightLayout L = weight_layout(n_out, k_in, bits, group);
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        PackedHeader h;
+        h.magic = kWeightMagic; h.version = 1; h.n_out = n_out; h.k_in = k_in; h.bits = bits; h.group = group;
+        h.n_groups = L.n_groups; h.has_bias = bias != nullptr;
+        h.off_codes = L.off_codes; h.off_scales = L.off_scales; h.off_bias = L.off_bias; h.total_bytes = L.total;
+        *reinterpret_cast<PackedHeader*>(blob) = h;
+    }
+    const int lane = threadIdx.x & 31;
+    const int qmax = bits == 8 ? 127 : 7;
+    const long long items = (long long)n_out * L.n_groups;
+    const long long warps_total = (long long)gridDim.x * (blockDim.x >> 5);
+    float* scales = reinterpret_cast<float*>(blob + L.off_scales);
+    float* bias_out = reinterpret_cast<float*>(blob + L.off_bias);
+    uint8_t* codes = blob + L.off_codes;
+    for (long long it = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); it < items; it += warps_total) {
+        const int n = (int)(it / L.n_groups), g = (int)(it % L.n_groups);
+        const int lo = g * L.group_len, hi = min(k_in, lo + L.group_len);
+        const float* wr = W + (size_t)n * k_in;
+        float a = 0.f;
+        for (int k = lo + lane; k < hi; k += 32) a = fmaxf(a, fabsf(wr[k]));
+        a = warp_max(a);
+        const float s = quant_scale(a, (float)qmax);
+        if (lane == 0) {
+            scales[(size_t)n * L.n_groups + g] = s;
+            if (g == 0) bias_out[n] = bias ? bias[n] : 0.f;
+        }
+        if (bits == 8) {
+            for (int k = lo + lane; k < hi; k += 32) ((int8_t*)codes)[(size_t)n * L.row_bytes + k] = (int8_t)quant_code(wr[k], s, qmax);
+        } else {
+            for (int k = lo + 2 * lane; k < hi; k += 64) {   // group bounds are even, so a byte never straddles groups
+                int q0 = quant_code(wr[k], s, qmax) + 8;
+                int q1 = quant_code(wr[k + 1], s, qmax) + 8;
+                codes[(size_t)n * L.row_bytes + (k >> 1)] = (uint8_t)(q0 | (q1 << 4));
+            }
+        }
+    }
+}
+
+cudaError_t launch_pack_weights(const taq_weight_desc& d, const float* W, const float* bias, void* packed, cudaStream_t stream) {
+    const WeightLayout L = weight_layout(d.n_out, d.k_in, d.bits, d.group);
+    long long items = (long long)d.n_out * L.n_groups;
+    long long blocks = (items + 7) / 8;
+    if (blocks > 148LL * 32) blocks = 148LL * 32;
+    pack_weights_kernel<<<(unsigned)blocks, 256, 0, stream>>>(W, bias, (uint8_t*)packed, d.n_out, d.k_in, d.bits, d.group);
+    return cudaGetLastError();
+}
+
+__global__ void __launch_bounds__(256) unpack_weights_kernel(const uint8_t* __restrict__ blob, int8_t* __restrict__ codes_out,
+                                                             float* __restrict__ scales_out, int n_out, int k_in, int bits, int group) {
+    const WeightLayout L = weight_layout(n_out, k_in, bits, group);
+    const long long total = (long long)n_out * k_in;
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
+        const int n = (int)(i / k_in), k = (int)(i % k_in);
+        codes_out[i] = (int8_t)load_code(blob + L.off_codes, L.row_bytes, bits, n, k);
+    }
+    const float* scales = reinterpret_cast<const float*>(blob + L.off_scales);
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < (long long)n_out * L.n_groups; i += stride) scales_out[i] = scales[i];
+}
+
+cudaError_t launch_unpack_weights(const taq_weight_desc& d, const void* packed, int8_t* codes, float* scales, cudaStream_t stream) {
+    long long total = (long long)d.n_out * d.k_in;
+    long long blocks = (total + 255) / 256;
+    if (blocks > 148LL * 16) blocks = 148LL * 16;
+    unpack_weights_kernel<<<(unsigned)blocks, 256, 0, stream>>>((const uint8_t*)packed, codes, scales, d.n_out, d.k_in, d.bits, d.group);
+    return cudaGetLastError();
+}
+
+}  // namespace taq

@@ -1,0 +1,116 @@
+"""Shared helpers of the GPU parity tests: run the CUDA path through the C-ABI binding on the seeded
+synthetic inputs, run the CPU oracle on the same arrays, and compare."""
+import numpy as np
+import torch
+
+from oracle import taq_oracle as orc
+from paper_2603_22943_b200 import binding as tb
+from paper_2603_22943_b200 import synth
+
+# Layer-output tolerances of the parity contract (fp16 outputs against the fp64 contract-mode oracle).
+TOL_MAX_ABS = 2e-2
+TOL_REL_L2 = 1e-3
+
+
+def dev(a: np.ndarray) -> torch.Tensor:
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def errors(got: np.ndarray, want: np.ndarray):
+    got = np.asarray(got, dtype=np.float64)
+    want = np.asarray(want, dtype=np.float64)
+    den = np.linalg.norm(want)
+    return float(np.max(np.abs(got - want))) if got.size else 0.0, float(np.linalg.norm(got - want) / den) if den > 0 else 0.0
+
+
+def assert_layer_close(got, want, what=""):
+    max_abs, rel = errors(got, want)
+    assert max_abs <= TOL_MAX_ABS and rel <= TOL_REL_L2, f"{what}: max-abs {max_abs:.3e} (<= {TOL_MAX_ABS}), rel-L2 {rel:.3e} (<= {TOL_REL_L2})"
+    return max_abs, rel
+
+
+def oracle_cfg(shape: synth.LayerShape, contract=True) -> orc.TaqConfig:
+    return orc.TaqConfig(heads=shape.heads, w_bits=shape.w_bits, w_group=shape.w_group, q_bits=shape.q_bits, contract=contract)
+
+
+def oracle_layer(shape: synth.LayerShape, data, contract=True, rows=None):
+    """Oracle on the whole layer, or on a subset of query rows (rows are independent)."""
+    X = data["X"] if rows is None else data["X"][:, rows]
+    return orc.taq_layer(X, data["ctx"], data["Wq"], data["Wk"], data["Wv"], data["Wout"], data["bout"], data["mask"],
+                         oracle_cfg(shape, contract))
+
+
+def gpu_desc(shape: synth.LayerShape, max_trigger=None, batch=None, n_query=None) -> tb.LayerDesc:
+    mt = max(1, len(shape.trigger)) if max_trigger is None else max_trigger
+    return tb.layer_desc(shape.batch if batch is None else batch, shape.n_query if n_query is None else n_query,
+                         shape.channels, shape.heads, shape.n_ctx, shape.ctx_dim, shape.w_bits, shape.w_group,
+                         q_bits=shape.q_bits, max_trigger=mt)
+
+
+def pack_layer_weights(shape: synth.LayerShape, data):
+    C_, Dc = shape.channels, shape.ctx_dim
+    wd_cc = tb.weight_desc(C_, C_, shape.w_bits, shape.w_group)
+    wd_cd = tb.weight_desc(C_, Dc, shape.w_bits, shape.w_group)
+    return {
+        "Wq": tb.taq_pack_weights(wd_cc, dev(data["Wq"])),
+        "Wk": tb.taq_pack_weights(wd_cd, dev(data["Wk"])),
+        "Wv": tb.taq_pack_weights(wd_cd, dev(data["Wv"])),
+        "Wout": tb.taq_pack_weights(wd_cc, dev(data["Wout"]), dev(data["bout"])),
+        "wd_cc": wd_cc, "wd_cd": wd_cd,
+    }
+
+
+def gpu_layer(shape: synth.LayerShape, data, max_trigger=None, return_parts=False):
+    """The whole CUDA path: pack, K/V projection with Eq. 2, then the per-step layer."""
+    desc = gpu_desc(shape, max_trigger)
+    P = pack_layer_weights(shape, data)
+    mask = dev(data["mask"])
+    kv = tb.taq_kv_project(desc, dev(data["ctx"]), P["Wk"], P["Wv"], mask)
+    y = tb.taq_layer_forward(desc, dev(data["X"]), P["Wq"], P["Wout"], kv, mask)
+    tb.taq_poll_device_status()
+    torch.cuda.synchronize()
+    if return_parts:
+        return y.cpu().numpy(), {"desc": desc, "packed": P, "kv": kv, "mask": mask}
+    return y.cpu().numpy()
+
+
+def parse_kv_block(desc: tb.LayerDesc, kv: torch.Tensor):
+    """Splits the K~/V~ blocks (layout documented in taq.h) into numpy arrays."""
+    lay = tb.taq_kv_layout_of(desc)
+    B, H, T, d, R = desc.batch, desc.heads, desc.n_ctx, desc.d_head, desc.max_trigger
+    raw = kv.cpu().numpy().reshape(-1)[: B * lay.block_bytes].reshape(B, lay.block_bytes)
+    out = {}
+    for nm, oc, osc, otr in (("K", lay.off_k_codes, lay.off_k_scales, lay.off_k_trigger), ("V", lay.off_v_codes, lay.off_v_scales, lay.off_v_trigger)):
+        out[nm + "_codes"] = np.stack([raw[b, oc: oc + H * T * d].view(np.int8).reshape(H, T, d) for b in range(B)])
+        out[nm + "_scales"] = np.stack([raw[b, osc: osc + H * T * 4].view(np.float32).reshape(H, T) for b in range(B)])
+        out[nm + "_trigger"] = np.stack([raw[b, otr: otr + R * H * d * 2].view(np.float16).reshape(R, H, d) for b in range(B)])
+    out["slot"] = np.stack([raw[b, lay.off_trig_slot: lay.off_trig_slot + 512].view(np.int32) for b in range(B)])
+    return out
+
+
+def build_kv_block(desc: tb.LayerDesc, K_codes, K_scales, V_codes, V_scales, K_rows, V_rows, mask) -> np.ndarray:
+    """Host-side packer used to feed the attention kernel with the oracle's own K~/V~ (test isolation)."""
+    lay = tb.taq_kv_layout_of(desc)
+    B, H, T, d, R = desc.batch, desc.heads, desc.n_ctx, desc.d_head, desc.max_trigger
+    raw = np.zeros((B, lay.block_bytes), dtype=np.uint8)
+    for b in range(B):
+        slot = np.full(128, -1, dtype=np.int32)
+        trig = [j for j in range(T) if mask[b, j]]
+        assert len(trig) <= R
+        kt = np.zeros((R, H, d), np.float16)
+        vt = np.zeros((R, H, d), np.float16)
+        kc, vc = K_codes[b].astype(np.int8).copy(), V_codes[b].astype(np.int8).copy()
+        ks, vs = K_scales[b].astype(np.float32).copy(), V_scales[b].astype(np.float32).copy()
+        for s, j in enumerate(trig):
+            slot[j] = s
+            kt[s] = K_rows[b, :, j].astype(np.float16)
+            vt[s] = V_rows[b, :, j].astype(np.float16)
+            kc[:, j] = 0; vc[:, j] = 0; ks[:, j] = 0; vs[:, j] = 0
+        raw[b, lay.off_k_codes: lay.off_k_codes + H * T * d] = kc.reshape(-1).view(np.uint8)
+        raw[b, lay.off_v_codes: lay.off_v_codes + H * T * d] = vc.reshape(-1).view(np.uint8)
+        raw[b, lay.off_k_scales: lay.off_k_scales + H * T * 4] = ks.reshape(-1).view(np.uint8)
+        raw[b, lay.off_v_scales: lay.off_v_scales + H * T * 4] = vs.reshape(-1).view(np.uint8)
+        raw[b, lay.off_k_trigger: lay.off_k_trigger + R * H * d * 2] = kt.reshape(-1).view(np.uint8)
+        raw[b, lay.off_v_trigger: lay.off_v_trigger + R * H * d * 2] = vt.reshape(-1).view(np.uint8)
+        raw[b, lay.off_trig_slot: lay.off_trig_slot + 512] = slot.view(np.uint8)
+    return raw.reshape(-1)
