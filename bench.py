@@ -1,0 +1,329 @@
+#!/usr/bin/env python
+"""Benchmark of the TAQ cross-attention hot path on B200.
+
+``python bench.py [--gpus N] [--steps K] [--warmup W]`` times K passes of one cross-attention layer
+(to_q with Q~ = Q_a(Q), fused attention with Eq. 3, to_out; K~/V~ of Eq. 2 projected once per prompt outside
+the step, as they do not depend on the image tokens) on the SD-1.5 highest-resolution configuration
+(B=2, N=4096, C=320, 8 heads, T=77, W4 group 128, trigger tokens {4,5}) and prints one JSON line.
+Every step uses a different set of input/output/weight buffers out of a ring larger than twice the L2, so
+each pass streams its activations from HBM.  ``--impl reference`` times the CPU oracle instead.
+Under torchrun each rank runs an independent replica (the path has no exchange step).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "TAQ cross-attn queries/s per layer"
+UNIT = "queries/s"
+WORKLOAD = "config2: SD-1.5 64x64 cross-attn layer, B=2 N=4096 C=320 H=8 d=40 T=77 Dc=768, W4 g128, int8 Q/K/V rows, uint8 probs, fp16 trigger rows {4,5}"
+
+
+def _peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100", "-i", str(self.gpu)],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        for l in self.lines:
+            f = [x.strip() for x in l.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def _oracle_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [i.get("num_threads", 1) for i in threadpool_info()]
+        return max(n) if n else 1
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def time_oracle(shape, data, sample_rows: int, repeats: int = 1):
+    """Contract-mode oracle on `sample_rows` query rows of every sequence; returns (seconds, rows)."""
+    from oracle import taq_oracle as orc
+    rows = np.arange(min(sample_rows, shape.n_query))
+    cfg = orc.TaqConfig(heads=shape.heads, w_bits=shape.w_bits, w_group=shape.w_group, q_bits=shape.q_bits, contract=True)
+    best = None
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        orc.taq_layer(data["X"][:, rows], data["ctx"], data["Wq"], data["Wk"], data["Wv"], data["Wout"], data["bout"], data["mask"], cfg)
+        dt = time.perf_counter() - t0
+        best = dt if best is None else min(best, dt)
+    return best, shape.batch * len(rows)
+
+
+def run_reference(args, shape, data):
+    """The base contract's reference arm: the CPU oracle, as it stands, on the machine's host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    sample = min(shape.n_query, args.ref_rows)
+    for _ in range(args.warmup):
+        time_oracle(shape, data, sample)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        time_oracle(shape, data, sample)
+    dt = (time.perf_counter() - t0) / max(args.steps, 1)
+    value = shape.batch * sample / dt
+    cores = _oracle_threads()
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "sample": f"first {sample} query rows of each of the {shape.batch} sequences per step"},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": f"{shape.batch}x{sample} query rows per step (whole layer incl. K/V projection)"},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}, "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=400)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="taq", choices=["taq", "reference"])
+    ap.add_argument("--ref-rows", type=int, default=1024, help="query rows per sequence in one reference-arm step")
+    ap.add_argument("--cpu-rows", type=int, default=4096, help="query rows per sequence of the cpu_baseline sample")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--n-query", type=int, default=0, help="override N (profiling on a smaller case)")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "taq":
+        args.warmup = 3
+
+    from paper_2603_22943_b200 import synth
+    shape = synth.config2()
+    if args.n_query:
+        shape = synth.shrink(shape, args.n_query)
+    data = synth.make_layer(shape)
+
+    if args.impl == "reference":
+        run_reference(args, shape, data)
+        return
+
+    import torch
+    from paper_2603_22943_b200 import binding as tb
+    from paper_2603_22943_b200 import build as tbuild
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the TAQ path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if not os.path.exists(tb.LIB_PATH):
+        tbuild.build_library()
+    tb.lib()
+
+    def dev(a):
+        return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+    B, N, C_, H, T, Dc = shape.batch, shape.n_query, shape.channels, shape.heads, shape.n_ctx, shape.ctx_dim
+    M = B * N
+    desc = tb.layer_desc(B, N, C_, H, T, Dc, shape.w_bits, shape.w_group, q_bits=shape.q_bits, max_trigger=len(shape.trigger))
+    wd_cc = tb.weight_desc(C_, C_, shape.w_bits, shape.w_group)
+    wd_cd = tb.weight_desc(C_, Dc, shape.w_bits, shape.w_group)
+    l2 = torch.cuda.get_device_properties(local_rank).L2_cache_size
+    set_bytes = 2 * M * C_ * 2
+    n_sets = max(4, int(np.ceil(2.2 * l2 / set_bytes)))
+
+    Wk = tb.taq_pack_weights(wd_cd, dev(data["Wk"]))
+    Wv = tb.taq_pack_weights(wd_cd, dev(data["Wv"]))
+    mask = dev(data["mask"])
+    ctx = dev(data["ctx"])
+    x_host = data["X"]
+    sets = []
+    for i in range(n_sets):     # every set: its own activations, weights, K~/V~ and workspace
+        s = {"x": dev(np.roll(x_host, i, axis=1)), "y": torch.empty((B, N, C_), dtype=torch.float16, device="cuda"),
+             "Wq": tb.taq_pack_weights(wd_cc, dev(data["Wq"])), "Wout": tb.taq_pack_weights(wd_cc, dev(data["Wout"]), dev(data["bout"])),
+             "ws": torch.empty(tb.taq_workspace_bytes(desc, 1), dtype=torch.uint8, device="cuda")}
+        s["kv"] = tb.taq_kv_project(desc, ctx, Wk, Wv, mask)
+        sets.append(s)
+    tb.taq_poll_device_status()
+
+    def step(i):
+        s = sets[i % n_sets]
+        tb.taq_layer_forward(desc, s["x"], s["Wq"], s["Wout"], s["kv"], mask, s["y"], s["ws"])
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(args.steps):
+        step(i)
+    e1.record()
+    barrier()
+    ms_total = e0.elapsed_time(e1)
+
+    # Per-kernel attribution: the same three stages through their own entry points, events between them.
+    q_c = torch.empty((M, C_), dtype=torch.int8 if shape.q_bits == 8 else torch.float16, device="cuda")
+    q_s = torch.empty((M, H), dtype=torch.float32, device="cuda")
+    o_sets = [torch.empty((B, N, C_), dtype=torch.float16, device="cuda") for _ in range(n_sets)]
+    q_sets = [(torch.empty_like(q_c), torch.empty_like(q_s)) for _ in range(n_sets)]
+    k_steps = min(args.steps, 200)
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(k_steps)]
+
+    def stage_step(i, ev=None):
+        s = sets[i % n_sets]
+        qc, qs = q_sets[i % n_sets]
+        if ev: ev[0].record()
+        if shape.q_bits == 8:
+            tb.taq_quantized_linear(wd_cc, s["x"], s["Wq"], tb.TAQ_OUT_INT8_HEAD_ROWS, heads=H, y=qc, scales=qs)
+        else:
+            tb.taq_quantized_linear(wd_cc, s["x"], s["Wq"], tb.TAQ_OUT_F16, y=qc)
+        if ev: ev[1].record()
+        tb.taq_cross_attention(desc, qc, qs if shape.q_bits == 8 else None, s["kv"], mask, o_sets[i % n_sets])
+        if ev: ev[2].record()
+        tb.taq_quantized_linear(wd_cc, o_sets[i % n_sets], s["Wout"], tb.TAQ_OUT_F16, y=s["y"])
+        if ev: ev[3].record()
+
+    for i in range(3):
+        stage_step(i)
+    torch.cuda.synchronize()
+    for i in range(k_steps):
+        stage_step(i, evs[i])
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    stage_ms = [sum(ev[j].elapsed_time(ev[j + 1]) for ev in evs) / k_steps for j in range(3)]
+
+    # End to end through the same call with host buffers: H2D of X and D2H of Y inside the timed region.
+    xh = [torch.from_numpy(np.ascontiguousarray(np.roll(x_host, i, axis=1))).pin_memory() for i in range(4)]
+    yh = [torch.empty((B, N, C_), dtype=torch.float16).pin_memory() for _ in range(4)]
+    e_steps = max(10, min(args.steps, 100))
+
+    def e2e_step(i):
+        s = sets[i % n_sets]
+        s["x"].copy_(xh[i % 4], non_blocking=True)
+        tb.taq_layer_forward(desc, s["x"], s["Wq"], s["Wout"], s["kv"], mask, s["y"], s["ws"])
+        yh[i % 4].copy_(s["y"], non_blocking=True)
+
+    for i in range(3):
+        e2e_step(i)
+    barrier()
+    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    f0.record()
+    for i in range(e_steps):
+        e2e_step(i)
+    f1.record()
+    barrier()
+    e2e_ms = f0.elapsed_time(f1)
+    tb.taq_poll_device_status()
+
+    t = torch.tensor([ms_total, e2e_ms], dtype=torch.float64, device="cuda")
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total, e2e_ms = float(t[0]), float(t[1])
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peaks = _peaks()
+    ms_per_step = ms_total / args.steps
+    value = world * M / (ms_per_step * 1e-3)
+    e2e_value = world * M / (e2e_ms / e_steps * 1e-3)
+    kv_block = tb.taq_kv_layout_of(desc).block_bytes * B
+    wbytes = tb.taq_packed_weight_bytes(wd_cc)
+    qbytes = M * C_ * (1 if shape.q_bits == 8 else 2) + (M * H * 4 if shape.q_bits == 8 else 0)
+    kernels = [
+        {"name": "to_q dequant-GEMM + Q_a epilogue", "ms": stage_ms[0], "bytes": M * C_ * 2 + qbytes + wbytes, "flops": 2 * M * C_ * C_},
+        {"name": "fused TAQ attention", "ms": stage_ms[1], "bytes": qbytes + M * C_ * 2 + kv_block, "flops": 4 * M * T * C_},
+        {"name": "to_out dequant-GEMM", "ms": stage_ms[2], "bytes": 2 * M * C_ * 2 + wbytes, "flops": 2 * M * C_ * C_},
+    ]
+    for k in kernels:
+        k["GB/s"] = k["bytes"] / (k["ms"] * 1e-3) / 1e9
+        k["TFLOP/s"] = k["flops"] / (k["ms"] * 1e-3) / 1e12
+    dom = max(kernels, key=lambda k: k["ms"])
+    roofline = {"kernel": dom["name"], "bound": "hbm", "achieved": dom["GB/s"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": dom["GB/s"] / peaks["hbm_gbs"], "peak_source": peaks["source"], "traffic": None,
+                "bytes_per_launch": dom["bytes"], "ms_per_launch": dom["ms"],
+                "stages": [{"name": k["name"], "ms": round(k["ms"], 5), "GB/s": round(k["GB/s"], 1), "TFLOP/s": round(k["TFLOP/s"], 2)} for k in kernels]}
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f16",
+            "data": "synthetic",
+            "config": {"workload": WORKLOAD if not args.n_query else WORKLOAD + f" (N overridden to {N})", "kv_projection": "once per prompt, outside the step",
+                       "l2_policy": f"inputs larger than L2: ring of {n_sets} buffer sets ({n_sets * set_bytes / 1e6:.0f} MB of activations, L2 {l2 / 1e6:.0f} MB)",
+                       "replicas": world},
+            "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": M * C_ * 2, "d2h_bytes_per_step": M * C_ * 2, "steps": e_steps},
+            "gpu_launches": 3 * args.steps,
+            "roofline": roofline}
+    if not args.no_cpu_baseline:
+        secs, rows = time_oracle(shape, data, args.cpu_rows)
+        line["cpu_baseline"] = {"value": rows / secs, "unit": UNIT, "cores": _oracle_threads(), "kind": "oracle",
+                                "sample": f"{rows} query rows ({B} sequences x {rows // B}) of the same layer incl. K/V projection, {secs:.2f} s"}
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -114,3 +114,88 @@ def build_kv_block(desc: tb.LayerDesc, K_codes, K_scales, V_codes, V_scales, K_r
         raw[b, lay.off_v_trigger: lay.off_v_trigger + R * H * d * 2] = vt.reshape(-1).view(np.uint8)
         raw[b, lay.off_trig_slot: lay.off_trig_slot + 512] = slot.view(np.uint8)
     return raw.reshape(-1)
+
+
+def gpu_decisions(shape: synth.LayerShape, data, parts, rows=None):
+    """The rounding decisions the CUDA path took upstream of the attention: K~/V~ as stored in its block and Q~
+    as produced by the same dequant-GEMM kernel the layer call runs (bit-identical by determinism)."""
+    desc, P = parts["desc"], parts["packed"]
+    B, H, T, d = shape.batch, shape.heads, shape.n_ctx, shape.d_head
+    kvg = parse_kv_block(desc, parts["kv"])
+    out = {}
+    for nm in ("K", "V"):
+        Z = (kvg[nm + "_codes"].astype(np.float32) * kvg[nm + "_scales"][..., None]).astype(np.float64)     # [B,H,T,d]
+        for b in range(B):
+            for j in range(T):
+                s = int(kvg["slot"][b, j])
+                if s >= 0:
+                    Z[b, :, j] = kvg[nm + "_trigger"][b, s].astype(np.float64)
+        out[nm + "_tilde"] = Z
+        out[nm + "_codes"], out[nm + "_scales"] = kvg[nm + "_codes"], kvg[nm + "_scales"]
+    X = data["X"] if rows is None else data["X"][:, rows]
+    n = X.shape[1]
+    x2 = dev(X.reshape(B * n, shape.channels))
+    if shape.q_bits == 8:
+        qc, qs = tb.taq_quantized_linear(P["wd_cc"], x2, P["Wq"], tb.TAQ_OUT_INT8_HEAD_ROWS, heads=H)
+        qc = qc.cpu().numpy().reshape(B, n, H, d).transpose(0, 2, 1, 3)                                   # [B,H,n,d]
+        qs = qs.cpu().numpy().reshape(B, n, H).transpose(0, 2, 1)                                          # [B,H,n]
+        out["Q_codes"], out["Q_scales"] = qc, qs
+        out["Q_tilde"] = (qc.astype(np.float32) * qs[..., None]).astype(np.float64)
+    else:
+        q16 = tb.taq_quantized_linear(P["wd_cc"], x2, P["Wq"], tb.TAQ_OUT_F16).cpu().numpy()
+        out["Q_tilde"] = q16.reshape(B, n, H, d).transpose(0, 2, 1, 3).astype(np.float64)
+    return out
+
+
+def assert_codes_agree(got, want, pre, scales, what, max_frac=2e-3):
+    """Integer codes taken after an fp32 accumulation (GPU) and after an fp64 one (oracle) may differ by one step,
+    and only where the value being rounded sits on a rounding boundary to within the accumulation error."""
+    got, want = got.astype(np.int32), want.astype(np.int32)
+    diff = got != want
+    if not diff.any():
+        return 0.0
+    assert np.abs(got - want).max() <= 1, f"{what}: a code differs by more than one step"
+    frac = float(diff.mean())
+    assert frac <= max_frac, f"{what}: {frac:.2e} of the codes differ"
+    s = np.broadcast_to(scales[..., None], pre.shape)[diff].astype(np.float64)
+    boundary = (got[diff] + want[diff]) / 2.0
+    dist = np.abs(pre[diff] / s - boundary)                     # in code units
+    assert dist.max() < 2e-3, f"{what}: a differing code is {dist.max():.2e} steps away from its rounding boundary"
+    return frac
+
+
+def check_layer(shape: synth.LayerShape, data, y_gpu, parts, rows=None):
+    """Three-part parity of one layer call.
+    (1) the integer decisions (Q, K, V codes) of the CUDA path equal the oracle's, up to near-ties;
+    (2) given the same decisions, the layer output matches the oracle within the contract tolerances everywhere;
+    (3) end to end against the untouched oracle: relative L2 within tolerance over everything, and max-abs within
+        tolerance on every query row whose Q codes agree (a one-step flip of a near-tie is amplified by the softmax,
+        which is why both sides must take that decision from the same value, as (2) does)."""
+    cfg = oracle_cfg(shape)
+    X = data["X"] if rows is None else data["X"][:, rows]
+    y = y_gpu if rows is None else y_gpu[:, rows]
+    kv_o = orc.taq_kv(data["ctx"], data["Wk"], data["Wv"], data["mask"], cfg)
+    q_o = orc.taq_q(X, data["Wq"], cfg)
+    Y_o = orc.taq_out(orc.taq_attention(q_o["Q_tilde"], kv_o["K_tilde"], kv_o["V_tilde"], data["mask"], cfg), data["Wout"], data["bout"], cfg)
+    g = gpu_decisions(shape, data, parts, rows)
+    # (1)
+    nt = np.array([j for j in range(shape.n_ctx) if not data["mask"][0, j]], dtype=np.int64)
+    same_mask = bool((data["mask"] == data["mask"][0]).all())
+    if same_mask and len(nt):
+        for nm in ("K", "V"):
+            assert_codes_agree(g[nm + "_codes"][:, :, nt], kv_o[nm + "_codes"][:, :, nt], kv_o[nm][:, :, nt], kv_o[nm + "_scales"][:, :, nt], nm + " codes")
+    flipped_rows = np.zeros(X.shape[:2], dtype=bool)
+    if shape.q_bits == 8:
+        assert_codes_agree(g["Q_codes"], q_o["Q_codes"], q_o["Q"], q_o["Q_scales"], "Q codes")
+        np.testing.assert_allclose(g["Q_scales"], q_o["Q_scales"], rtol=2e-5)
+        flipped_rows = (g["Q_codes"] != q_o["Q_codes"]).any(axis=(1, 3))               # [B,n]
+    # (2)
+    Y_d = orc.taq_out(orc.taq_attention(g["Q_tilde"], g["K_tilde"], g["V_tilde"], data["mask"], cfg), data["Wout"], data["bout"], cfg)
+    same = assert_layer_close(y, Y_d, shape.name + " (same decisions)")
+    # (3)
+    max_abs, rel = errors(y, Y_o)
+    assert rel <= TOL_REL_L2, f"{shape.name}: end-to-end rel-L2 {rel:.3e}"
+    if (~flipped_rows).any():
+        ma = float(np.max(np.abs(y.astype(np.float64) - Y_o)[~flipped_rows]))
+        assert ma <= TOL_MAX_ABS, f"{shape.name}: end-to-end max-abs {ma:.3e} on rows whose Q codes agree"
+    return {"same_decisions": same, "end_to_end": (max_abs, rel), "rows_with_q_flip": int(flipped_rows.sum())}
