@@ -212,7 +212,9 @@ def taq_attention(Q_tilde: np.ndarray, K_tilde: np.ndarray, V_tilde: np.ndarray,
     S = S - S.max(axis=-1, keepdims=True)
     E = np.exp(S)
     A = E / E.sum(axis=-1, keepdims=True)
-    kept = f16_round(A) if cfg.contract else A                   # trigger columns: stored fp16
+    # Trigger columns are kept in fp16.  The stored probability tensor uses one unit for all columns, 1/255:
+    # ordinary columns hold the uint8 code, trigger columns hold fp16(255 A).
+    kept = f16_round(A * 255.0) / 255.0 if cfg.contract else A
     if cfg.p_bits == 0:
         A_hat = np.where(M, kept, A)
     else:
