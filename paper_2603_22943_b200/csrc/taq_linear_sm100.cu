@@ -167,7 +167,7 @@ __global__ void __launch_bounds__(NTHREADS) linear_sm100_kernel(const __grid_con
                 for (int c = 0; c < BN; c += 16) {
                     uint32_t v[16];
                     ptx::tmem_ld16(taddr + c, v);
-                    ptx::tmem_ld_wait();
+                    ptx::tmem_ld_wait(v);
                     if (row < a.rows) {
                         const size_t o = ((size_t)z * a.rows + row) * a.n_out + col0 + c;
                         if (a.epi == EPI_F16) {
@@ -218,7 +218,7 @@ __global__ void __launch_bounds__(NTHREADS) linear_sm100_kernel(const __grid_con
                     for (int c = 0; c < d; c += 8) {
                         uint32_t v[8];
                         ptx::tmem_ld8(taddr + hh * d + c, v);
-                        ptx::tmem_ld_wait();
+                        ptx::tmem_ld_wait(v);
 #pragma unroll
                         for (int i = 0; i < 8; ++i) amax = fmaxf(amax, fabsf(__uint_as_float(v[i])));
                     }
@@ -227,7 +227,7 @@ __global__ void __launch_bounds__(NTHREADS) linear_sm100_kernel(const __grid_con
                     for (int c = 0; c < d; c += 8) {
                         uint32_t v[8];
                         ptx::tmem_ld8(taddr + hh * d + c, v);
-                        ptx::tmem_ld_wait();
+                        ptx::tmem_ld_wait(v);
                         if (row < a.rows) {
                         uint32_t lo = 0, hi = 0;
                         if (!(a.epi == EPI_KV && trig)) {

@@ -52,7 +52,7 @@ def test_kv_project(shape):
             g = got[nm + "_trigger"][:, s].astype(np.float64)               # [B,H,d]
             w = want[nm + "_tilde"][:, :, j]
             assert np.max(np.abs(g - w)) <= np.max(np.abs(w)) * 2.0 ** -10
-            assert (g != w).mean() < 0.01                                    # an fp16 tie broken differently is rare
+            assert (g != w).mean() < 0.03          # an fp16 rounding that lands on the other side is rare (~1 % with tensor-core accumulation)
         deq = got[nm + "_codes"].astype(np.float64) * got[nm + "_scales"][..., None]
         assert tl.errors(deq[:, :, nt], want[nm + "_tilde"][:, :, nt])[1] < 1e-3
     for b in range(shape.batch):
