@@ -184,6 +184,28 @@ taq_status taq_layer_forward_batched(const taq_layer_desc* desc, const taq_reque
 taq_status taq_kv_project_batched(const taq_layer_desc* desc, const taq_request* reqs_dev, int32_t n_requests,
                                   const void* ctx_f16_dev, void* stream);
 
+/* The same pass as taq_layer_forward for callers that cannot hand over a workspace.  The paper has no counterpart
+ * to this entry point; it exists for integration only.  Typical callers: an inference server that gave all of the
+ * GPU's memory to its own pool at start-up (a cudaMalloc there fails, or stalls every stream of the device while
+ * it runs), and a plug-in slot of a host framework that passes input and output pointers and nothing else.
+ *   - The scratch (Q~, its scales, O) is a fixed array of TAQ_STATIC_WORKSPACE_BYTES inside the library image:
+ *     every GPU on which the library is loaded keeps that much memory until the process ends.  The call performs
+ *     no device allocation or free of any kind.
+ *   - A layer whose taq_workspace_bytes(desc, 1) exceeds taq_static_workspace_capacity() is refused with
+ *     TAQ_ERR_BUFFER_TOO_SMALL before anything is launched (config 2 of the benchmark, B=2 N=4096 C=320, needs
+ *     8.1 MB and fits; B*N*(3C + 4H) bytes is the rule of thumb).
+ *   - The first call on each device looks up the array's device address (a host-side runtime query, with that
+ *     device current).  Make that first call outside any stream capture.
+ *   - All calls on one device share the one array.  Nothing in it has to be zero on entry and nothing is kept
+ *     for the caller, but two calls whose kernels can overlap on the GPU (different streams, no dependency) write
+ *     over each other's intermediate results: issue them on one stream or order them with events.
+ * Arguments as for taq_layer_forward, without the workspace pair. */
+#define TAQ_STATIC_WORKSPACE_BYTES (16u << 20)
+size_t taq_static_workspace_capacity(void);
+taq_status taq_layer_forward_static(const taq_layer_desc* desc, const void* x_f16_dev, const void* Wq_packed_dev,
+                                    const void* Wout_packed_dev, const void* kv_packed_dev,
+                                    const uint8_t* trig_mask_dev, void* y_f16_dev, void* stream);
+
 /* Device status word: kernels never trap; a bounded wait that runs out or a capacity violation records a code
  * and the block that saw it.  This call synchronises `stream`, returns that code (TAQ_OK if none) and clears
  * it.  block_id_out may be NULL. */

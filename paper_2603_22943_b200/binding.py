@@ -24,6 +24,7 @@ EXPORTS = [
     "taq_unpack_weights", "taq_quantize_rows", "taq_kv_layout_of", "taq_kv_bytes", "taq_kv_project",
     "taq_quantized_linear", "taq_cross_attention", "taq_workspace_bytes", "taq_layer_forward",
     "taq_layer_forward_batched", "taq_kv_project_batched", "taq_poll_device_status",
+    "taq_static_workspace_capacity", "taq_layer_forward_static",
 ]
 
 
@@ -89,6 +90,9 @@ def lib() -> C.CDLL:
         L.taq_layer_forward_batched.argtypes = [C.POINTER(LayerDesc), vp, i32, vp, vp, vp, sz, vp]
         L.taq_kv_project_batched.argtypes = [C.POINTER(LayerDesc), vp, i32, vp, vp]
         L.taq_poll_device_status.argtypes = [vp, C.POINTER(i32)]
+        L.taq_static_workspace_capacity.restype = sz
+        L.taq_static_workspace_capacity.argtypes = []
+        L.taq_layer_forward_static.argtypes = [C.POINTER(LayerDesc), vp, vp, vp, vp, vp, vp, vp]
         for name in EXPORTS:
             f = getattr(L, name)
             if f.restype is C.c_int and name not in ("taq_version",):
@@ -217,6 +221,19 @@ def taq_layer_forward(desc: LayerDesc, x: torch.Tensor, Wq_packed: torch.Tensor,
         workspace = torch.empty(max(taq_workspace_bytes(desc, 1), 128), dtype=torch.uint8, device=x.device)
     _check(lib().taq_layer_forward(C.byref(desc), _ptr(x), _ptr(Wq_packed), _ptr(Wout_packed), _ptr(kv), _ptr(trig_mask), _ptr(y),
                                    _ptr(workspace), workspace.numel(), _stream(stream)))
+    return y
+
+
+def taq_static_workspace_capacity() -> int:
+    return lib().taq_static_workspace_capacity()
+
+
+def taq_layer_forward_static(desc: LayerDesc, x: torch.Tensor, Wq_packed: torch.Tensor, Wout_packed: torch.Tensor,
+                             kv: torch.Tensor, trig_mask: torch.Tensor, y: torch.Tensor, stream=None) -> torch.Tensor:
+    """The layer pass on the library's built-in scratch array.  ``y`` must be supplied: this wrapper, like the
+    entry point under it, allocates nothing."""
+    _check(lib().taq_layer_forward_static(C.byref(desc), _ptr(x), _ptr(Wq_packed), _ptr(Wout_packed), _ptr(kv), _ptr(trig_mask),
+                                          _ptr(y), _stream(stream)))
     return y
 
 

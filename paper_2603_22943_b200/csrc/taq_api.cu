@@ -366,6 +366,58 @@ taq_status taq_layer_forward_batched(const taq_layer_desc* d, const taq_request*
     return layer_forward_impl(d, reqs_dev, n_requests, x_f16_dev, nullptr, nullptr, nullptr, nullptr, y_f16_dev, workspace_dev, (cudaStream_t)stream);
 }
 
+// ---------------------------------------------------------------------------------------------------------
+// taq_layer_forward_static: the layer pass for callers that cannot provide a workspace.
+// The scratch (Q~, its scales, O) lives in a fixed array inside the library image; each GPU that loads the
+// library holds one copy until the process exits.
+// ---------------------------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_static_workspace[TAQ_STATIC_WORKSPACE_BYTES];
+
+// Device address of the array on the current device.  In host code the array's name is only a handle for the
+// runtime, not an address a kernel can use, so the address is asked for once per device and remembered.
+static taq_status static_workspace_ptr(unsigned char** out) {
+    static unsigned char* cache[64] = {nullptr};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+    if (dev < 0 || dev >= 64) return fail(TAQ_ERR_UNSUPPORTED, "device ordinal %d out of range", dev);
+    if (!cache[dev]) {
+        void* p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_static_workspace);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaGetSymbolAddress(static workspace)");
+        cache[dev] = static_cast<unsigned char*>(p);
+    }
+    *out = cache[dev];
+    return TAQ_OK;
+}
+
+size_t taq_static_workspace_capacity(void) { return (size_t)TAQ_STATIC_WORKSPACE_BYTES; }
+
+taq_status taq_layer_forward_static(const taq_layer_desc* d, const void* x_f16_dev, const void* Wq_packed_dev, const void* Wout_packed_dev,
+                                    const void* kv_packed_dev, const uint8_t* trig_mask_dev, void* y_f16_dev, void* stream) {
+    taq_status s = check_layer_desc(d);
+    if (s != TAQ_OK) return s;
+    if (d->batch > 65535) return fail(TAQ_ERR_SHAPE, "batch must be at most 65535");
+    const size_t need = workspace_layout(d, 1).total;
+    if (need > (size_t)TAQ_STATIC_WORKSPACE_BYTES)
+        return fail(TAQ_ERR_BUFFER_TOO_SMALL, "this layer needs %zu bytes of scratch, the built-in workspace holds %zu; use taq_layer_forward with a caller-owned workspace",
+                    need, (size_t)TAQ_STATIC_WORKSPACE_BYTES);
+    if (d->batch == 0 || d->n_query == 0) return TAQ_OK;
+    TAQ_REQUIRE_PTR(x_f16_dev);
+    TAQ_REQUIRE_PTR(Wq_packed_dev);
+    TAQ_REQUIRE_PTR(Wout_packed_dev);
+    TAQ_REQUIRE_PTR(kv_packed_dev);
+    TAQ_REQUIRE_PTR(y_f16_dev);
+    if (!trig_mask_dev) return fail(TAQ_ERR_INVALID_ARG, "trig_mask_dev is NULL");
+    unsigned char* ws = nullptr;
+    s = static_workspace_ptr(&ws);
+    if (s != TAQ_OK) return s;
+    // Every byte of Q~, its scales and O that a later stage reads is written by the stage before it in this same
+    // call, so nothing in the array has to start at zero and what the previous call left there is never read.
+    return layer_forward_impl(d, nullptr, 1, x_f16_dev, Wq_packed_dev, Wout_packed_dev, kv_packed_dev, trig_mask_dev, y_f16_dev, ws,
+                              (cudaStream_t)stream);
+}
+
 taq_status taq_poll_device_status(void* stream, int32_t* block_id_out) {
     int* status = nullptr;
     taq_status s = status_ptr(&status);
