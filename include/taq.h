@@ -116,7 +116,21 @@ typedef struct {
     size_t off_k_trigger;  /* fp16 [max_trigger][H][d], slot order = increasing token position */
     size_t off_v_trigger;  /* fp16 [max_trigger][H][d] */
     size_t off_trig_slot;  /* int32 [128]: slot of token j, or -1 if j is an ordinary token */
+    size_t off_operands;   /* [H] images of operand_head_bytes each (see below); operand_head_bytes = 0 when the
+                              shape is outside the tensor-core attention kernel (d not in {40,64,80,160} or T > 80) */
+    size_t operand_head_bytes;
 } taq_kv_layout;
+/* Operand image of one head: the same K~ and V~ once more, laid out as the tensor-core attention kernel wants them
+ * in shared memory, so that staging a head is one bulk copy.  Keys are padded to 80, the head width to a multiple
+ * of 16 (dp); tiles are K-major with the 128-byte swizzle (rows of 64 fp16, 16-byte chunk index XOR row mod 8).
+ *   K~ tile   ceil(dp/64) blocks of [80 keys][64] fp16: an ordinary row holds its int8 codes as fp16 integers, a
+ *             trigger row its fp16 values, padding zeros
+ *   V~^T tile 2 blocks of [dp channels][64 keys] fp16: fp16(code * scale) for ordinary rows, the fp16 value for
+ *             trigger rows
+ *   constants 1024 bytes: fp32 [80] logit factor of key j (K scale, or 1 for a trigger row, times log2(e)/sqrt(d);
+ *             0 for padding), then u32 [4] bitmap of trigger keys
+ * The images are derived data: taq_kv_project writes them; a block assembled by hand gets them from
+ * taq_kv_finalize. */
 
 taq_status taq_kv_layout_of(const taq_layer_desc* desc, taq_kv_layout* out);
 size_t taq_kv_bytes(const taq_layer_desc* desc);               /* batch * block_bytes; 0 if invalid */
@@ -131,6 +145,10 @@ size_t taq_kv_bytes(const taq_layer_desc* desc);               /* batch * block_
 taq_status taq_kv_project(const taq_layer_desc* desc, const void* ctx_f16_dev, const void* Wk_packed_dev,
                           const void* Wv_packed_dev, const uint8_t* trig_mask_dev, void* kv_packed_dev,
                           size_t kv_bytes, void* stream);
+
+/* Rebuilds the operand images of `batch` blocks from their code / scale / trigger-row / slot sections.  Needed
+ * only for blocks that were not written by taq_kv_project. */
+taq_status taq_kv_finalize(const taq_layer_desc* desc, void* kv_packed_dev, size_t kv_bytes, void* stream);
 
 /* Dequant-GEMM on packed weights (the to_q / to_out projections; "quantizing all remaining ... pathways",
  * Sec. III-B last paragraph): y = x W^T (+ bias), W^ = fp16(code * scale) as the matrix operand, fp32

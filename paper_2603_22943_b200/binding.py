@@ -24,7 +24,7 @@ EXPORTS = [
     "taq_unpack_weights", "taq_quantize_rows", "taq_kv_layout_of", "taq_kv_bytes", "taq_kv_project",
     "taq_quantized_linear", "taq_cross_attention", "taq_workspace_bytes", "taq_layer_forward",
     "taq_layer_forward_batched", "taq_kv_project_batched", "taq_poll_device_status",
-    "taq_static_workspace_capacity", "taq_layer_forward_static",
+    "taq_static_workspace_capacity", "taq_layer_forward_static", "taq_kv_finalize",
 ]
 
 
@@ -49,7 +49,8 @@ class LayerDesc(C.Structure):
 
 class KvLayout(C.Structure):
     _fields_ = [(n, C.c_size_t) for n in ("block_bytes", "off_k_codes", "off_v_codes", "off_k_scales", "off_v_scales",
-                                           "off_k_trigger", "off_v_trigger", "off_trig_slot")]
+                                           "off_k_trigger", "off_v_trigger", "off_trig_slot", "off_operands",
+                                           "operand_head_bytes")]
 
 
 class Request(C.Structure):
@@ -82,6 +83,7 @@ def lib() -> C.CDLL:
         L.taq_kv_bytes.restype = sz
         L.taq_kv_bytes.argtypes = [C.POINTER(LayerDesc)]
         L.taq_kv_project.argtypes = [C.POINTER(LayerDesc), vp, vp, vp, vp, vp, sz, vp]
+        L.taq_kv_finalize.argtypes = [C.POINTER(LayerDesc), vp, sz, vp]
         L.taq_quantized_linear.argtypes = [C.POINTER(WeightDesc), vp, i64, vp, vp, i32, i32, vp, vp]
         L.taq_cross_attention.argtypes = [C.POINTER(LayerDesc), vp, vp, vp, vp, vp, vp]
         L.taq_workspace_bytes.restype = sz
@@ -185,6 +187,12 @@ def taq_kv_project(desc: LayerDesc, ctx: torch.Tensor, Wk_packed: torch.Tensor, 
         kv = torch.zeros(max(taq_kv_bytes(desc), 16), dtype=torch.uint8, device=ctx.device)
     _check(lib().taq_kv_project(C.byref(desc), _ptr(ctx), _ptr(Wk_packed), _ptr(Wv_packed), _ptr(trig_mask), _ptr(kv),
                                 kv.numel(), _stream(stream)))
+    return kv
+
+
+def taq_kv_finalize(desc: LayerDesc, kv: torch.Tensor, stream=None) -> torch.Tensor:
+    """Rebuilds the operand images of hand-assembled K~/V~ blocks."""
+    _check(lib().taq_kv_finalize(C.byref(desc), _ptr(kv), kv.numel(), _stream(stream)))
     return kv
 
 

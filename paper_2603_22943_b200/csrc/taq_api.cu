@@ -200,7 +200,9 @@ static taq_status kv_project_impl(const taq_layer_desc* d, const taq_request* re
         s = run_linear(a, n_z, st);
         if (s != TAQ_OK) return s;
     }
-    return TAQ_OK;
+    // the same rows once more as MMA-ready operand images for the attention kernel
+    cudaError_t e = launch_kv_operands(*d, kv, reqs, reqs ? n_z : d->batch, st);
+    return e == cudaSuccess ? TAQ_OK : cuda_fail(e, "K/V operand image launch");
 }
 
 taq_status taq_kv_project(const taq_layer_desc* d, const void* ctx_f16_dev, const void* Wk_packed_dev, const void* Wv_packed_dev,
@@ -208,6 +210,7 @@ taq_status taq_kv_project(const taq_layer_desc* d, const void* ctx_f16_dev, cons
     taq_status s = check_layer_desc(d);
     if (s != TAQ_OK) return s;
     if (d->batch == 0) return TAQ_OK;
+    if (d->batch > 65535) return fail(TAQ_ERR_SHAPE, "batch must be at most 65535");
     TAQ_REQUIRE_PTR(ctx_f16_dev);
     TAQ_REQUIRE_PTR(Wk_packed_dev);
     TAQ_REQUIRE_PTR(Wv_packed_dev);
@@ -216,6 +219,18 @@ taq_status taq_kv_project(const taq_layer_desc* d, const void* ctx_f16_dev, cons
     const size_t need = taq_kv_bytes(d);
     if (kv_bytes < need) return fail(TAQ_ERR_BUFFER_TOO_SMALL, "kv buffer has %zu bytes, %zu needed", kv_bytes, need);
     return kv_project_impl(d, nullptr, 1, ctx_f16_dev, Wk_packed_dev, Wv_packed_dev, trig_mask_dev, kv_packed_dev, (cudaStream_t)stream);
+}
+
+taq_status taq_kv_finalize(const taq_layer_desc* d, void* kv_packed_dev, size_t kv_bytes, void* stream) {
+    taq_status s = check_layer_desc(d);
+    if (s != TAQ_OK) return s;
+    if (d->batch == 0) return TAQ_OK;
+    if (d->batch > 65535) return fail(TAQ_ERR_SHAPE, "batch must be at most 65535");
+    TAQ_REQUIRE_PTR(kv_packed_dev);
+    const size_t need = taq_kv_bytes(d);
+    if (kv_bytes < need) return fail(TAQ_ERR_BUFFER_TOO_SMALL, "kv buffer has %zu bytes, %zu needed", kv_bytes, need);
+    cudaError_t e = launch_kv_operands(*d, kv_packed_dev, nullptr, d->batch, (cudaStream_t)stream);
+    return e == cudaSuccess ? TAQ_OK : cuda_fail(e, "K/V operand image launch");
 }
 
 taq_status taq_kv_project_batched(const taq_layer_desc* d, const taq_request* reqs_dev, int32_t n_requests, const void* ctx_f16_dev, void* stream) {

@@ -1,12 +1,15 @@
-// Fused TAQ attention on the Blackwell tensor cores (tcgen05 + TMEM), one pass, nothing but Q~ in and O out:
-//   S = Q~ K~^T          tcgen05.mma, fp16 operands holding the int8 codes exactly (trigger rows: their fp16 values)
-//   A = softmax(S * scale)   one thread per query row, the row's 80 scores live in its registers (TMEM lane)
-//   A^ (Eq. 3)            ordinary columns -> uint8 code, trigger columns -> fp16, both in units of 1/255
-//   O = A^ V~             tcgen05.mma with the probabilities as the A operand, V~^T (fp16) as B; O = acc / 255
-// A CTA owns 128 query rows of one sequence and walks over a group of heads.  Per head the four worker warps stage
-// the head's mixed-precision K~ and V~^T (Eq. 2) and the row tile of Q~ codes into 128-byte-swizzled K-major
-// operand tiles, a fifth warp issues the MMAs, and the workers (thread = row = TMEM lane) run the softmax and the
-// epilogue.  Several CTAs share an SM, so one CTA's staging overlaps another's MMA and softmax.
+// Fused TAQ attention on the Blackwell tensor cores (tcgen05 + TMEM): Q~ in, O out, nothing else touches HBM.
+//   S = Q~ K~^T             tcgen05.mma; the fp16 operands hold the int8 codes exactly (trigger rows: fp16 values)
+//   A = softmax(S * scale)  one thread per query row; the row's 80 scores live in its registers (TMEM lane)
+//   A^ (Eq. 3)              ordinary columns -> uint8 code, trigger columns -> fp16, both in units of 1/255
+//   O = A^ V~               tcgen05.mma with the probabilities as the A operand and V~^T (fp16) as B; O = acc/255
+// A CTA owns 128 query rows of one sequence and walks over a group of heads, software-pipelined:
+//   warps 0-3  thread = query row = TMEM lane: stage the row's Q~ codes of the next head as an fp16 operand tile,
+//              softmax + Eq. 3 of the current head, epilogue of the previous head;
+//   warp 4     one thread issues the MMAs: S of head h+1 is in flight while the rows are in the softmax of head h;
+//   warp 5     one thread fetches each head's K~/V~ operand image (written once per prompt by the K/V projection)
+//              with a single bulk copy, one head ahead.
+// Two CTAs share an SM for head widths up to 80, so one CTA's loads overlap the other's arithmetic.
 #include "taq_ptx.cuh"
 #include "taq_sm100.cuh"
 
@@ -14,10 +17,10 @@ namespace taq {
 
 namespace {
 
-constexpr int TP = 80;           // keys padded to a multiple of 16
+constexpr int TP = kOperandKeys;     // keys padded to a multiple of 16
 constexpr int ROWS = 128;
-constexpr int NWORK = 128;
-constexpr int ATT_THREADS = 160;
+constexpr int ATT_THREADS = 192;
+constexpr int MMA_WARP = 4, COPY_WARP = 5;
 
 template <int D>
 struct Cfg {
@@ -26,26 +29,28 @@ struct Cfg {
     static constexpr int A_BLOCK = ROWS * 128;
     static constexpr int K_BLOCK = TP * 128;
     static constexpr int VT_BLOCK = DP * 128;
-    static constexpr int KBP = 2;                            // k-blocks of the probability tile (64 + 16 keys)
-    static constexpr int OFF_A = 0;
-    static constexpr int OFF_K = OFF_A + KBQ * A_BLOCK;
-    static constexpr int OFF_VT = OFF_K + KBQ * K_BLOCK;
-    static constexpr int OFF_P = OFF_VT + KBP * VT_BLOCK;
-    static constexpr int OFF_MISC = OFF_P + KBP * A_BLOCK;
-    static constexpr int TOTAL = OFF_MISC + 2048 + 1024;     // misc block + slack for 1024-byte alignment
-    static constexpr uint32_t TMEM_COLS = (TP + DP) <= 128 ? 128 : 256;
-    static_assert(VT_BLOCK % 1024 == 0 && K_BLOCK % 1024 == 0, "operand blocks must keep 1024-byte alignment");
+    static constexpr int K_BYTES = KBQ * K_BLOCK;
+    static constexpr int VT_BYTES = 2 * VT_BLOCK;
+    static constexpr int HEAD_BYTES = K_BYTES + VT_BYTES + kOperandConstBytes;
+    static constexpr int KVBUF = D <= 64 ? 2 : 1;            // K~/V~ images in flight
+    static constexpr int OBUF = D == 40 ? 2 : 1;             // O accumulators in TMEM
+    static constexpr int OFF_KV = 0;
+    static constexpr int OFF_Q = OFF_KV + KVBUF * HEAD_BYTES;
+    static constexpr int OFF_P = OFF_Q + KBQ * A_BLOCK;
+    static constexpr int OFF_MISC = OFF_P + 2 * A_BLOCK;
+    static constexpr int TOTAL = OFF_MISC + 1024 + 1024;     // misc block + slack for 1024-byte alignment
+    static constexpr uint32_t TMEM_S = 0, TMEM_O = 2 * TP;
+    static constexpr uint32_t TMEM_COLS = (2 * TP + OBUF * DP) <= 256 ? 256 : 512;
+    static constexpr int CTAS_PER_SM = (2 * (TOTAL + 1024) <= 232448 && TMEM_COLS == 256) ? 2 : 1;
+    static_assert(HEAD_BYTES % 1024 == 0 && K_BYTES % 1024 == 0 && VT_BLOCK % 1024 == 0, "operand tiles must keep 1024-byte alignment");
+    static_assert(TOTAL <= 232448, "shared memory budget");
 };
 
 struct Misc {
-    uint64_t bar_ab, bar_s, bar_p, bar_o;
+    uint64_t kv_full[2], kv_free[2], q_full, s_full[2], p_full, o_full[2], drain;
     uint32_t tmem_base;
     volatile int abort_flag;
-    int slot[TP];            // fp16 slot of key j, -1 for an ordinary key, -2 for padding
-    float2 fm[TP];           // {logit factor of key j (K scale * log2 e / sqrt d), rounding constant of Eq. 3}
-    float vs[TP];            // V scale of key j
 };
-static_assert(sizeof(Misc) <= 2048, "misc block");
 
 __device__ __forceinline__ float ex2_approx(float x) {
     float y;
@@ -70,8 +75,41 @@ __device__ __forceinline__ uint4 codes8_to_half(uint2 raw) {
     return make_uint4(o[0], o[1], o[2], o[3]);
 }
 
-template <int D>
-__global__ void __launch_bounds__(ATT_THREADS, 2) attention_sm100_kernel(const AttnArgs a, const int heads_per_cta) {
+// Query codes (or fp16 values) of one row and head, held in registers between the global load and the store
+// into the operand tile.
+template <int D, bool Q8>
+struct QRegs {
+    static constexpr int CH = Cfg<D>::DP / 8;
+    uint4 v[Q8 ? (CH + 1) / 2 : CH];
+    __device__ __forceinline__ void load(const void* q, size_t elem_off, bool valid) {
+        if (Q8) {
+#pragma unroll
+            for (int i = 0; i < (CH + 1) / 2; ++i) {
+                uint2 lo = make_uint2(0, 0), hi = make_uint2(0, 0);
+                if (valid && (2 * i) * 8 < D) lo = *reinterpret_cast<const uint2*>((const int8_t*)q + elem_off + (2 * i) * 8);
+                if (valid && (2 * i + 1) * 8 < D) hi = *reinterpret_cast<const uint2*>((const int8_t*)q + elem_off + (2 * i + 1) * 8);
+                v[i] = make_uint4(lo.x, lo.y, hi.x, hi.y);
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < CH; ++i) {
+                v[i] = make_uint4(0, 0, 0, 0);
+                if (valid && i * 8 < D) v[i] = *reinterpret_cast<const uint4*>((const __half*)q + elem_off + i * 8);
+            }
+        }
+    }
+    // chunk cc (8 channels) as fp16 operands; channels beyond D are zero (a zero int8 code maps to fp16 zero)
+    __device__ __forceinline__ uint4 chunk(int cc) const {
+        if (Q8) {
+            const uint4 w = v[cc / 2];
+            return codes8_to_half((cc & 1) ? make_uint2(w.z, w.w) : make_uint2(w.x, w.y));
+        }
+        return v[cc];
+    }
+};
+
+template <int D, bool Q8, bool TAIL_ONLY>
+__global__ void __launch_bounds__(ATT_THREADS, Cfg<D>::CTAS_PER_SM) attention_sm100_kernel(const AttnArgs a, const int heads_per_cta) {
     using C = Cfg<D>;
     constexpr int DP = C::DP;
     extern __shared__ unsigned char smem_dyn[];
@@ -84,193 +122,108 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) attention_sm100_kernel(const A
     const int b = a.reqs ? 0 : zb;
     const int row0 = blockIdx.x * ROWS;
     const int h_begin = blockIdx.y * heads_per_cta;
+    const int HG = heads_per_cta;
 
     if (tid == 0) {
-        ptx::mbar_init(&misc->bar_ab, NWORK);
-        ptx::mbar_init(&misc->bar_s, 1);
-        ptx::mbar_init(&misc->bar_p, NWORK);
-        ptx::mbar_init(&misc->bar_o, 1);
+        for (int i = 0; i < 2; ++i) {
+            ptx::mbar_init(&misc->kv_full[i], 1);
+            ptx::mbar_init(&misc->kv_free[i], 1);
+            ptx::mbar_init(&misc->s_full[i], 1);
+            ptx::mbar_init(&misc->o_full[i], 1);
+        }
+        ptx::mbar_init(&misc->q_full, ROWS);
+        ptx::mbar_init(&misc->p_full, ROWS);
+        ptx::mbar_init(&misc->drain, 1);
         misc->abort_flag = 0;
         ptx::mbar_fence_init();
     }
-    if (warp == 4) ptx::tmem_alloc(&misc->tmem_base, C::TMEM_COLS);
+    if (warp == MMA_WARP) ptx::tmem_alloc(&misc->tmem_base, C::TMEM_COLS);
     ptx::tc_fence_before_sync();
     __syncthreads();
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = misc->tmem_base;
-    const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + TP;
 
-    if (warp == 4) {
+    const taq_kv_layout KL = kv_layout(H, T, D, a.max_trigger);
+    const uint8_t* blk = a.reqs ? (const uint8_t*)a.reqs[zb].kv : (const uint8_t*)a.kv + (size_t)b * KL.block_bytes;
+
+    if (warp == COPY_WARP) {
+        // ---------------- K~/V~ operand images, one head ahead ----------------
+        if (lane == 0) {
+            const uint8_t* img = blk + KL.off_operands + (size_t)h_begin * KL.operand_head_bytes;
+            int issued = 0;
+            for (int hi = 0; hi < HG; ++hi) {
+                const int buf = hi % C::KVBUF;
+                if (hi >= C::KVBUF && !ptx::mbar_wait(&misc->kv_free[buf], ((hi / C::KVBUF) - 1) & 1)) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; }
+                if (misc->abort_flag) break;
+                ptx::mbar_arrive_expect_tx(&misc->kv_full[buf], C::HEAD_BYTES);
+                ptx::bulk_load(smem + C::OFF_KV + buf * C::HEAD_BYTES, img + (size_t)hi * KL.operand_head_bytes, C::HEAD_BYTES, &misc->kv_full[buf]);
+                issued = hi + 1;
+            }
+            if (misc->abort_flag) {   // let copies that were issued land before the CTA goes away
+                for (int hi = issued > C::KVBUF ? issued - C::KVBUF : 0; hi < issued; ++hi) (void)ptx::mbar_wait(&misc->kv_full[hi % C::KVBUF], (hi / C::KVBUF) & 1);
+            }
+        }
+    } else if (warp == MMA_WARP) {
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
-            const uint32_t a_addr = ptx::smem_u32(smem + C::OFF_A), k_addr = ptx::smem_u32(smem + C::OFF_K);
-            const uint32_t p_addr = ptx::smem_u32(smem + C::OFF_P), vt_addr = ptx::smem_u32(smem + C::OFF_VT);
-            for (int hi = 0; hi < heads_per_cta; ++hi) {
-                const uint32_t ph = hi & 1;
-                if (!ptx::mbar_wait(&misc->bar_ab, ph)) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; }
-                if (misc->abort_flag) break;
+            const uint32_t q_addr = ptx::smem_u32(smem + C::OFF_Q), p_addr = ptx::smem_u32(smem + C::OFF_P);
+            auto issue_s = [&](int hi) -> bool {
+                const int buf = hi % C::KVBUF;
+                if (!ptx::mbar_wait(&misc->kv_full[buf], (hi / C::KVBUF) & 1) || !ptx::mbar_wait(&misc->q_full, hi & 1)) return false;
                 ptx::tc_fence_after_sync();
+                const uint32_t k_addr = ptx::smem_u32(smem + C::OFF_KV + buf * C::HEAD_BYTES);
 #pragma unroll
                 for (int ks = 0; ks < DP / 16; ++ks)
-                    ptx::mma_f16_ss(tmem_s, ptx::desc_k_sw128(a_addr + (ks / 4) * C::A_BLOCK + (ks % 4) * 32),
+                    ptx::mma_f16_ss(tmem_base + C::TMEM_S + (hi & 1) * TP, ptx::desc_k_sw128(q_addr + (ks / 4) * C::A_BLOCK + (ks % 4) * 32),
                                     ptx::desc_k_sw128(k_addr + (ks / 4) * C::K_BLOCK + (ks % 4) * 32), ptx::idesc_f16_m128(TP), ks != 0);
-                ptx::mma_commit(&misc->bar_s);
-                if (!ptx::mbar_wait(&misc->bar_p, ph)) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; }
-                if (misc->abort_flag) break;
+                ptx::mma_commit(&misc->s_full[hi & 1]);
+                return true;
+            };
+            auto issue_pv = [&](int hi) -> bool {
+                const int buf = hi % C::KVBUF;
+                if (!ptx::mbar_wait(&misc->p_full, hi & 1)) return false;
                 ptx::tc_fence_after_sync();
+                const uint32_t vt_addr = ptx::smem_u32(smem + C::OFF_KV + buf * C::HEAD_BYTES + C::K_BYTES);
 #pragma unroll
                 for (int ks = 0; ks < TP / 16; ++ks)
-                    ptx::mma_f16_ss(tmem_o, ptx::desc_k_sw128(p_addr + (ks / 4) * C::A_BLOCK + (ks % 4) * 32),
+                    ptx::mma_f16_ss(tmem_base + C::TMEM_O + (hi % C::OBUF) * DP, ptx::desc_k_sw128(p_addr + (ks / 4) * C::A_BLOCK + (ks % 4) * 32),
                                     ptx::desc_k_sw128(vt_addr + (ks / 4) * C::VT_BLOCK + (ks % 4) * 32), ptx::idesc_f16_m128(DP), ks != 0);
-                ptx::mma_commit(&misc->bar_o);
+                ptx::mma_commit(&misc->o_full[hi % C::OBUF]);
+                ptx::mma_commit(&misc->kv_free[buf]);
+                return true;
+            };
+            bool ok = issue_s(0);
+            for (int hi = 0; hi < HG && ok && !misc->abort_flag; ++hi) {
+                if (C::KVBUF == 2) {          // S of the next head first: it runs under this head's softmax
+                    if (hi + 1 < HG) ok = issue_s(hi + 1);
+                    if (ok) ok = issue_pv(hi);
+                } else {                      // one K~/V~ buffer: the next head's image lands only after this PV
+                    ok = issue_pv(hi);
+                    if (ok && hi + 1 < HG) ok = issue_s(hi + 1);
+                }
+            }
+            if (!ok) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; }
+            if (misc->abort_flag) {           // wait (bounded) for whatever was issued before TMEM is given back
+                ptx::mma_commit(&misc->drain);
+                (void)ptx::mbar_wait(&misc->drain, 0);
             }
         }
     } else {
-        // ---------------- workers: thread = query row = TMEM lane ----------------
-        const taq_kv_layout KL = kv_layout(H, T, D, a.max_trigger);
-        const uint8_t* blk = a.reqs ? (const uint8_t*)a.reqs[zb].kv : (const uint8_t*)a.kv + (size_t)b * KL.block_bytes;
-        const uint8_t* mask = a.reqs ? a.reqs[zb].trig_mask : a.mask + (size_t)b * T;
-        const int32_t* gslot = (const int32_t*)(blk + KL.off_trig_slot);
-        const __half* kt = (const __half*)(blk + KL.off_k_trigger);
-        const __half* vt = (const __half*)(blk + KL.off_v_trigger);
+        // ---------------- row threads: thread = query row = TMEM lane ----------------
         const int n = row0 + tid;
         const bool valid = n < a.n_query;
         const size_t grow = (size_t)zb * a.n_query + (valid ? n : 0);
-        const float logit_unit = 1.4426950408889634f / sqrtf((float)D);
         const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
+        const float inv255 = 1.0f / 255.0f;
         bool alive = true;
 
-        for (int hi = 0; hi < heads_per_cta && alive; ++hi) {
-            const int h = h_begin + hi;
-            const uint32_t ph = hi & 1;
-            const int8_t* kc = (const int8_t*)(blk + KL.off_k_codes) + (size_t)h * T * D;
-            const int8_t* vc = (const int8_t*)(blk + KL.off_v_codes) + (size_t)h * T * D;
-            const float* ks = (const float*)(blk + KL.off_k_scales) + (size_t)h * T;
-            const float* vs = (const float*)(blk + KL.off_v_scales) + (size_t)h * T;
-
-            // per-key constants of this head
-            if (tid < TP) {
-                const int j = tid;
-                int sl = -2;
-                float f = 0.f, m = 0.f, v = 0.f;
-                if (j < T) {
-                    sl = gslot[j];
-                    f = (sl >= 0 ? 1.0f : ks[j]) * logit_unit;
-                    m = mask[j] ? 0.f : 12582912.f;        // (x + 1.5*2^23) - 1.5*2^23 rounds x to the nearest-even integer
-                    v = vs[j];
-                }
-                misc->slot[j] = sl;
-                misc->fm[j] = make_float2(f, m);
-                misc->vs[j] = v;
-            }
-            asm volatile("bar.sync 1, 128;" ::: "memory");
-
-            // K~ tile: [TP keys][DP], ordinary rows as exact fp16 integers, trigger rows as their fp16 values (Eq. 2)
-            for (int idx = tid; idx < TP * (DP / 8); idx += NWORK) {
-                const int j = idx / (DP / 8), cc = idx % (DP / 8);
-                uint4 v = make_uint4(0, 0, 0, 0);
-                const int sl = misc->slot[j];
-                if (cc * 8 < D && sl != -2) {
-                    if (sl >= 0) v = *reinterpret_cast<const uint4*>(kt + ((size_t)sl * H + h) * D + cc * 8);
-                    else v = codes8_to_half(*reinterpret_cast<const uint2*>(kc + (size_t)j * D + cc * 8));
-                }
-                *reinterpret_cast<uint4*>(smem + C::OFF_K + (cc / 8) * C::K_BLOCK + ptx::sw128_offset(j, cc % 8)) = v;
-            }
-            // V~^T tile: [DP channels][TP keys]; ordinary rows are the fp16 operand of code * scale
-            for (int idx = tid; idx < DP * (TP / 8); idx += NWORK) {
-                const int c = idx % DP, jc = idx / DP;
-                uint32_t pk[4];
-#pragma unroll
-                for (int i2 = 0; i2 < 4; ++i2) {
-                    float v2[2];
-#pragma unroll
-                    for (int e = 0; e < 2; ++e) {
-                        const int j = jc * 8 + i2 * 2 + e;
-                        const int sl = misc->slot[j];
-                        float v = 0.f;
-                        if (c < D && sl != -2) {
-                            if (sl >= 0) v = __half2float(vt[((size_t)sl * H + h) * D + c]);
-                            else v = __fmul_rn((float)vc[(size_t)j * D + c], misc->vs[j]);
-                        }
-                        v2[e] = v;
-                    }
-                    __half2 hv = __floats2half2_rn(v2[0], v2[1]);
-                    pk[i2] = *reinterpret_cast<uint32_t*>(&hv);
-                }
-                *reinterpret_cast<uint4*>(smem + C::OFF_VT + (jc / 8) * C::VT_BLOCK + ptx::sw128_offset(c, jc % 8)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-            }
-            // Q~ tile: this thread's row
-            float sq = 1.0f;
-            {
-#pragma unroll
-                for (int cc = 0; cc < DP / 8; ++cc) {
-                    uint4 v = make_uint4(0, 0, 0, 0);
-                    if (cc * 8 < D && valid) {
-                        if (a.q_bits == 8) v = codes8_to_half(*reinterpret_cast<const uint2*>((const int8_t*)a.q + grow * Cch + h * D + cc * 8));
-                        else v = *reinterpret_cast<const uint4*>((const __half*)a.q + grow * Cch + h * D + cc * 8);
-                    }
-                    *reinterpret_cast<uint4*>(smem + C::OFF_A + (cc / 8) * C::A_BLOCK + ptx::sw128_offset(tid, cc % 8)) = v;
-                }
-                if (a.q_bits == 8) sq = valid ? a.q_scales[grow * H + h] : 0.f;
-            }
-            ptx::fence_proxy_async_smem();
-            ptx::mbar_arrive(&misc->bar_ab);
-
-            // ---- scores -> softmax -> Eq. 3 -> probability operand ----
-            alive = __all_sync(0xffffffffu, ptx::mbar_wait(&misc->bar_s, ph) && !misc->abort_flag);
-            if (!alive) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; break; }
-            ptx::tc_fence_after_sync();
-            uint32_t u[TP / 16][16];
-#pragma unroll
-            for (int c = 0; c < TP / 16; ++c) ptx::tmem_ld16(tmem_s + lane_addr + c * 16, u[c]);
-            ptx::tmem_ld_wait(u[0]);
-#pragma unroll
-            for (int c = 1; c < TP / 16; ++c) ptx::reg_fence(u[c]);
-            float s[TP];
-            float mx = -INFINITY;
-#pragma unroll
-            for (int j = 0; j < TP; ++j) {
-                s[j] = __uint_as_float(u[j / 16][j % 16]) * misc->fm[j].x;
-                if (j >= 64 || T <= 64) { if (j >= T) s[j] = -INFINITY; }
-                mx = fmaxf(mx, s[j]);
-            }
-            const float msq = mx * sq;
-            float sum = 0.f;
-#pragma unroll
-            for (int j = 0; j < TP; ++j) {
-                float arg = fmaf(s[j], sq, -msq);
-                if (j >= 64 || T <= 64) { if (j >= T) arg = -INFINITY; }      // padded keys: weight exactly 0, also when sq = 0
-                s[j] = ex2_approx(arg);
-                sum += s[j];
-            }
-            const float k255 = __fdividef(255.0f, sum);
-#pragma unroll
-            for (int jc = 0; jc < TP / 8; ++jc) {
-                uint32_t pk[4];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int j = jc * 8 + 2 * i;
-                    const float m0 = misc->fm[j].y, m1 = misc->fm[j + 1].y;
-                    const float x0 = __fadd_rn(__fadd_rn(s[j] * k255, m0), -m0);
-                    const float x1 = __fadd_rn(__fadd_rn(s[j + 1] * k255, m1), -m1);
-                    __half2 hv = __floats2half2_rn(x0, x1);
-                    pk[i] = *reinterpret_cast<uint32_t*>(&hv);
-                }
-                *reinterpret_cast<uint4*>(smem + C::OFF_P + (jc / 8) * C::A_BLOCK + ptx::sw128_offset(tid, jc % 8)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-            }
-            ptx::fence_proxy_async_smem();
-            ptx::tc_fence_before_sync();
-            ptx::mbar_arrive(&misc->bar_p);
-
-            // ---- O = acc / 255 -> fp16 ----
-            alive = __all_sync(0xffffffffu, ptx::mbar_wait(&misc->bar_o, ph) && !misc->abort_flag);
-            if (!alive) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; break; }
-            ptx::tc_fence_after_sync();
-            __half* orow = a.o + grow * Cch + h * D;
+        auto store_o = [&](int hi) {        // O of head hi: acc / 255 -> fp16
+            __half* orow = a.o + grow * Cch + (h_begin + hi) * D;
+            const uint32_t t_o = tmem_base + C::TMEM_O + (hi % C::OBUF) * DP + lane_addr;
 #pragma unroll
             for (int c = 0; c < DP; c += 16) {
                 uint32_t v[16];
-                ptx::tmem_ld16(tmem_o + lane_addr + c, v);
+                ptx::tmem_ld16(t_o + c, v);
                 ptx::tmem_ld_wait(v);
 #pragma unroll
                 for (int half8 = 0; half8 < 2; ++half8) {
@@ -278,7 +231,7 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) attention_sm100_kernel(const A
                         uint32_t pk[4];
 #pragma unroll
                         for (int i = 0; i < 4; ++i) {
-                            __half2 hv = __floats2half2_rn(__uint_as_float(v[half8 * 8 + 2 * i]) * (1.0f / 255.0f), __uint_as_float(v[half8 * 8 + 2 * i + 1]) * (1.0f / 255.0f));
+                            __half2 hv = __floats2half2_rn(__uint_as_float(v[half8 * 8 + 2 * i]) * inv255, __uint_as_float(v[half8 * 8 + 2 * i + 1]) * inv255);
                             pk[i] = *reinterpret_cast<uint32_t*>(&hv);
                         }
                         *reinterpret_cast<uint4*>(orow + c + half8 * 8) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
@@ -286,48 +239,171 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) attention_sm100_kernel(const A
                 }
             }
             ptx::tc_fence_before_sync();
+        };
+        auto stage_q = [&](const QRegs<D, Q8>& qr) {
+#pragma unroll
+            for (int cc = 0; cc < DP / 8; ++cc)
+                *reinterpret_cast<uint4*>(smem + C::OFF_Q + (cc / 8) * C::A_BLOCK + ptx::sw128_offset(tid, cc % 8)) = qr.chunk(cc);
+            ptx::fence_proxy_async_smem();
+            ptx::mbar_arrive(&misc->q_full);
+        };
+
+        QRegs<D, Q8> qr;
+        qr.load(a.q, grow * Cch + (size_t)h_begin * D, valid);
+        float sq = 1.0f, sq_next = 1.0f;
+        if (Q8) sq = valid ? a.q_scales[grow * H + h_begin] : 0.f;
+        stage_q(qr);
+
+        for (int hi = 0; hi < HG; ++hi) {
+            const uint32_t ph = hi & 1;
+            const bool more = hi + 1 < HG;
+            if (more) {                         // next head's query codes: in flight while this head's S is awaited
+                qr.load(a.q, grow * Cch + (size_t)(h_begin + hi + 1) * D, valid);
+                if (Q8) sq_next = valid ? a.q_scales[grow * H + h_begin + hi + 1] : 0.f;
+            }
+            alive = __all_sync(0xffffffffu, ptx::mbar_wait(&misc->s_full[ph], (hi >> 1) & 1) && !misc->abort_flag);
+            if (!alive) break;
+            ptx::tc_fence_after_sync();
+            uint32_t u[TP / 16][16];
+#pragma unroll
+            for (int c = 0; c < TP / 16; ++c) ptx::tmem_ld16(tmem_base + C::TMEM_S + ph * TP + lane_addr + c * 16, u[c]);
+            ptx::tmem_ld_wait(u[0]);
+#pragma unroll
+            for (int c = 1; c < TP / 16; ++c) ptx::reg_fence(u[c]);
+            ptx::tc_fence_before_sync();
+            if (more) stage_q(qr);              // S of this head is complete, so the Q~ tile is free again
+
+            // ---- softmax over the keys: logits in units of log2 ----
+            const OperandConsts* cst = reinterpret_cast<const OperandConsts*>(smem + C::OFF_KV + (hi % C::KVBUF) * C::HEAD_BYTES + C::K_BYTES + C::VT_BYTES);
+            float s[TP];
+#pragma unroll
+            for (int j4 = 0; j4 < TP / 4; ++j4) {
+                const float4 f = *reinterpret_cast<const float4*>(&cst->logit_factor[4 * j4]);
+                s[4 * j4 + 0] = __uint_as_float(u[j4 / 4][(j4 % 4) * 4 + 0]) * f.x;
+                s[4 * j4 + 1] = __uint_as_float(u[j4 / 4][(j4 % 4) * 4 + 1]) * f.y;
+                s[4 * j4 + 2] = __uint_as_float(u[j4 / 4][(j4 % 4) * 4 + 2]) * f.z;
+                s[4 * j4 + 3] = __uint_as_float(u[j4 / 4][(j4 % 4) * 4 + 3]) * f.w;
+            }
+            const uint32_t tb0 = cst->trig_bits[0], tb1 = cst->trig_bits[1], tb2 = cst->trig_bits[2];
+#pragma unroll
+            for (int j = 0; j < TP; ++j)
+                if (j >= 64 || !TAIL_ONLY) { if (j >= T) s[j] = -INFINITY; }
+            float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+            for (int j = 0; j < TP; ++j) m4[j & 3] = fmaxf(m4[j & 3], s[j]);
+            const float mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
+            const float msq = mx * sq;
+            float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int j = 0; j < TP; ++j) {
+                float arg = fmaf(s[j], sq, -msq);
+                if (j >= 64 || !TAIL_ONLY) { if (j >= T) arg = -INFINITY; }      // padded keys: weight exactly 0, also when sq = 0
+                s[j] = ex2_approx(arg);
+                sum4[j & 3] += s[j];
+            }
+            const float k255 = __fdividef(255.0f, (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]));
+
+            // the P tile is free once the previous head's PV has completed
+            if (hi > 0) {
+                alive = __all_sync(0xffffffffu, ptx::mbar_wait(&misc->o_full[(hi - 1) % C::OBUF], ((hi - 1) / C::OBUF) & 1) && !misc->abort_flag);
+                if (!alive) break;
+                ptx::tc_fence_after_sync();
+                if (C::OBUF == 1) store_o(hi - 1);   // one O accumulator: empty it before the next PV may start
+            }
+
+            // ---- Eq. 3: ordinary columns -> rint(255 p) (exact, ties to even), trigger columns -> fp16(255 p) ----
+            // fma(e, 255/sum, 1.5 * 2^23 + 0x6400) leaves the integer code in the low byte and 0x64 above it, which
+            // read as fp16 is 1024 + code.
+            const __half2 h1024 = __floats2half2_rn(1024.f, 1024.f);
+#pragma unroll
+            for (int jc = 0; jc < TP / 8; ++jc) {
+                const uint32_t word = jc < 4 ? tb0 : (jc < 8 ? tb1 : tb2);
+                const uint32_t bits = (word >> (8 * (jc % 4))) & 0xFFu;
+                uint32_t pk[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int j = jc * 8 + 2 * i;
+                    const uint32_t x0 = __float_as_uint(fmaf(s[j], k255, 12608512.0f));
+                    const uint32_t x1 = __float_as_uint(fmaf(s[j + 1], k255, 12608512.0f));
+                    uint32_t w = __byte_perm(x0, x1, 0x5410);
+                    __half2 hv = __hsub2(*reinterpret_cast<__half2*>(&w), h1024);
+                    pk[i] = *reinterpret_cast<uint32_t*>(&hv);
+                }
+                if (bits != 0) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int j = jc * 8 + 2 * i;
+                        __half2 raw = __floats2half2_rn(s[j] * k255, s[j + 1] * k255);
+                        const uint32_t sel = (((bits >> (2 * i)) & 1u) ? 0x0054u : 0x0010u) | (((bits >> (2 * i + 1)) & 1u) ? 0x7600u : 0x3200u);
+                        pk[i] = __byte_perm(pk[i], *reinterpret_cast<uint32_t*>(&raw), sel);
+                    }
+                }
+                *reinterpret_cast<uint4*>(smem + C::OFF_P + (jc / 8) * C::A_BLOCK + ptx::sw128_offset(tid, jc % 8)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+            }
+            ptx::fence_proxy_async_smem();
+            ptx::tc_fence_before_sync();
+            ptx::mbar_arrive(&misc->p_full);
+
+            if (hi > 0 && C::OBUF == 2) store_o(hi - 1);    // under this head's PV
+            sq = sq_next;
         }
+        if (alive) {
+            alive = __all_sync(0xffffffffu, ptx::mbar_wait(&misc->o_full[(HG - 1) % C::OBUF], ((HG - 1) / C::OBUF) & 1) && !misc->abort_flag);
+            if (alive) {
+                ptx::tc_fence_after_sync();
+                store_o(HG - 1);
+            }
+        }
+        if (!alive) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; }
     }
 
     ptx::tc_fence_before_sync();
     __syncthreads();
-    if (warp == 4) {
+    if (warp == MMA_WARP) {
         ptx::tc_fence_after_sync();
         ptx::tmem_dealloc(tmem_base, C::TMEM_COLS);
     }
 }
 
+template <int D>
 int pick_heads_per_cta(const AttnArgs& a, int n_z) {
+    // The largest head group that still fills the GPU's CTA slots to about three quarters.
     const long long tiles = (long long)((a.n_query + ROWS - 1) / ROWS) * n_z;
-    int best = 1;
-    for (int hg = a.heads; hg >= 1; --hg) {
+    const long long want = (long long)148 * Cfg<D>::CTAS_PER_SM * 3 / 4;
+    for (int hg = a.heads; hg > 1; --hg) {
         if (a.heads % hg) continue;
-        if (tiles * (a.heads / hg) >= 2 * 148 || hg == 1) { best = hg; break; }
+        if (tiles * (a.heads / hg) >= want) return hg;
     }
-    return best;
+    return 1;
+}
+
+template <int D, bool Q8, bool TAIL_ONLY>
+cudaError_t launch_k(const AttnArgs& a, int n_z, cudaStream_t stream) {
+    using C = Cfg<D>;
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(attention_sm100_kernel<D, Q8, TAIL_ONLY>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::TOTAL);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    const int hg = pick_heads_per_cta<D>(a, n_z);
+    dim3 grid((a.n_query + ROWS - 1) / ROWS, a.heads / hg, n_z);
+    attention_sm100_kernel<D, Q8, TAIL_ONLY><<<grid, ATT_THREADS, C::TOTAL, stream>>>(a, hg);
+    return cudaGetLastError();
 }
 
 template <int D>
 cudaError_t launch_d(const AttnArgs& a, int n_z, cudaStream_t stream) {
-    using C = Cfg<D>;
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(attention_sm100_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::TOTAL);
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
-    const int hg = pick_heads_per_cta(a, n_z);
-    dim3 grid((a.n_query + ROWS - 1) / ROWS, a.heads / hg, n_z);
-    attention_sm100_kernel<D><<<grid, ATT_THREADS, C::TOTAL, stream>>>(a, hg);
-    return cudaGetLastError();
+    const bool q8 = a.q_bits == 8, tail = a.n_ctx > 64;
+    if (q8) return tail ? launch_k<D, true, true>(a, n_z, stream) : launch_k<D, true, false>(a, n_z, stream);
+    return tail ? launch_k<D, false, true>(a, n_z, stream) : launch_k<D, false, false>(a, n_z, stream);
 }
 
 }  // namespace
 
 bool sm100_attention_supported(const AttnArgs& a) {
-    const int d = a.channels / a.heads;
-    if (d != 40 && d != 64 && d != 80 && d != 160) return false;
-    if (a.n_ctx > TP) return false;
+    OperandGeom g;
+    if (!operand_geom(a.channels / a.heads, a.n_ctx, &g)) return false;
     if (a.p_bits != 8) return false;
     if (a.heads > 65535) return false;
     return true;

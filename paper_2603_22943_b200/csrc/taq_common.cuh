@@ -40,6 +40,33 @@ __host__ __device__ inline WeightLayout weight_layout(int n_out, int k_in, int b
     return L;
 }
 
+// MMA-ready image of one head's K~ and V~ (layout documented in taq.h): present when the tensor-core attention
+// kernel covers the shape (head width 40/64/80/160, at most kOperandKeys text tokens).
+constexpr int kOperandKeys = 80;                // keys padded to a multiple of the MMA K step
+constexpr int kOperandConstBytes = 1024;
+struct OperandGeom {
+    int dp;                 // head width padded to a multiple of 16
+    int kbq;                // 64-wide blocks along the head width
+    size_t k_bytes;         // K~ tile: kbq blocks of [kOperandKeys rows][128 bytes]
+    size_t vt_bytes;        // V~^T tile: 2 blocks of [dp rows][128 bytes]
+    size_t head_bytes;      // k_bytes + vt_bytes + kOperandConstBytes
+};
+__host__ __device__ inline bool operand_geom(int d, int n_ctx, OperandGeom* g) {
+    if ((d != 40 && d != 64 && d != 80 && d != 160) || n_ctx > kOperandKeys) return false;
+    g->dp = (d + 15) / 16 * 16;
+    g->kbq = (g->dp + 63) / 64;
+    g->k_bytes = (size_t)g->kbq * kOperandKeys * 128;
+    g->vt_bytes = (size_t)2 * g->dp * 128;
+    g->head_bytes = g->k_bytes + g->vt_bytes + kOperandConstBytes;
+    return true;
+}
+// Constants block at the end of a head's image.
+struct OperandConsts {
+    float logit_factor[kOperandKeys];   // K scale of key j (1 for a trigger row) * log2(e) / sqrt(d); 0 for padding
+    uint32_t trig_bits[4];              // bit j set: key j is a trigger token (fp16 probability column, Eq. 3)
+};
+static_assert(sizeof(OperandConsts) <= kOperandConstBytes, "constants block");
+
 // K~/V~ block of one sequence (layout documented in taq.h).
 __host__ __device__ inline taq_kv_layout kv_layout(int heads, int n_ctx, int d, int max_trigger) {
     taq_kv_layout L;
@@ -53,7 +80,10 @@ __host__ __device__ inline taq_kv_layout kv_layout(int heads, int n_ctx, int d, 
     L.off_k_trigger = 2 * codes + 2 * scales;
     L.off_v_trigger = L.off_k_trigger + trig;
     L.off_trig_slot = L.off_v_trigger + trig;
-    L.block_bytes = L.off_trig_slot + sizeof(int32_t) * kMaxCtx;
+    L.off_operands = L.off_trig_slot + sizeof(int32_t) * kMaxCtx;
+    OperandGeom g;
+    L.operand_head_bytes = operand_geom(d, n_ctx, &g) ? g.head_bytes : 0;
+    L.block_bytes = L.off_operands + L.operand_head_bytes * heads;
     return L;
 }
 
@@ -126,6 +156,7 @@ cudaError_t launch_quantize_rows(const float* x, long long rows, int cols, int q
                                  cudaStream_t stream);
 cudaError_t launch_pack_weights(const taq_weight_desc& d, const float* W, const float* bias, void* packed,
                                 cudaStream_t stream);
+cudaError_t launch_kv_operands(const taq_layer_desc& d, void* kv, const taq_request* reqs, int n_z, cudaStream_t stream);
 cudaError_t launch_unpack_weights(const taq_weight_desc& d, const void* packed, int8_t* codes, float* scales,
                                   cudaStream_t stream);
 

@@ -63,7 +63,8 @@ def test_kv_layout(L):
     assert lay.off_k_codes == 0 and lay.off_v_codes == codes
     assert lay.off_k_scales == 2 * codes and lay.off_v_scales == 2 * codes + scales
     assert lay.off_k_trigger == 2 * codes + 2 * scales and lay.off_v_trigger == lay.off_k_trigger + trig
-    assert lay.off_trig_slot == lay.off_v_trigger + trig and lay.block_bytes == lay.off_trig_slot + 512
+    assert lay.off_trig_slot == lay.off_v_trigger + trig and lay.off_operands == lay.off_trig_slot + 512 and lay.block_bytes == lay.off_operands + 8 * lay.operand_head_bytes
+    assert lay.operand_head_bytes == 80 * 128 + 2 * 48 * 128 + 1024          # K~ tile, V~^T tile, constants (d = 40)
     assert tb.taq_kv_bytes(d) == 2 * lay.block_bytes
     assert tb.taq_workspace_bytes(d, 1) == 8192 * 320 + 8192 * 8 * 4 + 8192 * 320 * 2
     d0 = tb.layer_desc(2, 4096, 320, 8, 77, 768, 4, 128, q_bits=0)

@@ -132,10 +132,10 @@ def test_cross_attention_isolated(shape, n, q_bits):
     if q_bits == 8:
         qc = orc.merge_heads(q["Q_codes"]).astype(np.int8)
         qs = np.ascontiguousarray(q["Q_scales"].transpose(0, 2, 1)).astype(np.float32)        # [B,N,H]
-        o = tb.taq_cross_attention(desc, dev(qc), dev(qs), dev(blk), dev(data["mask"]))
+        o = tb.taq_cross_attention(desc, dev(qc), dev(qs), tb.taq_kv_finalize(desc, dev(blk)), dev(data["mask"]))
     else:
         q16 = orc.merge_heads(q["Q_tilde"]).astype(np.float16)
-        o = tb.taq_cross_attention(desc, dev(q16), None, dev(blk), dev(data["mask"]))
+        o = tb.taq_cross_attention(desc, dev(q16), None, tb.taq_kv_finalize(desc, dev(blk)), dev(data["mask"]))
     tb.taq_poll_device_status()
     max_abs, rel = tl.assert_layer_close(o.cpu().numpy(), want, "O")
     assert rel < 5e-4                                         # fp16 output rounding is the only modelled difference
