@@ -110,6 +110,10 @@ __device__ __forceinline__ void reg_fence(uint32_t (&r)[16]) {
                  :: "memory");
 }
 
+__device__ __forceinline__ void reg_fence8(uint32_t (&r)[8]) {
+    asm volatile("" : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]) :: "memory");
+}
+
 // ---- tcgen05.mma ------------------------------------------------------------------------------------
 // Shared-memory matrix descriptor of a K-major operand tile stored with the 128-byte swizzle: rows of 128 bytes
 // (64 fp16), groups of 8 rows 1024 bytes apart, 16-byte chunks XOR-ed with the row index inside the group.  The
