@@ -59,8 +59,10 @@ int taq_version(void);
  * Packed blob (relocatable, offsets from its start; every section 128-byte aligned):
  *   [0,64)  header: u32 magic 'TAQW', version, n_out, k_in, bits, group, n_groups, has_bias; u64 off_codes,
  *           off_scales, off_bias, total_bytes
- *   codes   bits=8: int8 [n_out][k_in];  bits=4: u8 [n_out][k_in/2], fan-in element 2i in the low nibble and
- *           2i+1 in the high nibble, each nibble = code + 8
+ *   codes   bits=8: int8 [n_out][k_in];  bits=4: u32 [n_out][k_in/8], eight consecutive fan-in elements per
+ *           little-endian word, each nibble = code + 8: even elements 0,2,4,6 in nibbles 0..3 (bits 0..15), odd
+ *           elements 1,3,5,7 in nibbles 4..7 (bits 16..31), so that (word >> 4i) & 0x000F000F yields elements
+ *           2i and 2i+1 in the two halves of a register
  *   scales  fp32 [n_out][n_groups]
  *   bias    fp32 [n_out] (zeros when no bias was given)
  * Restrictions: n_out >= 1, k_in a multiple of 8.
@@ -151,8 +153,9 @@ taq_status taq_kv_project(const taq_layer_desc* desc, const void* ctx_f16_dev, c
 taq_status taq_kv_finalize(const taq_layer_desc* desc, void* kv_packed_dev, size_t kv_bytes, void* stream);
 
 /* Dequant-GEMM on packed weights (the to_q / to_out projections; "quantizing all remaining ... pathways",
- * Sec. III-B last paragraph): y = x W^T (+ bias), W^ = fp16(code * scale) as the matrix operand, fp32
- * accumulation.
+ * Sec. III-B last paragraph): y = x W^T (+ bias) with W^ = code * scale.  The tensor cores multiply x by the
+ * integer codes (exact in fp16) with fp32 accumulation; each scale group's partial sum is multiplied by the
+ * group's scale in fp32.
  *   x_f16_dev fp16 [rows][k_in]
  *   out_kind TAQ_OUT_F16: y fp16 [rows][n_out], bias added.  TAQ_OUT_F32: y fp32, bias added.
  *   TAQ_OUT_INT8_HEAD_ROWS: the Q~ = Q_a(Q) epilogue - y int8 [rows][n_out], scales_dev fp32 [rows][heads],

@@ -25,8 +25,8 @@ integer codes are compared bit for bit; everything else is float64.
 
 Two modes.  ``ideal``: the equations in real (float64) arithmetic, quantizers as above, no other
 rounding.  ``contract``: the same, plus a round-to-nearest-even to fp16 wherever the layer stores an
-fp16 value ("full precision" of the trigger pathway is fp16 storage; dequantized weights and
-dequantized V rows are fp16 matrix operands; O and Y are fp16 tensors).  The CUDA path is graded
+fp16 value ("full precision" of the trigger pathway is fp16 storage; dequantized V rows are fp16
+matrix operands; O and Y are fp16 tensors).  Dequantized weights are exact in both modes (w^ = q * s).  The CUDA path is graded
 against ``contract``.
 
 Pins (tests/test_oracle_*.py, no GPU): empty mask == separately written uniform quantized
@@ -101,13 +101,12 @@ def quantize_weights(W: np.ndarray, bits: int, group: int) -> Tuple[np.ndarray, 
 
 
 def dequantize_weights(codes: np.ndarray, scales: np.ndarray, group: int, contract: bool) -> np.ndarray:
-    """w^ = q * s per group.  ideal: the exact product in float64.  contract: the matrix operand is
-    fp16, w16 = fp16(float32(q) * s)."""
+    """w^ = q * s per group: the exact product, in both modes.  The layer multiplies by the integer codes
+    and applies the scale of each group to that group's partial sum, so no rounding sits between the
+    code and the product (``contract`` is kept in the signature for symmetry with the other steps)."""
     n_out, k_in = codes.shape
     g = k_in if group == 0 else group
     s_full = np.repeat(scales, g, axis=1)[:, :k_in]
-    if contract:
-        return (codes.astype(F32) * s_full.astype(F32)).astype(F32).astype(np.float16).astype(F64)
     return codes.astype(F64) * s_full.astype(F64)
 
 

@@ -113,7 +113,7 @@ __global__ void __launch_bounds__(ATT_THREADS, Cfg<D>::CTAS_PER_SM) attention_sm
     using C = Cfg<D>;
     constexpr int DP = C::DP;
     extern __shared__ unsigned char smem_dyn[];
-    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
+    unsigned char* smem = smem_dyn + ((1024u - (ptx::smem_u32(smem_dyn) & 1023u)) & 1023u);   // 1024-byte aligned, still provably shared
     Misc* misc = reinterpret_cast<Misc*>(smem + C::OFF_MISC);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -131,8 +131,8 @@ __global__ void __launch_bounds__(ATT_THREADS, Cfg<D>::CTAS_PER_SM) attention_sm
             ptx::mbar_init(&misc->s_full[i], 1);
             ptx::mbar_init(&misc->o_full[i], 1);
         }
-        ptx::mbar_init(&misc->q_full, ROWS);
-        ptx::mbar_init(&misc->p_full, ROWS);
+        ptx::mbar_init(&misc->q_full, ROWS / 32);      // one arrival per row warp
+        ptx::mbar_init(&misc->p_full, ROWS / 32);
         ptx::mbar_init(&misc->drain, 1);
         misc->abort_flag = 0;
         ptx::mbar_fence_init();
@@ -245,7 +245,8 @@ __global__ void __launch_bounds__(ATT_THREADS, Cfg<D>::CTAS_PER_SM) attention_sm
             for (int cc = 0; cc < DP / 8; ++cc)
                 *reinterpret_cast<uint4*>(smem + C::OFF_Q + (cc / 8) * C::A_BLOCK + ptx::sw128_offset(tid, cc % 8)) = qr.chunk(cc);
             ptx::fence_proxy_async_smem();
-            ptx::mbar_arrive(&misc->q_full);
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&misc->q_full);
         };
 
         QRegs<D, Q8> qr;
@@ -342,7 +343,8 @@ __global__ void __launch_bounds__(ATT_THREADS, Cfg<D>::CTAS_PER_SM) attention_sm
             }
             ptx::fence_proxy_async_smem();
             ptx::tc_fence_before_sync();
-            ptx::mbar_arrive(&misc->p_full);
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&misc->p_full);
 
             if (hi > 0 && C::OBUF == 2) store_o(hi - 1);    // under this head's PV
             sq = sq_next;

@@ -103,15 +103,15 @@ __device__ inline int quant_code(float x, float scale, int qmax) {
     return (int)r;
 }
 
-// Matrix operand of a packed weight: fp16(float(code) * scale), returned as float.
-__device__ inline float dequant_w16(int code, float scale) {
-    return __half2float(__float2half_rn(__fmul_rn((float)code, scale)));
-}
+// Position of fan-in element e (0..7) of an aligned group of eight 4-bit codes inside their 32-bit word: even
+// elements fill nibbles 0..3, odd elements nibbles 4..7, so that (word >> 4i) & 0x000F000F holds elements 2i and
+// 2i+1 in the two halves of a register.
+__host__ __device__ inline int w4_nibble_pos(int e) { return (e >> 1) + ((e & 1) << 2); }
 
 __device__ inline int load_code(const uint8_t* codes, size_t row_bytes, int bits, int n, int k) {
     if (bits == 8) return (int)((const int8_t*)codes)[(size_t)n * row_bytes + k];
-    uint8_t byte = codes[(size_t)n * row_bytes + (k >> 1)];
-    return (int)((k & 1) ? (byte >> 4) : (byte & 0xF)) - 8;
+    const uint32_t word = *reinterpret_cast<const uint32_t*>(codes + (size_t)n * row_bytes + ((k >> 3) << 2));
+    return (int)((word >> (4 * w4_nibble_pos(k & 7))) & 0xFu) - 8;
 }
 
 // ------------------------------------------------------------------------------------------------------

@@ -1,4 +1,4 @@
-// Generic dequant-GEMM on CUDA cores: y = x W^T with W^ = fp16(code * scale), fp32 accumulation.
+// Generic dequant-GEMM on CUDA cores: y = x W^T with W^ = code * scale, fp32 accumulation.
 // This is the shape-agnostic path (any k_in multiple of 8, any head width up to 256); it also carries the
 // epilogues that quantize the result per (row, head): Q~ = Q_a(Q) and the mixed int8 / fp16 K~, V~ of Eq. 2.
 // A CTA computes 64 rows x TN*16 columns; for the per-head epilogues a CTA's columns are exactly one head, so
@@ -56,7 +56,7 @@ __global__ void __launch_bounds__(256) linear_simt_kernel(const LinearArgs a) {
             if (c < ncols && k0 + k < a.k_in) {
                 const int n = col0 + c;
                 const int q = load_code(codes, L.row_bytes, a.bits, n, k0 + k);
-                w = dequant_w16(q, wscales[(size_t)n * L.n_groups + (k0 + k) / L.group_len]);
+                w = __fmul_rn((float)q, wscales[(size_t)n * L.n_groups + (k0 + k) / L.group_len]);
             }
             Ws[k][c] = w;
         }

@@ -1,15 +1,20 @@
-// Dequant-GEMM on the Blackwell tensor cores: y = x W^T with W^ = fp16(code * scale), fp32 accumulation in TMEM.
+// Dequant-GEMM on the Blackwell tensor cores: y = x W^T with W^ = code * scale.
+//
+// The tensor cores never see a scale: the B operand holds the integer codes as fp16 (exact), every scale group
+// (128 fan-in elements for W4, the whole row for W8) is accumulated in its own pass into one of two TMEM
+// accumulators, and the worker threads fold each finished group into fp32 registers, y += scale[n][g] * acc_g,
+// while the tensor core is already on the next group.
 //
 // One CTA computes a 128-row x BN-column tile.  The packed codes of its BN output channels (a contiguous slice of
-// the blob), their scales and biases are fetched once with three bulk copies; K is then walked in blocks of 64
-// through a ring of shared-memory stages.  Roles:
+// the blob), their scales and biases are fetched once with three bulk copies; K is walked in blocks of 64 through
+// a ring of shared-memory stages.  Roles:
 //   warp 0       one thread issues the bulk copies and the TMA loads of the fp16 activation tile (128 x 64,
 //                128-byte swizzle);
 //   warp 1       owns the TMEM allocation; one thread issues tcgen05.mma (M=128, N=BN, K=16) and commits;
-//   warps 2..5   expand the 4/8-bit codes from shared memory into the fp16 weight tile (BN x 64, same swizzled
-//                K-major layout); afterwards they are the epilogue: each thread owns one accumulator row (TMEM
-//                lane) and applies bias / fp16 conversion, or the per-(row, head) int8 quantization Q_a of Eq. 2,
-//                or the mixed int8 / fp16 K~,V~ store of Eq. 2.
+//   warps 2..9   workers, two threads per accumulator row (TMEM lane), each owning half of the tile's columns:
+//                they expand the 4/8-bit codes from shared memory into the fp16 weight tile (BN x 64, swizzled
+//                K-major), fold finished groups into registers, and run the epilogue: bias / fp16 conversion, or
+//                the per-(row, head) int8 quantization Q_a of Eq. 2, or the mixed int8 / fp16 K~,V~ of Eq. 2.
 // The packed weights stay packed in HBM and are read once per CTA.
 #include "taq_ptx.cuh"
 #include "taq_sm100.cuh"
@@ -21,15 +26,19 @@ namespace {
 constexpr int BM = 128;
 constexpr int BK = 64;
 constexpr int MAX_STAGE = 6;
-constexpr int NTHREADS = 192;
+constexpr int NWORK = 256;                  // worker threads: two per accumulator row
+constexpr int NTHREADS = 64 + NWORK;
 constexpr int A_TILE_BYTES = BM * BK * 2;   // 16 KB
 constexpr int SMEM_LIMIT = 227 * 1024;
 
 template <int BN>
 struct Tile {
+    static constexpr int HC = BN / 2;                                         // columns per worker thread
     static constexpr int B_TILE_BYTES = ((BN * BK * 2 + 1023) / 1024) * 1024;
     static constexpr int STAGE_BYTES = A_TILE_BYTES + B_TILE_BYTES;
-    static constexpr uint32_t TMEM_COLS = BN <= 32 ? 32 : BN <= 64 ? 64 : BN <= 128 ? 128 : 256;
+    static constexpr uint32_t TMEM_COLS = 2 * BN <= 128 ? 128 : 2 * BN <= 256 ? 256 : 512;
+    static constexpr int CTAS_PER_SM = TMEM_COLS <= 256 ? 2 : 1;
+    static_assert(HC % 8 == 0, "a worker's columns come in groups of 8");
 };
 
 struct Bars {
@@ -37,36 +46,64 @@ struct Bars {
     uint64_t full_b[MAX_STAGE];
     uint64_t empty[MAX_STAGE];
     uint64_t w_full;
-    uint64_t acc_full;
+    uint64_t acc_full[2];
+    uint64_t acc_free[2];
     uint32_t tmem_base;
     volatile int abort_flag;
 };
 
 // Shared-memory plan of one launch (host and device agree through these numbers).
 struct Plan {
-    int nstage;
     int raw_bytes, scale_bytes, bias_bytes;   // BN rows of codes / scales / bias
-    int off_raw, off_scales, off_bias, off_bars, total;
+    int off_raw, off_scales, off_scales_t, off_bias, off_xchg, off_bars, total;
 };
 
 template <int BN>
 __host__ __device__ inline Plan make_plan(int k_in, int bits, int group, int nstage) {
     const WeightLayout L = weight_layout(BN, k_in, bits, group);
     Plan p;
-    p.nstage = nstage;
     p.raw_bytes = (int)(L.row_bytes * BN);
     p.scale_bytes = BN * L.n_groups * 4;
     p.bias_bytes = BN * 4;
     p.off_raw = nstage * Tile<BN>::STAGE_BYTES;
     p.off_scales = p.off_raw + (p.raw_bytes + 127) / 128 * 128;
-    p.off_bias = p.off_scales + (p.scale_bytes + 127) / 128 * 128;
-    p.off_bars = p.off_bias + (p.bias_bytes + 127) / 128 * 128;
+    p.off_scales_t = p.off_scales + (p.scale_bytes + 127) / 128 * 128;        // [n_groups][BN]
+    p.off_bias = p.off_scales_t + (p.scale_bytes + 127) / 128 * 128;
+    p.off_xchg = p.off_bias + (p.bias_bytes + 127) / 128 * 128;              // float [2][128]
+    p.off_bars = p.off_xchg + 1024;
     p.total = p.off_bars + 256 + 1024;        // barriers + slack to align the base to 1024
     return p;
 }
 
-// Eight consecutive weights of one output channel -> eight fp16 operands fp16(float(code) * s).
-// 0x4B000000 | n read as a float is 2^23 + n, so the integer-to-float conversion is a subtraction.
+// Eight 4-bit codes of one word -> eight fp16 integers in fan-in order.  0x6400 | n read as fp16 is 1024 + n.
+__device__ __forceinline__ uint4 codes_w4_to_half(uint32_t p) {
+    const __half2 off = __floats2half2_rn(1032.f, 1032.f);                     // 1024 + the nibble bias of 8
+    uint32_t o[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        uint32_t w = ((p >> (4 * i)) & 0x000F000Fu) | 0x64006400u;
+        __half2 h = __hsub2(*reinterpret_cast<__half2*>(&w), off);
+        o[i] = *reinterpret_cast<uint32_t*>(&h);
+    }
+    return make_uint4(o[0], o[1], o[2], o[3]);
+}
+// Eight int8 codes -> eight fp16 integers: (code + 128) rides in the mantissa of 0x64xx.
+__device__ __forceinline__ uint4 codes_w8_to_half(uint2 raw) {
+    const __half2 off = __floats2half2_rn(1152.f, 1152.f);
+    const uint32_t w[2] = {raw.x ^ 0x80808080u, raw.y ^ 0x80808080u};
+    uint32_t o[4];
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        uint32_t lo = __byte_perm(w[i], 0x64646464u, 0x5140);
+        uint32_t hi = __byte_perm(w[i], 0x64646464u, 0x5342);
+        __half2 a = __hsub2(*reinterpret_cast<__half2*>(&lo), off);
+        __half2 b = __hsub2(*reinterpret_cast<__half2*>(&hi), off);
+        o[2 * i] = *reinterpret_cast<uint32_t*>(&a);
+        o[2 * i + 1] = *reinterpret_cast<uint32_t*>(&b);
+    }
+    return make_uint4(o[0], o[1], o[2], o[3]);
+}
+
 __device__ __forceinline__ uint4 pack8(const float (&w)[8]) {
     uint4 out;
     __half2 h;
@@ -76,47 +113,23 @@ __device__ __forceinline__ uint4 pack8(const float (&w)[8]) {
     h = __floats2half2_rn(w[6], w[7]); out.w = *reinterpret_cast<uint32_t*>(&h);
     return out;
 }
-__device__ __forceinline__ uint4 dequant8_w4(uint32_t p, float s) {
-    const uint32_t lo = p & 0x0F0F0F0Fu, hi = (p >> 4) & 0x0F0F0F0Fu;    // nibbles 0,2,4,6 and 1,3,5,7
-    float w[8];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const uint32_t a = __byte_perm(lo, 0x4B000000u, 0x7440 + i);     // bytes {lo.b_i, 0, 0, 0x4B}
-        const uint32_t b = __byte_perm(hi, 0x4B000000u, 0x7440 + i);
-        w[2 * i] = __fmul_rn(__uint_as_float(a) - 8388616.0f, s);        // (2^23 + n) - (2^23 + 8) = code
-        w[2 * i + 1] = __fmul_rn(__uint_as_float(b) - 8388616.0f, s);
-    }
-    return pack8(w);
-}
-__device__ __forceinline__ uint4 dequant8_w8(uint2 p, float s) {
-    const uint32_t x0 = p.x ^ 0x80808080u, x1 = p.y ^ 0x80808080u;       // code + 128 in every byte
-    float w[8];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const uint32_t a = __byte_perm(x0, 0x4B000000u, 0x7440 + i);
-        const uint32_t b = __byte_perm(x1, 0x4B000000u, 0x7440 + i);
-        w[i] = __fmul_rn(__uint_as_float(a) - 8388736.0f, s);            // (2^23 + code + 128) - (2^23 + 128)
-        w[4 + i] = __fmul_rn(__uint_as_float(b) - 8388736.0f, s);
-    }
-    return pack8(w);
-}
 
-// Loads `n8` groups of 8 accumulator columns of this thread's row (all loads issued before the one wait).
-template <int N8>
-__device__ __forceinline__ void tmem_row_load(uint32_t taddr, uint32_t (&v)[N8][8], int n8) {
+// Eight values -> eight int8 codes rint(x * rs): fma(x, rs, 1.5 * 2^23) leaves the two's-complement code in the low byte.
+__device__ __forceinline__ uint2 quant8(const float* x, float rs) {
+    uint32_t b[8];
 #pragma unroll
-    for (int i = 0; i < N8; ++i)
-        if (i < n8) ptx::tmem_ld8(taddr + i * 8, v[i]);
-    ptx::tmem_ld_wait(v[0]);
-#pragma unroll
-    for (int i = 1; i < N8; ++i) ptx::reg_fence8(v[i]);
+    for (int e = 0; e < 8; ++e) b[e] = __float_as_uint(fmaf(x[e], rs, 12582912.0f));
+    const uint32_t lo = __byte_perm(__byte_perm(b[0], b[1], 0x0040), __byte_perm(b[2], b[3], 0x0040), 0x5410);
+    const uint32_t hi = __byte_perm(__byte_perm(b[4], b[5], 0x0040), __byte_perm(b[6], b[7], 0x0040), 0x5410);
+    return make_uint2(lo, hi);
 }
 
 template <int BN>
-__global__ void __launch_bounds__(NTHREADS) linear_sm100_kernel(const __grid_constant__ CUtensorMap tmap_x, const LinearArgs a, const int nstage) {
+__global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_kernel(const __grid_constant__ CUtensorMap tmap_x, const LinearArgs a, const int nstage) {
     using TL = Tile<BN>;
+    constexpr int HC = TL::HC;
     extern __shared__ unsigned char smem_dyn[];
-    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
+    unsigned char* smem = smem_dyn + ((1024u - (ptx::smem_u32(smem_dyn) & 1023u)) & 1023u);   // 1024-byte aligned, still provably shared
     const Plan P = make_plan<BN>(a.k_in, a.bits, a.group, nstage);
     Bars* bars = reinterpret_cast<Bars*>(smem + P.off_bars);
     constexpr uint32_t TMEM_COLS = TL::TMEM_COLS;
@@ -128,15 +141,20 @@ __global__ void __launch_bounds__(NTHREADS) linear_sm100_kernel(const __grid_con
     const int n_kb = a.k_in / BK;
     const uint8_t* blob = (const uint8_t*)(a.reqs ? (a.which == 0 ? a.reqs[z].Wq : a.reqs[z].Wout) : a.w);
     const WeightLayout L = weight_layout(a.n_out, a.k_in, a.bits, a.group);
+    const int n_groups = L.n_groups;
+    const int kb_per_group = L.group_len / BK;             // k-blocks in a full group (the last group may be shorter)
 
     if (tid == 0) {
         for (int s = 0; s < MAX_STAGE; ++s) {
             ptx::mbar_init(&bars->full_a[s], 1);
-            ptx::mbar_init(&bars->full_b[s], 128);
+            ptx::mbar_init(&bars->full_b[s], NWORK / 32);    // one arrival per worker warp
             ptx::mbar_init(&bars->empty[s], 1);
         }
         ptx::mbar_init(&bars->w_full, 1);
-        ptx::mbar_init(&bars->acc_full, 1);
+        for (int i = 0; i < 2; ++i) {
+            ptx::mbar_init(&bars->acc_full[i], 1);
+            ptx::mbar_init(&bars->acc_free[i], NWORK / 32);
+        }
         bars->abort_flag = 0;
         ptx::mbar_fence_init();
         ptx::tma_prefetch_desc(&tmap_x);
@@ -152,16 +170,17 @@ __global__ void __launch_bounds__(NTHREADS) linear_sm100_kernel(const __grid_con
         if (lane == 0) {
             ptx::mbar_arrive_expect_tx(&bars->w_full, (uint32_t)(P.raw_bytes + P.scale_bytes + P.bias_bytes));
             ptx::bulk_load(smem + P.off_raw, blob + L.off_codes + (size_t)col0 * L.row_bytes, (uint32_t)P.raw_bytes, &bars->w_full);
-            ptx::bulk_load(smem + P.off_scales, blob + L.off_scales + (size_t)col0 * L.n_groups * 4, (uint32_t)P.scale_bytes, &bars->w_full);
+            ptx::bulk_load(smem + P.off_scales, blob + L.off_scales + (size_t)col0 * n_groups * 4, (uint32_t)P.scale_bytes, &bars->w_full);
             ptx::bulk_load(smem + P.off_bias, blob + L.off_bias + (size_t)col0 * 4, (uint32_t)P.bias_bytes, &bars->w_full);
-            int issued = 0;
+            int issued = 0, s = 0;
+            uint32_t ph = 0;                               // parity of the ring pass
             for (int kb = 0; kb < n_kb; ++kb) {
-                const int s = kb % nstage;
-                if (kb >= nstage && !ptx::mbar_wait(&bars->empty[s], ((kb / nstage) & 1) ^ 1)) { raise_status(a.status, TAQ_ERR_TIMEOUT); bars->abort_flag = 1; }
+                if (kb >= nstage && !ptx::mbar_wait(&bars->empty[s], ph ^ 1)) { raise_status(a.status, TAQ_ERR_TIMEOUT); bars->abort_flag = 1; }
                 if (bars->abort_flag) break;
                 ptx::mbar_arrive_expect_tx(&bars->full_a[s], A_TILE_BYTES);
                 ptx::tma_load_3d(smem + s * TL::STAGE_BYTES, &tmap_x, &bars->full_a[s], kb * BK, row0, z);
                 issued = kb + 1;
+                if (++s == nstage) { s = 0; ph ^= 1; }
             }
             if (bars->abort_flag) {   // give copies that are still in flight a bounded chance to land before the CTA exits
                 (void)ptx::mbar_wait(&bars->w_full, 0);
@@ -169,202 +188,222 @@ __global__ void __launch_bounds__(NTHREADS) linear_sm100_kernel(const __grid_con
             }
         }
     } else if (warp == 1) {
-        // ---------------- MMA issuer ----------------
+        // ---------------- MMA issuer: one accumulation pass per scale group ----------------
         if (lane == 0) {
             constexpr uint32_t idesc = ptx::idesc_f16_m128(BN);
-            for (int kb = 0; kb < n_kb; ++kb) {
-                const int s = kb % nstage;
-                const uint32_t ph = (kb / nstage) & 1;
-                if (!ptx::mbar_wait(&bars->full_a[s], ph) || !ptx::mbar_wait(&bars->full_b[s], ph)) { raise_status(a.status, TAQ_ERR_TIMEOUT); bars->abort_flag = 1; }
-                if (bars->abort_flag) break;
+            int s = 0, kb = 0;
+            uint32_t ph = 0;
+            bool ok = true;
+            for (int g = 0; g < n_groups && ok; ++g) {
+                const int buf = g & 1;
+                if (g >= 2 && !ptx::mbar_wait(&bars->acc_free[buf], ((g >> 1) - 1) & 1)) ok = false;   // the workers have emptied this accumulator
                 ptx::tc_fence_after_sync();
-                const uint32_t a_addr = ptx::smem_u32(smem + s * TL::STAGE_BYTES);
-                const uint32_t b_addr = a_addr + A_TILE_BYTES;
+                const int kb_end = min(n_kb, kb + kb_per_group);
+                for (bool first = true; kb < kb_end && ok; ++kb) {
+                    if (!ptx::mbar_wait(&bars->full_a[s], ph) || !ptx::mbar_wait(&bars->full_b[s], ph) || bars->abort_flag) { ok = false; break; }
+                    ptx::tc_fence_after_sync();
+                    const uint32_t a_addr = ptx::smem_u32(smem + s * TL::STAGE_BYTES);
+                    const uint32_t b_addr = a_addr + A_TILE_BYTES;
 #pragma unroll
-                for (int k = 0; k < BK / 16; ++k) {
-                    ptx::mma_f16_ss(tmem_base, ptx::desc_k_sw128(a_addr + k * 32), ptx::desc_k_sw128(b_addr + k * 32), idesc, (kb | k) != 0);
+                    for (int k = 0; k < BK / 16; ++k) {
+                        ptx::mma_f16_ss(tmem_base + buf * BN, ptx::desc_k_sw128(a_addr + k * 32), ptx::desc_k_sw128(b_addr + k * 32), idesc, !(first && k == 0));
+                    }
+                    first = false;
+                    ptx::mma_commit(&bars->empty[s]);       // frees the stage once these MMAs have read it
+                    if (++s == nstage) { s = 0; ph ^= 1; }
                 }
-                ptx::mma_commit(&bars->empty[s]);       // frees the stage once these MMAs have read it
+                if (ok) ptx::mma_commit(&bars->acc_full[buf]);
             }
-            ptx::mma_commit(&bars->acc_full);            // accumulator complete (arrives even after an abort)
+            if (!ok) {
+                raise_status(a.status, TAQ_ERR_TIMEOUT);
+                bars->abort_flag = 1;
+                ptx::mma_commit(&bars->acc_full[0]);        // wake the workers; they see the abort flag
+                ptx::mma_commit(&bars->acc_full[1]);
+            }
         }
     } else {
-        // ---------------- weight expansion (warps 2..5) ----------------
-        const int wt = tid - 64;                          // 0..127
+        // ---------------- workers (warps 2..9) ----------------
+        const int wt = tid - 64;                          // 0..255
+        const int q = warp & 3;                           // TMEM lane quarter this warp may read
+        const int half = (warp - 2) >> 2;                 // which half of the tile's columns this thread owns
+        const int r = q * 32 + lane;
+        const long long row = (long long)row0 + r;
+        const int cb = half * HC;                         // first owned column inside the tile
+        const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + cb;
         const unsigned char* raw = smem + P.off_raw;
         const float* wscales = reinterpret_cast<const float*>(smem + P.off_scales);
+        float* scales_t = reinterpret_cast<float*>(smem + P.off_scales_t);
         const float* bias = reinterpret_cast<const float*>(smem + P.off_bias);
-        const int row_bytes = (int)L.row_bytes, n_groups = L.n_groups;
+        float* xchg = reinterpret_cast<float*>(smem + P.off_xchg);
+        const int row_bytes = (int)L.row_bytes;
         bool ok = ptx::mbar_wait(&bars->w_full, 0);
         if (!ok) { raise_status(a.status, TAQ_ERR_TIMEOUT); bars->abort_flag = 1; }
-        for (int kb = 0; kb < n_kb && ok; ++kb) {
-            const int s = kb % nstage;
-            if (kb >= nstage && !ptx::mbar_wait(&bars->empty[s], ((kb / nstage) & 1) ^ 1)) { raise_status(a.status, TAQ_ERR_TIMEOUT); bars->abort_flag = 1; }
-            if (bars->abort_flag) { ok = false; break; }
-            unsigned char* b_tile = smem + s * TL::STAGE_BYTES + A_TILE_BYTES;
-            const int g = (kb * BK) / L.group_len;
-#pragma unroll
-            for (int i = 0; i < (BN * 8 + 127) / 128; ++i) {   // 16-byte chunks: 8 per weight row
-                const int idx = wt + i * 128;
-                if ((BN * 8) % 128 == 0 || idx < BN * 8) {
-                    const int n = idx >> 3, c = idx & 7;
-                    const float sc = wscales[n * n_groups + g];
-                    uint4 v;
-                    if (a.bits == 4) v = dequant8_w4(*reinterpret_cast<const uint32_t*>(raw + n * row_bytes + ((kb * BK + c * 8) >> 1)), sc);
-                    else v = dequant8_w8(*reinterpret_cast<const uint2*>(raw + n * row_bytes + kb * BK + c * 8), sc);
-                    *reinterpret_cast<uint4*>(b_tile + ptx::sw128_offset(n, c)) = v;
-                }
-            }
-            ptx::fence_proxy_async_smem();                // make the generic-proxy writes visible to the tensor core
-            ptx::mbar_arrive(&bars->full_b[s]);
-        }
+        // scales [BN][n_groups] -> [n_groups][BN], so that a group's scales of consecutive columns are contiguous
+        for (int i = wt; i < BN * n_groups; i += NWORK) scales_t[(i % n_groups) * BN + i / n_groups] = wscales[i];
+        asm volatile("bar.sync 1, 256;" ::: "memory");
 
-        // ---------------- epilogue: one accumulator row per thread ----------------
-        const bool done = ptx::mbar_wait(&bars->acc_full, 0);
-        if (!done) { raise_status(a.status, TAQ_ERR_TIMEOUT); bars->abort_flag = 1; }
-        ptx::tc_fence_after_sync();
-        if (done && !bars->abort_flag) {
-            const int q = warp & 3;                       // TMEM lane quarter this warp may read
-            const int r = q * 32 + lane;
-            const long long row = (long long)row0 + r;
-            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
-            if (a.epi == EPI_F16 || a.epi == EPI_F32) {
-#pragma unroll 1
-                for (int c0 = 0; c0 < BN; c0 += 32) {
-                    uint32_t v[4][8];
-                    const int n8 = (BN - c0) >= 32 ? 4 : (BN - c0) / 8;
-                    tmem_row_load<4>(taddr + c0, v, n8);
-                    if (row < a.rows) {
-                        const size_t o = ((size_t)z * a.rows + row) * a.n_out + col0 + c0;
+        float y[HC];
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            if (i < n8) {
-                                float f[8];
+        for (int c = 0; c < HC; ++c) y[c] = 0.f;
+
+        // y += scale[g] * accumulator of group g (this thread's HC columns of its row)
+        auto fold_group = [&](int g) -> bool {
+            const int buf = g & 1;
+            if (!ptx::mbar_wait(&bars->acc_full[buf], (g >> 1) & 1) || bars->abort_flag) return false;
+            ptx::tc_fence_after_sync();
+            const float* sg = scales_t + g * BN + cb;
 #pragma unroll
-                                for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[i][e]) + bias[c0 + i * 8 + e];
-                                if (a.epi == EPI_F16) {
-                                    *reinterpret_cast<uint4*>((__half*)a.y + o + i * 8) = pack8(f);
-                                } else {
-                                    float4* dst = reinterpret_cast<float4*>((float*)a.y + o + i * 8);
-                                    dst[0] = make_float4(f[0], f[1], f[2], f[3]);
-                                    dst[1] = make_float4(f[4], f[5], f[6], f[7]);
-                                }
-                            }
-                        }
+            for (int c0 = 0; c0 < HC; c0 += 40) {
+                constexpr int N8MAX = 5;
+                uint32_t v[N8MAX][8];
+#pragma unroll
+                for (int i = 0; i < N8MAX; ++i)
+                    if (c0 + i * 8 < HC) ptx::tmem_ld8(taddr + buf * BN + c0 + i * 8, v[i]);
+                ptx::tmem_ld_wait(v[0]);
+#pragma unroll
+                for (int i = 1; i < N8MAX; ++i) ptx::reg_fence8(v[i]);
+#pragma unroll
+                for (int i = 0; i < N8MAX; ++i)
+                    if (c0 + i * 8 < HC) {
+                        const float4 s0 = *reinterpret_cast<const float4*>(sg + c0 + i * 8), s1 = *reinterpret_cast<const float4*>(sg + c0 + i * 8 + 4);
+                        float* yy = y + c0 + i * 8;
+                        yy[0] = fmaf(__uint_as_float(v[i][0]), s0.x, yy[0]); yy[1] = fmaf(__uint_as_float(v[i][1]), s0.y, yy[1]);
+                        yy[2] = fmaf(__uint_as_float(v[i][2]), s0.z, yy[2]); yy[3] = fmaf(__uint_as_float(v[i][3]), s0.w, yy[3]);
+                        yy[4] = fmaf(__uint_as_float(v[i][4]), s1.x, yy[4]); yy[5] = fmaf(__uint_as_float(v[i][5]), s1.y, yy[5]);
+                        yy[6] = fmaf(__uint_as_float(v[i][6]), s1.z, yy[6]); yy[7] = fmaf(__uint_as_float(v[i][7]), s1.w, yy[7]);
+                    }
+            }
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&bars->acc_free[buf]);
+            return true;
+        };
+
+        // expand the weight tiles of group g's k-blocks
+        int s = 0, kb = 0;
+        uint32_t ph = 0;
+        auto build_group = [&](int g) -> bool {
+            const int kb_end = min(n_kb, kb + kb_per_group);
+            for (; kb < kb_end; ++kb) {
+                if (kb >= nstage && !ptx::mbar_wait(&bars->empty[s], ph ^ 1)) return false;
+                if (bars->abort_flag) return false;
+                unsigned char* b_tile = smem + s * TL::STAGE_BYTES + A_TILE_BYTES;
+                // 16-byte chunks of the fp16 tile: 8 per weight row; this thread owns chunk c of rows n0, n0 + 32, ...
+                constexpr int NCH = (BN * 8 + NWORK - 1) / NWORK;
+                const int n0 = wt >> 3, c = wt & 7;
+                uint2 pw[NCH];
+#pragma unroll
+                for (int i = 0; i < NCH; ++i) {
+                    const int n = n0 + (NWORK / 8) * i;
+                    pw[i] = make_uint2(0, 0);
+                    if ((BN * 8) % NWORK == 0 || n < BN) {
+                        if (a.bits == 4) pw[i].x = *reinterpret_cast<const uint32_t*>(raw + n * row_bytes + kb * (BK / 2) + c * 4);
+                        else pw[i] = *reinterpret_cast<const uint2*>(raw + n * row_bytes + kb * BK + c * 8);
                     }
                 }
-            } else if (a.epi == EPI_Q8_HEAD) {
-                // Q~ = Q_a(Q): per (row, head) absmax, then codes = rint(x * (1/s)) by one fma whose low byte is the
-                // two's-complement code (1.5 * 2^23 + code).  Two passes over TMEM, 40 columns at a time.
-                const int d = a.n_out / a.heads;
-                const int heads_here = BN / d;
-#pragma unroll 1
-                for (int hh = 0; hh < heads_here; ++hh) {
-                    const int h = col0 / d + hh;
-                    float amax = 0.f;
-#pragma unroll 1
-                    for (int c0 = 0; c0 < d; c0 += 40) {
-                        uint32_t v[5][8];
-                        const int n8 = (d - c0) >= 40 ? 5 : (d - c0) / 8;
-                        tmem_row_load<5>(taddr + hh * d + c0, v, n8);
 #pragma unroll
-                        for (int i = 0; i < 5; ++i)
-                            if (i < n8) {
+                for (int i = 0; i < NCH; ++i) {
+                    const int n = n0 + (NWORK / 8) * i;
+                    if ((BN * 8) % NWORK == 0 || n < BN)
+                        *reinterpret_cast<uint4*>(b_tile + ptx::sw128_offset(n, c)) = a.bits == 4 ? codes_w4_to_half(pw[i].x) : codes_w8_to_half(pw[i]);
+                }
+                ptx::fence_proxy_async_smem();            // make the generic-proxy writes visible to the tensor core
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&bars->full_b[s]);
+                if (++s == nstage) { s = 0; ph ^= 1; }
+            }
+            return true;
+        };
+
+        for (int g = 0; g < n_groups && ok; ++g) {
+            ok = build_group(g);
+            if (ok && g >= 1) ok = fold_group(g - 1);
+        }
+        if (ok) ok = fold_group(n_groups - 1);
+        if (!ok) { raise_status(a.status, TAQ_ERR_TIMEOUT); bars->abort_flag = 1; }
+        asm volatile("bar.sync 1, 256;" ::: "memory");       // every worker gets here; the decision below is uniform
+        ok = !bars->abort_flag;
+
+        // ---------------- epilogue on this thread's HC columns ----------------
+        if (ok) {
+            if (a.epi == EPI_F16 || a.epi == EPI_F32) {
+                if (row < a.rows) {
+                    const size_t o = ((size_t)z * a.rows + row) * a.n_out + col0 + cb;
 #pragma unroll
-                                for (int e = 0; e < 8; ++e) amax = fmaxf(amax, fabsf(__uint_as_float(v[i][e])));
-                            }
-                    }
-                    const float s = quant_scale(amax, 127.f);
-                    const float rs = s > 0.f ? __frcp_rn(s) : 0.f;
-#pragma unroll 1
-                    for (int c0 = 0; c0 < d; c0 += 40) {
-                        uint32_t v[5][8];
-                        const int n8 = (d - c0) >= 40 ? 5 : (d - c0) / 8;
-                        tmem_row_load<5>(taddr + hh * d + c0, v, n8);
-                        if (row < a.rows) {
-                            int8_t* dst = (int8_t*)a.y + ((size_t)z * a.rows + row) * a.n_out + h * d + c0;
+                    for (int c = 0; c < HC; c += 8) {
+                        float f[8];
 #pragma unroll
-                            for (int i = 0; i < 5; ++i)
-                                if (i < n8) {
-                                    uint32_t x[8];
-#pragma unroll
-                                    for (int e = 0; e < 8; ++e) x[e] = __float_as_uint(fmaf(__uint_as_float(v[i][e]), rs, 12582912.0f));
-                                    const uint32_t lo = __byte_perm(__byte_perm(x[0], x[1], 0x0040), __byte_perm(x[2], x[3], 0x0040), 0x5410);
-                                    const uint32_t hi = __byte_perm(__byte_perm(x[4], x[5], 0x0040), __byte_perm(x[6], x[7], 0x0040), 0x5410);
-                                    *reinterpret_cast<uint2*>(dst + i * 8) = make_uint2(lo, hi);
-                                }
+                        for (int e = 0; e < 8; ++e) f[e] = y[c + e] + bias[cb + c + e];
+                        if (a.epi == EPI_F16) {
+                            *reinterpret_cast<uint4*>((__half*)a.y + o + c) = pack8(f);
+                        } else {
+                            float4* dst = reinterpret_cast<float4*>((float*)a.y + o + c);
+                            dst[0] = make_float4(f[0], f[1], f[2], f[3]);
+                            dst[1] = make_float4(f[4], f[5], f[6], f[7]);
                         }
                     }
-                    if (row < a.rows) a.scales[((size_t)z * a.rows + row) * a.heads + h] = s;
                 }
             } else {
-                // Eq. 2 for K or V: rows of ordinary tokens -> int8 codes + scale, rows of trigger tokens -> fp16
+                // Per-(row, head) symmetric int8.  A thread's columns are either one whole head (d = HC) or half of the
+                // tile's single head (d = BN); in the second case the row's two threads exchange their absmax.
                 const int d = a.n_out / a.heads;
-                const int heads_here = BN / d;
-                int b = 0, t = 0, slot = -1;
-                bool trig = false;
-                uint8_t* blk = nullptr;
-                taq_kv_layout KL;
-                if (row < a.rows) {
-                    b = a.reqs ? 0 : (int)(row / a.n_ctx);
-                    t = (int)(row % a.n_ctx);
+                const bool whole_head = d == HC;
+                const int h = (col0 + cb) / d;
+                float amax = 0.f;
+#pragma unroll
+                for (int c = 0; c < HC; ++c) amax = fmaxf(amax, fabsf(y[c]));
+                if (!whole_head) {
+                    xchg[half * 128 + r] = amax;
+                    asm volatile("bar.sync 2, 256;" ::: "memory");
+                    amax = fmaxf(amax, xchg[(half ^ 1) * 128 + r]);
+                }
+                const float s = quant_scale(amax, 127.f);
+                const float rs = s > 0.f ? __frcp_rn(s) : 0.f;
+                const int ch = (col0 + cb) - h * d;                   // first owned column inside the head
+                if (a.epi == EPI_Q8_HEAD) {
+                    // Q~ = Q_a(Q), Eq. 2 third line
+                    if (row < a.rows) {
+                        int8_t* dst = (int8_t*)a.y + ((size_t)z * a.rows + row) * a.n_out + col0 + cb;
+#pragma unroll
+                        for (int c = 0; c < HC; c += 8) *reinterpret_cast<uint2*>(dst + c) = quant8(y + c, rs);
+                        if (whole_head || half == 0) a.scales[((size_t)z * a.rows + row) * a.heads + h] = s;
+                    }
+                } else if (row < a.rows) {
+                    // Eq. 2 for K or V: rows of ordinary tokens -> int8 codes + scale, rows of trigger tokens -> fp16
+                    const int b = a.reqs ? 0 : (int)(row / a.n_ctx);
+                    const int t = (int)(row % a.n_ctx);
                     const uint8_t* mask = a.reqs ? a.reqs[z].trig_mask : a.mask + (size_t)b * a.n_ctx;
-                    KL = kv_layout(a.heads, a.n_ctx, d, a.max_trigger);
-                    blk = a.reqs ? (uint8_t*)a.reqs[z].kv : (uint8_t*)a.y + (size_t)b * KL.block_bytes;
-                    trig = mask[t] != 0;
+                    const taq_kv_layout KL = kv_layout(a.heads, a.n_ctx, d, a.max_trigger);
+                    uint8_t* blk = a.reqs ? (uint8_t*)a.reqs[z].kv : (uint8_t*)a.y + (size_t)b * KL.block_bytes;
+                    const bool trig = mask[t] != 0;
+                    int slot = -1;
                     if (trig) {
                         slot = 0;
                         for (int u = 0; u < t; ++u) slot += mask[u] != 0;
                         if (slot >= a.max_trigger) { raise_status(a.status, TAQ_ERR_SHAPE); slot = -2; }
                     }
-                }
-#pragma unroll 1
-                for (int hh = 0; hh < heads_here; ++hh) {
-                    const int h = col0 / d + hh;
-                    float amax = 0.f;
-#pragma unroll 1
-                    for (int c = 0; c < d; c += 8) {
-                        uint32_t v[8];
-                        ptx::tmem_ld8(taddr + hh * d + c, v);
-                        ptx::tmem_ld_wait(v);
+                    int8_t* cq = (int8_t*)(blk + (a.kv_which ? KL.off_v_codes : KL.off_k_codes)) + ((size_t)h * a.n_ctx + t) * d + ch;
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) amax = fmaxf(amax, fabsf(__uint_as_float(v[i])));
-                    }
-                    const float s = quant_scale(amax, 127.f);
-#pragma unroll 1
-                    for (int c = 0; c < d; c += 8) {
-                        uint32_t v[8];
-                        ptx::tmem_ld8(taddr + hh * d + c, v);
-                        ptx::tmem_ld_wait(v);
-                        if (row < a.rows) {
-                            uint32_t lo = 0, hi = 0;
-                            if (!trig) {
+                    for (int c = 0; c < HC; c += 8) *reinterpret_cast<uint2*>(cq + c) = trig ? make_uint2(0, 0) : quant8(y + c, rs);
+                    if (slot >= 0) {
+                        __half* tr = (__half*)(blk + (a.kv_which ? KL.off_v_trigger : KL.off_k_trigger)) + ((size_t)slot * a.heads + h) * d + ch;
 #pragma unroll
-                                for (int i = 0; i < 4; ++i) {
-                                    lo |= (uint32_t)(quant_code(__uint_as_float(v[i]), s, 127) & 0xFF) << (8 * i);
-                                    hi |= (uint32_t)(quant_code(__uint_as_float(v[4 + i]), s, 127) & 0xFF) << (8 * i);
-                                }
-                            }
-                            int8_t* cq = (int8_t*)(blk + (a.kv_which ? KL.off_v_codes : KL.off_k_codes)) + ((size_t)h * a.n_ctx + t) * d + c;
-                            *reinterpret_cast<uint2*>(cq) = make_uint2(lo, hi);
-                            if (slot >= 0) {
-                                __half* tr = (__half*)(blk + (a.kv_which ? KL.off_v_trigger : KL.off_k_trigger)) + ((size_t)slot * a.heads + h) * d + c;
-                                float f[8];
+                        for (int c = 0; c < HC; c += 8) {
+                            float f[8];
 #pragma unroll
-                                for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(v[i]);
-                                *reinterpret_cast<uint4*>(tr) = pack8(f);
-                            }
+                            for (int e = 0; e < 8; ++e) f[e] = y[c + e];
+                            *reinterpret_cast<uint4*>(tr + c) = pack8(f);
                         }
                     }
-                    if (row < a.rows) {
+                    if (whole_head || half == 0) {
                         ((float*)(blk + (a.kv_which ? KL.off_v_scales : KL.off_k_scales)))[(size_t)h * a.n_ctx + t] = trig ? 0.f : s;
                         if (h == 0 && a.kv_which == 0) ((int32_t*)(blk + KL.off_trig_slot))[t] = slot >= 0 ? slot : -1;
                     }
                 }
-                if (a.kv_which == 0 && blockIdx.x == 0 && blockIdx.y == 0) {   // slot table beyond T
+                if (a.epi == EPI_KV && a.kv_which == 0 && blockIdx.x == 0 && blockIdx.y == 0) {   // slot table beyond T
                     const int nb = a.reqs ? 1 : (int)(a.rows / a.n_ctx);
                     const taq_kv_layout K2 = kv_layout(a.heads, a.n_ctx, d, a.max_trigger);
-                    for (int i = wt; i < nb * (kMaxCtx - a.n_ctx); i += 128) {
+                    for (int i = wt; i < nb * (kMaxCtx - a.n_ctx); i += NWORK) {
                         const int bb = i / (kMaxCtx - a.n_ctx), tt = a.n_ctx + i % (kMaxCtx - a.n_ctx);
                         uint8_t* bk = a.reqs ? (uint8_t*)a.reqs[z].kv : (uint8_t*)a.y + (size_t)bb * K2.block_bytes;
                         ((int32_t*)(bk + K2.off_trig_slot))[tt] = -1;
@@ -402,8 +441,8 @@ EncodeTiledFn encode_tiled_fn() {
 int pick_bn(const LinearArgs& a) {
     if (a.epi == EPI_Q8_HEAD || a.epi == EPI_KV) {
         const int d = a.n_out / a.heads;
-        if (d == 40 && a.heads % 2 == 0) return 80;
-        if (d == 64 || d == 80 || d == 160) return d;
+        if (d == 40 && a.heads % 2 == 0) return 80;     // two heads per tile, one per worker thread of a row
+        if (d == 64 || d == 80 || d == 160) return d;   // one head per tile, split between the row's two threads
         return 0;
     }
     if (a.n_out % 160 == 0 && a.rows * (a.n_out / 160) >= 148LL * 128) return 160;
@@ -416,11 +455,12 @@ int pick_bn(const LinearArgs& a) {
 template <int BN>
 int pick_nstage(const LinearArgs& a) {
     const int n_kb = a.k_in / BK;
+    const int half_sm = Tile<BN>::CTAS_PER_SM == 2 ? SMEM_LIMIT / 2 : SMEM_LIMIT;
     int best = 0;
     for (int ns = 1; ns <= MAX_STAGE && ns <= (n_kb < 2 ? 2 : n_kb); ++ns) {
         const int total = make_plan<BN>(a.k_in, a.bits, a.group, ns).total;
         if (total > SMEM_LIMIT) break;
-        if (ns > 3 && total + 1024 > SMEM_LIMIT / 2 && make_plan<BN>(a.k_in, a.bits, a.group, 3).total + 1024 <= SMEM_LIMIT / 2) break;
+        if (ns > 3 && total + 1024 > half_sm && make_plan<BN>(a.k_in, a.bits, a.group, 3).total + 1024 <= half_sm) break;
         best = ns;
     }
     return best;

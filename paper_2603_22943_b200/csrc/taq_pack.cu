@@ -88,10 +88,11 @@ __global__ void __launch_bounds__(256) pack_weights_kernel(const float* __restri
         if (bits == 8) {
             for (int k = lo + lane; k < hi; k += 32) ((int8_t*)codes)[(size_t)n * L.row_bytes + k] = (int8_t)quant_code(wr[k], s, qmax);
         } else {
-            for (int k = lo + 2 * lane; k < hi; k += 64) {   // group bounds are even, so a byte never straddles groups
-                int q0 = quant_code(wr[k], s, qmax) + 8;
-                int q1 = quant_code(wr[k + 1], s, qmax) + 8;
-                codes[(size_t)n * L.row_bytes + (k >> 1)] = (uint8_t)(q0 | (q1 << 4));
+            for (int k = lo + 8 * lane; k < hi; k += 256) {   // group bounds are multiples of 8: a word never straddles groups
+                uint32_t word = 0;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) word |= (uint32_t)(quant_code(wr[k + e], s, qmax) + 8) << (4 * w4_nibble_pos(e));
+                *reinterpret_cast<uint32_t*>(codes + (size_t)n * L.row_bytes + (k >> 1)) = word;
             }
         }
     }
