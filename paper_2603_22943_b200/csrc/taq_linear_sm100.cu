@@ -344,60 +344,76 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
                     }
                 }
             } else {
-                // Per-(row, head) symmetric int8.  A thread's columns are either one whole head (d = HC) or half of the
-                // tile's single head (d = BN); in the second case the row's two threads exchange their absmax.
+                // Per-(row, head) symmetric int8.  A thread's columns are either whole heads (HC a multiple of d) or half
+                // of the tile's single head (d = BN); in the second case the row's two threads exchange their absmax.
                 const int d = a.n_out / a.heads;
-                const bool whole_head = d == HC;
-                const int h = (col0 + cb) / d;
-                float amax = 0.f;
-#pragma unroll
-                for (int c = 0; c < HC; ++c) amax = fmaxf(amax, fabsf(y[c]));
-                if (!whole_head) {
-                    xchg[half * 128 + r] = amax;
-                    asm volatile("bar.sync 2, 256;" ::: "memory");
-                    amax = fmaxf(amax, xchg[(half ^ 1) * 128 + r]);
-                }
-                const float s = quant_scale(amax, 127.f);
-                const float rs = s > 0.f ? __frcp_rn(s) : 0.f;
-                const int ch = (col0 + cb) - h * d;                   // first owned column inside the head
-                if (a.epi == EPI_Q8_HEAD) {
-                    // Q~ = Q_a(Q), Eq. 2 third line
-                    if (row < a.rows) {
-                        int8_t* dst = (int8_t*)a.y + ((size_t)z * a.rows + row) * a.n_out + col0 + cb;
-#pragma unroll
-                        for (int c = 0; c < HC; c += 8) *reinterpret_cast<uint2*>(dst + c) = quant8(y + c, rs);
-                        if (whole_head || half == 0) a.scales[((size_t)z * a.rows + row) * a.heads + h] = s;
-                    }
-                } else if (row < a.rows) {
-                    // Eq. 2 for K or V: rows of ordinary tokens -> int8 codes + scale, rows of trigger tokens -> fp16
+                const bool whole_heads = HC % d == 0;
+                const int dd = whole_heads ? d : HC;                  // columns of one head held by this thread
+                int slot = -1;
+                bool trig = false;
+                int t = 0;
+                uint8_t* blk = nullptr;
+                taq_kv_layout KL;
+                if (a.epi == EPI_KV && row < a.rows) {
                     const int b = a.reqs ? 0 : (int)(row / a.n_ctx);
-                    const int t = (int)(row % a.n_ctx);
+                    t = (int)(row % a.n_ctx);
                     const uint8_t* mask = a.reqs ? a.reqs[z].trig_mask : a.mask + (size_t)b * a.n_ctx;
-                    const taq_kv_layout KL = kv_layout(a.heads, a.n_ctx, d, a.max_trigger);
-                    uint8_t* blk = a.reqs ? (uint8_t*)a.reqs[z].kv : (uint8_t*)a.y + (size_t)b * KL.block_bytes;
-                    const bool trig = mask[t] != 0;
-                    int slot = -1;
+                    KL = kv_layout(a.heads, a.n_ctx, d, a.max_trigger);
+                    blk = a.reqs ? (uint8_t*)a.reqs[z].kv : (uint8_t*)a.y + (size_t)b * KL.block_bytes;
+                    trig = mask[t] != 0;
                     if (trig) {
                         slot = 0;
                         for (int u = 0; u < t; ++u) slot += mask[u] != 0;
                         if (slot >= a.max_trigger) { raise_status(a.status, TAQ_ERR_SHAPE); slot = -2; }
                     }
-                    int8_t* cq = (int8_t*)(blk + (a.kv_which ? KL.off_v_codes : KL.off_k_codes)) + ((size_t)h * a.n_ctx + t) * d + ch;
+                }
 #pragma unroll
-                    for (int c = 0; c < HC; c += 8) *reinterpret_cast<uint2*>(cq + c) = trig ? make_uint2(0, 0) : quant8(y + c, rs);
-                    if (slot >= 0) {
-                        __half* tr = (__half*)(blk + (a.kv_which ? KL.off_v_trigger : KL.off_k_trigger)) + ((size_t)slot * a.heads + h) * d + ch;
+                for (int hc = 0; hc < HC; hc += 40) {                 // heads are 40, 64, 80 or 160 wide: steps of 40 or the whole of HC
+                    if (hc % dd != 0) continue;
+                    const int h = (col0 + cb + hc) / d;
+                    const int ch = (col0 + cb + hc) - h * d;          // first column of this piece inside the head
+                    float amax = 0.f;
 #pragma unroll
-                        for (int c = 0; c < HC; c += 8) {
-                            float f[8];
-#pragma unroll
-                            for (int e = 0; e < 8; ++e) f[e] = y[c + e];
-                            *reinterpret_cast<uint4*>(tr + c) = pack8(f);
-                        }
+                    for (int c = 0; c < HC; ++c)
+                        if (c >= hc && c < hc + dd) amax = fmaxf(amax, fabsf(y[c]));
+                    if (!whole_heads) {
+                        xchg[half * 128 + r] = amax;
+                        asm volatile("bar.sync 2, 256;" ::: "memory");
+                        amax = fmaxf(amax, xchg[(half ^ 1) * 128 + r]);
                     }
-                    if (whole_head || half == 0) {
-                        ((float*)(blk + (a.kv_which ? KL.off_v_scales : KL.off_k_scales)))[(size_t)h * a.n_ctx + t] = trig ? 0.f : s;
-                        if (h == 0 && a.kv_which == 0) ((int32_t*)(blk + KL.off_trig_slot))[t] = slot >= 0 ? slot : -1;
+                    const float s = quant_scale(amax, 127.f);
+                    const float rs = s > 0.f ? __frcp_rn(s) : 0.f;
+                    const bool owner = whole_heads || half == 0;      // writes the head's scale
+                    if (a.epi == EPI_Q8_HEAD) {
+                        // Q~ = Q_a(Q), Eq. 2 third line
+                        if (row < a.rows) {
+                            int8_t* dst = (int8_t*)a.y + ((size_t)z * a.rows + row) * a.n_out + col0 + cb;
+#pragma unroll
+                            for (int c = 0; c < HC; c += 8)
+                                if (c >= hc && c < hc + dd) *reinterpret_cast<uint2*>(dst + c) = quant8(y + c, rs);
+                            if (owner) a.scales[((size_t)z * a.rows + row) * a.heads + h] = s;
+                        }
+                    } else if (row < a.rows) {
+                        // Eq. 2 for K or V: rows of ordinary tokens -> int8 codes + scale, rows of trigger tokens -> fp16
+                        int8_t* cq = (int8_t*)(blk + (a.kv_which ? KL.off_v_codes : KL.off_k_codes)) + ((size_t)h * a.n_ctx + t) * d + ch;
+#pragma unroll
+                        for (int c = 0; c < HC; c += 8)
+                            if (c >= hc && c < hc + dd) *reinterpret_cast<uint2*>(cq + c - hc) = trig ? make_uint2(0, 0) : quant8(y + c, rs);
+                        if (slot >= 0) {
+                            __half* tr = (__half*)(blk + (a.kv_which ? KL.off_v_trigger : KL.off_k_trigger)) + ((size_t)slot * a.heads + h) * d + ch;
+#pragma unroll
+                            for (int c = 0; c < HC; c += 8)
+                                if (c >= hc && c < hc + dd) {
+                                    float f[8];
+#pragma unroll
+                                    for (int e = 0; e < 8; ++e) f[e] = y[c + e];
+                                    *reinterpret_cast<uint4*>(tr + c - hc) = pack8(f);
+                                }
+                        }
+                        if (owner) {
+                            ((float*)(blk + (a.kv_which ? KL.off_v_scales : KL.off_k_scales)))[(size_t)h * a.n_ctx + t] = trig ? 0.f : s;
+                            if (h == 0 && a.kv_which == 0) ((int32_t*)(blk + KL.off_trig_slot))[t] = slot >= 0 ? slot : -1;
+                        }
                     }
                 }
                 if (a.epi == EPI_KV && a.kv_which == 0 && blockIdx.x == 0 && blockIdx.y == 0) {   // slot table beyond T
@@ -439,13 +455,17 @@ EncodeTiledFn encode_tiled_fn() {
 }
 
 int pick_bn(const LinearArgs& a) {
+    // Every column tile re-reads the activation rows, so tiles are as wide as the row count allows while the grid
+    // still covers most of the SMs.
+    const long long row_tiles = (a.rows + BM - 1) / BM;
     if (a.epi == EPI_Q8_HEAD || a.epi == EPI_KV) {
         const int d = a.n_out / a.heads;
-        if (d == 40 && a.heads % 2 == 0) return 80;     // two heads per tile, one per worker thread of a row
+        if (d == 40 && a.heads % 4 == 0 && row_tiles * (a.n_out / 160) >= 96) return 160;   // two heads per worker thread
+        if (d == 40 && a.heads % 2 == 0) return 80;     // one head per worker thread
         if (d == 64 || d == 80 || d == 160) return d;   // one head per tile, split between the row's two threads
         return 0;
     }
-    if (a.n_out % 160 == 0 && a.rows * (a.n_out / 160) >= 148LL * 128) return 160;
+    if (a.n_out % 160 == 0 && row_tiles * (a.n_out / 160) >= 96) return 160;
     if (a.n_out % 80 == 0) return 80;
     if (a.n_out % 64 == 0) return 64;
     return 0;

@@ -85,10 +85,11 @@ def test_pack_weights_codes_bit_exact(n_out, k_in, bits, group):
     offs = raw[32:64].view(np.uint64)
     assert offs[3] == raw.size == tb.taq_packed_weight_bytes(d)
     assert np.array_equal(raw[int(offs[2]): int(offs[2]) + 4 * n_out].view(np.float32), bias)
-    if bits == 4:                                           # nibble order: even fan-in index in the low nibble, code + 8
-        row0 = raw[int(offs[0]): int(offs[0]) + k_in // 2]
-        assert np.array_equal((row0 & 0xF).astype(np.int32) - 8, want_c[0, 0::2])
-        assert np.array_equal((row0 >> 4).astype(np.int32) - 8, want_c[0, 1::2])
+    if bits == 4:   # eight codes per little-endian word: even fan-in indices in nibbles 0..3, odd ones in nibbles 4..7, code + 8
+        words = raw[int(offs[0]): int(offs[0]) + k_in // 2].view(np.uint32).astype(np.int64)
+        for e in range(8):
+            pos = (e >> 1) + ((e & 1) << 2)
+            assert np.array_equal(((words >> (4 * pos)) & 0xF).astype(np.int32) - 8, want_c[0, e::8])
 
 
 def test_pack_is_deterministic_and_respects_buffer_bounds():
