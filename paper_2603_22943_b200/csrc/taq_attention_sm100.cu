@@ -142,6 +142,8 @@ __global__ void __launch_bounds__(ATT_THREADS, Cfg<D>::CTAS_PER_SM) attention_sm
     __syncthreads();
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = misc->tmem_base;
+    ptx::pdl_trigger();
+    ptx::pdl_wait();          // Q~ comes from the previous kernel in the stream
 
     const taq_kv_layout KL = kv_layout(H, T, D, a.max_trigger);
     const uint8_t* blk = a.reqs ? (const uint8_t*)a.reqs[zb].kv : (const uint8_t*)a.kv + (size_t)b * KL.block_bytes;
@@ -390,8 +392,7 @@ cudaError_t launch_k(const AttnArgs& a, int n_z, cudaStream_t stream) {
     }
     const int hg = pick_heads_per_cta<D>(a, n_z);
     dim3 grid((a.n_query + ROWS - 1) / ROWS, a.heads / hg, n_z);
-    attention_sm100_kernel<D, Q8, TAIL_ONLY><<<grid, ATT_THREADS, C::TOTAL, stream>>>(a, hg);
-    return cudaGetLastError();
+    return launch_pdl(attention_sm100_kernel<D, Q8, TAIL_ONLY>, grid, dim3(ATT_THREADS), (size_t)C::TOTAL, stream, a, hg);
 }
 
 template <int D>

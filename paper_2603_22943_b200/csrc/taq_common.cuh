@@ -150,6 +150,23 @@ struct AttnArgs {
     int* status;
 };
 
+// Launch with the programmatic-serialization attribute (see ptx::pdl_wait): the kernel's prologue may overlap the
+// tail of the previous kernel in the stream.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 cudaError_t launch_linear_simt(const LinearArgs& a, int n_z, cudaStream_t stream);
 cudaError_t launch_attention_simt(const AttnArgs& a, int n_z, cudaStream_t stream);
 cudaError_t launch_quantize_rows(const float* x, long long rows, int cols, int qmax, int8_t* codes, float* scales,

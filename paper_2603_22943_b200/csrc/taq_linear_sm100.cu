@@ -164,6 +164,8 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
     __syncthreads();
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = bars->tmem_base;
+    ptx::pdl_trigger();
+    ptx::pdl_wait();          // the activations (and, in general, the weights) may come from the previous kernel
 
     if (warp == 0) {
         // ---------------- producer: packed weights once, then activation tiles ----------------
@@ -506,8 +508,7 @@ cudaError_t launch_bn(const CUtensorMap& tmap, const LinearArgs& a, int n_z, cud
     const int ns = pick_nstage<BN>(a);
     const Plan P = make_plan<BN>(a.k_in, a.bits, a.group, ns);
     dim3 grid((unsigned)((a.rows + BM - 1) / BM), a.n_out / BN, n_z);
-    linear_sm100_kernel<BN><<<grid, NTHREADS, P.total, stream>>>(tmap, a, ns);
-    return cudaGetLastError();
+    return launch_pdl(linear_sm100_kernel<BN>, grid, dim3(NTHREADS), (size_t)P.total, stream, tmap, a, ns);
 }
 
 }  // namespace

@@ -42,6 +42,14 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
     return true;
 }
 
+// ---- programmatic dependent launch ---------------------------------------------------------------------
+// A kernel launched with the programmatic-serialization attribute may start while its predecessor in the stream
+// is still draining.  pdl_wait() returns once the predecessor has completed and its writes are visible; nothing
+// that the predecessor may have written (or may still read) is touched before it.  pdl_trigger() lets the
+// successor's CTAs be scheduled as soon as resources allow.  Both are no-ops for an ordinary launch.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---- proxies and fences -----------------------------------------------------------------------------
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
