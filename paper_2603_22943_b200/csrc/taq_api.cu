@@ -340,6 +340,7 @@ static taq_status layer_forward_impl(const taq_layer_desc* d, const taq_request*
     o.y = y;
     o.rows = rows_per_z; o.n_out = d->channels; o.k_in = d->channels; o.bits = d->w_bits; o.group = d->w_group;
     o.heads = 1; o.epi = EPI_F16; o.status = status;
+    o.early_weights = 1;        // the kernel before it in the stream is the attention above, which writes O only
     return run_linear(o, n_req, st);
 }
 

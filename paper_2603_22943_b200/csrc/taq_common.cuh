@@ -135,6 +135,8 @@ struct LinearArgs {
     int n_ctx, max_trigger;     // EPI_KV: rows = batch * n_ctx
     int kv_which;               // EPI_KV: 0 = K, 1 = V
     int epi;
+    int early_weights;          // the previous kernel in the stream is known not to write the weights: fetch and expand
+                                // them before waiting for it
     int* status;
 };
 

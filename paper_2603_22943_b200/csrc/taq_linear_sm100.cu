@@ -165,15 +165,16 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = bars->tmem_base;
     ptx::pdl_trigger();
-    ptx::pdl_wait();          // the activations (and, in general, the weights) may come from the previous kernel
 
     if (warp == 0) {
         // ---------------- producer: packed weights once, then activation tiles ----------------
         if (lane == 0) {
+            if (!a.early_weights) ptx::pdl_wait();        // in general the weights may come from the previous kernel
             ptx::mbar_arrive_expect_tx(&bars->w_full, (uint32_t)(P.raw_bytes + P.scale_bytes + P.bias_bytes));
             ptx::bulk_load(smem + P.off_raw, blob + L.off_codes + (size_t)col0 * L.row_bytes, (uint32_t)P.raw_bytes, &bars->w_full);
             ptx::bulk_load(smem + P.off_scales, blob + L.off_scales + (size_t)col0 * n_groups * 4, (uint32_t)P.scale_bytes, &bars->w_full);
             ptx::bulk_load(smem + P.off_bias, blob + L.off_bias + (size_t)col0 * 4, (uint32_t)P.bias_bytes, &bars->w_full);
+            if (a.early_weights) ptx::pdl_wait();         // the activations come from the previous kernel
             int issued = 0, s = 0;
             uint32_t ph = 0;                               // parity of the ring pass
             for (int kb = 0; kb < n_kb; ++kb) {
@@ -325,25 +326,34 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
         if (!ok) { raise_status(a.status, TAQ_ERR_TIMEOUT); bars->abort_flag = 1; }
         asm volatile("bar.sync 1, 256;" ::: "memory");       // every worker gets here; the decision below is uniform
         ok = !bars->abort_flag;
+        ptx::pdl_wait();                                     // (already satisfied: the activations have arrived) orders the stores below
 
         // ---------------- epilogue on this thread's HC columns ----------------
         if (ok) {
             if (a.epi == EPI_F16 || a.epi == EPI_F32) {
-                if (row < a.rows) {
-                    const size_t o = ((size_t)z * a.rows + row) * a.n_out + col0 + cb;
+                // The thread's HC outputs are one contiguous piece of its row: stage them in shared memory (the ring
+                // is free now; pieces are padded by 16 bytes against bank conflicts) and hand the piece to the copy
+                // engine, instead of 16-byte stores scattered over 128 rows per warp.
+                const int esz = a.epi == EPI_F16 ? 2 : 4;
+                unsigned char* seg = smem + (size_t)(half * 128 + r) * (HC * esz + 16);
+                const size_t o = ((size_t)z * a.rows + row) * a.n_out + col0 + cb;
 #pragma unroll
-                    for (int c = 0; c < HC; c += 8) {
-                        float f[8];
+                for (int c = 0; c < HC; c += 8) {
+                    float f[8];
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) f[e] = y[c + e] + bias[cb + c + e];
-                        if (a.epi == EPI_F16) {
-                            *reinterpret_cast<uint4*>((__half*)a.y + o + c) = pack8(f);
-                        } else {
-                            float4* dst = reinterpret_cast<float4*>((float*)a.y + o + c);
-                            dst[0] = make_float4(f[0], f[1], f[2], f[3]);
-                            dst[1] = make_float4(f[4], f[5], f[6], f[7]);
-                        }
+                    for (int e = 0; e < 8; ++e) f[e] = y[c + e] + bias[cb + c + e];
+                    if (a.epi == EPI_F16) {
+                        *reinterpret_cast<uint4*>(seg + c * 2) = pack8(f);
+                    } else {
+                        *reinterpret_cast<float4*>(seg + c * 4) = make_float4(f[0], f[1], f[2], f[3]);
+                        *reinterpret_cast<float4*>(seg + c * 4 + 16) = make_float4(f[4], f[5], f[6], f[7]);
                     }
+                }
+                ptx::fence_proxy_async_smem();
+                if (row < a.rows) {
+                    ptx::bulk_store((unsigned char*)a.y + o * esz, seg, HC * esz);
+                    ptx::bulk_store_commit();
+                    ptx::bulk_store_wait_read();
                 }
             } else {
                 // Per-(row, head) symmetric int8.  A thread's columns are either whole heads (HC a multiple of d) or half
@@ -388,13 +398,26 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
                     const bool owner = whole_heads || half == 0;      // writes the head's scale
                     if (a.epi == EPI_Q8_HEAD) {
                         // Q~ = Q_a(Q), Eq. 2 third line
-                        if (row < a.rows) {
-                            int8_t* dst = (int8_t*)a.y + ((size_t)z * a.rows + row) * a.n_out + col0 + cb;
+                        int8_t* dst = (int8_t*)a.y + ((size_t)z * a.rows + row) * a.n_out + col0 + cb;
+                        if (HC % 16 == 0) {       // the codes of the thread's piece leave through shared memory in one bulk store
+                            unsigned char* seg = smem + (size_t)(half * 128 + r) * (HC + 16);
+#pragma unroll
+                            for (int c = 0; c < HC; c += 8)
+                                if (c >= hc && c < hc + dd) *reinterpret_cast<uint2*>(seg + c) = quant8(y + c, rs);
+                            if (hc + dd >= HC) {  // last head of the piece
+                                ptx::fence_proxy_async_smem();
+                                if (row < a.rows) {
+                                    ptx::bulk_store(dst, seg, HC);
+                                    ptx::bulk_store_commit();
+                                    ptx::bulk_store_wait_read();
+                                }
+                            }
+                        } else if (row < a.rows) {
 #pragma unroll
                             for (int c = 0; c < HC; c += 8)
                                 if (c >= hc && c < hc + dd) *reinterpret_cast<uint2*>(dst + c) = quant8(y + c, rs);
-                            if (owner) a.scales[((size_t)z * a.rows + row) * a.heads + h] = s;
                         }
+                        if (row < a.rows && owner) a.scales[((size_t)z * a.rows + row) * a.heads + h] = s;
                     } else if (row < a.rows) {
                         // Eq. 2 for K or V: rows of ordinary tokens -> int8 codes + scale, rows of trigger tokens -> fp16
                         int8_t* cq = (int8_t*)(blk + (a.kv_which ? KL.off_v_codes : KL.off_k_codes)) + ((size_t)h * a.n_ctx + t) * d + ch;
