@@ -332,6 +332,7 @@ static taq_status layer_forward_impl(const taq_layer_desc* d, const taq_request*
     AttnArgs at = attn_args(d, status);                                 // softmax(Q~K~^T/sqrt(d)), Eq. 3, P.V
     at.q = wsb + W.off_q; at.q_scales = (const float*)(wsb + W.off_qs); at.kv = kv; at.mask = mask; at.reqs = reqs;
     at.o = (__half*)(wsb + W.off_o);
+    at.early_kv = 1;            // the kernel before it in the stream is to_q above, which writes the workspace only
     s = run_attention(at, reqs ? n_req : d->batch, st);
     if (s != TAQ_OK) return s;
 

@@ -4,10 +4,11 @@
 //   A^ (Eq. 3)              ordinary columns -> uint8 code, trigger columns -> fp16, both in units of 1/255
 //   O = A^ V~               tcgen05.mma with the probabilities as the A operand and V~^T (fp16) as B; O = acc/255
 // A CTA owns 128 query rows of one sequence and walks over a group of heads, software-pipelined:
-//   warps 0-3  thread = query row = TMEM lane: stage the row's Q~ codes of the next head as an fp16 operand tile,
-//              softmax + Eq. 3 of the current head, epilogue of the previous head;
-//   warp 4     one thread issues the MMAs: S of head h+1 is in flight while the rows are in the softmax of head h;
-//   warp 5     one thread fetches each head's K~/V~ operand image (written once per prompt by the K/V projection)
+//   warps 0-7  two threads per query row (TMEM lane), one per half of the keys: stage the row's Q~ codes of the next
+//              head as an fp16 operand tile, softmax + Eq. 3 of the current head (the two threads of a row exchange
+//              their partial maximum and sum once per head), epilogue of the previous head;
+//   warp 8     one thread issues the MMAs: S of head h+1 is in flight while the rows are in the softmax of head h;
+//   warp 9     one thread fetches each head's K~/V~ operand image (written once per prompt by the K/V projection)
 //              with a single bulk copy, one head ahead.
 // Two CTAs share an SM for head widths up to 80, so one CTA's loads overlap the other's arithmetic.
 #include "taq_ptx.cuh"
@@ -19,8 +20,9 @@ namespace {
 
 constexpr int TP = kOperandKeys;     // keys padded to a multiple of 16
 constexpr int ROWS = 128;
-constexpr int ATT_THREADS = 192;
-constexpr int MMA_WARP = 4, COPY_WARP = 5;
+constexpr int ROW_WARPS = 8;         // two threads per query row
+constexpr int MMA_WARP = 8, COPY_WARP = 9;
+constexpr int ATT_THREADS = 320;
 
 template <int D>
 struct Cfg {
@@ -38,7 +40,7 @@ struct Cfg {
     static constexpr int OFF_Q = OFF_KV + KVBUF * HEAD_BYTES;
     static constexpr int OFF_P = OFF_Q + KBQ * A_BLOCK;
     static constexpr int OFF_MISC = OFF_P + 2 * A_BLOCK;
-    static constexpr int TOTAL = OFF_MISC + 1024 + 1024;     // misc block + slack for 1024-byte alignment
+    static constexpr int TOTAL = OFF_MISC + 4096 + 128 + 1024;   // misc block + slack for 1024-byte alignment
     static constexpr uint32_t TMEM_S = 0, TMEM_O = 2 * TP;
     static constexpr uint32_t TMEM_COLS = (2 * TP + OBUF * DP) <= 256 ? 256 : 512;
     static constexpr int CTAS_PER_SM = (2 * (TOTAL + 1024) <= 232448 && TMEM_COLS == 256) ? 2 : 1;
@@ -50,7 +52,9 @@ struct Misc {
     uint64_t kv_full[2], kv_free[2], q_full, s_full[2], p_full, o_full[2], drain;
     uint32_t tmem_base;
     volatile int abort_flag;
+    float2 xchg[2][2][ROWS];     // [head parity][half][row]: (max, sum) of a thread's half of the softmax
 };
+static_assert(sizeof(Misc) <= 4096 + 128, "misc block");
 
 __device__ __forceinline__ float ex2_approx(float x) {
     float y;
@@ -75,38 +79,104 @@ __device__ __forceinline__ uint4 codes8_to_half(uint2 raw) {
     return make_uint4(o[0], o[1], o[2], o[3]);
 }
 
-// Query codes (or fp16 values) of one row and head, held in registers between the global load and the store
-// into the operand tile.
+// Half of the query codes (or fp16 values) of one row and head, held in registers between the global load and
+// the store into the operand tile: the row's two threads take the lower and the upper half of the 16-byte chunks.
 template <int D, bool Q8>
 struct QRegs {
-    static constexpr int CH = Cfg<D>::DP / 8;
-    uint4 v[Q8 ? (CH + 1) / 2 : CH];
-    __device__ __forceinline__ void load(const void* q, size_t elem_off, bool valid) {
+    static constexpr int CH2 = (Cfg<D>::DP / 8 + 1) / 2;      // chunks (8 channels) per thread
+    uint4 v[Q8 ? (CH2 + 1) / 2 : CH2];
+    __device__ __forceinline__ void load(const void* q, size_t elem_off, bool valid, int half) {
+        const int c0 = half * CH2;
         if (Q8) {
 #pragma unroll
-            for (int i = 0; i < (CH + 1) / 2; ++i) {
+            for (int i = 0; i < (CH2 + 1) / 2; ++i) {
                 uint2 lo = make_uint2(0, 0), hi = make_uint2(0, 0);
-                if (valid && (2 * i) * 8 < D) lo = *reinterpret_cast<const uint2*>((const int8_t*)q + elem_off + (2 * i) * 8);
-                if (valid && (2 * i + 1) * 8 < D) hi = *reinterpret_cast<const uint2*>((const int8_t*)q + elem_off + (2 * i + 1) * 8);
+                if (valid && (c0 + 2 * i) * 8 < D) lo = *reinterpret_cast<const uint2*>((const int8_t*)q + elem_off + (c0 + 2 * i) * 8);
+                if (valid && 2 * i + 1 < CH2 && (c0 + 2 * i + 1) * 8 < D) hi = *reinterpret_cast<const uint2*>((const int8_t*)q + elem_off + (c0 + 2 * i + 1) * 8);
                 v[i] = make_uint4(lo.x, lo.y, hi.x, hi.y);
             }
         } else {
 #pragma unroll
-            for (int i = 0; i < CH; ++i) {
+            for (int i = 0; i < CH2; ++i) {
                 v[i] = make_uint4(0, 0, 0, 0);
-                if (valid && i * 8 < D) v[i] = *reinterpret_cast<const uint4*>((const __half*)q + elem_off + i * 8);
+                if (valid && (c0 + i) * 8 < D) v[i] = *reinterpret_cast<const uint4*>((const __half*)q + elem_off + (c0 + i) * 8);
             }
         }
     }
-    // chunk cc (8 channels) as fp16 operands; channels beyond D are zero (a zero int8 code maps to fp16 zero)
-    __device__ __forceinline__ uint4 chunk(int cc) const {
+    // local chunk i (8 channels) as fp16 operands; channels beyond D are zero (a zero int8 code maps to fp16 zero)
+    __device__ __forceinline__ uint4 chunk(int i) const {
         if (Q8) {
-            const uint4 w = v[cc / 2];
-            return codes8_to_half((cc & 1) ? make_uint2(w.z, w.w) : make_uint2(w.x, w.y));
+            const uint4 w = v[i / 2];
+            return codes8_to_half((i & 1) ? make_uint2(w.z, w.w) : make_uint2(w.x, w.y));
         }
-        return v[cc];
+        return v[i];
     }
 };
+
+constexpr int HK = TP / 2;           // keys per thread: a row's scores are split between two threads
+
+// Softmax pieces of one thread: its HK raw scores u (integer dot products) -> e_j = 2^(s_j sq - m) with the
+// thread's own maximum m (log2 units), and their sum.  Keys at or beyond T get weight exactly 0.
+template <bool TAIL_ONLY>
+__device__ __forceinline__ void softmax_half(const uint32_t (&u)[HK], const float* factor, float sq, int T, int key0, float (&e)[HK], float& m_out, float& l_out) {
+#pragma unroll
+    for (int j4 = 0; j4 < HK / 4; ++j4) {
+        const float4 f = *reinterpret_cast<const float4*>(factor + 4 * j4);
+        e[4 * j4 + 0] = __uint_as_float(u[4 * j4 + 0]) * f.x;
+        e[4 * j4 + 1] = __uint_as_float(u[4 * j4 + 1]) * f.y;
+        e[4 * j4 + 2] = __uint_as_float(u[4 * j4 + 2]) * f.z;
+        e[4 * j4 + 3] = __uint_as_float(u[4 * j4 + 3]) * f.w;
+    }
+#pragma unroll
+    for (int j = 0; j < HK; ++j)
+        if (j >= 64 - HK || !TAIL_ONLY) { if (key0 + j >= T) e[j] = -INFINITY; }
+    float m4[4] = {-1e30f, -1e30f, -1e30f, -1e30f};          // finite floor: a thread whose keys are all padding
+#pragma unroll
+    for (int j = 0; j < HK; ++j) m4[j & 3] = fmaxf(m4[j & 3], e[j]);
+    const float msq = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])) * sq;
+    float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int j = 0; j < HK; ++j) {
+        float arg = fmaf(e[j], sq, -msq);
+        if (j >= 64 - HK || !TAIL_ONLY) { if (key0 + j >= T) arg = -INFINITY; }      // also when sq = 0
+        e[j] = ex2_approx(arg);
+        sum4[j & 3] += e[j];
+    }
+    m_out = msq;
+    l_out = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+}
+
+// Eq. 3 on the thread's HK probabilities e_j * k255 (units of 1/255): ordinary columns -> rint (exact, ties to even),
+// trigger columns -> fp16.  fma(e, k, 1.5 * 2^23 + 0x6400) leaves the integer code in the low byte and 0x64 above it,
+// which read as fp16 is 1024 + code.  `trig` holds the thread's HK trigger bits.  Writes chunks chunk0.. of row `r`.
+__device__ __forceinline__ void write_p_half(const float (&e)[HK], float k255, unsigned long long trig, unsigned char* p_tile, int a_block, int r, int chunk0) {
+    const __half2 h1024 = __floats2half2_rn(1024.f, 1024.f);
+#pragma unroll
+    for (int g = 0; g < HK / 8; ++g) {
+        const uint32_t bits = (uint32_t)(trig >> (8 * g)) & 0xFFu;
+        uint32_t pk[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int j = g * 8 + 2 * i;
+            const uint32_t x0 = __float_as_uint(fmaf(e[j], k255, 12608512.0f));
+            const uint32_t x1 = __float_as_uint(fmaf(e[j + 1], k255, 12608512.0f));
+            uint32_t w = __byte_perm(x0, x1, 0x5410);
+            __half2 hv = __hsub2(*reinterpret_cast<__half2*>(&w), h1024);
+            pk[i] = *reinterpret_cast<uint32_t*>(&hv);
+        }
+        if (bits != 0) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int j = g * 8 + 2 * i;
+                __half2 raw = __floats2half2_rn(e[j] * k255, e[j + 1] * k255);
+                const uint32_t sel = (((bits >> (2 * i)) & 1u) ? 0x0054u : 0x0010u) | (((bits >> (2 * i + 1)) & 1u) ? 0x7600u : 0x3200u);
+                pk[i] = __byte_perm(pk[i], *reinterpret_cast<uint32_t*>(&raw), sel);
+            }
+        }
+        const int chunk = chunk0 + g;
+        *reinterpret_cast<uint4*>(p_tile + (chunk >> 3) * a_block + ptx::sw128_offset(r, chunk & 7)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+    }
+}
 
 template <int D, bool Q8, bool TAIL_ONLY>
 __global__ void __launch_bounds__(ATT_THREADS, Cfg<D>::CTAS_PER_SM) attention_sm100_kernel(const AttnArgs a, const int heads_per_cta) {
@@ -131,8 +201,8 @@ __global__ void __launch_bounds__(ATT_THREADS, Cfg<D>::CTAS_PER_SM) attention_sm
             ptx::mbar_init(&misc->s_full[i], 1);
             ptx::mbar_init(&misc->o_full[i], 1);
         }
-        ptx::mbar_init(&misc->q_full, ROWS / 32);      // one arrival per row warp
-        ptx::mbar_init(&misc->p_full, ROWS / 32);
+        ptx::mbar_init(&misc->q_full, ROW_WARPS);      // one arrival per row warp
+        ptx::mbar_init(&misc->p_full, ROW_WARPS);
         ptx::mbar_init(&misc->drain, 1);
         misc->abort_flag = 0;
         ptx::mbar_fence_init();
@@ -143,14 +213,14 @@ __global__ void __launch_bounds__(ATT_THREADS, Cfg<D>::CTAS_PER_SM) attention_sm
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = misc->tmem_base;
     ptx::pdl_trigger();
-    ptx::pdl_wait();          // Q~ comes from the previous kernel in the stream
 
     const taq_kv_layout KL = kv_layout(H, T, D, a.max_trigger);
-    const uint8_t* blk = a.reqs ? (const uint8_t*)a.reqs[zb].kv : (const uint8_t*)a.kv + (size_t)b * KL.block_bytes;
 
     if (warp == COPY_WARP) {
         // ---------------- K~/V~ operand images, one head ahead ----------------
         if (lane == 0) {
+            if (!a.early_kv) ptx::pdl_wait();             // in general the images may come from the previous kernel
+            const uint8_t* blk = a.reqs ? (const uint8_t*)a.reqs[zb].kv : (const uint8_t*)a.kv + (size_t)b * KL.block_bytes;
             const uint8_t* img = blk + KL.off_operands + (size_t)h_begin * KL.operand_head_bytes;
             int issued = 0;
             for (int hi = 0; hi < HG; ++hi) {
@@ -211,48 +281,56 @@ __global__ void __launch_bounds__(ATT_THREADS, Cfg<D>::CTAS_PER_SM) attention_sm
             }
         }
     } else {
-        // ---------------- row threads: thread = query row = TMEM lane ----------------
-        const int n = row0 + tid;
+        // ---------------- row threads: two per query row (TMEM lane), each with half of the keys ----------------
+        const int q4 = warp & 3, half = warp >> 2;
+        const int r = q4 * 32 + lane;
+        const int n = row0 + r;
         const bool valid = n < a.n_query;
         const size_t grow = (size_t)zb * a.n_query + (valid ? n : 0);
-        const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
+        const uint32_t lane_addr = (uint32_t)(q4 * 32) << 16;
+        const int key0 = half * HK;
         const float inv255 = 1.0f / 255.0f;
+        constexpr int CH2 = QRegs<D, Q8>::CH2;
+        constexpr int OC = DP / 2;                       // O columns per thread
         bool alive = true;
+        ptx::pdl_wait();                                 // Q~ comes from the previous kernel in the stream
 
-        auto store_o = [&](int hi) {        // O of head hi: acc / 255 -> fp16
-            __half* orow = a.o + grow * Cch + (h_begin + hi) * D;
-            const uint32_t t_o = tmem_base + C::TMEM_O + (hi % C::OBUF) * DP + lane_addr;
+        auto store_o = [&](int hi) {        // this thread's half of O of head hi: acc / 255 -> fp16
+            __half* orow = a.o + grow * Cch + (h_begin + hi) * D + half * OC;
+            const uint32_t t_o = tmem_base + C::TMEM_O + (hi % C::OBUF) * DP + half * OC + lane_addr;
+            uint32_t v[OC / 8][8];
 #pragma unroll
-            for (int c = 0; c < DP; c += 16) {
-                uint32_t v[16];
-                ptx::tmem_ld16(t_o + c, v);
-                ptx::tmem_ld_wait(v);
+            for (int i = 0; i < OC / 8; ++i) ptx::tmem_ld8(t_o + i * 8, v[i]);
+            ptx::tmem_ld_wait(v[0]);
 #pragma unroll
-                for (int half8 = 0; half8 < 2; ++half8) {
-                    if (c + half8 * 8 < D && valid) {
-                        uint32_t pk[4];
+            for (int i = 1; i < OC / 8; ++i) ptx::reg_fence8(v[i]);
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            __half2 hv = __floats2half2_rn(__uint_as_float(v[half8 * 8 + 2 * i]) * inv255, __uint_as_float(v[half8 * 8 + 2 * i + 1]) * inv255);
-                            pk[i] = *reinterpret_cast<uint32_t*>(&hv);
-                        }
-                        *reinterpret_cast<uint4*>(orow + c + half8 * 8) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+            for (int i = 0; i < OC / 8; ++i) {
+                if (half * OC + i * 8 < D && valid) {
+                    uint32_t pk[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        __half2 hv = __floats2half2_rn(__uint_as_float(v[i][2 * e]) * inv255, __uint_as_float(v[i][2 * e + 1]) * inv255);
+                        pk[e] = *reinterpret_cast<uint32_t*>(&hv);
                     }
+                    *reinterpret_cast<uint4*>(orow + i * 8) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                 }
             }
             ptx::tc_fence_before_sync();
         };
         auto stage_q = [&](const QRegs<D, Q8>& qr) {
 #pragma unroll
-            for (int cc = 0; cc < DP / 8; ++cc)
-                *reinterpret_cast<uint4*>(smem + C::OFF_Q + (cc / 8) * C::A_BLOCK + ptx::sw128_offset(tid, cc % 8)) = qr.chunk(cc);
+            for (int i = 0; i < CH2; ++i) {
+                const int cc = half * CH2 + i;
+                if (cc < DP / 8) *reinterpret_cast<uint4*>(smem + C::OFF_Q + (cc >> 3) * C::A_BLOCK + ptx::sw128_offset(r, cc & 7)) = qr.chunk(i);
+            }
             ptx::fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(&misc->q_full);
         };
 
         QRegs<D, Q8> qr;
-        qr.load(a.q, grow * Cch + (size_t)h_begin * D, valid);
+        qr.load(a.q, grow * Cch + (size_t)h_begin * D, valid, half);
         float sq = 1.0f, sq_next = 1.0f;
         if (Q8) sq = valid ? a.q_scales[grow * H + h_begin] : 0.f;
         stage_q(qr);
@@ -261,50 +339,38 @@ __global__ void __launch_bounds__(ATT_THREADS, Cfg<D>::CTAS_PER_SM) attention_sm
             const uint32_t ph = hi & 1;
             const bool more = hi + 1 < HG;
             if (more) {                         // next head's query codes: in flight while this head's S is awaited
-                qr.load(a.q, grow * Cch + (size_t)(h_begin + hi + 1) * D, valid);
+                qr.load(a.q, grow * Cch + (size_t)(h_begin + hi + 1) * D, valid, half);
                 if (Q8) sq_next = valid ? a.q_scales[grow * H + h_begin + hi + 1] : 0.f;
             }
             alive = __all_sync(0xffffffffu, ptx::mbar_wait(&misc->s_full[ph], (hi >> 1) & 1) && !misc->abort_flag);
             if (!alive) break;
             ptx::tc_fence_after_sync();
-            uint32_t u[TP / 16][16];
+            uint32_t u[HK];
+            {
+                const uint32_t t_s = tmem_base + C::TMEM_S + ph * TP + key0 + lane_addr;
+                uint32_t (&u8)[HK / 8][8] = *reinterpret_cast<uint32_t (*)[HK / 8][8]>(&u);
 #pragma unroll
-            for (int c = 0; c < TP / 16; ++c) ptx::tmem_ld16(tmem_base + C::TMEM_S + ph * TP + lane_addr + c * 16, u[c]);
-            ptx::tmem_ld_wait(u[0]);
+                for (int i = 0; i < HK / 8; ++i) ptx::tmem_ld8(t_s + i * 8, u8[i]);
+                ptx::tmem_ld_wait(u8[0]);
 #pragma unroll
-            for (int c = 1; c < TP / 16; ++c) ptx::reg_fence(u[c]);
+                for (int i = 1; i < HK / 8; ++i) ptx::reg_fence8(u8[i]);
+            }
             ptx::tc_fence_before_sync();
             if (more) stage_q(qr);              // S of this head is complete, so the Q~ tile is free again
 
-            // ---- softmax over the keys: logits in units of log2 ----
+            // ---- this thread's half of the softmax; the row's two threads then exchange (max, sum) ----
             const OperandConsts* cst = reinterpret_cast<const OperandConsts*>(smem + C::OFF_KV + (hi % C::KVBUF) * C::HEAD_BYTES + C::K_BYTES + C::VT_BYTES);
-            float s[TP];
-#pragma unroll
-            for (int j4 = 0; j4 < TP / 4; ++j4) {
-                const float4 f = *reinterpret_cast<const float4*>(&cst->logit_factor[4 * j4]);
-                s[4 * j4 + 0] = __uint_as_float(u[j4 / 4][(j4 % 4) * 4 + 0]) * f.x;
-                s[4 * j4 + 1] = __uint_as_float(u[j4 / 4][(j4 % 4) * 4 + 1]) * f.y;
-                s[4 * j4 + 2] = __uint_as_float(u[j4 / 4][(j4 % 4) * 4 + 2]) * f.z;
-                s[4 * j4 + 3] = __uint_as_float(u[j4 / 4][(j4 % 4) * 4 + 3]) * f.w;
-            }
-            const uint32_t tb0 = cst->trig_bits[0], tb1 = cst->trig_bits[1], tb2 = cst->trig_bits[2];
-#pragma unroll
-            for (int j = 0; j < TP; ++j)
-                if (j >= 64 || !TAIL_ONLY) { if (j >= T) s[j] = -INFINITY; }
-            float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-            for (int j = 0; j < TP; ++j) m4[j & 3] = fmaxf(m4[j & 3], s[j]);
-            const float mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
-            const float msq = mx * sq;
-            float sum4[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-            for (int j = 0; j < TP; ++j) {
-                float arg = fmaf(s[j], sq, -msq);
-                if (j >= 64 || !TAIL_ONLY) { if (j >= T) arg = -INFINITY; }      // padded keys: weight exactly 0, also when sq = 0
-                s[j] = ex2_approx(arg);
-                sum4[j & 3] += s[j];
-            }
-            const float k255 = __fdividef(255.0f, (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]));
+            float e[HK];
+            float m_loc, l_loc;
+            softmax_half<TAIL_ONLY>(u, cst->logit_factor + key0, sq, T, key0, e, m_loc, l_loc);
+            const unsigned long long trig = half == 0 ? ((unsigned long long)cst->trig_bits[0] | ((unsigned long long)(cst->trig_bits[1] & 0xFFu) << 32))
+                                                      : ((unsigned long long)(cst->trig_bits[1] >> 8) | ((unsigned long long)cst->trig_bits[2] << 24));
+            misc->xchg[ph][half][r] = make_float2(m_loc, l_loc);
+            asm volatile("bar.sync %0, 64;" ::"r"(1 + q4) : "memory");
+            const float2 other = misc->xchg[ph][half ^ 1][r];
+            const float m_all = fmaxf(m_loc, other.x);
+            const float c_self = ex2_approx(m_loc - m_all), c_other = ex2_approx(other.x - m_all);
+            const float k255 = __fdividef(255.0f * c_self, fmaf(l_loc, c_self, other.y * c_other));
 
             // the P tile is free once the previous head's PV has completed
             if (hi > 0) {
@@ -313,36 +379,7 @@ __global__ void __launch_bounds__(ATT_THREADS, Cfg<D>::CTAS_PER_SM) attention_sm
                 ptx::tc_fence_after_sync();
                 if (C::OBUF == 1) store_o(hi - 1);   // one O accumulator: empty it before the next PV may start
             }
-
-            // ---- Eq. 3: ordinary columns -> rint(255 p) (exact, ties to even), trigger columns -> fp16(255 p) ----
-            // fma(e, 255/sum, 1.5 * 2^23 + 0x6400) leaves the integer code in the low byte and 0x64 above it, which
-            // read as fp16 is 1024 + code.
-            const __half2 h1024 = __floats2half2_rn(1024.f, 1024.f);
-#pragma unroll
-            for (int jc = 0; jc < TP / 8; ++jc) {
-                const uint32_t word = jc < 4 ? tb0 : (jc < 8 ? tb1 : tb2);
-                const uint32_t bits = (word >> (8 * (jc % 4))) & 0xFFu;
-                uint32_t pk[4];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int j = jc * 8 + 2 * i;
-                    const uint32_t x0 = __float_as_uint(fmaf(s[j], k255, 12608512.0f));
-                    const uint32_t x1 = __float_as_uint(fmaf(s[j + 1], k255, 12608512.0f));
-                    uint32_t w = __byte_perm(x0, x1, 0x5410);
-                    __half2 hv = __hsub2(*reinterpret_cast<__half2*>(&w), h1024);
-                    pk[i] = *reinterpret_cast<uint32_t*>(&hv);
-                }
-                if (bits != 0) {
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const int j = jc * 8 + 2 * i;
-                        __half2 raw = __floats2half2_rn(s[j] * k255, s[j + 1] * k255);
-                        const uint32_t sel = (((bits >> (2 * i)) & 1u) ? 0x0054u : 0x0010u) | (((bits >> (2 * i + 1)) & 1u) ? 0x7600u : 0x3200u);
-                        pk[i] = __byte_perm(pk[i], *reinterpret_cast<uint32_t*>(&raw), sel);
-                    }
-                }
-                *reinterpret_cast<uint4*>(smem + C::OFF_P + (jc / 8) * C::A_BLOCK + ptx::sw128_offset(tid, jc % 8)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-            }
+            write_p_half(e, k255, trig, smem + C::OFF_P, C::A_BLOCK, r, half * (HK / 8));
             ptx::fence_proxy_async_smem();
             ptx::tc_fence_before_sync();
             __syncwarp();
