@@ -319,6 +319,11 @@ static taq_status layer_forward_impl(const taq_layer_desc* d, const taq_request*
     uint8_t* wsb = (uint8_t*)ws;
     const long long rows_per_z = (long long)d->batch * d->n_query;   // weights are shared by the whole batch
 
+    bool fused = sm100_qattn_supported(*d);
+    if (fused) {                                                        // to_q, Q_a and the attention in one kernel
+        cudaError_t e = launch_qattn_sm100(*d, (const __half*)x, Wq, kv, reqs, (__half*)(wsb + W.off_o), reqs ? n_req : d->batch, status, st);
+        if (e != cudaSuccess) return cuda_fail(e, "fused to_q + attention launch");
+    }
     LinearArgs q{};                                                     // to_q (+ Q~ = Q_a(Q))
     q.x = (const __half*)x; q.w = Wq; q.reqs = reqs; q.which = 0;
     q.y = wsb + W.off_q; q.scales = (float*)(wsb + W.off_qs);
@@ -326,15 +331,19 @@ static taq_status layer_forward_impl(const taq_layer_desc* d, const taq_request*
     q.heads = d->q_bits == 8 ? d->heads : 1;
     q.epi = d->q_bits == 8 ? EPI_Q8_HEAD : EPI_F16;
     q.status = status;
-    s = run_linear(q, n_req, st);
-    if (s != TAQ_OK) return s;
+    if (!fused) {
+        s = run_linear(q, n_req, st);
+        if (s != TAQ_OK) return s;
+    }
 
     AttnArgs at = attn_args(d, status);                                 // softmax(Q~K~^T/sqrt(d)), Eq. 3, P.V
     at.q = wsb + W.off_q; at.q_scales = (const float*)(wsb + W.off_qs); at.kv = kv; at.mask = mask; at.reqs = reqs;
     at.o = (__half*)(wsb + W.off_o);
     at.early_kv = 1;            // the kernel before it in the stream is to_q above, which writes the workspace only
-    s = run_attention(at, reqs ? n_req : d->batch, st);
-    if (s != TAQ_OK) return s;
+    if (!fused) {
+        s = run_attention(at, reqs ? n_req : d->batch, st);
+        if (s != TAQ_OK) return s;
+    }
 
     LinearArgs o{};                                                     // to_out (+ bias)
     o.x = (const __half*)(wsb + W.off_o); o.w = Wout; o.reqs = reqs; o.which = 1;

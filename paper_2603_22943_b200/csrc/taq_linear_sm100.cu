@@ -18,10 +18,13 @@
 // The packed weights stay packed in HBM and are read once per CTA.
 #include "taq_ptx.cuh"
 #include "taq_sm100.cuh"
+#include "taq_sm100_parts.cuh"
 
 namespace taq {
 
 namespace {
+
+using namespace parts;
 
 constexpr int BM = 128;
 constexpr int BK = 64;
@@ -73,55 +76,6 @@ __host__ __device__ inline Plan make_plan(int k_in, int bits, int group, int nst
     p.off_bars = p.off_xchg + 1024;
     p.total = p.off_bars + 256 + 1024;        // barriers + slack to align the base to 1024
     return p;
-}
-
-// Eight 4-bit codes of one word -> eight fp16 integers in fan-in order.  0x6400 | n read as fp16 is 1024 + n.
-__device__ __forceinline__ uint4 codes_w4_to_half(uint32_t p) {
-    const __half2 off = __floats2half2_rn(1032.f, 1032.f);                     // 1024 + the nibble bias of 8
-    uint32_t o[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        uint32_t w = ((p >> (4 * i)) & 0x000F000Fu) | 0x64006400u;
-        __half2 h = __hsub2(*reinterpret_cast<__half2*>(&w), off);
-        o[i] = *reinterpret_cast<uint32_t*>(&h);
-    }
-    return make_uint4(o[0], o[1], o[2], o[3]);
-}
-// Eight int8 codes -> eight fp16 integers: (code + 128) rides in the mantissa of 0x64xx.
-__device__ __forceinline__ uint4 codes_w8_to_half(uint2 raw) {
-    const __half2 off = __floats2half2_rn(1152.f, 1152.f);
-    const uint32_t w[2] = {raw.x ^ 0x80808080u, raw.y ^ 0x80808080u};
-    uint32_t o[4];
-#pragma unroll
-    for (int i = 0; i < 2; ++i) {
-        uint32_t lo = __byte_perm(w[i], 0x64646464u, 0x5140);
-        uint32_t hi = __byte_perm(w[i], 0x64646464u, 0x5342);
-        __half2 a = __hsub2(*reinterpret_cast<__half2*>(&lo), off);
-        __half2 b = __hsub2(*reinterpret_cast<__half2*>(&hi), off);
-        o[2 * i] = *reinterpret_cast<uint32_t*>(&a);
-        o[2 * i + 1] = *reinterpret_cast<uint32_t*>(&b);
-    }
-    return make_uint4(o[0], o[1], o[2], o[3]);
-}
-
-__device__ __forceinline__ uint4 pack8(const float (&w)[8]) {
-    uint4 out;
-    __half2 h;
-    h = __floats2half2_rn(w[0], w[1]); out.x = *reinterpret_cast<uint32_t*>(&h);
-    h = __floats2half2_rn(w[2], w[3]); out.y = *reinterpret_cast<uint32_t*>(&h);
-    h = __floats2half2_rn(w[4], w[5]); out.z = *reinterpret_cast<uint32_t*>(&h);
-    h = __floats2half2_rn(w[6], w[7]); out.w = *reinterpret_cast<uint32_t*>(&h);
-    return out;
-}
-
-// Eight values -> eight int8 codes rint(x * rs): fma(x, rs, 1.5 * 2^23) leaves the two's-complement code in the low byte.
-__device__ __forceinline__ uint2 quant8(const float* x, float rs) {
-    uint32_t b[8];
-#pragma unroll
-    for (int e = 0; e < 8; ++e) b[e] = __float_as_uint(fmaf(x[e], rs, 12582912.0f));
-    const uint32_t lo = __byte_perm(__byte_perm(b[0], b[1], 0x0040), __byte_perm(b[2], b[3], 0x0040), 0x5410);
-    const uint32_t hi = __byte_perm(__byte_perm(b[4], b[5], 0x0040), __byte_perm(b[6], b[7], 0x0040), 0x5410);
-    return make_uint2(lo, hi);
 }
 
 template <int BN>

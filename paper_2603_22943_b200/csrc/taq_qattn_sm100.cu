@@ -1,0 +1,482 @@
+// to_q and the TAQ attention in one kernel for the SD-1.5 64x64 shape (C = 320, 8 heads of 40, W4): Q never leaves
+// the SM.  A CTA owns 128 query rows of one sequence and four heads (160 output channels of to_q):
+//   phase 1  Q = X Wq^T for its 160 channels: the dequant-GEMM of taq_linear_sm100.cu (integer-code operands, one
+//            accumulation pass per scale group, folded into registers by the workers);
+//   phase 2  Q~ = Q_a(Q) (Eq. 2, third line) per (row, head) straight from those registers into the fp16-integer
+//            operand tiles of the four heads; the row scales stay in shared memory;
+//   phase 3  per head: S = Q~ K~^T, softmax, Eq. 3, O = A^ V~ as in taq_attention_sm100.cu (two threads per row,
+//            S of head h+1 under the softmax of head h), O stored as fp16.
+// Shared memory is used twice: the X tile and the weight ring of phase 1 become the Q~ tiles and the P tile.
+// Warps: 0 producer (TMA / bulk copies), 1 MMA issuer, 2..9 workers (two threads per row).
+#include "taq_ptx.cuh"
+#include "taq_sm100.cuh"
+#include "taq_sm100_parts.cuh"
+
+namespace taq {
+
+namespace {
+
+using namespace parts;
+
+constexpr int D = 40, DP = 48, HG = 4;          // head width, padded width, heads per CTA
+constexpr int NQ = HG * D;                      // 160 to_q channels per CTA
+constexpr int HC = NQ / 2;                      // channels per worker thread (two heads)
+constexpr int KIN = 320, BK = 64, NKB = KIN / BK;
+constexpr int ROWS = 128;
+constexpr int NWORK = 256, NTHREADS = 64 + NWORK;
+constexpr int NBSTAGE = 3;                      // ring of expanded weight tiles
+
+constexpr int A_TILE = ROWS * 128;              // 16 KB: one 64-wide K block of X, or one head's Q~ tile, or half of P
+constexpr int B_TILE = NQ * 128;                // 20 KB
+constexpr int K_BLOCK = TP * 128, VT_BLOCK = DP * 128;
+constexpr int K_BYTES = K_BLOCK, VT_BYTES = 2 * VT_BLOCK;
+constexpr int HEAD_BYTES = K_BYTES + VT_BYTES + kOperandConstBytes;     // 23552
+constexpr int MAX_GROUPS = NKB;
+constexpr int RAW_BYTES = NQ * (KIN / 2);       // 25600 (W4)
+constexpr int SCALE_BYTES = ((NQ * MAX_GROUPS * 4 + 127) / 128) * 128;
+
+constexpr int OFF_A = 0;                                    // phase 1: X tile, 5 K blocks
+constexpr int OFF_B = OFF_A + NKB * A_TILE;                 // phase 1: weight ring
+constexpr int OFF_Q = 0;                                    // phase 3: Q~ tiles of the four heads
+constexpr int OFF_P = OFF_Q + HG * A_TILE;                  // phase 3: probability tile (two K blocks)
+constexpr int OFF_RAW = OFF_B + NBSTAGE * B_TILE;
+constexpr int OFF_SC = OFF_RAW + RAW_BYTES;
+constexpr int OFF_SCT = OFF_SC + SCALE_BYTES;
+constexpr int OFF_KV = ((OFF_SCT + SCALE_BYTES + 1023) / 1024) * 1024;
+constexpr int OFF_MISC = OFF_KV + 2 * HEAD_BYTES;
+static_assert(OFF_P + 2 * A_TILE <= OFF_RAW, "phase-3 tiles must fit into the phase-1 region");
+
+struct Misc {
+    uint64_t a_full[NKB], b_full[NBSTAGE], b_empty[NBSTAGE], w_full, acc_full[2], acc_free[2];
+    uint64_t q_all, kv_full[2], kv_free[2], s_full[2], p_full, o_full[2], drain;
+    uint32_t tmem_base;
+    volatile int abort_flag;
+    float sq[HG][ROWS];              // Q~ row scales
+    float2 xchg[2][2][ROWS];         // [head parity][half][row]
+};
+constexpr int TOTAL = OFF_MISC + (int)sizeof(Misc) + 1024;
+static_assert(TOTAL <= 232448, "shared memory budget");
+
+constexpr uint32_t TMEM_COLS = 512;
+constexpr uint32_t TMEM_ACC = 0;                 // phase 1: two accumulators of NQ columns
+constexpr uint32_t TMEM_S = 0, TMEM_O = 2 * TP;  // phase 3: S double-buffered, O double-buffered (reuses the columns)
+
+struct QAttnArgs {
+    const __half* x;            // [z][B][N][C]
+    const void* wq;             // packed [C][C] (single problem)
+    const void* kv;             // blocks [B] (single problem)
+    const taq_request* reqs;    // nullable; then one sequence per request
+    __half* o;                  // [z][B][N][C]
+    int n_query, heads, n_ctx, max_trigger, group, q_bits;
+    int* status;
+};
+
+template <bool TAIL_ONLY>
+__global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_constant__ CUtensorMap tmap_x, const QAttnArgs a) {
+    extern __shared__ unsigned char smem_dyn[];
+    unsigned char* smem = smem_dyn + ((1024u - (ptx::smem_u32(smem_dyn) & 1023u)) & 1023u);   // 1024-byte aligned, still provably shared
+    Misc* misc = reinterpret_cast<Misc*>(smem + OFF_MISC);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int T = a.n_ctx, H = a.heads;
+    const int zb = blockIdx.z;                      // sequence (batch entry or request)
+    const int row0 = blockIdx.x * ROWS;
+    const int h_begin = blockIdx.y * HG;
+    const int col0 = h_begin * D;
+    const WeightLayout L = weight_layout(KIN, KIN, 4, a.group);
+    const int n_groups = L.n_groups;
+    const int kb_per_group = L.group_len / BK;
+
+    if (tid == 0) {
+        for (int i = 0; i < NKB; ++i) ptx::mbar_init(&misc->a_full[i], 1);
+        for (int i = 0; i < NBSTAGE; ++i) {
+            ptx::mbar_init(&misc->b_full[i], NWORK / 32);
+            ptx::mbar_init(&misc->b_empty[i], 1);
+        }
+        ptx::mbar_init(&misc->w_full, 1);
+        for (int i = 0; i < 2; ++i) {
+            ptx::mbar_init(&misc->acc_full[i], 1);
+            ptx::mbar_init(&misc->acc_free[i], NWORK / 32);
+            ptx::mbar_init(&misc->kv_full[i], 1);
+            ptx::mbar_init(&misc->kv_free[i], 1);
+            ptx::mbar_init(&misc->s_full[i], 1);
+            ptx::mbar_init(&misc->o_full[i], 1);
+        }
+        ptx::mbar_init(&misc->q_all, NWORK / 32);
+        ptx::mbar_init(&misc->p_full, NWORK / 32);
+        ptx::mbar_init(&misc->drain, 1);
+        misc->abort_flag = 0;
+        ptx::mbar_fence_init();
+        ptx::tma_prefetch_desc(&tmap_x);
+    }
+    if (warp == 1) ptx::tmem_alloc(&misc->tmem_base, TMEM_COLS);
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_base = misc->tmem_base;
+    ptx::pdl_trigger();
+
+    const taq_kv_layout KL = kv_layout(H, T, D, a.max_trigger);
+
+    if (warp == 0) {
+        // ---------------- producer ----------------
+        if (lane == 0) {
+            ptx::pdl_wait();                              // X (and in general everything else) may come from the previous kernel
+            const uint8_t* blob = (const uint8_t*)(a.reqs ? a.reqs[zb].Wq : a.wq);
+            const uint32_t scale_bytes = (uint32_t)(NQ * n_groups * 4);
+            ptx::mbar_arrive_expect_tx(&misc->w_full, RAW_BYTES + scale_bytes);
+            ptx::bulk_load(smem + OFF_RAW, blob + L.off_codes + (size_t)col0 * L.row_bytes, RAW_BYTES, &misc->w_full);
+            ptx::bulk_load(smem + OFF_SC, blob + L.off_scales + (size_t)col0 * n_groups * 4, scale_bytes, &misc->w_full);
+            for (int kb = 0; kb < NKB; ++kb) {            // the whole X tile at once: every K block has its own buffer
+                ptx::mbar_arrive_expect_tx(&misc->a_full[kb], A_TILE);
+                ptx::tma_load_3d(smem + OFF_A + kb * A_TILE, &tmap_x, &misc->a_full[kb], kb * BK, row0, zb);
+            }
+            const uint8_t* blk = a.reqs ? (const uint8_t*)a.reqs[zb].kv : (const uint8_t*)a.kv + (size_t)zb * KL.block_bytes;
+            const uint8_t* img = blk + KL.off_operands + (size_t)h_begin * KL.operand_head_bytes;
+            int issued = 0;
+            for (int hi = 0; hi < HG; ++hi) {             // K~/V~ operand images, two buffers
+                const int buf = hi & 1;
+                if (hi >= 2 && !ptx::mbar_wait(&misc->kv_free[buf], ((hi >> 1) - 1) & 1)) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; }
+                if (misc->abort_flag) break;
+                ptx::mbar_arrive_expect_tx(&misc->kv_full[buf], HEAD_BYTES);
+                ptx::bulk_load(smem + OFF_KV + buf * HEAD_BYTES, img + (size_t)hi * KL.operand_head_bytes, HEAD_BYTES, &misc->kv_full[buf]);
+                issued = hi + 1;
+            }
+            if (misc->abort_flag) {   // give copies that are still in flight a bounded chance to land before the CTA exits
+                (void)ptx::mbar_wait(&misc->w_full, 0);
+                for (int kb = 0; kb < NKB; ++kb) (void)ptx::mbar_wait(&misc->a_full[kb], 0);
+                for (int hi = issued > 2 ? issued - 2 : 0; hi < issued; ++hi) (void)ptx::mbar_wait(&misc->kv_full[hi & 1], (hi >> 1) & 1);
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0) {
+            bool ok = true;
+            {   // phase 1: one accumulation pass per scale group
+                constexpr uint32_t idesc = ptx::idesc_f16_m128(NQ);
+                int s = 0, kb = 0;
+                uint32_t ph = 0;
+                for (int g = 0; g < n_groups && ok; ++g) {
+                    const int buf = g & 1;
+                    if (g >= 2 && !ptx::mbar_wait(&misc->acc_free[buf], ((g >> 1) - 1) & 1)) ok = false;
+                    ptx::tc_fence_after_sync();
+                    const int kb_end = min(NKB, kb + kb_per_group);
+                    for (bool first = true; kb < kb_end && ok; ++kb) {
+                        if (!ptx::mbar_wait(&misc->a_full[kb], 0) || !ptx::mbar_wait(&misc->b_full[s], ph) || misc->abort_flag) { ok = false; break; }
+                        ptx::tc_fence_after_sync();
+                        const uint32_t a_addr = ptx::smem_u32(smem + OFF_A + kb * A_TILE);
+                        const uint32_t b_addr = ptx::smem_u32(smem + OFF_B + s * B_TILE);
+#pragma unroll
+                        for (int k = 0; k < BK / 16; ++k)
+                            ptx::mma_f16_ss(tmem_base + TMEM_ACC + buf * NQ, ptx::desc_k_sw128(a_addr + k * 32), ptx::desc_k_sw128(b_addr + k * 32), idesc, !(first && k == 0));
+                        first = false;
+                        ptx::mma_commit(&misc->b_empty[s]);
+                        if (++s == NBSTAGE) { s = 0; ph ^= 1; }
+                    }
+                    if (ok) ptx::mma_commit(&misc->acc_full[buf]);
+                }
+            }
+            // phase 3: the Q~ tiles of all four heads are in place once every worker warp has arrived
+            if (ok && !ptx::mbar_wait(&misc->q_all, 0)) ok = false;
+            const uint32_t q_addr = ptx::smem_u32(smem + OFF_Q), p_addr = ptx::smem_u32(smem + OFF_P);
+            auto issue_s = [&](int hi) -> bool {
+                const int buf = hi & 1;
+                if (!ptx::mbar_wait(&misc->kv_full[buf], (hi >> 1) & 1) || misc->abort_flag) return false;
+                ptx::tc_fence_after_sync();
+                const uint32_t k_addr = ptx::smem_u32(smem + OFF_KV + buf * HEAD_BYTES);
+#pragma unroll
+                for (int ks = 0; ks < DP / 16; ++ks)
+                    ptx::mma_f16_ss(tmem_base + TMEM_S + buf * TP, ptx::desc_k_sw128(q_addr + hi * A_TILE + ks * 32), ptx::desc_k_sw128(k_addr + ks * 32), ptx::idesc_f16_m128(TP), ks != 0);
+                ptx::mma_commit(&misc->s_full[buf]);
+                return true;
+            };
+            auto issue_pv = [&](int hi) -> bool {
+                const int buf = hi & 1;
+                if (!ptx::mbar_wait(&misc->p_full, hi & 1) || misc->abort_flag) return false;
+                ptx::tc_fence_after_sync();
+                const uint32_t vt_addr = ptx::smem_u32(smem + OFF_KV + buf * HEAD_BYTES + K_BYTES);
+#pragma unroll
+                for (int ks = 0; ks < TP / 16; ++ks)
+                    ptx::mma_f16_ss(tmem_base + TMEM_O + buf * DP, ptx::desc_k_sw128(p_addr + (ks / 4) * A_TILE + (ks % 4) * 32),
+                                    ptx::desc_k_sw128(vt_addr + (ks / 4) * VT_BLOCK + (ks % 4) * 32), ptx::idesc_f16_m128(DP), ks != 0);
+                ptx::mma_commit(&misc->o_full[buf]);
+                ptx::mma_commit(&misc->kv_free[buf]);
+                return true;
+            };
+            if (ok) ok = issue_s(0);
+            for (int hi = 0; hi < HG && ok; ++hi) {
+                if (hi + 1 < HG) ok = issue_s(hi + 1);       // S of the next head runs under this head's softmax
+                if (ok) ok = issue_pv(hi);
+            }
+            if (!ok) {
+                raise_status(a.status, TAQ_ERR_TIMEOUT);
+                misc->abort_flag = 1;
+                ptx::mma_commit(&misc->drain);               // wait (bounded) for whatever was issued before TMEM is given back
+                (void)ptx::mbar_wait(&misc->drain, 0);
+            }
+        }
+    } else {
+        // ---------------- workers (warps 2..9): two threads per row ----------------
+        const int wt = tid - 64;
+        const int q4 = warp & 3, half = (warp - 2) >> 2;
+        const int r = q4 * 32 + lane;
+        const int n = row0 + r;
+        const bool valid = n < a.n_query;
+        const size_t grow = (size_t)zb * a.n_query + (valid ? n : 0);
+        const uint32_t lane_addr = (uint32_t)(q4 * 32) << 16;
+        const unsigned char* raw = smem + OFF_RAW;
+        const float* wscales = reinterpret_cast<const float*>(smem + OFF_SC);
+        float* scales_t = reinterpret_cast<float*>(smem + OFF_SCT);
+        bool ok = ptx::mbar_wait(&misc->w_full, 0);
+        for (int i = wt; i < NQ * n_groups; i += NWORK) scales_t[(i % n_groups) * NQ + i / n_groups] = wscales[i];
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+
+        // ---- phase 1: expand weight tiles, fold finished groups: y = this thread's 80 channels (two heads) of its row ----
+        float y[HC];
+#pragma unroll
+        for (int c = 0; c < HC; ++c) y[c] = 0.f;
+        const int cb = half * HC;
+        auto fold_group = [&](int g) -> bool {
+            const int buf = g & 1;
+            if (!ptx::mbar_wait(&misc->acc_full[buf], (g >> 1) & 1) || misc->abort_flag) return false;
+            ptx::tc_fence_after_sync();
+            const float* sg = scales_t + g * NQ + cb;
+            const uint32_t taddr = tmem_base + TMEM_ACC + buf * NQ + cb + lane_addr;
+#pragma unroll
+            for (int c0 = 0; c0 < HC; c0 += 40) {
+                uint32_t v[5][8];
+#pragma unroll
+                for (int i = 0; i < 5; ++i) ptx::tmem_ld8(taddr + c0 + i * 8, v[i]);
+                ptx::tmem_ld_wait(v[0]);
+#pragma unroll
+                for (int i = 1; i < 5; ++i) ptx::reg_fence8(v[i]);
+#pragma unroll
+                for (int i = 0; i < 5; ++i) {
+                    const float4 s0 = *reinterpret_cast<const float4*>(sg + c0 + i * 8), s1 = *reinterpret_cast<const float4*>(sg + c0 + i * 8 + 4);
+                    float* yy = y + c0 + i * 8;
+                    yy[0] = fmaf(__uint_as_float(v[i][0]), s0.x, yy[0]); yy[1] = fmaf(__uint_as_float(v[i][1]), s0.y, yy[1]);
+                    yy[2] = fmaf(__uint_as_float(v[i][2]), s0.z, yy[2]); yy[3] = fmaf(__uint_as_float(v[i][3]), s0.w, yy[3]);
+                    yy[4] = fmaf(__uint_as_float(v[i][4]), s1.x, yy[4]); yy[5] = fmaf(__uint_as_float(v[i][5]), s1.y, yy[5]);
+                    yy[6] = fmaf(__uint_as_float(v[i][6]), s1.z, yy[6]); yy[7] = fmaf(__uint_as_float(v[i][7]), s1.w, yy[7]);
+                }
+            }
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&misc->acc_free[buf]);
+            return true;
+        };
+        int s = 0, kb = 0;
+        uint32_t ph = 0;
+        auto build_group = [&]() -> bool {
+            const int kb_end = min(NKB, kb + kb_per_group);
+            for (; kb < kb_end; ++kb) {
+                if (kb >= NBSTAGE && !ptx::mbar_wait(&misc->b_empty[s], ph ^ 1)) return false;
+                if (misc->abort_flag) return false;
+                unsigned char* b_tile = smem + OFF_B + s * B_TILE;
+                constexpr int NCH = NQ * 8 / NWORK;         // 5 chunks of 8 weights per thread and K block
+                const int n0 = wt >> 3, c = wt & 7;
+                uint32_t pw[NCH];
+#pragma unroll
+                for (int i = 0; i < NCH; ++i) pw[i] = *reinterpret_cast<const uint32_t*>(raw + (n0 + 32 * i) * (KIN / 2) + kb * (BK / 2) + c * 4);
+#pragma unroll
+                for (int i = 0; i < NCH; ++i) *reinterpret_cast<uint4*>(b_tile + ptx::sw128_offset(n0 + 32 * i, c)) = codes_w4_to_half(pw[i]);
+                ptx::fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&misc->b_full[s]);
+                if (++s == NBSTAGE) { s = 0; ph ^= 1; }
+            }
+            return true;
+        };
+        for (int g = 0; g < n_groups && ok; ++g) {
+            ok = build_group();
+            if (ok && g >= 1) ok = fold_group(g - 1);
+        }
+        if (ok) ok = fold_group(n_groups - 1);
+        if (!ok) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; }
+        asm volatile("bar.sync 1, 256;" ::: "memory");       // all of phase 1 has been consumed: its shared memory is free
+        ok = !misc->abort_flag;
+
+        // ---- phase 2: Q~ = Q_a(Q) of this thread's two heads, written as fp16 integers into the heads' operand tiles ----
+        if (ok) {
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+                const int hi = half * 2 + hh;
+                float amax = 0.f;
+#pragma unroll
+                for (int c = 0; c < D; ++c) amax = fmaxf(amax, fabsf(y[hh * D + c]));
+                unsigned char* q_tile = smem + OFF_Q + hi * A_TILE;
+                if (a.q_bits == 8) {
+                    const float sc = quant_scale(amax, 127.f);
+                    const float rs = sc > 0.f ? __frcp_rn(sc) : 0.f;
+                    // fma(x, 1/s, 1.5 * 2^23 + 0x6480): the low half-word read as fp16 is 1152 + code
+                    const __half2 h1152 = __floats2half2_rn(1152.f, 1152.f);
+#pragma unroll
+                    for (int cc = 0; cc < D / 8; ++cc) {
+                        uint32_t pk[4];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const uint32_t x0 = __float_as_uint(fmaf(y[hh * D + cc * 8 + 2 * i], rs, 12608640.0f));
+                            const uint32_t x1 = __float_as_uint(fmaf(y[hh * D + cc * 8 + 2 * i + 1], rs, 12608640.0f));
+                            uint32_t w = __byte_perm(x0, x1, 0x5410);
+                            __half2 hv = __hsub2(*reinterpret_cast<__half2*>(&w), h1152);
+                            pk[i] = *reinterpret_cast<uint32_t*>(&hv);
+                        }
+                        *reinterpret_cast<uint4*>(q_tile + ptx::sw128_offset(r, cc)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    }
+                    misc->sq[hi][r] = valid ? sc : 0.f;
+                } else {                                    // Q stays fp16
+#pragma unroll
+                    for (int cc = 0; cc < D / 8; ++cc) {
+                        float f[8];
+#pragma unroll
+                        for (int e2 = 0; e2 < 8; ++e2) f[e2] = y[hh * D + cc * 8 + e2];
+                        *reinterpret_cast<uint4*>(q_tile + ptx::sw128_offset(r, cc)) = pack8(f);
+                    }
+                    misc->sq[hi][r] = 1.0f;
+                }
+                *reinterpret_cast<uint4*>(q_tile + ptx::sw128_offset(r, D / 8)) = make_uint4(0, 0, 0, 0);   // channels 40..47
+            }
+            ptx::fence_proxy_async_smem();
+        }
+        asm volatile("bar.sync 1, 256;" ::: "memory");       // the row scales of all heads are visible to both threads of a row
+        if (lane == 0) ptx::mbar_arrive(&misc->q_all);
+
+        // ---- phase 3: attention over the four heads; this thread has keys [40 half, 40 half + 40) of its row ----
+        const int key0 = half * HK;
+        const float inv255 = 1.0f / 255.0f;
+        constexpr int OC = DP / 2;
+        bool alive = ok;
+        auto store_o = [&](int hi) {
+            __half* orow = a.o + grow * (size_t)(H * D) + (h_begin + hi) * D + half * OC;
+            const uint32_t t_o = tmem_base + TMEM_O + (hi & 1) * DP + half * OC + lane_addr;
+            uint32_t v[OC / 8][8];
+#pragma unroll
+            for (int i = 0; i < OC / 8; ++i) ptx::tmem_ld8(t_o + i * 8, v[i]);
+            ptx::tmem_ld_wait(v[0]);
+#pragma unroll
+            for (int i = 1; i < OC / 8; ++i) ptx::reg_fence8(v[i]);
+#pragma unroll
+            for (int i = 0; i < OC / 8; ++i) {
+                if (half * OC + i * 8 < D && valid) {
+                    float f[8];
+#pragma unroll
+                    for (int e2 = 0; e2 < 8; ++e2) f[e2] = __uint_as_float(v[i][e2]) * inv255;
+                    *reinterpret_cast<uint4*>(orow + i * 8) = pack8(f);
+                }
+            }
+            ptx::tc_fence_before_sync();
+        };
+        for (int hi = 0; hi < HG && alive; ++hi) {
+            const uint32_t ph2 = hi & 1;
+            alive = __all_sync(0xffffffffu, ptx::mbar_wait(&misc->s_full[ph2], (hi >> 1) & 1) && !misc->abort_flag);
+            if (!alive) break;
+            ptx::tc_fence_after_sync();
+            uint32_t u[HK];
+            {
+                const uint32_t t_s = tmem_base + TMEM_S + ph2 * TP + key0 + lane_addr;
+                uint32_t (&u8)[HK / 8][8] = *reinterpret_cast<uint32_t (*)[HK / 8][8]>(&u);
+#pragma unroll
+                for (int i = 0; i < HK / 8; ++i) ptx::tmem_ld8(t_s + i * 8, u8[i]);
+                ptx::tmem_ld_wait(u8[0]);
+#pragma unroll
+                for (int i = 1; i < HK / 8; ++i) ptx::reg_fence8(u8[i]);
+            }
+            ptx::tc_fence_before_sync();
+            const OperandConsts* cst = reinterpret_cast<const OperandConsts*>(smem + OFF_KV + ph2 * HEAD_BYTES + K_BYTES + VT_BYTES);
+            const float sq = misc->sq[hi][r];
+            float e[HK];
+            float m_loc, l_loc;
+            softmax_half<TAIL_ONLY>(u, cst->logit_factor + key0, sq, T, key0, e, m_loc, l_loc);
+            const unsigned long long trig = half == 0 ? ((unsigned long long)cst->trig_bits[0] | ((unsigned long long)(cst->trig_bits[1] & 0xFFu) << 32))
+                                                      : ((unsigned long long)(cst->trig_bits[1] >> 8) | ((unsigned long long)cst->trig_bits[2] << 24));
+            misc->xchg[ph2][half][r] = make_float2(m_loc, l_loc);
+            asm volatile("bar.sync %0, 64;" ::"r"(2 + q4) : "memory");
+            const float2 other = misc->xchg[ph2][half ^ 1][r];
+            const float m_all = fmaxf(m_loc, other.x);
+            const float c_self = ex2_approx(m_loc - m_all), c_other = ex2_approx(other.x - m_all);
+            const float k255 = __fdividef(255.0f * c_self, fmaf(l_loc, c_self, other.y * c_other));
+            if (hi > 0) {       // the P tile is free once the previous head's PV has completed
+                alive = __all_sync(0xffffffffu, ptx::mbar_wait(&misc->o_full[(hi - 1) & 1], ((hi - 1) >> 1) & 1) && !misc->abort_flag);
+                if (!alive) break;
+                ptx::tc_fence_after_sync();
+            }
+            write_p_half(e, k255, trig, smem + OFF_P, A_TILE, r, half * (HK / 8));
+            ptx::fence_proxy_async_smem();
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&misc->p_full);
+            if (hi > 0) store_o(hi - 1);                    // under this head's PV
+        }
+        if (alive) {
+            alive = __all_sync(0xffffffffu, ptx::mbar_wait(&misc->o_full[(HG - 1) & 1], ((HG - 1) >> 1) & 1) && !misc->abort_flag);
+            if (alive) {
+                ptx::tc_fence_after_sync();
+                store_o(HG - 1);
+            }
+        }
+        if (!alive) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; }
+    }
+
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_tiled_fn2() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess && qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+}  // namespace
+
+bool sm100_qattn_supported(const taq_layer_desc& d) {
+    if (d.channels != KIN || d.heads * D != KIN) return false;
+    if (d.w_bits != 4) return false;
+    if (d.w_group != 0 && d.w_group % BK) return false;
+    if (d.n_ctx > TP || d.p_bits != 8) return false;
+    if (d.n_query < 1) return false;
+    return encode_tiled_fn2() != nullptr;
+}
+
+cudaError_t launch_qattn_sm100(const taq_layer_desc& d, const __half* x, const void* wq, const void* kv, const taq_request* reqs, __half* o,
+                               int n_z, int* status, cudaStream_t stream) {
+    if (n_z == 0 || d.n_query == 0) return cudaSuccess;
+    EncodeTiledFn enc = encode_tiled_fn2();
+    if (!enc) return cudaErrorNotSupported;
+    CUtensorMap tmap;
+    const cuuint64_t dims[3] = {(cuuint64_t)KIN, (cuuint64_t)d.n_query, (cuuint64_t)n_z};
+    const cuuint64_t strides[2] = {(cuuint64_t)KIN * 2, (cuuint64_t)KIN * 2 * (cuuint64_t)d.n_query};
+    const cuuint32_t box[3] = {BK, ROWS, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = enc(&tmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<__half*>(x), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+    QAttnArgs a{};
+    a.x = x; a.wq = wq; a.kv = kv; a.reqs = reqs; a.o = o;
+    a.n_query = d.n_query; a.heads = d.heads; a.n_ctx = d.n_ctx; a.max_trigger = d.max_trigger; a.group = d.w_group; a.q_bits = d.q_bits;
+    a.status = status;
+    dim3 grid((d.n_query + ROWS - 1) / ROWS, d.heads / HG, n_z);
+    static bool configured[2] = {false, false};
+    const bool tail = d.n_ctx > 64;
+    auto kern = tail ? qattn_c320_kernel<true> : qattn_c320_kernel<false>;
+    if (!configured[tail]) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TOTAL);
+        if (e != cudaSuccess) return e;
+        configured[tail] = true;
+    }
+    return launch_pdl(kern, grid, dim3(NTHREADS), (size_t)TOTAL, stream, tmap, a);
+}
+
+}  // namespace taq

@@ -11,4 +11,9 @@ cudaError_t launch_linear_sm100(const LinearArgs& a, int n_z, cudaStream_t strea
 bool sm100_attention_supported(const AttnArgs& a);
 cudaError_t launch_attention_sm100(const AttnArgs& a, int n_z, cudaStream_t stream);
 
+// to_q fused into the attention kernel (C = 320, 8 heads of 40, W4): x -> O without Q~ leaving the SM.
+bool sm100_qattn_supported(const taq_layer_desc& d);
+cudaError_t launch_qattn_sm100(const taq_layer_desc& d, const __half* x, const void* wq, const void* kv, const taq_request* reqs, __half* o,
+                               int n_z, int* status, cudaStream_t stream);
+
 }  // namespace taq
