@@ -1,7 +1,8 @@
 // to_q and the TAQ attention in one kernel for the SD-1.5 64x64 shape (C = 320, 8 heads of 40, W4): Q never leaves
 // the SM.  A CTA owns 128 query rows of one sequence and four heads (160 output channels of to_q):
 //   phase 1  Q = X Wq^T for its 160 channels: the dequant-GEMM of taq_linear_sm100.cu (integer-code operands, one
-//            accumulation pass per scale group, folded into registers by the workers);
+//            accumulation pass per scale group; here every group - at most three - has its own TMEM accumulator,
+//            so the tensor core never waits for the workers, who fold the groups into registers at the end);
 //   phase 2  Q~ = Q_a(Q) (Eq. 2, third line) per (row, head) straight from those registers into the fp16-integer
 //            operand tiles of the four heads; the row scales stay in shared memory;
 //   phase 3  per head: S = Q~ K~^T, softmax, Eq. 3, O = A^ V~ as in taq_attention_sm100.cu (two threads per row,
@@ -31,7 +32,7 @@ constexpr int B_TILE = NQ * 128;                // 20 KB
 constexpr int K_BLOCK = TP * 128, VT_BLOCK = DP * 128;
 constexpr int K_BYTES = K_BLOCK, VT_BYTES = 2 * VT_BLOCK;
 constexpr int HEAD_BYTES = K_BYTES + VT_BYTES + kOperandConstBytes;     // 23552
-constexpr int MAX_GROUPS = NKB;
+constexpr int MAX_GROUPS = 3;                    // one TMEM accumulator of NQ columns per scale group
 constexpr int RAW_BYTES = NQ * (KIN / 2);       // 25600 (W4)
 constexpr int SCALE_BYTES = ((NQ * MAX_GROUPS * 4 + 127) / 128) * 128;
 
@@ -47,7 +48,7 @@ constexpr int OFF_MISC = OFF_KV + 2 * HEAD_BYTES;
 static_assert(OFF_P + 2 * A_TILE <= OFF_RAW, "phase-3 tiles must fit into the phase-1 region");
 
 struct Misc {
-    uint64_t a_full[NKB], b_full[NBSTAGE], b_empty[NBSTAGE], w_full, acc_full[2], acc_free[2];
+    uint64_t a_full[NKB], b_full[NBSTAGE], b_empty[NBSTAGE], w_full, acc_full;
     uint64_t q_all, kv_full[2], kv_free[2], s_full[2], p_full, o_full[2], drain;
     uint32_t tmem_base;
     volatile int abort_flag;
@@ -58,7 +59,7 @@ constexpr int TOTAL = OFF_MISC + (int)sizeof(Misc) + 1024;
 static_assert(TOTAL <= 232448, "shared memory budget");
 
 constexpr uint32_t TMEM_COLS = 512;
-constexpr uint32_t TMEM_ACC = 0;                 // phase 1: two accumulators of NQ columns
+constexpr uint32_t TMEM_ACC = 0;                 // phase 1: up to three accumulators of NQ columns
 constexpr uint32_t TMEM_S = 0, TMEM_O = 2 * TP;  // phase 3: S double-buffered, O double-buffered (reuses the columns)
 
 struct QAttnArgs {
@@ -94,9 +95,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
             ptx::mbar_init(&misc->b_empty[i], 1);
         }
         ptx::mbar_init(&misc->w_full, 1);
+        ptx::mbar_init(&misc->acc_full, 1);
         for (int i = 0; i < 2; ++i) {
-            ptx::mbar_init(&misc->acc_full[i], 1);
-            ptx::mbar_init(&misc->acc_free[i], NWORK / 32);
             ptx::mbar_init(&misc->kv_full[i], 1);
             ptx::mbar_init(&misc->kv_free[i], 1);
             ptx::mbar_init(&misc->s_full[i], 1);
@@ -157,9 +157,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
                 int s = 0, kb = 0;
                 uint32_t ph = 0;
                 for (int g = 0; g < n_groups && ok; ++g) {
-                    const int buf = g & 1;
-                    if (g >= 2 && !ptx::mbar_wait(&misc->acc_free[buf], ((g >> 1) - 1) & 1)) ok = false;
-                    ptx::tc_fence_after_sync();
+                    const int buf = g;
                     const int kb_end = min(NKB, kb + kb_per_group);
                     for (bool first = true; kb < kb_end && ok; ++kb) {
                         if (!ptx::mbar_wait(&misc->a_full[kb], 0) || !ptx::mbar_wait(&misc->b_full[s], ph) || misc->abort_flag) { ok = false; break; }
@@ -173,8 +171,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
                         ptx::mma_commit(&misc->b_empty[s]);
                         if (++s == NBSTAGE) { s = 0; ph ^= 1; }
                     }
-                    if (ok) ptx::mma_commit(&misc->acc_full[buf]);
                 }
+                if (ok) ptx::mma_commit(&misc->acc_full);
             }
             // phase 3: the Q~ tiles of all four heads are in place once every worker warp has arrived
             if (ok && !ptx::mbar_wait(&misc->q_all, 0)) ok = false;
@@ -236,10 +234,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
 #pragma unroll
         for (int c = 0; c < HC; ++c) y[c] = 0.f;
         const int cb = half * HC;
-        auto fold_group = [&](int g) -> bool {
-            const int buf = g & 1;
-            if (!ptx::mbar_wait(&misc->acc_full[buf], (g >> 1) & 1) || misc->abort_flag) return false;
-            ptx::tc_fence_after_sync();
+        auto fold_group = [&](int g) {
+            const int buf = g;
             const float* sg = scales_t + g * NQ + cb;
             const uint32_t taddr = tmem_base + TMEM_ACC + buf * NQ + cb + lane_addr;
 #pragma unroll
@@ -260,10 +256,6 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
                     yy[6] = fmaf(__uint_as_float(v[i][6]), s1.z, yy[6]); yy[7] = fmaf(__uint_as_float(v[i][7]), s1.w, yy[7]);
                 }
             }
-            ptx::tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(&misc->acc_free[buf]);
-            return true;
         };
         int s = 0, kb = 0;
         uint32_t ph = 0;
@@ -287,11 +279,13 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
             }
             return true;
         };
-        for (int g = 0; g < n_groups && ok; ++g) {
-            ok = build_group();
-            if (ok && g >= 1) ok = fold_group(g - 1);
+        for (int g = 0; g < n_groups && ok; ++g) ok = build_group();
+        if (ok) ok = ptx::mbar_wait(&misc->acc_full, 0) && !misc->abort_flag;
+        if (ok) {
+            ptx::tc_fence_after_sync();
+            for (int g = 0; g < n_groups; ++g) fold_group(g);
+            ptx::tc_fence_before_sync();
         }
-        if (ok) ok = fold_group(n_groups - 1);
         if (!ok) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; }
         asm volatile("bar.sync 1, 256;" ::: "memory");       // all of phase 1 has been consumed: its shared memory is free
         ok = !misc->abort_flag;
@@ -444,7 +438,7 @@ EncodeTiledFn encode_tiled_fn2() {
 bool sm100_qattn_supported(const taq_layer_desc& d) {
     if (d.channels != KIN || d.heads * D != KIN) return false;
     if (d.w_bits != 4) return false;
-    if (d.w_group != 0 && d.w_group % BK) return false;
+    if (d.w_group != 0 && (d.w_group % BK || (KIN + d.w_group - 1) / d.w_group > MAX_GROUPS)) return false;
     if (d.n_ctx > TP || d.p_bits != 8) return false;
     if (d.n_query < 1) return false;
     return encode_tiled_fn2() != nullptr;
