@@ -5,10 +5,12 @@
 //            so the tensor core never waits for the workers, who fold the groups into registers at the end);
 //   phase 2  Q~ = Q_a(Q) (Eq. 2, third line) per (row, head) straight from those registers into the fp16-integer
 //            operand tiles of the four heads; the row scales stay in shared memory;
-//   phase 3  per head: S = Q~ K~^T, softmax, Eq. 3, O = A^ V~ as in taq_attention_sm100.cu (two threads per row,
-//            S of head h+1 under the softmax of head h), O stored as fp16.
-// Shared memory is used twice: the X tile and the weight ring of phase 1 become the Q~ tiles and the P tile.
-// Warps: 0 producer (TMA / bulk copies), 1 MMA issuer, 2..9 workers (two threads per row).
+//   phase 3  per head: S = Q~ K~^T, softmax, Eq. 3, O = A^ V~ as in taq_attention_sm100.cu.  The sixteen worker warps
+//            form two groups of eight (two threads per row each); group g takes heads g and g + 2, so that one
+//            group's exponentials overlap the other group's stores, exchanges and waits.  O is stored as fp16.
+// Shared memory is used twice: the X tile and the weight ring of phase 1 become the Q~ tiles and the two P tiles.
+// Warps: 0 producer (TMA / bulk copies), 1 MMA issuer, 2..17 workers (four threads per row: one head each in
+// phases 1 and 2, (group, key half) in phase 3).
 #include "taq_ptx.cuh"
 #include "taq_sm100.cuh"
 #include "taq_sm100_parts.cuh"
@@ -21,10 +23,10 @@ using namespace parts;
 
 constexpr int D = 40, DP = 48, HG = 4;          // head width, padded width, heads per CTA
 constexpr int NQ = HG * D;                      // 160 to_q channels per CTA
-constexpr int HC = NQ / 2;                      // channels per worker thread (two heads)
+constexpr int HC = D;                           // channels per worker thread in phases 1 and 2: one head
 constexpr int KIN = 320, BK = 64, NKB = KIN / BK;
 constexpr int ROWS = 128;
-constexpr int NWORK = 256, NTHREADS = 64 + NWORK;
+constexpr int NWORK = 512, NTHREADS = 64 + NWORK;
 constexpr int NBSTAGE = 3;                      // ring of expanded weight tiles
 
 constexpr int A_TILE = ROWS * 128;              // 16 KB: one 64-wide K block of X, or one head's Q~ tile, or half of P
@@ -39,28 +41,28 @@ constexpr int SCALE_BYTES = ((NQ * MAX_GROUPS * 4 + 127) / 128) * 128;
 constexpr int OFF_A = 0;                                    // phase 1: X tile, 5 K blocks
 constexpr int OFF_B = OFF_A + NKB * A_TILE;                 // phase 1: weight ring
 constexpr int OFF_Q = 0;                                    // phase 3: Q~ tiles of the four heads
-constexpr int OFF_P = OFF_Q + HG * A_TILE;                  // phase 3: probability tile (two K blocks)
+constexpr int OFF_P = OFF_Q + HG * A_TILE;                  // phase 3: one probability tile (two K blocks) per group
 constexpr int OFF_RAW = OFF_B + NBSTAGE * B_TILE;
 constexpr int OFF_SC = OFF_RAW + RAW_BYTES;
 constexpr int OFF_SCT = OFF_SC + SCALE_BYTES;
 constexpr int OFF_KV = ((OFF_SCT + SCALE_BYTES + 1023) / 1024) * 1024;
 constexpr int OFF_MISC = OFF_KV + 2 * HEAD_BYTES;
-static_assert(OFF_P + 2 * A_TILE <= OFF_RAW, "phase-3 tiles must fit into the phase-1 region");
+static_assert(OFF_P + 4 * A_TILE <= OFF_RAW, "phase-3 tiles must fit into the phase-1 region");
 
 struct Misc {
-    uint64_t a_full[NKB], b_full[NBSTAGE], b_empty[NBSTAGE], w_full, acc_full;
-    uint64_t q_all, kv_full[2], kv_free[2], s_full[2], p_full, o_full[2], drain;
+    uint64_t a_full[NKB], b_full[NBSTAGE], b_empty[NBSTAGE], w_full, acc_full[MAX_GROUPS];
+    uint64_t q_all, kv_full[2], kv_free[2], s_full[2], s_free[2], p_full[2], o_full[2], drain;
     uint32_t tmem_base;
     volatile int abort_flag;
     float sq[HG][ROWS];              // Q~ row scales
-    float2 xchg[2][2][ROWS];         // [head parity][half][row]
+    float2 xchg[2][2][2][ROWS];      // [iteration][group][half][row]
 };
 constexpr int TOTAL = OFF_MISC + (int)sizeof(Misc) + 1024;
 static_assert(TOTAL <= 232448, "shared memory budget");
 
 constexpr uint32_t TMEM_COLS = 512;
 constexpr uint32_t TMEM_ACC = 0;                 // phase 1: up to three accumulators of NQ columns
-constexpr uint32_t TMEM_S = 0, TMEM_O = 2 * TP;  // phase 3: S double-buffered, O double-buffered (reuses the columns)
+constexpr uint32_t TMEM_S = 0, TMEM_O = 2 * TP;  // phase 3: one S and one O accumulator per group (reuses the columns)
 
 struct QAttnArgs {
     const __half* x;            // [z][B][N][C]
@@ -95,15 +97,16 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
             ptx::mbar_init(&misc->b_empty[i], 1);
         }
         ptx::mbar_init(&misc->w_full, 1);
-        ptx::mbar_init(&misc->acc_full, 1);
+        for (int i = 0; i < MAX_GROUPS; ++i) ptx::mbar_init(&misc->acc_full[i], 1);
         for (int i = 0; i < 2; ++i) {
             ptx::mbar_init(&misc->kv_full[i], 1);
             ptx::mbar_init(&misc->kv_free[i], 1);
             ptx::mbar_init(&misc->s_full[i], 1);
+            ptx::mbar_init(&misc->s_free[i], NWORK / 64);     // one arrival per warp of the group
+            ptx::mbar_init(&misc->p_full[i], NWORK / 64);
             ptx::mbar_init(&misc->o_full[i], 1);
         }
         ptx::mbar_init(&misc->q_all, NWORK / 32);
-        ptx::mbar_init(&misc->p_full, NWORK / 32);
         ptx::mbar_init(&misc->drain, 1);
         misc->abort_flag = 0;
         ptx::mbar_fence_init();
@@ -171,40 +174,43 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
                         ptx::mma_commit(&misc->b_empty[s]);
                         if (++s == NBSTAGE) { s = 0; ph ^= 1; }
                     }
+                    if (ok) ptx::mma_commit(&misc->acc_full[buf]);
                 }
-                if (ok) ptx::mma_commit(&misc->acc_full);
             }
             // phase 3: the Q~ tiles of all four heads are in place once every worker warp has arrived
             if (ok && !ptx::mbar_wait(&misc->q_all, 0)) ok = false;
             const uint32_t q_addr = ptx::smem_u32(smem + OFF_Q), p_addr = ptx::smem_u32(smem + OFF_P);
-            auto issue_s = [&](int hi) -> bool {
-                const int buf = hi & 1;
-                if (!ptx::mbar_wait(&misc->kv_full[buf], (hi >> 1) & 1) || misc->abort_flag) return false;
+            // group g (heads g, g + 2) owns K~/V~ buffer g, S accumulator g, O accumulator g and P tile g
+            auto issue_s = [&](int g, int it) -> bool {
+                const int hi = g + 2 * it;
+                if (!ptx::mbar_wait(&misc->kv_full[g], it) || (it > 0 && !ptx::mbar_wait(&misc->s_free[g], it - 1)) || misc->abort_flag) return false;
                 ptx::tc_fence_after_sync();
-                const uint32_t k_addr = ptx::smem_u32(smem + OFF_KV + buf * HEAD_BYTES);
+                const uint32_t k_addr = ptx::smem_u32(smem + OFF_KV + g * HEAD_BYTES);
 #pragma unroll
                 for (int ks = 0; ks < DP / 16; ++ks)
-                    ptx::mma_f16_ss(tmem_base + TMEM_S + buf * TP, ptx::desc_k_sw128(q_addr + hi * A_TILE + ks * 32), ptx::desc_k_sw128(k_addr + ks * 32), ptx::idesc_f16_m128(TP), ks != 0);
-                ptx::mma_commit(&misc->s_full[buf]);
+                    ptx::mma_f16_ss(tmem_base + TMEM_S + g * TP, ptx::desc_k_sw128(q_addr + hi * A_TILE + ks * 32), ptx::desc_k_sw128(k_addr + ks * 32), ptx::idesc_f16_m128(TP), ks != 0);
+                ptx::mma_commit(&misc->s_full[g]);
                 return true;
             };
-            auto issue_pv = [&](int hi) -> bool {
-                const int buf = hi & 1;
-                if (!ptx::mbar_wait(&misc->p_full, hi & 1) || misc->abort_flag) return false;
+            auto issue_pv = [&](int g, int it) -> bool {
+                if (!ptx::mbar_wait(&misc->p_full[g], it) || misc->abort_flag) return false;     // (the group has emptied O before it arrives)
                 ptx::tc_fence_after_sync();
-                const uint32_t vt_addr = ptx::smem_u32(smem + OFF_KV + buf * HEAD_BYTES + K_BYTES);
+                const uint32_t vt_addr = ptx::smem_u32(smem + OFF_KV + g * HEAD_BYTES + K_BYTES);
+                const uint32_t pg_addr = p_addr + g * 2 * A_TILE;
 #pragma unroll
                 for (int ks = 0; ks < TP / 16; ++ks)
-                    ptx::mma_f16_ss(tmem_base + TMEM_O + buf * DP, ptx::desc_k_sw128(p_addr + (ks / 4) * A_TILE + (ks % 4) * 32),
+                    ptx::mma_f16_ss(tmem_base + TMEM_O + g * DP, ptx::desc_k_sw128(pg_addr + (ks / 4) * A_TILE + (ks % 4) * 32),
                                     ptx::desc_k_sw128(vt_addr + (ks / 4) * VT_BLOCK + (ks % 4) * 32), ptx::idesc_f16_m128(DP), ks != 0);
-                ptx::mma_commit(&misc->o_full[buf]);
-                ptx::mma_commit(&misc->kv_free[buf]);
+                ptx::mma_commit(&misc->o_full[g]);
+                ptx::mma_commit(&misc->kv_free[g]);
                 return true;
             };
-            if (ok) ok = issue_s(0);
-            for (int hi = 0; hi < HG && ok; ++hi) {
-                if (hi + 1 < HG) ok = issue_s(hi + 1);       // S of the next head runs under this head's softmax
-                if (ok) ok = issue_pv(hi);
+            if (ok) ok = issue_s(0, 0);
+            if (ok) ok = issue_s(1, 0);
+            for (int it = 0; it < 2 && ok; ++it) {
+                for (int g = 0; g < 2 && ok; ++g) ok = issue_pv(g, it);
+                if (it == 0)
+                    for (int g = 0; g < 2 && ok; ++g) ok = issue_s(g, 1);
             }
             if (!ok) {
                 raise_status(a.status, TAQ_ERR_TIMEOUT);
@@ -214,9 +220,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
             }
         }
     } else {
-        // ---------------- workers (warps 2..9): two threads per row ----------------
+        // ---------------- workers (warps 2..17): four threads per row ----------------
         const int wt = tid - 64;
-        const int q4 = warp & 3, half = (warp - 2) >> 2;
+        const int q4 = warp & 3, part = (warp - 2) >> 2;    // TMEM lane quarter; which head (phases 1, 2) / (group, half) (phase 3)
         const int r = q4 * 32 + lane;
         const int n = row0 + r;
         const bool valid = n < a.n_query;
@@ -227,122 +233,115 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
         float* scales_t = reinterpret_cast<float*>(smem + OFF_SCT);
         bool ok = ptx::mbar_wait(&misc->w_full, 0);
         for (int i = wt; i < NQ * n_groups; i += NWORK) scales_t[(i % n_groups) * NQ + i / n_groups] = wscales[i];
-        asm volatile("bar.sync 1, 256;" ::: "memory");
+        asm volatile("bar.sync 1, 512;" ::: "memory");
 
-        // ---- phase 1: expand weight tiles, fold finished groups: y = this thread's 80 channels (two heads) of its row ----
+        // ---- phase 1: expand weight tiles; fold each finished group: y = this thread's head (40 channels) of its row ----
         float y[HC];
 #pragma unroll
         for (int c = 0; c < HC; ++c) y[c] = 0.f;
-        const int cb = half * HC;
-        auto fold_group = [&](int g) {
-            const int buf = g;
-            const float* sg = scales_t + g * NQ + cb;
-            const uint32_t taddr = tmem_base + TMEM_ACC + buf * NQ + cb + lane_addr;
-#pragma unroll
-            for (int c0 = 0; c0 < HC; c0 += 40) {
-                uint32_t v[5][8];
-#pragma unroll
-                for (int i = 0; i < 5; ++i) ptx::tmem_ld8(taddr + c0 + i * 8, v[i]);
-                ptx::tmem_ld_wait(v[0]);
-#pragma unroll
-                for (int i = 1; i < 5; ++i) ptx::reg_fence8(v[i]);
-#pragma unroll
-                for (int i = 0; i < 5; ++i) {
-                    const float4 s0 = *reinterpret_cast<const float4*>(sg + c0 + i * 8), s1 = *reinterpret_cast<const float4*>(sg + c0 + i * 8 + 4);
-                    float* yy = y + c0 + i * 8;
-                    yy[0] = fmaf(__uint_as_float(v[i][0]), s0.x, yy[0]); yy[1] = fmaf(__uint_as_float(v[i][1]), s0.y, yy[1]);
-                    yy[2] = fmaf(__uint_as_float(v[i][2]), s0.z, yy[2]); yy[3] = fmaf(__uint_as_float(v[i][3]), s0.w, yy[3]);
-                    yy[4] = fmaf(__uint_as_float(v[i][4]), s1.x, yy[4]); yy[5] = fmaf(__uint_as_float(v[i][5]), s1.y, yy[5]);
-                    yy[6] = fmaf(__uint_as_float(v[i][6]), s1.z, yy[6]); yy[7] = fmaf(__uint_as_float(v[i][7]), s1.w, yy[7]);
-                }
-            }
-        };
-        int s = 0, kb = 0;
-        uint32_t ph = 0;
-        auto build_group = [&]() -> bool {
-            const int kb_end = min(NKB, kb + kb_per_group);
-            for (; kb < kb_end; ++kb) {
-                if (kb >= NBSTAGE && !ptx::mbar_wait(&misc->b_empty[s], ph ^ 1)) return false;
-                if (misc->abort_flag) return false;
+        const int cb = part * HC;
+        {
+            int s = 0;
+            uint32_t ph = 0;
+            for (int kb = 0; kb < NKB && ok; ++kb) {
+                if (kb >= NBSTAGE && !ptx::mbar_wait(&misc->b_empty[s], ph ^ 1)) ok = false;
+                if (!ok || misc->abort_flag) { ok = false; break; }
                 unsigned char* b_tile = smem + OFF_B + s * B_TILE;
-                constexpr int NCH = NQ * 8 / NWORK;         // 5 chunks of 8 weights per thread and K block
+                constexpr int NCH = (NQ * 8 + NWORK - 1) / NWORK;       // 16-byte chunks (8 weights) per thread and K block
                 const int n0 = wt >> 3, c = wt & 7;
                 uint32_t pw[NCH];
 #pragma unroll
-                for (int i = 0; i < NCH; ++i) pw[i] = *reinterpret_cast<const uint32_t*>(raw + (n0 + 32 * i) * (KIN / 2) + kb * (BK / 2) + c * 4);
+                for (int i = 0; i < NCH; ++i) {
+                    pw[i] = 0;
+                    if (n0 + (NWORK / 8) * i < NQ) pw[i] = *reinterpret_cast<const uint32_t*>(raw + (n0 + (NWORK / 8) * i) * (KIN / 2) + kb * (BK / 2) + c * 4);
+                }
 #pragma unroll
-                for (int i = 0; i < NCH; ++i) *reinterpret_cast<uint4*>(b_tile + ptx::sw128_offset(n0 + 32 * i, c)) = codes_w4_to_half(pw[i]);
+                for (int i = 0; i < NCH; ++i)
+                    if (n0 + (NWORK / 8) * i < NQ) *reinterpret_cast<uint4*>(b_tile + ptx::sw128_offset(n0 + (NWORK / 8) * i, c)) = codes_w4_to_half(pw[i]);
                 ptx::fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(&misc->b_full[s]);
                 if (++s == NBSTAGE) { s = 0; ph ^= 1; }
             }
-            return true;
-        };
-        for (int g = 0; g < n_groups && ok; ++g) ok = build_group();
-        if (ok) ok = ptx::mbar_wait(&misc->acc_full, 0) && !misc->abort_flag;
-        if (ok) {
-            ptx::tc_fence_after_sync();
-            for (int g = 0; g < n_groups; ++g) fold_group(g);
-            ptx::tc_fence_before_sync();
         }
+        for (int g = 0; g < n_groups && ok; ++g) {             // later groups are still being multiplied while this one is folded
+            ok = ptx::mbar_wait(&misc->acc_full[g], 0) && !misc->abort_flag;
+            if (!ok) break;
+            ptx::tc_fence_after_sync();
+            const float* sg = scales_t + g * NQ + cb;
+            const uint32_t taddr = tmem_base + TMEM_ACC + g * NQ + cb + lane_addr;
+            uint32_t v[5][8];
+#pragma unroll
+            for (int i = 0; i < 5; ++i) ptx::tmem_ld8(taddr + i * 8, v[i]);
+            ptx::tmem_ld_wait(v[0]);
+#pragma unroll
+            for (int i = 1; i < 5; ++i) ptx::reg_fence8(v[i]);
+#pragma unroll
+            for (int i = 0; i < 5; ++i) {
+                const float4 s0 = *reinterpret_cast<const float4*>(sg + i * 8), s1 = *reinterpret_cast<const float4*>(sg + i * 8 + 4);
+                float* yy = y + i * 8;
+                yy[0] = fmaf(__uint_as_float(v[i][0]), s0.x, yy[0]); yy[1] = fmaf(__uint_as_float(v[i][1]), s0.y, yy[1]);
+                yy[2] = fmaf(__uint_as_float(v[i][2]), s0.z, yy[2]); yy[3] = fmaf(__uint_as_float(v[i][3]), s0.w, yy[3]);
+                yy[4] = fmaf(__uint_as_float(v[i][4]), s1.x, yy[4]); yy[5] = fmaf(__uint_as_float(v[i][5]), s1.y, yy[5]);
+                yy[6] = fmaf(__uint_as_float(v[i][6]), s1.z, yy[6]); yy[7] = fmaf(__uint_as_float(v[i][7]), s1.w, yy[7]);
+            }
+        }
+        ptx::tc_fence_before_sync();
         if (!ok) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; }
-        asm volatile("bar.sync 1, 256;" ::: "memory");       // all of phase 1 has been consumed: its shared memory is free
+        asm volatile("bar.sync 1, 512;" ::: "memory");       // all of phase 1 has been consumed: its shared memory is free
         ok = !misc->abort_flag;
 
-        // ---- phase 2: Q~ = Q_a(Q) of this thread's two heads, written as fp16 integers into the heads' operand tiles ----
+        // ---- phase 2: Q~ = Q_a(Q) of this thread's head, written as fp16 integers into the head's operand tile ----
         if (ok) {
+            const int hi = part;
+            float amax = 0.f;
 #pragma unroll
-            for (int hh = 0; hh < 2; ++hh) {
-                const int hi = half * 2 + hh;
-                float amax = 0.f;
+            for (int c = 0; c < D; ++c) amax = fmaxf(amax, fabsf(y[c]));
+            unsigned char* q_tile = smem + OFF_Q + hi * A_TILE;
+            if (a.q_bits == 8) {
+                const float sc = quant_scale(amax, 127.f);
+                const float rs = sc > 0.f ? __frcp_rn(sc) : 0.f;
+                // fma(x, 1/s, 1.5 * 2^23 + 0x6480): the low half-word read as fp16 is 1152 + code
+                const __half2 h1152 = __floats2half2_rn(1152.f, 1152.f);
 #pragma unroll
-                for (int c = 0; c < D; ++c) amax = fmaxf(amax, fabsf(y[hh * D + c]));
-                unsigned char* q_tile = smem + OFF_Q + hi * A_TILE;
-                if (a.q_bits == 8) {
-                    const float sc = quant_scale(amax, 127.f);
-                    const float rs = sc > 0.f ? __frcp_rn(sc) : 0.f;
-                    // fma(x, 1/s, 1.5 * 2^23 + 0x6480): the low half-word read as fp16 is 1152 + code
-                    const __half2 h1152 = __floats2half2_rn(1152.f, 1152.f);
+                for (int cc = 0; cc < D / 8; ++cc) {
+                    uint32_t pk[4];
 #pragma unroll
-                    for (int cc = 0; cc < D / 8; ++cc) {
-                        uint32_t pk[4];
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const uint32_t x0 = __float_as_uint(fmaf(y[hh * D + cc * 8 + 2 * i], rs, 12608640.0f));
-                            const uint32_t x1 = __float_as_uint(fmaf(y[hh * D + cc * 8 + 2 * i + 1], rs, 12608640.0f));
-                            uint32_t w = __byte_perm(x0, x1, 0x5410);
-                            __half2 hv = __hsub2(*reinterpret_cast<__half2*>(&w), h1152);
-                            pk[i] = *reinterpret_cast<uint32_t*>(&hv);
-                        }
-                        *reinterpret_cast<uint4*>(q_tile + ptx::sw128_offset(r, cc)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    for (int i = 0; i < 4; ++i) {
+                        const uint32_t x0 = __float_as_uint(fmaf(y[cc * 8 + 2 * i], rs, 12608640.0f));
+                        const uint32_t x1 = __float_as_uint(fmaf(y[cc * 8 + 2 * i + 1], rs, 12608640.0f));
+                        uint32_t w = __byte_perm(x0, x1, 0x5410);
+                        __half2 hv = __hsub2(*reinterpret_cast<__half2*>(&w), h1152);
+                        pk[i] = *reinterpret_cast<uint32_t*>(&hv);
                     }
-                    misc->sq[hi][r] = valid ? sc : 0.f;
-                } else {                                    // Q stays fp16
-#pragma unroll
-                    for (int cc = 0; cc < D / 8; ++cc) {
-                        float f[8];
-#pragma unroll
-                        for (int e2 = 0; e2 < 8; ++e2) f[e2] = y[hh * D + cc * 8 + e2];
-                        *reinterpret_cast<uint4*>(q_tile + ptx::sw128_offset(r, cc)) = pack8(f);
-                    }
-                    misc->sq[hi][r] = 1.0f;
+                    *reinterpret_cast<uint4*>(q_tile + ptx::sw128_offset(r, cc)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                 }
-                *reinterpret_cast<uint4*>(q_tile + ptx::sw128_offset(r, D / 8)) = make_uint4(0, 0, 0, 0);   // channels 40..47
+                misc->sq[hi][r] = valid ? sc : 0.f;
+            } else {                                    // Q stays fp16
+#pragma unroll
+                for (int cc = 0; cc < D / 8; ++cc) {
+                    float f[8];
+#pragma unroll
+                    for (int e2 = 0; e2 < 8; ++e2) f[e2] = y[cc * 8 + e2];
+                    *reinterpret_cast<uint4*>(q_tile + ptx::sw128_offset(r, cc)) = pack8(f);
+                }
+                misc->sq[hi][r] = 1.0f;
             }
+            *reinterpret_cast<uint4*>(q_tile + ptx::sw128_offset(r, D / 8)) = make_uint4(0, 0, 0, 0);   // channels 40..47
             ptx::fence_proxy_async_smem();
         }
-        asm volatile("bar.sync 1, 256;" ::: "memory");       // the row scales of all heads are visible to both threads of a row
+        asm volatile("bar.sync 1, 512;" ::: "memory");       // the row scales of all heads are visible to every thread of the row
         if (lane == 0) ptx::mbar_arrive(&misc->q_all);
 
-        // ---- phase 3: attention over the four heads; this thread has keys [40 half, 40 half + 40) of its row ----
+        // ---- phase 3: group g = part / 2 takes heads g and g + 2; this thread has keys [40 half, 40 half + 40) of its row ----
+        const int grp = part >> 1, half = part & 1;
         const int key0 = half * HK;
         const float inv255 = 1.0f / 255.0f;
         constexpr int OC = DP / 2;
         bool alive = ok;
         auto store_o = [&](int hi) {
             __half* orow = a.o + grow * (size_t)(H * D) + (h_begin + hi) * D + half * OC;
-            const uint32_t t_o = tmem_base + TMEM_O + (hi & 1) * DP + half * OC + lane_addr;
+            const uint32_t t_o = tmem_base + TMEM_O + grp * DP + half * OC + lane_addr;
             uint32_t v[OC / 8][8];
 #pragma unroll
             for (int i = 0; i < OC / 8; ++i) ptx::tmem_ld8(t_o + i * 8, v[i]);
@@ -360,14 +359,14 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
             }
             ptx::tc_fence_before_sync();
         };
-        for (int hi = 0; hi < HG && alive; ++hi) {
-            const uint32_t ph2 = hi & 1;
-            alive = __all_sync(0xffffffffu, ptx::mbar_wait(&misc->s_full[ph2], (hi >> 1) & 1) && !misc->abort_flag);
+        for (int it = 0; it < 2 && alive; ++it) {
+            const int hi = grp + 2 * it;
+            alive = __all_sync(0xffffffffu, ptx::mbar_wait(&misc->s_full[grp], it) && !misc->abort_flag);
             if (!alive) break;
             ptx::tc_fence_after_sync();
             uint32_t u[HK];
             {
-                const uint32_t t_s = tmem_base + TMEM_S + ph2 * TP + key0 + lane_addr;
+                const uint32_t t_s = tmem_base + TMEM_S + grp * TP + key0 + lane_addr;
                 uint32_t (&u8)[HK / 8][8] = *reinterpret_cast<uint32_t (*)[HK / 8][8]>(&u);
 #pragma unroll
                 for (int i = 0; i < HK / 8; ++i) ptx::tmem_ld8(t_s + i * 8, u8[i]);
@@ -376,36 +375,38 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
                 for (int i = 1; i < HK / 8; ++i) ptx::reg_fence8(u8[i]);
             }
             ptx::tc_fence_before_sync();
-            const OperandConsts* cst = reinterpret_cast<const OperandConsts*>(smem + OFF_KV + ph2 * HEAD_BYTES + K_BYTES + VT_BYTES);
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&misc->s_free[grp]);      // the group's next S may overwrite the accumulator
+            const OperandConsts* cst = reinterpret_cast<const OperandConsts*>(smem + OFF_KV + grp * HEAD_BYTES + K_BYTES + VT_BYTES);
             const float sq = misc->sq[hi][r];
             float e[HK];
             float m_loc, l_loc;
             softmax_half<TAIL_ONLY>(u, cst->logit_factor + key0, sq, T, key0, e, m_loc, l_loc);
             const unsigned long long trig = half == 0 ? ((unsigned long long)cst->trig_bits[0] | ((unsigned long long)(cst->trig_bits[1] & 0xFFu) << 32))
                                                       : ((unsigned long long)(cst->trig_bits[1] >> 8) | ((unsigned long long)cst->trig_bits[2] << 24));
-            misc->xchg[ph2][half][r] = make_float2(m_loc, l_loc);
-            asm volatile("bar.sync %0, 64;" ::"r"(2 + q4) : "memory");
-            const float2 other = misc->xchg[ph2][half ^ 1][r];
+            misc->xchg[it][grp][half][r] = make_float2(m_loc, l_loc);
+            asm volatile("bar.sync %0, 64;" ::"r"(2 + grp * 4 + q4) : "memory");
+            const float2 other = misc->xchg[it][grp][half ^ 1][r];
             const float m_all = fmaxf(m_loc, other.x);
             const float c_self = ex2_approx(m_loc - m_all), c_other = ex2_approx(other.x - m_all);
             const float k255 = __fdividef(255.0f * c_self, fmaf(l_loc, c_self, other.y * c_other));
-            if (hi > 0) {       // the P tile is free once the previous head's PV has completed
-                alive = __all_sync(0xffffffffu, ptx::mbar_wait(&misc->o_full[(hi - 1) & 1], ((hi - 1) >> 1) & 1) && !misc->abort_flag);
+            if (it > 0) {       // the group's P tile and O accumulator are free once its previous PV is complete and O is stored
+                alive = __all_sync(0xffffffffu, ptx::mbar_wait(&misc->o_full[grp], 0) && !misc->abort_flag);
                 if (!alive) break;
                 ptx::tc_fence_after_sync();
+                store_o(hi - 2);
             }
-            write_p_half(e, k255, trig, smem + OFF_P, A_TILE, r, half * (HK / 8));
+            write_p_half(e, k255, trig, smem + OFF_P + grp * 2 * A_TILE, A_TILE, r, half * (HK / 8));
             ptx::fence_proxy_async_smem();
             ptx::tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(&misc->p_full);
-            if (hi > 0) store_o(hi - 1);                    // under this head's PV
+            if (lane == 0) ptx::mbar_arrive(&misc->p_full[grp]);
         }
         if (alive) {
-            alive = __all_sync(0xffffffffu, ptx::mbar_wait(&misc->o_full[(HG - 1) & 1], ((HG - 1) >> 1) & 1) && !misc->abort_flag);
+            alive = __all_sync(0xffffffffu, ptx::mbar_wait(&misc->o_full[grp], 1) && !misc->abort_flag);
             if (alive) {
                 ptx::tc_fence_after_sync();
-                store_o(HG - 1);
+                store_o(grp + 2);
             }
         }
         if (!alive) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; }
