@@ -41,7 +41,15 @@ def _newest_header() -> float:
     return max(os.path.getmtime(h) for h in hs)
 
 
-def build_library(force: bool = False, verbose: bool = False) -> str:
+def build_library(force: bool = False, verbose: bool = False, profile: bool = False) -> str:
+    """``profile=True`` builds ``libtaq_profile.so`` with the phase stamps of ``csrc/taq_prof.cuh`` compiled in
+    (into its own object directory); the normal library contains none of that code."""
+    if profile:
+        return _build(os.path.join(PKG, "_build_profile"), os.path.join(PKG, "libtaq_profile.so"), ["-DTAQ_PROFILE"], True, verbose)
+    return _build(BUILD, LIB, [], force, verbose)
+
+
+def _build(BUILD: str, LIB: str, extra: list, force: bool, verbose: bool) -> str:
     os.makedirs(BUILD, exist_ok=True)
     nvcc = _nvcc()
     hdr_time = _newest_header()
@@ -55,7 +63,7 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
 
     def compile_one(job):
         src, obj = job
-        cmd = [nvcc] + NVCC_FLAGS + ["-c", src, "-o", obj]
+        cmd = [nvcc] + NVCC_FLAGS + extra + ["-c", src, "-o", obj]
         p = subprocess.run(cmd, capture_output=True, text=True)
         log = os.path.join(BUILD, os.path.basename(src)[:-3] + ".log")
         with open(log, "w") as f:
@@ -78,4 +86,4 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
 
 
 if __name__ == "__main__":
-    print(build_library(force="--force" in sys.argv, verbose=True))
+    print(build_library(force="--force" in sys.argv, verbose=True, profile="--profile" in sys.argv))

@@ -19,6 +19,7 @@
 #include "taq_ptx.cuh"
 #include "taq_sm100.cuh"
 #include "taq_sm100_parts.cuh"
+#include "taq_prof.cuh"
 
 namespace taq {
 
@@ -98,6 +99,8 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
     const int n_groups = L.n_groups;
     const int kb_per_group = L.group_len / BK;             // k-blocks in a full group (the last group may be shorter)
 
+    TAQ_PROF_INIT
+    if (tid == 0) { TAQ_PROF(0); TAQ_GPROF(30); }
     if (tid == 0) {
         for (int s = 0; s < MAX_STAGE; ++s) {
             ptx::mbar_init(&bars->full_a[s], 1);
@@ -129,6 +132,7 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
             ptx::bulk_load(smem + P.off_scales, blob + L.off_scales + (size_t)col0 * n_groups * 4, (uint32_t)P.scale_bytes, &bars->w_full);
             ptx::bulk_load(smem + P.off_bias, blob + L.off_bias + (size_t)col0 * 4, (uint32_t)P.bias_bytes, &bars->w_full);
             if (a.early_weights) ptx::pdl_wait();         // the activations come from the previous kernel
+            TAQ_PROF(1); TAQ_GPROF(28);
             int issued = 0, s = 0;
             uint32_t ph = 0;                               // parity of the ring pass
             for (int kb = 0; kb < n_kb; ++kb) {
@@ -281,6 +285,7 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
         asm volatile("bar.sync 1, 256;" ::: "memory");       // every worker gets here; the decision below is uniform
         ok = !bars->abort_flag;
         ptx::pdl_wait();                                     // (already satisfied: the activations have arrived) orders the stores below
+        if (wt == 0) TAQ_PROF(7);
 
         // ---------------- epilogue on this thread's HC columns ----------------
         if (ok) {
@@ -411,6 +416,7 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
     // ---------------- teardown ----------------
     ptx::tc_fence_before_sync();
     __syncthreads();
+    if (tid == 0) { TAQ_PROF(9); TAQ_GPROF(29); }
     if (warp == 1) {
         ptx::tc_fence_after_sync();
         ptx::tmem_dealloc(tmem_base, TMEM_COLS);

@@ -14,6 +14,7 @@
 #include "taq_ptx.cuh"
 #include "taq_sm100.cuh"
 #include "taq_sm100_parts.cuh"
+#include "taq_prof.cuh"
 
 namespace taq {
 
@@ -90,6 +91,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
     const int n_groups = L.n_groups;
     const int kb_per_group = L.group_len / BK;
 
+    TAQ_PROF_INIT
+    if (tid == 0) { TAQ_PROF(0); TAQ_GPROF(30); }
     if (tid == 0) {
         for (int i = 0; i < NKB; ++i) ptx::mbar_init(&misc->a_full[i], 1);
         for (int i = 0; i < NBSTAGE; ++i) {
@@ -125,6 +128,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
         // ---------------- producer ----------------
         if (lane == 0) {
             ptx::pdl_wait();                              // X (and in general everything else) may come from the previous kernel
+            TAQ_PROF(1); TAQ_GPROF(28);
             const uint8_t* blob = (const uint8_t*)(a.reqs ? a.reqs[zb].Wq : a.wq);
             const uint32_t scale_bytes = (uint32_t)(NQ * n_groups * 4);
             ptx::mbar_arrive_expect_tx(&misc->w_full, RAW_BYTES + scale_bytes);
@@ -164,6 +168,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
                     const int kb_end = min(NKB, kb + kb_per_group);
                     for (bool first = true; kb < kb_end && ok; ++kb) {
                         if (!ptx::mbar_wait(&misc->a_full[kb], 0) || !ptx::mbar_wait(&misc->b_full[s], ph) || misc->abort_flag) { ok = false; break; }
+                        TAQ_PROF(2 + kb);
                         ptx::tc_fence_after_sync();
                         const uint32_t a_addr = ptx::smem_u32(smem + OFF_A + kb * A_TILE);
                         const uint32_t b_addr = ptx::smem_u32(smem + OFF_B + s * B_TILE);
@@ -288,6 +293,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
         }
         ptx::tc_fence_before_sync();
         if (!ok) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; }
+        if (wt == 0) TAQ_PROF(7);
         asm volatile("bar.sync 1, 512;" ::: "memory");       // all of phase 1 has been consumed: its shared memory is free
         ok = !misc->abort_flag;
 
@@ -332,6 +338,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
         }
         asm volatile("bar.sync 1, 512;" ::: "memory");       // the row scales of all heads are visible to every thread of the row
         if (lane == 0) ptx::mbar_arrive(&misc->q_all);
+        if (wt == 0) TAQ_PROF(8);
 
         // ---- phase 3: group g = part / 2 takes heads g and g + 2; this thread has keys [40 half, 40 half + 40) of its row ----
         const int grp = part >> 1, half = part & 1;
@@ -363,6 +370,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
             const int hi = grp + 2 * it;
             alive = __all_sync(0xffffffffu, ptx::mbar_wait(&misc->s_full[grp], it) && !misc->abort_flag);
             if (!alive) break;
+            if (lane == 0 && q4 == 0 && half == 0) TAQ_PROF(10 + 8 * grp + 4 * it);       // S seen
             ptx::tc_fence_after_sync();
             uint32_t u[HK];
             {
@@ -384,6 +392,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
             softmax_half<TAIL_ONLY>(u, cst->logit_factor + key0, sq, T, key0, e, m_loc, l_loc);
             const unsigned long long trig = half == 0 ? ((unsigned long long)cst->trig_bits[0] | ((unsigned long long)(cst->trig_bits[1] & 0xFFu) << 32))
                                                       : ((unsigned long long)(cst->trig_bits[1] >> 8) | ((unsigned long long)cst->trig_bits[2] << 24));
+            if (lane == 0 && q4 == 0 && half == 0) TAQ_PROF(11 + 8 * grp + 4 * it);       // exponentials done
             misc->xchg[it][grp][half][r] = make_float2(m_loc, l_loc);
             asm volatile("bar.sync %0, 64;" ::"r"(2 + grp * 4 + q4) : "memory");
             const float2 other = misc->xchg[it][grp][half ^ 1][r];
@@ -396,17 +405,20 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
                 ptx::tc_fence_after_sync();
                 store_o(hi - 2);
             }
+            if (lane == 0 && q4 == 0 && half == 0) TAQ_PROF(12 + 8 * grp + 4 * it);       // exchange (and previous O) done
             write_p_half(e, k255, trig, smem + OFF_P + grp * 2 * A_TILE, A_TILE, r, half * (HK / 8));
             ptx::fence_proxy_async_smem();
             ptx::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(&misc->p_full[grp]);
+            if (lane == 0 && q4 == 0 && half == 0) TAQ_PROF(13 + 8 * grp + 4 * it);       // P written
         }
         if (alive) {
             alive = __all_sync(0xffffffffu, ptx::mbar_wait(&misc->o_full[grp], 1) && !misc->abort_flag);
             if (alive) {
                 ptx::tc_fence_after_sync();
                 store_o(grp + 2);
+                if (lane == 0 && q4 == 0 && half == 0) TAQ_PROF(26 + grp);                 // last O stored
             }
         }
         if (!alive) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; }
@@ -414,6 +426,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
 
     ptx::tc_fence_before_sync();
     __syncthreads();
+    if (tid == 0) { TAQ_PROF(9); TAQ_GPROF(29); }
     if (warp == 1) {
         ptx::tc_fence_after_sync();
         ptx::tmem_dealloc(tmem_base, TMEM_COLS);
