@@ -6,11 +6,6 @@
 #include "taq_common.cuh"
 #include "taq_sm100.cuh"
 
-#ifdef TAQ_PROFILE
-namespace taq { __device__ unsigned long long* g_profile = nullptr; }
-extern "C" int taq_profile_set(unsigned long long* buf_dev) { return (int)cudaMemcpyToSymbol(taq::g_profile, &buf_dev, sizeof(buf_dev)); }
-#endif
-
 namespace taq {
 
 __device__ int g_status_word[2];   // {code, block id}; raised by kernels, read by taq_poll_device_status

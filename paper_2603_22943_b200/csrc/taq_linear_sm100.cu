@@ -21,6 +21,8 @@
 #include "taq_sm100_parts.cuh"
 #include "taq_prof.cuh"
 
+TAQ_PROF_DEFINE(linear)
+
 namespace taq {
 
 namespace {

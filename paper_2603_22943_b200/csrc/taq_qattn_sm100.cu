@@ -16,6 +16,8 @@
 #include "taq_sm100_parts.cuh"
 #include "taq_prof.cuh"
 
+TAQ_PROF_DEFINE(qattn)
+
 namespace taq {
 
 namespace {
@@ -43,20 +45,22 @@ constexpr int OFF_A = 0;                                    // phase 1: X tile, 
 constexpr int OFF_B = OFF_A + NKB * A_TILE;                 // phase 1: weight ring
 constexpr int OFF_Q = 0;                                    // phase 3: Q~ tiles of the four heads
 constexpr int OFF_P = OFF_Q + HG * A_TILE;                  // phase 3: one probability tile (two K blocks) per group
-constexpr int OFF_RAW = OFF_B + NBSTAGE * B_TILE;
+constexpr int OFF_RAW = OFF_B + NBSTAGE * B_TILE;            // phase 1: packed codes of the CTA's channels
+constexpr int OFF_XCHG = OFF_RAW;                           // phase 3: float2 [iteration][group][half][row], 8 KB
 constexpr int OFF_SC = OFF_RAW + RAW_BYTES;
 constexpr int OFF_SCT = OFF_SC + SCALE_BYTES;
-constexpr int OFF_KV = ((OFF_SCT + SCALE_BYTES + 1023) / 1024) * 1024;
-constexpr int OFF_MISC = OFF_KV + 2 * HEAD_BYTES;
+constexpr int OFF_K = ((OFF_SCT + SCALE_BYTES + 1023) / 1024) * 1024;    // K~ tiles, one buffer per group
+constexpr int OFF_VT = OFF_K + 2 * K_BYTES;                                // V~^T tiles, one buffer per group
+constexpr int OFF_CST = OFF_VT + 2 * VT_BYTES;                             // per-key constants of all four heads
+constexpr int OFF_MISC = OFF_CST + HG * kOperandConstBytes;
 static_assert(OFF_P + 4 * A_TILE <= OFF_RAW, "phase-3 tiles must fit into the phase-1 region");
 
 struct Misc {
     uint64_t a_full[NKB], b_full[NBSTAGE], b_empty[NBSTAGE], w_full, acc_full[MAX_GROUPS];
-    uint64_t q_all, kv_full[2], kv_free[2], s_full[2], s_free[2], p_full[2], o_full[2], drain;
+    uint64_t q_all, k_full[2], k_free[2], vt_full[2], vt_free[2], c_full, s_full[2], s_free[2], p_full[2], o_full[2], drain;
     uint32_t tmem_base;
     volatile int abort_flag;
     float sq[HG][ROWS];              // Q~ row scales
-    float2 xchg[2][2][2][ROWS];      // [iteration][group][half][row]
 };
 constexpr int TOTAL = OFF_MISC + (int)sizeof(Misc) + 1024;
 static_assert(TOTAL <= 232448, "shared memory budget");
@@ -102,13 +106,16 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
         ptx::mbar_init(&misc->w_full, 1);
         for (int i = 0; i < MAX_GROUPS; ++i) ptx::mbar_init(&misc->acc_full[i], 1);
         for (int i = 0; i < 2; ++i) {
-            ptx::mbar_init(&misc->kv_full[i], 1);
-            ptx::mbar_init(&misc->kv_free[i], 1);
+            ptx::mbar_init(&misc->k_full[i], 1);
+            ptx::mbar_init(&misc->k_free[i], 1);
+            ptx::mbar_init(&misc->vt_full[i], 1);
+            ptx::mbar_init(&misc->vt_free[i], 1);
             ptx::mbar_init(&misc->s_full[i], 1);
             ptx::mbar_init(&misc->s_free[i], NWORK / 64);     // one arrival per warp of the group
             ptx::mbar_init(&misc->p_full[i], NWORK / 64);
             ptx::mbar_init(&misc->o_full[i], 1);
         }
+        ptx::mbar_init(&misc->c_full, 1);
         ptx::mbar_init(&misc->q_all, NWORK / 32);
         ptx::mbar_init(&misc->drain, 1);
         misc->abort_flag = 0;
@@ -140,19 +147,38 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
             }
             const uint8_t* blk = a.reqs ? (const uint8_t*)a.reqs[zb].kv : (const uint8_t*)a.kv + (size_t)zb * KL.block_bytes;
             const uint8_t* img = blk + KL.off_operands + (size_t)h_begin * KL.operand_head_bytes;
-            int issued = 0;
-            for (int hi = 0; hi < HG; ++hi) {             // K~/V~ operand images, two buffers
-                const int buf = hi & 1;
-                if (hi >= 2 && !ptx::mbar_wait(&misc->kv_free[buf], ((hi >> 1) - 1) & 1)) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; }
-                if (misc->abort_flag) break;
-                ptx::mbar_arrive_expect_tx(&misc->kv_full[buf], HEAD_BYTES);
-                ptx::bulk_load(smem + OFF_KV + buf * HEAD_BYTES, img + (size_t)hi * KL.operand_head_bytes, HEAD_BYTES, &misc->kv_full[buf]);
-                issued = hi + 1;
+            // K~/V~ operand images: the constants of all four heads at once; K~ and V~^T tiles of head hi go to the
+            // buffers of group hi & 1.  A group's K~ buffer is free again as soon as its S has been computed, its V~^T
+            // buffer after its PV, so the second head's tiles arrive under the first head's softmax.
+            ptx::mbar_arrive_expect_tx(&misc->c_full, HG * kOperandConstBytes);
+            for (int hi = 0; hi < HG; ++hi)
+                ptx::bulk_load(smem + OFF_CST + hi * kOperandConstBytes, img + (size_t)hi * KL.operand_head_bytes + K_BYTES + VT_BYTES, kOperandConstBytes, &misc->c_full);
+            auto load_k = [&](int hi) {
+                ptx::mbar_arrive_expect_tx(&misc->k_full[hi & 1], K_BYTES);
+                ptx::bulk_load(smem + OFF_K + (hi & 1) * K_BYTES, img + (size_t)hi * KL.operand_head_bytes, K_BYTES, &misc->k_full[hi & 1]);
+            };
+            auto load_vt = [&](int hi) {
+                ptx::mbar_arrive_expect_tx(&misc->vt_full[hi & 1], VT_BYTES);
+                ptx::bulk_load(smem + OFF_VT + (hi & 1) * VT_BYTES, img + (size_t)hi * KL.operand_head_bytes + K_BYTES, VT_BYTES, &misc->vt_full[hi & 1]);
+            };
+            load_k(0); load_k(1); load_vt(0); load_vt(1);
+            int k_issued = 2, vt_issued = 2;
+            for (int g = 0; g < 2 && !misc->abort_flag; ++g) {
+                if (!ptx::mbar_wait(&misc->k_free[g], 0)) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; break; }
+                load_k(2 + g);
+                ++k_issued;
+            }
+            for (int g = 0; g < 2 && !misc->abort_flag; ++g) {
+                if (!ptx::mbar_wait(&misc->vt_free[g], 0)) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; break; }
+                load_vt(2 + g);
+                ++vt_issued;
             }
             if (misc->abort_flag) {   // give copies that are still in flight a bounded chance to land before the CTA exits
                 (void)ptx::mbar_wait(&misc->w_full, 0);
+                (void)ptx::mbar_wait(&misc->c_full, 0);
                 for (int kb = 0; kb < NKB; ++kb) (void)ptx::mbar_wait(&misc->a_full[kb], 0);
-                for (int hi = issued > 2 ? issued - 2 : 0; hi < issued; ++hi) (void)ptx::mbar_wait(&misc->kv_full[hi & 1], (hi >> 1) & 1);
+                for (int hi = k_issued - 2; hi < k_issued; ++hi) (void)ptx::mbar_wait(&misc->k_full[hi & 1], (hi >> 1) & 1);
+                for (int hi = vt_issued - 2; hi < vt_issued; ++hi) (void)ptx::mbar_wait(&misc->vt_full[hi & 1], (hi >> 1) & 1);
             }
         }
     } else if (warp == 1) {
@@ -188,35 +214,35 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
             // group g (heads g, g + 2) owns K~/V~ buffer g, S accumulator g, O accumulator g and P tile g
             auto issue_s = [&](int g, int it) -> bool {
                 const int hi = g + 2 * it;
-                if (!ptx::mbar_wait(&misc->kv_full[g], it) || (it > 0 && !ptx::mbar_wait(&misc->s_free[g], it - 1)) || misc->abort_flag) return false;
+                if (!ptx::mbar_wait(&misc->k_full[g], it) || (it > 0 && !ptx::mbar_wait(&misc->s_free[g], it - 1)) || misc->abort_flag) return false;
                 ptx::tc_fence_after_sync();
-                const uint32_t k_addr = ptx::smem_u32(smem + OFF_KV + g * HEAD_BYTES);
+                const uint32_t k_addr = ptx::smem_u32(smem + OFF_K + g * K_BYTES);
 #pragma unroll
                 for (int ks = 0; ks < DP / 16; ++ks)
                     ptx::mma_f16_ss(tmem_base + TMEM_S + g * TP, ptx::desc_k_sw128(q_addr + hi * A_TILE + ks * 32), ptx::desc_k_sw128(k_addr + ks * 32), ptx::idesc_f16_m128(TP), ks != 0);
                 ptx::mma_commit(&misc->s_full[g]);
+                ptx::mma_commit(&misc->k_free[g]);
                 return true;
             };
             auto issue_pv = [&](int g, int it) -> bool {
-                if (!ptx::mbar_wait(&misc->p_full[g], it) || misc->abort_flag) return false;     // (the group has emptied O before it arrives)
+                if (!ptx::mbar_wait(&misc->p_full[g], it) || !ptx::mbar_wait(&misc->vt_full[g], it) || misc->abort_flag) return false;     // (the group has emptied O before it arrives)
                 ptx::tc_fence_after_sync();
-                const uint32_t vt_addr = ptx::smem_u32(smem + OFF_KV + g * HEAD_BYTES + K_BYTES);
+                const uint32_t vt_addr = ptx::smem_u32(smem + OFF_VT + g * VT_BYTES);
                 const uint32_t pg_addr = p_addr + g * 2 * A_TILE;
 #pragma unroll
                 for (int ks = 0; ks < TP / 16; ++ks)
                     ptx::mma_f16_ss(tmem_base + TMEM_O + g * DP, ptx::desc_k_sw128(pg_addr + (ks / 4) * A_TILE + (ks % 4) * 32),
                                     ptx::desc_k_sw128(vt_addr + (ks / 4) * VT_BLOCK + (ks % 4) * 32), ptx::idesc_f16_m128(DP), ks != 0);
                 ptx::mma_commit(&misc->o_full[g]);
-                ptx::mma_commit(&misc->kv_free[g]);
+                ptx::mma_commit(&misc->vt_free[g]);
                 return true;
             };
-            if (ok) ok = issue_s(0, 0);
-            if (ok) ok = issue_s(1, 0);
-            for (int it = 0; it < 2 && ok; ++it) {
+            // S of a group's second head is issued as soon as its K~ tile has arrived and the group holds the first
+            // head's scores in registers, i.e. under the first head's softmax
+            for (int it = 0; it < 2 && ok; ++it)
+                for (int g = 0; g < 2 && ok; ++g) ok = issue_s(g, it);
+            for (int it = 0; it < 2 && ok; ++it)
                 for (int g = 0; g < 2 && ok; ++g) ok = issue_pv(g, it);
-                if (it == 0)
-                    for (int g = 0; g < 2 && ok; ++g) ok = issue_s(g, 1);
-            }
             if (!ok) {
                 raise_status(a.status, TAQ_ERR_TIMEOUT);
                 misc->abort_flag = 1;
@@ -294,8 +320,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
         ptx::tc_fence_before_sync();
         if (!ok) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; }
         if (wt == 0) TAQ_PROF(7);
-        asm volatile("bar.sync 1, 512;" ::: "memory");       // all of phase 1 has been consumed: its shared memory is free
-        ok = !misc->abort_flag;
+        // The last group's accumulator is complete, hence every MMA of phase 1 has finished reading shared memory and
+        // every weight tile has been built: the phase-1 region may be overwritten without a barrier.
 
         // ---- phase 2: Q~ = Q_a(Q) of this thread's head, written as fp16 integers into the head's operand tile ----
         if (ok) {
@@ -337,7 +363,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
             ptx::fence_proxy_async_smem();
         }
         asm volatile("bar.sync 1, 512;" ::: "memory");       // the row scales of all heads are visible to every thread of the row
+        ok = !misc->abort_flag;
         if (lane == 0) ptx::mbar_arrive(&misc->q_all);
+        if (ok && !ptx::mbar_wait(&misc->c_full, 0)) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; ok = false; }
         if (wt == 0) TAQ_PROF(8);
 
         // ---- phase 3: group g = part / 2 takes heads g and g + 2; this thread has keys [40 half, 40 half + 40) of its row ----
@@ -385,7 +413,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
             ptx::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(&misc->s_free[grp]);      // the group's next S may overwrite the accumulator
-            const OperandConsts* cst = reinterpret_cast<const OperandConsts*>(smem + OFF_KV + grp * HEAD_BYTES + K_BYTES + VT_BYTES);
+            const OperandConsts* cst = reinterpret_cast<const OperandConsts*>(smem + OFF_CST + hi * kOperandConstBytes);
             const float sq = misc->sq[hi][r];
             float e[HK];
             float m_loc, l_loc;
@@ -393,9 +421,10 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
             const unsigned long long trig = half == 0 ? ((unsigned long long)cst->trig_bits[0] | ((unsigned long long)(cst->trig_bits[1] & 0xFFu) << 32))
                                                       : ((unsigned long long)(cst->trig_bits[1] >> 8) | ((unsigned long long)cst->trig_bits[2] << 24));
             if (lane == 0 && q4 == 0 && half == 0) TAQ_PROF(11 + 8 * grp + 4 * it);       // exponentials done
-            misc->xchg[it][grp][half][r] = make_float2(m_loc, l_loc);
+            float2* xchg = reinterpret_cast<float2*>(smem + OFF_XCHG) + (size_t)((it * 2 + grp) * 2) * ROWS;     // [half][row] of this head
+            xchg[half * ROWS + r] = make_float2(m_loc, l_loc);
             asm volatile("bar.sync %0, 64;" ::"r"(2 + grp * 4 + q4) : "memory");
-            const float2 other = misc->xchg[it][grp][half ^ 1][r];
+            const float2 other = xchg[(half ^ 1) * ROWS + r];
             const float m_all = fmaxf(m_loc, other.x);
             const float c_self = ex2_approx(m_loc - m_all), c_other = ex2_approx(other.x - m_all);
             const float k255 = __fdividef(255.0f * c_self, fmaf(l_loc, c_self, other.y * c_other));
