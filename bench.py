@@ -27,6 +27,9 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 METRIC = "TAQ cross-attn queries/s per layer"
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/ (bytes); a
+# kernel that changed since its capture is listed as None.
+TRAFFIC = {"qattn": None, "to_out": None}
 UNIT = "queries/s"
 WORKLOAD = "config2: SD-1.5 64x64 cross-attn layer, B=2 N=4096 C=320 H=8 d=40 T=77 Dc=768, W4 g128, int8 Q/K/V rows, uint8 probs, fp16 trigger rows {4,5}"
 
@@ -247,12 +250,18 @@ def main():
     barrier()
     ms_total = e0.elapsed_time(e1)
 
-    # Per-kernel attribution: each stage through its own entry point, one graph of n_sets back-to-back launches of
-    # that stage over the buffer ring (so every launch streams its inputs from HBM), CUDA events around the graph.
+    # Per-kernel attribution: each kernel of the step through its own entry point, one graph of n_sets back-to-back
+    # launches of that stage over the buffer ring (so every launch streams its inputs from HBM), CUDA events around the
+    # graph.  A step is two launches: the fused to_q + Q_a + attention kernel and the to_out dequant-GEMM.  The three
+    # stand-alone entry points (to_q, attention, to_out as separate kernels) are timed the same way for comparison.
     q_c = torch.empty((M, C_), dtype=torch.int8 if shape.q_bits == 8 else torch.float16, device="cuda")
     q_s = torch.empty((M, H), dtype=torch.float32, device="cuda")
     o_sets = [torch.empty((B, N, C_), dtype=torch.float16, device="cuda") for _ in range(n_sets)]
     q_sets = [(torch.empty_like(q_c), torch.empty_like(q_s)) for _ in range(n_sets)]
+
+    def stage_qattn(i):
+        s = sets[i % n_sets]
+        tb.taq_query_attention(desc, s["x"], s["Wq"], s["kv"], mask, o_sets[i % n_sets], s["ws"])
 
     def stage_q(i):
         s = sets[i % n_sets]
@@ -271,13 +280,13 @@ def main():
         s = sets[i % n_sets]
         tb.taq_quantized_linear(wd_cc, o_sets[i % n_sets], s["Wout"], tb.TAQ_OUT_F16, y=s["y"])
 
-    stage_ms = []
-    for fn in (stage_q, stage_attn, stage_out):
+    stage_ms = {}
+    for name, fn in (("qattn", stage_qattn), ("to_q", stage_q), ("attn", stage_attn), ("to_out", stage_out)):
         for i in range(n_sets):
             fn(i)
         torch.cuda.synchronize()
         g = capture(fn, n_sets)
-        stage_ms.append(time_graph(g, replays=max(1, min(args.steps, 200) // n_sets)) / n_sets)
+        stage_ms[name] = time_graph(g, replays=max(1, min(args.steps, 200) // n_sets)) / n_sets
     clocks = sampler.stop()
 
     # End to end through the same call with host buffers: H2D of X and D2H of Y inside the timed region.
@@ -319,29 +328,36 @@ def main():
     kv_block = tb.taq_kv_layout_of(desc).block_bytes * B
     wbytes = tb.taq_packed_weight_bytes(wd_cc)
     qbytes = M * C_ * (1 if shape.q_bits == 8 else 2) + (M * H * 4 if shape.q_bits == 8 else 0)
+    img_bytes = tb.taq_kv_layout_of(desc).operand_head_bytes * H * B
     kernels = [
-        {"name": "to_q dequant-GEMM + Q_a epilogue", "ms": stage_ms[0], "bytes": M * C_ * 2 + qbytes + wbytes, "flops": 2 * M * C_ * C_},
-        {"name": "fused TAQ attention", "ms": stage_ms[1], "bytes": qbytes + M * C_ * 2 + kv_block, "flops": 4 * M * T * C_},
-        {"name": "to_out dequant-GEMM", "ms": stage_ms[2], "bytes": 2 * M * C_ * 2 + wbytes, "flops": 2 * M * C_ * C_},
+        {"name": "qattn_c320_kernel: to_q + Q_a + attention, one kernel (taq_query_attention)", "ms": stage_ms["qattn"], "in_step": True,
+         "bytes": 2 * M * C_ * 2 + wbytes + img_bytes, "flops": 2 * M * C_ * C_ + 4 * M * T * C_, "traffic": TRAFFIC.get("qattn")},
+        {"name": "linear_sm100_kernel<160>: to_out dequant-GEMM (taq_quantized_linear)", "ms": stage_ms["to_out"], "in_step": True,
+         "bytes": 2 * M * C_ * 2 + wbytes, "flops": 2 * M * C_ * C_, "traffic": TRAFFIC.get("to_out")},
+        {"name": "linear_sm100_kernel<160>: to_q dequant-GEMM + Q_a epilogue, stand-alone", "ms": stage_ms["to_q"], "in_step": False,
+         "bytes": M * C_ * 2 + qbytes + wbytes, "flops": 2 * M * C_ * C_, "traffic": None},
+        {"name": "attention_sm100_kernel<40>: attention, stand-alone (taq_cross_attention)", "ms": stage_ms["attn"], "in_step": False,
+         "bytes": qbytes + M * C_ * 2 + img_bytes, "flops": 4 * M * T * C_, "traffic": None},
     ]
     for k in kernels:
         k["GB/s"] = k["bytes"] / (k["ms"] * 1e-3) / 1e9
         k["TFLOP/s"] = k["flops"] / (k["ms"] * 1e-3) / 1e12
-    dom = max(kernels, key=lambda k: k["ms"])
+    dom = max((k for k in kernels if k["in_step"]), key=lambda k: k["ms"])
     roofline = {"kernel": dom["name"], "bound": "hbm", "achieved": dom["GB/s"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": dom["GB/s"] / peaks["hbm_gbs"], "peak_source": peaks["source"], "traffic": None,
+                "frac": dom["GB/s"] / peaks["hbm_gbs"], "peak_source": peaks["source"] + " (burst copy figure; of measured)", "traffic": dom["traffic"],
                 "bytes_per_launch": dom["bytes"], "ms_per_launch": dom["ms"],
-                "stages": [{"name": k["name"], "ms": round(k["ms"], 5), "GB/s": round(k["GB/s"], 1), "TFLOP/s": round(k["TFLOP/s"], 2)} for k in kernels]}
+                "tensor": {"achieved_tflops": dom["TFLOP/s"], "peak_tflops": peaks["bf16_tflops"], "frac": dom["TFLOP/s"] / peaks["bf16_tflops"]},
+                "stages": [{"name": k["name"], "in_step": k["in_step"], "ms": round(k["ms"], 5), "GB/s": round(k["GB/s"], 1), "TFLOP/s": round(k["TFLOP/s"], 2)} for k in kernels]}
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f16",
             "data": "synthetic",
             "config": {"workload": WORKLOAD if not args.n_query else WORKLOAD + f" (N overridden to {N})", "kv_projection": "once per prompt, outside the step",
-                       "launch": "the K timed steps are one CUDA graph (3 kernel launches per step)",
+                       "launch": "the K timed steps are one CUDA graph (2 kernel launches per step: fused to_q+attention, to_out)",
                        "l2_policy": f"inputs larger than L2: ring of {n_sets} buffer sets ({n_sets * set_bytes / 1e6:.0f} MB of activations, L2 {l2 / 1e6:.0f} MB)",
                        "replicas": world},
             "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": M * C_ * 2, "d2h_bytes_per_step": M * C_ * 2, "steps": e_steps},
-            "gpu_launches": 3 * args.steps,
+            "gpu_launches": 2 * args.steps,
             "roofline": roofline}
     if not args.no_cpu_baseline:
         secs, rows = time_oracle(shape, data, args.cpu_rows)

@@ -176,6 +176,14 @@ taq_status taq_cross_attention(const taq_layer_desc* desc, const void* q_dev, co
                                const void* kv_packed_dev, const uint8_t* trig_mask_dev, void* o_f16_dev,
                                void* stream);
 
+/* to_q, Q~ = Q_a(Q) and the attention core in one call: x fp16 [B][N][C] -> O fp16 [B][N][C] (the input of to_out).
+ * For the SD-1.5 64x64 shape (C = 320, 8 heads of 40, W4) this is a single kernel in which Q~ never leaves the SM
+ * (Eq. 2 third line, Sec. III-B first paragraph, Eq. 3); other shapes run taq_quantized_linear's and
+ * taq_cross_attention's kernels back to back with Q~ in the workspace.  Arguments as for taq_layer_forward. */
+taq_status taq_query_attention(const taq_layer_desc* desc, const void* x_f16_dev, const void* Wq_packed_dev,
+                               const void* kv_packed_dev, const uint8_t* trig_mask_dev, void* o_f16_dev,
+                               void* workspace_dev, size_t workspace_bytes, void* stream);
+
 /* One denoising-step pass of the layer, K~/V~ already projected: to_q (+ Q_a), attention, to_out (+ bias).
  *   x_f16_dev fp16 [B][N][C] -> y_f16_dev fp16 [B][N][C];  Wq/Wout blobs of shape [C][C]
  *   workspace_dev >= taq_workspace_bytes(desc, 1), 128-byte aligned; contents are scratch. */

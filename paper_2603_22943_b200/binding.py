@@ -24,7 +24,7 @@ EXPORTS = [
     "taq_unpack_weights", "taq_quantize_rows", "taq_kv_layout_of", "taq_kv_bytes", "taq_kv_project",
     "taq_quantized_linear", "taq_cross_attention", "taq_workspace_bytes", "taq_layer_forward",
     "taq_layer_forward_batched", "taq_kv_project_batched", "taq_poll_device_status",
-    "taq_static_workspace_capacity", "taq_layer_forward_static", "taq_kv_finalize",
+    "taq_static_workspace_capacity", "taq_layer_forward_static", "taq_kv_finalize", "taq_query_attention",
 ]
 
 
@@ -89,6 +89,7 @@ def lib() -> C.CDLL:
         L.taq_workspace_bytes.restype = sz
         L.taq_workspace_bytes.argtypes = [C.POINTER(LayerDesc), i32]
         L.taq_layer_forward.argtypes = [C.POINTER(LayerDesc), vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.taq_query_attention.argtypes = [C.POINTER(LayerDesc), vp, vp, vp, vp, vp, vp, sz, vp]
         L.taq_layer_forward_batched.argtypes = [C.POINTER(LayerDesc), vp, i32, vp, vp, vp, sz, vp]
         L.taq_kv_project_batched.argtypes = [C.POINTER(LayerDesc), vp, i32, vp, vp]
         L.taq_poll_device_status.argtypes = [vp, C.POINTER(i32)]
@@ -230,6 +231,18 @@ def taq_layer_forward(desc: LayerDesc, x: torch.Tensor, Wq_packed: torch.Tensor,
     _check(lib().taq_layer_forward(C.byref(desc), _ptr(x), _ptr(Wq_packed), _ptr(Wout_packed), _ptr(kv), _ptr(trig_mask), _ptr(y),
                                    _ptr(workspace), workspace.numel(), _stream(stream)))
     return y
+
+
+def taq_query_attention(desc: LayerDesc, x: torch.Tensor, Wq_packed: torch.Tensor, kv: torch.Tensor, trig_mask: torch.Tensor,
+                        o: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """x -> O (to_q, Q_a, attention); one fused kernel for C = 320 / 8 heads / W4."""
+    if o is None:
+        o = torch.empty((desc.batch, desc.n_query, desc.channels), dtype=torch.float16, device=x.device)
+    if workspace is None:
+        workspace = torch.empty(max(taq_workspace_bytes(desc, 1), 128), dtype=torch.uint8, device=x.device)
+    _check(lib().taq_query_attention(C.byref(desc), _ptr(x), _ptr(Wq_packed), _ptr(kv), _ptr(trig_mask), _ptr(o), _ptr(workspace),
+                                     workspace.numel(), _stream(stream)))
+    return o
 
 
 def taq_static_workspace_capacity() -> int:

@@ -310,19 +310,16 @@ size_t taq_workspace_bytes(const taq_layer_desc* d, int32_t n_requests) {
     return workspace_layout(d, n_requests).total;
 }
 
-static taq_status layer_forward_impl(const taq_layer_desc* d, const taq_request* reqs, int n_req, const void* x, const void* Wq,
-                                     const void* Wout, const void* kv, const uint8_t* mask, void* y, void* ws, cudaStream_t st) {
-    int* status = nullptr;
-    taq_status s = status_ptr(&status);
-    if (s != TAQ_OK) return s;
+// x -> O: to_q, Q~ = Q_a(Q), attention.  One kernel where the fused kernel covers the shape, otherwise two with Q~
+// in the workspace.
+static taq_status q_attention_impl(const taq_layer_desc* d, const taq_request* reqs, int n_req, const void* x, const void* Wq, const void* kv,
+                                   const uint8_t* mask, void* o_dst, void* ws, int* status, cudaStream_t st) {
     const Workspace W = workspace_layout(d, n_req);
     uint8_t* wsb = (uint8_t*)ws;
     const long long rows_per_z = (long long)d->batch * d->n_query;   // weights are shared by the whole batch
-
-    bool fused = sm100_qattn_supported(*d);
-    if (fused) {                                                        // to_q, Q_a and the attention in one kernel
-        cudaError_t e = launch_qattn_sm100(*d, (const __half*)x, Wq, kv, reqs, (__half*)(wsb + W.off_o), reqs ? n_req : d->batch, status, st);
-        if (e != cudaSuccess) return cuda_fail(e, "fused to_q + attention launch");
+    if (sm100_qattn_supported(*d)) {
+        cudaError_t e = launch_qattn_sm100(*d, (const __half*)x, Wq, kv, reqs, (__half*)o_dst, reqs ? n_req : d->batch, status, st);
+        return e == cudaSuccess ? TAQ_OK : cuda_fail(e, "fused to_q + attention launch");
     }
     LinearArgs q{};                                                     // to_q (+ Q~ = Q_a(Q))
     q.x = (const __half*)x; q.w = Wq; q.reqs = reqs; q.which = 0;
@@ -331,24 +328,30 @@ static taq_status layer_forward_impl(const taq_layer_desc* d, const taq_request*
     q.heads = d->q_bits == 8 ? d->heads : 1;
     q.epi = d->q_bits == 8 ? EPI_Q8_HEAD : EPI_F16;
     q.status = status;
-    if (!fused) {
-        s = run_linear(q, n_req, st);
-        if (s != TAQ_OK) return s;
-    }
+    taq_status s = run_linear(q, n_req, st);
+    if (s != TAQ_OK) return s;
 
     AttnArgs at = attn_args(d, status);                                 // softmax(Q~K~^T/sqrt(d)), Eq. 3, P.V
     at.q = wsb + W.off_q; at.q_scales = (const float*)(wsb + W.off_qs); at.kv = kv; at.mask = mask; at.reqs = reqs;
-    at.o = (__half*)(wsb + W.off_o);
+    at.o = (__half*)o_dst;
     at.early_kv = 1;            // the kernel before it in the stream is to_q above, which writes the workspace only
-    if (!fused) {
-        s = run_attention(at, reqs ? n_req : d->batch, st);
-        if (s != TAQ_OK) return s;
-    }
+    return run_attention(at, reqs ? n_req : d->batch, st);
+}
+
+static taq_status layer_forward_impl(const taq_layer_desc* d, const taq_request* reqs, int n_req, const void* x, const void* Wq,
+                                     const void* Wout, const void* kv, const uint8_t* mask, void* y, void* ws, cudaStream_t st) {
+    int* status = nullptr;
+    taq_status s = status_ptr(&status);
+    if (s != TAQ_OK) return s;
+    const Workspace W = workspace_layout(d, n_req);
+    uint8_t* wsb = (uint8_t*)ws;
+    s = q_attention_impl(d, reqs, n_req, x, Wq, kv, mask, wsb + W.off_o, ws, status, st);
+    if (s != TAQ_OK) return s;
 
     LinearArgs o{};                                                     // to_out (+ bias)
     o.x = (const __half*)(wsb + W.off_o); o.w = Wout; o.reqs = reqs; o.which = 1;
     o.y = y;
-    o.rows = rows_per_z; o.n_out = d->channels; o.k_in = d->channels; o.bits = d->w_bits; o.group = d->w_group;
+    o.rows = (long long)d->batch * d->n_query; o.n_out = d->channels; o.k_in = d->channels; o.bits = d->w_bits; o.group = d->w_group;
     o.heads = 1; o.epi = EPI_F16; o.status = status;
     o.early_weights = 1;        // the kernel before it in the stream is the attention above, which writes O only
     return run_linear(o, n_req, st);
@@ -373,6 +376,27 @@ taq_status taq_layer_forward(const taq_layer_desc* d, const void* x_f16_dev, con
     if (workspace_bytes < need) return fail(TAQ_ERR_BUFFER_TOO_SMALL, "workspace has %zu bytes, %zu needed", workspace_bytes, need);
     return layer_forward_impl(d, nullptr, 1, x_f16_dev, Wq_packed_dev, Wout_packed_dev, kv_packed_dev, trig_mask_dev, y_f16_dev,
                               workspace_dev, (cudaStream_t)stream);
+}
+
+taq_status taq_query_attention(const taq_layer_desc* d, const void* x_f16_dev, const void* Wq_packed_dev, const void* kv_packed_dev,
+                               const uint8_t* trig_mask_dev, void* o_f16_dev, void* workspace_dev, size_t workspace_bytes, void* stream) {
+    taq_status s = check_layer_desc(d);
+    if (s != TAQ_OK) return s;
+    if (d->batch > 65535) return fail(TAQ_ERR_SHAPE, "batch must be at most 65535");
+    if (d->batch == 0 || d->n_query == 0) return TAQ_OK;
+    TAQ_REQUIRE_PTR(x_f16_dev);
+    TAQ_REQUIRE_PTR(Wq_packed_dev);
+    TAQ_REQUIRE_PTR(kv_packed_dev);
+    TAQ_REQUIRE_PTR(o_f16_dev);
+    TAQ_REQUIRE_PTR(workspace_dev);
+    if (!trig_mask_dev) return fail(TAQ_ERR_INVALID_ARG, "trig_mask_dev is NULL");
+    if (reinterpret_cast<uintptr_t>(workspace_dev) & 127u) return fail(TAQ_ERR_ALIGNMENT, "workspace_dev is not 128-byte aligned");
+    const size_t need = taq_workspace_bytes(d, 1);
+    if (workspace_bytes < need) return fail(TAQ_ERR_BUFFER_TOO_SMALL, "workspace has %zu bytes, %zu needed", workspace_bytes, need);
+    int* status = nullptr;
+    s = status_ptr(&status);
+    if (s != TAQ_OK) return s;
+    return q_attention_impl(d, nullptr, 1, x_f16_dev, Wq_packed_dev, kv_packed_dev, trig_mask_dev, o_f16_dev, workspace_dev, status, (cudaStream_t)stream);
 }
 
 taq_status taq_layer_forward_batched(const taq_layer_desc* d, const taq_request* reqs_dev, int32_t n_requests, const void* x_f16_dev,

@@ -153,6 +153,37 @@ def _layer_case(shape, sample_rows=None, max_trigger=None):
     return tl.check_layer(shape, data, y, parts, rows)
 
 
+@pytest.mark.parametrize("shape_fn,n", [(synth.config2, 4096), (synth.config2, 333), (lambda: synth.config3_layers()[5], 200)],
+                         ids=["config2_full", "config2_ragged", "C640_unfused"])
+@pytest.mark.parametrize("q_bits", [8, 0])
+def test_query_attention_equals_the_two_step_path(shape_fn, n, q_bits):
+    """taq_query_attention (one fused kernel at C = 320) against taq_quantized_linear + taq_cross_attention on the same
+    inputs: the same arithmetic in the same order, hence bit-identical O; and against the oracle's O on sampled rows."""
+    from dataclasses import replace
+    shape = replace(_small(shape_fn(), n), q_bits=q_bits)
+    data = synth.make_layer(shape)
+    desc = tl.gpu_desc(shape)
+    P = tl.pack_layer_weights(shape, data)
+    mask = dev(data["mask"])
+    kv = tb.taq_kv_project(desc, dev(data["ctx"]), P["Wk"], P["Wv"], mask)
+    x = dev(data["X"])
+    o_fused = tb.taq_query_attention(desc, x, P["Wq"], kv, mask)
+    x2 = x.reshape(-1, shape.channels)
+    if q_bits == 8:
+        qc, qs = tb.taq_quantized_linear(P["wd_cc"], x2, P["Wq"], tb.TAQ_OUT_INT8_HEAD_ROWS, heads=shape.heads)
+        o_two = tb.taq_cross_attention(desc, qc, qs, kv, mask)
+    else:
+        q16 = tb.taq_quantized_linear(P["wd_cc"], x2, P["Wq"], tb.TAQ_OUT_F16)
+        o_two = tb.taq_cross_attention(desc, q16, None, kv, mask)
+    tb.taq_poll_device_status()
+    assert torch.equal(o_fused.view(torch.int16), o_two.view(torch.int16))
+    rows = np.arange(0, shape.n_query, max(1, shape.n_query // 64))
+    cfg = tl.oracle_cfg(shape)
+    g = tl.gpu_decisions(shape, data, {"desc": desc, "packed": P, "kv": kv, "mask": mask}, rows)
+    want = orc.taq_attention(g["Q_tilde"], g["K_tilde"], g["V_tilde"], data["mask"], cfg)
+    tl.assert_layer_close(o_fused.cpu().numpy()[:, rows], want, shape.name + " O (same decisions)")
+
+
 def test_layer_config1_full():
     _layer_case(synth.config1())
 
