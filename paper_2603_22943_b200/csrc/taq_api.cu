@@ -343,6 +343,10 @@ static taq_status layer_forward_impl(const taq_layer_desc* d, const taq_request*
     int* status = nullptr;
     taq_status s = status_ptr(&status);
     if (s != TAQ_OK) return s;
+    if (sm100_layer_supported(*d)) {                                    // the whole pass in one kernel
+        cudaError_t e = launch_layer_sm100(*d, (const __half*)x, Wq, Wout, kv, reqs, (__half*)y, reqs ? n_req : d->batch, status, st);
+        return e == cudaSuccess ? TAQ_OK : cuda_fail(e, "fused layer launch");
+    }
     const Workspace W = workspace_layout(d, n_req);
     uint8_t* wsb = (uint8_t*)ws;
     s = q_attention_impl(d, reqs, n_req, x, Wq, kv, mask, wsb + W.off_o, ws, status, st);

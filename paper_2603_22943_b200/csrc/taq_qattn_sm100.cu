@@ -8,6 +8,10 @@
 //   phase 3  per head: S = Q~ K~^T, softmax, Eq. 3, O = A^ V~ as in taq_attention_sm100.cu.  The sixteen worker warps
 //            form two groups of eight (two threads per row each); group g takes heads g and g + 2, so that one
 //            group's exponentials overlap the other group's stores, exchanges and waits.  O is stored as fp16.
+//   phase 4  (layer variant only) to_out: the two CTAs that share a row tile form a cluster.  Each writes its four
+//            heads' O, as fp16 operand tiles, into its own and into its partner's shared memory, and then computes
+//            Y = O Wout^T + b for its own 160 output channels over all 320 channels of O with the machinery of
+//            phase 1.  Neither Q~ nor O ever reaches global memory.
 // Shared memory is used twice: the X tile and the weight ring of phase 1 become the Q~ tiles and the two P tiles.
 // Warps: 0 producer (TMA / bulk copies), 1 MMA issuer, 2..17 workers (four threads per row: one head each in
 // phases 1 and 2, (group, key half) in phase 3).
@@ -45,11 +49,13 @@ constexpr int OFF_A = 0;                                    // phase 1: X tile, 
 constexpr int OFF_B = OFF_A + NKB * A_TILE;                 // phase 1: weight ring
 constexpr int OFF_Q = 0;                                    // phase 3: Q~ tiles of the four heads
 constexpr int OFF_P = OFF_Q + HG * A_TILE;                  // phase 3: one probability tile (two K blocks) per group
-constexpr int OFF_RAW = OFF_B + NBSTAGE * B_TILE;            // phase 1: packed codes of the CTA's channels
-constexpr int OFF_XCHG = OFF_RAW;                           // phase 3: float2 [iteration][group][half][row], 8 KB
+constexpr int OFF_XCHG = OFF_P + 4 * A_TILE;                // phase 3: float2 [iteration][group][half][row], 8 KB
+constexpr int OFF_RAW = OFF_B + NBSTAGE * B_TILE;            // packed codes of the CTA's 160 channels (Wq, later Wout)
+static_assert(OFF_XCHG + 8192 <= OFF_RAW, "exchange buffer must fit behind the P tiles");
 constexpr int OFF_SC = OFF_RAW + RAW_BYTES;
 constexpr int OFF_SCT = OFF_SC + SCALE_BYTES;
-constexpr int OFF_K = ((OFF_SCT + SCALE_BYTES + 1023) / 1024) * 1024;    // K~ tiles, one buffer per group
+constexpr int OFF_BIAS = OFF_SCT + SCALE_BYTES;                            // phase 4: bias of the CTA's 160 channels
+constexpr int OFF_K = ((OFF_BIAS + NQ * 4 + 1023) / 1024) * 1024;          // K~ tiles, one buffer per group
 constexpr int OFF_VT = OFF_K + 2 * K_BYTES;                                // V~^T tiles, one buffer per group
 constexpr int OFF_CST = OFF_VT + 2 * VT_BYTES;                             // per-key constants of all four heads
 constexpr int OFF_MISC = OFF_CST + HG * kOperandConstBytes;
@@ -57,6 +63,7 @@ static_assert(OFF_P + 4 * A_TILE <= OFF_RAW, "phase-3 tiles must fit into the ph
 
 struct Misc {
     uint64_t a_full[NKB], b_full[NBSTAGE], b_empty[NBSTAGE], w_full, acc_full[MAX_GROUPS];
+    uint64_t w2_full, s_done, pv_done, peer_ready, o_all;       // layer variant (phase 4)
     uint64_t q_all, k_full[2], k_free[2], vt_full[2], vt_free[2], c_full, s_full[2], s_free[2], p_full[2], o_full[2], drain;
     uint32_t tmem_base;
     volatile int abort_flag;
@@ -74,12 +81,19 @@ struct QAttnArgs {
     const void* wq;             // packed [C][C] (single problem)
     const void* kv;             // blocks [B] (single problem)
     const taq_request* reqs;    // nullable; then one sequence per request
-    __half* o;                  // [z][B][N][C]
+    __half* o;                  // [z][B][N][C]  (query-attention variant)
+    const void* wout;           // packed [C][C] (layer variant, single problem)
+    __half* y;                  // [z][B][N][C]  (layer variant)
     int n_query, heads, n_ctx, max_trigger, group, q_bits;
     int* status;
 };
 
-template <bool TAIL_ONLY>
+// O tile of phase 4: K block kb (channels 64 kb .. 64 kb + 63 of O).  Blocks 0..3 reuse the Q~ tiles, block 4 the K~
+// buffers; both are dead once the S products of all four heads have been computed.
+__device__ __forceinline__ int o_tile_offset(int kb) { return kb < 4 ? OFF_Q + kb * A_TILE : OFF_K; }
+static_assert(2 * K_BYTES >= A_TILE, "the K~ buffers must hold one O tile");
+
+template <bool TAIL_ONLY, bool FUSE_OUT>
 __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_constant__ CUtensorMap tmap_x, const QAttnArgs a) {
     extern __shared__ unsigned char smem_dyn[];
     unsigned char* smem = smem_dyn + ((1024u - (ptx::smem_u32(smem_dyn) & 1023u)) & 1023u);   // 1024-byte aligned, still provably shared
@@ -116,6 +130,11 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
             ptx::mbar_init(&misc->o_full[i], 1);
         }
         ptx::mbar_init(&misc->c_full, 1);
+        ptx::mbar_init(&misc->w2_full, 1);
+        ptx::mbar_init(&misc->s_done, 1);
+        ptx::mbar_init(&misc->pv_done, 1);
+        ptx::mbar_init(&misc->peer_ready, 1);
+        ptx::mbar_init(&misc->o_all, 2 * (NWORK / 32));      // every worker warp of this CTA and of its partner
         ptx::mbar_init(&misc->q_all, NWORK / 32);
         ptx::mbar_init(&misc->drain, 1);
         misc->abort_flag = 0;
@@ -128,6 +147,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = misc->tmem_base;
     ptx::pdl_trigger();
+    if (FUSE_OUT) ptx::cluster_sync_all();                   // the partner's barriers exist before anything arrives on them
+    const uint32_t peer = FUSE_OUT ? (ptx::cluster_ctarank() ^ 1u) : 0u;
 
     const taq_kv_layout KL = kv_layout(H, T, D, a.max_trigger);
 
@@ -163,6 +184,16 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
             };
             load_k(0); load_k(1); load_vt(0); load_vt(1);
             int k_issued = 2, vt_issued = 2;
+            if (FUSE_OUT) {       // phase 1 no longer needs the packed Wq: fetch the packed Wout rows of this CTA's output channels
+                if (!ptx::mbar_wait(&misc->acc_full[n_groups - 1], 0)) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; }
+                if (!misc->abort_flag) {
+                    const uint8_t* blob2 = (const uint8_t*)(a.reqs ? a.reqs[zb].Wout : a.wout);
+                    ptx::mbar_arrive_expect_tx(&misc->w2_full, RAW_BYTES + scale_bytes + NQ * 4);
+                    ptx::bulk_load(smem + OFF_RAW, blob2 + L.off_codes + (size_t)col0 * L.row_bytes, RAW_BYTES, &misc->w2_full);
+                    ptx::bulk_load(smem + OFF_SC, blob2 + L.off_scales + (size_t)col0 * n_groups * 4, scale_bytes, &misc->w2_full);
+                    ptx::bulk_load(smem + OFF_BIAS, blob2 + L.off_bias + (size_t)col0 * 4, NQ * 4, &misc->w2_full);
+                }
+            }
             for (int g = 0; g < 2 && !misc->abort_flag; ++g) {
                 if (!ptx::mbar_wait(&misc->k_free[g], 0)) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; break; }
                 load_k(2 + g);
@@ -176,6 +207,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
             if (misc->abort_flag) {   // give copies that are still in flight a bounded chance to land before the CTA exits
                 (void)ptx::mbar_wait(&misc->w_full, 0);
                 (void)ptx::mbar_wait(&misc->c_full, 0);
+                if (FUSE_OUT) (void)ptx::mbar_wait(&misc->w2_full, 0);
                 for (int kb = 0; kb < NKB; ++kb) (void)ptx::mbar_wait(&misc->a_full[kb], 0);
                 for (int hi = k_issued - 2; hi < k_issued; ++hi) (void)ptx::mbar_wait(&misc->k_full[hi & 1], (hi >> 1) & 1);
                 for (int hi = vt_issued - 2; hi < vt_issued; ++hi) (void)ptx::mbar_wait(&misc->vt_full[hi & 1], (hi >> 1) & 1);
@@ -185,10 +217,11 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
             bool ok = true;
+            constexpr uint32_t idesc = ptx::idesc_f16_m128(NQ);
+            int s = 0;                                       // weight ring position and pass parity, continued in phase 4
+            uint32_t ph = 0;
             {   // phase 1: one accumulation pass per scale group
-                constexpr uint32_t idesc = ptx::idesc_f16_m128(NQ);
-                int s = 0, kb = 0;
-                uint32_t ph = 0;
+                int kb = 0;
                 for (int g = 0; g < n_groups && ok; ++g) {
                     const int buf = g;
                     const int kb_end = min(NKB, kb + kb_per_group);
@@ -241,8 +274,36 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
             // head's scores in registers, i.e. under the first head's softmax
             for (int it = 0; it < 2 && ok; ++it)
                 for (int g = 0; g < 2 && ok; ++g) ok = issue_s(g, it);
+            if (FUSE_OUT && ok) {     // all S products done: the Q~ tiles and K~ buffers of this CTA may receive O tiles
+                ptx::mma_commit(&misc->s_done);
+                ok = ptx::mbar_wait(&misc->s_done, 0);
+                if (ok) ptx::mbar_arrive_cluster(ptx::map_to_cta(ptx::smem_u32(&misc->peer_ready), peer));
+            }
             for (int it = 0; it < 2 && ok; ++it)
                 for (int g = 0; g < 2 && ok; ++g) ok = issue_pv(g, it);
+            if (FUSE_OUT && ok) {
+                ptx::mma_commit(&misc->pv_done);             // the P tiles become the weight ring of phase 4
+                // phase 4: Y = O Wout^T for this CTA's 160 output channels, once both CTAs' O tiles are complete
+                ok = ptx::mbar_wait_cluster(&misc->o_all, 0) && !misc->abort_flag;
+                ptx::tc_fence_after_sync();
+                int kb = 0;
+                for (int g = 0; g < n_groups && ok; ++g) {
+                    const int kb_end = min(NKB, kb + kb_per_group);
+                    for (bool first = true; kb < kb_end && ok; ++kb) {
+                        if (!ptx::mbar_wait(&misc->b_full[s], ph) || misc->abort_flag) { ok = false; break; }
+                        ptx::tc_fence_after_sync();
+                        const uint32_t a_addr = ptx::smem_u32(smem + o_tile_offset(kb));
+                        const uint32_t b_addr = ptx::smem_u32(smem + OFF_B + s * B_TILE);
+#pragma unroll
+                        for (int k = 0; k < BK / 16; ++k)
+                            ptx::mma_f16_ss(tmem_base + TMEM_ACC + g * NQ, ptx::desc_k_sw128(a_addr + k * 32), ptx::desc_k_sw128(b_addr + k * 32), idesc, !(first && k == 0));
+                        first = false;
+                        ptx::mma_commit(&misc->b_empty[s]);
+                        if (++s == NBSTAGE) { s = 0; ph ^= 1; }
+                    }
+                    if (ok) ptx::mma_commit(&misc->acc_full[g]);
+                }
+            }
             if (!ok) {
                 raise_status(a.status, TAQ_ERR_TIMEOUT);
                 misc->abort_flag = 1;
@@ -271,11 +332,11 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
 #pragma unroll
         for (int c = 0; c < HC; ++c) y[c] = 0.f;
         const int cb = part * HC;
-        {
-            int s = 0;
-            uint32_t ph = 0;
+        int s = 0;                                           // weight ring position and pass parity, continued in phase 4
+        uint32_t ph = 0;
+        auto build_tiles = [&](int first_pass) {             // expand the packed codes at OFF_RAW into the ring, K block by K block
             for (int kb = 0; kb < NKB && ok; ++kb) {
-                if (kb >= NBSTAGE && !ptx::mbar_wait(&misc->b_empty[s], ph ^ 1)) ok = false;
+                if ((!first_pass || kb >= NBSTAGE) && !ptx::mbar_wait(&misc->b_empty[s], ph ^ 1)) ok = false;
                 if (!ok || misc->abort_flag) { ok = false; break; }
                 unsigned char* b_tile = smem + OFF_B + s * B_TILE;
                 constexpr int NCH = (NQ * 8 + NWORK - 1) / NWORK;       // 16-byte chunks (8 weights) per thread and K block
@@ -294,9 +355,10 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
                 if (lane == 0) ptx::mbar_arrive(&misc->b_full[s]);
                 if (++s == NBSTAGE) { s = 0; ph ^= 1; }
             }
-        }
+        };
+        auto fold_groups = [&](uint32_t parity) {            // y += scale[g] * accumulator g, as each group completes
         for (int g = 0; g < n_groups && ok; ++g) {             // later groups are still being multiplied while this one is folded
-            ok = ptx::mbar_wait(&misc->acc_full[g], 0) && !misc->abort_flag;
+            ok = ptx::mbar_wait(&misc->acc_full[g], parity) && !misc->abort_flag;
             if (!ok) break;
             ptx::tc_fence_after_sync();
             const float* sg = scales_t + g * NQ + cb;
@@ -318,6 +380,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
             }
         }
         ptx::tc_fence_before_sync();
+        };
+        build_tiles(1);
+        fold_groups(0);
         if (!ok) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; }
         if (wt == 0) TAQ_PROF(7);
         // The last group's accumulator is complete, hence every MMA of phase 1 has finished reading shared memory and
@@ -374,7 +439,12 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
         const float inv255 = 1.0f / 255.0f;
         constexpr int OC = DP / 2;
         bool alive = ok;
+        bool peer_ok = !FUSE_OUT;                        // the partner has announced that its tiles may be written
         auto store_o = [&](int hi) {
+            if (!peer_ok) {
+                peer_ok = ptx::mbar_wait_cluster(&misc->peer_ready, 0);
+                if (!peer_ok) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; return; }
+            }
             __half* orow = a.o + grow * (size_t)(H * D) + (h_begin + hi) * D + half * OC;
             const uint32_t t_o = tmem_base + TMEM_O + grp * DP + half * OC + lane_addr;
             uint32_t v[OC / 8][8];
@@ -385,15 +455,24 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
             for (int i = 1; i < OC / 8; ++i) ptx::reg_fence8(v[i]);
 #pragma unroll
             for (int i = 0; i < OC / 8; ++i) {
-                if (half * OC + i * 8 < D && valid) {
+                if (half * OC + i * 8 < D) {
                     float f[8];
 #pragma unroll
                     for (int e2 = 0; e2 < 8; ++e2) f[e2] = __uint_as_float(v[i][e2]) * inv255;
-                    *reinterpret_cast<uint4*>(orow + i * 8) = pack8(f);
+                    const uint4 o8 = pack8(f);
+                    if (FUSE_OUT) {       // 8 channels of O as one chunk of the to_out operand tiles, here and in the partner CTA
+                        const int cg = (h_begin + hi) * D + half * OC + i * 8;       // channel of O (0..319)
+                        unsigned char* dst = smem + o_tile_offset(cg >> 6) + ptx::sw128_offset(r, (cg & 63) >> 3);
+                        *reinterpret_cast<uint4*>(dst) = o8;
+                        ptx::st_cluster_v4(ptx::map_to_cta(ptx::smem_u32(dst), peer), o8);
+                    } else if (valid) {
+                        *reinterpret_cast<uint4*>(orow + i * 8) = o8;
+                    }
                 }
             }
             ptx::tc_fence_before_sync();
         };
+
         for (int it = 0; it < 2 && alive; ++it) {
             const int hi = grp + 2 * it;
             alive = __all_sync(0xffffffffu, ptx::mbar_wait(&misc->s_full[grp], it) && !misc->abort_flag);
@@ -451,8 +530,46 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
             }
         }
         if (!alive) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; }
+
+        if (FUSE_OUT) {
+            // ---- phase 4: Y = O Wout^T + b for this CTA's 160 output channels ----
+            ptx::fence_proxy_async_all();                        // this thread's O chunks, here and in the partner CTA
+            __syncwarp();
+            if (lane == 0) {
+                ptx::mbar_arrive_cluster(ptx::map_to_cta(ptx::smem_u32(&misc->o_all), ptx::cluster_ctarank()));
+                ptx::mbar_arrive_cluster(ptx::map_to_cta(ptx::smem_u32(&misc->o_all), peer));
+            }
+            ok = alive && ptx::mbar_wait(&misc->w2_full, 0) && ptx::mbar_wait(&misc->pv_done, 0) && !misc->abort_flag;
+            asm volatile("bar.sync 1, 512;" ::: "memory");       // nobody reads the old scale table or the exchange buffer any more
+            for (int i = wt; i < NQ * n_groups; i += NWORK) scales_t[(i % n_groups) * NQ + i / n_groups] = wscales[i];
+            asm volatile("bar.sync 1, 512;" ::: "memory");
+#pragma unroll
+            for (int c = 0; c < HC; ++c) y[c] = 0.f;
+            build_tiles(0);
+            fold_groups(1);
+            if (!ok) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; }
+            if (ok) {
+                // every MMA of phase 4 is complete: the ring is free and stages the output pieces (80 bytes per thread)
+                const float* bias = reinterpret_cast<const float*>(smem + OFF_BIAS);
+                unsigned char* seg = smem + OFF_B + (size_t)(part * ROWS + r) * (HC * 2 + 16);
+#pragma unroll
+                for (int c = 0; c < HC; c += 8) {
+                    float f[8];
+#pragma unroll
+                    for (int e2 = 0; e2 < 8; ++e2) f[e2] = y[c + e2] + bias[cb + c + e2];
+                    *reinterpret_cast<uint4*>(seg + c * 2) = pack8(f);
+                }
+                ptx::fence_proxy_async_smem();
+                if (valid) {
+                    ptx::bulk_store(a.y + grow * (size_t)KIN + col0 + cb, seg, HC * 2);
+                    ptx::bulk_store_commit();
+                    ptx::bulk_store_wait_read();
+                }
+            }
+        }
     }
 
+    if (FUSE_OUT) ptx::cluster_sync_all();                   // neither CTA's shared memory goes away while its partner may still write to it
     ptx::tc_fence_before_sync();
     __syncthreads();
     if (tid == 0) { TAQ_PROF(9); TAQ_GPROF(29); }
@@ -478,6 +595,8 @@ EncodeTiledFn encode_tiled_fn2() {
 
 }  // namespace
 
+bool sm100_layer_supported(const taq_layer_desc& d) { return sm100_qattn_supported(d); }
+
 bool sm100_qattn_supported(const taq_layer_desc& d) {
     if (d.channels != KIN || d.heads * D != KIN) return false;
     if (d.w_bits != 4) return false;
@@ -487,8 +606,8 @@ bool sm100_qattn_supported(const taq_layer_desc& d) {
     return encode_tiled_fn2() != nullptr;
 }
 
-cudaError_t launch_qattn_sm100(const taq_layer_desc& d, const __half* x, const void* wq, const void* kv, const taq_request* reqs, __half* o,
-                               int n_z, int* status, cudaStream_t stream) {
+static cudaError_t launch_c320(const taq_layer_desc& d, const __half* x, const void* wq, const void* kv, const taq_request* reqs, __half* o,
+                               const void* wout, __half* y, int n_z, int* status, cudaStream_t stream) {
     if (n_z == 0 || d.n_query == 0) return cudaSuccess;
     EncodeTiledFn enc = encode_tiled_fn2();
     if (!enc) return cudaErrorNotSupported;
@@ -501,19 +620,32 @@ cudaError_t launch_qattn_sm100(const taq_layer_desc& d, const __half* x, const v
                      CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
     QAttnArgs a{};
-    a.x = x; a.wq = wq; a.kv = kv; a.reqs = reqs; a.o = o;
+    a.x = x; a.wq = wq; a.kv = kv; a.reqs = reqs; a.o = o; a.wout = wout; a.y = y;
     a.n_query = d.n_query; a.heads = d.heads; a.n_ctx = d.n_ctx; a.max_trigger = d.max_trigger; a.group = d.w_group; a.q_bits = d.q_bits;
     a.status = status;
     dim3 grid((d.n_query + ROWS - 1) / ROWS, d.heads / HG, n_z);
-    static bool configured[2] = {false, false};
-    const bool tail = d.n_ctx > 64;
-    auto kern = tail ? qattn_c320_kernel<true> : qattn_c320_kernel<false>;
-    if (!configured[tail]) {
+    static bool configured[4] = {false, false, false, false};
+    const bool tail = d.n_ctx > 64, fuse_out = y != nullptr;
+    void (*kern)(const CUtensorMap, const QAttnArgs) =
+        fuse_out ? (tail ? qattn_c320_kernel<true, true> : qattn_c320_kernel<false, true>) : (tail ? qattn_c320_kernel<true, false> : qattn_c320_kernel<false, false>);
+    const int ci = (tail ? 1 : 0) + (fuse_out ? 2 : 0);
+    if (!configured[ci]) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TOTAL);
         if (e != cudaSuccess) return e;
-        configured[tail] = true;
+        configured[ci] = true;
     }
+    if (fuse_out) return launch_pdl_cluster(kern, grid, dim3(1, 2, 1), dim3(NTHREADS), (size_t)TOTAL, stream, tmap, a);
     return launch_pdl(kern, grid, dim3(NTHREADS), (size_t)TOTAL, stream, tmap, a);
+}
+
+cudaError_t launch_qattn_sm100(const taq_layer_desc& d, const __half* x, const void* wq, const void* kv, const taq_request* reqs, __half* o,
+                               int n_z, int* status, cudaStream_t stream) {
+    return launch_c320(d, x, wq, kv, reqs, o, nullptr, nullptr, n_z, status, stream);
+}
+
+cudaError_t launch_layer_sm100(const taq_layer_desc& d, const __half* x, const void* wq, const void* wout, const void* kv, const taq_request* reqs,
+                               __half* y, int n_z, int* status, cudaStream_t stream) {
+    return launch_c320(d, x, wq, kv, reqs, nullptr, wout, y, n_z, status, stream);
 }
 
 }  // namespace taq

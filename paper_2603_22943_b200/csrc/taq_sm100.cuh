@@ -16,4 +16,10 @@ bool sm100_qattn_supported(const taq_layer_desc& d);
 cudaError_t launch_qattn_sm100(const taq_layer_desc& d, const __half* x, const void* wq, const void* kv, const taq_request* reqs, __half* o,
                                int n_z, int* status, cudaStream_t stream);
 
+// The whole layer pass (to_q, Q_a, attention, to_out) in one kernel for the same shape: pairs of CTAs exchange their
+// halves of O through distributed shared memory.
+bool sm100_layer_supported(const taq_layer_desc& d);
+cudaError_t launch_layer_sm100(const taq_layer_desc& d, const __half* x, const void* wq, const void* wout, const void* kv, const taq_request* reqs,
+                               __half* y, int n_z, int* status, cudaStream_t stream);
+
 }  // namespace taq
