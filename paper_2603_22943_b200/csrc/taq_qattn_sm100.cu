@@ -285,12 +285,14 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
                 ptx::mma_commit(&misc->pv_done);             // the P tiles become the weight ring of phase 4
                 // phase 4: Y = O Wout^T for this CTA's 160 output channels, once both CTAs' O tiles are complete
                 ok = ptx::mbar_wait_cluster(&misc->o_all, 0) && !misc->abort_flag;
+                TAQ_PROF(38);
                 ptx::tc_fence_after_sync();
                 int kb = 0;
                 for (int g = 0; g < n_groups && ok; ++g) {
                     const int kb_end = min(NKB, kb + kb_per_group);
                     for (bool first = true; kb < kb_end && ok; ++kb) {
                         if (!ptx::mbar_wait(&misc->b_full[s], ph) || misc->abort_flag) { ok = false; break; }
+                        TAQ_PROF(40 + kb);
                         ptx::tc_fence_after_sync();
                         const uint32_t a_addr = ptx::smem_u32(smem + o_tile_offset(kb));
                         const uint32_t b_addr = ptx::smem_u32(smem + OFF_B + s * B_TILE);
@@ -539,14 +541,19 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
                 ptx::mbar_arrive_cluster(ptx::map_to_cta(ptx::smem_u32(&misc->o_all), ptx::cluster_ctarank()));
                 ptx::mbar_arrive_cluster(ptx::map_to_cta(ptx::smem_u32(&misc->o_all), peer));
             }
+            if (wt == 0) TAQ_PROF(32);
             ok = alive && ptx::mbar_wait(&misc->w2_full, 0) && ptx::mbar_wait(&misc->pv_done, 0) && !misc->abort_flag;
+            if (wt == 0) TAQ_PROF(33);
             asm volatile("bar.sync 1, 512;" ::: "memory");       // nobody reads the old scale table or the exchange buffer any more
             for (int i = wt; i < NQ * n_groups; i += NWORK) scales_t[(i % n_groups) * NQ + i / n_groups] = wscales[i];
             asm volatile("bar.sync 1, 512;" ::: "memory");
 #pragma unroll
             for (int c = 0; c < HC; ++c) y[c] = 0.f;
+            if (wt == 0) TAQ_PROF(34);
             build_tiles(0);
+            if (wt == 0) TAQ_PROF(35);
             fold_groups(1);
+            if (wt == 0) TAQ_PROF(36);
             if (!ok) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; }
             if (ok) {
                 // every MMA of phase 4 is complete: the ring is free and stages the output pieces (80 bytes per thread)
@@ -566,6 +573,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
                     ptx::bulk_store_wait_read();
                 }
             }
+            if (wt == 0) TAQ_PROF(37);
         }
     }
 

@@ -184,6 +184,26 @@ def test_query_attention_equals_the_two_step_path(shape_fn, n, q_bits):
     tl.assert_layer_close(o_fused.cpu().numpy()[:, rows], want, shape.name + " O (same decisions)")
 
 
+@pytest.mark.parametrize("n,q_bits", [(4096, 8), (333, 8), (130, 0)])
+def test_one_kernel_layer_equals_the_step_by_step_path(n, q_bits):
+    """At C = 320 taq_layer_forward is a single kernel (pairs of CTAs exchange O through distributed shared memory and
+    run to_out themselves).  Its Y must equal, bit for bit, taq_query_attention followed by taq_quantized_linear: the
+    same products accumulated in the same order."""
+    from dataclasses import replace
+    shape = replace(_small(synth.config2(), n), q_bits=q_bits)
+    data = synth.make_layer(shape)
+    desc = tl.gpu_desc(shape)
+    P = tl.pack_layer_weights(shape, data)
+    mask = dev(data["mask"])
+    kv = tb.taq_kv_project(desc, dev(data["ctx"]), P["Wk"], P["Wv"], mask)
+    x = dev(data["X"])
+    y_one = tb.taq_layer_forward(desc, x, P["Wq"], P["Wout"], kv, mask)
+    o = tb.taq_query_attention(desc, x, P["Wq"], kv, mask)
+    y_two = tb.taq_quantized_linear(P["wd_cc"], o.reshape(-1, shape.channels), P["Wout"], tb.TAQ_OUT_F16).reshape(y_one.shape)
+    tb.taq_poll_device_status()
+    assert torch.equal(y_one.view(torch.int16), y_two.view(torch.int16))
+
+
 def test_layer_config1_full():
     _layer_case(synth.config1())
 
