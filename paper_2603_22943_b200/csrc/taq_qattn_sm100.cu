@@ -542,11 +542,12 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
                 ptx::mbar_arrive_cluster(ptx::map_to_cta(ptx::smem_u32(&misc->o_all), peer));
             }
             if (wt == 0) TAQ_PROF(32);
-            ok = alive && ptx::mbar_wait(&misc->w2_full, 0) && ptx::mbar_wait(&misc->pv_done, 0) && !misc->abort_flag;
-            if (wt == 0) TAQ_PROF(33);
-            asm volatile("bar.sync 1, 512;" ::: "memory");       // nobody reads the old scale table or the exchange buffer any more
+            ok = alive && ptx::mbar_wait(&misc->w2_full, 0) && !misc->abort_flag;
+            // (the old scale table was last read in phase 1)
             for (int i = wt; i < NQ * n_groups; i += NWORK) scales_t[(i % n_groups) * NQ + i / n_groups] = wscales[i];
-            asm volatile("bar.sync 1, 512;" ::: "memory");
+            ok = ok && ptx::mbar_wait(&misc->pv_done, 0) && !misc->abort_flag;          // the P tiles become the weight ring
+            if (wt == 0) TAQ_PROF(33);
+            asm volatile("bar.sync 1, 512;" ::: "memory");       // scale table complete; nobody uses the exchange buffer any more
 #pragma unroll
             for (int c = 0; c < HC; ++c) y[c] = 0.f;
             if (wt == 0) TAQ_PROF(34);
@@ -555,22 +556,29 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
             fold_groups(1);
             if (wt == 0) TAQ_PROF(36);
             if (!ok) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; }
+            // Every MMA of phase 4 is complete: the ring is free.  The 128 x 160 fp16 output tile is staged there (row
+            // pitch padded to 336 bytes: conflict-free for the row-per-lane writes) and then copied out by all threads
+            // with 16 bytes per lane, consecutive lanes on consecutive chunks of a row.
+            constexpr int PITCH = NQ * 2 + 16;
+            unsigned char* stage = smem + OFF_B;
             if (ok) {
-                // every MMA of phase 4 is complete: the ring is free and stages the output pieces (80 bytes per thread)
                 const float* bias = reinterpret_cast<const float*>(smem + OFF_BIAS);
-                unsigned char* seg = smem + OFF_B + (size_t)(part * ROWS + r) * (HC * 2 + 16);
 #pragma unroll
                 for (int c = 0; c < HC; c += 8) {
                     float f[8];
 #pragma unroll
                     for (int e2 = 0; e2 < 8; ++e2) f[e2] = y[c + e2] + bias[cb + c + e2];
-                    *reinterpret_cast<uint4*>(seg + c * 2) = pack8(f);
+                    *reinterpret_cast<uint4*>(stage + r * PITCH + (cb + c) * 2) = pack8(f);
                 }
-                ptx::fence_proxy_async_smem();
-                if (valid) {
-                    ptx::bulk_store(a.y + grow * (size_t)KIN + col0 + cb, seg, HC * 2);
-                    ptx::bulk_store_commit();
-                    ptx::bulk_store_wait_read();
+            }
+            asm volatile("bar.sync 1, 512;" ::: "memory");
+            if (!misc->abort_flag) {
+                constexpr int CPR = NQ * 2 / 16;                 // 16-byte chunks per row of the tile
+#pragma unroll
+                for (int i = 0; i < ROWS * CPR / NWORK; ++i) {
+                    const int id = i * NWORK + wt, rr = id / CPR, cc = id % CPR;
+                    if (row0 + rr < a.n_query)
+                        *reinterpret_cast<uint4*>(a.y + ((size_t)zb * a.n_query + row0 + rr) * KIN + col0 + cc * 8) = *reinterpret_cast<const uint4*>(stage + rr * PITCH + cc * 16);
                 }
             }
             if (wt == 0) TAQ_PROF(37);
