@@ -429,8 +429,10 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
             *reinterpret_cast<uint4*>(q_tile + ptx::sw128_offset(r, D / 8)) = make_uint4(0, 0, 0, 0);   // channels 40..47
             ptx::fence_proxy_async_smem();
         }
-        asm volatile("bar.sync 1, 512;" ::: "memory");       // the row scales of all heads are visible to every thread of the row
-        ok = !misc->abort_flag;
+        // No CTA barrier here: a thread reads another thread's row scale only after it has seen that head's S complete,
+        // and S is issued only after every worker warp has arrived on q_all below (release), i.e. after all scales and
+        // Q~ tiles were written.
+        __syncwarp();
         if (lane == 0) ptx::mbar_arrive(&misc->q_all);
         if (ok && !ptx::mbar_wait(&misc->c_full, 0)) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; ok = false; }
         if (wt == 0) TAQ_PROF(8);
