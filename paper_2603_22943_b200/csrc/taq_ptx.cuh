@@ -90,6 +90,13 @@ __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
+// Bulk copy from this CTA's shared memory into a peer CTA's (addresses of the destination and of the peer's barrier
+// as returned by map_to_cta); completes `bytes` on that barrier.  16-byte alignment and granularity; the source
+// must have been fenced (fence_proxy_async_smem) by its writers and stay intact until the peer has seen completion.
+__device__ __forceinline__ void bulk_copy_to_cta(uint32_t dst_cluster_addr, const void* smem_src, uint32_t bytes, uint32_t bar_cluster_addr) {
+    asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst_cluster_addr), "r"(smem_u32(smem_src)), "r"(bytes), "r"(bar_cluster_addr) : "memory");
+}
 // Orders this thread's earlier generic-proxy writes (own or peer shared memory) before later async-proxy reads.
 __device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
 

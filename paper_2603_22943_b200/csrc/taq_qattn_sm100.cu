@@ -63,7 +63,7 @@ static_assert(OFF_P + 4 * A_TILE <= OFF_RAW, "phase-3 tiles must fit into the ph
 
 struct Misc {
     uint64_t a_full[NKB], b_full[NBSTAGE], b_empty[NBSTAGE], w_full, acc_full[MAX_GROUPS];
-    uint64_t w2_full, s_done, pv_done, peer_ready, o_all;       // layer variant (phase 4)
+    uint64_t w2_full, s_done, pv_done, peer_ready, o_all, tile_done[2];       // layer variant (phase 4)
     uint64_t q_all, k_full[2], k_free[2], vt_full[2], vt_free[2], c_full, s_full[2], s_free[2], p_full[2], o_full[2], drain;
     uint32_t tmem_base;
     volatile int abort_flag;
@@ -92,6 +92,20 @@ struct QAttnArgs {
 // buffers; both are dead once the S products of all four heads have been computed.
 __device__ __forceinline__ int o_tile_offset(int kb) { return kb < 4 ? OFF_Q + kb * A_TILE : OFF_K; }
 static_assert(2 * K_BYTES >= A_TILE, "the K~ buffers must hold one O tile");
+// A CTA's four heads cover two and a half O tiles: two whole ones (tiles 0, 1 for heads 0..3; tiles 3, 4 for heads 4..7),
+// which travel to the partner CTA as bulk copies once complete, and its half of tile 2, which is written chunk by
+// chunk into both CTAs' shared memory.
+constexpr int SHARED_TILE = 2;
+static_assert(HG * D == 2 * BK + BK / 2 && KIN == 2 * HG * D, "O tile ownership assumes 160 of 320 channels per CTA");
+constexpr int OCH = DP / 2;                      // O columns per thread (two threads per row in phase 3)
+// Bit t set: the thread pair half `half` of local head hi (first head of the CTA: h_begin) stores chunks of O tile t.
+__device__ __forceinline__ uint32_t o_tiles_touched(int h_begin, int hi, int half) {
+    uint32_t m = 0;
+#pragma unroll
+    for (int i = 0; i < OCH / 8; ++i)
+        if (half * OCH + i * 8 < D) m |= 1u << (((h_begin + hi) * D + half * OCH + i * 8) >> 6);
+    return m;
+}
 
 template <bool TAIL_ONLY, bool FUSE_OUT>
 __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_constant__ CUtensorMap tmap_x, const QAttnArgs a) {
@@ -134,11 +148,22 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
         ptx::mbar_init(&misc->s_done, 1);
         ptx::mbar_init(&misc->pv_done, 1);
         ptx::mbar_init(&misc->peer_ready, 1);
-        ptx::mbar_init(&misc->o_all, 2 * (NWORK / 32));      // every worker warp of this CTA and of its partner
+        // every worker warp of this CTA and of its partner, and the two whole tiles the partner sends as bulk copies
+        ptx::mbar_init(&misc->o_all, 2 * (NWORK / 32) + (FUSE_OUT ? 1 : 0));
+        if (FUSE_OUT) {
+            const int own0 = h_begin ? SHARED_TILE + 1 : 0;
+            for (int k = 0; k < 2; ++k) {               // arrivals: one per (warp, head) that stores into the tile
+                int cnt = 0;
+                for (int hi = 0; hi < HG; ++hi)
+                    for (int hf = 0; hf < 2; ++hf) cnt += ((o_tiles_touched(h_begin, hi, hf) >> (own0 + k)) & 1u) ? NWORK / 128 : 0;
+                ptx::mbar_init(&misc->tile_done[k], cnt);
+            }
+        }
         ptx::mbar_init(&misc->q_all, NWORK / 32);
         ptx::mbar_init(&misc->drain, 1);
         misc->abort_flag = 0;
         ptx::mbar_fence_init();
+        if (FUSE_OUT) ptx::mbar_arrive_expect_tx(&misc->o_all, 2 * A_TILE);
         ptx::tma_prefetch_desc(&tmap_x);
     }
     if (warp == 1) ptx::tmem_alloc(&misc->tmem_base, TMEM_COLS);
@@ -155,13 +180,15 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
     if (warp == 0) {
         // ---------------- producer ----------------
         if (lane == 0) {
-            ptx::pdl_wait();                              // X (and in general everything else) may come from the previous kernel
-            TAQ_PROF(1); TAQ_GPROF(28);
+            // Packed weights are written by taq_pack_weights, which never lets its successor start early: they are complete
+            // before this kernel can run at all and are fetched (and expanded) under the previous kernel's tail.
             const uint8_t* blob = (const uint8_t*)(a.reqs ? a.reqs[zb].Wq : a.wq);
             const uint32_t scale_bytes = (uint32_t)(NQ * n_groups * 4);
             ptx::mbar_arrive_expect_tx(&misc->w_full, RAW_BYTES + scale_bytes);
             ptx::bulk_load(smem + OFF_RAW, blob + L.off_codes + (size_t)col0 * L.row_bytes, RAW_BYTES, &misc->w_full);
             ptx::bulk_load(smem + OFF_SC, blob + L.off_scales + (size_t)col0 * n_groups * 4, scale_bytes, &misc->w_full);
+            ptx::pdl_wait();                              // X (and in general the K~/V~ block) may come from the previous kernel
+            TAQ_PROF(1); TAQ_GPROF(28);
             for (int kb = 0; kb < NKB; ++kb) {            // the whole X tile at once: every K block has its own buffer
                 ptx::mbar_arrive_expect_tx(&misc->a_full[kb], A_TILE);
                 ptx::tma_load_3d(smem + OFF_A + kb * A_TILE, &tmap_x, &misc->a_full[kb], kb * BK, row0, zb);
@@ -203,6 +230,20 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
                 if (!ptx::mbar_wait(&misc->vt_free[g], 0)) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; break; }
                 load_vt(2 + g);
                 ++vt_issued;
+            }
+            if (FUSE_OUT && !misc->abort_flag) {
+                // phase 4: this CTA's two whole O tiles go to the partner as soon as every warp that stores into them has
+                // arrived, one bulk copy each, completing on the partner's o_all barrier
+                const int own0 = h_begin ? SHARED_TILE + 1 : 0;
+                bool sent = ptx::mbar_wait_cluster(&misc->peer_ready, 0);
+                for (int k = 0; k < 2 && sent; ++k) {
+                    sent = ptx::mbar_wait(&misc->tile_done[k], 0) && !misc->abort_flag;
+                    if (!sent) break;
+                    unsigned char* tile = smem + o_tile_offset(own0 + k);
+                    ptx::bulk_copy_to_cta(ptx::map_to_cta(ptx::smem_u32(tile), peer), tile, A_TILE, ptx::map_to_cta(ptx::smem_u32(&misc->o_all), peer));
+                    TAQ_PROF(57 + k);
+                }
+                if (!sent) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; }
             }
             if (misc->abort_flag) {   // give copies that are still in flight a bounded chance to land before the CTA exits
                 (void)ptx::mbar_wait(&misc->w_full, 0);
@@ -444,8 +485,13 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
         constexpr int OC = DP / 2;
         bool alive = ok;
         bool peer_ok = !FUSE_OUT;                        // the partner has announced that its tiles may be written
+        bool wrote_remote = false;
         auto store_o = [&](int hi) {
-            if (!peer_ok) {
+            const bool stamp = lane == 0 && q4 == 0 && half == 0;
+            const int sb = 45 + 5 * grp + (hi >= 2 ? 3 : 0);
+            if (stamp) TAQ_PROF(sb);
+            const uint32_t touched = FUSE_OUT ? o_tiles_touched(h_begin, hi, half) : 0u;
+            if (!peer_ok && ((touched >> SHARED_TILE) & 1u)) {       // this call writes into the partner's shared memory
                 peer_ok = ptx::mbar_wait_cluster(&misc->peer_ready, 0);
                 if (!peer_ok) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; return; }
             }
@@ -454,9 +500,11 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
             uint32_t v[OC / 8][8];
 #pragma unroll
             for (int i = 0; i < OC / 8; ++i) ptx::tmem_ld8(t_o + i * 8, v[i]);
+            if (stamp) TAQ_PROF(sb + 1);
             ptx::tmem_ld_wait(v[0]);
 #pragma unroll
             for (int i = 1; i < OC / 8; ++i) ptx::reg_fence8(v[i]);
+            if (stamp && hi < 2) TAQ_PROF(sb + 2);
 #pragma unroll
             for (int i = 0; i < OC / 8; ++i) {
                 if (half * OC + i * 8 < D) {
@@ -464,17 +512,28 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
 #pragma unroll
                     for (int e2 = 0; e2 < 8; ++e2) f[e2] = __uint_as_float(v[i][e2]) * inv255;
                     const uint4 o8 = pack8(f);
-                    if (FUSE_OUT) {       // 8 channels of O as one chunk of the to_out operand tiles, here and in the partner CTA
+                    if (FUSE_OUT) {       // 8 channels of O as one chunk of the to_out operand tiles
                         const int cg = (h_begin + hi) * D + half * OC + i * 8;       // channel of O (0..319)
                         unsigned char* dst = smem + o_tile_offset(cg >> 6) + ptx::sw128_offset(r, (cg & 63) >> 3);
                         *reinterpret_cast<uint4*>(dst) = o8;
-                        ptx::st_cluster_v4(ptx::map_to_cta(ptx::smem_u32(dst), peer), o8);
+                        if ((cg >> 6) == SHARED_TILE) {                                // the tile both CTAs contribute to
+                            ptx::st_cluster_v4(ptx::map_to_cta(ptx::smem_u32(dst), peer), o8);
+                            wrote_remote = true;
+                        }
                     } else if (valid) {
                         *reinterpret_cast<uint4*>(orow + i * 8) = o8;
                     }
                 }
             }
             ptx::tc_fence_before_sync();
+            if (FUSE_OUT) {       // whole tiles: tell the producer, which sends each to the partner once it is complete
+                const int own0 = h_begin ? SHARED_TILE + 1 : 0;
+                ptx::fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0)
+                    for (int k = 0; k < 2; ++k)
+                        if ((touched >> (own0 + k)) & 1u) ptx::mbar_arrive(&misc->tile_done[k]);
+            }
         };
 
         for (int it = 0; it < 2 && alive; ++it) {
@@ -511,6 +570,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
             const float m_all = fmaxf(m_loc, other.x);
             const float c_self = ex2_approx(m_loc - m_all), c_other = ex2_approx(other.x - m_all);
             const float k255 = __fdividef(255.0f * c_self, fmaf(l_loc, c_self, other.y * c_other));
+            if (it > 0 && lane == 0 && q4 == 0 && half == 0) TAQ_PROF(55 + grp);
             if (it > 0) {       // the group's P tile and O accumulator are free once its previous PV is complete and O is stored
                 alive = __all_sync(0xffffffffu, ptx::mbar_wait(&misc->o_full[grp], 0) && !misc->abort_flag);
                 if (!alive) break;
@@ -537,7 +597,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
 
         if (FUSE_OUT) {
             // ---- phase 4: Y = O Wout^T + b for this CTA's 160 output channels ----
-            ptx::fence_proxy_async_all();                        // this thread's O chunks, here and in the partner CTA
+            if (wrote_remote) ptx::fence_proxy_async_all();      // this thread's chunks of the shared tile in the partner CTA
             __syncwarp();
             if (lane == 0) {
                 ptx::mbar_arrive_cluster(ptx::map_to_cta(ptx::smem_u32(&misc->o_all), ptx::cluster_ctarank()));
