@@ -69,6 +69,10 @@ __device__ __forceinline__ void st_cluster_v4(uint32_t cluster_addr, uint4 v) {
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
+// Arrival without memory ordering: a pure "go ahead" for the peer (nothing this thread wrote is read by it).
+__device__ __forceinline__ void mbar_arrive_cluster_relaxed(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
 // Bounded wait with acquire at cluster scope: pairs with mbar_arrive_cluster from the peer CTA.
 __device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity) {
     const long long t0 = clock64();
@@ -195,6 +199,17 @@ __device__ __forceinline__ uint64_t desc_k_sw128(uint32_t smem_addr_bytes) {
     d |= (uint64_t)2 << 61;                                     // 128-byte swizzle
     return d;
 }
+// The same for the 64-byte swizzle: rows of 64 bytes (32 fp16), groups of 8 rows 512 bytes apart, the 16-byte chunk
+// index XOR-ed with bits 1..2 of the row index (address bits 4..5 with bits 7..8).
+__device__ __forceinline__ uint64_t desc_k_sw64(uint32_t smem_addr_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr_bytes >> 4) & 0x3FFF);
+    d |= (uint64_t)1 << 16;
+    d |= (uint64_t)(512 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)4 << 61;                                     // 64-byte swizzle
+    return d;
+}
 // Instruction descriptor: fp16 x fp16 -> fp32, both operands K-major, M = 128, N = n.
 __host__ __device__ constexpr uint32_t idesc_f16_m128(int n) {
     return (1u << 4) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
@@ -213,6 +228,10 @@ __device__ __forceinline__ void mma_commit(uint64_t* bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
+// Byte offset of 16-byte chunk `chunk` (0..3) of row `row` in a tile stored with the 64-byte swizzle.
+__device__ __forceinline__ uint32_t sw64_offset(int row, int chunk) {
+    return (uint32_t)(row * 64 + ((chunk ^ ((row >> 1) & 3)) << 4));
+}
 // Byte offset of the 16-byte chunk `chunk` (0..7) of row `row` inside a 128-byte-swizzled K-major tile.
 __device__ __forceinline__ uint32_t sw128_offset(int row, int chunk) {
     return (uint32_t)((row >> 3) * 1024 + (row & 7) * 128 + ((chunk ^ (row & 7)) << 4));

@@ -9,9 +9,10 @@
 //            form two groups of eight (two threads per row each); group g takes heads g and g + 2, so that one
 //            group's exponentials overlap the other group's stores, exchanges and waits.  O is stored as fp16.
 //   phase 4  (layer variant only) to_out: the two CTAs that share a row tile form a cluster.  Each writes its four
-//            heads' O, as fp16 operand tiles, into its own and into its partner's shared memory, and then computes
-//            Y = O Wout^T + b for its own 160 output channels over all 320 channels of O with the machinery of
-//            phase 1.  Neither Q~ nor O ever reaches global memory.
+//            heads' O as fp16 operand tiles (32 channels each) into its own shared memory; the producer thread sends
+//            them to the partner CTA with bulk copies between the two shared memories as they complete.  Then each
+//            CTA computes Y = O Wout^T + b for its own 160 output channels over all 320 channels of O with the
+//            machinery of phase 1.  Neither Q~ nor O ever reaches global memory.
 // Shared memory is used twice: the X tile and the weight ring of phase 1 become the Q~ tiles and the two P tiles.
 // Warps: 0 producer (TMA / bulk copies), 1 MMA issuer, 2..17 workers (four threads per row: one head each in
 // phases 1 and 2, (group, key half) in phase 3).
@@ -63,7 +64,7 @@ static_assert(OFF_P + 4 * A_TILE <= OFF_RAW, "phase-3 tiles must fit into the ph
 
 struct Misc {
     uint64_t a_full[NKB], b_full[NBSTAGE], b_empty[NBSTAGE], w_full, acc_full[MAX_GROUPS];
-    uint64_t w2_full, s_done, pv_done, peer_ready, o_all, tile_done[2];       // layer variant (phase 4)
+    uint64_t w2_full, s_done, pv_done, peer_ready, o_all, piece_done[3];      // layer variant (phase 4)
     uint64_t q_all, k_full[2], k_free[2], vt_full[2], vt_free[2], c_full, s_full[2], s_free[2], p_full[2], o_full[2], drain;
     uint32_t tmem_base;
     volatile int abort_flag;
@@ -88,23 +89,31 @@ struct QAttnArgs {
     int* status;
 };
 
-// O tile of phase 4: K block kb (channels 64 kb .. 64 kb + 63 of O).  Blocks 0..3 reuse the Q~ tiles, block 4 the K~
-// buffers; both are dead once the S products of all four heads have been computed.
-__device__ __forceinline__ int o_tile_offset(int kb) { return kb < 4 ? OFF_Q + kb * A_TILE : OFF_K; }
-static_assert(2 * K_BYTES >= A_TILE, "the K~ buffers must hold one O tile");
-// A CTA's four heads cover two and a half O tiles: two whole ones (tiles 0, 1 for heads 0..3; tiles 3, 4 for heads 4..7),
-// which travel to the partner CTA as bulk copies once complete, and its half of tile 2, which is written chunk by
-// chunk into both CTAs' shared memory.
-constexpr int SHARED_TILE = 2;
-static_assert(HG * D == 2 * BK + BK / 2 && KIN == 2 * HG * D, "O tile ownership assumes 160 of 320 channels per CTA");
+// O of phase 4 (the A operand of to_out) lives in ten tiles of 32 channels: 128 rows of 64 bytes with the 64-byte swizzle.
+// Tiles 0..7 reuse the Q~ tiles, tiles 8 and 9 the K~ buffers; both are dead once the S products of all four heads have
+// been computed.  A CTA produces five of them (heads 0..3: tiles 0..4, heads 4..7: tiles 5..9) and receives the other
+// five from its partner, as bulk copies of contiguous runs of tiles ("pieces") that leave as soon as they are complete.
+constexpr int O_TILE = ROWS * 64;                // 8 KB
+constexpr int N_OTILE = KIN / 32;
+__device__ __forceinline__ int o_tile_offset(int t) { return t < 8 ? OFF_Q + t * O_TILE : OFF_K + (t - 8) * O_TILE; }
+static_assert(8 * O_TILE == HG * A_TILE && 2 * K_BYTES >= 2 * O_TILE, "the Q~ tiles and K~ buffers must hold the ten O tiles");
+static_assert(HG * D == 5 * 32 && KIN == 2 * HG * D, "O tile ownership assumes 160 of 320 channels per CTA");
 constexpr int OCH = DP / 2;                      // O columns per thread (two threads per row in phase 3)
-// Bit t set: the thread pair half `half` of local head hi (first head of the CTA: h_begin) stores chunks of O tile t.
-__device__ __forceinline__ uint32_t o_tiles_touched(int h_begin, int hi, int half) {
+// Bit t set: the threads of half `half` of head h (0..7) store chunks of O tile t.
+__device__ __forceinline__ uint32_t o_tiles_touched(int h, int half) {
     uint32_t m = 0;
 #pragma unroll
     for (int i = 0; i < OCH / 8; ++i)
-        if (half * OCH + i * 8 < D) m |= 1u << (((h_begin + hi) * D + half * OCH + i * 8) >> 6);
+        if (half * OCH + i * 8 < D) m |= 1u << ((h * D + half * OCH + i * 8) >> 5);
     return m;
+}
+// Pieces of a CTA's five tiles: the first leaves after the first head of each group (80 channels cover two tiles and a
+// half), the rest after the second; tiles 7 and 8 are not adjacent in shared memory.
+constexpr int MAX_PIECES = 3;
+__device__ __forceinline__ int o_pieces(int h_begin, int (&first)[MAX_PIECES], int (&count)[MAX_PIECES]) {
+    if (h_begin == 0) { first[0] = 0; count[0] = 2; first[1] = 2; count[1] = 3; first[2] = 0; count[2] = 0; return 2; }
+    first[0] = 5; count[0] = 2; first[1] = 7; count[1] = 1; first[2] = 8; count[2] = 2;
+    return 3;
 }
 
 template <bool TAIL_ONLY, bool FUSE_OUT>
@@ -148,22 +157,24 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
         ptx::mbar_init(&misc->s_done, 1);
         ptx::mbar_init(&misc->pv_done, 1);
         ptx::mbar_init(&misc->peer_ready, 1);
-        // every worker warp of this CTA and of its partner, and the two whole tiles the partner sends as bulk copies
-        ptx::mbar_init(&misc->o_all, 2 * (NWORK / 32) + (FUSE_OUT ? 1 : 0));
-        if (FUSE_OUT) {
-            const int own0 = h_begin ? SHARED_TILE + 1 : 0;
-            for (int k = 0; k < 2; ++k) {               // arrivals: one per (warp, head) that stores into the tile
+        // every worker warp of this CTA, and one arrival that announces the bytes of the partner's five tiles
+        ptx::mbar_init(&misc->o_all, NWORK / 32 + 1);
+        {
+            int first[MAX_PIECES], count[MAX_PIECES];
+            const int np = o_pieces(h_begin, first, count);
+            for (int k = 0; k < MAX_PIECES; ++k) {      // arrivals: one per (warp, head) that stores into the piece
+                const uint32_t pm = k < np ? ((1u << count[k]) - 1u) << first[k] : 0u;
                 int cnt = 0;
                 for (int hi = 0; hi < HG; ++hi)
-                    for (int hf = 0; hf < 2; ++hf) cnt += ((o_tiles_touched(h_begin, hi, hf) >> (own0 + k)) & 1u) ? NWORK / 128 : 0;
-                ptx::mbar_init(&misc->tile_done[k], cnt);
+                    for (int hf = 0; hf < 2; ++hf) cnt += (o_tiles_touched(h_begin + hi, hf) & pm) ? NWORK / 128 : 0;
+                ptx::mbar_init(&misc->piece_done[k], cnt > 0 ? cnt : 1);
             }
         }
         ptx::mbar_init(&misc->q_all, NWORK / 32);
         ptx::mbar_init(&misc->drain, 1);
         misc->abort_flag = 0;
         ptx::mbar_fence_init();
-        if (FUSE_OUT) ptx::mbar_arrive_expect_tx(&misc->o_all, 2 * A_TILE);
+        if (FUSE_OUT) ptx::mbar_arrive_expect_tx(&misc->o_all, (N_OTILE / 2) * O_TILE);
         ptx::tma_prefetch_desc(&tmap_x);
     }
     if (warp == 1) ptx::tmem_alloc(&misc->tmem_base, TMEM_COLS);
@@ -232,15 +243,18 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
                 ++vt_issued;
             }
             if (FUSE_OUT && !misc->abort_flag) {
-                // phase 4: this CTA's two whole O tiles go to the partner as soon as every warp that stores into them has
-                // arrived, one bulk copy each, completing on the partner's o_all barrier
-                const int own0 = h_begin ? SHARED_TILE + 1 : 0;
-                bool sent = ptx::mbar_wait_cluster(&misc->peer_ready, 0);
-                for (int k = 0; k < 2 && sent; ++k) {
-                    sent = ptx::mbar_wait(&misc->tile_done[k], 0) && !misc->abort_flag;
+                // phase 4: this CTA's O tiles go to the partner, piece by piece, as soon as every warp that stores into a
+                // piece has arrived and the partner has announced that its Q~ tiles and K~ buffers are dead; the copies
+                // complete on the partner's o_all barrier
+                int first[MAX_PIECES], count[MAX_PIECES];
+                const int np = o_pieces(h_begin, first, count);
+                bool sent = ptx::mbar_wait(&misc->peer_ready, 0);
+                for (int k = 0; k < np && sent; ++k) {
+                    sent = ptx::mbar_wait(&misc->piece_done[k], 0) && !misc->abort_flag;
                     if (!sent) break;
-                    unsigned char* tile = smem + o_tile_offset(own0 + k);
-                    ptx::bulk_copy_to_cta(ptx::map_to_cta(ptx::smem_u32(tile), peer), tile, A_TILE, ptx::map_to_cta(ptx::smem_u32(&misc->o_all), peer));
+                    unsigned char* piece = smem + o_tile_offset(first[k]);
+                    ptx::bulk_copy_to_cta(ptx::map_to_cta(ptx::smem_u32(piece), peer), piece, (uint32_t)(count[k] * O_TILE),
+                                          ptx::map_to_cta(ptx::smem_u32(&misc->o_all), peer));
                     TAQ_PROF(57 + k);
                 }
                 if (!sent) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; }
@@ -318,14 +332,14 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
             if (FUSE_OUT && ok) {     // all S products done: the Q~ tiles and K~ buffers of this CTA may receive O tiles
                 ptx::mma_commit(&misc->s_done);
                 ok = ptx::mbar_wait(&misc->s_done, 0);
-                if (ok) ptx::mbar_arrive_cluster(ptx::map_to_cta(ptx::smem_u32(&misc->peer_ready), peer));
+                if (ok) ptx::mbar_arrive_cluster_relaxed(ptx::map_to_cta(ptx::smem_u32(&misc->peer_ready), peer));
             }
             for (int it = 0; it < 2 && ok; ++it)
                 for (int g = 0; g < 2 && ok; ++g) ok = issue_pv(g, it);
             if (FUSE_OUT && ok) {
                 ptx::mma_commit(&misc->pv_done);             // the P tiles become the weight ring of phase 4
                 // phase 4: Y = O Wout^T for this CTA's 160 output channels, once both CTAs' O tiles are complete
-                ok = ptx::mbar_wait_cluster(&misc->o_all, 0) && !misc->abort_flag;
+                ok = ptx::mbar_wait(&misc->o_all, 0) && !misc->abort_flag;
                 TAQ_PROF(38);
                 ptx::tc_fence_after_sync();
                 int kb = 0;
@@ -335,11 +349,11 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
                         if (!ptx::mbar_wait(&misc->b_full[s], ph) || misc->abort_flag) { ok = false; break; }
                         TAQ_PROF(40 + kb);
                         ptx::tc_fence_after_sync();
-                        const uint32_t a_addr = ptx::smem_u32(smem + o_tile_offset(kb));
+                        const uint32_t a_addr[2] = {ptx::smem_u32(smem + o_tile_offset(2 * kb)), ptx::smem_u32(smem + o_tile_offset(2 * kb + 1))};
                         const uint32_t b_addr = ptx::smem_u32(smem + OFF_B + s * B_TILE);
 #pragma unroll
-                        for (int k = 0; k < BK / 16; ++k)
-                            ptx::mma_f16_ss(tmem_base + TMEM_ACC + g * NQ, ptx::desc_k_sw128(a_addr + k * 32), ptx::desc_k_sw128(b_addr + k * 32), idesc, !(first && k == 0));
+                        for (int k = 0; k < BK / 16; ++k)      // the 64-wide weight block spans two O tiles
+                            ptx::mma_f16_ss(tmem_base + TMEM_ACC + g * NQ, ptx::desc_k_sw64(a_addr[k >> 1] + (k & 1) * 32), ptx::desc_k_sw128(b_addr + k * 32), idesc, !(first && k == 0));
                         first = false;
                         ptx::mma_commit(&misc->b_empty[s]);
                         if (++s == NBSTAGE) { s = 0; ph ^= 1; }
@@ -484,17 +498,10 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
         const float inv255 = 1.0f / 255.0f;
         constexpr int OC = DP / 2;
         bool alive = ok;
-        bool peer_ok = !FUSE_OUT;                        // the partner has announced that its tiles may be written
-        bool wrote_remote = false;
         auto store_o = [&](int hi) {
             const bool stamp = lane == 0 && q4 == 0 && half == 0;
             const int sb = 45 + 5 * grp + (hi >= 2 ? 3 : 0);
             if (stamp) TAQ_PROF(sb);
-            const uint32_t touched = FUSE_OUT ? o_tiles_touched(h_begin, hi, half) : 0u;
-            if (!peer_ok && ((touched >> SHARED_TILE) & 1u)) {       // this call writes into the partner's shared memory
-                peer_ok = ptx::mbar_wait_cluster(&misc->peer_ready, 0);
-                if (!peer_ok) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; return; }
-            }
             __half* orow = a.o + grow * (size_t)(H * D) + (h_begin + hi) * D + half * OC;
             const uint32_t t_o = tmem_base + TMEM_O + grp * DP + half * OC + lane_addr;
             uint32_t v[OC / 8][8];
@@ -514,25 +521,22 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
                     const uint4 o8 = pack8(f);
                     if (FUSE_OUT) {       // 8 channels of O as one chunk of the to_out operand tiles
                         const int cg = (h_begin + hi) * D + half * OC + i * 8;       // channel of O (0..319)
-                        unsigned char* dst = smem + o_tile_offset(cg >> 6) + ptx::sw128_offset(r, (cg & 63) >> 3);
-                        *reinterpret_cast<uint4*>(dst) = o8;
-                        if ((cg >> 6) == SHARED_TILE) {                                // the tile both CTAs contribute to
-                            ptx::st_cluster_v4(ptx::map_to_cta(ptx::smem_u32(dst), peer), o8);
-                            wrote_remote = true;
-                        }
+                        *reinterpret_cast<uint4*>(smem + o_tile_offset(cg >> 5) + ptx::sw64_offset(r, (cg & 31) >> 3)) = o8;
                     } else if (valid) {
                         *reinterpret_cast<uint4*>(orow + i * 8) = o8;
                     }
                 }
             }
             ptx::tc_fence_before_sync();
-            if (FUSE_OUT) {       // whole tiles: tell the producer, which sends each to the partner once it is complete
-                const int own0 = h_begin ? SHARED_TILE + 1 : 0;
+            if (FUSE_OUT) {       // tell the producer, which sends each piece to the partner once it is complete
+                int first[MAX_PIECES], count[MAX_PIECES];
+                const int np = o_pieces(h_begin, first, count);
+                const uint32_t touched = o_tiles_touched(h_begin + hi, half);
                 ptx::fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0)
-                    for (int k = 0; k < 2; ++k)
-                        if ((touched >> (own0 + k)) & 1u) ptx::mbar_arrive(&misc->tile_done[k]);
+                    for (int k = 0; k < np; ++k)
+                        if (touched & (((1u << count[k]) - 1u) << first[k])) ptx::mbar_arrive(&misc->piece_done[k]);
             }
         };
 
@@ -597,12 +601,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
 
         if (FUSE_OUT) {
             // ---- phase 4: Y = O Wout^T + b for this CTA's 160 output channels ----
-            if (wrote_remote) ptx::fence_proxy_async_all();      // this thread's chunks of the shared tile in the partner CTA
-            __syncwarp();
-            if (lane == 0) {
-                ptx::mbar_arrive_cluster(ptx::map_to_cta(ptx::smem_u32(&misc->o_all), ptx::cluster_ctarank()));
-                ptx::mbar_arrive_cluster(ptx::map_to_cta(ptx::smem_u32(&misc->o_all), peer));
-            }
+            __syncwarp();                                        // (every store_o ended with a proxy fence)
+            if (lane == 0) ptx::mbar_arrive(&misc->o_all);
             if (wt == 0) TAQ_PROF(32);
             ok = alive && ptx::mbar_wait(&misc->w2_full, 0) && !misc->abort_flag;
             // (the old scale table was last read in phase 1)
