@@ -42,6 +42,14 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
     return true;
 }
 
+// One lane of the (converged) warp: the others get false.  The warp that issues tcgen05.mma walks its control flow
+// with all lanes, so that addresses and loop state stay warp-uniform, and only the elected lane issues.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t e;
+    asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(e));
+    return e != 0;
+}
+
 // ---- programmatic dependent launch ---------------------------------------------------------------------
 // A kernel launched with the programmatic-serialization attribute may start while its predecessor in the stream
 // is still draining.  pdl_wait() returns once the predecessor has completed and its writes are visible; nothing
@@ -210,6 +218,13 @@ __device__ __forceinline__ uint64_t desc_k_sw64(uint32_t smem_addr_bytes) {
     d |= (uint64_t)4 << 61;                                     // 64-byte swizzle
     return d;
 }
+// The two halves of those descriptors, for issue loops that advance the start address only: the low word of a tile
+// at shared-memory address `a` is desc_lo(a); 16 bytes further is +1 (shared-memory addresses stay below 2^18, so
+// the 14-bit field never wraps), the high word is a constant of the layout.
+__device__ __forceinline__ uint32_t desc_lo(uint32_t smem_addr_bytes) { return ((smem_addr_bytes >> 4) & 0x3FFFu) | (1u << 16); }
+constexpr uint32_t kDescHiSw128 = (1024u >> 4) | (1u << 14) | (2u << 29);
+constexpr uint32_t kDescHiSw64 = (512u >> 4) | (1u << 14) | (4u << 29);
+__device__ __forceinline__ uint64_t desc_join(uint32_t hi, uint32_t lo) { return ((uint64_t)hi << 32) | lo; }
 // Instruction descriptor: fp16 x fp16 -> fp32, both operands K-major, M = 128, N = n.
 __host__ __device__ constexpr uint32_t idesc_f16_m128(int n) {
     return (1u << 4) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);

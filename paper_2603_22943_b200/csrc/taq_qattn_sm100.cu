@@ -270,103 +270,117 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
-        if (lane == 0) {
-            bool ok = true;
-            constexpr uint32_t idesc = ptx::idesc_f16_m128(NQ);
-            int s = 0;                                       // weight ring position and pass parity, continued in phase 4
-            uint32_t ph = 0;
-            {   // phase 1: one accumulation pass per scale group
-                int kb = 0;
-                for (int g = 0; g < n_groups && ok; ++g) {
-                    const int buf = g;
-                    const int kb_end = min(NKB, kb + kb_per_group);
-                    for (bool first = true; kb < kb_end && ok; ++kb) {
-                        if (!ptx::mbar_wait(&misc->a_full[kb], 0) || !ptx::mbar_wait(&misc->b_full[s], ph) || misc->abort_flag) { ok = false; break; }
+        // All 32 lanes walk the control flow (waits, loop state, descriptor words stay warp-uniform and cheap); one
+        // elected lane issues the MMAs and commits.  The issue path is kept short on purpose: this warp shares its
+        // scheduler with four worker warps, and every instruction it needs between two MMAs delays the tensor core.
+        const bool leader = ptx::elect_one();
+        bool ok = true;
+        auto wait = [&](uint64_t* bar, uint32_t parity) -> bool { return __all_sync(0xffffffffu, ptx::mbar_wait(bar, parity) && !misc->abort_flag) != 0; };
+        constexpr uint32_t idesc = ptx::idesc_f16_m128(NQ);
+        constexpr uint32_t HI128 = ptx::kDescHiSw128, HI64 = ptx::kDescHiSw64;
+        const uint32_t a_lo0 = ptx::desc_lo(ptx::smem_u32(smem + OFF_A)), b_lo0 = ptx::desc_lo(ptx::smem_u32(smem + OFF_B));
+        const uint32_t q_lo0 = ptx::desc_lo(ptx::smem_u32(smem + OFF_Q)), p_lo0 = ptx::desc_lo(ptx::smem_u32(smem + OFF_P));
+        const uint32_t k_lo0 = ptx::desc_lo(ptx::smem_u32(smem + OFF_K)), vt_lo0 = ptx::desc_lo(ptx::smem_u32(smem + OFF_VT));
+        int s = 0;                                       // weight ring position and pass parity, continued in phase 4
+        uint32_t ph = 0;
+        {   // phase 1: one accumulation pass per scale group
+            int kb = 0;
+            for (int g = 0; g < n_groups && ok; ++g) {
+                const int kb_end = min(NKB, kb + kb_per_group);
+                for (bool first = true; kb < kb_end && ok; ++kb) {
+                    if (!wait(&misc->a_full[kb], 0) || !wait(&misc->b_full[s], ph)) { ok = false; break; }
+                    if (leader) {
                         TAQ_PROF(2 + kb);
-                        ptx::tc_fence_after_sync();
-                        const uint32_t a_addr = ptx::smem_u32(smem + OFF_A + kb * A_TILE);
-                        const uint32_t b_addr = ptx::smem_u32(smem + OFF_B + s * B_TILE);
+                        const uint32_t a_lo = a_lo0 + kb * (A_TILE >> 4), b_lo = b_lo0 + s * (B_TILE >> 4);
 #pragma unroll
                         for (int k = 0; k < BK / 16; ++k)
-                            ptx::mma_f16_ss(tmem_base + TMEM_ACC + buf * NQ, ptx::desc_k_sw128(a_addr + k * 32), ptx::desc_k_sw128(b_addr + k * 32), idesc, !(first && k == 0));
-                        first = false;
+                            ptx::mma_f16_ss(tmem_base + TMEM_ACC + g * NQ, ptx::desc_join(HI128, a_lo + 2 * k), ptx::desc_join(HI128, b_lo + 2 * k), idesc, !(first && k == 0));
                         ptx::mma_commit(&misc->b_empty[s]);
-                        if (++s == NBSTAGE) { s = 0; ph ^= 1; }
+                        if (kb + 1 == kb_end) ptx::mma_commit(&misc->acc_full[g]);
                     }
-                    if (ok) ptx::mma_commit(&misc->acc_full[buf]);
+                    first = false;
+                    if (++s == NBSTAGE) { s = 0; ph ^= 1; }
                 }
             }
-            // phase 3: the Q~ tiles of all four heads are in place once every worker warp has arrived
-            if (ok && !ptx::mbar_wait(&misc->q_all, 0)) ok = false;
-            const uint32_t q_addr = ptx::smem_u32(smem + OFF_Q), p_addr = ptx::smem_u32(smem + OFF_P);
-            // group g (heads g, g + 2) owns K~/V~ buffer g, S accumulator g, O accumulator g and P tile g
-            auto issue_s = [&](int g, int it) -> bool {
-                const int hi = g + 2 * it;
-                if (!ptx::mbar_wait(&misc->k_full[g], it) || (it > 0 && !ptx::mbar_wait(&misc->s_free[g], it - 1)) || misc->abort_flag) return false;
-                ptx::tc_fence_after_sync();
-                const uint32_t k_addr = ptx::smem_u32(smem + OFF_K + g * K_BYTES);
+        }
+        // phase 3: the Q~ tiles of all four heads are in place once every worker warp has arrived (their reads of the
+        // phase-1 accumulators, whose columns S and O reuse, are ordered before that arrival)
+        ok = ok && wait(&misc->q_all, 0);
+        ptx::tc_fence_after_sync();
+        // group g (heads g, g + 2) owns K~/V~ buffer g, S accumulator g, O accumulator g and P tile g
+        auto issue_s = [&](int g, int it) -> bool {
+            const int hi = g + 2 * it;
+            if (!wait(&misc->k_full[g], it) || (it > 0 && !wait(&misc->s_free[g], it - 1))) return false;
+            ptx::tc_fence_after_sync();                  // the group's loads of its previous S
+            if (leader) {
+                const uint32_t qh_lo = q_lo0 + hi * (A_TILE >> 4), kg_lo = k_lo0 + g * (K_BYTES >> 4);
 #pragma unroll
                 for (int ks = 0; ks < DP / 16; ++ks)
-                    ptx::mma_f16_ss(tmem_base + TMEM_S + g * TP, ptx::desc_k_sw128(q_addr + hi * A_TILE + ks * 32), ptx::desc_k_sw128(k_addr + ks * 32), ptx::idesc_f16_m128(TP), ks != 0);
+                    ptx::mma_f16_ss(tmem_base + TMEM_S + g * TP, ptx::desc_join(HI128, qh_lo + 2 * ks), ptx::desc_join(HI128, kg_lo + 2 * ks), ptx::idesc_f16_m128(TP), ks != 0);
                 ptx::mma_commit(&misc->s_full[g]);
                 ptx::mma_commit(&misc->k_free[g]);
-                return true;
-            };
-            auto issue_pv = [&](int g, int it) -> bool {
-                if (!ptx::mbar_wait(&misc->p_full[g], it) || !ptx::mbar_wait(&misc->vt_full[g], it) || misc->abort_flag) return false;     // (the group has emptied O before it arrives)
-                ptx::tc_fence_after_sync();
-                const uint32_t vt_addr = ptx::smem_u32(smem + OFF_VT + g * VT_BYTES);
-                const uint32_t pg_addr = p_addr + g * 2 * A_TILE;
+            }
+            return true;
+        };
+        auto issue_pv = [&](int g, int it) -> bool {
+            if (!wait(&misc->p_full[g], it) || !wait(&misc->vt_full[g], it)) return false;     // (the group has emptied O before it arrives)
+            ptx::tc_fence_after_sync();
+            if (leader) {
+                const uint32_t pg_lo = p_lo0 + g * 2 * (A_TILE >> 4), vg_lo = vt_lo0 + g * (VT_BYTES >> 4);
 #pragma unroll
                 for (int ks = 0; ks < TP / 16; ++ks)
-                    ptx::mma_f16_ss(tmem_base + TMEM_O + g * DP, ptx::desc_k_sw128(pg_addr + (ks / 4) * A_TILE + (ks % 4) * 32),
-                                    ptx::desc_k_sw128(vt_addr + (ks / 4) * VT_BLOCK + (ks % 4) * 32), ptx::idesc_f16_m128(DP), ks != 0);
+                    ptx::mma_f16_ss(tmem_base + TMEM_O + g * DP, ptx::desc_join(HI128, pg_lo + (ks / 4) * (A_TILE >> 4) + (ks % 4) * 2),
+                                    ptx::desc_join(HI128, vg_lo + (ks / 4) * (VT_BLOCK >> 4) + (ks % 4) * 2), ptx::idesc_f16_m128(DP), ks != 0);
                 ptx::mma_commit(&misc->o_full[g]);
                 ptx::mma_commit(&misc->vt_free[g]);
-                return true;
-            };
-            // S of a group's second head is issued as soon as its K~ tile has arrived and the group holds the first
-            // head's scores in registers, i.e. under the first head's softmax
-            for (int it = 0; it < 2 && ok; ++it)
-                for (int g = 0; g < 2 && ok; ++g) ok = issue_s(g, it);
-            if (FUSE_OUT && ok) {     // all S products done: the Q~ tiles and K~ buffers of this CTA may receive O tiles
-                ptx::mma_commit(&misc->s_done);
-                ok = ptx::mbar_wait(&misc->s_done, 0);
-                if (ok) ptx::mbar_arrive_cluster_relaxed(ptx::map_to_cta(ptx::smem_u32(&misc->peer_ready), peer));
             }
-            for (int it = 0; it < 2 && ok; ++it)
-                for (int g = 0; g < 2 && ok; ++g) ok = issue_pv(g, it);
-            if (FUSE_OUT && ok) {
-                ptx::mma_commit(&misc->pv_done);             // the P tiles become the weight ring of phase 4
-                // phase 4: Y = O Wout^T for this CTA's 160 output channels, once both CTAs' O tiles are complete
-                ok = ptx::mbar_wait(&misc->o_all, 0) && !misc->abort_flag;
-                TAQ_PROF(38);
-                ptx::tc_fence_after_sync();
-                int kb = 0;
-                for (int g = 0; g < n_groups && ok; ++g) {
-                    const int kb_end = min(NKB, kb + kb_per_group);
-                    for (bool first = true; kb < kb_end && ok; ++kb) {
-                        if (!ptx::mbar_wait(&misc->b_full[s], ph) || misc->abort_flag) { ok = false; break; }
+            return true;
+        };
+        // S of a group's second head is issued as soon as its K~ tile has arrived and the group holds the first
+        // head's scores in registers, i.e. under the first head's softmax
+        for (int it = 0; it < 2 && ok; ++it)
+            for (int g = 0; g < 2 && ok; ++g) ok = issue_s(g, it);
+        if (FUSE_OUT && ok) {     // all S products done: the Q~ tiles and K~ buffers of this CTA may receive O tiles
+            if (leader) ptx::mma_commit(&misc->s_done);
+            ok = wait(&misc->s_done, 0);
+            if (ok && leader) ptx::mbar_arrive_cluster_relaxed(ptx::map_to_cta(ptx::smem_u32(&misc->peer_ready), peer));
+        }
+        for (int it = 0; it < 2 && ok; ++it)
+            for (int g = 0; g < 2 && ok; ++g) ok = issue_pv(g, it);
+        if (FUSE_OUT && ok) {
+            if (leader) ptx::mma_commit(&misc->pv_done);             // the P tiles become the weight ring of phase 4
+            // phase 4: Y = O Wout^T for this CTA's 160 output channels, once both CTAs' O tiles are complete
+            ok = wait(&misc->o_all, 0);
+            if (leader) TAQ_PROF(38);
+            ptx::tc_fence_after_sync();                  // the workers' loads of the last O accumulators
+            int kb = 0;
+            for (int g = 0; g < n_groups && ok; ++g) {
+                const int kb_end = min(NKB, kb + kb_per_group);
+                for (bool first = true; kb < kb_end && ok; ++kb) {
+                    if (!wait(&misc->b_full[s], ph)) { ok = false; break; }
+                    if (leader) {
                         TAQ_PROF(40 + kb);
-                        ptx::tc_fence_after_sync();
-                        const uint32_t a_addr[2] = {ptx::smem_u32(smem + o_tile_offset(2 * kb)), ptx::smem_u32(smem + o_tile_offset(2 * kb + 1))};
-                        const uint32_t b_addr = ptx::smem_u32(smem + OFF_B + s * B_TILE);
+                        // the 64-wide weight block spans O tiles 2 kb and 2 kb + 1 (adjacent, except tiles 7 and 8)
+                        const uint32_t o_lo = kb < 4 ? q_lo0 + 2 * kb * (O_TILE >> 4) : k_lo0;
+                        const uint32_t b_lo = b_lo0 + s * (B_TILE >> 4);
 #pragma unroll
-                        for (int k = 0; k < BK / 16; ++k)      // the 64-wide weight block spans two O tiles
-                            ptx::mma_f16_ss(tmem_base + TMEM_ACC + g * NQ, ptx::desc_k_sw64(a_addr[k >> 1] + (k & 1) * 32), ptx::desc_k_sw128(b_addr + k * 32), idesc, !(first && k == 0));
-                        first = false;
+                        for (int k = 0; k < BK / 16; ++k)
+                            ptx::mma_f16_ss(tmem_base + TMEM_ACC + g * NQ, ptx::desc_join(HI64, o_lo + (k >> 1) * (O_TILE >> 4) + (k & 1) * 2), ptx::desc_join(HI128, b_lo + 2 * k), idesc, !(first && k == 0));
                         ptx::mma_commit(&misc->b_empty[s]);
-                        if (++s == NBSTAGE) { s = 0; ph ^= 1; }
+                        if (kb + 1 == kb_end) ptx::mma_commit(&misc->acc_full[g]);
                     }
-                    if (ok) ptx::mma_commit(&misc->acc_full[g]);
+                    first = false;
+                    if (++s == NBSTAGE) { s = 0; ph ^= 1; }
                 }
             }
-            if (!ok) {
+        }
+        if (!ok) {
+            if (leader) {
                 raise_status(a.status, TAQ_ERR_TIMEOUT);
                 misc->abort_flag = 1;
                 ptx::mma_commit(&misc->drain);               // wait (bounded) for whatever was issued before TMEM is given back
-                (void)ptx::mbar_wait(&misc->drain, 0);
             }
+            (void)ptx::mbar_wait(&misc->drain, 0);
         }
     } else {
         // ---------------- workers (warps 2..17): four threads per row ----------------
@@ -395,6 +409,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
             for (int kb = 0; kb < NKB && ok; ++kb) {
                 if ((!first_pass || kb >= NBSTAGE) && !ptx::mbar_wait(&misc->b_empty[s], ph ^ 1)) ok = false;
                 if (!ok || misc->abort_flag) { ok = false; break; }
+                if (wt == 0) TAQ_PROF((first_pass ? 95 : 90) + kb);
                 unsigned char* b_tile = smem + OFF_B + s * B_TILE;
                 constexpr int NCH = (NQ * 8 + NWORK - 1) / NWORK;       // 16-byte chunks (8 weights) per thread and K block
                 const int n0 = wt >> 3, c = wt & 7;
@@ -410,6 +425,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
                 ptx::fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(&misc->b_full[s]);
+                if (wt == 0) TAQ_PROF((first_pass ? 85 : 80) + kb);
                 if (++s == NBSTAGE) { s = 0; ph ^= 1; }
             }
         };
