@@ -64,7 +64,7 @@ static_assert(OFF_P + 4 * A_TILE <= OFF_RAW, "phase-3 tiles must fit into the ph
 
 struct Misc {
     uint64_t a_full[NKB], b_full[NBSTAGE], b_empty[NBSTAGE], w_full, acc_full[MAX_GROUPS];
-    uint64_t w2_full, s_done, pv_done, peer_ready, o_all, piece_done[3];      // layer variant (phase 4)
+    uint64_t w2_full, s_done, pv_done, peer_ready, peer_got, o_all, piece_done[3];      // layer variant (phase 4)
     uint64_t q_all, k_full[2], k_free[2], vt_full[2], vt_free[2], c_full, s_full[2], s_free[2], p_full[2], o_full[2], drain;
     uint32_t tmem_base;
     volatile int abort_flag;
@@ -117,7 +117,7 @@ __device__ __forceinline__ int o_pieces(int h_begin, int (&first)[MAX_PIECES], i
 }
 
 template <bool TAIL_ONLY, bool FUSE_OUT>
-__global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_constant__ CUtensorMap tmap_x, const QAttnArgs a) {
+__global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_y, const QAttnArgs a) {
     extern __shared__ unsigned char smem_dyn[];
     unsigned char* smem = smem_dyn + ((1024u - (ptx::smem_u32(smem_dyn) & 1023u)) & 1023u);   // 1024-byte aligned, still provably shared
     Misc* misc = reinterpret_cast<Misc*>(smem + OFF_MISC);
@@ -157,6 +157,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
         ptx::mbar_init(&misc->s_done, 1);
         ptx::mbar_init(&misc->pv_done, 1);
         ptx::mbar_init(&misc->peer_ready, 1);
+        ptx::mbar_init(&misc->peer_got, 1);
         // every worker warp of this CTA, and one arrival that announces the bytes of the partner's five tiles
         ptx::mbar_init(&misc->o_all, NWORK / 32 + 1);
         {
@@ -176,6 +177,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
         ptx::mbar_fence_init();
         if (FUSE_OUT) ptx::mbar_arrive_expect_tx(&misc->o_all, (N_OTILE / 2) * O_TILE);
         ptx::tma_prefetch_desc(&tmap_x);
+        if (FUSE_OUT) ptx::tma_prefetch_desc(&tmap_y);
     }
     if (warp == 1) ptx::tmem_alloc(&misc->tmem_base, TMEM_COLS);
     ptx::tc_fence_before_sync();
@@ -351,6 +353,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
             if (leader) ptx::mma_commit(&misc->pv_done);             // the P tiles become the weight ring of phase 4
             // phase 4: Y = O Wout^T for this CTA's 160 output channels, once both CTAs' O tiles are complete
             ok = wait(&misc->o_all, 0);
+            // the partner's copies have landed: it may leave without waiting for this CTA any longer
+            if (ok && leader) ptx::mbar_arrive_cluster_relaxed(ptx::map_to_cta(ptx::smem_u32(&misc->peer_got), peer));
             if (leader) TAQ_PROF(38);
             ptx::tc_fence_after_sync();                  // the workers' loads of the last O accumulators
             int kb = 0;
@@ -634,10 +638,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
             fold_groups(1);
             if (wt == 0) TAQ_PROF(36);
             if (!ok) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; }
-            // Every MMA of phase 4 is complete: the ring is free.  The 128 x 160 fp16 output tile is staged there (row
-            // pitch padded to 336 bytes: conflict-free for the row-per-lane writes) and then copied out by all threads
-            // with 16 bytes per lane, consecutive lanes on consecutive chunks of a row.
-            constexpr int PITCH = NQ * 2 + 16;
+            // Every MMA of phase 4 is complete: the ring is free.  The 128 x 160 fp16 output tile is staged there as five
+            // tiles of 32 channels (64-byte rows, 64-byte swizzle: conflict-free for the row-per-lane writes), which one
+            // thread hands to the TMA unit as tensor stores; rows beyond n_query are clipped by the tensor map.
             unsigned char* stage = smem + OFF_B;
             if (ok) {
                 const float* bias = reinterpret_cast<const float*>(smem + OFF_BIAS);
@@ -646,24 +649,25 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
                     float f[8];
 #pragma unroll
                     for (int e2 = 0; e2 < 8; ++e2) f[e2] = y[c + e2] + bias[cb + c + e2];
-                    *reinterpret_cast<uint4*>(stage + r * PITCH + (cb + c) * 2) = pack8(f);
+                    const int c8 = (cb + c) >> 3;
+                    *reinterpret_cast<uint4*>(stage + (c8 >> 2) * O_TILE + ptx::sw64_offset(r, c8 & 3)) = pack8(f);
                 }
             }
+            ptx::fence_proxy_async_smem();
             asm volatile("bar.sync 1, 512;" ::: "memory");
-            if (!misc->abort_flag) {
-                constexpr int CPR = NQ * 2 / 16;                 // 16-byte chunks per row of the tile
+            if (wt == 0 && !misc->abort_flag) {
 #pragma unroll
-                for (int i = 0; i < ROWS * CPR / NWORK; ++i) {
-                    const int id = i * NWORK + wt, rr = id / CPR, cc = id % CPR;
-                    if (row0 + rr < a.n_query)
-                        *reinterpret_cast<uint4*>(a.y + ((size_t)zb * a.n_query + row0 + rr) * KIN + col0 + cc * 8) = *reinterpret_cast<const uint4*>(stage + rr * PITCH + cc * 16);
-                }
+                for (int t = 0; t < NQ / 32; ++t) ptx::tma_store_3d(&tmap_y, stage + t * O_TILE, col0 + 32 * t, row0, zb);
+                ptx::bulk_store_commit();
+                ptx::bulk_store_wait_read();                     // shared memory is given back only after the stores have read it
             }
             if (wt == 0) TAQ_PROF(37);
         }
     }
 
-    if (FUSE_OUT) ptx::cluster_sync_all();                   // neither CTA's shared memory goes away while its partner may still write to it
+    // Neither CTA's shared memory may go away while the partner still writes to it or reads from it: each CTA has told
+    // its partner (peer_got) that everything it expects from it has landed, and leaves only after hearing the same.
+    if (FUSE_OUT && tid == 0 && !ptx::mbar_wait(&misc->peer_got, 0)) raise_status(a.status, TAQ_ERR_TIMEOUT);
     ptx::tc_fence_before_sync();
     __syncthreads();
     if (tid == 0) { TAQ_PROF(9); TAQ_GPROF(29); }
@@ -720,7 +724,14 @@ static cudaError_t launch_c320(const taq_layer_desc& d, const __half* x, const v
     dim3 grid((d.n_query + ROWS - 1) / ROWS, d.heads / HG, n_z);
     static bool configured[4] = {false, false, false, false};
     const bool tail = d.n_ctx > 64, fuse_out = y != nullptr;
-    void (*kern)(const CUtensorMap, const QAttnArgs) =
+    CUtensorMap tmap_y = tmap;                        // (unused by the variant that stores O)
+    if (fuse_out) {
+        const cuuint32_t ybox[3] = {32, ROWS, 1};
+        r = enc(&tmap_y, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, y, dims, strides, ybox, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+    }
+    void (*kern)(const CUtensorMap, const CUtensorMap, const QAttnArgs) =
         fuse_out ? (tail ? qattn_c320_kernel<true, true> : qattn_c320_kernel<false, true>) : (tail ? qattn_c320_kernel<true, false> : qattn_c320_kernel<false, false>);
     const int ci = (tail ? 1 : 0) + (fuse_out ? 2 : 0);
     if (!configured[ci]) {
@@ -728,8 +739,8 @@ static cudaError_t launch_c320(const taq_layer_desc& d, const __half* x, const v
         if (e != cudaSuccess) return e;
         configured[ci] = true;
     }
-    if (fuse_out) return launch_pdl_cluster(kern, grid, dim3(1, 2, 1), dim3(NTHREADS), (size_t)TOTAL, stream, tmap, a);
-    return launch_pdl(kern, grid, dim3(NTHREADS), (size_t)TOTAL, stream, tmap, a);
+    if (fuse_out) return launch_pdl_cluster(kern, grid, dim3(1, 2, 1), dim3(NTHREADS), (size_t)TOTAL, stream, tmap, tmap_y, a);
+    return launch_pdl(kern, grid, dim3(NTHREADS), (size_t)TOTAL, stream, tmap, tmap_y, a);
 }
 
 cudaError_t launch_qattn_sm100(const taq_layer_desc& d, const __half* x, const void* wq, const void* kv, const taq_request* reqs, __half* o,
