@@ -116,6 +116,35 @@ __device__ __forceinline__ int o_pieces(int h_begin, int (&first)[MAX_PIECES], i
     return 3;
 }
 
+// Expands the packed 4-bit codes at OFF_RAW into the ring of fp16 weight tiles, K block by K block (all worker threads).
+// One copy of this code serves phase 1 and phase 4.  Takes and returns the ring position: bits 0..1 stage, bit 2 pass
+// parity, bit 3 set when a wait ran out.
+__device__ __noinline__ uint32_t build_weight_tiles(unsigned char* smem, Misc* misc, int first_pass, int wt, int lane, int s, uint32_t ph) {
+    const unsigned char* raw = smem + OFF_RAW;
+    bool ok = true;
+    for (int kb = 0; kb < NKB; ++kb) {
+        if ((!first_pass || kb >= NBSTAGE) && !ptx::mbar_wait(&misc->b_empty[s], ph ^ 1)) ok = false;
+        if (!ok || misc->abort_flag) { ok = false; break; }
+        unsigned char* b_tile = smem + OFF_B + s * B_TILE;
+        constexpr int NCH = (NQ * 8 + NWORK - 1) / NWORK;       // 16-byte chunks (8 weights) per thread and K block
+        const int n0 = wt >> 3, c = wt & 7;
+        uint32_t pw[NCH];
+#pragma unroll
+        for (int i = 0; i < NCH; ++i) {
+            pw[i] = 0;
+            if (n0 + (NWORK / 8) * i < NQ) pw[i] = *reinterpret_cast<const uint32_t*>(raw + (n0 + (NWORK / 8) * i) * (KIN / 2) + kb * (BK / 2) + c * 4);
+        }
+#pragma unroll
+        for (int i = 0; i < NCH; ++i)
+            if (n0 + (NWORK / 8) * i < NQ) *reinterpret_cast<uint4*>(b_tile + ptx::sw128_offset(n0 + (NWORK / 8) * i, c)) = codes_w4_to_half(pw[i]);
+        ptx::fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&misc->b_full[s]);
+        if (++s == NBSTAGE) { s = 0; ph ^= 1; }
+    }
+    return (uint32_t)s | (ph << 2) | (ok ? 0u : 8u);
+}
+
 template <bool TAIL_ONLY, bool FUSE_OUT>
 __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_y, const QAttnArgs a) {
     extern __shared__ unsigned char smem_dyn[];
@@ -409,29 +438,10 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
         const int cb = part * HC;
         int s = 0;                                           // weight ring position and pass parity, continued in phase 4
         uint32_t ph = 0;
-        auto build_tiles = [&](int first_pass) {             // expand the packed codes at OFF_RAW into the ring, K block by K block
-            for (int kb = 0; kb < NKB && ok; ++kb) {
-                if ((!first_pass || kb >= NBSTAGE) && !ptx::mbar_wait(&misc->b_empty[s], ph ^ 1)) ok = false;
-                if (!ok || misc->abort_flag) { ok = false; break; }
-                if (wt == 0) TAQ_PROF((first_pass ? 95 : 90) + kb);
-                unsigned char* b_tile = smem + OFF_B + s * B_TILE;
-                constexpr int NCH = (NQ * 8 + NWORK - 1) / NWORK;       // 16-byte chunks (8 weights) per thread and K block
-                const int n0 = wt >> 3, c = wt & 7;
-                uint32_t pw[NCH];
-#pragma unroll
-                for (int i = 0; i < NCH; ++i) {
-                    pw[i] = 0;
-                    if (n0 + (NWORK / 8) * i < NQ) pw[i] = *reinterpret_cast<const uint32_t*>(raw + (n0 + (NWORK / 8) * i) * (KIN / 2) + kb * (BK / 2) + c * 4);
-                }
-#pragma unroll
-                for (int i = 0; i < NCH; ++i)
-                    if (n0 + (NWORK / 8) * i < NQ) *reinterpret_cast<uint4*>(b_tile + ptx::sw128_offset(n0 + (NWORK / 8) * i, c)) = codes_w4_to_half(pw[i]);
-                ptx::fence_proxy_async_smem();
-                __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(&misc->b_full[s]);
-                if (wt == 0) TAQ_PROF((first_pass ? 85 : 80) + kb);
-                if (++s == NBSTAGE) { s = 0; ph ^= 1; }
-            }
+        auto build_tiles = [&](int first_pass) {
+            const uint32_t st = build_weight_tiles(smem, misc, first_pass, wt, lane, s, ph);
+            s = (int)(st & 3u); ph = (st >> 2) & 1u;
+            if (st >> 3) ok = false;
         };
         auto fold_groups = [&](uint32_t parity) {            // y += scale[g] * accumulator g, as each group completes
         for (int g = 0; g < n_groups && ok; ++g) {             // later groups are still being multiplied while this one is folded
