@@ -151,48 +151,58 @@ __global__ void __launch_bounds__(ATT_THREADS, Cfg<D>::CTAS_PER_SM) attention_sm
         }
     } else if (warp == MMA_WARP) {
         // ---------------- MMA issuer ----------------
-        if (lane == 0) {
-            const uint32_t q_addr = ptx::smem_u32(smem + C::OFF_Q), p_addr = ptx::smem_u32(smem + C::OFF_P);
-            auto issue_s = [&](int hi) -> bool {
-                const int buf = hi % C::KVBUF;
-                if (!ptx::mbar_wait(&misc->kv_full[buf], (hi / C::KVBUF) & 1) || !ptx::mbar_wait(&misc->q_full, hi & 1)) return false;
-                ptx::tc_fence_after_sync();
-                const uint32_t k_addr = ptx::smem_u32(smem + C::OFF_KV + buf * C::HEAD_BYTES);
+        // All 32 lanes walk the control flow (warp-uniform loop state and descriptor words); one elected lane issues.
+        const bool leader = ptx::elect_one();
+        auto wait = [&](uint64_t* bar, uint32_t parity) -> bool { return __all_sync(0xffffffffu, ptx::mbar_wait(bar, parity) && !misc->abort_flag) != 0; };
+        constexpr uint32_t HI = ptx::kDescHiSw128;
+        const uint32_t q_lo0 = ptx::desc_lo(ptx::smem_u32(smem + C::OFF_Q)), p_lo0 = ptx::desc_lo(ptx::smem_u32(smem + C::OFF_P));
+        const uint32_t kv_lo0 = ptx::desc_lo(ptx::smem_u32(smem + C::OFF_KV));
+        auto issue_s = [&](int hi) -> bool {
+            const int buf = hi % C::KVBUF;
+            if (!wait(&misc->kv_full[buf], (hi / C::KVBUF) & 1) || !wait(&misc->q_full, hi & 1)) return false;
+            ptx::tc_fence_after_sync();
+            if (leader) {
+                const uint32_t k_lo = kv_lo0 + buf * (C::HEAD_BYTES >> 4);
 #pragma unroll
                 for (int ks = 0; ks < DP / 16; ++ks)
-                    ptx::mma_f16_ss(tmem_base + C::TMEM_S + (hi & 1) * TP, ptx::desc_k_sw128(q_addr + (ks / 4) * C::A_BLOCK + (ks % 4) * 32),
-                                    ptx::desc_k_sw128(k_addr + (ks / 4) * C::K_BLOCK + (ks % 4) * 32), ptx::idesc_f16_m128(TP), ks != 0);
+                    ptx::mma_f16_ss(tmem_base + C::TMEM_S + (hi & 1) * TP, ptx::desc_join(HI, q_lo0 + (ks / 4) * (C::A_BLOCK >> 4) + (ks % 4) * 2),
+                                    ptx::desc_join(HI, k_lo + (ks / 4) * (C::K_BLOCK >> 4) + (ks % 4) * 2), ptx::idesc_f16_m128(TP), ks != 0);
                 ptx::mma_commit(&misc->s_full[hi & 1]);
-                return true;
-            };
-            auto issue_pv = [&](int hi) -> bool {
-                const int buf = hi % C::KVBUF;
-                if (!ptx::mbar_wait(&misc->p_full, hi & 1)) return false;
-                ptx::tc_fence_after_sync();
-                const uint32_t vt_addr = ptx::smem_u32(smem + C::OFF_KV + buf * C::HEAD_BYTES + C::K_BYTES);
+            }
+            return true;
+        };
+        auto issue_pv = [&](int hi) -> bool {
+            const int buf = hi % C::KVBUF;
+            if (!wait(&misc->p_full, hi & 1)) return false;
+            ptx::tc_fence_after_sync();
+            if (leader) {
+                const uint32_t vt_lo = kv_lo0 + ((buf * C::HEAD_BYTES + C::K_BYTES) >> 4);
 #pragma unroll
                 for (int ks = 0; ks < TP / 16; ++ks)
-                    ptx::mma_f16_ss(tmem_base + C::TMEM_O + (hi % C::OBUF) * DP, ptx::desc_k_sw128(p_addr + (ks / 4) * C::A_BLOCK + (ks % 4) * 32),
-                                    ptx::desc_k_sw128(vt_addr + (ks / 4) * C::VT_BLOCK + (ks % 4) * 32), ptx::idesc_f16_m128(DP), ks != 0);
+                    ptx::mma_f16_ss(tmem_base + C::TMEM_O + (hi % C::OBUF) * DP, ptx::desc_join(HI, p_lo0 + (ks / 4) * (C::A_BLOCK >> 4) + (ks % 4) * 2),
+                                    ptx::desc_join(HI, vt_lo + (ks / 4) * (C::VT_BLOCK >> 4) + (ks % 4) * 2), ptx::idesc_f16_m128(DP), ks != 0);
                 ptx::mma_commit(&misc->o_full[hi % C::OBUF]);
                 ptx::mma_commit(&misc->kv_free[buf]);
-                return true;
-            };
-            bool ok = issue_s(0);
-            for (int hi = 0; hi < HG && ok && !misc->abort_flag; ++hi) {
-                if (C::KVBUF == 2) {          // S of the next head first: it runs under this head's softmax
-                    if (hi + 1 < HG) ok = issue_s(hi + 1);
-                    if (ok) ok = issue_pv(hi);
-                } else {                      // one K~/V~ buffer: the next head's image lands only after this PV
-                    ok = issue_pv(hi);
-                    if (ok && hi + 1 < HG) ok = issue_s(hi + 1);
-                }
             }
-            if (!ok) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; }
-            if (misc->abort_flag) {           // wait (bounded) for whatever was issued before TMEM is given back
+            return true;
+        };
+        bool ok = issue_s(0);
+        for (int hi = 0; hi < HG && ok; ++hi) {
+            if (C::KVBUF == 2) {          // S of the next head first: it runs under this head's softmax
+                if (hi + 1 < HG) ok = issue_s(hi + 1);
+                if (ok) ok = issue_pv(hi);
+            } else {                      // one K~/V~ buffer: the next head's image lands only after this PV
+                ok = issue_pv(hi);
+                if (ok && hi + 1 < HG) ok = issue_s(hi + 1);
+            }
+        }
+        if (!ok) {                        // wait (bounded) for whatever was issued before TMEM is given back
+            if (leader) {
+                raise_status(a.status, TAQ_ERR_TIMEOUT);
+                misc->abort_flag = 1;
                 ptx::mma_commit(&misc->drain);
-                (void)ptx::mbar_wait(&misc->drain, 0);
             }
+            (void)ptx::mbar_wait(&misc->drain, 0);
         }
     } else {
         // ---------------- row threads: two per query row (TMEM lane), each with half of the keys ----------------

@@ -152,37 +152,42 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer: one accumulation pass per scale group ----------------
-        if (lane == 0) {
-            constexpr uint32_t idesc = ptx::idesc_f16_m128(BN);
-            int s = 0, kb = 0;
-            uint32_t ph = 0;
-            bool ok = true;
-            for (int g = 0; g < n_groups && ok; ++g) {
-                const int buf = g & 1;
-                if (g >= 2 && !ptx::mbar_wait(&bars->acc_free[buf], ((g >> 1) - 1) & 1)) ok = false;   // the workers have emptied this accumulator
+        // All 32 lanes walk the control flow, so that loop state and descriptor words stay warp-uniform; one elected lane
+        // issues.  The path between two MMAs is kept short: this warp shares its scheduler with worker warps.
+        const bool leader = ptx::elect_one();
+        auto wait = [&](uint64_t* bar, uint32_t parity) -> bool { return __all_sync(0xffffffffu, ptx::mbar_wait(bar, parity) && !bars->abort_flag) != 0; };
+        constexpr uint32_t idesc = ptx::idesc_f16_m128(BN);
+        constexpr uint32_t HI = ptx::kDescHiSw128;
+        const uint32_t lo0 = ptx::desc_lo(ptx::smem_u32(smem));
+        int s = 0, kb = 0;
+        uint32_t ph = 0;
+        bool ok = true;
+        for (int g = 0; g < n_groups && ok; ++g) {
+            const int buf = g & 1;
+            if (g >= 2) {                                   // the workers have emptied this accumulator
+                if (!wait(&bars->acc_free[buf], ((g >> 1) - 1) & 1)) { ok = false; break; }
                 ptx::tc_fence_after_sync();
-                const int kb_end = min(n_kb, kb + kb_per_group);
-                for (bool first = true; kb < kb_end && ok; ++kb) {
-                    if (!ptx::mbar_wait(&bars->full_a[s], ph) || !ptx::mbar_wait(&bars->full_b[s], ph) || bars->abort_flag) { ok = false; break; }
-                    ptx::tc_fence_after_sync();
-                    const uint32_t a_addr = ptx::smem_u32(smem + s * TL::STAGE_BYTES);
-                    const uint32_t b_addr = a_addr + A_TILE_BYTES;
+            }
+            const int kb_end = min(n_kb, kb + kb_per_group);
+            for (bool first = true; kb < kb_end && ok; ++kb) {
+                if (!wait(&bars->full_a[s], ph) || !wait(&bars->full_b[s], ph)) { ok = false; break; }
+                if (leader) {
+                    const uint32_t a_lo = lo0 + s * (TL::STAGE_BYTES >> 4), b_lo = a_lo + (A_TILE_BYTES >> 4);
 #pragma unroll
-                    for (int k = 0; k < BK / 16; ++k) {
-                        ptx::mma_f16_ss(tmem_base + buf * BN, ptx::desc_k_sw128(a_addr + k * 32), ptx::desc_k_sw128(b_addr + k * 32), idesc, !(first && k == 0));
-                    }
-                    first = false;
+                    for (int k = 0; k < BK / 16; ++k)
+                        ptx::mma_f16_ss(tmem_base + buf * BN, ptx::desc_join(HI, a_lo + 2 * k), ptx::desc_join(HI, b_lo + 2 * k), idesc, !(first && k == 0));
                     ptx::mma_commit(&bars->empty[s]);       // frees the stage once these MMAs have read it
-                    if (++s == nstage) { s = 0; ph ^= 1; }
+                    if (kb + 1 == kb_end) ptx::mma_commit(&bars->acc_full[buf]);
                 }
-                if (ok) ptx::mma_commit(&bars->acc_full[buf]);
+                first = false;
+                if (++s == nstage) { s = 0; ph ^= 1; }
             }
-            if (!ok) {
-                raise_status(a.status, TAQ_ERR_TIMEOUT);
-                bars->abort_flag = 1;
-                ptx::mma_commit(&bars->acc_full[0]);        // wake the workers; they see the abort flag
-                ptx::mma_commit(&bars->acc_full[1]);
-            }
+        }
+        if (!ok && leader) {
+            raise_status(a.status, TAQ_ERR_TIMEOUT);
+            bars->abort_flag = 1;
+            ptx::mma_commit(&bars->acc_full[0]);        // wake the workers; they see the abort flag
+            ptx::mma_commit(&bars->acc_full[1]);
         }
     } else {
         // ---------------- workers (warps 2..9) ----------------
