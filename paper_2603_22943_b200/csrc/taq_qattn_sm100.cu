@@ -41,7 +41,6 @@ constexpr int A_TILE = ROWS * 128;              // 16 KB: one 64-wide K block of
 constexpr int B_TILE = NQ * 128;                // 20 KB
 constexpr int K_BLOCK = TP * 128, VT_BLOCK = DP * 128;
 constexpr int K_BYTES = K_BLOCK, VT_BYTES = 2 * VT_BLOCK;
-constexpr int HEAD_BYTES = K_BYTES + VT_BYTES + kOperandConstBytes;     // 23552
 constexpr int MAX_GROUPS = 3;                    // one TMEM accumulator of NQ columns per scale group
 constexpr int RAW_BYTES = NQ * (KIN / 2);       // 25600 (W4)
 constexpr int SCALE_BYTES = ((NQ * MAX_GROUPS * 4 + 127) / 128) * 128;
@@ -424,7 +423,6 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
         const bool valid = n < a.n_query;
         const size_t grow = (size_t)zb * a.n_query + (valid ? n : 0);
         const uint32_t lane_addr = (uint32_t)(q4 * 32) << 16;
-        const unsigned char* raw = smem + OFF_RAW;
         const float* wscales = reinterpret_cast<const float*>(smem + OFF_SC);
         float* scales_t = reinterpret_cast<float*>(smem + OFF_SCT);
         bool ok = ptx::mbar_wait(&misc->w_full, 0);
@@ -530,7 +528,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
         bool alive = ok;
         auto store_o = [&](int hi) {
             const bool stamp = lane == 0 && q4 == 0 && half == 0;
-            const int sb = 45 + 5 * grp + (hi >= 2 ? 3 : 0);
+            [[maybe_unused]] const int sb = 45 + 5 * grp + (hi >= 2 ? 3 : 0);
             if (stamp) TAQ_PROF(sb);
             __half* orow = a.o + grow * (size_t)(H * D) + (h_begin + hi) * D + half * OC;
             const uint32_t t_o = tmem_base + TMEM_O + grp * DP + half * OC + lane_addr;
