@@ -23,6 +23,13 @@ fixed by the benchmark configuration: symmetric, dynamic, round-to-nearest-even;
 The quantizer itself is evaluated in IEEE binary32 (numpy float32, no fused multiply-add), because
 integer codes are compared bit for bit; everything else is float64.
 
+Integer activations (``a_bits = 8``): the paper's W/A bit-widths (Table 1, "W/A" column) and its BOPs
+accounting count activation bits for every layer, which read literally means that the inputs of the four
+projections - the hidden states X, the text context and the attention output O - are quantized too.  With
+``a_bits = 8`` each token's row of all C (or Dc) channels passes through the same symmetric int8 quantizer
+before its projection, so that a projection is an integer product scaled by (row scale) x (weight scale).
+``a_bits = 0`` (the default, and the configuration the benchmark names) leaves these inputs in fp16.
+
 Two modes.  ``ideal``: the equations in real (float64) arithmetic, quantizers as above, no other
 rounding.  ``contract``: the same, plus a round-to-nearest-even to fp16 wherever the layer stores an
 fp16 value ("full precision" of the trigger pathway is fp16 storage; dequantized V rows are fp16
@@ -137,6 +144,7 @@ class TaqConfig:
     q_bits: int = 8          # 8 = Eq. 2's Q~ = Q_a(Q); 0 = Q left unquantized
     kv_bits: int = 8         # 8 = non-trigger K/V rows int8; 0 = no K/V quantization at all
     p_bits: int = 8          # 8 = non-trigger probabilities uint8; 0 = no probability quantization
+    a_bits: int = 0          # 8 = inputs of the projections (X, ctx, O) int8 per token; 0 = left in fp16
     contract: bool = True    # fp16 storage roundings on (contract) or off (ideal)
 
 
@@ -146,6 +154,18 @@ def effective_weight(W: np.ndarray, cfg: TaqConfig) -> np.ndarray:
         return np.asarray(W, dtype=F64)
     codes, scales = quantize_weights(W, cfg.w_bits, cfg.w_group)
     return dequantize_weights(codes, scales, cfg.w_group, cfg.contract)
+
+
+def quantize_activations(x: np.ndarray, cfg: TaqConfig) -> np.ndarray:
+    """Input of a projection under ``a_bits``: x~ = q * s with (q, s) = Q_a(row), one row per token over all of
+    its channels; the product is exact (the projection multiplies the integer codes and applies s afterwards)."""
+    x = np.asarray(x, dtype=F64)
+    if cfg.a_bits == 0:
+        return x
+    if cfg.a_bits != 8:
+        raise ValueError("a_bits must be 0 or 8")
+    codes, scales = quantize_rows(x.astype(F32), 127)
+    return codes.astype(F64) * scales.astype(F64)[..., None]
 
 
 def split_heads(x: np.ndarray, heads: int) -> np.ndarray:
@@ -166,7 +186,7 @@ def taq_kv(ctx: np.ndarray, Wk: np.ndarray, Wv: np.ndarray, mask_kv: np.ndarray,
     ctx [B,T,Dc] (fp16 data), Wk/Wv [C,Dc] float32, mask_kv [B,T] (1 = trigger row kept).
     Returns K~, V~ as float64 [B,H,T,d] plus the integer codes / scales of the quantized rows.
     """
-    ctx = np.asarray(ctx, dtype=F64)
+    ctx = quantize_activations(ctx, cfg)
     K = split_heads(ctx @ effective_weight(Wk, cfg).T, cfg.heads)
     V = split_heads(ctx @ effective_weight(Wv, cfg).T, cfg.heads)
     M = (np.asarray(mask_kv) != 0)[:, None, :, None]           # broadcast over heads and channels
@@ -189,7 +209,7 @@ def taq_kv(ctx: np.ndarray, Wk: np.ndarray, Wv: np.ndarray, mask_kv: np.ndarray,
 
 def taq_q(X: np.ndarray, Wq: np.ndarray, cfg: TaqConfig) -> Dict[str, np.ndarray]:
     """Query projection and Eq. 2 (third line): Q~ = Q_a(Q) per (batch, head, token) row."""
-    X = np.asarray(X, dtype=F64)
+    X = quantize_activations(X, cfg)
     Q = split_heads(X @ effective_weight(Wq, cfg).T, cfg.heads)
     if cfg.q_bits == 0:
         Qt = f16_round(Q) if cfg.contract else Q                  # unquantized Q is an fp16 tensor
@@ -229,7 +249,7 @@ def taq_attention(Q_tilde: np.ndarray, K_tilde: np.ndarray, V_tilde: np.ndarray,
 
 
 def taq_out(O: np.ndarray, Wout: np.ndarray, bout: Optional[np.ndarray], cfg: TaqConfig) -> np.ndarray:
-    Y = np.asarray(O, dtype=F64) @ effective_weight(Wout, cfg).T
+    Y = quantize_activations(O, cfg) @ effective_weight(Wout, cfg).T
     if bout is not None:
         Y = Y + np.asarray(bout, dtype=F64)
     return f16_round(Y) if cfg.contract else Y

@@ -408,9 +408,78 @@ def check_contract_close_to_ideal(o):
     assert np.array_equal(yc, yc.astype(np.float16).astype(np.float64))      # Y is fp16 data
 
 
+def check_integer_activations(o):
+    """a_bits = 8 (the W/A reading of Table 1: the inputs of the projections are int8 per token).
+    (i) the projection is an integer product: Q[b,n,c] = s_x[b,n] * sum_g s_w[c,g] * sum_{k in g} xq[b,n,k] wq[c,k],
+    checked in exact rational arithmetic; (ii) inputs that already lie on an int8 grid whose largest code is 127 pass
+    through unchanged, so the layer equals the a_bits = 0 layer; (iii) |x - x~| <= s/2, one scale per token."""
+    B, N, H, d, T, Dc = 1, 3, 2, 8, 4, 16
+    X, ctx, Wq, Wk, Wv, Wo, bo = _tiny_layer(41, B=B, N=N, H=H, d=d, T=T, Dc=Dc)
+    C = H * d
+    cfg = o.TaqConfig(heads=H, w_bits=4, w_group=8, q_bits=0, a_bits=8, contract=False)
+    Q = o.merge_heads(o.taq_q(X, Wq, cfg)["Q"])
+    xq, sx = o.quantize_rows(X.astype(np.float32), 127)
+    wq, sw = o.quantize_weights(Wq, 4, 8)
+    assert sx.shape == (B, N) and np.all(np.max(np.abs(xq), axis=-1) == 127)
+    for n in range(N):
+        for c in range(C):
+            acc = Fraction(0)
+            for g in range(C // 8):
+                part = sum(int(xq[0, n, k]) * int(wq[c, k]) for k in range(8 * g, 8 * g + 8))
+                acc += Fraction(float(sw[c, g])) * part
+            want = float(Fraction(float(sx[0, n])) * acc)
+            assert abs(Q[0, n, c] - want) <= 1e-12 * max(1.0, abs(want))
+    # the same for to_out (with its bias) and for the K projection of the text context
+    Oin = X
+    Y = o.taq_out(Oin, Wo, bo, cfg)
+    wo, swo = o.quantize_weights(Wo, 4, 8)
+    for n in range(N):
+        for c in range(0, C, 5):
+            acc = sum(Fraction(float(swo[c, g])) * sum(int(xq[0, n, k]) * int(wo[c, k]) for k in range(8 * g, 8 * g + 8)) for g in range(C // 8))
+            want = float(Fraction(float(sx[0, n])) * acc + Fraction(float(bo[c])))
+            assert abs(Y[0, n, c] - want) <= 1e-12 * max(1.0, abs(want))
+    cq, sc = o.quantize_rows(ctx.astype(np.float32), 127)
+    wk, swk = o.quantize_weights(Wk, 4, 8)
+    K = o.merge_heads(o.taq_kv(ctx, Wk, Wv, np.zeros((B, T), np.uint8), cfg)["K"])
+    for t in range(T):
+        for c in range(0, C, 3):
+            acc = sum(Fraction(float(swk[c, g])) * sum(int(cq[0, t, k]) * int(wk[c, k]) for k in range(8 * g, 8 * g + 8)) for g in range(Dc // 8))
+            want = float(Fraction(float(sc[0, t])) * acc)
+            assert abs(K[0, t, c] - want) <= 1e-12 * max(1.0, abs(want))
+    xt = o.quantize_activations(X, cfg)
+    assert np.all(np.abs(xt - X.astype(np.float64)) <= sx[..., None].astype(np.float64) * 0.5000001)
+    # (ii) grid inputs: codes with absmax 127 times a power of two are fixed points of the quantizer
+    r = _rng(42)
+    def grid(shape):
+        c = r.integers(-127, 128, size=shape)
+        c[..., 0] = 127
+        return (c * 2.0 ** -6).astype(np.float16)
+    Xg, ctxg = grid((B, N, C)), grid((B, T, Dc))
+    mask = np.zeros((B, T), np.uint8); mask[0, 1] = 1
+    base = dict(heads=H, w_bits=4, w_group=8, contract=False)
+    q0 = o.taq_q(Xg, Wq, o.TaqConfig(a_bits=0, **base))
+    q8 = o.taq_q(Xg, Wq, o.TaqConfig(a_bits=8, **base))
+    np.testing.assert_allclose(q8["Q"], q0["Q"], rtol=1e-13, atol=0)
+    k0 = o.taq_kv(ctxg, Wk, Wv, mask, o.TaqConfig(a_bits=0, **base))
+    k8 = o.taq_kv(ctxg, Wk, Wv, mask, o.TaqConfig(a_bits=8, **base))
+    np.testing.assert_allclose(k8["K"], k0["K"], rtol=1e-13, atol=0)
+    np.testing.assert_allclose(k8["V"], k0["V"], rtol=1e-13, atol=0)
+    Og = grid((B, N, C))
+    np.testing.assert_allclose(o.taq_out(Og, Wo, bo, o.TaqConfig(a_bits=8, **base)), o.taq_out(Og, Wo, bo, o.TaqConfig(a_bits=0, **base)), rtol=1e-13, atol=1e-15)
+    # and on ordinary inputs the integer-activation layer stays close to the fp16-activation layer
+    X2, ctx2, Wq2, Wk2, Wv2, Wo2, bo2 = _tiny_layer(43, B=1, N=16, H=2, d=16, T=9, Dc=32)
+    m2 = np.zeros((1, 9), np.uint8); m2[0, 3] = 1
+    y0 = o.taq_layer(X2, ctx2, Wq2, Wk2, Wv2, Wo2, bo2, m2, o.TaqConfig(heads=2, w_bits=8, a_bits=0))["Y"]
+    y8 = o.taq_layer(X2, ctx2, Wq2, Wk2, Wv2, Wo2, bo2, m2, o.TaqConfig(heads=2, w_bits=8, a_bits=8))["Y"]
+    rel = np.linalg.norm(y8 - y0) / np.linalg.norm(y0)
+    assert 0 < rel < 0.05
+    with pytest.raises(ValueError):
+        o.quantize_activations(X, o.TaqConfig(heads=H, a_bits=4))
+
+
 LAYER_CHECKS = [check_all_trigger_is_textbook_attention, check_empty_mask_is_uniform_quantization,
                 check_trigger_rows_pass_through, check_closed_forms, check_structure, check_brute_force,
-                check_contract_close_to_ideal]
+                check_contract_close_to_ideal, check_integer_activations]
 
 
 @pytest.mark.parametrize("check", LAYER_CHECKS)
@@ -476,6 +545,11 @@ MUTATIONS = {
     "renormalised_probs": [("A_hat = np.where(M, kept, Aq)                             # Eq. 3",
                             "A_hat = np.where(M, kept, Aq); A_hat = A_hat / A_hat.sum(-1, keepdims=True)")],
     "group_ignored": [("g = k_in if group == 0 else group\n    n_groups", "g = k_in\n    n_groups")],
+    "activation_scale_dropped": [("return codes.astype(F64) * scales.astype(F64)[..., None]", "return codes.astype(F64)")],
+    "activations_not_quantized": [("    if cfg.a_bits == 0:\n        return x\n", "    if True:\n        return x\n")],
+    "out_input_not_quantized": [("Y = quantize_activations(O, cfg) @ effective_weight(Wout, cfg).T", "Y = np.asarray(O, dtype=F64) @ effective_weight(Wout, cfg).T")],
+    "activation_scale_per_tensor": [("    codes, scales = quantize_rows(x.astype(F32), 127)\n    return codes.astype(F64) * scales",
+                                     "    codes, scales = quantize_rows(x.astype(F32).reshape(1, -1), 127)\n    codes = codes.reshape(x.shape); scales = np.broadcast_to(scales, x.shape[:-1])\n    return codes.astype(F64) * scales")],
     "heads_interleaved": [("return x.reshape(B, L, heads, d).transpose(0, 2, 1, 3)", "return x.reshape(B, L, d, heads).transpose(0, 3, 1, 2)")],
 }
 
