@@ -193,6 +193,45 @@ taq_status taq_layer_forward(const taq_layer_desc* desc, const void* x_f16_dev, 
                              const uint8_t* trig_mask_dev, void* y_f16_dev, void* workspace_dev,
                              size_t workspace_bytes, void* stream);
 
+/* --------------------------------------------------------------------------------------------------------
+ * Integer-activation projections ("W8A8", "W4A8": the W/A column of Table 1 and the BOPs accounting of
+ * Sec. IV count activation bits for every layer; Sec. III-B last paragraph: "remaining ... pathways" are
+ * quantized).  Read literally, the inputs of the four projections - hidden states X, text context, attention
+ * output O - are int8 as well: each token's row of all its channels goes through the symmetric quantizer Q_a
+ * of Eq. 2 (one fp32 scale per token), and a projection is an exact int8 x int8 -> int32 product on the tensor
+ * cores, one accumulation per weight scale group, times (weight scale) x (token scale) in fp32.  The entry
+ * points above keep these inputs in fp16 (the configuration the benchmark names); the ones below are the
+ * integer reading.  They need the tensor-core kernel: k_in a multiple of 16, group 0 or 128, n_out a multiple
+ * of 64 or 80; otherwise TAQ_ERR_UNSUPPORTED.
+ * -------------------------------------------------------------------------------------------------------- */
+
+/* Q_a per token on fp16 data: x fp16 [rows][cols] (cols a multiple of 8) -> int8 codes [rows][cols], fp32
+ * scales [rows].  Same arithmetic as taq_quantize_rows (qmax 127) on the fp16 values converted to fp32. */
+taq_status taq_quantize_rows_f16(const void* x_f16_dev, int64_t rows, int32_t cols, int8_t* codes_dev,
+                                 float* scales_dev, void* stream);
+
+/* y = (x_codes * x_scale) W^T (+ bias): the integer product described above.  x_codes_dev int8 [rows][k_in],
+ * x_scales_dev fp32 [rows]; W, y, out_kind, heads, scales_dev as for taq_quantized_linear. */
+taq_status taq_quantized_linear_i8(const taq_weight_desc* desc, const int8_t* x_codes_dev, const float* x_scales_dev,
+                                   int64_t rows, const void* W_packed_dev, void* y_dev, int32_t out_kind,
+                                   int32_t heads, float* scales_dev, void* stream);
+
+/* taq_layer_forward with int8 X and O: Q_a(X) per token, integer to_q (+ Q_a per head row), attention as
+ * before, Q_a(O) per token on the fp16 O, integer to_out (+ bias).  Five kernels; workspace_dev >=
+ * taq_workspace_bytes_a8(desc), 128-byte aligned. */
+size_t taq_workspace_bytes_a8(const taq_layer_desc* desc);
+taq_status taq_layer_forward_a8(const taq_layer_desc* desc, const void* x_f16_dev, const void* Wq_packed_dev,
+                                const void* Wout_packed_dev, const void* kv_packed_dev,
+                                const uint8_t* trig_mask_dev, void* y_f16_dev, void* workspace_dev,
+                                size_t workspace_bytes, void* stream);
+
+/* taq_kv_project with an int8 text context: Q_a(ctx) per token, integer to_k / to_v, Eq. 2 as before.
+ * workspace_dev >= taq_kv_project_a8_workspace_bytes(desc), 128-byte aligned (the context's codes and scales). */
+size_t taq_kv_project_a8_workspace_bytes(const taq_layer_desc* desc);
+taq_status taq_kv_project_a8(const taq_layer_desc* desc, const void* ctx_f16_dev, const void* Wk_packed_dev,
+                             const void* Wv_packed_dev, const uint8_t* trig_mask_dev, void* kv_packed_dev,
+                             size_t kv_bytes, void* workspace_dev, size_t workspace_bytes, void* stream);
+
 /* Batched serving (Sec. I: many personalized checkpoints served concurrently): request r is one sequence
  * (desc->batch must be 1) whose activations are slice r of x/y [n_requests][N][C] and which carries its own
  * checkpoint's packed weights, its own K~/V~ block and its own trigger mask.  `reqs_dev` is a DEVICE array of

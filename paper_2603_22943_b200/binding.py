@@ -25,6 +25,8 @@ EXPORTS = [
     "taq_quantized_linear", "taq_cross_attention", "taq_workspace_bytes", "taq_layer_forward",
     "taq_layer_forward_batched", "taq_kv_project_batched", "taq_poll_device_status",
     "taq_static_workspace_capacity", "taq_layer_forward_static", "taq_kv_finalize", "taq_query_attention",
+    "taq_quantize_rows_f16", "taq_quantized_linear_i8", "taq_workspace_bytes_a8", "taq_layer_forward_a8",
+    "taq_kv_project_a8_workspace_bytes", "taq_kv_project_a8",
 ]
 
 
@@ -96,6 +98,14 @@ def lib() -> C.CDLL:
         L.taq_static_workspace_capacity.restype = sz
         L.taq_static_workspace_capacity.argtypes = []
         L.taq_layer_forward_static.argtypes = [C.POINTER(LayerDesc), vp, vp, vp, vp, vp, vp, vp]
+        L.taq_quantize_rows_f16.argtypes = [vp, i64, i32, vp, vp, vp]
+        L.taq_quantized_linear_i8.argtypes = [C.POINTER(WeightDesc), vp, vp, i64, vp, vp, i32, i32, vp, vp]
+        L.taq_workspace_bytes_a8.restype = sz
+        L.taq_workspace_bytes_a8.argtypes = [C.POINTER(LayerDesc)]
+        L.taq_layer_forward_a8.argtypes = [C.POINTER(LayerDesc), vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.taq_kv_project_a8_workspace_bytes.restype = sz
+        L.taq_kv_project_a8_workspace_bytes.argtypes = [C.POINTER(LayerDesc)]
+        L.taq_kv_project_a8.argtypes = [C.POINTER(LayerDesc), vp, vp, vp, vp, vp, sz, vp, sz, vp]
         for name in EXPORTS:
             f = getattr(L, name)
             if f.restype is C.c_int and name not in ("taq_version",):
@@ -207,6 +217,61 @@ def taq_quantized_linear(desc: WeightDesc, x: torch.Tensor, W_packed: torch.Tens
         scales = torch.empty((rows, heads), dtype=torch.float32, device=x.device)
     _check(lib().taq_quantized_linear(C.byref(desc), _ptr(x), rows, _ptr(W_packed), _ptr(y), out_kind, heads, _ptr(scales), _stream(stream)))
     return (y, scales) if out_kind == TAQ_OUT_INT8_HEAD_ROWS else y
+
+
+def taq_quantize_rows_f16(x: torch.Tensor, stream=None):
+    """Q_a per token on fp16 data: returns (int8 codes of x's shape, fp32 scales without the last axis)."""
+    cols = x.shape[-1]
+    rows = x.numel() // cols
+    codes = torch.empty(x.shape, dtype=torch.int8, device=x.device)
+    scales = torch.empty(x.shape[:-1], dtype=torch.float32, device=x.device)
+    _check(lib().taq_quantize_rows_f16(_ptr(x), rows, cols, _ptr(codes), _ptr(scales), _stream(stream)))
+    return codes, scales
+
+
+def taq_quantized_linear_i8(desc: WeightDesc, x_codes: torch.Tensor, x_scales: torch.Tensor, W_packed: torch.Tensor,
+                            out_kind: int = TAQ_OUT_F16, heads: int = 1, y: Optional[torch.Tensor] = None,
+                            scales: Optional[torch.Tensor] = None, stream=None):
+    """The integer-activation projection: int8 codes and per-token scales in."""
+    rows = x_codes.numel() // desc.k_in
+    if y is None:
+        dt = {TAQ_OUT_F16: torch.float16, TAQ_OUT_F32: torch.float32, TAQ_OUT_INT8_HEAD_ROWS: torch.int8}[out_kind]
+        y = torch.empty((rows, desc.n_out), dtype=dt, device=x_codes.device)
+    if out_kind == TAQ_OUT_INT8_HEAD_ROWS and scales is None:
+        scales = torch.empty((rows, heads), dtype=torch.float32, device=x_codes.device)
+    _check(lib().taq_quantized_linear_i8(C.byref(desc), _ptr(x_codes), _ptr(x_scales), rows, _ptr(W_packed), _ptr(y), out_kind, heads,
+                                         _ptr(scales), _stream(stream)))
+    return (y, scales) if out_kind == TAQ_OUT_INT8_HEAD_ROWS else y
+
+
+def taq_workspace_bytes_a8(desc: LayerDesc) -> int:
+    return lib().taq_workspace_bytes_a8(C.byref(desc))
+
+
+def taq_layer_forward_a8(desc: LayerDesc, x: torch.Tensor, Wq_packed: torch.Tensor, Wout_packed: torch.Tensor, kv: torch.Tensor,
+                         trig_mask: torch.Tensor, y: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                         stream=None) -> torch.Tensor:
+    """The layer pass with int8 X and O (integer to_q and to_out)."""
+    if y is None:
+        y = torch.empty((desc.batch, desc.n_query, desc.channels), dtype=torch.float16, device=x.device)
+    if workspace is None:
+        workspace = torch.empty(max(taq_workspace_bytes_a8(desc), 128), dtype=torch.uint8, device=x.device)
+    _check(lib().taq_layer_forward_a8(C.byref(desc), _ptr(x), _ptr(Wq_packed), _ptr(Wout_packed), _ptr(kv), _ptr(trig_mask), _ptr(y),
+                                      _ptr(workspace), workspace.numel(), _stream(stream)))
+    return y
+
+
+def taq_kv_project_a8(desc: LayerDesc, ctx: torch.Tensor, Wk_packed: torch.Tensor, Wv_packed: torch.Tensor,
+                      trig_mask: torch.Tensor, kv: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                      stream=None) -> torch.Tensor:
+    """K/V projection with an int8 text context."""
+    if kv is None:
+        kv = torch.zeros(max(taq_kv_bytes(desc), 16), dtype=torch.uint8, device=ctx.device)
+    if workspace is None:
+        workspace = torch.empty(max(lib().taq_kv_project_a8_workspace_bytes(C.byref(desc)), 128), dtype=torch.uint8, device=ctx.device)
+    _check(lib().taq_kv_project_a8(C.byref(desc), _ptr(ctx), _ptr(Wk_packed), _ptr(Wv_packed), _ptr(trig_mask), _ptr(kv), kv.numel(),
+                                   _ptr(workspace), workspace.numel(), _stream(stream)))
+    return kv
 
 
 def taq_cross_attention(desc: LayerDesc, q: torch.Tensor, q_scales: Optional[torch.Tensor], kv: torch.Tensor,

@@ -382,6 +382,182 @@ taq_status taq_layer_forward(const taq_layer_desc* d, const void* x_f16_dev, con
                               workspace_dev, (cudaStream_t)stream);
 }
 
+// ---- integer-activation variants (a_bits = 8): per-token int8 inputs of the projections ----------------------------
+
+taq_status taq_quantize_rows_f16(const void* x_f16_dev, int64_t rows, int32_t cols, int8_t* codes_dev, float* scales_dev, void* stream) {
+    if (rows < 0 || cols < 8 || cols % 8) return fail(TAQ_ERR_SHAPE, "rows >= 0 and cols a positive multiple of 8 required (rows=%lld cols=%d)", (long long)rows, cols);
+    if (rows == 0) return TAQ_OK;
+    TAQ_REQUIRE_PTR(x_f16_dev);
+    TAQ_REQUIRE_PTR(codes_dev);
+    TAQ_REQUIRE_PTR(scales_dev);
+    cudaError_t e = launch_quantize_rows_f16((const __half*)x_f16_dev, rows, cols, codes_dev, scales_dev, (cudaStream_t)stream);
+    return e == cudaSuccess ? TAQ_OK : cuda_fail(e, "quantize_rows_f16 launch");
+}
+
+static taq_status run_linear_i8(const LinearArgs& a, cudaStream_t st) {
+    if (!sm100_linear_supported(a))
+        return fail(TAQ_ERR_UNSUPPORTED, "integer-activation GEMM: needs k_in a multiple of 16, group 0 or 128, n_out a multiple of 64 or 80 (per-head output: head width 40, 64, 80 or 160)");
+    cudaError_t e = launch_linear_sm100(a, 1, st);
+    return e == cudaSuccess ? TAQ_OK : cuda_fail(e, "integer-activation GEMM launch");
+}
+
+taq_status taq_quantized_linear_i8(const taq_weight_desc* d, const int8_t* x_codes_dev, const float* x_scales_dev, int64_t rows,
+                                   const void* W_packed_dev, void* y_dev, int32_t out_kind, int32_t heads, float* scales_dev, void* stream) {
+    taq_status s = check_weight_desc(d);
+    if (s != TAQ_OK) return s;
+    if (rows < 0 || rows > (1LL << 31) - 1) return fail(TAQ_ERR_SHAPE, "rows out of range");
+    if (out_kind != TAQ_OUT_F16 && out_kind != TAQ_OUT_F32 && out_kind != TAQ_OUT_INT8_HEAD_ROWS) return fail(TAQ_ERR_INVALID_ARG, "unknown out_kind %d", out_kind);
+    if (out_kind == TAQ_OUT_INT8_HEAD_ROWS) {
+        if (heads < 1 || d->n_out % heads) return fail(TAQ_ERR_SHAPE, "n_out (%d) must be a multiple of heads (%d)", d->n_out, heads);
+        if (heads > 65535) return fail(TAQ_ERR_SHAPE, "too many heads");
+    }
+    if (rows == 0) return TAQ_OK;
+    TAQ_REQUIRE_PTR(x_codes_dev);
+    TAQ_REQUIRE_PTR(x_scales_dev);
+    TAQ_REQUIRE_PTR(W_packed_dev);
+    TAQ_REQUIRE_PTR(y_dev);
+    if (out_kind == TAQ_OUT_INT8_HEAD_ROWS) TAQ_REQUIRE_PTR(scales_dev);
+    int* status = nullptr;
+    s = status_ptr(&status);
+    if (s != TAQ_OK) return s;
+    LinearArgs a{};
+    a.xq = x_codes_dev; a.x_scales = x_scales_dev;
+    a.w = W_packed_dev;
+    a.y = y_dev;
+    a.scales = scales_dev;
+    a.rows = rows;
+    a.n_out = d->n_out; a.k_in = d->k_in; a.bits = d->bits; a.group = d->group;
+    a.heads = out_kind == TAQ_OUT_INT8_HEAD_ROWS ? heads : 1;
+    a.epi = out_kind == TAQ_OUT_F16 ? EPI_F16 : out_kind == TAQ_OUT_F32 ? EPI_F32 : EPI_Q8_HEAD;
+    a.status = status;
+    return run_linear_i8(a, (cudaStream_t)stream);
+}
+
+// Workspace of the integer-activation layer pass: activation codes and scales (X, later O), then the sections of the
+// ordinary pass.
+struct WorkspaceA8 { size_t off_xq, off_xs, base, total; };
+static WorkspaceA8 workspace_a8_layout(const taq_layer_desc* d) {
+    const size_t rows = (size_t)d->batch * d->n_query;
+    WorkspaceA8 w;
+    w.off_xq = 0;
+    w.off_xs = align_up(rows * d->channels, 128);
+    w.base = w.off_xs + align_up(rows * sizeof(float), 128);
+    w.total = w.base + workspace_layout(d, 1).total;
+    return w;
+}
+
+size_t taq_workspace_bytes_a8(const taq_layer_desc* d) {
+    if (check_layer_desc(d) != TAQ_OK) return 0;
+    return workspace_a8_layout(d).total;
+}
+
+taq_status taq_layer_forward_a8(const taq_layer_desc* d, const void* x_f16_dev, const void* Wq_packed_dev, const void* Wout_packed_dev,
+                                const void* kv_packed_dev, const uint8_t* trig_mask_dev, void* y_f16_dev, void* workspace_dev,
+                                size_t workspace_bytes, void* stream) {
+    taq_status s = check_layer_desc(d);
+    if (s != TAQ_OK) return s;
+    if (d->batch > 65535) return fail(TAQ_ERR_SHAPE, "batch must be at most 65535");
+    if (d->batch == 0 || d->n_query == 0) return TAQ_OK;
+    TAQ_REQUIRE_PTR(x_f16_dev);
+    TAQ_REQUIRE_PTR(Wq_packed_dev);
+    TAQ_REQUIRE_PTR(Wout_packed_dev);
+    TAQ_REQUIRE_PTR(kv_packed_dev);
+    TAQ_REQUIRE_PTR(y_f16_dev);
+    TAQ_REQUIRE_PTR(workspace_dev);
+    if (!trig_mask_dev) return fail(TAQ_ERR_INVALID_ARG, "trig_mask_dev is NULL");
+    if (reinterpret_cast<uintptr_t>(workspace_dev) & 127u) return fail(TAQ_ERR_ALIGNMENT, "workspace_dev is not 128-byte aligned");
+    const WorkspaceA8 WA = workspace_a8_layout(d);
+    if (workspace_bytes < WA.total) return fail(TAQ_ERR_BUFFER_TOO_SMALL, "workspace has %zu bytes, %zu needed", workspace_bytes, WA.total);
+    cudaStream_t st = (cudaStream_t)stream;
+    int* status = nullptr;
+    s = status_ptr(&status);
+    if (s != TAQ_OK) return s;
+    uint8_t* wsb = (uint8_t*)workspace_dev;
+    int8_t* xq = (int8_t*)(wsb + WA.off_xq);
+    float* xs = (float*)(wsb + WA.off_xs);
+    uint8_t* base = wsb + WA.base;
+    const Workspace W = workspace_layout(d, 1);
+    const long long rows = (long long)d->batch * d->n_query;
+
+    cudaError_t e = launch_quantize_rows_f16((const __half*)x_f16_dev, rows, d->channels, xq, xs, st);      // X~ = Q_a(X) per token
+    if (e != cudaSuccess) return cuda_fail(e, "quantize_rows_f16 launch");
+    LinearArgs q{};                                                                                           // to_q (+ Q~ = Q_a(Q))
+    q.xq = xq; q.x_scales = xs; q.w = Wq_packed_dev;
+    q.y = base + W.off_q; q.scales = (float*)(base + W.off_qs);
+    q.rows = rows; q.n_out = d->channels; q.k_in = d->channels; q.bits = d->w_bits; q.group = d->w_group;
+    q.heads = d->q_bits == 8 ? d->heads : 1;
+    q.epi = d->q_bits == 8 ? EPI_Q8_HEAD : EPI_F16;
+    q.status = status;
+    s = run_linear_i8(q, st);
+    if (s != TAQ_OK) return s;
+    AttnArgs at = attn_args(d, status);
+    at.q = base + W.off_q; at.q_scales = (const float*)(base + W.off_qs); at.kv = kv_packed_dev; at.mask = trig_mask_dev;
+    at.o = (__half*)(base + W.off_o);
+    at.early_kv = 1;
+    s = run_attention(at, d->batch, st);
+    if (s != TAQ_OK) return s;
+    e = launch_quantize_rows_f16((const __half*)(base + W.off_o), rows, d->channels, xq, xs, st);            // O~ = Q_a(O) per token
+    if (e != cudaSuccess) return cuda_fail(e, "quantize_rows_f16 launch");
+    LinearArgs o{};                                                                                           // to_out (+ bias)
+    o.xq = xq; o.x_scales = xs; o.w = Wout_packed_dev;
+    o.y = y_f16_dev;
+    o.rows = rows; o.n_out = d->channels; o.k_in = d->channels; o.bits = d->w_bits; o.group = d->w_group;
+    o.heads = 1; o.epi = EPI_F16; o.status = status;
+    return run_linear_i8(o, st);
+}
+
+size_t taq_kv_project_a8_workspace_bytes(const taq_layer_desc* d) {
+    if (check_layer_desc(d) != TAQ_OK) return 0;
+    const size_t rows = (size_t)d->batch * d->n_ctx;
+    return align_up(rows * d->ctx_dim, 128) + align_up(rows * sizeof(float), 128);
+}
+
+taq_status taq_kv_project_a8(const taq_layer_desc* d, const void* ctx_f16_dev, const void* Wk_packed_dev, const void* Wv_packed_dev,
+                             const uint8_t* trig_mask_dev, void* kv_packed_dev, size_t kv_bytes, void* workspace_dev, size_t workspace_bytes,
+                             void* stream) {
+    taq_status s = check_layer_desc(d);
+    if (s != TAQ_OK) return s;
+    if (d->batch == 0) return TAQ_OK;
+    if (d->batch > 65535) return fail(TAQ_ERR_SHAPE, "batch must be at most 65535");
+    TAQ_REQUIRE_PTR(ctx_f16_dev);
+    TAQ_REQUIRE_PTR(Wk_packed_dev);
+    TAQ_REQUIRE_PTR(Wv_packed_dev);
+    TAQ_REQUIRE_PTR(kv_packed_dev);
+    TAQ_REQUIRE_PTR(workspace_dev);
+    if (!trig_mask_dev) return fail(TAQ_ERR_INVALID_ARG, "trig_mask_dev is NULL");
+    if (reinterpret_cast<uintptr_t>(workspace_dev) & 127u) return fail(TAQ_ERR_ALIGNMENT, "workspace_dev is not 128-byte aligned");
+    const size_t need = taq_kv_bytes(d), wneed = taq_kv_project_a8_workspace_bytes(d);
+    if (kv_bytes < need) return fail(TAQ_ERR_BUFFER_TOO_SMALL, "kv buffer has %zu bytes, %zu needed", kv_bytes, need);
+    if (workspace_bytes < wneed) return fail(TAQ_ERR_BUFFER_TOO_SMALL, "workspace has %zu bytes, %zu needed", workspace_bytes, wneed);
+    cudaStream_t st = (cudaStream_t)stream;
+    int* status = nullptr;
+    s = status_ptr(&status);
+    if (s != TAQ_OK) return s;
+    const long long rows = (long long)d->batch * d->n_ctx;
+    int8_t* cq = (int8_t*)workspace_dev;
+    float* cs = (float*)((uint8_t*)workspace_dev + align_up((size_t)rows * d->ctx_dim, 128));
+    cudaError_t e = launch_quantize_rows_f16((const __half*)ctx_f16_dev, rows, d->ctx_dim, cq, cs, st);
+    if (e != cudaSuccess) return cuda_fail(e, "quantize_rows_f16 launch");
+    LinearArgs a{};
+    a.xq = cq; a.x_scales = cs;
+    a.y = kv_packed_dev;
+    a.mask = trig_mask_dev;
+    a.rows = rows;
+    a.n_out = d->channels; a.k_in = d->ctx_dim; a.bits = d->w_bits; a.group = d->w_group;
+    a.heads = d->heads; a.n_ctx = d->n_ctx; a.max_trigger = d->max_trigger;
+    a.epi = EPI_KV;
+    a.status = status;
+    for (int which = 0; which < 2; ++which) {
+        a.w = which ? Wv_packed_dev : Wk_packed_dev;
+        a.which = which;
+        a.kv_which = which;
+        s = run_linear_i8(a, st);
+        if (s != TAQ_OK) return s;
+    }
+    e = launch_kv_operands(*d, kv_packed_dev, nullptr, d->batch, st);
+    return e == cudaSuccess ? TAQ_OK : cuda_fail(e, "K/V operand image launch");
+}
+
 taq_status taq_query_attention(const taq_layer_desc* d, const void* x_f16_dev, const void* Wq_packed_dev, const void* kv_packed_dev,
                                const uint8_t* trig_mask_dev, void* o_f16_dev, void* workspace_dev, size_t workspace_bytes, void* stream) {
     taq_status s = check_layer_desc(d);

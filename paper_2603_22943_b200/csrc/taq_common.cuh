@@ -123,6 +123,8 @@ enum Epilogue : int { EPI_F16 = 0, EPI_F32 = 1, EPI_Q8_HEAD = 2, EPI_KV = 3 };
 // (and, for EPI_KV, the output block and mask) come from the request table.
 struct LinearArgs {
     const __half* x;            // [z][rows][k_in]
+    const int8_t* xq;           // integer-activation variant: int8 codes [z][rows][k_in] instead of x ...
+    const float* x_scales;      // ... and one fp32 scale per row [z][rows]
     const void* w;              // packed blob (single problem)
     const taq_request* reqs;    // nullable
     int which;                  // 0: reqs[z].Wq, 1: reqs[z].Wout
@@ -191,6 +193,7 @@ inline cudaError_t launch_pdl_cluster(void (*kernel)(KArgs...), dim3 grid, dim3 
 
 cudaError_t launch_linear_simt(const LinearArgs& a, int n_z, cudaStream_t stream);
 cudaError_t launch_attention_simt(const AttnArgs& a, int n_z, cudaStream_t stream);
+cudaError_t launch_quantize_rows_f16(const __half* x, long long rows, int cols, int8_t* codes, float* scales, cudaStream_t stream);
 cudaError_t launch_quantize_rows(const float* x, long long rows, int cols, int qmax, int8_t* codes, float* scales,
                                  cudaStream_t stream);
 cudaError_t launch_pack_weights(const taq_weight_desc& d, const float* W, const float* bias, void* packed,

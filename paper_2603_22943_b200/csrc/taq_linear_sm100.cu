@@ -30,7 +30,7 @@ namespace {
 using namespace parts;
 
 constexpr int BM = 128;
-constexpr int BK = 64;
+constexpr int BK = 64;                     // fp16 elements per 128-byte operand row; the int8 variant has 2 BK
 constexpr int MAX_STAGE = 6;
 constexpr int NWORK = 256;                  // worker threads: two per accumulator row
 constexpr int NTHREADS = 64 + NWORK;
@@ -81,9 +81,13 @@ __host__ __device__ inline Plan make_plan(int k_in, int bits, int group, int nst
     return p;
 }
 
-template <int BN>
+// I8: the integer-activation variant (the literal W/A reading of Table 1).  The A operand is the int8 codes of the
+// per-token-quantized activations, the B operand the int8 weight codes, the accumulators are exact int32; a K block is
+// 128 elements (one W4 scale group), and the row's activation scale multiplies the folded sum at the end.
+template <int BN, bool I8>
 __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_kernel(const __grid_constant__ CUtensorMap tmap_x, const LinearArgs a, const int nstage) {
     using TL = Tile<BN>;
+    constexpr int BKE = I8 ? 2 * BK : BK;             // elements per K block
     constexpr int HC = TL::HC;
     extern __shared__ unsigned char smem_dyn[];
     unsigned char* smem = smem_dyn + ((1024u - (ptx::smem_u32(smem_dyn) & 1023u)) & 1023u);   // 1024-byte aligned, still provably shared
@@ -95,11 +99,11 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
     const int z = blockIdx.z;
     const int row0 = blockIdx.x * BM;
     const int col0 = blockIdx.y * BN;
-    const int n_kb = a.k_in / BK;
+    const int n_kb = (a.k_in + BKE - 1) / BKE;          // (int8: the last block may be ragged; TMA and the expansion zero-fill)
     const uint8_t* blob = (const uint8_t*)(a.reqs ? (a.which == 0 ? a.reqs[z].Wq : a.reqs[z].Wout) : a.w);
     const WeightLayout L = weight_layout(a.n_out, a.k_in, a.bits, a.group);
     const int n_groups = L.n_groups;
-    const int kb_per_group = L.group_len / BK;             // k-blocks in a full group (the last group may be shorter)
+    const int kb_per_group = n_groups == 1 ? n_kb : L.group_len / BKE;   // k-blocks in a full group (the last group may be shorter)
 
     TAQ_PROF_INIT
     if (tid == 0) { TAQ_PROF(0); TAQ_GPROF(30); }
@@ -141,7 +145,7 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
                 if (kb >= nstage && !ptx::mbar_wait(&bars->empty[s], ph ^ 1)) { raise_status(a.status, TAQ_ERR_TIMEOUT); bars->abort_flag = 1; }
                 if (bars->abort_flag) break;
                 ptx::mbar_arrive_expect_tx(&bars->full_a[s], A_TILE_BYTES);
-                ptx::tma_load_3d(smem + s * TL::STAGE_BYTES, &tmap_x, &bars->full_a[s], kb * BK, row0, z);
+                ptx::tma_load_3d(smem + s * TL::STAGE_BYTES, &tmap_x, &bars->full_a[s], kb * BKE, row0, z);
                 issued = kb + 1;
                 if (++s == nstage) { s = 0; ph ^= 1; }
             }
@@ -156,7 +160,7 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
         // issues.  The path between two MMAs is kept short: this warp shares its scheduler with worker warps.
         const bool leader = ptx::elect_one();
         auto wait = [&](uint64_t* bar, uint32_t parity) -> bool { return __all_sync(0xffffffffu, ptx::mbar_wait(bar, parity) && !bars->abort_flag) != 0; };
-        constexpr uint32_t idesc = ptx::idesc_f16_m128(BN);
+        constexpr uint32_t idesc = I8 ? ptx::idesc_i8_m128(BN) : ptx::idesc_f16_m128(BN);
         constexpr uint32_t HI = ptx::kDescHiSw128;
         const uint32_t lo0 = ptx::desc_lo(ptx::smem_u32(smem));
         int s = 0, kb = 0;
@@ -174,8 +178,10 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
                 if (leader) {
                     const uint32_t a_lo = lo0 + s * (TL::STAGE_BYTES >> 4), b_lo = a_lo + (A_TILE_BYTES >> 4);
 #pragma unroll
-                    for (int k = 0; k < BK / 16; ++k)
-                        ptx::mma_f16_ss(tmem_base + buf * BN, ptx::desc_join(HI, a_lo + 2 * k), ptx::desc_join(HI, b_lo + 2 * k), idesc, !(first && k == 0));
+                    for (int k = 0; k < 4; ++k) {            // four 32-byte K slices per 128-byte operand row
+                        if (I8) ptx::mma_i8_ss(tmem_base + buf * BN, ptx::desc_join(HI, a_lo + 2 * k), ptx::desc_join(HI, b_lo + 2 * k), idesc, !(first && k == 0));
+                        else ptx::mma_f16_ss(tmem_base + buf * BN, ptx::desc_join(HI, a_lo + 2 * k), ptx::desc_join(HI, b_lo + 2 * k), idesc, !(first && k == 0));
+                    }
                     ptx::mma_commit(&bars->empty[s]);       // frees the stage once these MMAs have read it
                     if (kb + 1 == kb_end) ptx::mma_commit(&bars->acc_full[buf]);
                 }
@@ -235,10 +241,13 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
                     if (c0 + i * 8 < HC) {
                         const float4 s0 = *reinterpret_cast<const float4*>(sg + c0 + i * 8), s1 = *reinterpret_cast<const float4*>(sg + c0 + i * 8 + 4);
                         float* yy = y + c0 + i * 8;
-                        yy[0] = fmaf(__uint_as_float(v[i][0]), s0.x, yy[0]); yy[1] = fmaf(__uint_as_float(v[i][1]), s0.y, yy[1]);
-                        yy[2] = fmaf(__uint_as_float(v[i][2]), s0.z, yy[2]); yy[3] = fmaf(__uint_as_float(v[i][3]), s0.w, yy[3]);
-                        yy[4] = fmaf(__uint_as_float(v[i][4]), s1.x, yy[4]); yy[5] = fmaf(__uint_as_float(v[i][5]), s1.y, yy[5]);
-                        yy[6] = fmaf(__uint_as_float(v[i][6]), s1.z, yy[6]); yy[7] = fmaf(__uint_as_float(v[i][7]), s1.w, yy[7]);
+                        float f[8];
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) f[e] = I8 ? __int2float_rn((int)v[i][e]) : __uint_as_float(v[i][e]);
+                        yy[0] = fmaf(f[0], s0.x, yy[0]); yy[1] = fmaf(f[1], s0.y, yy[1]);
+                        yy[2] = fmaf(f[2], s0.z, yy[2]); yy[3] = fmaf(f[3], s0.w, yy[3]);
+                        yy[4] = fmaf(f[4], s1.x, yy[4]); yy[5] = fmaf(f[5], s1.y, yy[5]);
+                        yy[6] = fmaf(f[6], s1.z, yy[6]); yy[7] = fmaf(f[7], s1.w, yy[7]);
                     }
             }
             ptx::tc_fence_before_sync();
@@ -259,6 +268,30 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
                 // 16-byte chunks of the fp16 tile: 8 per weight row; this thread owns chunk c of rows n0, n0 + 32, ...
                 constexpr int NCH = (BN * 8 + NWORK - 1) / NWORK;
                 const int n0 = wt >> 3, c = wt & 7;
+                if (I8) {
+                    // int8 tile: a chunk is 16 fan-in elements; chunks at or beyond k_in (ragged last block) are zero
+                    const int k0 = kb * BKE + c * 16;
+                    uint4 cw[NCH];
+#pragma unroll
+                    for (int i = 0; i < NCH; ++i) {
+                        const int n = n0 + (NWORK / 8) * i;
+                        cw[i] = make_uint4(0, 0, 0, 0);
+                        if (((BN * 8) % NWORK == 0 || n < BN) && k0 < a.k_in) {
+                            if (a.bits == 4) {
+                                const uint2 p = *reinterpret_cast<const uint2*>(raw + n * row_bytes + (k0 >> 1));
+                                const uint2 lo = codes_w4_to_i8(p.x), hi = codes_w4_to_i8(p.y);
+                                cw[i] = make_uint4(lo.x, lo.y, hi.x, hi.y);
+                            } else {
+                                cw[i] = *reinterpret_cast<const uint4*>(raw + n * row_bytes + k0);
+                            }
+                        }
+                    }
+#pragma unroll
+                    for (int i = 0; i < NCH; ++i) {
+                        const int n = n0 + (NWORK / 8) * i;
+                        if ((BN * 8) % NWORK == 0 || n < BN) *reinterpret_cast<uint4*>(b_tile + ptx::sw128_offset(n, c)) = cw[i];
+                    }
+                } else {
                 uint2 pw[NCH];
 #pragma unroll
                 for (int i = 0; i < NCH; ++i) {
@@ -274,6 +307,7 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
                     const int n = n0 + (NWORK / 8) * i;
                     if ((BN * 8) % NWORK == 0 || n < BN)
                         *reinterpret_cast<uint4*>(b_tile + ptx::sw128_offset(n, c)) = a.bits == 4 ? codes_w4_to_half(pw[i].x) : codes_w8_to_half(pw[i]);
+                }
                 }
                 ptx::fence_proxy_async_smem();            // make the generic-proxy writes visible to the tensor core
                 __syncwarp();
@@ -293,6 +327,11 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
         ok = !bars->abort_flag;
         ptx::pdl_wait();                                     // (already satisfied: the activations have arrived) orders the stores below
         if (wt == 0) TAQ_PROF(7);
+        if (I8 && ok) {                                      // x~ = code * s_x: the row's activation scale
+            const float sx = row < a.rows ? a.x_scales[(size_t)z * a.rows + row] : 0.f;
+#pragma unroll
+            for (int c = 0; c < HC; ++c) y[c] *= sx;
+        }
 
         // ---------------- epilogue on this thread's HC columns ----------------
         if (ok) {
@@ -466,7 +505,8 @@ int pick_bn(const LinearArgs& a) {
 // Ring depth: as deep as the K loop needs, but no deeper than three stages when that keeps two CTAs on an SM.
 template <int BN>
 int pick_nstage(const LinearArgs& a) {
-    const int n_kb = a.k_in / BK;
+    const int bke = a.xq ? 2 * BK : BK;
+    const int n_kb = (a.k_in + bke - 1) / bke;
     const int half_sm = Tile<BN>::CTAS_PER_SM == 2 ? SMEM_LIMIT / 2 : SMEM_LIMIT;
     int best = 0;
     for (int ns = 1; ns <= MAX_STAGE && ns <= (n_kb < 2 ? 2 : n_kb); ++ns) {
@@ -489,25 +529,33 @@ int nstage_for(const LinearArgs& a, int bn) {
 
 template <int BN>
 cudaError_t launch_bn(const CUtensorMap& tmap, const LinearArgs& a, int n_z, cudaStream_t stream) {
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(linear_sm100_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT);
+    static bool configured[2] = {false, false};
+    const bool i8 = a.xq != nullptr;
+    void (*kern)(const CUtensorMap, const LinearArgs, const int) = i8 ? linear_sm100_kernel<BN, true> : linear_sm100_kernel<BN, false>;
+    if (!configured[i8]) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT);
         if (e != cudaSuccess) return e;
-        configured = true;
+        configured[i8] = true;
     }
     const int ns = pick_nstage<BN>(a);
     const Plan P = make_plan<BN>(a.k_in, a.bits, a.group, ns);
     dim3 grid((unsigned)((a.rows + BM - 1) / BM), a.n_out / BN, n_z);
-    return launch_pdl(linear_sm100_kernel<BN>, grid, dim3(NTHREADS), (size_t)P.total, stream, tmap, a, ns);
+    return launch_pdl(kern, grid, dim3(NTHREADS), (size_t)P.total, stream, tmap, a, ns);
 }
 
 }  // namespace
 
 bool sm100_linear_supported(const LinearArgs& a) {
-    if (a.k_in % BK) return false;
-    if (a.group != 0 && a.group % BK) return false;
+    if (a.xq) {       // int8 activations: rows of 16-byte granularity, a scale group = one 128-element K block
+        if (a.k_in % 16) return false;
+        if (a.group != 0 && a.group != 2 * BK && a.group < a.k_in) return false;
+        if (reinterpret_cast<uintptr_t>(a.xq) & 15u) return false;
+    } else {
+        if (a.k_in % BK) return false;
+        if (a.group != 0 && a.group % BK) return false;
+        if (reinterpret_cast<uintptr_t>(a.x) & 15u) return false;
+    }
     if (a.rows < 1 || a.rows > (1LL << 31) - 1) return false;
-    if (reinterpret_cast<uintptr_t>(a.x) & 15u) return false;
     const int bn = pick_bn(a);
     if (bn == 0) return false;
     if (nstage_for(a, bn) < 2) return false;
@@ -519,11 +567,14 @@ cudaError_t launch_linear_sm100(const LinearArgs& a, int n_z, cudaStream_t strea
     EncodeTiledFn enc = encode_tiled_fn();
     if (!enc) return cudaErrorNotSupported;
     CUtensorMap tmap;
+    const bool i8 = a.xq != nullptr;
+    const cuuint64_t esz = i8 ? 1 : 2;
     const cuuint64_t dims[3] = {(cuuint64_t)a.k_in, (cuuint64_t)a.rows, (cuuint64_t)n_z};
-    const cuuint64_t strides[2] = {(cuuint64_t)a.k_in * 2, (cuuint64_t)a.k_in * 2 * (cuuint64_t)a.rows};
-    const cuuint32_t box[3] = {BK, BM, 1};
+    const cuuint64_t strides[2] = {(cuuint64_t)a.k_in * esz, (cuuint64_t)a.k_in * esz * (cuuint64_t)a.rows};
+    const cuuint32_t box[3] = {(cuuint32_t)(i8 ? 2 * BK : BK), BM, 1};       // 128 bytes of K either way; elements beyond k_in read as zero
     const cuuint32_t estr[3] = {1, 1, 1};
-    CUresult r = enc(&tmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<__half*>(a.x), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+    CUresult r = enc(&tmap, i8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3,
+                     i8 ? (void*)const_cast<int8_t*>(a.xq) : (void*)const_cast<__half*>(a.x), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                      CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
     switch (pick_bn(a)) {

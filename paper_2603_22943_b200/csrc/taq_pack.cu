@@ -55,6 +55,65 @@ cudaError_t launch_quantize_rows(const float* x, long long rows, int cols, int q
     return cudaGetLastError();
 }
 
+// Per-token quantizer of fp16 activations (the inputs of the integer-activation projections): one warp per row of
+// `cols` fp16 values (a multiple of 8), which it keeps in registers between the absmax pass and the code pass when the
+// row is short enough (up to 2048 columns), so that the row is read once.  Same arithmetic as quantize_rows_kernel.
+__global__ void __launch_bounds__(256) quantize_rows_f16_kernel(const __half* __restrict__ x, long long rows, int cols,
+                                                                int8_t* __restrict__ codes, float* __restrict__ scales) {
+    const int lane = threadIdx.x & 31;
+    const long long warps_total = (long long)gridDim.x * (blockDim.x >> 5);
+    const int chunks = cols / 8;                                 // 16-byte chunks of a row
+    for (long long r = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); r < rows; r += warps_total) {
+        const uint4* xr = reinterpret_cast<const uint4*>(x + r * cols);
+        constexpr int KEEP = 8;                                  // chunks a lane keeps: 8 x 32 x 8 = 2048 columns
+        uint4 keep[KEEP];
+        float a = 0.f;
+#pragma unroll
+        for (int j = 0; j < KEEP; ++j) {
+            const int i = lane + 32 * j;
+            keep[j] = make_uint4(0, 0, 0, 0);
+            if (i < chunks) keep[j] = xr[i];
+            const __half2* h = reinterpret_cast<const __half2*>(&keep[j]);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) { const float2 f = __half22float2(h[e]); a = fmaxf(a, fmaxf(fabsf(f.x), fabsf(f.y))); }
+        }
+        for (int i = lane + 32 * KEEP; i < chunks; i += 32) {
+            const uint4 v = xr[i];
+            const __half2* h = reinterpret_cast<const __half2*>(&v);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) { const float2 f = __half22float2(h[e]); a = fmaxf(a, fmaxf(fabsf(f.x), fabsf(f.y))); }
+        }
+        a = warp_max(a);
+        const float s = quant_scale(a, 127.f);
+        if (lane == 0) scales[r] = s;
+        uint2* cr = reinterpret_cast<uint2*>(codes + r * cols);
+        auto encode = [&](const uint4& v) {
+            const __half2* h = reinterpret_cast<const __half2*>(&v);
+            uint32_t w[2] = {0, 0};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float2 f = __half22float2(h[e]);
+                w[e >> 1] |= ((uint32_t)(quant_code(f.x, s, 127) & 0xFF) | ((uint32_t)(quant_code(f.y, s, 127) & 0xFF) << 8)) << (16 * (e & 1));
+            }
+            return make_uint2(w[0], w[1]);
+        };
+#pragma unroll
+        for (int j = 0; j < KEEP; ++j) {
+            const int i = lane + 32 * j;
+            if (i < chunks) cr[i] = encode(keep[j]);
+        }
+        for (int i = lane + 32 * KEEP; i < chunks; i += 32) cr[i] = encode(xr[i]);
+    }
+}
+
+cudaError_t launch_quantize_rows_f16(const __half* x, long long rows, int cols, int8_t* codes, float* scales, cudaStream_t stream) {
+    if (rows == 0) return cudaSuccess;
+    long long blocks = (rows + 7) / 8;
+    if (blocks > 148LL * 32) blocks = 148LL * 32;
+    quantize_rows_f16_kernel<<<(unsigned)blocks, 256, 0, stream>>>(x, rows, cols, codes, scales);
+    return cudaGetLastError();
+}
+
 // One warp per (output channel, group).
 __global__ void __launch_bounds__(256) pack_weights_kernel(const float* __restrict__ W, const float* __restrict__ bias, uint8_t* __restrict__ blob,
                                                            int n_out, int k_in, int bits, int group) {

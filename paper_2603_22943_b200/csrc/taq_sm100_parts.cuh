@@ -38,6 +38,13 @@ __device__ __forceinline__ uint4 codes_w8_to_half(uint2 raw) {
     return make_uint4(o[0], o[1], o[2], o[3]);
 }
 
+// Eight 4-bit codes of one word -> eight int8 codes in fan-in order (the integer-activation GEMM's weight operand).
+__device__ __forceinline__ uint2 codes_w4_to_i8(uint32_t p) {
+    const uint32_t even = p & 0x0F0F0F0Fu;              // bytes: elements 0, 4, 1, 5 (+8)
+    const uint32_t odd = (p >> 4) & 0x0F0F0F0Fu;        // bytes: elements 2, 6, 3, 7 (+8)
+    return make_uint2(__vsub4(__byte_perm(even, odd, 0x6420), 0x08080808u), __vsub4(__byte_perm(even, odd, 0x7531), 0x08080808u));
+}
+
 __device__ __forceinline__ uint4 pack8(const float (&w)[8]) {
     uint4 out;
     __half2 h;

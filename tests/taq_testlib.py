@@ -29,8 +29,8 @@ def assert_layer_close(got, want, what=""):
     return max_abs, rel
 
 
-def oracle_cfg(shape: synth.LayerShape, contract=True) -> orc.TaqConfig:
-    return orc.TaqConfig(heads=shape.heads, w_bits=shape.w_bits, w_group=shape.w_group, q_bits=shape.q_bits, contract=contract)
+def oracle_cfg(shape: synth.LayerShape, contract=True, a_bits=0) -> orc.TaqConfig:
+    return orc.TaqConfig(heads=shape.heads, w_bits=shape.w_bits, w_group=shape.w_group, q_bits=shape.q_bits, contract=contract, a_bits=a_bits)
 
 
 def oracle_layer(shape: synth.LayerShape, data, contract=True, rows=None):
@@ -116,7 +116,7 @@ def build_kv_block(desc: tb.LayerDesc, K_codes, K_scales, V_codes, V_scales, K_r
     return raw.reshape(-1)
 
 
-def gpu_decisions(shape: synth.LayerShape, data, parts, rows=None):
+def gpu_decisions(shape: synth.LayerShape, data, parts, rows=None, a_bits=0):
     """The rounding decisions the CUDA path took upstream of the attention: K~/V~ as stored in its block and Q~
     as produced by the same dequant-GEMM kernel the layer call runs (bit-identical by determinism)."""
     desc, P = parts["desc"], parts["packed"]
@@ -135,14 +135,20 @@ def gpu_decisions(shape: synth.LayerShape, data, parts, rows=None):
     X = data["X"] if rows is None else data["X"][:, rows]
     n = X.shape[1]
     x2 = dev(X.reshape(B * n, shape.channels))
+    if a_bits == 8:                      # the integer-activation projection, as taq_layer_forward_a8 runs it
+        xc, xs = tb.taq_quantize_rows_f16(x2)
+        out["X_codes"], out["X_scales"] = xc.cpu().numpy().reshape(B, n, -1), xs.cpu().numpy().reshape(B, n)
+        linear = lambda kind, **kw: tb.taq_quantized_linear_i8(P["wd_cc"], xc, xs, P["Wq"], kind, **kw)
+    else:
+        linear = lambda kind, **kw: tb.taq_quantized_linear(P["wd_cc"], x2, P["Wq"], kind, **kw)
     if shape.q_bits == 8:
-        qc, qs = tb.taq_quantized_linear(P["wd_cc"], x2, P["Wq"], tb.TAQ_OUT_INT8_HEAD_ROWS, heads=H)
+        qc, qs = linear(tb.TAQ_OUT_INT8_HEAD_ROWS, heads=H)
         qc = qc.cpu().numpy().reshape(B, n, H, d).transpose(0, 2, 1, 3)                                   # [B,H,n,d]
         qs = qs.cpu().numpy().reshape(B, n, H).transpose(0, 2, 1)                                          # [B,H,n]
         out["Q_codes"], out["Q_scales"] = qc, qs
         out["Q_tilde"] = (qc.astype(np.float32) * qs[..., None]).astype(np.float64)
     else:
-        q16 = tb.taq_quantized_linear(P["wd_cc"], x2, P["Wq"], tb.TAQ_OUT_F16).cpu().numpy()
+        q16 = linear(tb.TAQ_OUT_F16).cpu().numpy()
         out["Q_tilde"] = q16.reshape(B, n, H, d).transpose(0, 2, 1, 3).astype(np.float64)
     return out
 
@@ -164,20 +170,23 @@ def assert_codes_agree(got, want, pre, scales, what, max_frac=2e-3):
     return frac
 
 
-def check_layer(shape: synth.LayerShape, data, y_gpu, parts, rows=None):
+def check_layer(shape: synth.LayerShape, data, y_gpu, parts, rows=None, a_bits=0):
     """Three-part parity of one layer call.
     (1) the integer decisions (Q, K, V codes) of the CUDA path equal the oracle's, up to near-ties;
     (2) given the same decisions, the layer output matches the oracle within the contract tolerances everywhere;
     (3) end to end against the untouched oracle: relative L2 within tolerance over everything, and max-abs within
         tolerance on every query row whose Q codes agree (a one-step flip of a near-tie is amplified by the softmax,
         which is why both sides must take that decision from the same value, as (2) does)."""
-    cfg = oracle_cfg(shape)
+    cfg = oracle_cfg(shape, a_bits=a_bits)
     X = data["X"] if rows is None else data["X"][:, rows]
     y = y_gpu if rows is None else y_gpu[:, rows]
     kv_o = orc.taq_kv(data["ctx"], data["Wk"], data["Wv"], data["mask"], cfg)
     q_o = orc.taq_q(X, data["Wq"], cfg)
     Y_o = orc.taq_out(orc.taq_attention(q_o["Q_tilde"], kv_o["K_tilde"], kv_o["V_tilde"], data["mask"], cfg), data["Wout"], data["bout"], cfg)
-    g = gpu_decisions(shape, data, parts, rows)
+    g = gpu_decisions(shape, data, parts, rows, a_bits)
+    if a_bits == 8:                      # the per-token codes of X are a stand-alone quantizer's: bit-exact
+        xc, xs = orc.quantize_rows(X.astype(np.float32), 127)
+        assert np.array_equal(g["X_codes"], xc) and np.array_equal(g["X_scales"], xs), "X codes / scales"
     # (1)
     nt = np.array([j for j in range(shape.n_ctx) if not data["mask"][0, j]], dtype=np.int64)
     same_mask = bool((data["mask"] == data["mask"][0]).all())
