@@ -137,6 +137,8 @@ struct LinearArgs {
     int n_ctx, max_trigger;     // EPI_KV: rows = batch * n_ctx
     int kv_which;               // EPI_KV: 0 = K, 1 = V
     int epi;
+    int w_direct;               // (set by the launcher) int8 activations and 8-bit weights: the weight codes are the B
+                                // operand as they are and go from the blob into the ring by TMA, no staging or expansion
     int early_weights;          // the previous kernel in the stream is known not to write the weights: fetch and expand
                                 // them before waiting for it
     int* status;

@@ -65,10 +65,10 @@ struct Plan {
 };
 
 template <int BN>
-__host__ __device__ inline Plan make_plan(int k_in, int bits, int group, int nstage) {
+__host__ __device__ inline Plan make_plan(int k_in, int bits, int group, int nstage, bool direct) {
     const WeightLayout L = weight_layout(BN, k_in, bits, group);
     Plan p;
-    p.raw_bytes = (int)(L.row_bytes * BN);
+    p.raw_bytes = direct ? 0 : (int)(L.row_bytes * BN);    // (direct: no staged codes)
     p.scale_bytes = BN * L.n_groups * 4;
     p.bias_bytes = BN * 4;
     p.off_raw = nstage * Tile<BN>::STAGE_BYTES;
@@ -85,13 +85,13 @@ __host__ __device__ inline Plan make_plan(int k_in, int bits, int group, int nst
 // per-token-quantized activations, the B operand the int8 weight codes, the accumulators are exact int32; a K block is
 // 128 elements (one W4 scale group), and the row's activation scale multiplies the folded sum at the end.
 template <int BN, bool I8>
-__global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_kernel(const __grid_constant__ CUtensorMap tmap_x, const LinearArgs a, const int nstage) {
+__global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w, const LinearArgs a, const int nstage) {
     using TL = Tile<BN>;
     constexpr int BKE = I8 ? 2 * BK : BK;             // elements per K block
     constexpr int HC = TL::HC;
     extern __shared__ unsigned char smem_dyn[];
     unsigned char* smem = smem_dyn + ((1024u - (ptx::smem_u32(smem_dyn) & 1023u)) & 1023u);   // 1024-byte aligned, still provably shared
-    const Plan P = make_plan<BN>(a.k_in, a.bits, a.group, nstage);
+    const Plan P = make_plan<BN>(a.k_in, a.bits, a.group, nstage, a.w_direct != 0);
     Bars* bars = reinterpret_cast<Bars*>(smem + P.off_bars);
     constexpr uint32_t TMEM_COLS = TL::TMEM_COLS;
 
@@ -134,7 +134,7 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
         if (lane == 0) {
             if (!a.early_weights) ptx::pdl_wait();        // in general the weights may come from the previous kernel
             ptx::mbar_arrive_expect_tx(&bars->w_full, (uint32_t)(P.raw_bytes + P.scale_bytes + P.bias_bytes));
-            ptx::bulk_load(smem + P.off_raw, blob + L.off_codes + (size_t)col0 * L.row_bytes, (uint32_t)P.raw_bytes, &bars->w_full);
+            if (P.raw_bytes) ptx::bulk_load(smem + P.off_raw, blob + L.off_codes + (size_t)col0 * L.row_bytes, (uint32_t)P.raw_bytes, &bars->w_full);
             ptx::bulk_load(smem + P.off_scales, blob + L.off_scales + (size_t)col0 * n_groups * 4, (uint32_t)P.scale_bytes, &bars->w_full);
             ptx::bulk_load(smem + P.off_bias, blob + L.off_bias + (size_t)col0 * 4, (uint32_t)P.bias_bytes, &bars->w_full);
             if (a.early_weights) ptx::pdl_wait();         // the activations come from the previous kernel
@@ -144,8 +144,9 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
             for (int kb = 0; kb < n_kb; ++kb) {
                 if (kb >= nstage && !ptx::mbar_wait(&bars->empty[s], ph ^ 1)) { raise_status(a.status, TAQ_ERR_TIMEOUT); bars->abort_flag = 1; }
                 if (bars->abort_flag) break;
-                ptx::mbar_arrive_expect_tx(&bars->full_a[s], A_TILE_BYTES);
+                ptx::mbar_arrive_expect_tx(&bars->full_a[s], A_TILE_BYTES + (a.w_direct ? BN * 128 : 0));
                 ptx::tma_load_3d(smem + s * TL::STAGE_BYTES, &tmap_x, &bars->full_a[s], kb * BKE, row0, z);
+                if (a.w_direct) ptx::tma_load_3d(smem + s * TL::STAGE_BYTES + A_TILE_BYTES, &tmap_w, &bars->full_a[s], kb * BKE, col0, 0);
                 issued = kb + 1;
                 if (++s == nstage) { s = 0; ph ^= 1; }
             }
@@ -174,7 +175,7 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
             }
             const int kb_end = min(n_kb, kb + kb_per_group);
             for (bool first = true; kb < kb_end && ok; ++kb) {
-                if (!wait(&bars->full_a[s], ph) || !wait(&bars->full_b[s], ph)) { ok = false; break; }
+                if (!wait(&bars->full_a[s], ph) || (!a.w_direct && !wait(&bars->full_b[s], ph))) { ok = false; break; }
                 if (leader) {
                     const uint32_t a_lo = lo0 + s * (TL::STAGE_BYTES >> 4), b_lo = a_lo + (A_TILE_BYTES >> 4);
 #pragma unroll
@@ -318,7 +319,7 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
         };
 
         for (int g = 0; g < n_groups && ok; ++g) {
-            ok = build_group(g);
+            ok = a.w_direct ? true : build_group(g);
             if (ok && g >= 1) ok = fold_group(g - 1);
         }
         if (ok) ok = fold_group(n_groups - 1);
@@ -506,13 +507,14 @@ int pick_bn(const LinearArgs& a) {
 template <int BN>
 int pick_nstage(const LinearArgs& a) {
     const int bke = a.xq ? 2 * BK : BK;
+    const bool direct = a.xq && a.bits == 8 && !a.reqs;
     const int n_kb = (a.k_in + bke - 1) / bke;
     const int half_sm = Tile<BN>::CTAS_PER_SM == 2 ? SMEM_LIMIT / 2 : SMEM_LIMIT;
     int best = 0;
     for (int ns = 1; ns <= MAX_STAGE && ns <= (n_kb < 2 ? 2 : n_kb); ++ns) {
-        const int total = make_plan<BN>(a.k_in, a.bits, a.group, ns).total;
+        const int total = make_plan<BN>(a.k_in, a.bits, a.group, ns, direct).total;
         if (total > SMEM_LIMIT) break;
-        if (ns > 3 && total + 1024 > half_sm && make_plan<BN>(a.k_in, a.bits, a.group, 3).total + 1024 <= half_sm) break;
+        if (ns > 3 && total + 1024 > half_sm && make_plan<BN>(a.k_in, a.bits, a.group, 3, direct).total + 1024 <= half_sm) break;
         best = ns;
     }
     return best;
@@ -528,19 +530,30 @@ int nstage_for(const LinearArgs& a, int bn) {
 }
 
 template <int BN>
-cudaError_t launch_bn(const CUtensorMap& tmap, const LinearArgs& a, int n_z, cudaStream_t stream) {
+cudaError_t launch_bn(const CUtensorMap& tmap, EncodeTiledFn enc, LinearArgs a, int n_z, cudaStream_t stream) {
     static bool configured[2] = {false, false};
     const bool i8 = a.xq != nullptr;
-    void (*kern)(const CUtensorMap, const LinearArgs, const int) = i8 ? linear_sm100_kernel<BN, true> : linear_sm100_kernel<BN, false>;
+    void (*kern)(const CUtensorMap, const CUtensorMap, const LinearArgs, const int) = i8 ? linear_sm100_kernel<BN, true> : linear_sm100_kernel<BN, false>;
+    a.w_direct = i8 && a.bits == 8 && !a.reqs;
+    CUtensorMap tmap_w = tmap;                        // (unused unless w_direct)
+    if (a.w_direct) {                                 // the codes section of the blob as an int8 matrix [n_out][k_in]
+        const WeightLayout L = weight_layout(a.n_out, a.k_in, a.bits, a.group);
+        const cuuint64_t dims[3] = {(cuuint64_t)a.k_in, (cuuint64_t)a.n_out, 1};
+        const cuuint64_t strides[2] = {(cuuint64_t)L.row_bytes, (cuuint64_t)L.row_bytes * (cuuint64_t)a.n_out};
+        const cuuint32_t box[3] = {2 * BK, BN, 1}, estr[3] = {1, 1, 1};
+        CUresult r = enc(&tmap_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, (void*)((const uint8_t*)a.w + L.off_codes), dims, strides, box, estr,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+    }
     if (!configured[i8]) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT);
         if (e != cudaSuccess) return e;
         configured[i8] = true;
     }
     const int ns = pick_nstage<BN>(a);
-    const Plan P = make_plan<BN>(a.k_in, a.bits, a.group, ns);
+    const Plan P = make_plan<BN>(a.k_in, a.bits, a.group, ns, a.w_direct != 0);
     dim3 grid((unsigned)((a.rows + BM - 1) / BM), a.n_out / BN, n_z);
-    return launch_pdl(kern, grid, dim3(NTHREADS), (size_t)P.total, stream, tmap, a, ns);
+    return launch_pdl(kern, grid, dim3(NTHREADS), (size_t)P.total, stream, tmap, tmap_w, a, ns);
 }
 
 }  // namespace
@@ -578,9 +591,9 @@ cudaError_t launch_linear_sm100(const LinearArgs& a, int n_z, cudaStream_t strea
                      CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
     switch (pick_bn(a)) {
-        case 64: return launch_bn<64>(tmap, a, n_z, stream);
-        case 80: return launch_bn<80>(tmap, a, n_z, stream);
-        case 160: return launch_bn<160>(tmap, a, n_z, stream);
+        case 64: return launch_bn<64>(tmap, enc, a, n_z, stream);
+        case 80: return launch_bn<80>(tmap, enc, a, n_z, stream);
+        case 160: return launch_bn<160>(tmap, enc, a, n_z, stream);
     }
     return cudaErrorNotSupported;
 }
