@@ -294,8 +294,23 @@ def main():
         s = sets[i % n_sets]
         tb.taq_quantized_linear(wd_cc, o_sets[i % n_sets], s["Wout"], tb.TAQ_OUT_F16, y=s["y"])
 
+    # the integer-activation reading (int8 X and O, tcgen05 kind::i8): the five-kernel layer pass, and its to_out GEMM
+    # alone on codes quantized beforehand
+    ws_a8 = torch.empty(tb.taq_workspace_bytes_a8(desc), dtype=torch.uint8, device="cuda")
+    oq_sets = [tb.taq_quantize_rows_f16(sets[i]["x"].view(M, C_)) for i in range(n_sets)]
+
+    def stage_layer_a8(i):
+        s = sets[i % n_sets]
+        tb.taq_layer_forward_a8(desc, s["x"], s["Wq"], s["Wout"], s["kv"], mask, s["y"], ws_a8)
+
+    def stage_out_i8(i):
+        s = sets[i % n_sets]
+        oc, os_ = oq_sets[i % n_sets]
+        tb.taq_quantized_linear_i8(wd_cc, oc, os_, s["Wout"], tb.TAQ_OUT_F16, y=s["y"])
+
     stage_ms = {}
-    for name, fn in (("qattn", stage_qattn), ("to_q", stage_q), ("attn", stage_attn), ("to_out", stage_out)):
+    for name, fn in (("qattn", stage_qattn), ("to_q", stage_q), ("attn", stage_attn), ("to_out", stage_out),
+                     ("layer_a8", stage_layer_a8), ("to_out_i8", stage_out_i8)):
         for i in range(n_sets):
             fn(i)
         torch.cuda.synchronize()
@@ -351,6 +366,10 @@ def main():
          "bytes": M * C_ * 2 + qbytes + wbytes, "flops": 2 * M * C_ * C_, "traffic": None},
         {"name": "attention_sm100_kernel<40>: attention, stand-alone (taq_cross_attention)", "ms": stage_ms["attn"], "in_step": False,
          "bytes": qbytes + M * C_ * 2 + img_bytes, "flops": 4 * M * T * C_, "traffic": None},
+        {"name": "integer-activation layer pass, 5 kernels: Q_a(X), int8 to_q, attention, Q_a(O), int8 to_out (taq_layer_forward_a8)", "ms": stage_ms["layer_a8"],
+         "in_step": False, "bytes": 2 * M * C_ * 2 + 2 * wbytes + img_bytes, "flops": 4 * M * C_ * C_ + 4 * M * T * C_, "traffic": None},
+        {"name": "linear_sm100_kernel<160,int8>: to_out as int8 x int8 -> int32 GEMM, stand-alone (taq_quantized_linear_i8)", "ms": stage_ms["to_out_i8"],
+         "in_step": False, "bytes": M * C_ + M * 4 + M * C_ * 2 + wbytes, "flops": 2 * M * C_ * C_, "traffic": None},
     ]
     for k in kernels:
         k["GB/s"] = k["bytes"] / (k["ms"] * 1e-3) / 1e9
