@@ -488,6 +488,7 @@ taq_status taq_layer_forward_a8(const taq_layer_desc* d, const void* x_f16_dev, 
     q.heads = d->q_bits == 8 ? d->heads : 1;
     q.epi = d->q_bits == 8 ? EPI_Q8_HEAD : EPI_F16;
     q.status = status;
+    q.early_weights = 1;        // the kernel before it in the stream is the quantizer above, which writes xq / xs only
     s = run_linear_i8(q, st);
     if (s != TAQ_OK) return s;
     AttnArgs at = attn_args(d, status);
@@ -503,6 +504,7 @@ taq_status taq_layer_forward_a8(const taq_layer_desc* d, const void* x_f16_dev, 
     o.y = y_f16_dev;
     o.rows = rows; o.n_out = d->channels; o.k_in = d->channels; o.bits = d->w_bits; o.group = d->w_group;
     o.heads = 1; o.epi = EPI_F16; o.status = status;
+    o.early_weights = 1;
     return run_linear_i8(o, st);
 }
 

@@ -55,45 +55,61 @@ cudaError_t launch_quantize_rows(const float* x, long long rows, int cols, int q
     return cudaGetLastError();
 }
 
+// rint(x / s) clamped to +-127, bit-identical to quant_code (one IEEE division, then rintf) at a fraction of its cost:
+// the product with the reciprocal is within 3e-5 of the quotient for |x / s| <= 127, so both round to the same integer
+// unless the product lies within 1e-3 of a half-integer; only then the division decides.
+__device__ __forceinline__ int quant_code_127(float x, float s, float rs) {
+    const float t = x * rs;
+    float q = rintf(t);
+    if (fabsf(t - q) > 0.499f) q = rintf(__fdiv_rn(x, s));
+    return (int)fminf(fmaxf(q, -127.f), 127.f);
+}
+
 // Per-token quantizer of fp16 activations (the inputs of the integer-activation projections): one warp per row of
 // `cols` fp16 values (a multiple of 8), which it keeps in registers between the absmax pass and the code pass when the
-// row is short enough (up to 2048 columns), so that the row is read once.  Same arithmetic as quantize_rows_kernel.
+// row is short enough (KEEP x 256 columns), so that the row is read once.  Same results as quantize_rows_kernel.
+template <int KEEP>
 __global__ void __launch_bounds__(256) quantize_rows_f16_kernel(const __half* __restrict__ x, long long rows, int cols,
                                                                 int8_t* __restrict__ codes, float* __restrict__ scales) {
+    // Launched with the programmatic-serialization attribute: the successor (the integer GEMM) may start its prologue
+    // now; this kernel's input may come from the predecessor, so it is read only after the wait.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int lane = threadIdx.x & 31;
     const long long warps_total = (long long)gridDim.x * (blockDim.x >> 5);
     const int chunks = cols / 8;                                 // 16-byte chunks of a row
     for (long long r = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); r < rows; r += warps_total) {
         const uint4* xr = reinterpret_cast<const uint4*>(x + r * cols);
-        constexpr int KEEP = 8;                                  // chunks a lane keeps: 8 x 32 x 8 = 2048 columns
         uint4 keep[KEEP];
         float a = 0.f;
+        auto absmax8 = [&](const uint4& v) {
+            const __half2* h = reinterpret_cast<const __half2*>(&v);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) { const float2 f = __half22float2(h[e]); a = fmaxf(a, fmaxf(fabsf(f.x), fabsf(f.y))); }
+        };
 #pragma unroll
         for (int j = 0; j < KEEP; ++j) {
             const int i = lane + 32 * j;
             keep[j] = make_uint4(0, 0, 0, 0);
             if (i < chunks) keep[j] = xr[i];
-            const __half2* h = reinterpret_cast<const __half2*>(&keep[j]);
-#pragma unroll
-            for (int e = 0; e < 4; ++e) { const float2 f = __half22float2(h[e]); a = fmaxf(a, fmaxf(fabsf(f.x), fabsf(f.y))); }
         }
-        for (int i = lane + 32 * KEEP; i < chunks; i += 32) {
-            const uint4 v = xr[i];
-            const __half2* h = reinterpret_cast<const __half2*>(&v);
 #pragma unroll
-            for (int e = 0; e < 4; ++e) { const float2 f = __half22float2(h[e]); a = fmaxf(a, fmaxf(fabsf(f.x), fabsf(f.y))); }
-        }
+        for (int j = 0; j < KEEP; ++j) absmax8(keep[j]);
+        for (int i = lane + 32 * KEEP; i < chunks; i += 32) absmax8(xr[i]);
         a = warp_max(a);
         const float s = quant_scale(a, 127.f);
+        const float rs = s > 0.f ? __frcp_rn(s) : 0.f;
         if (lane == 0) scales[r] = s;
         uint2* cr = reinterpret_cast<uint2*>(codes + r * cols);
         auto encode = [&](const uint4& v) {
             const __half2* h = reinterpret_cast<const __half2*>(&v);
             uint32_t w[2] = {0, 0};
+            if (s > 0.f) {
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const float2 f = __half22float2(h[e]);
-                w[e >> 1] |= ((uint32_t)(quant_code(f.x, s, 127) & 0xFF) | ((uint32_t)(quant_code(f.y, s, 127) & 0xFF) << 8)) << (16 * (e & 1));
+                for (int e = 0; e < 4; ++e) {
+                    const float2 f = __half22float2(h[e]);
+                    w[e >> 1] |= ((uint32_t)(quant_code_127(f.x, s, rs) & 0xFF) | ((uint32_t)(quant_code_127(f.y, s, rs) & 0xFF) << 8)) << (16 * (e & 1));
+                }
             }
             return make_uint2(w[0], w[1]);
         };
@@ -110,8 +126,8 @@ cudaError_t launch_quantize_rows_f16(const __half* x, long long rows, int cols, 
     if (rows == 0) return cudaSuccess;
     long long blocks = (rows + 7) / 8;
     if (blocks > 148LL * 32) blocks = 148LL * 32;
-    quantize_rows_f16_kernel<<<(unsigned)blocks, 256, 0, stream>>>(x, rows, cols, codes, scales);
-    return cudaGetLastError();
+    if (cols <= 512) return launch_pdl(quantize_rows_f16_kernel<2>, dim3((unsigned)blocks), dim3(256), 0, stream, x, rows, cols, codes, scales);
+    return launch_pdl(quantize_rows_f16_kernel<8>, dim3((unsigned)blocks), dim3(256), 0, stream, x, rows, cols, codes, scales);
 }
 
 // One warp per (output channel, group).

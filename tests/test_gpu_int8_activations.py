@@ -28,6 +28,11 @@ def test_quantize_rows_f16_is_bit_exact(rows, cols):
     x[rows // 2] = 0                                      # an all-zero token: scale 0, codes 0
     if rows > 2:
         x[1, :] = np.float16(0.5) * np.sign(x[1, :])      # every element at the row maximum: codes +-127
+    if rows > 4 and cols >= 16:                           # exact ties: absmax 127 gives scale 1, half-integers round to even
+        x[3, :] = (r.integers(-126, 126, cols) + 0.5).astype(np.float16)
+        x[3, 0] = 127
+        x[4, :] = (r.integers(-252, 252, cols) * 0.25).astype(np.float16)       # scale 1/2 (absmax 63.5): quarter steps
+        x[4, 0] = 63.5
     codes, scales = tb.taq_quantize_rows_f16(dev(x))
     want_c, want_s = orc.quantize_rows(x.astype(np.float32), 127)
     assert np.array_equal(scales.cpu().numpy(), want_s)
