@@ -117,13 +117,15 @@ def dequantize_weights(codes: np.ndarray, scales: np.ndarray, group: int, contra
     return codes.astype(F64) * s_full.astype(F64)
 
 
-def quantize_prob(A: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
-    """uint8 quantizer of attention probabilities over [0,1]: code = rint(255 p) in float32,
-    p^ = float32(code) / 255.  Returns (codes int32, p^ float64)."""
+def quantize_prob(A: np.ndarray, bits: int = 8) -> Tuple[np.ndarray, np.ndarray]:
+    """Unsigned quantizer of attention probabilities over [0,1] with 2^bits levels: code = rint(pmax p) in
+    float32 with pmax = 2^bits - 1 (255 for uint8, 15 for the 4-bit rows of Table 1), p^ = float32(code) / pmax.
+    Returns (codes int32, p^ float64)."""
+    pmax = F32(2 ** bits - 1)
     p = np.asarray(A, dtype=F32)
-    code = np.rint((p * F32(255.0)).astype(F32))
-    code = np.clip(code, 0, 255).astype(np.int32)
-    p_hat = (code.astype(F32) / F32(255.0)).astype(F32)
+    code = np.rint((p * pmax).astype(F32))
+    code = np.clip(code, 0, int(pmax)).astype(np.int32)
+    p_hat = (code.astype(F32) / pmax).astype(F32)
     return code, p_hat.astype(F64)
 
 
@@ -142,8 +144,8 @@ class TaqConfig:
     w_bits: int = 8          # 0 = weights left unquantized
     w_group: int = 0
     q_bits: int = 8          # 8 = Eq. 2's Q~ = Q_a(Q); 0 = Q left unquantized
-    kv_bits: int = 8         # 8 = non-trigger K/V rows int8; 0 = no K/V quantization at all
-    p_bits: int = 8          # 8 = non-trigger probabilities uint8; 0 = no probability quantization
+    kv_bits: int = 8         # 8 / 4 = non-trigger K/V rows int8 / 4-bit (qmax 7); 0 = no K/V quantization at all
+    p_bits: int = 8          # 8 / 4 = non-trigger probabilities uint8 / 4-bit (15 levels); 0 = no probability quantization
     a_bits: int = 0          # 8 = inputs of the projections (X, ctx, O) int8 per token; 0 = left in fp16
     contract: bool = True    # fp16 storage roundings on (contract) or off (ideal)
 
@@ -198,7 +200,9 @@ def taq_kv(ctx: np.ndarray, Wk: np.ndarray, Wv: np.ndarray, mask_kv: np.ndarray,
             codes = np.zeros(Z.shape, dtype=np.int32)
             scales = np.zeros(Z.shape[:-1], dtype=F32)
         else:
-            codes, scales = quantize_rows(Z.astype(F32), 127)
+            if cfg.kv_bits not in (4, 8):
+                raise ValueError("kv_bits must be 0, 4 or 8")
+            codes, scales = quantize_rows(Z.astype(F32), 127 if cfg.kv_bits == 8 else 7)
             Zq = dequantize_rows(codes, scales).astype(F64)
             Zt = np.where(M, kept, Zq)                            # Eq. 2
         out[name + "_tilde"] = Zt
@@ -231,13 +235,16 @@ def taq_attention(Q_tilde: np.ndarray, K_tilde: np.ndarray, V_tilde: np.ndarray,
     S = S - S.max(axis=-1, keepdims=True)
     E = np.exp(S)
     A = E / E.sum(axis=-1, keepdims=True)
-    # Trigger columns are kept in fp16.  The stored probability tensor uses one unit for all columns, 1/255:
-    # ordinary columns hold the uint8 code, trigger columns hold fp16(255 A).
-    kept = f16_round(A * 255.0) / 255.0 if cfg.contract else A
+    # Trigger columns are kept in fp16.  The stored probability tensor uses one unit for all columns, 1/pmax
+    # (1/255 for uint8 codes): ordinary columns hold the integer code, trigger columns hold fp16(pmax A).
+    if cfg.p_bits not in (0, 4, 8):
+        raise ValueError("p_bits must be 0, 4 or 8")
+    pmax = float(2 ** cfg.p_bits - 1) if cfg.p_bits else 255.0
+    kept = f16_round(A * pmax) / pmax if cfg.contract else A
     if cfg.p_bits == 0:
         A_hat = np.where(M, kept, A)
     else:
-        _, Aq = quantize_prob(A)
+        _, Aq = quantize_prob(A, cfg.p_bits)
         A_hat = np.where(M, kept, Aq)                             # Eq. 3
     if cfg.contract:
         # Dequantized non-trigger V rows are fp16 matrix operands; trigger rows already are fp16.
@@ -265,6 +272,26 @@ def taq_layer(X, ctx, Wq, Wk, Wv, Wout, bout, mask, cfg: TaqConfig, mask_a=None)
     O = taq_attention(q["Q_tilde"], kv["K_tilde"], kv["V_tilde"], mask_a, cfg)
     Y = taq_out(O, Wout, bout, cfg)
     return {"Y": Y, "O": O, **{k: v for k, v in q.items()}, **{k: v for k, v in kv.items()}}
+
+
+def token_sensitivity(X, ctx, Wq, Wk, Wv, Wout, bout, cfg: TaqConfig, bits: int) -> np.ndarray:
+    """Per-token quantization sensitivity, Eq. 1, restated at the level of one layer: Delta_i(b) is the mean
+    squared difference between the layer output with ONLY the K and V rows of text token i quantized to b bits
+    and the output y* with no K/V row quantized.  Everything else is as ``cfg`` says in both runs (the paper
+    keeps it in full precision: pass w_bits = q_bits = 0); attention probabilities are not quantized in either
+    run (M_A all ones: the experiment touches K and V only).  Returns Delta [T], averaged over the batch."""
+    from dataclasses import replace
+    B, T = np.asarray(ctx).shape[:2]
+    ones = np.ones((B, T), dtype=np.uint8)
+    c = replace(cfg, kv_bits=bits)
+    y_star = taq_layer(X, ctx, Wq, Wk, Wv, Wout, bout, ones, c, mask_a=ones)["Y"]
+    delta = np.zeros(T, dtype=F64)
+    for i in range(T):
+        m = ones.copy()
+        m[:, i] = 0                                                # only token i's K/V rows pass through Q_b
+        y = taq_layer(X, ctx, Wq, Wk, Wv, Wout, bout, m, c, mask_a=ones)["Y"]
+        delta[i] = np.mean((y - y_star) ** 2)
+    return delta
 
 
 # ----------------------------------------------------------------------------------------------

@@ -477,9 +477,80 @@ def check_integer_activations(o):
         o.quantize_activations(X, o.TaqConfig(heads=H, a_bits=4))
 
 
+def check_four_bit_rows_and_probabilities(o):
+    """The 4-bit rows of Table 1 ("8/4"): K/V rows with qmax 7 and probabilities with 15 levels."""
+    code, ph = o.quantize_prob(np.array([0.0, 1.0, 1 / 15, 7.4 / 15, 7.6 / 15, 0.5]), 4)
+    assert code.tolist() == [0, 15, 1, 7, 8, 8] and abs(ph[2] - 1 / 15) < 1e-7       # 7.5 is a tie: to even
+    r = _rng(50)
+    A = r.dirichlet(np.ones(9), size=50)
+    c4, a4 = o.quantize_prob(A, 4)
+    assert c4.max() <= 15 and np.all(np.abs(a4 - A) <= 1 / 30 + 1e-7)
+    X, ctx, Wq, Wk, Wv, Wo, bo = _tiny_layer(51, B=1, N=4, H=2, d=8, T=6, Dc=16)
+    mask = np.zeros((1, 6), np.uint8); mask[0, 2] = 1
+    kv4 = o.taq_kv(ctx, Wk, Wv, mask, o.TaqConfig(heads=2, w_bits=0, kv_bits=4, contract=False))
+    assert np.abs(kv4["K_codes"]).max() == 7 and np.abs(kv4["V_codes"]).max() == 7
+    nt = [0, 1, 3, 4, 5]
+    assert np.all(np.max(np.abs(kv4["K_codes"][:, :, nt]), axis=-1) == 7)
+    np.testing.assert_array_equal(kv4["K_tilde"][:, :, 2], kv4["K"][:, :, 2])                 # the trigger row is untouched
+    err4 = np.abs(kv4["K_tilde"] - kv4["K"])[:, :, nt]
+    assert np.all(err4 <= kv4["K_scales"][:, :, nt, None] * 0.5000001)
+    kv8 = o.taq_kv(ctx, Wk, Wv, mask, o.TaqConfig(heads=2, w_bits=0, kv_bits=8, contract=False))
+    assert err4.mean() > 8 * np.abs(kv8["K_tilde"] - kv8["K"])[:, :, nt].mean()              # 127/7 = 18 times coarser
+    # empty mask, 4-bit everything == separately written uniform 4-bit attention
+    Q = o.split_heads(X.astype(np.float64) @ Wq.astype(np.float64).T, 2)
+    K, V = kv4["K"], kv4["V"]
+    def q4(Z):
+        cc, ss = o.quantize_rows(Z.astype(np.float32), 7)
+        return (cc.astype(np.float32) * ss[..., None]).astype(np.float64)
+    S = np.einsum("bhnd,bhtd->bhnt", Q, q4(K)) / np.sqrt(8.0)
+    E = np.exp(S - S.max(-1, keepdims=True)); Af = E / E.sum(-1, keepdims=True)
+    Ah = np.rint((Af.astype(np.float32) * np.float32(15)).astype(np.float32)).astype(np.float32) / np.float32(15)
+    want = o.merge_heads(np.einsum("bhnt,bhtd->bhnd", Ah.astype(np.float64), q4(V)))
+    got = o.taq_attention(Q, q4(K), q4(V), np.zeros((1, 6), np.uint8), o.TaqConfig(heads=2, p_bits=4, contract=False))
+    np.testing.assert_allclose(got, want, rtol=0, atol=1e-12)
+    with pytest.raises(ValueError):
+        o.taq_kv(ctx, Wk, Wv, mask, o.TaqConfig(heads=2, kv_bits=3))
+
+
+def check_token_sensitivity(o):
+    """Eq. 1 at layer level.  (i) one text token: the attention weight is 1, so y - y* = (V^ - V) Wout^T whatever the
+    queries are: Delta has a closed form; (ii) K/V rows that already lie on the b-bit grid give Delta = 0; (iii) 4 bits
+    hurt more than 8, and a row three times larger (the trigger rows of the workload) is more sensitive in absolute
+    terms than the others."""
+    full = dict(w_bits=0, q_bits=0, p_bits=0, contract=False)
+    X, ctx, Wq, Wk, Wv, Wo, bo = _tiny_layer(60, B=1, N=3, H=2, d=4, T=1, Dc=8)
+    for bits, qmax in ((8, 127), (4, 7)):
+        d = o.token_sensitivity(X, ctx, Wq, Wk, Wv, Wo, bo, o.TaqConfig(heads=2, **full), bits)
+        V = o.split_heads(ctx.astype(np.float64) @ Wv.astype(np.float64).T, 2)                 # [1,H,1,d]
+        c, s = o.quantize_rows(V.astype(np.float32), qmax)
+        dv = o.merge_heads((c.astype(np.float32) * s[..., None]).astype(np.float64) - V)[0, 0]  # [C]
+        want = np.mean((dv @ Wo.astype(np.float64).T) ** 2)
+        assert d.shape == (1,) and abs(d[0] - want) <= 1e-12 * want
+    # (ii): weights and context built so that K = V = integer codes with absmax 7 per (head, token) row
+    H, dd, T, Dc = 2, 4, 5, 8
+    C = H * dd
+    r = _rng(61)
+    ctxg = np.zeros((1, T, Dc), np.float16); ctxg[0, np.arange(T), np.arange(T)] = 1           # one-hot tokens
+    rows = r.integers(-7, 8, size=(T, C)).astype(np.float32)
+    rows[:, 0] = 7; rows[:, dd] = -7                                                            # absmax 7 in both heads
+    Wg = np.zeros((C, Dc), np.float32); Wg[:, :T] = rows.T
+    Xg = r.standard_normal((1, 3, C)).astype(np.float16)
+    Wqg = (r.standard_normal((C, C)) * 0.3).astype(np.float32)
+    dz = o.token_sensitivity(Xg, ctxg, Wqg, Wg, Wg, Wo[:C, :C] if Wo.shape[0] >= C else Wo, None, o.TaqConfig(heads=H, **full), 4)
+    assert np.all(dz == 0)
+    # (iii)
+    X3, ctx3, Wq3, Wk3, Wv3, Wo3, bo3 = _tiny_layer(62, B=2, N=24, H=2, d=8, T=8, Dc=32)
+    ctx3 = ctx3.astype(np.float32); ctx3[:, 3] *= 3; ctx3 = ctx3.astype(np.float16)
+    d8 = o.token_sensitivity(X3, ctx3, Wq3, Wk3, Wv3, Wo3, bo3, o.TaqConfig(heads=2, **full), 8)
+    d4 = o.token_sensitivity(X3, ctx3, Wq3, Wk3, Wv3, Wo3, bo3, o.TaqConfig(heads=2, **full), 4)
+    assert np.all(d8 > 0) and np.all(d4 > 20 * d8)
+    assert np.argmax(d4) == 3 and np.argmax(d8) == 3
+
+
 LAYER_CHECKS = [check_all_trigger_is_textbook_attention, check_empty_mask_is_uniform_quantization,
                 check_trigger_rows_pass_through, check_closed_forms, check_structure, check_brute_force,
-                check_contract_close_to_ideal, check_integer_activations]
+                check_contract_close_to_ideal, check_integer_activations, check_four_bit_rows_and_probabilities,
+                check_token_sensitivity]
 
 
 @pytest.mark.parametrize("check", LAYER_CHECKS)
@@ -539,7 +610,7 @@ MUTATIONS = {
     "k_v_swapped": [("taq_attention(q[\"Q_tilde\"], kv[\"K_tilde\"], kv[\"V_tilde\"]", "taq_attention(q[\"Q_tilde\"], kv[\"V_tilde\"], kv[\"K_tilde\"]")],
     "transposed_weight": [("ctx @ effective_weight(Wk, cfg).T", "ctx @ effective_weight(Wk, cfg)")],
     "q_not_quantized": [("if cfg.q_bits == 0:", "if True:")],
-    "prob_scale_256": [("code = np.rint((p * F32(255.0)).astype(F32))", "code = np.rint((p * F32(256.0)).astype(F32))")],
+    "prob_scale_256": [("pmax = F32(2 ** bits - 1)", "pmax = F32(2 ** bits)")],
     "clamp_asymmetric": [("q = np.clip(q, -qmax, qmax)", "q = np.clip(q, -qmax - 1, qmax - 1)")],
     "bias_dropped": [("Y = Y + np.asarray(bout, dtype=F64)", "Y = Y")],
     "renormalised_probs": [("A_hat = np.where(M, kept, Aq)                             # Eq. 3",
@@ -550,6 +621,10 @@ MUTATIONS = {
     "out_input_not_quantized": [("Y = quantize_activations(O, cfg) @ effective_weight(Wout, cfg).T", "Y = np.asarray(O, dtype=F64) @ effective_weight(Wout, cfg).T")],
     "activation_scale_per_tensor": [("    codes, scales = quantize_rows(x.astype(F32), 127)\n    return codes.astype(F64) * scales",
                                      "    codes, scales = quantize_rows(x.astype(F32).reshape(1, -1), 127)\n    codes = codes.reshape(x.shape); scales = np.broadcast_to(scales, x.shape[:-1])\n    return codes.astype(F64) * scales")],
+    "four_bit_rows_use_qmax_8": [("127 if cfg.kv_bits == 8 else 7", "127 if cfg.kv_bits == 8 else 8")],
+    "four_bit_probs_use_8_bit_levels": [("_, Aq = quantize_prob(A, cfg.p_bits)", "_, Aq = quantize_prob(A, 8)")],
+    "sensitivity_quantizes_all_but_i": [("        m = ones.copy()\n        m[:, i] = 0", "        m = 1 - ones\n        m[:, i] = 1")],
+    "sensitivity_reference_quantized": [("y_star = taq_layer(X, ctx, Wq, Wk, Wv, Wout, bout, ones, c, mask_a=ones)", "y_star = taq_layer(X, ctx, Wq, Wk, Wv, Wout, bout, 1 - ones, c, mask_a=ones)")],
     "heads_interleaved": [("return x.reshape(B, L, heads, d).transpose(0, 2, 1, 3)", "return x.reshape(B, L, d, heads).transpose(0, 3, 1, 2)")],
 }
 
