@@ -103,8 +103,9 @@ typedef struct {
     int32_t w_bits;       /* 4 or 8: format of all four packed projections of the layer */
     int32_t w_group;      /* 0 or group length */
     int32_t q_bits;       /* 8: Q~ = Q_a(Q) (Eq. 2, third line); 0: Q stays fp16 */
-    int32_t kv_bits;      /* 8 */
-    int32_t p_bits;       /* 8 */
+    int32_t kv_bits;      /* 8: ordinary K/V rows int8 (codes in [-127,127]); 4: 4-bit rows (codes in [-7,7], the "8/4" rows
+                             of Table 1; stored one code per byte) */
+    int32_t p_bits;       /* 8: ordinary probabilities uint8, code = rint(255 p); 4: 16 levels, code = rint(15 p) */
     int32_t max_trigger;  /* capacity of fp16 trigger rows per sequence, 0..n_ctx */
 } taq_layer_desc;
 
@@ -231,6 +232,27 @@ size_t taq_kv_project_a8_workspace_bytes(const taq_layer_desc* desc);
 taq_status taq_kv_project_a8(const taq_layer_desc* desc, const void* ctx_f16_dev, const void* Wk_packed_dev,
                              const void* Wv_packed_dev, const uint8_t* trig_mask_dev, void* kv_packed_dev,
                              size_t kv_bytes, void* workspace_dev, size_t workspace_bytes, void* stream);
+
+/* --------------------------------------------------------------------------------------------------------
+ * Token-specific quantization sensitivity (Sec. III-B, Eq. 1), restated for one layer: Delta_i(b) = mean squared
+ * difference between the layer output with ONLY the K and V rows of text token i quantized to b bits and the
+ * output y* with no K/V row quantized.  b = desc->kv_bits (8 or 4); everything else as desc says in both runs
+ * (weights as packed, q_bits; no attention probability is quantized in either run: Eq. 3's M_A is all ones,
+ * the experiment touches K and V only).  desc->max_trigger must equal n_ctx.  n_ctx + 1 K/V projections and
+ * layer passes plus n_ctx reductions are enqueued; delta_dev receives fp64 [n_ctx].
+ * -------------------------------------------------------------------------------------------------------- */
+size_t taq_token_sensitivity_workspace_bytes(const taq_layer_desc* desc);
+taq_status taq_token_sensitivity(const taq_layer_desc* desc, const void* x_f16_dev, const void* ctx_f16_dev,
+                                 const void* Wq_packed_dev, const void* Wk_packed_dev, const void* Wv_packed_dev,
+                                 const void* Wout_packed_dev, double* delta_dev, void* workspace_dev,
+                                 size_t workspace_bytes, void* stream);
+
+/* Eq. 3's mask M_A chosen independently of Eq. 2's M_KV (by default a probability column stays fp16 exactly when
+ * its K/V rows do): rewrites the operand images of `batch` blocks so that the columns marked in mask_a_dev
+ * (u8 [B][T]) stay fp16 and the others become codes.  Pass the same mask as trig_mask_dev to the attention and
+ * layer calls that use the blocks. */
+taq_status taq_kv_set_prob_mask(const taq_layer_desc* desc, void* kv_packed_dev, size_t kv_bytes,
+                                const uint8_t* mask_a_dev, void* stream);
 
 /* Batched serving (Sec. I: many personalized checkpoints served concurrently): request r is one sequence
  * (desc->batch must be 1) whose activations are slice r of x/y [n_requests][N][C] and which carries its own

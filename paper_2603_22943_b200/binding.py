@@ -26,7 +26,8 @@ EXPORTS = [
     "taq_layer_forward_batched", "taq_kv_project_batched", "taq_poll_device_status",
     "taq_static_workspace_capacity", "taq_layer_forward_static", "taq_kv_finalize", "taq_query_attention",
     "taq_quantize_rows_f16", "taq_quantized_linear_i8", "taq_workspace_bytes_a8", "taq_layer_forward_a8",
-    "taq_kv_project_a8_workspace_bytes", "taq_kv_project_a8",
+    "taq_kv_project_a8_workspace_bytes", "taq_kv_project_a8", "taq_token_sensitivity_workspace_bytes",
+    "taq_token_sensitivity", "taq_kv_set_prob_mask",
 ]
 
 
@@ -106,6 +107,10 @@ def lib() -> C.CDLL:
         L.taq_kv_project_a8_workspace_bytes.restype = sz
         L.taq_kv_project_a8_workspace_bytes.argtypes = [C.POINTER(LayerDesc)]
         L.taq_kv_project_a8.argtypes = [C.POINTER(LayerDesc), vp, vp, vp, vp, vp, sz, vp, sz, vp]
+        L.taq_token_sensitivity_workspace_bytes.restype = sz
+        L.taq_token_sensitivity_workspace_bytes.argtypes = [C.POINTER(LayerDesc)]
+        L.taq_token_sensitivity.argtypes = [C.POINTER(LayerDesc), vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.taq_kv_set_prob_mask.argtypes = [C.POINTER(LayerDesc), vp, sz, vp, vp]
         for name in EXPORTS:
             f = getattr(L, name)
             if f.restype is C.c_int and name not in ("taq_version",):
@@ -272,6 +277,22 @@ def taq_kv_project_a8(desc: LayerDesc, ctx: torch.Tensor, Wk_packed: torch.Tenso
     _check(lib().taq_kv_project_a8(C.byref(desc), _ptr(ctx), _ptr(Wk_packed), _ptr(Wv_packed), _ptr(trig_mask), _ptr(kv), kv.numel(),
                                    _ptr(workspace), workspace.numel(), _stream(stream)))
     return kv
+
+
+def taq_kv_set_prob_mask(desc: LayerDesc, kv: torch.Tensor, mask_a: torch.Tensor, stream=None) -> torch.Tensor:
+    """Eq. 3's M_A independent of Eq. 2's M_KV: the columns marked in mask_a stay fp16."""
+    _check(lib().taq_kv_set_prob_mask(C.byref(desc), _ptr(kv), kv.numel(), _ptr(mask_a), _stream(stream)))
+    return kv
+
+
+def taq_token_sensitivity(desc: LayerDesc, x: torch.Tensor, ctx: torch.Tensor, Wq_packed: torch.Tensor, Wk_packed: torch.Tensor,
+                          Wv_packed: torch.Tensor, Wout_packed: torch.Tensor, stream=None) -> torch.Tensor:
+    """Eq. 1 at layer level: fp64 [n_ctx], Delta_i for b = desc.kv_bits."""
+    delta = torch.zeros(desc.n_ctx, dtype=torch.float64, device=x.device)
+    ws = torch.empty(max(lib().taq_token_sensitivity_workspace_bytes(C.byref(desc)), 128), dtype=torch.uint8, device=x.device)
+    _check(lib().taq_token_sensitivity(C.byref(desc), _ptr(x), _ptr(ctx), _ptr(Wq_packed), _ptr(Wk_packed), _ptr(Wv_packed),
+                                       _ptr(Wout_packed), _ptr(delta), _ptr(ws), ws.numel(), _stream(stream)))
+    return delta
 
 
 def taq_cross_attention(desc: LayerDesc, q: torch.Tensor, q_scales: Optional[torch.Tensor], kv: torch.Tensor,

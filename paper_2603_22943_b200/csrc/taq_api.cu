@@ -63,8 +63,8 @@ static taq_status check_layer_desc(const taq_layer_desc* d) {
     if (d->ctx_dim < 8 || d->ctx_dim % 8) return fail(TAQ_ERR_SHAPE, "ctx_dim must be a positive multiple of 8, got %d", d->ctx_dim);
     if (d->w_bits != 4 && d->w_bits != 8) return fail(TAQ_ERR_INVALID_ARG, "w_bits must be 4 or 8, got %d", d->w_bits);
     if (d->q_bits != 0 && d->q_bits != 8) return fail(TAQ_ERR_INVALID_ARG, "q_bits must be 0 or 8, got %d", d->q_bits);
-    if (d->kv_bits != 8) return fail(TAQ_ERR_UNSUPPORTED, "kv_bits must be 8, got %d", d->kv_bits);
-    if (d->p_bits != 8) return fail(TAQ_ERR_UNSUPPORTED, "p_bits must be 8, got %d", d->p_bits);
+    if (d->kv_bits != 8 && d->kv_bits != 4) return fail(TAQ_ERR_UNSUPPORTED, "kv_bits must be 8 or 4, got %d", d->kv_bits);
+    if (d->p_bits != 8 && d->p_bits != 4) return fail(TAQ_ERR_UNSUPPORTED, "p_bits must be 8 or 4, got %d", d->p_bits);
     if (d->max_trigger < 0 || d->max_trigger > d->n_ctx) return fail(TAQ_ERR_SHAPE, "max_trigger must be in [0,n_ctx], got %d", d->max_trigger);
     if ((long long)d->batch * d->n_query > (1LL << 31) - 1) return fail(TAQ_ERR_SHAPE, "batch * n_query too large");
     taq_weight_desc w{d->channels, d->channels, d->w_bits, d->w_group};
@@ -191,7 +191,7 @@ static taq_status kv_project_impl(const taq_layer_desc* d, const taq_request* re
     a.rows = (long long)d->batch * d->n_ctx;
     a.n_out = d->channels; a.k_in = d->ctx_dim; a.bits = d->w_bits; a.group = d->w_group;
     a.heads = d->heads; a.n_ctx = d->n_ctx; a.max_trigger = d->max_trigger;
-    a.epi = EPI_KV;
+    a.epi = EPI_KV; a.kv_qmax = d->kv_bits == 4 ? 7 : 127;
     a.status = status;
     for (int which = 0; which < 2; ++which) {
         a.w = which ? Wv : Wk;
@@ -547,7 +547,7 @@ taq_status taq_kv_project_a8(const taq_layer_desc* d, const void* ctx_f16_dev, c
     a.rows = rows;
     a.n_out = d->channels; a.k_in = d->ctx_dim; a.bits = d->w_bits; a.group = d->w_group;
     a.heads = d->heads; a.n_ctx = d->n_ctx; a.max_trigger = d->max_trigger;
-    a.epi = EPI_KV;
+    a.epi = EPI_KV; a.kv_qmax = d->kv_bits == 4 ? 7 : 127;
     a.status = status;
     for (int which = 0; which < 2; ++which) {
         a.w = which ? Wv_packed_dev : Wk_packed_dev;
@@ -558,6 +558,84 @@ taq_status taq_kv_project_a8(const taq_layer_desc* d, const void* ctx_f16_dev, c
     }
     e = launch_kv_operands(*d, kv_packed_dev, nullptr, d->batch, st);
     return e == cudaSuccess ? TAQ_OK : cuda_fail(e, "K/V operand image launch");
+}
+
+// ---- Eq. 3's M_A chosen independently of Eq. 2's M_KV; the token-sensitivity sweep of Eq. 1 -------------------------
+
+taq_status taq_kv_set_prob_mask(const taq_layer_desc* d, void* kv_packed_dev, size_t kv_bytes, const uint8_t* mask_a_dev, void* stream) {
+    taq_status s = check_layer_desc(d);
+    if (s != TAQ_OK) return s;
+    if (d->batch == 0) return TAQ_OK;
+    if (d->batch > 65535) return fail(TAQ_ERR_SHAPE, "batch must be at most 65535");
+    TAQ_REQUIRE_PTR(kv_packed_dev);
+    if (!mask_a_dev) return fail(TAQ_ERR_INVALID_ARG, "mask_a_dev is NULL");
+    const size_t need = taq_kv_bytes(d);
+    if (kv_bytes < need) return fail(TAQ_ERR_BUFFER_TOO_SMALL, "kv buffer has %zu bytes, %zu needed", kv_bytes, need);
+    cudaError_t e = launch_kv_operands(*d, kv_packed_dev, nullptr, d->batch, (cudaStream_t)stream, mask_a_dev);
+    return e == cudaSuccess ? TAQ_OK : cuda_fail(e, "K/V operand image launch");
+}
+
+struct SensWorkspace { size_t off_masks, off_kv, off_ystar, off_y, off_partials, off_layer, total; };
+static SensWorkspace sens_layout(const taq_layer_desc* d) {
+    SensWorkspace w;
+    const size_t act = align_up((size_t)d->batch * d->n_query * d->channels * sizeof(__half), 128);
+    w.off_masks = 0;
+    w.off_kv = align_up((size_t)(d->n_ctx + 1) * d->batch * d->n_ctx, 128);
+    w.off_ystar = w.off_kv + align_up(taq_kv_bytes(d), 128);
+    w.off_y = w.off_ystar + act;
+    w.off_partials = w.off_y + act;
+    w.off_layer = w.off_partials + align_up(256 * sizeof(double), 128);
+    w.total = w.off_layer + workspace_layout(d, 1).total;
+    return w;
+}
+
+size_t taq_token_sensitivity_workspace_bytes(const taq_layer_desc* d) {
+    if (check_layer_desc(d) != TAQ_OK) return 0;
+    return sens_layout(d).total;
+}
+
+taq_status taq_token_sensitivity(const taq_layer_desc* d, const void* x_f16_dev, const void* ctx_f16_dev, const void* Wq_packed_dev,
+                                 const void* Wk_packed_dev, const void* Wv_packed_dev, const void* Wout_packed_dev, double* delta_dev,
+                                 void* workspace_dev, size_t workspace_bytes, void* stream) {
+    taq_status s = check_layer_desc(d);
+    if (s != TAQ_OK) return s;
+    if (d->batch < 1 || d->n_query < 1) return fail(TAQ_ERR_SHAPE, "batch and n_query must be positive");
+    if (d->batch > 65535) return fail(TAQ_ERR_SHAPE, "batch must be at most 65535");
+    if (d->max_trigger < d->n_ctx) return fail(TAQ_ERR_SHAPE, "the sweep keeps up to n_ctx rows in fp16: max_trigger (%d) must equal n_ctx (%d)", d->max_trigger, d->n_ctx);
+    TAQ_REQUIRE_PTR(x_f16_dev);
+    TAQ_REQUIRE_PTR(ctx_f16_dev);
+    TAQ_REQUIRE_PTR(Wq_packed_dev);
+    TAQ_REQUIRE_PTR(Wk_packed_dev);
+    TAQ_REQUIRE_PTR(Wv_packed_dev);
+    TAQ_REQUIRE_PTR(Wout_packed_dev);
+    TAQ_REQUIRE_PTR(delta_dev);
+    TAQ_REQUIRE_PTR(workspace_dev);
+    if (reinterpret_cast<uintptr_t>(workspace_dev) & 127u) return fail(TAQ_ERR_ALIGNMENT, "workspace_dev is not 128-byte aligned");
+    const SensWorkspace W = sens_layout(d);
+    if (workspace_bytes < W.total) return fail(TAQ_ERR_BUFFER_TOO_SMALL, "workspace has %zu bytes, %zu needed", workspace_bytes, W.total);
+    cudaStream_t st = (cudaStream_t)stream;
+    uint8_t* wsb = (uint8_t*)workspace_dev;
+    uint8_t* masks = wsb + W.off_masks;
+    const size_t mask_stride = (size_t)d->batch * d->n_ctx;
+    const uint8_t* ones = masks + (size_t)d->n_ctx * mask_stride;
+    const long long n = (long long)d->batch * d->n_query * d->channels;
+    cudaError_t e = launch_sensitivity_masks(masks, d->batch, d->n_ctx, st);
+    if (e != cudaSuccess) return cuda_fail(e, "sensitivity mask launch");
+    for (int i = d->n_ctx; i >= 0; --i) {       // i = n_ctx first: the reference y* with no K/V row quantized
+        const int which = (i == d->n_ctx) ? d->n_ctx : i;
+        void* y = wsb + (which == d->n_ctx ? W.off_ystar : W.off_y);
+        s = kv_project_impl(d, nullptr, 1, ctx_f16_dev, Wk_packed_dev, Wv_packed_dev, masks + (size_t)which * mask_stride, wsb + W.off_kv, st);
+        if (s != TAQ_OK) return s;
+        e = launch_kv_operands(*d, wsb + W.off_kv, nullptr, d->batch, st, ones);      // M_A: every probability column stays fp16
+        if (e != cudaSuccess) return cuda_fail(e, "K/V operand image launch");
+        s = layer_forward_impl(d, nullptr, 1, x_f16_dev, Wq_packed_dev, Wout_packed_dev, wsb + W.off_kv, ones, y, wsb + W.off_layer, st);
+        if (s != TAQ_OK) return s;
+        if (which != d->n_ctx) {
+            e = launch_mse_f16((const __half*)(wsb + W.off_y), (const __half*)(wsb + W.off_ystar), n, (double*)(wsb + W.off_partials), delta_dev + which, st);
+            if (e != cudaSuccess) return cuda_fail(e, "mse launch");
+        }
+    }
+    return TAQ_OK;
 }
 
 taq_status taq_query_attention(const taq_layer_desc* d, const void* x_f16_dev, const void* Wq_packed_dev, const void* kv_packed_dev,

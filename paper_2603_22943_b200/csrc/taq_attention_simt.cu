@@ -108,8 +108,9 @@ __global__ void __launch_bounds__(ATT_WARPS * 32) attention_simt_kernel(const At
             if (j < T) {
                 const float pj = __fdiv_rn(s[u], sum);
                 float ph;
-                if (msk[j] || a.p_bits == 0) ph = __fdiv_rn(__half2float(__float2half_rn(__fmul_rn(pj, 255.0f))), 255.0f);   // Eq. 3, trigger column: fp16 in units of 1/255
-                else ph = __fdiv_rn(rintf(__fmul_rn(pj, 255.0f)), 255.0f);                           // Eq. 3, uint8 code / 255
+                const float pmax = a.p_bits == 4 ? 15.0f : 255.0f;                                  // levels of the code: 2^bits - 1
+                if (msk[j] || a.p_bits == 0) ph = __fdiv_rn(__half2float(__float2half_rn(__fmul_rn(pj, pmax))), pmax);     // Eq. 3, trigger column: fp16 in units of 1/pmax
+                else ph = __fdiv_rn(rintf(__fmul_rn(pj, pmax)), pmax);                               // Eq. 3, integer code / pmax
                 p[j] = ph;
             }
         }

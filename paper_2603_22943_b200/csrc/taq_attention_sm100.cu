@@ -213,7 +213,8 @@ __global__ void __launch_bounds__(ATT_THREADS, Cfg<D>::CTAS_PER_SM) attention_sm
         const size_t grow = (size_t)zb * a.n_query + (valid ? n : 0);
         const uint32_t lane_addr = (uint32_t)(q4 * 32) << 16;
         const int key0 = half * HK;
-        const float inv255 = 1.0f / 255.0f;
+        const float pmax = a.p_bits == 4 ? 15.0f : 255.0f;     // probabilities are held in units of 1 / pmax (uint8 or 4-bit codes)
+        const float inv255 = 1.0f / pmax;
         constexpr int CH2 = QRegs<D, Q8>::CH2;
         constexpr int OC = DP / 2;                       // O columns per thread
         bool alive = true;
@@ -294,7 +295,7 @@ __global__ void __launch_bounds__(ATT_THREADS, Cfg<D>::CTAS_PER_SM) attention_sm
             const float2 other = misc->xchg[ph][half ^ 1][r];
             const float m_all = fmaxf(m_loc, other.x);
             const float c_self = ex2_approx(m_loc - m_all), c_other = ex2_approx(other.x - m_all);
-            const float k255 = __fdividef(255.0f * c_self, fmaf(l_loc, c_self, other.y * c_other));
+            const float k255 = __fdividef(pmax * c_self, fmaf(l_loc, c_self, other.y * c_other));
 
             // the P tile is free once the previous head's PV has completed
             if (hi > 0) {
@@ -368,7 +369,7 @@ cudaError_t launch_d(const AttnArgs& a, int n_z, cudaStream_t stream) {
 bool sm100_attention_supported(const AttnArgs& a) {
     OperandGeom g;
     if (!operand_geom(a.channels / a.heads, a.n_ctx, &g)) return false;
-    if (a.p_bits != 8) return false;
+    if (a.p_bits != 8 && a.p_bits != 4) return false;
     if (a.heads > 65535) return false;
     return true;
 }

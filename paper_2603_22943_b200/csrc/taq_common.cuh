@@ -136,6 +136,7 @@ struct LinearArgs {
     int heads;                  // EPI_Q8_HEAD / EPI_KV
     int n_ctx, max_trigger;     // EPI_KV: rows = batch * n_ctx
     int kv_which;               // EPI_KV: 0 = K, 1 = V
+    int kv_qmax;                // EPI_KV: 127 (int8 rows) or 7 (4-bit rows); 0 is read as 127
     int epi;
     int w_direct;               // (set by the launcher) int8 activations and 8-bit weights: the weight codes are the B
                                 // operand as they are and go from the blob into the ring by TMA, no staging or expansion
@@ -200,7 +201,11 @@ cudaError_t launch_quantize_rows(const float* x, long long rows, int cols, int q
                                  cudaStream_t stream);
 cudaError_t launch_pack_weights(const taq_weight_desc& d, const float* W, const float* bias, void* packed,
                                 cudaStream_t stream);
-cudaError_t launch_kv_operands(const taq_layer_desc& d, void* kv, const taq_request* reqs, int n_z, cudaStream_t stream);
+cudaError_t launch_kv_operands(const taq_layer_desc& d, void* kv, const taq_request* reqs, int n_z, cudaStream_t stream, const uint8_t* mask_a = nullptr);
+// Mean squared difference of two fp16 arrays into *out (fp64), deterministic two-stage sum; partials: 256 doubles of scratch.
+cudaError_t launch_mse_f16(const __half* a, const __half* b, long long n, double* partials, double* out, cudaStream_t stream);
+// masks[i][b][t] = (t != i) for i < T, all ones for i = T  (u8 [T+1][B][T])
+cudaError_t launch_sensitivity_masks(uint8_t* masks, int batch, int n_ctx, cudaStream_t stream);
 cudaError_t launch_unpack_weights(const taq_weight_desc& d, const void* packed, int8_t* codes, float* scales,
                                   cudaStream_t stream);
 

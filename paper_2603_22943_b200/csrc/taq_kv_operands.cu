@@ -10,7 +10,9 @@ namespace taq {
 namespace {
 
 // One CTA per (head, sequence).
-__global__ void __launch_bounds__(256) kv_operands_kernel(const taq_layer_desc d, uint8_t* kv, const taq_request* reqs) {
+// `mask_a` (nullable, u8 [sequences][T]) overrides which probability columns stay fp16 (Eq. 3's M_A); by default they
+// are the columns of the fp16 K/V rows (M_A = M_KV).
+__global__ void __launch_bounds__(256) kv_operands_kernel(const taq_layer_desc d, uint8_t* kv, const taq_request* reqs, const uint8_t* mask_a) {
     const int H = d.heads, T = d.n_ctx, D = d.channels / d.heads;
     const int h = blockIdx.x, z = blockIdx.y;
     const taq_kv_layout KL = kv_layout(H, T, D, d.max_trigger);
@@ -58,7 +60,7 @@ __global__ void __launch_bounds__(256) kv_operands_kernel(const taq_layer_desc d
         uint32_t bits = 0;
         for (int i = 0; i < 32; ++i) {
             const int j = threadIdx.x * 32 + i;
-            if (j < T && slot[j] >= 0) bits |= 1u << i;
+            if (j < T && (mask_a ? mask_a[(size_t)z * T + j] != 0 : slot[j] >= 0)) bits |= 1u << i;
         }
         cst->trig_bits[threadIdx.x] = bits;
     }
@@ -66,11 +68,11 @@ __global__ void __launch_bounds__(256) kv_operands_kernel(const taq_layer_desc d
 
 }  // namespace
 
-cudaError_t launch_kv_operands(const taq_layer_desc& d, void* kv, const taq_request* reqs, int n_z, cudaStream_t stream) {
+cudaError_t launch_kv_operands(const taq_layer_desc& d, void* kv, const taq_request* reqs, int n_z, cudaStream_t stream, const uint8_t* mask_a) {
     OperandGeom g;
     if (n_z == 0 || !operand_geom(d.channels / d.heads, d.n_ctx, &g)) return cudaSuccess;
     dim3 grid(d.heads, n_z);
-    kv_operands_kernel<<<grid, 256, 0, stream>>>(d, (uint8_t*)kv, reqs);
+    kv_operands_kernel<<<grid, 256, 0, stream>>>(d, (uint8_t*)kv, reqs, mask_a);
     return cudaGetLastError();
 }
 

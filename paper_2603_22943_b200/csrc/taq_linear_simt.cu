@@ -106,7 +106,8 @@ __global__ void __launch_bounds__(256) linear_simt_kernel(const LinearArgs a) {
 #pragma unroll
         for (int o = 8; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
         if (row >= a.rows) continue;
-        const float s = quant_scale(amax, 127.f);
+        const int qmax = a.epi == EPI_KV && a.kv_qmax ? a.kv_qmax : 127;
+        const float s = quant_scale(amax, (float)qmax);
         if (a.epi == EPI_Q8_HEAD) {
             int8_t* yq = (int8_t*)a.y + ((size_t)z * a.rows + row) * a.n_out + col0;
 #pragma unroll
@@ -132,7 +133,7 @@ __global__ void __launch_bounds__(256) linear_simt_kernel(const LinearArgs a) {
             for (int j = 0; j < TN; ++j) {
                 const int c = tx + 16 * j;
                 if (c >= ncols) continue;
-                cq[c] = trig ? (int8_t)0 : (int8_t)quant_code(acc[i][j], s, 127);
+                cq[c] = trig ? (int8_t)0 : (int8_t)quant_code(acc[i][j], s, qmax);
                 if (slot >= 0) tr[((size_t)slot * a.heads + h) * d + c] = __float2half_rn(acc[i][j]);
             }
             if (tx == 0) {

@@ -399,7 +399,7 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
                         asm volatile("bar.sync 2, 256;" ::: "memory");
                         amax = fmaxf(amax, xchg[(half ^ 1) * 128 + r]);
                     }
-                    const float s = quant_scale(amax, 127.f);
+                    const float s = quant_scale(amax, a.epi == EPI_KV && a.kv_qmax ? (float)a.kv_qmax : 127.f);
                     const float rs = s > 0.f ? __frcp_rn(s) : 0.f;
                     const bool owner = whole_heads || half == 0;      // writes the head's scale
                     if (a.epi == EPI_Q8_HEAD) {

@@ -130,6 +130,49 @@ cudaError_t launch_quantize_rows_f16(const __half* x, long long rows, int cols, 
     return launch_pdl(quantize_rows_f16_kernel<8>, dim3((unsigned)blocks), dim3(256), 0, stream, x, rows, cols, codes, scales);
 }
 
+// ---- helpers of the token-sensitivity sweep (Eq. 1) -------------------------------------------------------------
+__global__ void __launch_bounds__(256) mse_partial_kernel(const __half* __restrict__ a, const __half* __restrict__ b, long long n, double* __restrict__ partials) {
+    double acc = 0.0;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+        const float dlt = __half2float(a[i]) - __half2float(b[i]);
+        acc += (double)dlt * (double)dlt;
+    }
+    __shared__ double sh[256];
+    sh[threadIdx.x] = acc;
+    __syncthreads();
+    for (int s = 128; s > 0; s >>= 1) {           // fixed tree: the same sum for the same inputs
+        if (threadIdx.x < s) sh[threadIdx.x] += sh[threadIdx.x + s];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) partials[blockIdx.x] = sh[0];
+}
+__global__ void __launch_bounds__(256) mse_final_kernel(const double* __restrict__ partials, long long n, double* __restrict__ out) {
+    __shared__ double sh[256];
+    sh[threadIdx.x] = partials[threadIdx.x];
+    __syncthreads();
+    for (int s = 128; s > 0; s >>= 1) {
+        if (threadIdx.x < s) sh[threadIdx.x] += sh[threadIdx.x + s];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) *out = sh[0] / (double)n;
+}
+cudaError_t launch_mse_f16(const __half* a, const __half* b, long long n, double* partials, double* out, cudaStream_t stream) {
+    mse_partial_kernel<<<256, 256, 0, stream>>>(a, b, n, partials);
+    mse_final_kernel<<<1, 256, 0, stream>>>(partials, n, out);
+    return cudaGetLastError();
+}
+__global__ void sensitivity_masks_kernel(uint8_t* masks, int batch, int n_ctx) {
+    const long long total = (long long)(n_ctx + 1) * batch * n_ctx;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+        const int t = (int)(i % n_ctx), which = (int)(i / ((long long)batch * n_ctx));
+        masks[i] = (which == n_ctx || t != which) ? 1 : 0;
+    }
+}
+cudaError_t launch_sensitivity_masks(uint8_t* masks, int batch, int n_ctx, cudaStream_t stream) {
+    sensitivity_masks_kernel<<<64, 256, 0, stream>>>(masks, batch, n_ctx);
+    return cudaGetLastError();
+}
+
 // One warp per (output channel, group).
 __global__ void __launch_bounds__(256) pack_weights_kernel(const float* __restrict__ W, const float* __restrict__ bias, uint8_t* __restrict__ blob,
                                                            int n_out, int k_in, int bits, int group) {

@@ -84,7 +84,7 @@ struct QAttnArgs {
     __half* o;                  // [z][B][N][C]  (query-attention variant)
     const void* wout;           // packed [C][C] (layer variant, single problem)
     __half* y;                  // [z][B][N][C]  (layer variant)
-    int n_query, heads, n_ctx, max_trigger, group, q_bits;
+    int n_query, heads, n_ctx, max_trigger, group, q_bits, p_bits;
     int* status;
 };
 
@@ -523,7 +523,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
         // ---- phase 3: group g = part / 2 takes heads g and g + 2; this thread has keys [40 half, 40 half + 40) of its row ----
         const int grp = part >> 1, half = part & 1;
         const int key0 = half * HK;
-        const float inv255 = 1.0f / 255.0f;
+        const float pmax = a.p_bits == 4 ? 15.0f : 255.0f;     // probabilities are held in units of 1 / pmax (uint8 or 4-bit codes)
+        const float inv255 = 1.0f / pmax;
         constexpr int OC = DP / 2;
         bool alive = ok;
         auto store_o = [&](int hi) {
@@ -601,7 +602,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
             const float2 other = xchg[(half ^ 1) * ROWS + r];
             const float m_all = fmaxf(m_loc, other.x);
             const float c_self = ex2_approx(m_loc - m_all), c_other = ex2_approx(other.x - m_all);
-            const float k255 = __fdividef(255.0f * c_self, fmaf(l_loc, c_self, other.y * c_other));
+            const float k255 = __fdividef(pmax * c_self, fmaf(l_loc, c_self, other.y * c_other));
             if (it > 0 && lane == 0 && q4 == 0 && half == 0) TAQ_PROF(55 + grp);
             if (it > 0) {       // the group's P tile and O accumulator are free once its previous PV is complete and O is stored
                 alive = __all_sync(0xffffffffu, ptx::mbar_wait(&misc->o_full[grp], 0) && !misc->abort_flag);
@@ -707,7 +708,7 @@ bool sm100_qattn_supported(const taq_layer_desc& d) {
     if (d.channels != KIN || d.heads * D != KIN) return false;
     if (d.w_bits != 4) return false;
     if (d.w_group != 0 && (d.w_group % BK || (KIN + d.w_group - 1) / d.w_group > MAX_GROUPS)) return false;
-    if (d.n_ctx > TP || d.p_bits != 8) return false;
+    if (d.n_ctx > TP || (d.p_bits != 8 && d.p_bits != 4)) return false;
     if (d.n_query < 1) return false;
     return encode_tiled_fn2() != nullptr;
 }
@@ -727,7 +728,7 @@ static cudaError_t launch_c320(const taq_layer_desc& d, const __half* x, const v
     if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
     QAttnArgs a{};
     a.x = x; a.wq = wq; a.kv = kv; a.reqs = reqs; a.o = o; a.wout = wout; a.y = y;
-    a.n_query = d.n_query; a.heads = d.heads; a.n_ctx = d.n_ctx; a.max_trigger = d.max_trigger; a.group = d.w_group; a.q_bits = d.q_bits;
+    a.n_query = d.n_query; a.heads = d.heads; a.n_ctx = d.n_ctx; a.max_trigger = d.max_trigger; a.group = d.w_group; a.q_bits = d.q_bits; a.p_bits = d.p_bits;
     a.status = status;
     dim3 grid((d.n_query + ROWS - 1) / ROWS, d.heads / HG, n_z);
     static bool configured[4] = {false, false, false, false};

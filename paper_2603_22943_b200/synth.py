@@ -37,6 +37,8 @@ class LayerShape:
     w_group: int         # 0 = one scale per output channel, 128 = groups along fan-in
     trigger: Tuple[int, ...]  # trigger span positions (I_sks)
     q_bits: int = 8      # 8: Q is quantized (Eq. 2, third line); 0: Q stays unquantized
+    kv_bits: int = 8     # 8 or 4: width of the ordinary K/V rows (Table 1 lists 8 and 4)
+    p_bits: int = 8      # 8 or 4: width of the ordinary attention probabilities
     seed: int = 0
     name: str = ""
 

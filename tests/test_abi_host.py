@@ -77,8 +77,8 @@ def test_kv_layout(L):
     (dict(n_ctx=0), tb.TAQ_ERR_SHAPE),
     (dict(w_bits=5), tb.TAQ_ERR_INVALID_ARG),
     (dict(q_bits=4), tb.TAQ_ERR_INVALID_ARG),
-    (dict(kv_bits=4), tb.TAQ_ERR_UNSUPPORTED),
-    (dict(p_bits=4), tb.TAQ_ERR_UNSUPPORTED),
+    (dict(kv_bits=3), tb.TAQ_ERR_UNSUPPORTED),
+    (dict(p_bits=2), tb.TAQ_ERR_UNSUPPORTED),
     (dict(max_trigger=78), tb.TAQ_ERR_SHAPE),
     (dict(ctx_dim=100), tb.TAQ_ERR_SHAPE),
     (dict(channels=324, heads=81), tb.TAQ_ERR_SHAPE),  # head width 4
