@@ -9,7 +9,9 @@ namespace taq {
 
 namespace {
 
-// One CTA per (head, sequence).
+// One CTA per (head, sequence).  The head's codes and scales are staged in shared memory (coalesced 8-byte loads);
+// every thread then builds whole 16-byte chunks of the tiles: 8 channels of one key for K~, 8 keys of one channel for
+// V~^T (the transposition happens in shared memory).
 // `mask_a` (nullable, u8 [sequences][T]) overrides which probability columns stay fp16 (Eq. 3's M_A); by default they
 // are the columns of the fp16 K/V rows (M_A = M_KV).
 __global__ void __launch_bounds__(256) kv_operands_kernel(const taq_layer_desc d, uint8_t* kv, const taq_request* reqs, const uint8_t* mask_a) {
@@ -19,48 +21,80 @@ __global__ void __launch_bounds__(256) kv_operands_kernel(const taq_layer_desc d
     OperandGeom g;
     if (!operand_geom(D, T, &g)) return;
     uint8_t* blk = reqs ? (uint8_t*)reqs[z].kv : kv + (size_t)z * KL.block_bytes;
-    const int8_t* kc = (const int8_t*)(blk + KL.off_k_codes) + (size_t)h * T * D;
-    const int8_t* vc = (const int8_t*)(blk + KL.off_v_codes) + (size_t)h * T * D;
-    const float* ks = (const float*)(blk + KL.off_k_scales) + (size_t)h * T;
-    const float* vs = (const float*)(blk + KL.off_v_scales) + (size_t)h * T;
     const __half* kt = (const __half*)(blk + KL.off_k_trigger);
     const __half* vt = (const __half*)(blk + KL.off_v_trigger);
-    const int32_t* slot = (const int32_t*)(blk + KL.off_trig_slot);
     uint8_t* img = blk + KL.off_operands + (size_t)h * KL.operand_head_bytes;
     uint8_t* k_img = img;
     uint8_t* vt_img = img + g.k_bytes;
     OperandConsts* cst = reinterpret_cast<OperandConsts*>(img + g.k_bytes + g.vt_bytes);
     const size_t k_block = (size_t)kOperandKeys * 128, vt_block = (size_t)g.dp * 128;
 
-    // K~ tile: element (key j, channel c)
-    for (int idx = threadIdx.x; idx < kOperandKeys * g.kbq * 64; idx += blockDim.x) {
-        const int j = idx / (g.kbq * 64), c = idx % (g.kbq * 64);
-        __half v = __float2half_rn(0.f);
-        if (j < T && c < D) {
-            const int sl = slot[j];
-            v = sl >= 0 ? kt[((size_t)sl * H + h) * D + c] : __int2half_rn((int)kc[(size_t)j * D + c]);
+    __shared__ __align__(16) int8_t s_kc[kOperandKeys * kMaxHeadDim];
+    __shared__ __align__(16) int8_t s_vc[kOperandKeys * kMaxHeadDim];
+    __shared__ float s_ks[kOperandKeys], s_vs[kOperandKeys];
+    __shared__ int s_slot[kOperandKeys];
+    {
+        const uint2* kc8 = reinterpret_cast<const uint2*>(blk + KL.off_k_codes + (size_t)h * T * D);      // T * D is a multiple of 8
+        const uint2* vc8 = reinterpret_cast<const uint2*>(blk + KL.off_v_codes + (size_t)h * T * D);
+        for (int i = threadIdx.x; i < T * D / 8; i += blockDim.x) {
+            reinterpret_cast<uint2*>(s_kc)[i] = kc8[i];
+            reinterpret_cast<uint2*>(s_vc)[i] = vc8[i];
         }
-        *reinterpret_cast<__half*>(k_img + (c / 64) * k_block + ptx::sw128_offset(j, (c % 64) / 8) + (c % 8) * 2) = v;
+        const float* ks = (const float*)(blk + KL.off_k_scales) + (size_t)h * T;
+        const float* vs = (const float*)(blk + KL.off_v_scales) + (size_t)h * T;
+        const int32_t* slot = (const int32_t*)(blk + KL.off_trig_slot);
+        for (int j = threadIdx.x; j < kOperandKeys; j += blockDim.x) {
+            s_ks[j] = j < T ? ks[j] : 0.f;
+            s_vs[j] = j < T ? vs[j] : 0.f;
+            s_slot[j] = j < T ? slot[j] : -1;
+        }
     }
-    // V~^T tile: element (channel c, key j); ordinary rows are the fp16 operand of code * scale
-    for (int idx = threadIdx.x; idx < g.dp * 128; idx += blockDim.x) {
-        const int c = idx / 128, j = idx % 128;
-        __half v = __float2half_rn(0.f);
-        if (j < T && c < D) {
-            const int sl = slot[j];
-            v = sl >= 0 ? vt[((size_t)sl * H + h) * D + c] : __float2half_rn(__fmul_rn((float)vc[(size_t)j * D + c], vs[j]));
+    __syncthreads();
+
+    // K~ tile: chunk = 8 channels of key j
+    const int kch = g.kbq * 8;
+    for (int idx = threadIdx.x; idx < kOperandKeys * kch; idx += blockDim.x) {
+        const int j = idx / kch, cc = idx % kch, c0 = cc * 8;
+        uint4 out = make_uint4(0, 0, 0, 0);
+        if (j < T && c0 < D) {
+            const int sl = s_slot[j];
+            if (sl >= 0) {
+                out = *reinterpret_cast<const uint4*>(kt + ((size_t)sl * H + h) * D + c0);
+            } else {
+                __half2 hv[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    hv[e] = __halves2half2(__int2half_rn((int)s_kc[j * D + c0 + 2 * e]), __int2half_rn((int)s_kc[j * D + c0 + 2 * e + 1]));
+                out = *reinterpret_cast<uint4*>(hv);
+            }
         }
-        *reinterpret_cast<__half*>(vt_img + (j / 64) * vt_block + ptx::sw128_offset(c, (j % 64) / 8) + (j % 8) * 2) = v;
+        *reinterpret_cast<uint4*>(k_img + (cc / 8) * k_block + ptx::sw128_offset(j, cc % 8)) = out;
+    }
+    // V~^T tile: chunk = 8 keys of channel c; ordinary rows are the fp16 operand of code * scale
+    for (int idx = threadIdx.x; idx < g.dp * 16; idx += blockDim.x) {
+        const int c = idx / 16, jc = idx % 16;
+        __half hv[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const int j = jc * 8 + e;
+            __half v = __float2half_rn(0.f);
+            if (j < T && c < D) {
+                const int sl = s_slot[j];
+                v = sl >= 0 ? vt[((size_t)sl * H + h) * D + c] : __float2half_rn(__fmul_rn((float)s_vc[j * D + c], s_vs[j]));
+            }
+            hv[e] = v;
+        }
+        *reinterpret_cast<uint4*>(vt_img + (jc / 8) * vt_block + ptx::sw128_offset(c, jc % 8)) = *reinterpret_cast<uint4*>(hv);
     }
     // constants
     const float logit_unit = 1.4426950408889634f / sqrtf((float)D);
     for (int j = threadIdx.x; j < kOperandKeys; j += blockDim.x)
-        cst->logit_factor[j] = j < T ? (slot[j] >= 0 ? 1.0f : ks[j]) * logit_unit : 0.f;
+        cst->logit_factor[j] = j < T ? (s_slot[j] >= 0 ? 1.0f : s_ks[j]) * logit_unit : 0.f;
     if (threadIdx.x < 4) {
         uint32_t bits = 0;
         for (int i = 0; i < 32; ++i) {
             const int j = threadIdx.x * 32 + i;
-            if (j < T && (mask_a ? mask_a[(size_t)z * T + j] != 0 : slot[j] >= 0)) bits |= 1u << i;
+            if (j < T && (mask_a ? mask_a[(size_t)z * T + j] != 0 : s_slot[j] >= 0)) bits |= 1u << i;
         }
         cst->trig_bits[threadIdx.x] = bits;
     }
