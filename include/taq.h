@@ -254,6 +254,31 @@ taq_status taq_token_sensitivity(const taq_layer_desc* desc, const void* x_f16_d
 taq_status taq_kv_set_prob_mask(const taq_layer_desc* desc, void* kv_packed_dev, size_t kv_bytes,
                                 const uint8_t* mask_a_dev, void* stream);
 
+/* --------------------------------------------------------------------------------------------------------
+ * K~/V~ cache for serving (Sec. I: many personalized checkpoints served concurrently; Sec. III-B: the keys and
+ * values come from the text alone).  K~/V~ of a (checkpoint, prompt) pair are the same at every denoising step
+ * and for every request with that pair - the unconditional prompt of classifier-free guidance is one shared
+ * entry per checkpoint - so admission projects them once (taq_kv_project_batched) into an entry of this cache.
+ * Host-side bookkeeping only: the cache hands out fixed-size entries of a caller-owned device arena (entry_bytes:
+ * e.g. the K~/V~ blocks of all layers for one prompt; a multiple of 128, arena 128-byte aligned), never touches
+ * the device and is safe to call from several host threads.  Entries in use by requests in flight are pinned;
+ * a miss takes a free entry or evicts the least recently used unpinned one.
+ * -------------------------------------------------------------------------------------------------------- */
+typedef struct taq_kv_cache taq_kv_cache;
+typedef struct { int64_t capacity, used, hits, misses, evictions; } taq_kv_cache_stats;
+
+/* 64-bit FNV-1a over the token ids (little-endian bytes): the prompt part of a cache key. */
+uint64_t taq_hash_prompt(const int32_t* token_ids, int32_t n_tokens);
+taq_kv_cache* taq_kv_cache_create(void* arena_dev, size_t arena_bytes, size_t entry_bytes);   /* NULL on bad arguments */
+void taq_kv_cache_destroy(taq_kv_cache* cache);
+/* *hit = 1: *entry_dev holds the pair's K~/V~.  *hit = 0: *entry_dev is the entry to fill before use.  Either way
+ * the entry is pinned until taq_kv_cache_release.  TAQ_ERR_BUFFER_TOO_SMALL when every entry is pinned. */
+taq_status taq_kv_cache_acquire(taq_kv_cache* cache, uint64_t checkpoint, uint64_t prompt, void** entry_dev, int32_t* hit);
+taq_status taq_kv_cache_release(taq_kv_cache* cache, uint64_t checkpoint, uint64_t prompt);
+/* Forgets every entry of a checkpoint (e.g. when it is unloaded); refused while one of them is pinned. */
+taq_status taq_kv_cache_drop_checkpoint(taq_kv_cache* cache, uint64_t checkpoint);
+taq_status taq_kv_cache_get_stats(taq_kv_cache* cache, taq_kv_cache_stats* out);
+
 /* Batched serving (Sec. I: many personalized checkpoints served concurrently): request r is one sequence
  * (desc->batch must be 1) whose activations are slice r of x/y [n_requests][N][C] and which carries its own
  * checkpoint's packed weights, its own K~/V~ block and its own trigger mask.  `reqs_dev` is a DEVICE array of

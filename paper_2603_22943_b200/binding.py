@@ -27,7 +27,8 @@ EXPORTS = [
     "taq_static_workspace_capacity", "taq_layer_forward_static", "taq_kv_finalize", "taq_query_attention",
     "taq_quantize_rows_f16", "taq_quantized_linear_i8", "taq_workspace_bytes_a8", "taq_layer_forward_a8",
     "taq_kv_project_a8_workspace_bytes", "taq_kv_project_a8", "taq_token_sensitivity_workspace_bytes",
-    "taq_token_sensitivity", "taq_kv_set_prob_mask",
+    "taq_token_sensitivity", "taq_kv_set_prob_mask", "taq_hash_prompt", "taq_kv_cache_create", "taq_kv_cache_destroy",
+    "taq_kv_cache_acquire", "taq_kv_cache_release", "taq_kv_cache_drop_checkpoint", "taq_kv_cache_get_stats",
 ]
 
 
@@ -48,6 +49,10 @@ class LayerDesc(C.Structure):
     @property
     def d_head(self) -> int:
         return self.channels // self.heads
+
+
+class KvCacheStats(C.Structure):
+    _fields_ = [(n, C.c_int64) for n in ("capacity", "used", "hits", "misses", "evictions")]
 
 
 class KvLayout(C.Structure):
@@ -111,6 +116,17 @@ def lib() -> C.CDLL:
         L.taq_token_sensitivity_workspace_bytes.argtypes = [C.POINTER(LayerDesc)]
         L.taq_token_sensitivity.argtypes = [C.POINTER(LayerDesc), vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.taq_kv_set_prob_mask.argtypes = [C.POINTER(LayerDesc), vp, sz, vp, vp]
+        u64 = C.c_uint64
+        L.taq_hash_prompt.restype = u64
+        L.taq_hash_prompt.argtypes = [C.POINTER(i32), i32]
+        L.taq_kv_cache_create.restype = vp
+        L.taq_kv_cache_create.argtypes = [vp, sz, sz]
+        L.taq_kv_cache_destroy.restype = None
+        L.taq_kv_cache_destroy.argtypes = [vp]
+        L.taq_kv_cache_acquire.argtypes = [vp, u64, u64, C.POINTER(vp), C.POINTER(i32)]
+        L.taq_kv_cache_release.argtypes = [vp, u64, u64]
+        L.taq_kv_cache_drop_checkpoint.argtypes = [vp, u64]
+        L.taq_kv_cache_get_stats.argtypes = [vp, C.POINTER(KvCacheStats)]
         for name in EXPORTS:
             f = getattr(L, name)
             if f.restype is C.c_int and name not in ("taq_version",):
@@ -277,6 +293,52 @@ def taq_kv_project_a8(desc: LayerDesc, ctx: torch.Tensor, Wk_packed: torch.Tenso
     _check(lib().taq_kv_project_a8(C.byref(desc), _ptr(ctx), _ptr(Wk_packed), _ptr(Wv_packed), _ptr(trig_mask), _ptr(kv), kv.numel(),
                                    _ptr(workspace), workspace.numel(), _stream(stream)))
     return kv
+
+
+def taq_hash_prompt(token_ids) -> int:
+    ids = (C.c_int32 * len(token_ids))(*[int(t) for t in token_ids])
+    return int(lib().taq_hash_prompt(ids, len(token_ids)))
+
+
+class KvCache:
+    """Host-side K~/V~ cache over a device arena (address + size; the cache never touches the memory)."""
+
+    def __init__(self, arena_ptr: int, arena_bytes: int, entry_bytes: int):
+        self._h = lib().taq_kv_cache_create(arena_ptr, arena_bytes, entry_bytes)
+        if not self._h:
+            raise ValueError("taq_kv_cache_create refused its arguments (arena and entry size must be 128-byte aligned, at least one entry)")
+        self.arena_ptr, self.entry_bytes = arena_ptr, entry_bytes
+
+    def acquire(self, checkpoint: int, prompt: int):
+        """Returns (entry address, hit)."""
+        p, hit = C.c_void_p(), C.c_int32()
+        st = lib().taq_kv_cache_acquire(self._h, checkpoint, prompt, C.byref(p), C.byref(hit))
+        if st != TAQ_OK:
+            raise TaqError(st, "every cache entry is pinned" if st == TAQ_ERR_BUFFER_TOO_SMALL else "kv cache acquire")
+        return int(p.value), bool(hit.value)
+
+    def release(self, checkpoint: int, prompt: int) -> None:
+        st = lib().taq_kv_cache_release(self._h, checkpoint, prompt)
+        if st != TAQ_OK:
+            raise TaqError(st, "release of an entry that is not pinned")
+
+    def drop_checkpoint(self, checkpoint: int) -> None:
+        st = lib().taq_kv_cache_drop_checkpoint(self._h, checkpoint)
+        if st != TAQ_OK:
+            raise TaqError(st, "checkpoint still has pinned entries")
+
+    def stats(self) -> dict:
+        s = KvCacheStats()
+        lib().taq_kv_cache_get_stats(self._h, C.byref(s))
+        return {n: getattr(s, n) for n, _ in KvCacheStats._fields_}
+
+    def close(self) -> None:
+        if self._h:
+            lib().taq_kv_cache_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        self.close()
 
 
 def taq_kv_set_prob_mask(desc: LayerDesc, kv: torch.Tensor, mask_a: torch.Tensor, stream=None) -> torch.Tensor:
