@@ -150,6 +150,130 @@ def run_reference(args, shape, data):
     print(json.dumps(line), flush=True)
 
 
+def _graph_time(torch, fn, count, replays):
+    """Captures `count` calls of fn(i) into one CUDA graph and returns the milliseconds of one replay (device time)."""
+    for i in range(min(count, 8)):
+        fn(i)
+    torch.cuda.synchronize()
+    st = torch.cuda.Stream()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=st):
+        for i in range(count):
+            fn(i)
+    g.replay()
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(replays):
+        g.replay()
+    b.record()
+    torch.cuda.synchronize()
+    return a.elapsed_time(b) / replays
+
+
+def run_other_workload(args):
+    """The other measured configurations (not the headline line): `config3`, one SD-1.5 UNet step of all 16
+    cross-attention layers; `config5`, the multi-checkpoint serving sweep on the 64x64 layer.  One GPU."""
+    import torch
+    from paper_2603_22943_b200 import binding as tb
+    from paper_2603_22943_b200 import synth
+    torch.cuda.set_device(0)
+    tb.lib()
+    peaks = _peaks()
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    sampler = ClockSampler(0)
+    sampler.start()
+    if args.workload == "config3":
+        layers = synth.config3_layers()
+        n_sets = 3                                    # 3 x 108 MB of activations per step > 2 x L2
+        sets = []
+        for k in range(n_sets):
+            L = []
+            for shp in layers:
+                data = synth.make_layer(shp)
+                desc = tb.layer_desc(shp.batch, shp.n_query, shp.channels, shp.heads, shp.n_ctx, shp.ctx_dim, shp.w_bits, shp.w_group,
+                                     q_bits=shp.q_bits, max_trigger=len(shp.trigger))
+                wd_cc = tb.weight_desc(shp.channels, shp.channels, shp.w_bits, shp.w_group)
+                wd_cd = tb.weight_desc(shp.channels, shp.ctx_dim, shp.w_bits, shp.w_group)
+                mask = dev(data["mask"])
+                kv = tb.taq_kv_project(desc, dev(data["ctx"]), tb.taq_pack_weights(wd_cd, dev(data["Wk"])), tb.taq_pack_weights(wd_cd, dev(data["Wv"])), mask)
+                L.append((desc, dev(np.roll(data["X"], k, axis=1)), tb.taq_pack_weights(wd_cc, dev(data["Wq"])),
+                          tb.taq_pack_weights(wd_cc, dev(data["Wout"]), dev(data["bout"])), kv, mask,
+                          torch.empty((shp.batch, shp.n_query, shp.channels), dtype=torch.float16, device="cuda"),
+                          torch.empty(tb.taq_workspace_bytes(desc, 1), dtype=torch.uint8, device="cuda")))
+            sets.append(L)
+        tb.taq_poll_device_status()
+
+        def step(i):
+            for (desc, x, Wq, Wo, kv, mask, y, ws) in sets[i % n_sets]:
+                tb.taq_layer_forward(desc, x, Wq, Wo, kv, mask, y, ws)
+
+        steps = max(6, min(args.steps, 60))
+        ms = _graph_time(torch, step, steps, 3) / steps
+        rows = sum(l.batch * l.n_query for l in layers)
+        flops = sum(4 * l.batch * l.n_query * l.channels * l.channels + 4 * l.batch * l.n_query * l.n_ctx * l.channels for l in layers)
+        nbytes = sum(2 * l.batch * l.n_query * l.channels * 2 for l in layers)
+        tb.taq_poll_device_status()
+        line = {"metric": "TAQ cross-attn queries/s over one SD-1.5 UNet step (16 layers)", "value": rows / (ms * 1e-3), "unit": UNIT, "n_gpus": 1,
+                "steps": steps, "warmup": 8, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f16",
+                "data": "synthetic",
+                "config": {"workload": "config3: all 16 SD-1.5 cross-attn layers (5x(N=4096,C=320), 5x(1024,640), 5x(256,1280), 1x(64,1280)), B=2, T=77, W4 g128, trigger {4,5}",
+                           "launch": "one CUDA graph of the steps; C=320 layers: one kernel each, other layers: three kernels each",
+                           "l2_policy": f"ring of {n_sets} buffer sets ({n_sets * nbytes / 1e6:.0f} MB of activations)"},
+                "clocks": sampler.stop(), "gpu_launches": steps * (5 + 11 * 3),
+                "roofline": {"bound": "tensor", "achieved": flops / (ms * 1e-3) / 1e12, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                             "frac": flops / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"], "traffic": None,
+                             "hbm": {"achieved_GBps": nbytes / (ms * 1e-3) / 1e9, "peak_GBps": peaks["hbm_gbs"]}}}
+        print(json.dumps(line), flush=True)
+        return
+    # config5: 64 checkpoints resident, requests routed to random checkpoints, the N=4096 x C=320 layer
+    n_ckpt, N, C_, H, T, Dc = 64, 4096, 320, 8, 77, 768
+    wd_cc, wd_cd = tb.weight_desc(C_, C_, 4, 128), tb.weight_desc(C_, Dc, 4, 128)
+    desc1 = tb.layer_desc(1, N, C_, H, T, Dc, 4, 128, q_bits=8, max_trigger=3)
+    ck = []
+    for c in range(n_ckpt):
+        cp = synth.make_checkpoint(c, C_, Dc, T)
+        w = cp.weights
+        ck.append((cp, tb.taq_pack_weights(wd_cc, dev(w["Wq"])), tb.taq_pack_weights(wd_cc, dev(w["Wout"]), dev(w["bout"])),
+                   tb.taq_pack_weights(wd_cd, dev(w["Wk"])), tb.taq_pack_weights(wd_cd, dev(w["Wv"]))))
+    n_slots = 64
+    route = synth.make_request_batch(n_slots, n_ckpt, 0)
+    slot = []
+    for r in range(n_slots):
+        cp, Wq, Wo, Wk, Wv = ck[int(route[r])]
+        act = synth.make_request_activations(cp, N, C_, Dc, T, r)
+        mask = dev(act["mask"])
+        kv = tb.taq_kv_project(desc1, dev(act["ctx"]), Wk, Wv, mask)
+        slot.append((Wq, Wo, kv, mask, act["X"]))
+    x_all = dev(np.concatenate([s_[4] for s_ in slot], axis=0))              # [64][N][C]
+    y_all = torch.empty_like(x_all)
+    per_ckpt_all_layers = sum(2 * tb.taq_packed_weight_bytes(tb.weight_desc(l.channels, l.channels, 4, 128)) +
+                              2 * tb.taq_packed_weight_bytes(tb.weight_desc(l.channels, l.ctx_dim, 4, 128)) for l in synth.config3_layers())
+    results = []
+    for nb in (1, 8, 32, 64):
+        groups = n_slots // nb
+        tables = [tb.make_request_table([slot[g * nb + j][:4] for j in range(nb)], "cuda") for g in range(groups)]
+        ws = torch.empty(tb.taq_workspace_bytes(desc1, nb), dtype=torch.uint8, device="cuda")
+
+        def step(i, nb=nb, groups=groups, tables=tables, ws=ws):
+            g = i % groups
+            tb.taq_layer_forward_batched(desc1, tables[g], nb, x_all[g * nb:(g + 1) * nb], y_all[g * nb:(g + 1) * nb], ws)
+
+        count = max(groups, 16)
+        ms = _graph_time(torch, step, count, 5) / count
+        results.append({"requests_per_batch": nb, "ms_per_batch": round(ms, 5), "requests_per_s": nb / (ms * 1e-3), "queries_per_s": nb * N / (ms * 1e-3)})
+    tb.taq_poll_device_status()
+    best = results[-1]
+    line = {"metric": "TAQ multi-checkpoint serving, requests/s on the N=4096 x C=320 layer", "value": best["requests_per_s"], "unit": "requests/s", "n_gpus": 1,
+            "steps": 16, "warmup": 8, "ms_per_step": best["ms_per_batch"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f16",
+            "data": "synthetic",
+            "config": {"workload": "config5: 64 synthetic checkpoints resident (packed W4 g128), each request routed to a random checkpoint with its own weights, K~/V~ and trigger span (1-3 tokens)",
+                       "launch": "one kernel per batch (grid.z = request), batches rotate over 64 resident request slots (168 MB of activations)",
+                       "packed_bytes_per_checkpoint_all_16_layers": per_ckpt_all_layers, "fp16_bytes_per_checkpoint_all_16_layers": int(per_ckpt_all_layers / 4.25 * 16)},
+            "sweep": results, "clocks": sampler.stop(), "gpu_launches": 16}
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -161,7 +285,12 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=10.0, help="CPU time to spend on the cpu_baseline sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--n-query", type=int, default=0, help="override N (profiling on a smaller case)")
+    ap.add_argument("--workload", default="config2", choices=["config2", "config3", "config5"],
+                    help="config2 (default) is the headline line; config3 / config5 print the other measured configurations")
     args = ap.parse_args()
+    if args.workload != "config2":
+        run_other_workload(args)
+        return
     if args.warmup < 3 and args.impl == "taq":
         args.warmup = 3
 
@@ -323,20 +452,41 @@ def main():
     yh = [torch.empty((B, N, C_), dtype=torch.float16).pin_memory() for _ in range(4)]
     e_steps = max(10, min(args.steps, 100))
 
+    # Three streams: the upload of step i + 1 and the download of step i - 1 run under the kernel of step i (PCIe is full
+    # duplex), every copy is inside the timed region, and a buffer set is reused only after its previous user is done.
+    s_in, s_cmp, s_out = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
+    ev_in, ev_cmp, ev_out = {}, {}, {}
+
     def e2e_step(i):
         s = sets[i % n_sets]
-        s["x"].copy_(xh[i % 4], non_blocking=True)
-        tb.taq_layer_forward(desc, s["x"], s["Wq"], s["Wout"], s["kv"], mask, s["y"], s["ws"])
-        yh[i % 4].copy_(s["y"], non_blocking=True)
+        with torch.cuda.stream(s_in):
+            if i - n_sets in ev_cmp:
+                s_in.wait_event(ev_cmp[i - n_sets])          # the set's X is no longer being read
+            s["x"].copy_(xh[i % 4], non_blocking=True)
+            ev_in[i] = torch.cuda.Event()
+            ev_in[i].record(s_in)
+        with torch.cuda.stream(s_cmp):
+            s_cmp.wait_event(ev_in[i])
+            if i - n_sets in ev_out:
+                s_cmp.wait_event(ev_out[i - n_sets])         # the set's Y has been downloaded
+            tb.taq_layer_forward(desc, s["x"], s["Wq"], s["Wout"], s["kv"], mask, s["y"], s["ws"])
+            ev_cmp[i] = torch.cuda.Event()
+            ev_cmp[i].record(s_cmp)
+        with torch.cuda.stream(s_out):
+            s_out.wait_event(ev_cmp[i])
+            yh[i % 4].copy_(s["y"], non_blocking=True)
+            ev_out[i] = torch.cuda.Event()
+            ev_out[i].record(s_out)
 
     for i in range(3):
         e2e_step(i)
     barrier()
+    ev_in.clear(); ev_cmp.clear(); ev_out.clear()
     f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    f0.record()
+    f0.record(s_in)
     for i in range(e_steps):
         e2e_step(i)
-    f1.record()
+    f1.record(s_out)
     barrier()
     e2e_ms = f0.elapsed_time(f1)
     tb.taq_poll_device_status()
