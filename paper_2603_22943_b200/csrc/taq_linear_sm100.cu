@@ -177,6 +177,7 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
             for (bool first = true; kb < kb_end && ok; ++kb) {
                 if (!wait(&bars->full_a[s], ph) || (!a.w_direct && !wait(&bars->full_b[s], ph))) { ok = false; break; }
                 if (leader) {
+                    if (kb < 20) TAQ_PROF(40 + kb);
                     const uint32_t a_lo = lo0 + s * (TL::STAGE_BYTES >> 4), b_lo = a_lo + (A_TILE_BYTES >> 4);
 #pragma unroll
                     for (int k = 0; k < 4; ++k) {            // four 32-byte K slices per 128-byte operand row
@@ -212,6 +213,7 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
         float* xchg = reinterpret_cast<float*>(smem + P.off_xchg);
         const int row_bytes = (int)L.row_bytes;
         bool ok = ptx::mbar_wait(&bars->w_full, 0);
+        if (wt == 0) TAQ_PROF(2);
         if (!ok) { raise_status(a.status, TAQ_ERR_TIMEOUT); bars->abort_flag = 1; }
         // scales [BN][n_groups] -> [n_groups][BN], so that a group's scales of consecutive columns are contiguous
         for (int i = wt; i < BN * n_groups; i += NWORK) scales_t[(i % n_groups) * BN + i / n_groups] = wscales[i];
@@ -313,6 +315,7 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
                 ptx::fence_proxy_async_smem();            // make the generic-proxy writes visible to the tensor core
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(&bars->full_b[s]);
+                if (wt == 0 && kb < 20) TAQ_PROF(60 + kb);
                 if (++s == nstage) { s = 0; ph ^= 1; }
             }
             return true;
@@ -461,6 +464,7 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
     }
 
     // ---------------- teardown ----------------
+    if (tid == 64) TAQ_PROF(8);
     ptx::tc_fence_before_sync();
     __syncthreads();
     if (tid == 0) { TAQ_PROF(9); TAQ_GPROF(29); }
