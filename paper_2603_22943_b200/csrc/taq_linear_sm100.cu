@@ -44,8 +44,6 @@ struct Tile {
     static constexpr int STAGE_BYTES = A_TILE_BYTES + B_TILE_BYTES;
     static constexpr uint32_t TMEM_COLS = 2 * BN <= 128 ? 128 : 2 * BN <= 256 ? 256 : 512;
     static constexpr int CTAS_PER_SM = TMEM_COLS <= 256 ? 2 : 1;
-    static constexpr int NACC = TMEM_COLS / BN;                               // accumulators (one scale group each) in flight
-    static_assert(NACC >= 2 && NACC <= 4, "accumulator ring");
     static_assert(HC % 8 == 0, "a worker's columns come in groups of 8");
 };
 
@@ -54,8 +52,8 @@ struct Bars {
     uint64_t full_b[MAX_STAGE];
     uint64_t empty[MAX_STAGE];
     uint64_t w_full;
-    uint64_t acc_full[4];
-    uint64_t acc_free[4];
+    uint64_t acc_full[2];
+    uint64_t acc_free[2];
     uint32_t tmem_base;
     volatile int abort_flag;
 };
@@ -116,7 +114,7 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
             ptx::mbar_init(&bars->empty[s], 1);
         }
         ptx::mbar_init(&bars->w_full, 1);
-        for (int i = 0; i < 4; ++i) {
+        for (int i = 0; i < 2; ++i) {
             ptx::mbar_init(&bars->acc_full[i], 1);
             ptx::mbar_init(&bars->acc_free[i], NWORK / 32);
         }
@@ -170,9 +168,9 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
         uint32_t ph = 0;
         bool ok = true;
         for (int g = 0; g < n_groups && ok; ++g) {
-            const int buf = g % TL::NACC;
-            if (g >= TL::NACC) {                            // the workers have emptied this accumulator
-                if (!wait(&bars->acc_free[buf], ((g / TL::NACC) - 1) & 1)) { ok = false; break; }
+            const int buf = g & 1;
+            if (g >= 2) {                                   // the workers have emptied this accumulator
+                if (!wait(&bars->acc_free[buf], ((g >> 1) - 1) & 1)) { ok = false; break; }
                 ptx::tc_fence_after_sync();
             }
             const int kb_end = min(n_kb, kb + kb_per_group);
@@ -196,7 +194,8 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
         if (!ok && leader) {
             raise_status(a.status, TAQ_ERR_TIMEOUT);
             bars->abort_flag = 1;
-            for (int i = 0; i < TL::NACC; ++i) ptx::mma_commit(&bars->acc_full[i]);        // wake the workers; they see the abort flag
+            ptx::mma_commit(&bars->acc_full[0]);        // wake the workers; they see the abort flag
+            ptx::mma_commit(&bars->acc_full[1]);
         }
     } else {
         // ---------------- workers (warps 2..9) ----------------
@@ -226,8 +225,8 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
 
         // y += scale[g] * accumulator of group g (this thread's HC columns of its row)
         auto fold_group = [&](int g) -> bool {
-            const int buf = g % TL::NACC;
-            if (!ptx::mbar_wait(&bars->acc_full[buf], (g / TL::NACC) & 1) || bars->abort_flag) return false;
+            const int buf = g & 1;
+            if (!ptx::mbar_wait(&bars->acc_full[buf], (g >> 1) & 1) || bars->abort_flag) return false;
             ptx::tc_fence_after_sync();
             const float* sg = scales_t + g * BN + cb;
 #pragma unroll
@@ -263,8 +262,11 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
         // expand the weight tiles of group g's k-blocks
         int s = 0, kb = 0;
         uint32_t ph = 0;
-        auto build_tile = [&]() -> bool {                    // tile kb into stage s (the caller has seen the stage free)
-            {
+        auto build_group = [&](int g) -> bool {
+            const int kb_end = min(n_kb, kb + kb_per_group);
+            for (; kb < kb_end; ++kb) {
+                if (kb >= nstage && !ptx::mbar_wait(&bars->empty[s], ph ^ 1)) return false;
+                if (bars->abort_flag) return false;
                 unsigned char* b_tile = smem + s * TL::STAGE_BYTES + A_TILE_BYTES;
                 // 16-byte chunks of the fp16 tile: 8 per weight row; this thread owns chunk c of rows n0, n0 + 32, ...
                 constexpr int NCH = (BN * 8 + NWORK - 1) / NWORK;
@@ -315,39 +317,15 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
                 if (lane == 0) ptx::mbar_arrive(&bars->full_b[s]);
                 if (wt == 0 && kb < 20) TAQ_PROF(60 + kb);
                 if (++s == nstage) { s = 0; ph ^= 1; }
-                ++kb;
             }
             return true;
         };
 
-        // Each warp expands the next tile whenever its ring stage is free and folds the next scale group whenever its
-        // accumulator is complete, whichever comes first (the decision is taken by the whole warp); it never blocks on
-        // one of the two alone, because the tensor core waits for both: tiles to multiply and accumulators to reuse.
-        {
-            const int n_build = a.w_direct ? 0 : n_kb;
-            if (a.w_direct) kb = n_kb;
-            int gf = 0;
-            long long idle_since = 0;
-            while (ok && (kb < n_build || gf < n_groups)) {
-                if (__any_sync(0xffffffffu, bars->abort_flag != 0)) { ok = false; break; }      // (one decision per warp)
-                const bool can_build = kb < n_build && (kb < nstage || __all_sync(0xffffffffu, ptx::mbar_try_wait(&bars->empty[s], ph ^ 1)));
-                if (can_build) {
-                    ok = build_tile();
-                    idle_since = 0;
-                    continue;
-                }
-                const bool can_fold = gf < n_groups && __all_sync(0xffffffffu, ptx::mbar_try_wait(&bars->acc_full[gf % TL::NACC], (gf / TL::NACC) & 1));
-                if (can_fold) {
-                    ok = fold_group(gf);
-                    ++gf;
-                    idle_since = 0;
-                    continue;
-                }
-                const long long now = clock64();
-                if (idle_since == 0) idle_since = now;
-                else if (__any_sync(0xffffffffu, now - idle_since > (1LL << 31))) { ok = false; break; }
-            }
+        for (int g = 0; g < n_groups && ok; ++g) {
+            ok = a.w_direct ? true : build_group(g);
+            if (ok && g >= 1) ok = fold_group(g - 1);
         }
+        if (ok) ok = fold_group(n_groups - 1);
         if (!ok) { raise_status(a.status, TAQ_ERR_TIMEOUT); bars->abort_flag = 1; }
         asm volatile("bar.sync 1, 256;" ::: "memory");       // every worker gets here; the decision below is uniform
         ok = !bars->abort_flag;
