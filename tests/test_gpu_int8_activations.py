@@ -115,3 +115,48 @@ def test_layer_forward_a8_matches_the_oracle(shape):
     # the integer path is a different quantized network from the fp16-activation one, not a copy of it
     y16 = tl.gpu_layer(shape, data)
     assert tl.errors(y, y16)[1] > 1e-3, res
+
+
+def test_a8_pass_is_deterministic_and_stays_inside_its_buffers():
+    shape = replace(synth.shrink(synth.config2(), 333), seed=25)          # 2.6 row tiles per sequence
+    data = synth.make_layer(shape)
+    desc = tl.gpu_desc(shape)
+    P = tl.pack_layer_weights(shape, data)
+    mask = dev(data["mask"])
+    guard = 1024
+    kvn = tb.taq_kv_bytes(desc)
+    kvbuf = torch.full((kvn + 2 * guard,), 0x5A, dtype=torch.uint8, device="cuda")
+    wkn = tb.lib().taq_kv_project_a8_workspace_bytes(tb.C.byref(desc))
+    wkbuf = torch.full((wkn + 2 * guard,), 0x5A, dtype=torch.uint8, device="cuda")
+    tb.taq_kv_project_a8(desc, dev(data["ctx"]), P["Wk"], P["Wv"], mask, kvbuf[guard: guard + kvn], wkbuf[guard: guard + wkn])
+    n = shape.rows * shape.channels
+    ybuf = torch.full((n + 2 * guard,), -7.0, dtype=torch.float16, device="cuda")
+    wsn = tb.taq_workspace_bytes_a8(desc)
+    wsbuf = torch.full((wsn + 2 * guard,), 0x5A, dtype=torch.uint8, device="cuda")
+    x = dev(data["X"])
+    outs = []
+    for _ in range(2):
+        tb.taq_layer_forward_a8(desc, x, P["Wq"], P["Wout"], kvbuf[guard: guard + kvn], mask, ybuf[guard: guard + n], wsbuf[guard: guard + wsn])
+        torch.cuda.synchronize()
+        outs.append(ybuf.cpu().numpy().copy())
+    assert np.array_equal(outs[0].view(np.uint16), outs[1].view(np.uint16))
+    assert np.all(outs[0][:guard] == -7.0) and np.all(outs[0][-guard:] == -7.0)
+    for buf in (kvbuf, wkbuf, wsbuf):
+        b = buf.cpu().numpy()
+        assert np.all(b[:guard] == 0x5A) and np.all(b[-guard:] == 0x5A)
+    tb.taq_poll_device_status()
+
+
+def test_a8_empty_inputs_and_bad_arguments():
+    shape = synth.shrink(synth.config2(), 64)
+    desc0 = tl.gpu_desc(shape, n_query=0)
+    z = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    assert tb.taq_layer_forward_a8(desc0, z, z, z, z, z, y=z, workspace=z) is z          # nothing to do, nothing launched
+    desc = tl.gpu_desc(shape)
+    with pytest.raises(tb.TaqError) as e:                                                 # workspace too small
+        tb.taq_layer_forward_a8(desc, z, z, z, z, z, y=z, workspace=z)
+    assert e.value.status == tb.TAQ_ERR_BUFFER_TOO_SMALL
+    with pytest.raises(tb.TaqError) as e:                                                 # columns not a multiple of 8
+        tb.lib().taq_quantize_rows_f16.restype = tb.C.c_int
+        tb._check(tb.lib().taq_quantize_rows_f16(z.data_ptr(), 4, 12, z.data_ptr(), z.data_ptr(), None))
+    assert e.value.status == tb.TAQ_ERR_SHAPE
