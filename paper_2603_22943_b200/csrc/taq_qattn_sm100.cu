@@ -64,7 +64,7 @@ static_assert(OFF_P + 4 * A_TILE <= OFF_RAW, "phase-3 tiles must fit into the ph
 struct Misc {
     uint64_t a_full[NKB], b_full[NBSTAGE], b_empty[NBSTAGE], w_full, acc_full[MAX_GROUPS];
     uint64_t w2_full, s_done, pv_done, peer_ready, peer_got, o_all, piece_done[3];      // layer variant (phase 4)
-    uint64_t q_all, k_full[2], k_free[2], vt_full[2], vt_free[2], c_full, s_full[2], s_free[2], p_full[2], o_full[2], drain;
+    uint64_t q_all, k_full[2], vt_full[2], c_full, s_full[2], s_free[2], p_full[2], o_full[2], drain;
     uint32_t tmem_base;
     volatile int abort_flag;
     float sq[HG][ROWS];              // Q~ row scales
@@ -107,10 +107,11 @@ __device__ __forceinline__ uint32_t o_tiles_touched(int h, int half) {
     return m;
 }
 // Pieces of a CTA's five tiles: the first leaves after the first head of each group (80 channels cover two tiles and a
-// half), the rest after the second; tiles 7 and 8 are not adjacent in shared memory.
+// half), the next when group 0 has stored its second head, the last when group 1 has; tiles 7 and 8 are not adjacent in
+// shared memory.
 constexpr int MAX_PIECES = 3;
 __device__ __forceinline__ int o_pieces(int h_begin, int (&first)[MAX_PIECES], int (&count)[MAX_PIECES]) {
-    if (h_begin == 0) { first[0] = 0; count[0] = 2; first[1] = 2; count[1] = 3; first[2] = 0; count[2] = 0; return 2; }
+    if (h_begin == 0) { first[0] = 0; count[0] = 2; first[1] = 2; count[1] = 1; first[2] = 3; count[2] = 2; return 3; }
     first[0] = 5; count[0] = 2; first[1] = 7; count[1] = 1; first[2] = 8; count[2] = 2;
     return 3;
 }
@@ -172,9 +173,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
         for (int i = 0; i < MAX_GROUPS; ++i) ptx::mbar_init(&misc->acc_full[i], 1);
         for (int i = 0; i < 2; ++i) {
             ptx::mbar_init(&misc->k_full[i], 1);
-            ptx::mbar_init(&misc->k_free[i], 1);
             ptx::mbar_init(&misc->vt_full[i], 1);
-            ptx::mbar_init(&misc->vt_free[i], 1);
             ptx::mbar_init(&misc->s_full[i], 1);
             ptx::mbar_init(&misc->s_free[i], NWORK / 64);     // one arrival per warp of the group
             ptx::mbar_init(&misc->p_full[i], NWORK / 64);
@@ -263,12 +262,12 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
                 }
             }
             for (int g = 0; g < 2 && !misc->abort_flag; ++g) {
-                if (!ptx::mbar_wait(&misc->k_free[g], 0)) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; break; }
+                if (!ptx::mbar_wait(&misc->s_full[g], 0)) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; break; }
                 load_k(2 + g);
                 ++k_issued;
             }
             for (int g = 0; g < 2 && !misc->abort_flag; ++g) {
-                if (!ptx::mbar_wait(&misc->vt_free[g], 0)) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; break; }
+                if (!ptx::mbar_wait(&misc->o_full[g], 0)) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; break; }
                 load_vt(2 + g);
                 ++vt_issued;
             }
@@ -347,8 +346,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
 #pragma unroll
                 for (int ks = 0; ks < DP / 16; ++ks)
                     ptx::mma_f16_ss(tmem_base + TMEM_S + g * TP, ptx::desc_join(HI128, qh_lo + 2 * ks), ptx::desc_join(HI128, kg_lo + 2 * ks), ptx::idesc_f16_m128(TP), ks != 0);
-                ptx::mma_commit(&misc->s_full[g]);
-                ptx::mma_commit(&misc->k_free[g]);
+                ptx::mma_commit(&misc->s_full[g]);       // (also tells the producer that the group's K~ buffer is free)
             }
             return true;
         };
@@ -361,8 +359,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
                 for (int ks = 0; ks < TP / 16; ++ks)
                     ptx::mma_f16_ss(tmem_base + TMEM_O + g * DP, ptx::desc_join(HI128, pg_lo + (ks / 4) * (A_TILE >> 4) + (ks % 4) * 2),
                                     ptx::desc_join(HI128, vg_lo + (ks / 4) * (VT_BLOCK >> 4) + (ks % 4) * 2), ptx::idesc_f16_m128(DP), ks != 0);
-                ptx::mma_commit(&misc->o_full[g]);
-                ptx::mma_commit(&misc->vt_free[g]);
+                ptx::mma_commit(&misc->o_full[g]);       // (also tells the producer that the group's V~^T buffer is free)
             }
             return true;
         };
