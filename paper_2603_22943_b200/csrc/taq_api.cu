@@ -472,6 +472,11 @@ taq_status taq_layer_forward_a8(const taq_layer_desc* d, const void* x_f16_dev, 
     int* status = nullptr;
     s = status_ptr(&status);
     if (s != TAQ_OK) return s;
+    if (sm100_layer_a8_supported(*d)) {                                   // the whole integer-activation pass in one kernel
+        cudaError_t e1 = launch_layer_a8_sm100(*d, (const __half*)x_f16_dev, Wq_packed_dev, Wout_packed_dev, kv_packed_dev, (__half*)y_f16_dev,
+                                               d->batch, status, st);
+        return e1 == cudaSuccess ? TAQ_OK : cuda_fail(e1, "fused integer-activation layer launch");
+    }
     uint8_t* wsb = (uint8_t*)workspace_dev;
     int8_t* xq = (int8_t*)(wsb + WA.off_xq);
     float* xs = (float*)(wsb + WA.off_xs);

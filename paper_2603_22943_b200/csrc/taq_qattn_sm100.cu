@@ -68,6 +68,9 @@ struct Misc {
     uint32_t tmem_base;
     volatile int abort_flag;
     float sq[HG][ROWS];              // Q~ row scales
+    uint64_t xq_full;                // integer-activation variant: the int8 activation tiles are in place (X, later O)
+    float sx[ROWS];                  //   per-token scale of X, later of O
+    float xmax[4][ROWS];             //   partial absmax of a row's four threads
 };
 constexpr int TOTAL = OFF_MISC + (int)sizeof(Misc) + 1024;
 static_assert(TOTAL <= 232448, "shared memory budget");
@@ -145,7 +148,53 @@ __device__ __noinline__ uint32_t build_weight_tiles(unsigned char* smem, Misc* m
     return (uint32_t)s | (ph << 2) | (ok ? 0u : 8u);
 }
 
-template <bool TAIL_ONLY, bool FUSE_OUT>
+// Integer-activation variant: the same codes as int8, one tile per 128-element K block (= one scale group of the W4
+// format); the ring of three stages holds all three blocks of a projection at once.  Same calling convention.
+constexpr int NKB8 = (KIN + 127) / 128;
+static_assert(NKB8 == NBSTAGE, "the three int8 K blocks fill the ring exactly");
+__device__ __noinline__ uint32_t build_weight_tiles_i8(unsigned char* smem, Misc* misc, int first_pass, int wt, int lane, int s, uint32_t ph) {
+    const unsigned char* raw = smem + OFF_RAW;
+    bool ok = true;
+    for (int kb = 0; kb < NKB8; ++kb) {
+        if (!first_pass && !ptx::mbar_wait(&misc->b_empty[s], ph ^ 1)) ok = false;
+        if (!ok || misc->abort_flag) { ok = false; break; }
+        unsigned char* b_tile = smem + OFF_B + s * B_TILE;
+        constexpr int NCH = (NQ * 8 + NWORK - 1) / NWORK;       // 16-byte chunks (16 weights) per thread and K block
+        const int n0 = wt >> 3, c = wt & 7;
+        const int k0 = kb * 128 + c * 16;                       // first fan-in element of the chunk; beyond KIN: zeros
+        uint2 pw[NCH];
+#pragma unroll
+        for (int i = 0; i < NCH; ++i) {
+            pw[i] = make_uint2(0x88888888u, 0x88888888u);       // nibble 8 = code 0
+            if (n0 + (NWORK / 8) * i < NQ && k0 < KIN) pw[i] = *reinterpret_cast<const uint2*>(raw + (n0 + (NWORK / 8) * i) * (KIN / 2) + (k0 >> 1));
+        }
+#pragma unroll
+        for (int i = 0; i < NCH; ++i)
+            if (n0 + (NWORK / 8) * i < NQ) {
+                const uint2 lo = codes_w4_to_i8(pw[i].x), hi = codes_w4_to_i8(pw[i].y);
+                *reinterpret_cast<uint4*>(b_tile + ptx::sw128_offset(n0 + (NWORK / 8) * i, c)) = make_uint4(lo.x, lo.y, hi.x, hi.y);
+            }
+        ptx::fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&misc->b_full[s]);
+        if (++s == NBSTAGE) { s = 0; ph ^= 1; }
+    }
+    return (uint32_t)s | (ph << 2) | (ok ? 0u : 8u);
+}
+
+// rint(x / s) clamped to +-127 exactly as the stand-alone quantizer defines it (one IEEE division, then rintf): the product
+// with the reciprocal decides unless it lies within 1e-3 of a half-integer; then the division does.
+__device__ __forceinline__ int quant_code_exact(float x, float s, float rs) {
+    const float t = x * rs;
+    float q = rintf(t);
+    if (fabsf(t - q) > 0.499f) q = rintf(__fdiv_rn(x, s));
+    return (int)fminf(fmaxf(q, -127.f), 127.f);
+}
+
+// A8: the integer-activation layer pass.  X is quantized per token (Q_a over all 320 channels) inside the CTA, to_q and
+// to_out run as int8 x int8 -> int32 MMAs with one accumulator per 128-wide scale group, and O is quantized per token
+// from its fp16 tiles once both CTAs' halves are there.
+template <bool TAIL_ONLY, bool FUSE_OUT, bool A8 = false>
 __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_y, const QAttnArgs a) {
     extern __shared__ unsigned char smem_dyn[];
     unsigned char* smem = smem_dyn + ((1024u - (ptx::smem_u32(smem_dyn) & 1023u)) & 1023u);   // 1024-byte aligned, still provably shared
@@ -199,6 +248,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
             }
         }
         ptx::mbar_init(&misc->q_all, NWORK / 32);
+        ptx::mbar_init(&misc->xq_full, NWORK / 32);
         ptx::mbar_init(&misc->drain, 1);
         misc->abort_flag = 0;
         ptx::mbar_fence_init();
@@ -312,7 +362,22 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
         const uint32_t k_lo0 = ptx::desc_lo(ptx::smem_u32(smem + OFF_K)), vt_lo0 = ptx::desc_lo(ptx::smem_u32(smem + OFF_VT));
         int s = 0;                                       // weight ring position and pass parity, continued in phase 4
         uint32_t ph = 0;
-        {   // phase 1: one accumulation pass per scale group
+        if (A8) {   // phase 1, integer: K block g is scale group g, all three weight tiles fit the ring
+            ok = wait(&misc->xq_full, 0);
+            for (int g = 0; g < NKB8 && ok; ++g) {
+                if (!wait(&misc->b_full[g], 0)) { ok = false; break; }
+                if (leader) {
+                    TAQ_PROF(2 + g);
+                    const uint32_t a_lo = a_lo0 + g * (A_TILE >> 4), b_lo = b_lo0 + g * (B_TILE >> 4);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        ptx::mma_i8_ss(tmem_base + TMEM_ACC + g * NQ, ptx::desc_join(HI128, a_lo + 2 * k), ptx::desc_join(HI128, b_lo + 2 * k), ptx::idesc_i8_m128(NQ), k != 0);
+                    ptx::mma_commit(&misc->b_empty[g]);
+                    ptx::mma_commit(&misc->acc_full[g]);
+                }
+            }
+            s = 0; ph = 1;                               // the ring has been passed once
+        } else {   // phase 1: one accumulation pass per scale group
             int kb = 0;
             for (int g = 0; g < n_groups && ok; ++g) {
                 const int kb_end = min(NKB, kb + kb_per_group);
@@ -382,8 +447,23 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
             if (ok && leader) ptx::mbar_arrive_cluster_relaxed(ptx::map_to_cta(ptx::smem_u32(&misc->peer_got), peer));
             if (leader) TAQ_PROF(38);
             ptx::tc_fence_after_sync();                  // the workers' loads of the last O accumulators
+            if (A8) {    // integer to_out: the workers have turned the fp16 O tiles into three int8 tiles (in the Q~ region)
+                ok = ok && wait(&misc->xq_full, 1);
+                for (int g = 0; g < NKB8 && ok; ++g) {
+                    if (!wait(&misc->b_full[g], 1)) { ok = false; break; }
+                    if (leader) {
+                        TAQ_PROF(40 + g);
+                        const uint32_t o_lo = q_lo0 + g * (A_TILE >> 4), b_lo = b_lo0 + g * (B_TILE >> 4);
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)
+                            ptx::mma_i8_ss(tmem_base + TMEM_ACC + g * NQ, ptx::desc_join(HI128, o_lo + 2 * k), ptx::desc_join(HI128, b_lo + 2 * k), ptx::idesc_i8_m128(NQ), k != 0);
+                        ptx::mma_commit(&misc->b_empty[g]);
+                        ptx::mma_commit(&misc->acc_full[g]);
+                    }
+                }
+            }
             int kb = 0;
-            for (int g = 0; g < n_groups && ok; ++g) {
+            for (int g = 0; g < n_groups && ok && !A8; ++g) {
                 const int kb_end = min(NKB, kb + kb_per_group);
                 for (bool first = true; kb < kb_end && ok; ++kb) {
                     if (!wait(&misc->b_full[s], ph)) { ok = false; break; }
@@ -434,7 +514,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
         int s = 0;                                           // weight ring position and pass parity, continued in phase 4
         uint32_t ph = 0;
         auto build_tiles = [&](int first_pass) {
-            const uint32_t st = build_weight_tiles(smem, misc, first_pass, wt, lane, s, ph);
+            const uint32_t st = A8 ? build_weight_tiles_i8(smem, misc, first_pass, wt, lane, s, ph) : build_weight_tiles(smem, misc, first_pass, wt, lane, s, ph);
             s = (int)(st & 3u); ph = (st >> 2) & 1u;
             if (st >> 3) ok = false;
         };
@@ -455,16 +535,75 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
             for (int i = 0; i < 5; ++i) {
                 const float4 s0 = *reinterpret_cast<const float4*>(sg + i * 8), s1 = *reinterpret_cast<const float4*>(sg + i * 8 + 4);
                 float* yy = y + i * 8;
-                yy[0] = fmaf(__uint_as_float(v[i][0]), s0.x, yy[0]); yy[1] = fmaf(__uint_as_float(v[i][1]), s0.y, yy[1]);
-                yy[2] = fmaf(__uint_as_float(v[i][2]), s0.z, yy[2]); yy[3] = fmaf(__uint_as_float(v[i][3]), s0.w, yy[3]);
-                yy[4] = fmaf(__uint_as_float(v[i][4]), s1.x, yy[4]); yy[5] = fmaf(__uint_as_float(v[i][5]), s1.y, yy[5]);
-                yy[6] = fmaf(__uint_as_float(v[i][6]), s1.z, yy[6]); yy[7] = fmaf(__uint_as_float(v[i][7]), s1.w, yy[7]);
+                float f[8];
+#pragma unroll
+                for (int e2 = 0; e2 < 8; ++e2) f[e2] = A8 ? __int2float_rn((int)v[i][e2]) : __uint_as_float(v[i][e2]);
+                yy[0] = fmaf(f[0], s0.x, yy[0]); yy[1] = fmaf(f[1], s0.y, yy[1]);
+                yy[2] = fmaf(f[2], s0.z, yy[2]); yy[3] = fmaf(f[3], s0.w, yy[3]);
+                yy[4] = fmaf(f[4], s1.x, yy[4]); yy[5] = fmaf(f[5], s1.y, yy[5]);
+                yy[6] = fmaf(f[6], s1.z, yy[6]); yy[7] = fmaf(f[7], s1.w, yy[7]);
             }
         }
         ptx::tc_fence_before_sync();
         };
+        // Integer-activation variant: Q_a per token on this thread's 80 channels of its row, held as `vals` (ten 16-byte
+        // chunks of fp16 read from the tiles by the caller).  The row's four threads exchange their absmax; every thread
+        // has read its values before that barrier, so the int8 tiles may overwrite the fp16 tiles they were read from.
+        // Tiles: three K blocks of 128 channels at OFF_A (= OFF_Q), 128-byte rows, 128-byte swizzle; channels 320..383 zero.
+        auto quantize_row_piece = [&](const uint4 (&vals)[10], uint32_t parity) {
+            float amax = 0.f;
+#pragma unroll
+            for (int j = 0; j < 10; ++j) {
+                const __half2* h = reinterpret_cast<const __half2*>(&vals[j]);
+#pragma unroll
+                for (int e2 = 0; e2 < 4; ++e2) { const float2 f = __half22float2(h[e2]); amax = fmaxf(amax, fmaxf(fabsf(f.x), fabsf(f.y))); }
+            }
+            misc->xmax[part][r] = amax;
+            asm volatile("bar.sync 1, 512;" ::: "memory");
+            amax = fmaxf(fmaxf(misc->xmax[0][r], misc->xmax[1][r]), fmaxf(misc->xmax[2][r], misc->xmax[3][r]));
+            const float sc = quant_scale(amax, 127.f);
+            const float rs = sc > 0.f ? __frcp_rn(sc) : 0.f;
+            if (part == 0) misc->sx[r] = sc;
+#pragma unroll
+            for (int j = 0; j < 5; ++j) {                    // 16 channels -> one 16-byte chunk of int8 codes
+                uint32_t w[4] = {0, 0, 0, 0};
+                if (sc > 0.f) {
+#pragma unroll
+                    for (int u = 0; u < 2; ++u) {
+                        const __half2* h = reinterpret_cast<const __half2*>(&vals[2 * j + u]);
+#pragma unroll
+                        for (int e2 = 0; e2 < 4; ++e2) {
+                            const float2 f = __half22float2(h[e2]);
+                            w[2 * u + (e2 >> 1)] |= ((uint32_t)(quant_code_exact(f.x, sc, rs) & 0xFF) | ((uint32_t)(quant_code_exact(f.y, sc, rs) & 0xFF) << 8)) << (16 * (e2 & 1));
+                        }
+                    }
+                }
+                const int c16 = 5 * part + j;                // 16-channel chunk of the row, 0..19
+                *reinterpret_cast<uint4*>(smem + OFF_A + (c16 >> 3) * A_TILE + ptx::sw128_offset(r, c16 & 7)) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+            *reinterpret_cast<uint4*>(smem + OFF_A + 2 * A_TILE + ptx::sw128_offset(r, 4 + part)) = make_uint4(0, 0, 0, 0);
+            ptx::fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&misc->xq_full);
+            (void)parity;
+        };
         build_tiles(1);
+        if (A8) {                                            // X~ = Q_a(X) per token, from the fp16 tile that TMA brought
+            for (int kb = 0; kb < NKB && ok; ++kb) ok = ptx::mbar_wait(&misc->a_full[kb], 0) && !misc->abort_flag;
+            uint4 vals[10];
+#pragma unroll
+            for (int j = 0; j < 10; ++j) {
+                const int cg = 10 * part + j;                // 8-channel chunk of the row, 0..39
+                vals[j] = *reinterpret_cast<const uint4*>(smem + OFF_A + (cg >> 3) * A_TILE + ptx::sw128_offset(r, cg & 7));
+            }
+            quantize_row_piece(vals, 0);
+        }
         fold_groups(0);
+        if (A8) {
+            const float sxr = misc->sx[r];
+#pragma unroll
+            for (int c = 0; c < HC; ++c) y[c] *= sxr;
+        }
         if (!ok) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; }
         if (wt == 0) TAQ_PROF(7);
         // The last group's accumulator is complete, hence every MMA of phase 1 has finished reading shared memory and
@@ -641,7 +780,24 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
             if (wt == 0) TAQ_PROF(34);
             build_tiles(0);
             if (wt == 0) TAQ_PROF(35);
+            if (A8) {
+                // O~ = Q_a(O) per token from the fp16 tiles, once the partner's half has landed (o_all) and the partner has
+                // confirmed that this CTA's own tiles, which the int8 tiles overwrite, have arrived there (peer_got)
+                ok = ok && ptx::mbar_wait(&misc->o_all, 0) && ptx::mbar_wait(&misc->peer_got, 0) && !misc->abort_flag;
+                uint4 vals[10];
+#pragma unroll
+                for (int j = 0; j < 10; ++j) {
+                    const int cg = 10 * part + j;                // 8-channel chunk of the row, 0..39
+                    vals[j] = *reinterpret_cast<const uint4*>(smem + o_tile_offset(cg >> 2) + ptx::sw64_offset(r, cg & 3));
+                }
+                quantize_row_piece(vals, 1);
+            }
             fold_groups(1);
+            if (A8) {
+                const float sxr = misc->sx[r];
+#pragma unroll
+                for (int c = 0; c < HC; ++c) y[c] *= sxr;
+            }
             if (wt == 0) TAQ_PROF(36);
             if (!ok) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; }
             // Every MMA of phase 4 is complete: the ring is free.  The 128 x 160 fp16 output tile is staged there as five
@@ -711,7 +867,7 @@ bool sm100_qattn_supported(const taq_layer_desc& d) {
 }
 
 static cudaError_t launch_c320(const taq_layer_desc& d, const __half* x, const void* wq, const void* kv, const taq_request* reqs, __half* o,
-                               const void* wout, __half* y, int n_z, int* status, cudaStream_t stream) {
+                               const void* wout, __half* y, int n_z, int* status, cudaStream_t stream, bool a8 = false) {
     if (n_z == 0 || d.n_query == 0) return cudaSuccess;
     EncodeTiledFn enc = encode_tiled_fn2();
     if (!enc) return cudaErrorNotSupported;
@@ -728,7 +884,7 @@ static cudaError_t launch_c320(const taq_layer_desc& d, const __half* x, const v
     a.n_query = d.n_query; a.heads = d.heads; a.n_ctx = d.n_ctx; a.max_trigger = d.max_trigger; a.group = d.w_group; a.q_bits = d.q_bits; a.p_bits = d.p_bits;
     a.status = status;
     dim3 grid((d.n_query + ROWS - 1) / ROWS, d.heads / HG, n_z);
-    static bool configured[4] = {false, false, false, false};
+    static bool configured[8] = {false, false, false, false, false, false, false, false};
     const bool tail = d.n_ctx > 64, fuse_out = y != nullptr;
     CUtensorMap tmap_y = tmap;                        // (unused by the variant that stores O)
     if (fuse_out) {
@@ -738,8 +894,9 @@ static cudaError_t launch_c320(const taq_layer_desc& d, const __half* x, const v
         if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
     }
     void (*kern)(const CUtensorMap, const CUtensorMap, const QAttnArgs) =
-        fuse_out ? (tail ? qattn_c320_kernel<true, true> : qattn_c320_kernel<false, true>) : (tail ? qattn_c320_kernel<true, false> : qattn_c320_kernel<false, false>);
-    const int ci = (tail ? 1 : 0) + (fuse_out ? 2 : 0);
+        a8 ? (tail ? qattn_c320_kernel<true, true, true> : qattn_c320_kernel<false, true, true>)
+           : fuse_out ? (tail ? qattn_c320_kernel<true, true> : qattn_c320_kernel<false, true>) : (tail ? qattn_c320_kernel<true, false> : qattn_c320_kernel<false, false>);
+    const int ci = (tail ? 1 : 0) + (fuse_out ? 2 : 0) + (a8 ? 4 : 0);
     if (!configured[ci]) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TOTAL);
         if (e != cudaSuccess) return e;
@@ -757,6 +914,13 @@ cudaError_t launch_qattn_sm100(const taq_layer_desc& d, const __half* x, const v
 cudaError_t launch_layer_sm100(const taq_layer_desc& d, const __half* x, const void* wq, const void* wout, const void* kv, const taq_request* reqs,
                                __half* y, int n_z, int* status, cudaStream_t stream) {
     return launch_c320(d, x, wq, kv, reqs, nullptr, wout, y, n_z, status, stream);
+}
+
+bool sm100_layer_a8_supported(const taq_layer_desc& d) { return sm100_qattn_supported(d) && d.w_group == 128; }
+
+cudaError_t launch_layer_a8_sm100(const taq_layer_desc& d, const __half* x, const void* wq, const void* wout, const void* kv, __half* y, int n_z,
+                                  int* status, cudaStream_t stream) {
+    return launch_c320(d, x, wq, kv, nullptr, nullptr, wout, y, n_z, status, stream, true);
 }
 
 }  // namespace taq

@@ -22,4 +22,9 @@ bool sm100_layer_supported(const taq_layer_desc& d);
 cudaError_t launch_layer_sm100(const taq_layer_desc& d, const __half* x, const void* wq, const void* wout, const void* kv, const taq_request* reqs,
                                __half* y, int n_z, int* status, cudaStream_t stream);
 
+// The same with int8 X and O (per-token Q_a inside the kernel, int8 x int8 -> int32 projections); needs W4 groups of 128.
+bool sm100_layer_a8_supported(const taq_layer_desc& d);
+cudaError_t launch_layer_a8_sm100(const taq_layer_desc& d, const __half* x, const void* wq, const void* wout, const void* kv, __half* y, int n_z,
+                                  int* status, cudaStream_t stream);
+
 }  // namespace taq
