@@ -182,13 +182,87 @@ __device__ __noinline__ uint32_t build_weight_tiles_i8(unsigned char* smem, Misc
     return (uint32_t)s | (ph << 2) | (ok ? 0u : 8u);
 }
 
-// rint(x / s) clamped to +-127 exactly as the stand-alone quantizer defines it (one IEEE division, then rintf): the product
-// with the reciprocal decides unless it lies within 1e-3 of a half-integer; then the division does.
-__device__ __forceinline__ int quant_code_exact(float x, float s, float rs) {
-    const float t = x * rs;
-    float q = rintf(t);
-    if (fabsf(t - q) > 0.499f) q = rintf(__fdiv_rn(x, s));
-    return (int)fminf(fmaxf(q, -127.f), 127.f);
+// Sixteen codes rint(x / s), clamped to +-127, exactly as the stand-alone quantizer defines them (one IEEE division each,
+// then rintf): the rare path.
+__device__ __noinline__ uint4 quant16_by_division(uint4 lo8, uint4 hi8, float s) {
+    uint32_t w[4] = {0, 0, 0, 0};
+    const uint4 v[2] = {lo8, hi8};
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+        const __half2* h = reinterpret_cast<const __half2*>(&v[u]);
+#pragma unroll
+        for (int e2 = 0; e2 < 4; ++e2) {
+            const float2 f = __half22float2(h[e2]);
+            const int a = (int)fminf(fmaxf(rintf(__fdiv_rn(f.x, s)), -127.f), 127.f), b = (int)fminf(fmaxf(rintf(__fdiv_rn(f.y, s)), -127.f), 127.f);
+            w[2 * u + (e2 >> 1)] |= ((uint32_t)(a & 0xFF) | ((uint32_t)(b & 0xFF) << 8)) << (16 * (e2 & 1));
+        }
+    }
+    return make_uint4(w[0], w[1], w[2], w[3]);
+}
+// The same sixteen codes on the fast path: fma(x, 1/s, 1.5 * 2^23) leaves rint(x / s) in the low byte unless x / s lies
+// within 4e-5 of a half-integer (the product with the rounded reciprocal is within 2.3e-5 of the rounded quotient for
+// |x / s| <= 127); such a chunk - about one in a thousand - is redone by division.
+__device__ __forceinline__ uint4 quant16(uint4 lo8, uint4 hi8, float s, float rs) {
+    const uint4 v[2] = {lo8, hi8};
+    uint32_t b[16];
+    float dmax = 0.f;
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+        const __half2* h = reinterpret_cast<const __half2*>(&v[u]);
+#pragma unroll
+        for (int e2 = 0; e2 < 4; ++e2) {
+            const float2 f = __half22float2(h[e2]);
+            const float u0 = fmaf(f.x, rs, 12582912.0f), u1 = fmaf(f.y, rs, 12582912.0f);
+            dmax = fmaxf(dmax, fmaxf(fabsf(fmaf(f.x, rs, 12582912.0f - u0)), fabsf(fmaf(f.y, rs, 12582912.0f - u1))));
+            b[8 * u + 2 * e2] = __float_as_uint(u0);
+            b[8 * u + 2 * e2 + 1] = __float_as_uint(u1);
+        }
+    }
+    if (dmax > 0.49996f) return quant16_by_division(lo8, hi8, s);
+    uint4 out;
+    out.x = __byte_perm(__byte_perm(b[0], b[1], 0x0040), __byte_perm(b[2], b[3], 0x0040), 0x5410);
+    out.y = __byte_perm(__byte_perm(b[4], b[5], 0x0040), __byte_perm(b[6], b[7], 0x0040), 0x5410);
+    out.z = __byte_perm(__byte_perm(b[8], b[9], 0x0040), __byte_perm(b[10], b[11], 0x0040), 0x5410);
+    out.w = __byte_perm(__byte_perm(b[12], b[13], 0x0040), __byte_perm(b[14], b[15], 0x0040), 0x5410);
+    return out;
+}
+
+// Integer-activation variant: Q_a per token inside the CTA (all 512 worker threads; four threads per row, 80 channels
+// each).  `from_o` = 0: the row's fp16 values are read from the X tile (five 64-channel blocks, 128-byte swizzle);
+// 1: from the ten 32-channel O tiles (64-byte swizzle).  Two streaming passes over the row piece, written as real loops
+// (this code runs once per CTA: short code is fetch time saved): absmax, exchanged between the row's four threads
+// through shared memory, then the codes, which go into three int8 tiles elsewhere in shared memory (K blocks of 128
+// channels, 128-byte rows and swizzle, channels 320..383 zero) at the offsets dst[0..2].
+__device__ __noinline__ void quantize_tokens(unsigned char* smem, Misc* misc, int from_o, int r, int part, int lane, int dst0, int dst1, int dst2) {
+    auto chunk = [&](int cg) -> uint4 {                  // 8-channel chunk cg (0..39) of row r
+        const unsigned char* src = from_o ? smem + o_tile_offset(cg >> 2) + ptx::sw64_offset(r, cg & 3)
+                                          : smem + OFF_A + (cg >> 3) * A_TILE + ptx::sw128_offset(r, cg & 7);
+        return *reinterpret_cast<const uint4*>(src);
+    };
+    __half2 m2 = __floats2half2_rn(0.f, 0.f);
+#pragma unroll 1
+    for (int j = 0; j < 10; ++j) {
+        const uint4 v = chunk(10 * part + j);
+        const __half2* h = reinterpret_cast<const __half2*>(&v);
+        m2 = __hmax2(m2, __hmax2(__hmax2(__habs2(h[0]), __habs2(h[1])), __hmax2(__habs2(h[2]), __habs2(h[3]))));
+    }
+    misc->xmax[part][r] = fmaxf(__low2float(m2), __high2float(m2));
+    asm volatile("bar.sync 1, 512;" ::: "memory");
+    const float amax = fmaxf(fmaxf(misc->xmax[0][r], misc->xmax[1][r]), fmaxf(misc->xmax[2][r], misc->xmax[3][r]));
+    const float sc = quant_scale(amax, 127.f);
+    const float rs = sc > 0.f ? __frcp_rn(sc) : 0.f;
+    if (part == 0) misc->sx[r] = sc;
+#pragma unroll 1
+    for (int j = 0; j < 5; ++j) {                        // 16 channels -> one 16-byte chunk of int8 codes
+        const int c16 = 5 * part + j;                    // 16-channel chunk of the row, 0..19
+        const uint4 codes = sc > 0.f ? quant16(chunk(2 * c16), chunk(2 * c16 + 1), sc, rs) : make_uint4(0, 0, 0, 0);
+        const int tile = c16 >> 3;
+        *reinterpret_cast<uint4*>(smem + (tile == 0 ? dst0 : tile == 1 ? dst1 : dst2) + ptx::sw128_offset(r, c16 & 7)) = codes;
+    }
+    *reinterpret_cast<uint4*>(smem + dst2 + ptx::sw128_offset(r, 4 + part)) = make_uint4(0, 0, 0, 0);
+    ptx::fence_proxy_async_smem();
+    __syncwarp();
+    if (lane == 0) ptx::mbar_arrive(&misc->xq_full);
 }
 
 // A8: the integer-activation layer pass.  X is quantized per token (Q_a over all 320 channels) inside the CTA, to_q and
@@ -288,9 +362,11 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
             // K~/V~ operand images: the constants of all four heads at once; K~ and V~^T tiles of head hi go to the
             // buffers of group hi & 1.  A group's K~ buffer is free again as soon as its S has been computed, its V~^T
             // buffer after its PV, so the second head's tiles arrive under the first head's softmax.
-            ptx::mbar_arrive_expect_tx(&misc->c_full, HG * kOperandConstBytes);
-            for (int hi = 0; hi < HG; ++hi)
-                ptx::bulk_load(smem + OFF_CST + hi * kOperandConstBytes, img + (size_t)hi * KL.operand_head_bytes + K_BYTES + VT_BYTES, kOperandConstBytes, &misc->c_full);
+            auto load_consts = [&]() {
+                ptx::mbar_arrive_expect_tx(&misc->c_full, HG * kOperandConstBytes);
+                for (int hi = 0; hi < HG; ++hi)
+                    ptx::bulk_load(smem + OFF_CST + hi * kOperandConstBytes, img + (size_t)hi * KL.operand_head_bytes + K_BYTES + VT_BYTES, kOperandConstBytes, &misc->c_full);
+            };
             auto load_k = [&](int hi) {
                 ptx::mbar_arrive_expect_tx(&misc->k_full[hi & 1], K_BYTES);
                 ptx::bulk_load(smem + OFF_K + (hi & 1) * K_BYTES, img + (size_t)hi * KL.operand_head_bytes, K_BYTES, &misc->k_full[hi & 1]);
@@ -299,7 +375,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
                 ptx::mbar_arrive_expect_tx(&misc->vt_full[hi & 1], VT_BYTES);
                 ptx::bulk_load(smem + OFF_VT + (hi & 1) * VT_BYTES, img + (size_t)hi * KL.operand_head_bytes + K_BYTES, VT_BYTES, &misc->vt_full[hi & 1]);
             };
-            load_k(0); load_k(1); load_vt(0); load_vt(1);
+            // (integer-activation variant: the int8 X tiles occupy this region during phase 1; the images follow below)
+            if (!A8) { load_consts(); load_k(0); load_k(1); load_vt(0); load_vt(1); }
             int k_issued = 2, vt_issued = 2;
             if (FUSE_OUT) {       // phase 1 no longer needs the packed Wq: fetch the packed Wout rows of this CTA's output channels
                 if (!ptx::mbar_wait(&misc->acc_full[n_groups - 1], 0)) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; }
@@ -311,6 +388,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
                     ptx::bulk_load(smem + OFF_BIAS, blob2 + L.off_bias + (size_t)col0 * 4, NQ * 4, &misc->w2_full);
                 }
             }
+            if (A8 && !misc->abort_flag) { load_consts(); load_k(0); load_k(1); load_vt(0); load_vt(1); }    // phase 1 is over
             for (int g = 0; g < 2 && !misc->abort_flag; ++g) {
                 if (!ptx::mbar_wait(&misc->s_full[g], 0)) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; break; }
                 load_k(2 + g);
@@ -368,7 +446,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
                 if (!wait(&misc->b_full[g], 0)) { ok = false; break; }
                 if (leader) {
                     TAQ_PROF(2 + g);
-                    const uint32_t a_lo = a_lo0 + g * (A_TILE >> 4), b_lo = b_lo0 + g * (B_TILE >> 4);
+                    const uint32_t a_lo = k_lo0 + g * (A_TILE >> 4), b_lo = b_lo0 + g * (B_TILE >> 4);      // X~ tiles sit in the K~/V~ region
 #pragma unroll
                     for (int k = 0; k < 4; ++k)
                         ptx::mma_i8_ss(tmem_base + TMEM_ACC + g * NQ, ptx::desc_join(HI128, a_lo + 2 * k), ptx::desc_join(HI128, b_lo + 2 * k), ptx::idesc_i8_m128(NQ), k != 0);
@@ -453,7 +531,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
                     if (!wait(&misc->b_full[g], 1)) { ok = false; break; }
                     if (leader) {
                         TAQ_PROF(40 + g);
-                        const uint32_t o_lo = q_lo0 + g * (A_TILE >> 4), b_lo = b_lo0 + g * (B_TILE >> 4);
+                        const uint32_t o_lo = g == 0 ? p_lo0 : g == 1 ? vt_lo0 : ptx::desc_lo(ptx::smem_u32(smem + OFF_RAW));
+                        const uint32_t b_lo = b_lo0 + g * (B_TILE >> 4);
 #pragma unroll
                         for (int k = 0; k < 4; ++k)
                             ptx::mma_i8_ss(tmem_base + TMEM_ACC + g * NQ, ptx::desc_join(HI128, o_lo + 2 * k), ptx::desc_join(HI128, b_lo + 2 * k), ptx::idesc_i8_m128(NQ), k != 0);
@@ -546,57 +625,10 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
         }
         ptx::tc_fence_before_sync();
         };
-        // Integer-activation variant: Q_a per token on this thread's 80 channels of its row, held as `vals` (ten 16-byte
-        // chunks of fp16 read from the tiles by the caller).  The row's four threads exchange their absmax; every thread
-        // has read its values before that barrier, so the int8 tiles may overwrite the fp16 tiles they were read from.
-        // Tiles: three K blocks of 128 channels at OFF_A (= OFF_Q), 128-byte rows, 128-byte swizzle; channels 320..383 zero.
-        auto quantize_row_piece = [&](const uint4 (&vals)[10], uint32_t parity) {
-            float amax = 0.f;
-#pragma unroll
-            for (int j = 0; j < 10; ++j) {
-                const __half2* h = reinterpret_cast<const __half2*>(&vals[j]);
-#pragma unroll
-                for (int e2 = 0; e2 < 4; ++e2) { const float2 f = __half22float2(h[e2]); amax = fmaxf(amax, fmaxf(fabsf(f.x), fabsf(f.y))); }
-            }
-            misc->xmax[part][r] = amax;
-            asm volatile("bar.sync 1, 512;" ::: "memory");
-            amax = fmaxf(fmaxf(misc->xmax[0][r], misc->xmax[1][r]), fmaxf(misc->xmax[2][r], misc->xmax[3][r]));
-            const float sc = quant_scale(amax, 127.f);
-            const float rs = sc > 0.f ? __frcp_rn(sc) : 0.f;
-            if (part == 0) misc->sx[r] = sc;
-#pragma unroll
-            for (int j = 0; j < 5; ++j) {                    // 16 channels -> one 16-byte chunk of int8 codes
-                uint32_t w[4] = {0, 0, 0, 0};
-                if (sc > 0.f) {
-#pragma unroll
-                    for (int u = 0; u < 2; ++u) {
-                        const __half2* h = reinterpret_cast<const __half2*>(&vals[2 * j + u]);
-#pragma unroll
-                        for (int e2 = 0; e2 < 4; ++e2) {
-                            const float2 f = __half22float2(h[e2]);
-                            w[2 * u + (e2 >> 1)] |= ((uint32_t)(quant_code_exact(f.x, sc, rs) & 0xFF) | ((uint32_t)(quant_code_exact(f.y, sc, rs) & 0xFF) << 8)) << (16 * (e2 & 1));
-                        }
-                    }
-                }
-                const int c16 = 5 * part + j;                // 16-channel chunk of the row, 0..19
-                *reinterpret_cast<uint4*>(smem + OFF_A + (c16 >> 3) * A_TILE + ptx::sw128_offset(r, c16 & 7)) = make_uint4(w[0], w[1], w[2], w[3]);
-            }
-            *reinterpret_cast<uint4*>(smem + OFF_A + 2 * A_TILE + ptx::sw128_offset(r, 4 + part)) = make_uint4(0, 0, 0, 0);
-            ptx::fence_proxy_async_smem();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(&misc->xq_full);
-            (void)parity;
-        };
         build_tiles(1);
         if (A8) {                                            // X~ = Q_a(X) per token, from the fp16 tile that TMA brought
             for (int kb = 0; kb < NKB && ok; ++kb) ok = ptx::mbar_wait(&misc->a_full[kb], 0) && !misc->abort_flag;
-            uint4 vals[10];
-#pragma unroll
-            for (int j = 0; j < 10; ++j) {
-                const int cg = 10 * part + j;                // 8-channel chunk of the row, 0..39
-                vals[j] = *reinterpret_cast<const uint4*>(smem + OFF_A + (cg >> 3) * A_TILE + ptx::sw128_offset(r, cg & 7));
-            }
-            quantize_row_piece(vals, 0);
+            quantize_tokens(smem, misc, 0, r, part, lane, OFF_K, OFF_K + A_TILE, OFF_K + 2 * A_TILE);
         }
         fold_groups(0);
         if (A8) {
@@ -781,16 +813,11 @@ __global__ void __launch_bounds__(NTHREADS, 1) qattn_c320_kernel(const __grid_co
             build_tiles(0);
             if (wt == 0) TAQ_PROF(35);
             if (A8) {
-                // O~ = Q_a(O) per token from the fp16 tiles, once the partner's half has landed (o_all) and the partner has
-                // confirmed that this CTA's own tiles, which the int8 tiles overwrite, have arrived there (peer_got)
-                ok = ok && ptx::mbar_wait(&misc->o_all, 0) && ptx::mbar_wait(&misc->peer_got, 0) && !misc->abort_flag;
-                uint4 vals[10];
-#pragma unroll
-                for (int j = 0; j < 10; ++j) {
-                    const int cg = 10 * part + j;                // 8-channel chunk of the row, 0..39
-                    vals[j] = *reinterpret_cast<const uint4*>(smem + o_tile_offset(cg >> 2) + ptx::sw64_offset(r, cg & 3));
-                }
-                quantize_row_piece(vals, 1);
+                // O~ = Q_a(O) per token from the fp16 tiles, once the partner's half has landed (o_all).  The int8 tiles go
+                // where nothing is live any more: the first P block, the V~^T buffers, and the packed Wout codes, which
+                // every warp has finished expanding when it passes the barrier inside.
+                ok = ok && ptx::mbar_wait(&misc->o_all, 0) && !misc->abort_flag;
+                quantize_tokens(smem, misc, 1, r, part, lane, OFF_P, OFF_VT, OFF_RAW);
             }
             fold_groups(1);
             if (A8) {

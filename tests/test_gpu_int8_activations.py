@@ -160,3 +160,30 @@ def test_a8_empty_inputs_and_bad_arguments():
         tb.lib().taq_quantize_rows_f16.restype = tb.C.c_int
         tb._check(tb.lib().taq_quantize_rows_f16(z.data_ptr(), 4, 12, z.data_ptr(), z.data_ptr(), None))
     assert e.value.status == tb.TAQ_ERR_SHAPE
+
+
+@pytest.mark.parametrize("n,q_bits", [(4096, 8), (333, 8), (130, 0)])
+def test_one_kernel_a8_layer_equals_the_step_by_step_composition(n, q_bits):
+    """At C = 320 / 8 heads / W4 g128 the integer-activation pass is one kernel (Q_a of X and O inside the CTA).  The same
+    pass composed from the stand-alone entry points - quantize, integer to_q, attention, quantize, integer to_out - gives
+    the same bits: the per-token codes are the stand-alone quantizer's, the integer products are exact, and the fp32
+    combinations run in the same order."""
+    shape = replace(synth.shrink(synth.config2(), n), seed=26, q_bits=q_bits)
+    data = synth.make_layer(shape)
+    desc = tl.gpu_desc(shape)
+    P = tl.pack_layer_weights(shape, data)
+    mask = dev(data["mask"])
+    kv = tb.taq_kv_project_a8(desc, dev(data["ctx"]), P["Wk"], P["Wv"], mask)
+    x = dev(data["X"])
+    y = tb.taq_layer_forward_a8(desc, x, P["Wq"], P["Wout"], kv, mask)
+    M, C_, H = shape.rows, shape.channels, shape.heads
+    xc, xs = tb.taq_quantize_rows_f16(x.view(M, C_))
+    if q_bits == 8:
+        qc, qs = tb.taq_quantized_linear_i8(P["wd_cc"], xc, xs, P["Wq"], tb.TAQ_OUT_INT8_HEAD_ROWS, heads=H)
+    else:
+        qc, qs = tb.taq_quantized_linear_i8(P["wd_cc"], xc, xs, P["Wq"], tb.TAQ_OUT_F16), None
+    o = tb.taq_cross_attention(desc, qc, qs, kv, mask)
+    oc, os_ = tb.taq_quantize_rows_f16(o.view(M, C_))
+    want = tb.taq_quantized_linear_i8(P["wd_cc"], oc, os_, P["Wout"], tb.TAQ_OUT_F16)
+    tb.taq_poll_device_status()
+    assert torch.equal(y.view(M, C_).view(torch.int16), want.view(torch.int16))
