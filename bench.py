@@ -423,8 +423,8 @@ def main():
         s = sets[i % n_sets]
         tb.taq_quantized_linear(wd_cc, o_sets[i % n_sets], s["Wout"], tb.TAQ_OUT_F16, y=s["y"])
 
-    # the integer-activation reading (int8 X and O, tcgen05 kind::i8): the five-kernel layer pass, and its to_out GEMM
-    # alone on codes quantized beforehand
+    # the integer-activation reading (int8 X and O, tcgen05 kind::i8): the layer pass, and its to_out GEMM alone on codes
+    # quantized beforehand
     ws_a8 = torch.empty(tb.taq_workspace_bytes_a8(desc), dtype=torch.uint8, device="cuda")
     oq_sets = [tb.taq_quantize_rows_f16(sets[i]["x"].view(M, C_)) for i in range(n_sets)]
 
@@ -516,7 +516,7 @@ def main():
          "bytes": M * C_ * 2 + qbytes + wbytes, "flops": 2 * M * C_ * C_, "traffic": None},
         {"name": "attention_sm100_kernel<40>: attention, stand-alone (taq_cross_attention)", "ms": stage_ms["attn"], "in_step": False,
          "bytes": qbytes + M * C_ * 2 + img_bytes, "flops": 4 * M * T * C_, "traffic": None},
-        {"name": "integer-activation layer pass, 5 kernels: Q_a(X), int8 to_q, attention, Q_a(O), int8 to_out (taq_layer_forward_a8)", "ms": stage_ms["layer_a8"],
+        {"name": "qattn_c320_kernel<.,true,int8>: integer-activation layer pass in one kernel, Q_a(X) and Q_a(O) inside the CTA (taq_layer_forward_a8)", "ms": stage_ms["layer_a8"],
          "in_step": False, "bytes": 2 * M * C_ * 2 + 2 * wbytes + img_bytes, "flops": 4 * M * C_ * C_ + 4 * M * T * C_, "traffic": None},
         {"name": "linear_sm100_kernel<160,int8>: to_out as int8 x int8 -> int32 GEMM, stand-alone (taq_quantized_linear_i8)", "ms": stage_ms["to_out_i8"],
          "in_step": False, "bytes": M * C_ + M * 4 + M * C_ * 2 + wbytes, "flops": 2 * M * C_ * C_, "traffic": None},

@@ -218,8 +218,9 @@ taq_status taq_quantized_linear_i8(const taq_weight_desc* desc, const int8_t* x_
                                    int32_t heads, float* scales_dev, void* stream);
 
 /* taq_layer_forward with int8 X and O: Q_a(X) per token, integer to_q (+ Q_a per head row), attention as
- * before, Q_a(O) per token on the fp16 O, integer to_out (+ bias).  Five kernels; workspace_dev >=
- * taq_workspace_bytes_a8(desc), 128-byte aligned. */
+ * before, Q_a(O) per token on the fp16 O, integer to_out (+ bias).  One kernel for the SD-1.5 64x64 shape (C = 320,
+ * 8 heads, W4 groups of 128: both quantizers run inside the CTA), five kernels otherwise; the results are the same
+ * bits.  workspace_dev >= taq_workspace_bytes_a8(desc), 128-byte aligned. */
 size_t taq_workspace_bytes_a8(const taq_layer_desc* desc);
 taq_status taq_layer_forward_a8(const taq_layer_desc* desc, const void* x_f16_dev, const void* Wq_packed_dev,
                                 const void* Wout_packed_dev, const void* kv_packed_dev,
