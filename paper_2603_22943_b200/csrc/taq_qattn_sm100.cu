@@ -200,8 +200,8 @@ __device__ __noinline__ uint4 quant16_by_division(uint4 lo8, uint4 hi8, float s)
     return make_uint4(w[0], w[1], w[2], w[3]);
 }
 // The same sixteen codes on the fast path: fma(x, 1/s, 1.5 * 2^23) leaves rint(x / s) in the low byte unless x / s lies
-// within 4e-5 of a half-integer (the product with the rounded reciprocal is within 2.3e-5 of the rounded quotient for
-// |x / s| <= 127); such a chunk - about one in a thousand - is redone by division.
+// within 2e-5 of a half-integer (the product with the correctly rounded reciprocal is within 1.6e-5 of the rounded
+// quotient for |x / s| <= 127: two relative errors of 2^-24); such a chunk - about one in 1500 - is redone by division.
 __device__ __forceinline__ uint4 quant16(uint4 lo8, uint4 hi8, float s, float rs) {
     const uint4 v[2] = {lo8, hi8};
     uint32_t b[16];
@@ -218,7 +218,7 @@ __device__ __forceinline__ uint4 quant16(uint4 lo8, uint4 hi8, float s, float rs
             b[8 * u + 2 * e2 + 1] = __float_as_uint(u1);
         }
     }
-    if (dmax > 0.49996f) return quant16_by_division(lo8, hi8, s);
+    if (dmax > 0.49998f) return quant16_by_division(lo8, hi8, s);
     uint4 out;
     out.x = __byte_perm(__byte_perm(b[0], b[1], 0x0040), __byte_perm(b[2], b[3], 0x0040), 0x5410);
     out.y = __byte_perm(__byte_perm(b[4], b[5], 0x0040), __byte_perm(b[6], b[7], 0x0040), 0x5410);
