@@ -55,14 +55,14 @@ cudaError_t launch_quantize_rows(const float* x, long long rows, int cols, int q
     return cudaGetLastError();
 }
 
-// rint(x / s) clamped to +-127, bit-identical to quant_code (one IEEE division, then rintf) at a fraction of its cost:
-// the product with the reciprocal is within 3e-5 of the quotient for |x / s| <= 127, so both round to the same integer
-// unless the product lies within 1e-3 of a half-integer; only then the division decides.
-__device__ __forceinline__ int quant_code_127(float x, float s, float rs) {
-    const float t = x * rs;
-    float q = rintf(t);
-    if (fabsf(t - q) > 0.499f) q = rintf(__fdiv_rn(x, s));
-    return (int)fminf(fmaxf(q, -127.f), 127.f);
+// rint(x / s) clamped to +-127, bit-identical to quant_code (one IEEE division, then rintf) at a fraction of its cost.
+// fma(x, r, 1.5 * 2^23) leaves rint(x r) in the low bits.  The rounded quotient fl(x / s) and the product with the
+// correctly rounded reciprocal both lie between x r_lo and x r_hi (r two ulps down and up), so when both ends round to
+// the same integer that integer is the code; only otherwise the division decides.
+__device__ __forceinline__ int quant_code_127(float x, float s, float r_lo, float r_hi) {
+    const uint32_t a = __float_as_uint(fmaf(x, r_lo, 12582912.0f)), c = __float_as_uint(fmaf(x, r_hi, 12582912.0f));
+    if (a != c) return (int)fminf(fmaxf(rintf(__fdiv_rn(x, s)), -127.f), 127.f);
+    return (int)(a << 24) >> 24;                       // the low byte, sign-extended
 }
 
 // Per-token quantizer of fp16 activations (the inputs of the integer-activation projections): one warp per row of
@@ -99,6 +99,7 @@ __global__ void __launch_bounds__(256) quantize_rows_f16_kernel(const __half* __
         a = warp_max(a);
         const float s = quant_scale(a, 127.f);
         const float rs = s > 0.f ? __frcp_rn(s) : 0.f;
+        const float r_lo = __uint_as_float(__float_as_uint(rs) - 2u), r_hi = __uint_as_float(__float_as_uint(rs) + 2u);
         if (lane == 0) scales[r] = s;
         uint2* cr = reinterpret_cast<uint2*>(codes + r * cols);
         auto encode = [&](const uint4& v) {
@@ -108,7 +109,7 @@ __global__ void __launch_bounds__(256) quantize_rows_f16_kernel(const __half* __
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
                     const float2 f = __half22float2(h[e]);
-                    w[e >> 1] |= ((uint32_t)(quant_code_127(f.x, s, rs) & 0xFF) | ((uint32_t)(quant_code_127(f.y, s, rs) & 0xFF) << 8)) << (16 * (e & 1));
+                    w[e >> 1] |= ((uint32_t)(quant_code_127(f.x, s, r_lo, r_hi) & 0xFF) | ((uint32_t)(quant_code_127(f.y, s, r_lo, r_hi) & 0xFF) << 8)) << (16 * (e & 1));
                 }
             }
             return make_uint2(w[0], w[1]);

@@ -199,26 +199,30 @@ __device__ __noinline__ uint4 quant16_by_division(uint4 lo8, uint4 hi8, float s)
     }
     return make_uint4(w[0], w[1], w[2], w[3]);
 }
-// The same sixteen codes on the fast path: fma(x, 1/s, 1.5 * 2^23) leaves rint(x / s) in the low byte unless x / s lies
-// within 2e-5 of a half-integer (the product with the correctly rounded reciprocal is within 1.6e-5 of the rounded
-// quotient for |x / s| <= 127: two relative errors of 2^-24); such a chunk - about one in 1500 - is redone by division.
+// The same sixteen codes on the fast path.  fma(x, r, 1.5 * 2^23) leaves rint(x r) in the low byte.  The definition's
+// rounded quotient fl(x / s) and the product with the correctly rounded reciprocal both lie between x r_lo and x r_hi
+// (r two ulps down and up: each of them is off the exact quotient by at most one relative 2^-24), so when both ends
+// round to the same integer that integer is the definition's code; otherwise - about one chunk in 150 - the chunk is
+// redone by division.
 __device__ __forceinline__ uint4 quant16(uint4 lo8, uint4 hi8, float s, float rs) {
+    const float r_lo = __uint_as_float(__float_as_uint(rs) - 2u), r_hi = __uint_as_float(__float_as_uint(rs) + 2u);
     const uint4 v[2] = {lo8, hi8};
     uint32_t b[16];
-    float dmax = 0.f;
+    uint32_t differ = 0;
 #pragma unroll
     for (int u = 0; u < 2; ++u) {
         const __half2* h = reinterpret_cast<const __half2*>(&v[u]);
 #pragma unroll
         for (int e2 = 0; e2 < 4; ++e2) {
             const float2 f = __half22float2(h[e2]);
-            const float u0 = fmaf(f.x, rs, 12582912.0f), u1 = fmaf(f.y, rs, 12582912.0f);
-            dmax = fmaxf(dmax, fmaxf(fabsf(fmaf(f.x, rs, 12582912.0f - u0)), fabsf(fmaf(f.y, rs, 12582912.0f - u1))));
-            b[8 * u + 2 * e2] = __float_as_uint(u0);
-            b[8 * u + 2 * e2 + 1] = __float_as_uint(u1);
+            const uint32_t a0 = __float_as_uint(fmaf(f.x, r_lo, 12582912.0f)), a1 = __float_as_uint(fmaf(f.y, r_lo, 12582912.0f));
+            const uint32_t c0 = __float_as_uint(fmaf(f.x, r_hi, 12582912.0f)), c1 = __float_as_uint(fmaf(f.y, r_hi, 12582912.0f));
+            differ |= (a0 ^ c0) | (a1 ^ c1);
+            b[8 * u + 2 * e2] = a0;
+            b[8 * u + 2 * e2 + 1] = a1;
         }
     }
-    if (dmax > 0.49998f) return quant16_by_division(lo8, hi8, s);
+    if (differ) return quant16_by_division(lo8, hi8, s);
     uint4 out;
     out.x = __byte_perm(__byte_perm(b[0], b[1], 0x0040), __byte_perm(b[2], b[3], 0x0040), 0x5410);
     out.y = __byte_perm(__byte_perm(b[4], b[5], 0x0040), __byte_perm(b[6], b[7], 0x0040), 0x5410);
