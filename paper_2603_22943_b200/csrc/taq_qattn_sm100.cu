@@ -182,28 +182,17 @@ __device__ __noinline__ uint32_t build_weight_tiles_i8(unsigned char* smem, Misc
     return (uint32_t)s | (ph << 2) | (ok ? 0u : 8u);
 }
 
-// Sixteen codes rint(x / s), clamped to +-127, exactly as the stand-alone quantizer defines them (one IEEE division each,
-// then rintf): the rare path.
-__device__ __noinline__ uint4 quant16_by_division(uint4 lo8, uint4 hi8, float s) {
-    uint32_t w[4] = {0, 0, 0, 0};
-    const uint4 v[2] = {lo8, hi8};
-#pragma unroll
-    for (int u = 0; u < 2; ++u) {
-        const __half2* h = reinterpret_cast<const __half2*>(&v[u]);
-#pragma unroll
-        for (int e2 = 0; e2 < 4; ++e2) {
-            const float2 f = __half22float2(h[e2]);
-            const int a = (int)fminf(fmaxf(rintf(__fdiv_rn(f.x, s)), -127.f), 127.f), b = (int)fminf(fmaxf(rintf(__fdiv_rn(f.y, s)), -127.f), 127.f);
-            w[2 * u + (e2 >> 1)] |= ((uint32_t)(a & 0xFF) | ((uint32_t)(b & 0xFF) << 8)) << (16 * (e2 & 1));
-        }
-    }
-    return make_uint4(w[0], w[1], w[2], w[3]);
+// One code rint(x / s), clamped to +-127, exactly as the stand-alone quantizer defines it (one IEEE division, then rintf):
+// the rare path of quant16 below, one shared copy of the division.
+__device__ __noinline__ uint32_t code_by_division(float x, float s) {
+    return (uint32_t)(int)fminf(fmaxf(rintf(__fdiv_rn(x, s)), -127.f), 127.f);
 }
-// The same sixteen codes on the fast path.  fma(x, r, 1.5 * 2^23) leaves rint(x r) in the low byte.  The definition's
-// rounded quotient fl(x / s) and the product with the correctly rounded reciprocal both lie between x r_lo and x r_hi
-// (r two ulps down and up: each of them is off the exact quotient by at most one relative 2^-24), so when both ends
-// round to the same integer that integer is the definition's code; otherwise - about one chunk in 150 - the chunk is
-// redone by division.
+// Sixteen codes.  fma(x, r, 1.5 * 2^23) leaves rint(x r) in the low byte.  The definition's rounded quotient fl(x / s) and
+// the product with the correctly rounded reciprocal both lie between x r_lo and x r_hi (r two ulps down and up: each of
+// them is off the exact quotient by at most one relative 2^-24), so when both ends round to the same integer that
+// integer is the definition's code.  Otherwise the element is divided.  fp16 data makes that less rare than one would
+// think - a value that is exactly half of the row maximum sits exactly on a boundary - about 4 codes in 10000, so the
+// fix-up touches single elements, not the chunk.
 __device__ __forceinline__ uint4 quant16(uint4 lo8, uint4 hi8, float s, float rs) {
     const float r_lo = __uint_as_float(__float_as_uint(rs) - 2u), r_hi = __uint_as_float(__float_as_uint(rs) + 2u);
     const uint4 v[2] = {lo8, hi8};
@@ -216,13 +205,23 @@ __device__ __forceinline__ uint4 quant16(uint4 lo8, uint4 hi8, float s, float rs
         for (int e2 = 0; e2 < 4; ++e2) {
             const float2 f = __half22float2(h[e2]);
             const uint32_t a0 = __float_as_uint(fmaf(f.x, r_lo, 12582912.0f)), a1 = __float_as_uint(fmaf(f.y, r_lo, 12582912.0f));
-            const uint32_t c0 = __float_as_uint(fmaf(f.x, r_hi, 12582912.0f)), c1 = __float_as_uint(fmaf(f.y, r_hi, 12582912.0f));
-            differ |= (a0 ^ c0) | (a1 ^ c1);
+            differ |= (a0 ^ __float_as_uint(fmaf(f.x, r_hi, 12582912.0f))) | (a1 ^ __float_as_uint(fmaf(f.y, r_hi, 12582912.0f)));
             b[8 * u + 2 * e2] = a0;
             b[8 * u + 2 * e2 + 1] = a1;
         }
     }
-    if (differ) return quant16_by_division(lo8, hi8, s);
+    if (differ) {
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const __half2* h = reinterpret_cast<const __half2*>(&v[u]);
+#pragma unroll
+            for (int e2 = 0; e2 < 4; ++e2) {
+                const float2 f = __half22float2(h[e2]);
+                if (b[8 * u + 2 * e2] != __float_as_uint(fmaf(f.x, r_hi, 12582912.0f))) b[8 * u + 2 * e2] = code_by_division(f.x, s);
+                if (b[8 * u + 2 * e2 + 1] != __float_as_uint(fmaf(f.y, r_hi, 12582912.0f))) b[8 * u + 2 * e2 + 1] = code_by_division(f.y, s);
+            }
+        }
+    }
     uint4 out;
     out.x = __byte_perm(__byte_perm(b[0], b[1], 0x0040), __byte_perm(b[2], b[3], 0x0040), 0x5410);
     out.y = __byte_perm(__byte_perm(b[4], b[5], 0x0040), __byte_perm(b[6], b[7], 0x0040), 0x5410);

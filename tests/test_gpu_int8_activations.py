@@ -33,6 +33,9 @@ def test_quantize_rows_f16_is_bit_exact(rows, cols):
         x[3, 0] = 127
         x[4, :] = (r.integers(-252, 252, cols) * 0.25).astype(np.float16)       # scale 1/2 (absmax 63.5): quarter steps
         x[4, 0] = 63.5
+    if rows > 6:
+        x[5, :] = (r.integers(-40, 41, cols) * 2.0 ** -24).astype(np.float16)   # subnormal fp16 values: the scale is tiny, not zero
+        x[6, :] = np.clip(r.standard_normal(cols) * 3e4, -65504, 65504).astype(np.float16)   # near the top of the fp16 range
     codes, scales = tb.taq_quantize_rows_f16(dev(x))
     want_c, want_s = orc.quantize_rows(x.astype(np.float32), 127)
     assert np.array_equal(scales.cpu().numpy(), want_s)
