@@ -29,7 +29,7 @@ if ROOT not in sys.path:
 METRIC = "TAQ cross-attn queries/s per layer"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/ (bytes); a
 # kernel that changed since its capture is listed as None.
-TRAFFIC = {"layer": 5804544}     # profiles/layer_c320_config2.md: 5.80 MB read, 0 written (Y was still in L2 when the capture ended)
+TRAFFIC = {"layer": 5804288}     # profiles/layer_c320_config2.md: 5.80 MB read, 0 written (Y was still in L2 when the capture ended)
 UNIT = "queries/s"
 WORKLOAD = "config2: SD-1.5 64x64 cross-attn layer, B=2 N=4096 C=320 H=8 d=40 T=77 Dc=768, W4 g128, int8 Q/K/V rows, uint8 probs, fp16 trigger rows {4,5}"
 
