@@ -54,6 +54,7 @@ struct Bars {
     uint64_t w_full;
     uint64_t acc_full[2];
     uint64_t acc_free[2];
+    uint64_t part_full, part_got, peer_ready;   // K loop split over a CTA pair: hand-over of the second CTA's partial sums
     uint32_t tmem_base;
     volatile int abort_flag;
 };
@@ -84,7 +85,10 @@ __host__ __device__ inline Plan make_plan(int k_in, int bits, int group, int nst
 // I8: the integer-activation variant (the literal W/A reading of Table 1).  The A operand is the int8 codes of the
 // per-token-quantized activations, the B operand the int8 weight codes, the accumulators are exact int32; a K block is
 // 128 elements (one W4 scale group), and the row's activation scale multiplies the folded sum at the end.
-template <int BN, bool I8>
+// SPLIT: for launches with few tiles and a long K loop, two CTAs (a cluster of two along x) share one output tile: the first
+// takes the lower half of the scale groups, the second the upper half; the second hands its folded fp32 partial sums to
+// the first through a bulk copy between the two shared memories, and the first adds them and runs the epilogue.
+template <int BN, bool I8, bool SPLIT>
 __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w, const LinearArgs a, const int nstage) {
     using TL = Tile<BN>;
     constexpr int BKE = I8 ? 2 * BK : BK;             // elements per K block
@@ -97,13 +101,18 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int z = blockIdx.z;
-    const int row0 = blockIdx.x * BM;
+    const int rank = SPLIT ? (int)(blockIdx.x & 1) : 0;
+    const int row0 = (SPLIT ? (int)(blockIdx.x >> 1) : (int)blockIdx.x) * BM;
     const int col0 = blockIdx.y * BN;
     const int n_kb = (a.k_in + BKE - 1) / BKE;          // (int8: the last block may be ragged; TMA and the expansion zero-fill)
     const uint8_t* blob = (const uint8_t*)(a.reqs ? (a.which == 0 ? a.reqs[z].Wq : a.reqs[z].Wout) : a.w);
     const WeightLayout L = weight_layout(a.n_out, a.k_in, a.bits, a.group);
     const int n_groups = L.n_groups;
     const int kb_per_group = n_groups == 1 ? n_kb : L.group_len / BKE;   // k-blocks in a full group (the last group may be shorter)
+    // this CTA's share of the K loop: all of it, or one half of the scale groups
+    const int g_begin = SPLIT && rank ? n_groups / 2 : 0, g_end = SPLIT && !rank ? n_groups / 2 : n_groups;
+    const int kb_begin = g_begin * kb_per_group, kb_stop = min(n_kb, g_end * kb_per_group);
+    constexpr uint32_t PART_BYTES = (uint32_t)BN * 128u * 4u;        // fp32 partial sums of the tile
 
     TAQ_PROF_INIT
     if (tid == 0) { TAQ_PROF(0); TAQ_GPROF(30); }
@@ -118,8 +127,12 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
             ptx::mbar_init(&bars->acc_full[i], 1);
             ptx::mbar_init(&bars->acc_free[i], NWORK / 32);
         }
+        ptx::mbar_init(&bars->part_full, 1);
+        ptx::mbar_init(&bars->part_got, 1);
+        ptx::mbar_init(&bars->peer_ready, 1);
         bars->abort_flag = 0;
         ptx::mbar_fence_init();
+        if (SPLIT && rank == 0) ptx::mbar_arrive_expect_tx(&bars->part_full, PART_BYTES);
         ptx::tma_prefetch_desc(&tmap_x);
     }
     if (warp == 1) ptx::tmem_alloc(&bars->tmem_base, TMEM_COLS);
@@ -128,6 +141,7 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = bars->tmem_base;
     ptx::pdl_trigger();
+    if (SPLIT) ptx::cluster_sync_all();                    // the partner's barriers exist before anything arrives on them
 
     if (warp == 0) {
         // ---------------- producer: packed weights once, then activation tiles ----------------
@@ -141,13 +155,13 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
             TAQ_PROF(1); TAQ_GPROF(28);
             int issued = 0, s = 0;
             uint32_t ph = 0;                               // parity of the ring pass
-            for (int kb = 0; kb < n_kb; ++kb) {
-                if (kb >= nstage && !ptx::mbar_wait(&bars->empty[s], ph ^ 1)) { raise_status(a.status, TAQ_ERR_TIMEOUT); bars->abort_flag = 1; }
+            for (int kb = kb_begin; kb < kb_stop; ++kb) {
+                if (kb - kb_begin >= nstage && !ptx::mbar_wait(&bars->empty[s], ph ^ 1)) { raise_status(a.status, TAQ_ERR_TIMEOUT); bars->abort_flag = 1; }
                 if (bars->abort_flag) break;
                 ptx::mbar_arrive_expect_tx(&bars->full_a[s], A_TILE_BYTES + (a.w_direct ? BN * 128 : 0));
                 ptx::tma_load_3d(smem + s * TL::STAGE_BYTES, &tmap_x, &bars->full_a[s], kb * BKE, row0, z);
                 if (a.w_direct) ptx::tma_load_3d(smem + s * TL::STAGE_BYTES + A_TILE_BYTES, &tmap_w, &bars->full_a[s], kb * BKE, col0, 0);
-                issued = kb + 1;
+                issued = kb - kb_begin + 1;
                 if (++s == nstage) { s = 0; ph ^= 1; }
             }
             if (bars->abort_flag) {   // give copies that are still in flight a bounded chance to land before the CTA exits
@@ -164,13 +178,14 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
         constexpr uint32_t idesc = I8 ? ptx::idesc_i8_m128(BN) : ptx::idesc_f16_m128(BN);
         constexpr uint32_t HI = ptx::kDescHiSw128;
         const uint32_t lo0 = ptx::desc_lo(ptx::smem_u32(smem));
-        int s = 0, kb = 0;
+        int s = 0, kb = kb_begin;
         uint32_t ph = 0;
         bool ok = true;
-        for (int g = 0; g < n_groups && ok; ++g) {
-            const int buf = g & 1;
-            if (g >= 2) {                                   // the workers have emptied this accumulator
-                if (!wait(&bars->acc_free[buf], ((g >> 1) - 1) & 1)) { ok = false; break; }
+        for (int g = g_begin; g < g_end && ok; ++g) {
+            const int gl = g - g_begin;
+            const int buf = gl & 1;
+            if (gl >= 2) {                                  // the workers have emptied this accumulator
+                if (!wait(&bars->acc_free[buf], ((gl >> 1) - 1) & 1)) { ok = false; break; }
                 ptx::tc_fence_after_sync();
             }
             const int kb_end = min(n_kb, kb + kb_per_group);
@@ -225,8 +240,8 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
 
         // y += scale[g] * accumulator of group g (this thread's HC columns of its row)
         auto fold_group = [&](int g) -> bool {
-            const int buf = g & 1;
-            if (!ptx::mbar_wait(&bars->acc_full[buf], (g >> 1) & 1) || bars->abort_flag) return false;
+            const int buf = (g - g_begin) & 1;
+            if (!ptx::mbar_wait(&bars->acc_full[buf], ((g - g_begin) >> 1) & 1) || bars->abort_flag) return false;
             ptx::tc_fence_after_sync();
             const float* sg = scales_t + g * BN + cb;
 #pragma unroll
@@ -260,12 +275,12 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
         };
 
         // expand the weight tiles of group g's k-blocks
-        int s = 0, kb = 0;
+        int s = 0, kb = kb_begin;
         uint32_t ph = 0;
         auto build_group = [&](int g) -> bool {
             const int kb_end = min(n_kb, kb + kb_per_group);
             for (; kb < kb_end; ++kb) {
-                if (kb >= nstage && !ptx::mbar_wait(&bars->empty[s], ph ^ 1)) return false;
+                if (kb - kb_begin >= nstage && !ptx::mbar_wait(&bars->empty[s], ph ^ 1)) return false;
                 if (bars->abort_flag) return false;
                 unsigned char* b_tile = smem + s * TL::STAGE_BYTES + A_TILE_BYTES;
                 // 16-byte chunks of the fp16 tile: 8 per weight row; this thread owns chunk c of rows n0, n0 + 32, ...
@@ -321,16 +336,48 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
             return true;
         };
 
-        for (int g = 0; g < n_groups && ok; ++g) {
+        for (int g = g_begin; g < g_end && ok; ++g) {
             ok = a.w_direct ? true : build_group(g);
-            if (ok && g >= 1) ok = fold_group(g - 1);
+            if (ok && g > g_begin) ok = fold_group(g - 1);
         }
-        if (ok) ok = fold_group(n_groups - 1);
+        if (ok) ok = fold_group(g_end - 1);
         if (!ok) { raise_status(a.status, TAQ_ERR_TIMEOUT); bars->abort_flag = 1; }
         asm volatile("bar.sync 1, 256;" ::: "memory");       // every worker gets here; the decision below is uniform
         ok = !bars->abort_flag;
         ptx::pdl_wait();                                     // (already satisfied: the activations have arrived) orders the stores below
         if (wt == 0) TAQ_PROF(7);
+        if (SPLIT) {
+            // All of this CTA's MMAs are complete (every group was folded), so its ring is free: it holds the partial sums
+            // in transit, 128 x BN fp32, each thread's piece at the same place in both CTAs.
+            float* piece = reinterpret_cast<float*>(smem) + (size_t)(half * 128 + r) * HC;
+            if (rank == 1) {
+#pragma unroll
+                for (int c = 0; c < HC; c += 4) *reinterpret_cast<float4*>(piece + c) = make_float4(y[c], y[c + 1], y[c + 2], y[c + 3]);
+                ptx::fence_proxy_async_smem();
+                asm volatile("bar.sync 1, 256;" ::: "memory");
+                if (wt == 0) {
+                    bool sent = ptx::mbar_wait(&bars->peer_ready, 0) && !bars->abort_flag;       // the first CTA's ring is free, too
+                    if (sent) {
+                        ptx::bulk_copy_to_cta(ptx::map_to_cta(ptx::smem_u32(smem), 0), smem, PART_BYTES, ptx::map_to_cta(ptx::smem_u32(&bars->part_full), 0));
+                        sent = ptx::mbar_wait(&bars->part_got, 0);                               // this CTA's shared memory is the source: stay until it was read
+                    }
+                    if (!sent) { raise_status(a.status, TAQ_ERR_TIMEOUT); bars->abort_flag = 1; }
+                }
+                ok = false;                                  // nothing to store from this CTA
+            } else {
+                if (wt == 0) ptx::mbar_arrive_cluster_relaxed(ptx::map_to_cta(ptx::smem_u32(&bars->peer_ready), 1));
+                if (!ptx::mbar_wait(&bars->part_full, 0)) { raise_status(a.status, TAQ_ERR_TIMEOUT); bars->abort_flag = 1; ok = false; }
+                if (ok) {
+#pragma unroll
+                    for (int c = 0; c < HC; c += 4) {
+                        const float4 p4 = *reinterpret_cast<const float4*>(piece + c);
+                        y[c] += p4.x; y[c + 1] += p4.y; y[c + 2] += p4.z; y[c + 3] += p4.w;
+                    }
+                }
+                asm volatile("bar.sync 1, 256;" ::: "memory");   // every thread has read its piece (the epilogue stages output there)
+                if (wt == 0) ptx::mbar_arrive_cluster_relaxed(ptx::map_to_cta(ptx::smem_u32(&bars->part_got), 1));
+            }
+        }
         if (I8 && ok) {                                      // x~ = code * s_x: the row's activation scale
             const float sx = row < a.rows ? a.x_scales[(size_t)z * a.rows + row] : 0.f;
 #pragma unroll
@@ -535,9 +582,17 @@ int nstage_for(const LinearArgs& a, int bn) {
 
 template <int BN>
 cudaError_t launch_bn(const CUtensorMap& tmap, EncodeTiledFn enc, LinearArgs a, int n_z, cudaStream_t stream) {
-    static bool configured[2] = {false, false};
+    static bool configured[4] = {false, false, false, false};
     const bool i8 = a.xq != nullptr;
-    void (*kern)(const CUtensorMap, const CUtensorMap, const LinearArgs, const int) = i8 ? linear_sm100_kernel<BN, true> : linear_sm100_kernel<BN, false>;
+    const int ns = pick_nstage<BN>(a);
+    const WeightLayout Lw = weight_layout(a.n_out, a.k_in, a.bits, a.group);
+    const int bke = i8 ? 2 * BK : BK;
+    const long long tiles = ((a.rows + BM - 1) / BM) * (a.n_out / BN) * (long long)n_z;
+    // few tiles and a long K loop: two CTAs per tile, each with half of the scale groups
+    const bool split = Lw.n_groups >= 2 && tiles <= 74 && (a.k_in + bke - 1) / bke >= 6 && (long long)ns * Tile<BN>::STAGE_BYTES >= (long long)BN * 512;
+    void (*kern)(const CUtensorMap, const CUtensorMap, const LinearArgs, const int) =
+        split ? (i8 ? linear_sm100_kernel<BN, true, true> : linear_sm100_kernel<BN, false, true>)
+              : (i8 ? linear_sm100_kernel<BN, true, false> : linear_sm100_kernel<BN, false, false>);
     a.w_direct = i8 && a.bits == 8 && !a.reqs;
     CUtensorMap tmap_w = tmap;                        // (unused unless w_direct)
     if (a.w_direct) {                                 // the codes section of the blob as an int8 matrix [n_out][k_in]
@@ -549,14 +604,14 @@ cudaError_t launch_bn(const CUtensorMap& tmap, EncodeTiledFn enc, LinearArgs a, 
                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
     }
-    if (!configured[i8]) {
+    if (!configured[i8 + 2 * split]) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT);
         if (e != cudaSuccess) return e;
-        configured[i8] = true;
+        configured[i8 + 2 * split] = true;
     }
-    const int ns = pick_nstage<BN>(a);
     const Plan P = make_plan<BN>(a.k_in, a.bits, a.group, ns, a.w_direct != 0);
-    dim3 grid((unsigned)((a.rows + BM - 1) / BM), a.n_out / BN, n_z);
+    dim3 grid((unsigned)((a.rows + BM - 1) / BM) * (split ? 2u : 1u), a.n_out / BN, n_z);
+    if (split) return launch_pdl_cluster(kern, grid, dim3(2, 1, 1), dim3(NTHREADS), (size_t)P.total, stream, tmap, tmap_w, a, ns);
     return launch_pdl(kern, grid, dim3(NTHREADS), (size_t)P.total, stream, tmap, tmap_w, a, ns);
 }
 
