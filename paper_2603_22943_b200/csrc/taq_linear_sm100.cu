@@ -589,7 +589,7 @@ cudaError_t launch_bn(const CUtensorMap& tmap, EncodeTiledFn enc, LinearArgs a, 
     const int bke = i8 ? 2 * BK : BK;
     const long long tiles = ((a.rows + BM - 1) / BM) * (a.n_out / BN) * (long long)n_z;
     // few tiles and a long K loop: two CTAs per tile, each with half of the scale groups
-    const bool split = Lw.n_groups >= 2 && tiles <= 74 && (a.k_in + bke - 1) / bke >= 6 && (long long)ns * Tile<BN>::STAGE_BYTES >= (long long)BN * 512;
+    const bool split = Lw.n_groups >= 2 && tiles <= 74 * Tile<BN>::CTAS_PER_SM && (a.k_in + bke - 1) / bke >= 6 && (long long)ns * Tile<BN>::STAGE_BYTES >= (long long)BN * 512;
     void (*kern)(const CUtensorMap, const CUtensorMap, const LinearArgs, const int) =
         split ? (i8 ? linear_sm100_kernel<BN, true, true> : linear_sm100_kernel<BN, false, true>)
               : (i8 ? linear_sm100_kernel<BN, true, false> : linear_sm100_kernel<BN, false, false>);
