@@ -481,32 +481,12 @@ def main():
     for i in range(3):
         e2e_step(i)
     barrier()
-    # The pipelined steps are recorded once as a CUDA graph (copy nodes on the two copy streams, the kernel on the third) and
-    # replayed: the host then issues one launch per E2E_CHUNK steps instead of a dozen calls per step, which at 16 us of
-    # kernel time per step would otherwise bound the rate.  The pipeline drains at the end of each replay.
-    E2E_CHUNK = 25
     ev_in.clear(); ev_cmp.clear(); ev_out.clear()
-    g_e2e = torch.cuda.CUDAGraph()
-    with torch.cuda.graph(g_e2e, stream=s_cmp):
-        fork = torch.cuda.Event()
-        fork.record(s_cmp)
-        s_in.wait_event(fork)
-        s_out.wait_event(fork)
-        for i in range(E2E_CHUNK):
-            e2e_step(i)
-        for side in (s_in, s_out):
-            join = torch.cuda.Event()
-            join.record(side)
-            s_cmp.wait_event(join)
-    e_replays = max(1, e_steps // E2E_CHUNK)
-    e_steps = e_replays * E2E_CHUNK
-    g_e2e.replay()
-    barrier()
     f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    f0.record()
-    for _ in range(e_replays):
-        g_e2e.replay()
-    f1.record()
+    f0.record(s_in)
+    for i in range(e_steps):
+        e2e_step(i)
+    f1.record(s_out)
     barrier()
     e2e_ms = f0.elapsed_time(f1)
     tb.taq_poll_device_status()
@@ -560,8 +540,7 @@ def main():
                        "l2_policy": f"inputs larger than L2: ring of {n_sets} buffer sets ({n_sets * set_bytes / 1e6:.0f} MB of activations, L2 {l2 / 1e6:.0f} MB)",
                        "replicas": world},
             "clocks": clocks,
-            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": M * C_ * 2, "d2h_bytes_per_step": M * C_ * 2, "steps": e_steps,
-                    "launch": f"three streams (upload, kernel, download) recorded as one CUDA graph per {E2E_CHUNK} steps"},
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": M * C_ * 2, "d2h_bytes_per_step": M * C_ * 2, "steps": e_steps},
             "gpu_launches": args.steps,
             "roofline": roofline}
     if not args.no_cpu_baseline:

@@ -54,7 +54,7 @@ struct Bars {
     uint64_t w_full;
     uint64_t acc_full[2];
     uint64_t acc_free[2];
-    uint64_t part_full, part_got, peer_ready;   // K loop split over a CTA pair: hand-over of the second CTA's partial sums
+    uint64_t part_full[8], part_got, peer_ready;   // K loop split over a CTA pair: hand-over of the second CTA's partial sums
     uint32_t tmem_base;
     volatile int abort_flag;
 };
@@ -112,7 +112,7 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
     // this CTA's share of the K loop: all of it, or one half of the scale groups
     const int g_begin = SPLIT && rank ? n_groups / 2 : 0, g_end = SPLIT && !rank ? n_groups / 2 : n_groups;
     const int kb_begin = g_begin * kb_per_group, kb_stop = min(n_kb, g_end * kb_per_group);
-    constexpr uint32_t PART_BYTES = (uint32_t)BN * 128u * 4u;        // fp32 partial sums of the tile
+    constexpr uint32_t PART_ROW = (uint32_t)BN * 2u + 16u;           // a thread's fp32 partial sums (BN / 2 columns), padded against bank conflicts
 
     TAQ_PROF_INIT
     if (tid == 0) { TAQ_PROF(0); TAQ_GPROF(30); }
@@ -127,12 +127,13 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
             ptx::mbar_init(&bars->acc_full[i], 1);
             ptx::mbar_init(&bars->acc_free[i], NWORK / 32);
         }
-        ptx::mbar_init(&bars->part_full, 1);
-        ptx::mbar_init(&bars->part_got, 1);
+        for (int i = 0; i < 8; ++i) ptx::mbar_init(&bars->part_full[i], 1);
+        ptx::mbar_init(&bars->part_got, NWORK / 32);
         ptx::mbar_init(&bars->peer_ready, 1);
         bars->abort_flag = 0;
         ptx::mbar_fence_init();
-        if (SPLIT && rank == 0) ptx::mbar_arrive_expect_tx(&bars->part_full, PART_BYTES);
+        if (SPLIT && rank == 0)
+            for (int i = 0; i < 8; ++i) ptx::mbar_arrive_expect_tx(&bars->part_full[i], 32u * PART_ROW);
         ptx::tma_prefetch_desc(&tmap_x);
     }
     if (warp == 1) ptx::tmem_alloc(&bars->tmem_base, TMEM_COLS);
@@ -348,25 +349,29 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
         if (wt == 0) TAQ_PROF(7);
         if (SPLIT) {
             // All of this CTA's MMAs are complete (every group was folded), so its ring is free: it holds the partial sums
-            // in transit, 128 x BN fp32, each thread's piece at the same place in both CTAs.
-            float* piece = reinterpret_cast<float*>(smem) + (size_t)(half * 128 + r) * HC;
+            // in transit, each thread's piece at the same place in both CTAs.  Every worker warp hands its 32 rows over by
+            // itself (one bulk copy, one barrier per warp), so the copies overlap the staging of the other warps.
+            const int ww = wt >> 5, wl = wt & 31;
+            unsigned char* warp_part = smem + (size_t)ww * 32 * PART_ROW;
+            float* piece = reinterpret_cast<float*>(warp_part + (size_t)wl * PART_ROW);
             if (rank == 1) {
 #pragma unroll
                 for (int c = 0; c < HC; c += 4) *reinterpret_cast<float4*>(piece + c) = make_float4(y[c], y[c + 1], y[c + 2], y[c + 3]);
                 ptx::fence_proxy_async_smem();
-                asm volatile("bar.sync 1, 256;" ::: "memory");
-                if (wt == 0) {
-                    bool sent = ptx::mbar_wait(&bars->peer_ready, 0) && !bars->abort_flag;       // the first CTA's ring is free, too
-                    if (sent) {
-                        ptx::bulk_copy_to_cta(ptx::map_to_cta(ptx::smem_u32(smem), 0), smem, PART_BYTES, ptx::map_to_cta(ptx::smem_u32(&bars->part_full), 0));
-                        sent = ptx::mbar_wait(&bars->part_got, 0);                               // this CTA's shared memory is the source: stay until it was read
-                    }
-                    if (!sent) { raise_status(a.status, TAQ_ERR_TIMEOUT); bars->abort_flag = 1; }
+                __syncwarp();
+                if (wl == 0) {
+                    if (ww == 0) TAQ_PROF(11);
+                    const bool go = ptx::mbar_wait(&bars->peer_ready, 0) && !bars->abort_flag;   // the first CTA's ring is free, too
+                    if (ww == 0) TAQ_PROF(12);
+                    if (go) ptx::bulk_copy_to_cta(ptx::map_to_cta(ptx::smem_u32(warp_part), 0), warp_part, 32u * PART_ROW, ptx::map_to_cta(ptx::smem_u32(&bars->part_full[ww]), 0));
+                    else { raise_status(a.status, TAQ_ERR_TIMEOUT); bars->abort_flag = 1; }
                 }
+                // this CTA's shared memory is the source: stay until every warp of the first CTA has read its piece
+                if (wt == 0 && !ptx::mbar_wait(&bars->part_got, 0)) { raise_status(a.status, TAQ_ERR_TIMEOUT); bars->abort_flag = 1; }
                 ok = false;                                  // nothing to store from this CTA
             } else {
                 if (wt == 0) ptx::mbar_arrive_cluster_relaxed(ptx::map_to_cta(ptx::smem_u32(&bars->peer_ready), 1));
-                if (!ptx::mbar_wait(&bars->part_full, 0)) { raise_status(a.status, TAQ_ERR_TIMEOUT); bars->abort_flag = 1; ok = false; }
+                if (!ptx::mbar_wait(&bars->part_full[ww], 0)) { raise_status(a.status, TAQ_ERR_TIMEOUT); bars->abort_flag = 1; ok = false; }
                 if (ok) {
 #pragma unroll
                     for (int c = 0; c < HC; c += 4) {
@@ -374,9 +379,12 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
                         y[c] += p4.x; y[c + 1] += p4.y; y[c + 2] += p4.z; y[c + 3] += p4.w;
                     }
                 }
+                __syncwarp();
+                if (wl == 0) ptx::mbar_arrive_cluster_relaxed(ptx::map_to_cta(ptx::smem_u32(&bars->part_got), 1));
                 asm volatile("bar.sync 1, 256;" ::: "memory");   // every thread has read its piece (the epilogue stages output there)
-                if (wt == 0) ptx::mbar_arrive_cluster_relaxed(ptx::map_to_cta(ptx::smem_u32(&bars->part_got), 1));
+                ok = !bars->abort_flag;
             }
+            if (wt == 0) TAQ_PROF(10);
         }
         if (I8 && ok) {                                      // x~ = code * s_x: the row's activation scale
             const float sx = row < a.rows ? a.x_scales[(size_t)z * a.rows + row] : 0.f;
@@ -589,7 +597,7 @@ cudaError_t launch_bn(const CUtensorMap& tmap, EncodeTiledFn enc, LinearArgs a, 
     const int bke = i8 ? 2 * BK : BK;
     const long long tiles = ((a.rows + BM - 1) / BM) * (a.n_out / BN) * (long long)n_z;
     // few tiles and a long K loop: two CTAs per tile, each with half of the scale groups
-    const bool split = Lw.n_groups >= 2 && tiles <= 74 * Tile<BN>::CTAS_PER_SM && (a.k_in + bke - 1) / bke >= 6 && (long long)ns * Tile<BN>::STAGE_BYTES >= (long long)BN * 512;
+    const bool split = Lw.n_groups >= 2 && tiles <= 74 * Tile<BN>::CTAS_PER_SM && (a.k_in + bke - 1) / bke >= 6 && (long long)ns * Tile<BN>::STAGE_BYTES >= 256LL * (BN * 2 + 16);
     void (*kern)(const CUtensorMap, const CUtensorMap, const LinearArgs, const int) =
         split ? (i8 ? linear_sm100_kernel<BN, true, true> : linear_sm100_kernel<BN, false, true>)
               : (i8 ? linear_sm100_kernel<BN, true, false> : linear_sm100_kernel<BN, false, false>);
