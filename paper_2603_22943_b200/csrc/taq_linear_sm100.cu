@@ -280,47 +280,6 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
         uint32_t ph = 0;
         auto build_group = [&](int g) -> bool {
             const int kb_end = min(n_kb, kb + kb_per_group);
-            if (!I8) {
-                // fp16 tiles two at a time: the code loads, expansions and stores of both tiles overlap, and one proxy fence
-                // covers both (a worker's chain of latencies per tile, not its instruction count, bounds the K loop)
-                constexpr int NCH = (BN * 8 + NWORK - 1) / NWORK;
-                const int n0 = wt >> 3, c = wt & 7;
-                for (; kb + 1 < kb_end; kb += 2) {
-                    const int s2 = s + 1 == nstage ? 0 : s + 1;
-                    const uint32_t ph2 = s + 1 == nstage ? ph ^ 1 : ph;
-                    if (kb - kb_begin >= nstage && !ptx::mbar_wait(&bars->empty[s], ph ^ 1)) return false;
-                    if (kb + 1 - kb_begin >= nstage && !ptx::mbar_wait(&bars->empty[s2], ph2 ^ 1)) return false;
-                    if (bars->abort_flag) return false;
-                    uint2 pw[2][NCH];
-#pragma unroll
-                    for (int j = 0; j < 2; ++j)
-#pragma unroll
-                        for (int i = 0; i < NCH; ++i) {
-                            const int n = n0 + (NWORK / 8) * i;
-                            pw[j][i] = make_uint2(0, 0);
-                            if ((BN * 8) % NWORK == 0 || n < BN) {
-                                if (a.bits == 4) pw[j][i].x = *reinterpret_cast<const uint32_t*>(raw + n * row_bytes + (kb + j) * (BK / 2) + c * 4);
-                                else pw[j][i] = *reinterpret_cast<const uint2*>(raw + n * row_bytes + (kb + j) * BK + c * 8);
-                            }
-                        }
-#pragma unroll
-                    for (int j = 0; j < 2; ++j) {
-                        unsigned char* b_tile = smem + (j ? s2 : s) * TL::STAGE_BYTES + A_TILE_BYTES;
-#pragma unroll
-                        for (int i = 0; i < NCH; ++i) {
-                            const int n = n0 + (NWORK / 8) * i;
-                            if ((BN * 8) % NWORK == 0 || n < BN)
-                                *reinterpret_cast<uint4*>(b_tile + ptx::sw128_offset(n, c)) = a.bits == 4 ? codes_w4_to_half(pw[j][i].x) : codes_w8_to_half(pw[j][i]);
-                        }
-                    }
-                    ptx::fence_proxy_async_smem();        // make the generic-proxy writes visible to the tensor core
-                    __syncwarp();
-                    if (lane == 0) { ptx::mbar_arrive(&bars->full_b[s]); ptx::mbar_arrive(&bars->full_b[s2]); }
-                    if (wt == 0 && kb + 1 < 20) { TAQ_PROF(60 + kb); TAQ_PROF(61 + kb); }
-                    s = s2; ph = ph2;
-                    if (++s == nstage) { s = 0; ph ^= 1; }
-                }
-            }
             for (; kb < kb_end; ++kb) {
                 if (kb - kb_begin >= nstage && !ptx::mbar_wait(&bars->empty[s], ph ^ 1)) return false;
                 if (bars->abort_flag) return false;
