@@ -54,7 +54,7 @@ struct Bars {
     uint64_t w_full;
     uint64_t acc_full[2];
     uint64_t acc_free[2];
-    uint64_t part_full[8], part_got, peer_ready;   // K loop split over a CTA pair: hand-over of the second CTA's partial sums
+    uint64_t part_full[8], part_got[8], peer_ready;   // K loop split over a CTA pair: hand-over of the second CTA's partial sums
     uint32_t tmem_base;
     volatile int abort_flag;
 };
@@ -127,13 +127,13 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
             ptx::mbar_init(&bars->acc_full[i], 1);
             ptx::mbar_init(&bars->acc_free[i], NWORK / 32);
         }
-        for (int i = 0; i < 8; ++i) ptx::mbar_init(&bars->part_full[i], 1);
-        ptx::mbar_init(&bars->part_got, NWORK / 32);
+        for (int i = 0; i < 8; ++i) { ptx::mbar_init(&bars->part_full[i], 1); ptx::mbar_init(&bars->part_got[i], 1); }
         ptx::mbar_init(&bars->peer_ready, 1);
         bars->abort_flag = 0;
         ptx::mbar_fence_init();
-        if (SPLIT && rank == 0)
-            for (int i = 0; i < 8; ++i) ptx::mbar_arrive_expect_tx(&bars->part_full[i], 32u * PART_ROW);
+        if (SPLIT)                                          // the worker warps whose rows this CTA finishes receive a piece each
+            for (int i = 0; i < 8; ++i)
+                if (((i & 3) >> 1) == rank) ptx::mbar_arrive_expect_tx(&bars->part_full[i], 32u * PART_ROW);
         ptx::tma_prefetch_desc(&tmap_x);
     }
     if (warp == 1) ptx::tmem_alloc(&bars->tmem_base, TMEM_COLS);
@@ -219,7 +219,7 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
         const int q = warp & 3;                           // TMEM lane quarter this warp may read
         const int half = (warp - 2) >> 2;                 // which half of the tile's columns this thread owns
         const int r = q * 32 + lane;
-        const long long row = (long long)row0 + r;
+        long long row = (long long)row0 + r;
         const int cb = half * HC;                         // first owned column inside the tile
         const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + cb;
         const unsigned char* raw = smem + P.off_raw;
@@ -349,30 +349,38 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
         if (wt == 0) TAQ_PROF(7);
         if (SPLIT) {
             // All of this CTA's MMAs are complete (every group was folded), so its ring is free: it holds the partial sums
-            // in transit, each thread's piece at the same place in both CTAs.  Every worker warp hands its 32 rows over by
-            // itself (one bulk copy, one barrier per warp), so the copies overlap the staging of the other warps.
+            // in transit, each thread's piece at the same place in both CTAs.  The first CTA finishes rows 0..63 of the
+            // tile, the second rows 64..127: a worker warp either hands its 32 rows over (one bulk copy between the shared
+            // memories, one barrier per warp) or receives the partner's piece and adds it, so both directions of the
+            // exchange run at once and each CTA stores half of the tile.
             const int ww = wt >> 5, wl = wt & 31;
+            const uint32_t peer = (uint32_t)rank ^ 1u;
+            const bool keep = ((ww & 3) >> 1) == rank;
             unsigned char* warp_part = smem + (size_t)ww * 32 * PART_ROW;
             float* piece = reinterpret_cast<float*>(warp_part + (size_t)wl * PART_ROW);
-            if (rank == 1) {
+            if (wt == 0) ptx::mbar_arrive_cluster_relaxed(ptx::map_to_cta(ptx::smem_u32(&bars->peer_ready), peer));
+            if (!keep) {
 #pragma unroll
                 for (int c = 0; c < HC; c += 4) *reinterpret_cast<float4*>(piece + c) = make_float4(y[c], y[c + 1], y[c + 2], y[c + 3]);
                 ptx::fence_proxy_async_smem();
                 __syncwarp();
                 if (wl == 0) {
-                    if (ww == 0) TAQ_PROF(11);
-                    const bool go = ptx::mbar_wait(&bars->peer_ready, 0) && !bars->abort_flag;   // the first CTA's ring is free, too
-                    if (ww == 0) TAQ_PROF(12);
-                    if (go) ptx::bulk_copy_to_cta(ptx::map_to_cta(ptx::smem_u32(warp_part), 0), warp_part, 32u * PART_ROW, ptx::map_to_cta(ptx::smem_u32(&bars->part_full[ww]), 0));
-                    else { raise_status(a.status, TAQ_ERR_TIMEOUT); bars->abort_flag = 1; }
+                    if (ww == 2) TAQ_PROF(11);
+                    bool go = ptx::mbar_wait(&bars->peer_ready, 0) && !bars->abort_flag;         // the partner's ring is free, too
+                    if (ww == 2) TAQ_PROF(12);
+                    if (go) {
+                        ptx::bulk_copy_to_cta(ptx::map_to_cta(ptx::smem_u32(warp_part), peer), warp_part, 32u * PART_ROW,
+                                              ptx::map_to_cta(ptx::smem_u32(&bars->part_full[ww]), peer));
+                        go = ptx::mbar_wait(&bars->part_got[ww], 0);     // this CTA's shared memory is the source: stay until it was read
+                    }
+                    if (!go) { raise_status(a.status, TAQ_ERR_TIMEOUT); bars->abort_flag = 1; }
                 }
-                // this CTA's shared memory is the source: stay until every warp of the first CTA has read its piece
-                if (wt == 0 && !ptx::mbar_wait(&bars->part_got, 0)) { raise_status(a.status, TAQ_ERR_TIMEOUT); bars->abort_flag = 1; }
-                ok = false;                                  // nothing to store from this CTA
+                row = a.rows;                                // these rows are stored by the partner
             } else {
-                if (wt == 0) ptx::mbar_arrive_cluster_relaxed(ptx::map_to_cta(ptx::smem_u32(&bars->peer_ready), 1));
-                if (!ptx::mbar_wait(&bars->part_full[ww], 0)) { raise_status(a.status, TAQ_ERR_TIMEOUT); bars->abort_flag = 1; ok = false; }
-                if (ok) {
+                if (!ptx::mbar_wait(&bars->part_full[ww], 0)) {
+                    raise_status(a.status, TAQ_ERR_TIMEOUT);
+                    bars->abort_flag = 1;
+                } else {
 #pragma unroll
                     for (int c = 0; c < HC; c += 4) {
                         const float4 p4 = *reinterpret_cast<const float4*>(piece + c);
@@ -380,10 +388,10 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
                     }
                 }
                 __syncwarp();
-                if (wl == 0) ptx::mbar_arrive_cluster_relaxed(ptx::map_to_cta(ptx::smem_u32(&bars->part_got), 1));
-                asm volatile("bar.sync 1, 256;" ::: "memory");   // every thread has read its piece (the epilogue stages output there)
-                ok = !bars->abort_flag;
+                if (wl == 0) ptx::mbar_arrive_cluster_relaxed(ptx::map_to_cta(ptx::smem_u32(&bars->part_got[ww]), peer));
             }
+            asm volatile("bar.sync 1, 256;" ::: "memory");   // pieces read, outgoing copies done: the epilogue stages output there
+            ok = !bars->abort_flag;
             if (wt == 0) TAQ_PROF(10);
         }
         if (I8 && ok) {                                      // x~ = code * s_x: the row's activation scale
