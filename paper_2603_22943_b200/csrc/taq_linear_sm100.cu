@@ -109,9 +109,12 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
     const WeightLayout L = weight_layout(a.n_out, a.k_in, a.bits, a.group);
     const int n_groups = L.n_groups;
     const int kb_per_group = n_groups == 1 ? n_kb : L.group_len / BKE;   // k-blocks in a full group (the last group may be shorter)
-    // this CTA's share of the K loop: all of it, or one half of the scale groups
-    const int g_begin = SPLIT && rank ? n_groups / 2 : 0, g_end = SPLIT && !rank ? n_groups / 2 : n_groups;
-    const int kb_begin = g_begin * kb_per_group, kb_stop = min(n_kb, g_end * kb_per_group);
+    // this CTA's share of the K loop: all of it, one half of the scale groups, or (one scale per output channel) one half
+    // of the k-blocks of the only group
+    const bool split_kb = SPLIT && n_groups == 1;
+    const int g_begin = SPLIT && !split_kb && rank ? n_groups / 2 : 0, g_end = SPLIT && !split_kb && !rank ? n_groups / 2 : n_groups;
+    const int kb_begin = split_kb ? (rank ? n_kb / 2 : 0) : g_begin * kb_per_group;
+    const int kb_stop = split_kb ? (rank ? n_kb : n_kb / 2) : min(n_kb, g_end * kb_per_group);
     constexpr uint32_t PART_ROW = (uint32_t)BN * 2u + 16u;           // a thread's fp32 partial sums (BN / 2 columns), padded against bank conflicts
 
     TAQ_PROF_INIT
@@ -189,7 +192,7 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
                 if (!wait(&bars->acc_free[buf], ((gl >> 1) - 1) & 1)) { ok = false; break; }
                 ptx::tc_fence_after_sync();
             }
-            const int kb_end = min(n_kb, kb + kb_per_group);
+            const int kb_end = min(kb_stop, kb + kb_per_group);
             for (bool first = true; kb < kb_end && ok; ++kb) {
                 if (!wait(&bars->full_a[s], ph) || (!a.w_direct && !wait(&bars->full_b[s], ph))) { ok = false; break; }
                 if (leader) {
@@ -279,7 +282,7 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
         int s = 0, kb = kb_begin;
         uint32_t ph = 0;
         auto build_group = [&](int g) -> bool {
-            const int kb_end = min(n_kb, kb + kb_per_group);
+            const int kb_end = min(kb_stop, kb + kb_per_group);
             for (; kb < kb_end; ++kb) {
                 if (kb - kb_begin >= nstage && !ptx::mbar_wait(&bars->empty[s], ph ^ 1)) return false;
                 if (bars->abort_flag) return false;
@@ -604,8 +607,9 @@ cudaError_t launch_bn(const CUtensorMap& tmap, EncodeTiledFn enc, LinearArgs a, 
     const WeightLayout Lw = weight_layout(a.n_out, a.k_in, a.bits, a.group);
     const int bke = i8 ? 2 * BK : BK;
     const long long tiles = ((a.rows + BM - 1) / BM) * (a.n_out / BN) * (long long)n_z;
-    // few tiles and a long K loop: two CTAs per tile, each with half of the scale groups
-    const bool split = Lw.n_groups >= 2 && tiles <= 74 * Tile<BN>::CTAS_PER_SM && (a.k_in + bke - 1) / bke >= 6 && (long long)ns * Tile<BN>::STAGE_BYTES >= 256LL * (BN * 2 + 16);
+    // few tiles and a long K loop: two CTAs per tile, each with half of the scale groups (or of the k-blocks of a single
+    // group: not for integer activations, where a group's sum stays one exact int32 accumulation)
+    const bool split = (Lw.n_groups >= 2 || !i8) && tiles <= 74 * Tile<BN>::CTAS_PER_SM && (a.k_in + bke - 1) / bke >= 6 && (long long)ns * Tile<BN>::STAGE_BYTES >= 256LL * (BN * 2 + 16);
     void (*kern)(const CUtensorMap, const CUtensorMap, const LinearArgs, const int) =
         split ? (i8 ? linear_sm100_kernel<BN, true, true> : linear_sm100_kernel<BN, false, true>)
               : (i8 ? linear_sm100_kernel<BN, true, false> : linear_sm100_kernel<BN, false, false>);
