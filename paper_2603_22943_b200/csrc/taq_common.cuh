@@ -138,8 +138,10 @@ struct LinearArgs {
     int kv_which;               // EPI_KV: 0 = K, 1 = V
     int kv_qmax;                // EPI_KV: 127 (int8 rows) or 7 (4-bit rows); 0 is read as 127
     int epi;
-    int w_direct;               // (set by the launcher) int8 activations and 8-bit weights: the weight codes are the B
-                                // operand as they are and go from the blob into the ring by TMA, no staging or expansion
+    int w_direct;               // (set by the launcher) 1: int8 activations and 8-bit weights: the weight codes are the B
+                                // operand as they are and go from the blob into the ring by TMA, no staging or expansion;
+                                // 2: fp16 activations and 8-bit weights too large to stage whole: a slice of the codes per
+                                // k-block by TMA, expanded by the workers; 0: all codes staged once
     int early_weights;          // the previous kernel in the stream is known not to write the weights: fetch and expand
                                 // them before waiting for it
     int* status;

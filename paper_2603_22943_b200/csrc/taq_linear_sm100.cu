@@ -66,10 +66,12 @@ struct Plan {
 };
 
 template <int BN>
-__host__ __device__ inline Plan make_plan(int k_in, int bits, int group, int nstage, bool direct) {
+__host__ __device__ inline Plan make_plan(int k_in, int bits, int group, int nstage, int mode) {
     const WeightLayout L = weight_layout(BN, k_in, bits, group);
     Plan p;
-    p.raw_bytes = direct ? 0 : (int)(L.row_bytes * BN);    // (direct: no staged codes)
+    // codes of the BN channels over the whole fan-in; mode 1: none (the codes are the B operand); mode 2: one 64-byte slice
+    // per channel and ring stage
+    p.raw_bytes = mode == 1 ? 0 : mode == 2 ? nstage * BN * BK : (int)(L.row_bytes * BN);
     p.scale_bytes = BN * L.n_groups * 4;
     p.bias_bytes = BN * 4;
     p.off_raw = nstage * Tile<BN>::STAGE_BYTES;
@@ -95,7 +97,7 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
     constexpr int HC = TL::HC;
     extern __shared__ unsigned char smem_dyn[];
     unsigned char* smem = smem_dyn + ((1024u - (ptx::smem_u32(smem_dyn) & 1023u)) & 1023u);   // 1024-byte aligned, still provably shared
-    const Plan P = make_plan<BN>(a.k_in, a.bits, a.group, nstage, a.w_direct != 0);
+    const Plan P = make_plan<BN>(a.k_in, a.bits, a.group, nstage, a.w_direct);
     Bars* bars = reinterpret_cast<Bars*>(smem + P.off_bars);
     constexpr uint32_t TMEM_COLS = TL::TMEM_COLS;
 
@@ -151,8 +153,9 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
         // ---------------- producer: packed weights once, then activation tiles ----------------
         if (lane == 0) {
             if (!a.early_weights) ptx::pdl_wait();        // in general the weights may come from the previous kernel
-            ptx::mbar_arrive_expect_tx(&bars->w_full, (uint32_t)(P.raw_bytes + P.scale_bytes + P.bias_bytes));
-            if (P.raw_bytes) ptx::bulk_load(smem + P.off_raw, blob + L.off_codes + (size_t)col0 * L.row_bytes, (uint32_t)P.raw_bytes, &bars->w_full);
+            const int staged = a.w_direct ? 0 : P.raw_bytes;
+            ptx::mbar_arrive_expect_tx(&bars->w_full, (uint32_t)(staged + P.scale_bytes + P.bias_bytes));
+            if (staged) ptx::bulk_load(smem + P.off_raw, blob + L.off_codes + (size_t)col0 * L.row_bytes, (uint32_t)P.raw_bytes, &bars->w_full);
             ptx::bulk_load(smem + P.off_scales, blob + L.off_scales + (size_t)col0 * n_groups * 4, (uint32_t)P.scale_bytes, &bars->w_full);
             ptx::bulk_load(smem + P.off_bias, blob + L.off_bias + (size_t)col0 * 4, (uint32_t)P.bias_bytes, &bars->w_full);
             if (a.early_weights) ptx::pdl_wait();         // the activations come from the previous kernel
@@ -162,9 +165,10 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
             for (int kb = kb_begin; kb < kb_stop; ++kb) {
                 if (kb - kb_begin >= nstage && !ptx::mbar_wait(&bars->empty[s], ph ^ 1)) { raise_status(a.status, TAQ_ERR_TIMEOUT); bars->abort_flag = 1; }
                 if (bars->abort_flag) break;
-                ptx::mbar_arrive_expect_tx(&bars->full_a[s], A_TILE_BYTES + (a.w_direct ? BN * 128 : 0));
+                ptx::mbar_arrive_expect_tx(&bars->full_a[s], A_TILE_BYTES + (a.w_direct == 1 ? BN * 128 : a.w_direct == 2 ? BN * BK : 0));
                 ptx::tma_load_3d(smem + s * TL::STAGE_BYTES, &tmap_x, &bars->full_a[s], kb * BKE, row0, z);
-                if (a.w_direct) ptx::tma_load_3d(smem + s * TL::STAGE_BYTES + A_TILE_BYTES, &tmap_w, &bars->full_a[s], kb * BKE, col0, 0);
+                if (a.w_direct == 1) ptx::tma_load_3d(smem + s * TL::STAGE_BYTES + A_TILE_BYTES, &tmap_w, &bars->full_a[s], kb * BKE, col0, 0);
+                if (a.w_direct == 2) ptx::tma_load_3d(smem + P.off_raw + s * (BN * BK), &tmap_w, &bars->full_a[s], kb * BK, col0, 0);
                 issued = kb - kb_begin + 1;
                 if (++s == nstage) { s = 0; ph ^= 1; }
             }
@@ -194,7 +198,7 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
             }
             const int kb_end = min(kb_stop, kb + kb_per_group);
             for (bool first = true; kb < kb_end && ok; ++kb) {
-                if (!wait(&bars->full_a[s], ph) || (!a.w_direct && !wait(&bars->full_b[s], ph))) { ok = false; break; }
+                if (!wait(&bars->full_a[s], ph) || (a.w_direct != 1 && !wait(&bars->full_b[s], ph))) { ok = false; break; }
                 if (leader) {
                     if (kb < 20) TAQ_PROF(40 + kb);
                     const uint32_t a_lo = lo0 + s * (TL::STAGE_BYTES >> 4), b_lo = a_lo + (A_TILE_BYTES >> 4);
@@ -286,6 +290,7 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
             for (; kb < kb_end; ++kb) {
                 if (kb - kb_begin >= nstage && !ptx::mbar_wait(&bars->empty[s], ph ^ 1)) return false;
                 if (bars->abort_flag) return false;
+                if (a.w_direct == 2 && !ptx::mbar_wait(&bars->full_a[s], ph)) return false;    // this k-block's slice of the codes has arrived
                 unsigned char* b_tile = smem + s * TL::STAGE_BYTES + A_TILE_BYTES;
                 // 16-byte chunks of the fp16 tile: 8 per weight row; this thread owns chunk c of rows n0, n0 + 32, ...
                 constexpr int NCH = (BN * 8 + NWORK - 1) / NWORK;
@@ -321,6 +326,7 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
                     pw[i] = make_uint2(0, 0);
                     if ((BN * 8) % NWORK == 0 || n < BN) {
                         if (a.bits == 4) pw[i].x = *reinterpret_cast<const uint32_t*>(raw + n * row_bytes + kb * (BK / 2) + c * 4);
+                        else if (a.w_direct == 2) pw[i] = *reinterpret_cast<const uint2*>(raw + s * (BN * BK) + n * BK + c * 8);
                         else pw[i] = *reinterpret_cast<const uint2*>(raw + n * row_bytes + kb * BK + c * 8);
                     }
                 }
@@ -341,7 +347,7 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
         };
 
         for (int g = g_begin; g < g_end && ok; ++g) {
-            ok = a.w_direct ? true : build_group(g);
+            ok = a.w_direct == 1 ? true : build_group(g);
             if (ok && g > g_begin) ok = fold_group(g - 1);
         }
         if (ok) ok = fold_group(g_end - 1);
@@ -573,11 +579,22 @@ int pick_bn(const LinearArgs& a) {
     return 0;
 }
 
+// How the kernel gets at the weight codes: 0 = all codes of the tile's channels staged in shared memory once; 1 = int8
+// activations and 8-bit weights: the codes are the B operand, by TMA per k-block; 2 = fp16 activations and 8-bit weights whose
+// staged codes would not fit beside a two-stage ring (a 160-wide tile at a fan-in of 1280): a 64-byte slice per channel
+// arrives by TMA with every k-block's activations and the workers expand from it.
+template <int BN>
+int weight_mode(const LinearArgs& a) {
+    if (a.bits != 8 || a.reqs) return 0;
+    if (a.xq) return 1;
+    return make_plan<BN>(a.k_in, a.bits, a.group, 2, 0).total > SMEM_LIMIT ? 2 : 0;
+}
+
 // Ring depth: as deep as the K loop needs, but no deeper than three stages when that keeps two CTAs on an SM.
 template <int BN>
 int pick_nstage(const LinearArgs& a) {
     const int bke = a.xq ? 2 * BK : BK;
-    const bool direct = a.xq && a.bits == 8 && !a.reqs;
+    const int direct = weight_mode<BN>(a);
     const int n_kb = (a.k_in + bke - 1) / bke;
     const int half_sm = Tile<BN>::CTAS_PER_SM == 2 ? SMEM_LIMIT / 2 : SMEM_LIMIT;
     int best = 0;
@@ -613,15 +630,15 @@ cudaError_t launch_bn(const CUtensorMap& tmap, EncodeTiledFn enc, LinearArgs a, 
     void (*kern)(const CUtensorMap, const CUtensorMap, const LinearArgs, const int) =
         split ? (i8 ? linear_sm100_kernel<BN, true, true> : linear_sm100_kernel<BN, false, true>)
               : (i8 ? linear_sm100_kernel<BN, true, false> : linear_sm100_kernel<BN, false, false>);
-    a.w_direct = i8 && a.bits == 8 && !a.reqs;
+    a.w_direct = weight_mode<BN>(a);
     CUtensorMap tmap_w = tmap;                        // (unused unless w_direct)
     if (a.w_direct) {                                 // the codes section of the blob as an int8 matrix [n_out][k_in]
         const WeightLayout L = weight_layout(a.n_out, a.k_in, a.bits, a.group);
         const cuuint64_t dims[3] = {(cuuint64_t)a.k_in, (cuuint64_t)a.n_out, 1};
         const cuuint64_t strides[2] = {(cuuint64_t)L.row_bytes, (cuuint64_t)L.row_bytes * (cuuint64_t)a.n_out};
-        const cuuint32_t box[3] = {2 * BK, BN, 1}, estr[3] = {1, 1, 1};
+        const cuuint32_t box[3] = {a.w_direct == 1 ? 2 * BK : BK, BN, 1}, estr[3] = {1, 1, 1};    // mode 2: plain rows of 64 codes
         CUresult r = enc(&tmap_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, (void*)((const uint8_t*)a.w + L.off_codes), dims, strides, box, estr,
-                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, a.w_direct == 1 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
     }
     if (!configured[i8 + 2 * split]) {
@@ -629,7 +646,7 @@ cudaError_t launch_bn(const CUtensorMap& tmap, EncodeTiledFn enc, LinearArgs a, 
         if (e != cudaSuccess) return e;
         configured[i8 + 2 * split] = true;
     }
-    const Plan P = make_plan<BN>(a.k_in, a.bits, a.group, ns, a.w_direct != 0);
+    const Plan P = make_plan<BN>(a.k_in, a.bits, a.group, ns, a.w_direct);
     dim3 grid((unsigned)((a.rows + BM - 1) / BM) * (split ? 2u : 1u), a.n_out / BN, n_z);
     if (split) return launch_pdl_cluster(kern, grid, dim3(2, 1, 1), dim3(NTHREADS), (size_t)P.total, stream, tmap, tmap_w, a, ns);
     return launch_pdl(kern, grid, dim3(NTHREADS), (size_t)P.total, stream, tmap, tmap_w, a, ns);
