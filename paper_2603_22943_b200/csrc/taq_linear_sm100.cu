@@ -88,8 +88,9 @@ __host__ __device__ inline Plan make_plan(int k_in, int bits, int group, int nst
 // per-token-quantized activations, the B operand the int8 weight codes, the accumulators are exact int32; a K block is
 // 128 elements (one W4 scale group), and the row's activation scale multiplies the folded sum at the end.
 // SPLIT: for launches with few tiles and a long K loop, two CTAs (a cluster of two along x) share one output tile: the first
-// takes the lower half of the scale groups, the second the upper half; the second hands its folded fp32 partial sums to
-// the first through a bulk copy between the two shared memories, and the first adds them and runs the epilogue.
+// takes the lower half of the scale groups (of the k-blocks, when there is one group), the second the upper half; then
+// they exchange folded fp32 partial sums through bulk copies between the two shared memories, the first CTA adding and
+// storing rows 0..63 of the tile, the second rows 64..127.
 template <int BN, bool I8, bool SPLIT>
 __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w, const LinearArgs a, const int nstage) {
     using TL = Tile<BN>;
