@@ -327,6 +327,42 @@ taq_status taq_layer_forward_static(const taq_layer_desc* desc, const void* x_f1
  * it.  block_id_out may be NULL. */
 taq_status taq_poll_device_status(void* stream, int32_t* block_id_out);
 
+/* ---- Diagnostics (no counterpart in the paper; none of them touches a tensor) ----------------------------------
+ *
+ * Which kernel family served the calls so far.  The library prefers its tensor-core kernels and keeps generic
+ * CUDA-core kernels for shapes they do not cover; the generic ones are 10-40x slower, so a caller (or a test) that
+ * cares can check that none ran.  Counters are per process, counted on the host at launch time, and are not
+ * synchronised with the GPU.  counts_out: int64 [n]; entries beyond TAQ_N_KERNEL_FAMILIES read 0. */
+enum {
+    TAQ_KERNEL_LINEAR_TENSOR = 0,          /* dequant-GEMM on tcgen05 (also the integer-activation variant) */
+    TAQ_KERNEL_LINEAR_GENERIC = 1,         /* dequant-GEMM on CUDA cores */
+    TAQ_KERNEL_ATTENTION_TENSOR = 2,       /* stand-alone attention on tcgen05 */
+    TAQ_KERNEL_ATTENTION_GENERIC = 3,      /* stand-alone attention on CUDA cores */
+    TAQ_KERNEL_QUERY_ATTENTION_FUSED = 4,  /* to_q + Q_a + attention in one kernel */
+    TAQ_KERNEL_LAYER_FUSED = 5,            /* the whole layer pass in one kernel */
+    TAQ_KERNEL_LAYER_FUSED_A8 = 6,         /* the same with int8 activations */
+    TAQ_N_KERNEL_FAMILIES = 7
+};
+taq_status taq_dispatch_counts(int64_t* counts_out, int32_t n);
+void taq_dispatch_reset(void);
+
+/* The launch plan the tensor-core dequant-GEMM would take for a problem (host arithmetic only; nothing is launched
+ * and no GPU is needed).  plan_out: int32 [10] = {tile width BN (0: the tensor-core kernel does not take the
+ * problem), ring stages, weight mode (0 codes staged once, 1 codes are the operand, 2 codes sliced per K block), bytes
+ * of the ring, bytes of the ring the epilogue reuses as its staging area, offset of the staged codes, offset of the
+ * bias, offset of the barriers, total shared memory, shared-memory limit}.  Every region must lie inside `total`, the
+ * staging area inside the ring.  int8_activations / batched select the variant as taq_quantized_linear_i8 and the
+ * per-request calls do. */
+taq_status taq_linear_plan(const taq_weight_desc* desc, int64_t rows, int32_t out_kind, int32_t heads,
+                           int32_t int8_activations, int32_t batched, int32_t* plan_out);
+
+/* Failure-detection self-test.  Every wait inside the kernels is bounded (about one second of SM clock); when one
+ * runs out the block records TAQ_ERR_TIMEOUT in the device status word and returns.  This call launches one block
+ * whose only work is such a wait, on a barrier towards which nothing was ever issued, with a limit of `limit_cycles`
+ * SM cycles (1 .. 2^31): no pipeline is disturbed, nothing faults, and the next taq_poll_device_status reports the
+ * time-out and clears it. */
+taq_status taq_selftest_wait_expiry(int64_t limit_cycles, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

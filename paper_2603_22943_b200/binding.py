@@ -29,6 +29,7 @@ EXPORTS = [
     "taq_kv_project_a8_workspace_bytes", "taq_kv_project_a8", "taq_token_sensitivity_workspace_bytes",
     "taq_token_sensitivity", "taq_kv_set_prob_mask", "taq_hash_prompt", "taq_kv_cache_create", "taq_kv_cache_destroy",
     "taq_kv_cache_acquire", "taq_kv_cache_release", "taq_kv_cache_drop_checkpoint", "taq_kv_cache_get_stats",
+    "taq_dispatch_counts", "taq_dispatch_reset", "taq_linear_plan", "taq_selftest_wait_expiry",
 ]
 
 
@@ -101,6 +102,11 @@ def lib() -> C.CDLL:
         L.taq_layer_forward_batched.argtypes = [C.POINTER(LayerDesc), vp, i32, vp, vp, vp, sz, vp]
         L.taq_kv_project_batched.argtypes = [C.POINTER(LayerDesc), vp, i32, vp, vp]
         L.taq_poll_device_status.argtypes = [vp, C.POINTER(i32)]
+        L.taq_dispatch_counts.argtypes = [C.POINTER(i64), i32]
+        L.taq_dispatch_reset.restype = None
+        L.taq_dispatch_reset.argtypes = []
+        L.taq_linear_plan.argtypes = [C.POINTER(WeightDesc), i64, i32, i32, i32, i32, C.POINTER(i32)]
+        L.taq_selftest_wait_expiry.argtypes = [i64, vp]
         L.taq_static_workspace_capacity.restype = sz
         L.taq_static_workspace_capacity.argtypes = []
         L.taq_layer_forward_static.argtypes = [C.POINTER(LayerDesc), vp, vp, vp, vp, vp, vp, vp]
@@ -427,6 +433,36 @@ def taq_layer_forward_batched(desc: LayerDesc, reqs: torch.Tensor, n_requests: i
 
 def taq_kv_project_batched(desc: LayerDesc, reqs: torch.Tensor, n_requests: int, ctx: torch.Tensor, stream=None) -> None:
     _check(lib().taq_kv_project_batched(C.byref(desc), _ptr(reqs), n_requests, _ptr(ctx), _stream(stream)))
+
+
+KERNEL_FAMILIES = ("linear_tensor", "linear_generic", "attention_tensor", "attention_generic", "query_attention_fused",
+                   "layer_fused", "layer_fused_a8")
+
+
+def taq_dispatch_counts() -> dict:
+    """Launches per kernel family since the last taq_dispatch_reset()."""
+    arr = (C.c_int64 * len(KERNEL_FAMILIES))()
+    _check(lib().taq_dispatch_counts(arr, len(KERNEL_FAMILIES)))
+    return {k: int(arr[i]) for i, k in enumerate(KERNEL_FAMILIES)}
+
+
+def taq_dispatch_reset() -> None:
+    lib().taq_dispatch_reset()
+
+
+LINEAR_PLAN_FIELDS = ("bn", "nstage", "mode", "ring_bytes", "staging_bytes", "off_raw", "off_bias", "off_bars", "total", "limit")
+
+
+def taq_linear_plan(desc: "WeightDesc", rows: int, out_kind: int, heads: int = 1, int8_activations: bool = False, batched: bool = False) -> dict:
+    """Shared-memory plan of the tensor-core dequant-GEMM for a problem (host arithmetic; needs no GPU)."""
+    arr = (C.c_int32 * 10)()
+    _check(lib().taq_linear_plan(C.byref(desc), rows, out_kind, heads, int(int8_activations), int(batched), arr))
+    return {k: int(arr[i]) for i, k in enumerate(LINEAR_PLAN_FIELDS)}
+
+
+def taq_selftest_wait_expiry(limit_cycles: int, stream=None) -> None:
+    """Launches one block that waits (bounded by limit_cycles) on a barrier nothing arrives on."""
+    _check(lib().taq_selftest_wait_expiry(limit_cycles, _stream(stream)))
 
 
 def taq_poll_device_status(stream=None) -> int:

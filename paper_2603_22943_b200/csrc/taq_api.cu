@@ -1,9 +1,11 @@
 // C ABI of the TAQ library: host-side validation and kernel dispatch.  Nothing here allocates device memory.
+#include <atomic>
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
 
 #include "taq_common.cuh"
+#include "taq_ptx.cuh"
 #include "taq_sm100.cuh"
 
 namespace taq {
@@ -89,18 +91,33 @@ static Workspace workspace_layout(const taq_layer_desc* d, int n_requests) {
     return w;
 }
 
+// Launches per kernel family since the last taq_dispatch_reset (host-side counters; see taq_dispatch_counts in taq.h).
+static std::atomic<long long> g_dispatch[TAQ_N_KERNEL_FAMILIES];
+static void count_launch(int family) { g_dispatch[family].fetch_add(1, std::memory_order_relaxed); }
+
 static taq_status run_linear(const LinearArgs& a, int n_z, cudaStream_t st) {
     cudaError_t e;
-    if (sm100_linear_supported(a)) e = launch_linear_sm100(a, n_z, st);
-    else e = launch_linear_simt(a, n_z, st);
+    if (sm100_linear_supported(a)) { count_launch(TAQ_KERNEL_LINEAR_TENSOR); e = launch_linear_sm100(a, n_z, st); }
+    else { count_launch(TAQ_KERNEL_LINEAR_GENERIC); e = launch_linear_simt(a, n_z, st); }
     return e == cudaSuccess ? TAQ_OK : cuda_fail(e, "dequant-GEMM launch");
 }
 
 static taq_status run_attention(const AttnArgs& a, int n_z, cudaStream_t st) {
     cudaError_t e;
-    if (sm100_attention_supported(a)) e = launch_attention_sm100(a, n_z, st);
-    else e = launch_attention_simt(a, n_z, st);
+    if (sm100_attention_supported(a)) { count_launch(TAQ_KERNEL_ATTENTION_TENSOR); e = launch_attention_sm100(a, n_z, st); }
+    else { count_launch(TAQ_KERNEL_ATTENTION_GENERIC); e = launch_attention_simt(a, n_z, st); }
     return e == cudaSuccess ? TAQ_OK : cuda_fail(e, "attention launch");
+}
+
+// A kernel whose only work is a wait that nothing satisfies: the barrier is initialised and no arrival or copy is ever
+// directed at it, so the bounded wait runs out after `limit` cycles, the block records TAQ_ERR_TIMEOUT and returns.
+__global__ void wait_expiry_kernel(long long limit, int* status) {
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        ptx::mbar_init(&bar, 1);
+        ptx::mbar_fence_init();
+        if (!ptx::mbar_wait(&bar, 0, limit)) raise_status(status, TAQ_ERR_TIMEOUT);
+    }
 }
 
 }  // namespace taq
@@ -318,6 +335,7 @@ static taq_status q_attention_impl(const taq_layer_desc* d, const taq_request* r
     uint8_t* wsb = (uint8_t*)ws;
     const long long rows_per_z = (long long)d->batch * d->n_query;   // weights are shared by the whole batch
     if (sm100_qattn_supported(*d)) {
+        count_launch(TAQ_KERNEL_QUERY_ATTENTION_FUSED);
         cudaError_t e = launch_qattn_sm100(*d, (const __half*)x, Wq, kv, reqs, (__half*)o_dst, reqs ? n_req : d->batch, status, st);
         return e == cudaSuccess ? TAQ_OK : cuda_fail(e, "fused to_q + attention launch");
     }
@@ -344,6 +362,7 @@ static taq_status layer_forward_impl(const taq_layer_desc* d, const taq_request*
     taq_status s = status_ptr(&status);
     if (s != TAQ_OK) return s;
     if (sm100_layer_supported(*d)) {                                    // the whole pass in one kernel
+        count_launch(TAQ_KERNEL_LAYER_FUSED);
         cudaError_t e = launch_layer_sm100(*d, (const __half*)x, Wq, Wout, kv, reqs, (__half*)y, reqs ? n_req : d->batch, status, st);
         return e == cudaSuccess ? TAQ_OK : cuda_fail(e, "fused layer launch");
     }
@@ -395,6 +414,7 @@ taq_status taq_quantize_rows_f16(const void* x_f16_dev, int64_t rows, int32_t co
 }
 
 static taq_status run_linear_i8(const LinearArgs& a, cudaStream_t st) {
+    count_launch(TAQ_KERNEL_LINEAR_TENSOR);
     if (!sm100_linear_supported(a))
         return fail(TAQ_ERR_UNSUPPORTED, "integer-activation GEMM: needs k_in a multiple of 16, group 0 or 128, n_out a multiple of 64 or 80 (per-head output: head width 40, 64, 80 or 160)");
     cudaError_t e = launch_linear_sm100(a, 1, st);
@@ -473,6 +493,7 @@ taq_status taq_layer_forward_a8(const taq_layer_desc* d, const void* x_f16_dev, 
     s = status_ptr(&status);
     if (s != TAQ_OK) return s;
     if (sm100_layer_a8_supported(*d)) {                                   // the whole integer-activation pass in one kernel
+        count_launch(TAQ_KERNEL_LAYER_FUSED_A8);
         cudaError_t e1 = launch_layer_a8_sm100(*d, (const __half*)x_f16_dev, Wq_packed_dev, Wout_packed_dev, kv_packed_dev, (__half*)y_f16_dev,
                                                d->batch, status, st);
         return e1 == cudaSuccess ? TAQ_OK : cuda_fail(e1, "fused integer-activation layer launch");
@@ -731,6 +752,48 @@ taq_status taq_layer_forward_static(const taq_layer_desc* d, const void* x_f16_d
     // call, so nothing in the array has to start at zero and what the previous call left there is never read.
     return layer_forward_impl(d, nullptr, 1, x_f16_dev, Wq_packed_dev, Wout_packed_dev, kv_packed_dev, trig_mask_dev, y_f16_dev, ws,
                               (cudaStream_t)stream);
+}
+
+taq_status taq_dispatch_counts(int64_t* counts_out, int32_t n) {
+    if (!counts_out || n < 0) return fail(TAQ_ERR_INVALID_ARG, "counts_out is NULL or n negative");
+    for (int i = 0; i < n; ++i) counts_out[i] = i < TAQ_N_KERNEL_FAMILIES ? (int64_t)g_dispatch[i].load(std::memory_order_relaxed) : 0;
+    return TAQ_OK;
+}
+
+void taq_dispatch_reset(void) {
+    for (int i = 0; i < TAQ_N_KERNEL_FAMILIES; ++i) g_dispatch[i].store(0, std::memory_order_relaxed);
+}
+
+taq_status taq_linear_plan(const taq_weight_desc* d, int64_t rows, int32_t out_kind, int32_t heads, int32_t int8_activations,
+                           int32_t batched, int32_t* plan_out) {
+    taq_status s = check_weight_desc(d);
+    if (s != TAQ_OK) return s;
+    if (!plan_out) return fail(TAQ_ERR_INVALID_ARG, "plan_out is NULL");
+    if (out_kind != TAQ_OUT_F16 && out_kind != TAQ_OUT_F32 && out_kind != TAQ_OUT_INT8_HEAD_ROWS) return fail(TAQ_ERR_INVALID_ARG, "unknown out_kind %d", out_kind);
+    if (out_kind == TAQ_OUT_INT8_HEAD_ROWS && (heads < 1 || d->n_out % heads)) return fail(TAQ_ERR_SHAPE, "n_out (%d) must be a multiple of heads (%d)", d->n_out, heads);
+    static const taq_request dummy_req = {};
+    alignas(16) static const char dummy[16] = {};
+    LinearArgs a{};
+    if (int8_activations) a.xq = (const int8_t*)dummy; else a.x = (const __half*)dummy;
+    a.reqs = batched ? &dummy_req : nullptr;
+    a.rows = rows;
+    a.n_out = d->n_out; a.k_in = d->k_in; a.bits = d->bits; a.group = d->group;
+    a.heads = out_kind == TAQ_OUT_INT8_HEAD_ROWS ? heads : 1;
+    a.epi = out_kind == TAQ_OUT_F16 ? EPI_F16 : out_kind == TAQ_OUT_F32 ? EPI_F32 : EPI_Q8_HEAD;
+    int out[10];
+    linear_plan_of(a, out);
+    for (int i = 0; i < 10; ++i) plan_out[i] = out[i];
+    return TAQ_OK;
+}
+
+taq_status taq_selftest_wait_expiry(int64_t limit_cycles, void* stream) {
+    if (limit_cycles < 1 || limit_cycles > (1LL << 31)) return fail(TAQ_ERR_INVALID_ARG, "limit_cycles must be in [1, 2^31]");
+    int* status = nullptr;
+    taq_status s = status_ptr(&status);
+    if (s != TAQ_OK) return s;
+    wait_expiry_kernel<<<1, 32, 0, (cudaStream_t)stream>>>((long long)limit_cycles, status);
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? TAQ_OK : cuda_fail(e, "wait-expiry self-test launch");
 }
 
 taq_status taq_poll_device_status(void* stream, int32_t* block_id_out) {

@@ -86,7 +86,7 @@ struct QRegs {
     __device__ __forceinline__ uint4 chunk(int i) const {
         if (Q8) {
             const uint4 w = v[i / 2];
-            return codes8_to_half((i & 1) ? make_uint2(w.z, w.w) : make_uint2(w.x, w.y));
+            return codes_w8_to_half((i & 1) ? make_uint2(w.z, w.w) : make_uint2(w.x, w.y));
         }
         return v[i];
     }

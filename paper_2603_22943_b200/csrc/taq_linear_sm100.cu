@@ -563,49 +563,46 @@ EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
-int pick_bn(const LinearArgs& a) {
-    // Every column tile re-reads the activation rows, so tiles are as wide as the row count allows while the grid
-    // still covers most of the SMs.
-    const long long row_tiles = (a.rows + BM - 1) / BM;
-    if (a.epi == EPI_Q8_HEAD || a.epi == EPI_KV) {
-        const int d = a.n_out / a.heads;
-        if (d == 40 && a.heads % 4 == 0 && row_tiles * (a.n_out / 160) >= 96) return 160;   // two heads per worker thread
-        if (d == 40 && a.heads % 2 == 0) return 80;     // one head per worker thread
-        if (d == 64 || d == 80 || d == 160) return d;   // one head per tile, split between the row's two threads
-        return 0;
-    }
-    if (a.n_out % 160 == 0 && row_tiles * (a.n_out / 160) >= 96) return 160;
-    if (a.n_out % 80 == 0) return 80;
-    if (a.n_out % 64 == 0) return 64;
-    return 0;
-}
-
 // How the kernel gets at the weight codes: 0 = all codes of the tile's channels staged in shared memory once; 1 = int8
 // activations and 8-bit weights: the codes are the B operand, by TMA per k-block; 2 = fp16 activations and 8-bit weights whose
 // staged codes would not fit beside a two-stage ring (a 160-wide tile at a fan-in of 1280): a 64-byte slice per channel
 // arrives by TMA with every k-block's activations and the workers expand from it.
 template <int BN>
 int weight_mode(const LinearArgs& a) {
-    if (a.bits != 8 || a.reqs) return 0;
-    if (a.xq) return 1;
-    return make_plan<BN>(a.k_in, a.bits, a.group, 2, 0).total > SMEM_LIMIT ? 2 : 0;
+    if (a.bits != 8) return 0;
+    if (a.xq) return a.reqs ? 0 : 1;      // (per-request blobs have no common tensor map: their codes are staged)
+    return make_plan<BN>(a.k_in, a.bits, a.group, 2, 0).total > SMEM_LIMIT ? (a.reqs ? 0 : 2) : 0;
 }
 
-// Ring depth: as deep as the K loop needs, but no deeper than three stages when that keeps two CTAs on an SM.
+// Bytes of the ring that the epilogue reuses to stage a tile's output before the bulk stores: every one of the 256 worker
+// threads owns one piece of HC elements plus 16 bytes of padding.
+template <int BN>
+int epilogue_staging_bytes(const LinearArgs& a) {
+    constexpr int HC = Tile<BN>::HC;
+    if (a.epi == EPI_F16) return NWORK * (HC * 2 + 16);
+    if (a.epi == EPI_F32) return NWORK * (HC * 4 + 16);
+    if (a.epi == EPI_Q8_HEAD && HC % 16 == 0) return NWORK * (HC + 16);
+    return 0;
+}
+
+// Ring depth: as deep as the K loop needs, but no deeper than three stages when that keeps two CTAs on an SM, and never
+// shallower than the epilogue's staging area (which lives in the ring).  0: this tile width does not fit.
 template <int BN>
 int pick_nstage(const LinearArgs& a) {
     const int bke = a.xq ? 2 * BK : BK;
     const int direct = weight_mode<BN>(a);
     const int n_kb = (a.k_in + bke - 1) / bke;
     const int half_sm = Tile<BN>::CTAS_PER_SM == 2 ? SMEM_LIMIT / 2 : SMEM_LIMIT;
+    const int ns_min = (epilogue_staging_bytes<BN>(a) + Tile<BN>::STAGE_BYTES - 1) / Tile<BN>::STAGE_BYTES;
+    const int ns_max = n_kb < 2 ? 2 : n_kb;
     int best = 0;
-    for (int ns = 1; ns <= MAX_STAGE && ns <= (n_kb < 2 ? 2 : n_kb); ++ns) {
+    for (int ns = 1; ns <= MAX_STAGE && ns <= (ns_max > ns_min ? ns_max : ns_min); ++ns) {
         const int total = make_plan<BN>(a.k_in, a.bits, a.group, ns, direct).total;
         if (total > SMEM_LIMIT) break;
-        if (ns > 3 && total + 1024 > half_sm && make_plan<BN>(a.k_in, a.bits, a.group, 3, direct).total + 1024 <= half_sm) break;
+        if (ns > 3 && ns > ns_min && total + 1024 > half_sm && make_plan<BN>(a.k_in, a.bits, a.group, 3, direct).total + 1024 <= half_sm) break;
         best = ns;
     }
-    return best;
+    return best >= ns_min ? best : 0;
 }
 
 int nstage_for(const LinearArgs& a, int bn) {
@@ -617,9 +614,26 @@ int nstage_for(const LinearArgs& a, int bn) {
     return 0;
 }
 
+int pick_bn(const LinearArgs& a) {
+    // Every column tile re-reads the activation rows, so tiles are as wide as the row count allows while the grid
+    // still covers most of the SMs; a width whose ring and staging do not fit shared memory is passed over.
+    const long long row_tiles = (a.rows + BM - 1) / BM;
+    auto fits = [&](int bn) { return nstage_for(a, bn) >= 2; };
+    if (a.epi == EPI_Q8_HEAD || a.epi == EPI_KV) {
+        const int d = a.n_out / a.heads;
+        if (d == 40 && a.heads % 4 == 0 && row_tiles * (a.n_out / 160) >= 96 && fits(160)) return 160;   // two heads per worker thread
+        if (d == 40 && a.heads % 2 == 0) return fits(80) ? 80 : 0;     // one head per worker thread
+        if (d == 64 || d == 80 || d == 160) return fits(d) ? d : 0;   // one head per tile, split between the row's two threads
+        return 0;
+    }
+    if (a.n_out % 160 == 0 && row_tiles * (a.n_out / 160) >= 96 && fits(160)) return 160;
+    if (a.n_out % 80 == 0 && fits(80)) return 80;
+    if (a.n_out % 64 == 0 && fits(64)) return 64;
+    return 0;
+}
+
 template <int BN>
 cudaError_t launch_bn(const CUtensorMap& tmap, EncodeTiledFn enc, LinearArgs a, int n_z, cudaStream_t stream) {
-    static bool configured[4] = {false, false, false, false};
     const bool i8 = a.xq != nullptr;
     const int ns = pick_nstage<BN>(a);
     const WeightLayout Lw = weight_layout(a.n_out, a.k_in, a.bits, a.group);
@@ -642,10 +656,9 @@ cudaError_t launch_bn(const CUtensorMap& tmap, EncodeTiledFn enc, LinearArgs a, 
                          CU_TENSOR_MAP_INTERLEAVE_NONE, a.w_direct == 1 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
     }
-    if (!configured[i8 + 2 * split]) {
+    {   // (the attribute belongs to the current device's copy of the function: set on every launch, it is cheap)
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT);
         if (e != cudaSuccess) return e;
-        configured[i8 + 2 * split] = true;
     }
     const Plan P = make_plan<BN>(a.k_in, a.bits, a.group, ns, a.w_direct);
     dim3 grid((unsigned)((a.rows + BM - 1) / BM) * (split ? 2u : 1u), a.n_out / BN, n_z);
@@ -670,6 +683,32 @@ bool sm100_linear_supported(const LinearArgs& a) {
     if (bn == 0) return false;
     if (nstage_for(a, bn) < 2) return false;
     return encode_tiled_fn() != nullptr;
+}
+
+// The launch plan of a dequant-GEMM as the launcher would take it (no GPU needed): tile width, ring depth, how the codes
+// reach the CTA, and the byte ranges of shared memory that the ring, the epilogue's staging area and the fixed sections
+// occupy.  out: {bn, nstage, mode, ring_bytes, staging_bytes, off_raw, off_bias, off_bars, total, limit}.  bn = 0: the
+// tensor-core kernel does not take this problem.
+void linear_plan_of(const LinearArgs& a, int out[10]) {
+    for (int i = 0; i < 10; ++i) out[i] = 0;
+    out[9] = SMEM_LIMIT;
+    bool ok = a.rows >= 1;
+    if (a.xq) ok = ok && a.k_in % 16 == 0 && (a.group == 0 || a.group == 2 * BK || a.group >= a.k_in);
+    else ok = ok && a.k_in % BK == 0 && (a.group == 0 || a.group % BK == 0);
+    if (!ok) return;
+    const int bn = pick_bn(a);
+    if (bn == 0) return;
+    const int ns = nstage_for(a, bn);
+    if (ns < 2) return;
+    Plan P;
+    int stage_bytes = 0, staging = 0, mode = 0;
+    switch (bn) {
+        case 64: mode = weight_mode<64>(a); P = make_plan<64>(a.k_in, a.bits, a.group, ns, mode); stage_bytes = Tile<64>::STAGE_BYTES; staging = epilogue_staging_bytes<64>(a); break;
+        case 80: mode = weight_mode<80>(a); P = make_plan<80>(a.k_in, a.bits, a.group, ns, mode); stage_bytes = Tile<80>::STAGE_BYTES; staging = epilogue_staging_bytes<80>(a); break;
+        default: mode = weight_mode<160>(a); P = make_plan<160>(a.k_in, a.bits, a.group, ns, mode); stage_bytes = Tile<160>::STAGE_BYTES; staging = epilogue_staging_bytes<160>(a); break;
+    }
+    out[0] = bn; out[1] = ns; out[2] = mode; out[3] = ns * stage_bytes; out[4] = staging;
+    out[5] = P.off_raw; out[6] = P.off_bias; out[7] = P.off_bars; out[8] = P.total;
 }
 
 cudaError_t launch_linear_sm100(const LinearArgs& a, int n_z, cudaStream_t stream) {

@@ -32,12 +32,14 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// Waits for the phase with the given parity to complete, for at most ~1 s of SM clock.  Returns false on expiry.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+// Waits for the phase with the given parity to complete, for at most `limit` cycles of SM clock (default: about one
+// second).  Returns false on expiry.
+constexpr long long kWaitCycles = 1LL << 31;
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, long long limit = kWaitCycles) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     while (!mbar_try_wait(bar, parity)) {
-        if (clock64() - t0 > (1LL << 31)) return false;
+        if (clock64() - t0 > limit) return false;
     }
     return true;
 }
@@ -145,6 +147,12 @@ __device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t (&r)[8]) {
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
                  : "r"(taddr));
 }
+// One column: thread l of the warp receives lane (lane_base + l); the value is valid after tmem_ld_wait().
+__device__ __forceinline__ uint32_t tmem_ld1_wait(uint32_t taddr) {
+    uint32_t r;
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];\n\ttcgen05.wait::ld.sync.aligned;" : "=r"(r) : "r"(taddr) : "memory");
+    return r;
+}
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
@@ -206,6 +214,7 @@ __device__ __forceinline__ uint64_t desc_k_sw64(uint32_t smem_addr_bytes) {
 __device__ __forceinline__ uint32_t desc_lo(uint32_t smem_addr_bytes) { return ((smem_addr_bytes >> 4) & 0x3FFFu) | (1u << 16); }
 constexpr uint32_t kDescHiSw128 = (1024u >> 4) | (1u << 14) | (2u << 29);
 constexpr uint32_t kDescHiSw64 = (512u >> 4) | (1u << 14) | (4u << 29);
+constexpr uint32_t kDescHiSw32 = (256u >> 4) | (1u << 14) | (6u << 29);      // rows of 32 bytes, groups of 8 rows 256 bytes apart
 __device__ __forceinline__ uint64_t desc_join(uint32_t hi, uint32_t lo) { return ((uint64_t)hi << 32) | lo; }
 // Instruction descriptor: fp16 x fp16 -> fp32, both operands K-major, M = 128, N = n.
 __host__ __device__ constexpr uint32_t idesc_f16_m128(int n) {
@@ -240,6 +249,10 @@ __device__ __forceinline__ void mma_commit(uint64_t* bar) {
 // Byte offset of 16-byte chunk `chunk` (0..3) of row `row` in a tile stored with the 64-byte swizzle.
 __device__ __forceinline__ uint32_t sw64_offset(int row, int chunk) {
     return (uint32_t)(row * 64 + ((chunk ^ ((row >> 1) & 3)) << 4));
+}
+// The same for the 32-byte swizzle (rows of 32 bytes = one K step of fp16): address bit 4 XOR-ed with bit 7.
+__device__ __forceinline__ uint32_t sw32_offset(int row, int chunk) {
+    return (uint32_t)(row * 32 + ((chunk ^ ((row >> 2) & 1)) << 4));
 }
 // Byte offset of the 16-byte chunk `chunk` (0..7) of row `row` inside a 128-byte-swizzled K-major tile.
 __device__ __forceinline__ uint32_t sw128_offset(int row, int chunk) {

@@ -1,5 +1,6 @@
-// to_q and the TAQ attention in one kernel for the SD-1.5 64x64 shape (C = 320, 8 heads of 40, W4): Q never leaves
-// the SM.  A CTA owns 128 query rows of one sequence and four heads (160 output channels of to_q):
+// The integer-activation (int8 X and O) layer pass in one kernel for the SD-1.5 64x64 shape (C = 320, 8 heads of 40, W4);
+// the fp16-activation pass lives in taq_layer_c320_sm100.cu.  Only the A8 instantiation of the template below is built.
+// to_q and the TAQ attention in one kernel: Q never leaves the SM.  A CTA owns 128 query rows of one sequence and four heads (160 output channels of to_q):
 //   phase 1  Q = X Wq^T for its 160 channels: the dequant-GEMM of taq_linear_sm100.cu (integer-code operands, one
 //            accumulation pass per scale group; here every group - at most three - has its own TMEM accumulator,
 //            so the tensor core never waits for the workers, who fold the groups into registers at the end);
@@ -885,17 +886,6 @@ EncodeTiledFn encode_tiled_fn2() {
 
 }  // namespace
 
-bool sm100_layer_supported(const taq_layer_desc& d) { return sm100_qattn_supported(d); }
-
-bool sm100_qattn_supported(const taq_layer_desc& d) {
-    if (d.channels != KIN || d.heads * D != KIN) return false;
-    if (d.w_bits != 4) return false;
-    if (d.w_group != 0 && (d.w_group % BK || (KIN + d.w_group - 1) / d.w_group > MAX_GROUPS)) return false;
-    if (d.n_ctx > TP || (d.p_bits != 8 && d.p_bits != 4)) return false;
-    if (d.n_query < 1) return false;
-    return encode_tiled_fn2() != nullptr;
-}
-
 static cudaError_t launch_c320(const taq_layer_desc& d, const __half* x, const void* wq, const void* kv, const taq_request* reqs, __half* o,
                                const void* wout, __half* y, int n_z, int* status, cudaStream_t stream, bool a8 = false) {
     if (n_z == 0 || d.n_query == 0) return cudaSuccess;
@@ -914,7 +904,6 @@ static cudaError_t launch_c320(const taq_layer_desc& d, const __half* x, const v
     a.n_query = d.n_query; a.heads = d.heads; a.n_ctx = d.n_ctx; a.max_trigger = d.max_trigger; a.group = d.w_group; a.q_bits = d.q_bits; a.p_bits = d.p_bits;
     a.status = status;
     dim3 grid((d.n_query + ROWS - 1) / ROWS, d.heads / HG, n_z);
-    static bool configured[8] = {false, false, false, false, false, false, false, false};
     const bool tail = d.n_ctx > 64, fuse_out = y != nullptr;
     CUtensorMap tmap_y = tmap;                        // (unused by the variant that stores O)
     if (fuse_out) {
@@ -923,27 +912,13 @@ static cudaError_t launch_c320(const taq_layer_desc& d, const __half* x, const v
                 CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
     }
-    void (*kern)(const CUtensorMap, const CUtensorMap, const QAttnArgs) =
-        a8 ? (tail ? qattn_c320_kernel<true, true, true> : qattn_c320_kernel<false, true, true>)
-           : fuse_out ? (tail ? qattn_c320_kernel<true, true> : qattn_c320_kernel<false, true>) : (tail ? qattn_c320_kernel<true, false> : qattn_c320_kernel<false, false>);
-    const int ci = (tail ? 1 : 0) + (fuse_out ? 2 : 0) + (a8 ? 4 : 0);
-    if (!configured[ci]) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TOTAL);
-        if (e != cudaSuccess) return e;
-        configured[ci] = true;
-    }
+    (void)a8;                                         // only the integer-activation variant is built from this file
+    void (*kern)(const CUtensorMap, const CUtensorMap, const QAttnArgs) = tail ? qattn_c320_kernel<true, true, true> : qattn_c320_kernel<false, true, true>;
+    // (the attribute belongs to the current device's copy of the function: set on every launch, it is cheap)
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TOTAL);
+    if (e != cudaSuccess) return e;
     if (fuse_out) return launch_pdl_cluster(kern, grid, dim3(1, 2, 1), dim3(NTHREADS), (size_t)TOTAL, stream, tmap, tmap_y, a);
     return launch_pdl(kern, grid, dim3(NTHREADS), (size_t)TOTAL, stream, tmap, tmap_y, a);
-}
-
-cudaError_t launch_qattn_sm100(const taq_layer_desc& d, const __half* x, const void* wq, const void* kv, const taq_request* reqs, __half* o,
-                               int n_z, int* status, cudaStream_t stream) {
-    return launch_c320(d, x, wq, kv, reqs, o, nullptr, nullptr, n_z, status, stream);
-}
-
-cudaError_t launch_layer_sm100(const taq_layer_desc& d, const __half* x, const void* wq, const void* wout, const void* kv, const taq_request* reqs,
-                               __half* y, int n_z, int* status, cudaStream_t stream) {
-    return launch_c320(d, x, wq, kv, reqs, nullptr, wout, y, n_z, status, stream);
 }
 
 bool sm100_layer_a8_supported(const taq_layer_desc& d) { return sm100_qattn_supported(d) && d.w_group == 128; }

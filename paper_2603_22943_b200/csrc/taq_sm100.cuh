@@ -7,6 +7,8 @@ namespace taq {
 // True when the tensor-core dequant-GEMM covers this problem; otherwise the generic kernel runs.
 bool sm100_linear_supported(const LinearArgs& a);
 cudaError_t launch_linear_sm100(const LinearArgs& a, int n_z, cudaStream_t stream);
+// Launch plan of the tensor-core dequant-GEMM for a problem (host arithmetic only): see taq_linear_plan in taq.h.
+void linear_plan_of(const LinearArgs& a, int out[10]);
 
 bool sm100_attention_supported(const AttnArgs& a);
 cudaError_t launch_attention_sm100(const AttnArgs& a, int n_z, cudaStream_t stream);

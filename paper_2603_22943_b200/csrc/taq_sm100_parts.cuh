@@ -71,8 +71,6 @@ __device__ __forceinline__ float ex2_approx(float x) {
     return y;
 }
 
-__device__ __forceinline__ uint4 codes8_to_half(uint2 raw) { return codes_w8_to_half(raw); }
-
 constexpr int HK = TP / 2;           // keys per thread: a row's scores are split between two threads
 
 // Softmax pieces of one thread: its HK raw scores u (integer dot products) -> e_j = 2^(s_j sq - m) with the

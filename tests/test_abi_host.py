@@ -125,3 +125,44 @@ def test_binding_fails_loudly_without_the_library(monkeypatch, tmp_path):
     monkeypatch.setattr(tb, "LIB_PATH", str(tmp_path / "libtaq.so"))
     with pytest.raises(RuntimeError, match="no fallback"):
         tb.lib()
+
+
+def test_linear_plan_keeps_every_region_inside_shared_memory(L):
+    """The dequant-GEMM's epilogue stages a tile's output in the ring of operand stages.  For every problem the
+    tensor-core kernel accepts, the ring must hold that staging area and every fixed section must lie inside the
+    shared memory the launch asks for (a two-stage ring at a short fan-in once was too small for a 160-wide fp32 tile)."""
+    seen = 0
+    for n_out in (64, 80, 160, 320, 640, 1280):
+        for k_in in (64, 128, 192, 256, 320, 640, 768, 1280, 1536, 2048):
+            for bits, group in ((4, 128), (4, 0), (4, 64), (8, 0)):
+                for rows in (77, 128, 8192, 65536):
+                    for kind, heads in ((tb.TAQ_OUT_F16, 1), (tb.TAQ_OUT_F32, 1), (tb.TAQ_OUT_INT8_HEAD_ROWS, max(1, n_out // 40)),
+                                        (tb.TAQ_OUT_INT8_HEAD_ROWS, max(1, n_out // 160))):
+                        for i8 in (False, True):
+                            for batched in (False, True):
+                                if kind == tb.TAQ_OUT_INT8_HEAD_ROWS and n_out % heads:
+                                    continue
+                                plan = tb.taq_linear_plan(tb.weight_desc(n_out, k_in, bits, group), rows, kind, heads, i8, batched)
+                                if plan["bn"] == 0:
+                                    continue
+                                seen += 1
+                                what = (n_out, k_in, bits, group, rows, kind, heads, i8, batched, plan)
+                                assert plan["nstage"] >= 2, what
+                                assert plan["staging_bytes"] <= plan["ring_bytes"], what
+                                assert plan["ring_bytes"] <= plan["off_raw"] <= plan["off_bias"] < plan["off_bars"] < plan["total"], what
+                                assert plan["total"] <= plan["limit"], what
+    assert seen > 1000
+    # the case that used to overflow: a 160-wide fp32 tile over a fan-in of 128 (two K blocks)
+    plan = tb.taq_linear_plan(tb.weight_desc(320, 128, 4, 128), 8192, tb.TAQ_OUT_F32)
+    assert plan["bn"] == 160 and plan["staging_bytes"] == 256 * (80 * 4 + 16) and plan["ring_bytes"] >= plan["staging_bytes"]
+
+
+def test_dispatch_counters_start_at_zero_and_reset(L):
+    tb.taq_dispatch_reset()
+    assert set(tb.taq_dispatch_counts().values()) == {0}
+    assert len(tb.taq_dispatch_counts()) == 7
+
+
+def test_wait_expiry_selftest_rejects_bad_limits(L):
+    for bad in (0, -5, (1 << 31) + 1):                 # (refused on the host: nothing is launched)
+        assert L.taq_selftest_wait_expiry(bad, None) == tb.TAQ_ERR_INVALID_ARG

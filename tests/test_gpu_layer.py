@@ -153,12 +153,28 @@ def _layer_case(shape, sample_rows=None, max_trigger=None):
     return tl.check_layer(shape, data, y, parts, rows)
 
 
+def _assert_same_up_to_code_ties(a, b, what):
+    """Two GPU routes through the same arithmetic: equal except where a sum taken in another order moved an fp16
+    rounding (one ulp) or a probability code on a tie (1/255 of a value row)."""
+    a = a.float().cpu().numpy().astype(np.float64)
+    b = b.float().cpu().numpy().astype(np.float64)
+    diff = np.abs(a - b)
+    ulp = 2.0 ** -10 * np.maximum(np.abs(a), np.abs(b)) + 1e-6
+    assert diff.max() <= tl.TOL_MAX_ABS, f"{what}: max difference {diff.max():.3e} at {np.unravel_index(diff.argmax(), diff.shape)}"
+    frac = float(np.mean(diff > 2 * ulp))
+    assert frac <= 2e-3, f"{what}: {frac:.2e} of the values differ by more than two fp16 ulps"
+    rel = np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-30)
+    assert rel <= 2e-4, f"{what}: relative L2 difference {rel:.3e}"
+
+
 @pytest.mark.parametrize("shape_fn,n", [(synth.config2, 4096), (synth.config2, 333), (lambda: synth.config3_layers()[5], 200)],
                          ids=["config2_full", "config2_ragged", "C640_unfused"])
 @pytest.mark.parametrize("q_bits", [8, 0])
 def test_query_attention_equals_the_two_step_path(shape_fn, n, q_bits):
     """taq_query_attention (one fused kernel at C = 320) against taq_quantized_linear + taq_cross_attention on the same
-    inputs: the same arithmetic in the same order, hence bit-identical O; and against the oracle's O on sampled rows."""
+    inputs: the same Q~ codes and scores; the fused kernel sums a row's 80 exponentials in one thread, the stand-alone
+    kernel in two, so a probability that sits on a rounding boundary may take the neighbouring code (1/255 of one value
+    row): O agrees to that, and both are checked against the oracle's O on sampled rows."""
     from dataclasses import replace
     shape = replace(_small(shape_fn(), n), q_bits=q_bits)
     data = synth.make_layer(shape)
@@ -176,7 +192,7 @@ def test_query_attention_equals_the_two_step_path(shape_fn, n, q_bits):
         q16 = tb.taq_quantized_linear(P["wd_cc"], x2, P["Wq"], tb.TAQ_OUT_F16)
         o_two = tb.taq_cross_attention(desc, q16, None, kv, mask)
     tb.taq_poll_device_status()
-    assert torch.equal(o_fused.view(torch.int16), o_two.view(torch.int16))
+    _assert_same_up_to_code_ties(o_fused, o_two, "O")
     rows = np.arange(0, shape.n_query, max(1, shape.n_query // 64))
     cfg = tl.oracle_cfg(shape)
     g = tl.gpu_decisions(shape, data, {"desc": desc, "packed": P, "kv": kv, "mask": mask}, rows)
@@ -187,8 +203,9 @@ def test_query_attention_equals_the_two_step_path(shape_fn, n, q_bits):
 @pytest.mark.parametrize("n,q_bits", [(4096, 8), (333, 8), (130, 0)])
 def test_one_kernel_layer_equals_the_step_by_step_path(n, q_bits):
     """At C = 320 taq_layer_forward is a single kernel (pairs of CTAs exchange O through distributed shared memory and
-    run to_out themselves).  Its Y must equal, bit for bit, taq_query_attention followed by taq_quantized_linear: the
-    same products accumulated in the same order."""
+    run to_out themselves).  Its Y must equal taq_query_attention followed by taq_quantized_linear up to the order in
+    which the scale groups' partial sums are added (the second CTA of a pair walks the K blocks downwards) and to the
+    fp16 rounding of Y that this moves; the oracle comparison at the full tolerance is test_layer_config2_full."""
     from dataclasses import replace
     shape = replace(_small(synth.config2(), n), q_bits=q_bits)
     data = synth.make_layer(shape)
@@ -201,7 +218,7 @@ def test_one_kernel_layer_equals_the_step_by_step_path(n, q_bits):
     o = tb.taq_query_attention(desc, x, P["Wq"], kv, mask)
     y_two = tb.taq_quantized_linear(P["wd_cc"], o.reshape(-1, shape.channels), P["Wout"], tb.TAQ_OUT_F16).reshape(y_one.shape)
     tb.taq_poll_device_status()
-    assert torch.equal(y_one.view(torch.int16), y_two.view(torch.int16))
+    _assert_same_up_to_code_ties(y_one, y_two, "Y")
 
 
 def test_layer_config1_full():

@@ -408,6 +408,42 @@ def check_contract_close_to_ideal(o):
     assert np.array_equal(yc, yc.astype(np.float16).astype(np.float64))      # Y is fp16 data
 
 
+def check_contract_roundings(o):
+    """Every fp16 rounding point of contract mode on a hand-built case whose expected value is typed in as a literal
+    (worked out by hand from the fp16 grid: spacing 2^-4 in [64,128), 2^-9 in [2,4), 2^-10 in [1,2), 2^-14 in [1/16,1/8))."""
+    cfg = o.TaqConfig(heads=1, w_bits=0, q_bits=0, kv_bits=8, p_bits=8, contract=True)
+    one = np.ones((1, 1, 1, 1))
+    # (1) a trigger probability column is stored in the unit of the uint8 codes, 1/255, as fp16(255 A) / 255.
+    #     Two keys with logits (0, ln(154.7 / 100.3)): A = (100.3, 154.7) / 255.  255 A_0 = 100.3 lies between the fp16
+    #     numbers 100.25 and 100.3125 and is nearer the second; A_0 itself (0.39333...) would round to 0.393310546875.
+    K = np.array([0.0, np.log(154.7 / 100.3)]).reshape(1, 1, 2, 1)
+    V = np.array([1.0, 0.0]).reshape(1, 1, 2, 1)
+    _, A, A_hat = o.taq_attention(one, K, V, np.array([[1, 0]], np.uint8), cfg, return_probs=True)
+    assert abs(A[0, 0, 0, 0] - 100.3 / 255) < 1e-12
+    assert A_hat[0, 0, 0, 0] == 100.3125 / 255                           # not A, not fp16(A) = 0.393310546875
+    assert abs(A_hat[0, 0, 0, 1] - 155.0 / 255) < 1e-7                   # the ordinary column: rint(154.7) = 155, dequantized in binary32
+    # (2), (3) the value operand of an ordinary row is fp16(code * scale), and O is fp16.  Logits (0, ln 2): A = (1/3, 2/3),
+    #     codes (85, 170), so A^ = (1/3, 2/3) exactly.  V~ = (3.001, 0): fp16(3.001) = 3.001953125 (3.001 is 0.00095 from it
+    #     and 0.001 from 3.0); a third of that, 1.00065..., rounds to 1.0009765625.  With V~ left unrounded the product is
+    #     1.00033..., which rounds to 1.0; with O left unrounded it stays 1.00065104....
+    K = np.array([0.0, np.log(2.0)]).reshape(1, 1, 2, 1)
+    V = np.array([3.001, 0.0]).reshape(1, 1, 2, 1)
+    O = o.taq_attention(one, K, V, np.zeros((1, 2), np.uint8), cfg)
+    assert O.shape == (1, 1, 1) and O[0, 0, 0] == 1.0009765625
+    O_ideal = o.taq_attention(one, K, V, np.zeros((1, 2), np.uint8), o.TaqConfig(heads=1, w_bits=0, q_bits=0, contract=False))
+    assert abs(O_ideal[0, 0, 0] - 3.001 / 3) < 1e-7                      # (the code 85 is dequantized in binary32)
+    # (4) an unquantized Q (q_bits = 0) is an fp16 tensor: 1.0 * fp32(0.1) -> 0.0999755859375 (spacing 2^-14 there)
+    q = o.taq_q(np.ones((1, 1, 1), np.float16), np.array([[0.1]], np.float32), cfg)
+    assert q["Q_tilde"].shape == (1, 1, 1, 1) and q["Q_tilde"][0, 0, 0, 0] == 0.0999755859375
+    assert abs(q["Q"][0, 0, 0, 0] - np.float64(np.float32(0.1))) < 1e-15
+    # (5) a trigger K/V row is fp16 of the projected row: ctx 1.0, weights 0.1 and 0.3 -> 0.0999755859375, 0.300048828125
+    kv = o.taq_kv(np.ones((1, 1, 1), np.float16), np.array([[0.1]], np.float32), np.array([[0.3]], np.float32), np.ones((1, 1), np.uint8), cfg)
+    assert kv["K_tilde"][0, 0, 0, 0] == 0.0999755859375 and kv["V_tilde"][0, 0, 0, 0] == 0.300048828125
+    # (6) Y is fp16: O = 1 (fp16 data), weight 0.1, bias 0.2 -> fp64 0.3000000014901161 -> 0.300048828125
+    Y = o.taq_out(np.ones((1, 1, 1)), np.array([[0.1]], np.float32), np.array([0.2], np.float32), cfg)
+    assert Y[0, 0, 0] == 0.300048828125
+
+
 def check_integer_activations(o):
     """a_bits = 8 (the W/A reading of Table 1: the inputs of the projections are int8 per token).
     (i) the projection is an integer product: Q[b,n,c] = s_x[b,n] * sum_g s_w[c,g] * sum_{k in g} xq[b,n,k] wq[c,k],
@@ -549,7 +585,7 @@ def check_token_sensitivity(o):
 
 LAYER_CHECKS = [check_all_trigger_is_textbook_attention, check_empty_mask_is_uniform_quantization,
                 check_trigger_rows_pass_through, check_closed_forms, check_structure, check_brute_force,
-                check_contract_close_to_ideal, check_integer_activations, check_four_bit_rows_and_probabilities,
+                check_contract_close_to_ideal, check_contract_roundings, check_integer_activations, check_four_bit_rows_and_probabilities,
                 check_token_sensitivity]
 
 
@@ -625,6 +661,13 @@ MUTATIONS = {
     "four_bit_probs_use_8_bit_levels": [("_, Aq = quantize_prob(A, cfg.p_bits)", "_, Aq = quantize_prob(A, 8)")],
     "sensitivity_quantizes_all_but_i": [("        m = ones.copy()\n        m[:, i] = 0", "        m = 1 - ones\n        m[:, i] = 1")],
     "sensitivity_reference_quantized": [("y_star = taq_layer(X, ctx, Wq, Wk, Wv, Wout, bout, ones, c, mask_a=ones)", "y_star = taq_layer(X, ctx, Wq, Wk, Wv, Wout, bout, 1 - ones, c, mask_a=ones)")],
+    "contract_v_not_rounded": [("        V_tilde = f16_round(V_tilde)\n", "        V_tilde = V_tilde\n")],
+    "contract_kept_prob_rounded_in_unit_1": [("kept = f16_round(A * pmax) / pmax if cfg.contract else A", "kept = f16_round(A) if cfg.contract else A")],
+    "contract_kept_prob_not_rounded": [("kept = f16_round(A * pmax) / pmax if cfg.contract else A", "kept = A")],
+    "contract_o_not_rounded": [("    if cfg.contract:\n        O = f16_round(O)\n", "")],
+    "contract_q16_not_rounded": [("Qt = f16_round(Q) if cfg.contract else Q", "Qt = Q")],
+    "contract_trigger_rows_not_rounded": [("kept = f16_round(Z) if cfg.contract else Z", "kept = Z")],
+    "contract_y_not_rounded": [("    return f16_round(Y) if cfg.contract else Y", "    return Y")],
     "heads_interleaved": [("return x.reshape(B, L, heads, d).transpose(0, 2, 1, 3)", "return x.reshape(B, L, d, heads).transpose(0, 3, 1, 2)")],
 }
 

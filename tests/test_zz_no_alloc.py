@@ -4,7 +4,9 @@ It serves callers that have no way to obtain a workspace: a server whose memory 
 GPU (a fresh device allocation would fail or stall every stream), or a plug-in interface that hands over
 nothing but input and output pointers.  Its result must equal `taq_layer_forward`'s, which runs the same
 kernels on a caller-owned workspace.  The shared array keeps whatever the last call left in it, so the check
-is made on two calls in a row with different inputs: a stale intermediate result would show up in the second.
+is made on two calls in a row with different inputs, both on shapes whose pass really goes through the scratch
+(three kernels with Q~ and O in between; the one-kernel shape never touches it): the second call's sections lie
+over other bytes of what the first one left, so a stale intermediate result would show up there.
 The file name sorts last on purpose, so that a run stopping at the first failure has already run the rest.
 """
 import numpy as np
@@ -31,15 +33,20 @@ def _inputs(shape):
 
 def test_static_workspace_matches_caller_workspace_on_two_calls_in_a_row():
     from dataclasses import replace
-    first = replace(synth.shrink(synth.config2(), 700), seed=11)              # 5.5 row tiles per sequence, W4
-    second = replace(synth.shrink(synth.config3_layers()[5], 300), seed=12)   # other width and head size, fewer rows
+    first = replace(synth.shrink(synth.config3_layers()[10], 700), seed=11)   # C = 1280, 5.5 row tiles per sequence, Q~ int8
+    second = replace(synth.shrink(synth.config3_layers()[5], 300), seed=12, q_bits=0)   # C = 640, fewer rows, Q stays fp16
     for shape in (first, second):
         data, desc, P, mask, kv, x = _inputs(shape)
-        assert tb.taq_workspace_bytes(desc, 1) <= tb.taq_static_workspace_capacity()
+        assert 0 < tb.taq_workspace_bytes(desc, 1) <= tb.taq_static_workspace_capacity()
         want = tb.taq_layer_forward(desc, x, P["Wq"], P["Wout"], kv, mask)
         got = torch.full_like(want, float("nan"))
+        tb.taq_dispatch_reset()
         tb.taq_layer_forward_static(desc, x, P["Wq"], P["Wout"], kv, mask, got)
         tb.taq_poll_device_status()
+        ran = tb.taq_dispatch_counts()
+        # the pass went through the scratch: two dequant-GEMMs and the attention as separate kernels, none of them generic
+        assert ran["layer_fused"] == 0 and ran["linear_tensor"] == 2 and ran["attention_tensor"] == 1, ran
+        assert ran["linear_generic"] == 0 and ran["attention_generic"] == 0, ran
         # same kernels, same inputs, other scratch address: the outputs agree bit for bit, hence within the
         # layer tolerance used throughout (2e-2 max-abs, 1e-3 relative L2)
         tl.assert_layer_close(got.cpu().numpy(), want.cpu().numpy(), shape.name)
