@@ -27,10 +27,24 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 METRIC = "TAQ cross-attn queries/s per layer"
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/ (bytes); a
-# kernel that changed since its capture is listed as None.
-TRAFFIC = {"layer": 5804288}     # profiles/layer_c320_config2.md: 5.80 MB read, 0 written (Y was still in L2 when the capture ended)
 UNIT = "queries/s"
+
+
+def measured_traffic(kernel: str):
+    """DRAM bytes per launch (read + write) of `kernel` from the last ncu capture, as recorded by
+    `python -m paper_2603_22943_b200.profile_traffic`; None when there is no record or the kernel's source has changed
+    since the counters were taken."""
+    import hashlib
+    path = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    if not os.path.exists(path):
+        return None
+    rec = json.load(open(path)).get(kernel)
+    if not rec:
+        return None
+    src = os.path.join(ROOT, rec["source"])
+    if not os.path.exists(src) or hashlib.sha256(open(src, "rb").read()).hexdigest() != rec["source_sha256"]:
+        return None
+    return int(rec["dram_bytes_per_launch"])
 WORKLOAD = "config2: SD-1.5 64x64 cross-attn layer, B=2 N=4096 C=320 H=8 d=40 T=77 Dc=768, W4 g128, int8 Q/K/V rows, uint8 probs, fp16 trigger rows {4,5}"
 
 
@@ -55,7 +69,7 @@ class ClockSampler:
 
     def start(self):
         try:
-            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100", "-i", str(self.gpu)],
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "20", "-i", str(self.gpu)],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -150,6 +164,28 @@ def run_reference(args, shape, data):
     print(json.dumps(line), flush=True)
 
 
+def time_replays(torch, g, min_total_ms=400.0, min_replays=5, max_replays=20000):
+    """Replays a captured graph until at least `min_total_ms` of device time have been timed; every replay has its own
+    pair of CUDA events on the launching stream.  Returns the per-replay milliseconds: median, min, max, and the count."""
+    g.replay()
+    torch.cuda.synchronize()
+    times = []
+    total = 0.0
+    while (total < min_total_ms or len(times) < min_replays) and len(times) < max_replays:
+        n = 16 if times else 4
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
+        for a, b in evs:
+            a.record()
+            g.replay()
+            b.record()
+        torch.cuda.synchronize()
+        for a, b in evs:
+            t = a.elapsed_time(b)
+            times.append(t)
+            total += t
+    return {"median": statistics.median(times), "min": min(times), "max": max(times), "replays": len(times)}
+
+
 def _graph_time(torch, fn, count, replays):
     """Captures `count` calls of fn(i) into one CUDA graph and returns the milliseconds of one replay (device time)."""
     for i in range(min(count, 8)):
@@ -171,9 +207,85 @@ def _graph_time(torch, fn, count, replays):
     return a.elapsed_time(b) / replays
 
 
+def _layer_flops_bytes(tb, l):
+    """Algorithmic FLOPs and bytes of one layer pass (a3..a9): X in, Y out, the two packed weight matrices and the K~/V~
+    operand images once."""
+    rows = l.batch * l.n_query
+    flops = 4 * rows * l.channels * l.channels + 4 * rows * l.n_ctx * l.channels
+    desc = tb.layer_desc(l.batch, l.n_query, l.channels, l.heads, l.n_ctx, l.ctx_dim, l.w_bits, l.w_group, q_bits=l.q_bits, max_trigger=len(l.trigger))
+    wbytes = tb.taq_packed_weight_bytes(tb.weight_desc(l.channels, l.channels, l.w_bits, l.w_group))
+    nbytes = 2 * rows * l.channels * 2 + 2 * wbytes + tb.taq_kv_layout_of(desc).operand_head_bytes * l.heads * l.batch
+    return flops, nbytes
+
+
+def _bench_layers(torch, tb, synth, dev, layers, n_sets, steps):
+    """One step = taq_layer_forward on every layer of `layers`; every step uses another of `n_sets` buffer sets.  Returns
+    the replay statistics (ms per step), launches per step by kernel family, and the per-step bytes of a buffer set."""
+    sets = []
+    for k in range(n_sets):
+        L = []
+        for shp in layers:
+            data = synth.make_layer(shp)
+            desc = tb.layer_desc(shp.batch, shp.n_query, shp.channels, shp.heads, shp.n_ctx, shp.ctx_dim, shp.w_bits, shp.w_group,
+                                 q_bits=shp.q_bits, max_trigger=len(shp.trigger))
+            wd_cc = tb.weight_desc(shp.channels, shp.channels, shp.w_bits, shp.w_group)
+            wd_cd = tb.weight_desc(shp.channels, shp.ctx_dim, shp.w_bits, shp.w_group)
+            mask = dev(data["mask"])
+            kv = tb.taq_kv_project(desc, dev(data["ctx"]), tb.taq_pack_weights(wd_cd, dev(data["Wk"])), tb.taq_pack_weights(wd_cd, dev(data["Wv"])), mask)
+            L.append((desc, dev(np.roll(data["X"], k, axis=1)), tb.taq_pack_weights(wd_cc, dev(data["Wq"])),
+                      tb.taq_pack_weights(wd_cc, dev(data["Wout"]), dev(data["bout"])), kv, mask,
+                      torch.empty((shp.batch, shp.n_query, shp.channels), dtype=torch.float16, device="cuda"),
+                      torch.empty(tb.taq_workspace_bytes(desc, 1), dtype=torch.uint8, device="cuda")))
+        sets.append(L)
+    tb.taq_poll_device_status()
+
+    def step(i):
+        for (desc, x, Wq, Wo, kv, mask, y, ws) in sets[i % n_sets]:
+            tb.taq_layer_forward(desc, x, Wq, Wo, kv, mask, y, ws)
+
+    for i in range(min(steps, 8)):
+        step(i)
+    torch.cuda.synchronize()
+    tb.taq_dispatch_reset()
+    step(0)
+    per_step = tb.taq_dispatch_counts()
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=torch.cuda.Stream()):
+        for i in range(steps):
+            step(i)
+    rep = time_replays(torch, g)
+    tb.taq_poll_device_status()
+    return {k: v / steps for k, v in rep.items() if k != "replays"} | {"replays": rep["replays"]}, per_step
+
+
+def _workload_line(metric, workload, layers, ms, rep, per_step, steps, n_sets, peaks, clocks, tb, bound):
+    rows = sum(l.batch * l.n_query for l in layers)
+    fb = [_layer_flops_bytes(tb, l) for l in layers]
+    flops, nbytes = sum(f for f, _ in fb), sum(b for _, b in fb)
+    tf, gbs = flops / (ms * 1e-3) / 1e12, nbytes / (ms * 1e-3) / 1e9
+    launches = sum(per_step.values())
+    roof = {"bound": bound, "traffic": None, "flops_per_step": flops, "bytes_per_step": nbytes,
+            "tensor": {"achieved_TFLOPs": tf, "peak_TFLOPs": peaks["bf16_tflops"], "frac": tf / peaks["bf16_tflops"]},
+            "hbm": {"achieved_GBps": gbs, "peak_GBps": peaks["hbm_gbs"], "frac": gbs / peaks["hbm_gbs"]},
+            "peak_source": peaks["source"]}
+    if bound == "tensor":
+        roof.update({"achieved": tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": tf / peaks["bf16_tflops"]})
+    else:
+        roof.update({"achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"]})
+    return {"metric": metric, "value": rows / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": steps, "warmup": 8, "ms_per_step": ms,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f16", "data": "synthetic",
+            "config": {"workload": workload, "launch": "one CUDA graph of the steps, replayed until 0.4 s are timed; value = median replay",
+                       "l2_policy": f"ring of {n_sets} buffer sets ({n_sets * nbytes / 1e6:.0f} MB of activations and weights)"},
+            "timing": {"replays": rep["replays"], "ms_per_step_min": rep["min"], "ms_per_step_max": rep["max"]},
+            "kernel_launches_per_step": per_step, "generic_kernel_launches": per_step["linear_generic"] + per_step["attention_generic"],
+            "clocks": clocks, "gpu_launches": launches * steps, "roofline": roof}
+
+
 def run_other_workload(args):
-    """The other measured configurations (not the headline line): `config3`, one SD-1.5 UNet step of all 16
-    cross-attention layers; `config5`, the multi-checkpoint serving sweep on the 64x64 layer.  One GPU."""
+    """The other measured configurations (not the headline line): `config1`, the SD-1.5 lowest-resolution layer (W8);
+    `config3`, one SD-1.5 UNet step of all 16 cross-attention layers; `config4`, the two SDXL-shaped layers (one line
+    each); `config5`, the multi-checkpoint serving sweep on the 64x64 layer.  One GPU."""
     import torch
     from paper_2603_22943_b200 import binding as tb
     from paper_2603_22943_b200 import synth
@@ -181,50 +293,30 @@ def run_other_workload(args):
     tb.lib()
     peaks = _peaks()
     dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    l2 = torch.cuda.get_device_properties(0).L2_cache_size
     sampler = ClockSampler(0)
     sampler.start()
-    if args.workload == "config3":
-        layers = synth.config3_layers()
-        n_sets = 3                                    # 3 x 108 MB of activations per step > 2 x L2
-        sets = []
-        for k in range(n_sets):
-            L = []
-            for shp in layers:
-                data = synth.make_layer(shp)
-                desc = tb.layer_desc(shp.batch, shp.n_query, shp.channels, shp.heads, shp.n_ctx, shp.ctx_dim, shp.w_bits, shp.w_group,
-                                     q_bits=shp.q_bits, max_trigger=len(shp.trigger))
-                wd_cc = tb.weight_desc(shp.channels, shp.channels, shp.w_bits, shp.w_group)
-                wd_cd = tb.weight_desc(shp.channels, shp.ctx_dim, shp.w_bits, shp.w_group)
-                mask = dev(data["mask"])
-                kv = tb.taq_kv_project(desc, dev(data["ctx"]), tb.taq_pack_weights(wd_cd, dev(data["Wk"])), tb.taq_pack_weights(wd_cd, dev(data["Wv"])), mask)
-                L.append((desc, dev(np.roll(data["X"], k, axis=1)), tb.taq_pack_weights(wd_cc, dev(data["Wq"])),
-                          tb.taq_pack_weights(wd_cc, dev(data["Wout"]), dev(data["bout"])), kv, mask,
-                          torch.empty((shp.batch, shp.n_query, shp.channels), dtype=torch.float16, device="cuda"),
-                          torch.empty(tb.taq_workspace_bytes(desc, 1), dtype=torch.uint8, device="cuda")))
-            sets.append(L)
-        tb.taq_poll_device_status()
-
-        def step(i):
-            for (desc, x, Wq, Wo, kv, mask, y, ws) in sets[i % n_sets]:
-                tb.taq_layer_forward(desc, x, Wq, Wo, kv, mask, y, ws)
-
-        steps = max(6, min(args.steps, 60))
-        ms = _graph_time(torch, step, steps, 3) / steps
-        rows = sum(l.batch * l.n_query for l in layers)
-        flops = sum(4 * l.batch * l.n_query * l.channels * l.channels + 4 * l.batch * l.n_query * l.n_ctx * l.channels for l in layers)
-        nbytes = sum(2 * l.batch * l.n_query * l.channels * 2 for l in layers)
-        tb.taq_poll_device_status()
-        line = {"metric": "TAQ cross-attn queries/s over one SD-1.5 UNet step (16 layers)", "value": rows / (ms * 1e-3), "unit": UNIT, "n_gpus": 1,
-                "steps": steps, "warmup": 8, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f16",
-                "data": "synthetic",
-                "config": {"workload": "config3: all 16 SD-1.5 cross-attn layers (5x(N=4096,C=320), 5x(1024,640), 5x(256,1280), 1x(64,1280)), B=2, T=77, W4 g128, trigger {4,5}",
-                           "launch": "one CUDA graph of the steps; C=320 layers: one kernel each, other layers: three kernels each",
-                           "l2_policy": f"ring of {n_sets} buffer sets ({n_sets * nbytes / 1e6:.0f} MB of activations)"},
-                "clocks": sampler.stop(), "gpu_launches": steps * (5 + 11 * 3),
-                "roofline": {"bound": "tensor", "achieved": flops / (ms * 1e-3) / 1e12, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                             "frac": flops / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"], "traffic": None,
-                             "hbm": {"achieved_GBps": nbytes / (ms * 1e-3) / 1e9, "peak_GBps": peaks["hbm_gbs"]}}}
-        print(json.dumps(line), flush=True)
+    if args.workload in ("config1", "config3", "config4"):
+        if args.workload == "config1":
+            cases = [("TAQ cross-attn queries/s per layer", "config1: SD-1.5 8x8 cross-attn layer, B=1 N=64 C=1280 H=8 d=160 T=77 Dc=768, W8 per-channel, trigger {5}",
+                      [synth.config1()], "hbm")]
+        elif args.workload == "config4":
+            cases = [("TAQ cross-attn queries/s per layer", f"config4: SDXL-shaped cross-attn layer, B=2 N={l.n_query} C={l.channels} H={l.heads} d=64 T=77 Dc=2048, W4 g128, trigger {{3,4,5}}",
+                      [l], "tensor") for l in synth.config4_layers()]
+        else:
+            cases = [("TAQ cross-attn queries/s over one SD-1.5 UNet step (16 layers)",
+                      "config3: all 16 SD-1.5 cross-attn layers (5x(N=4096,C=320), 5x(1024,640), 5x(256,1280), 1x(64,1280)), B=2, T=77, W4 g128, trigger {4,5}",
+                      synth.config3_layers(), "tensor")]
+        lines = []
+        for metric, workload, layers, bound in cases:
+            set_bytes = sum(_layer_flops_bytes(tb, l)[1] for l in layers)
+            n_sets = max(3, int(np.ceil(2.2 * l2 / set_bytes)))
+            steps = max(n_sets, min(args.steps, 96 if set_bytes < 20e6 else 12))
+            rep, per_step = _bench_layers(torch, tb, synth, dev, layers, n_sets, steps)
+            lines.append((metric, workload, layers, rep, per_step, steps, n_sets, bound))
+        clocks = sampler.stop()
+        for metric, workload, layers, rep, per_step, steps, n_sets, bound in lines:
+            print(json.dumps(_workload_line(metric, workload, layers, rep["median"], rep, per_step, steps, n_sets, peaks, clocks, tb, bound)), flush=True)
         return
     # config5: 64 checkpoints resident, requests routed to random checkpoints, the N=4096 x C=320 layer
     n_ckpt, N, C_, H, T, Dc = 64, 4096, 320, 8, 77, 768
@@ -260,17 +352,33 @@ def run_other_workload(args):
             tb.taq_layer_forward_batched(desc1, tables[g], nb, x_all[g * nb:(g + 1) * nb], y_all[g * nb:(g + 1) * nb], ws)
 
         count = max(groups, 16)
-        ms = _graph_time(torch, step, count, 5) / count
-        results.append({"requests_per_batch": nb, "ms_per_batch": round(ms, 5), "requests_per_s": nb / (ms * 1e-3), "queries_per_s": nb * N / (ms * 1e-3)})
+        for i in range(min(count, 8)):
+            step(i)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=torch.cuda.Stream()):
+            for i in range(count):
+                step(i)
+        rep = time_replays(torch, g, min_total_ms=200.0)
+        ms = rep["median"] / count
+        flops = nb * (4 * N * C_ * C_ + 4 * N * T * C_)
+        results.append({"requests_per_batch": nb, "ms_per_batch": round(ms, 5), "ms_per_batch_min": round(rep["min"] / count, 5), "ms_per_batch_max": round(rep["max"] / count, 5),
+                        "requests_per_s": nb / (ms * 1e-3), "queries_per_s": nb * N / (ms * 1e-3),
+                        "TFLOP/s": flops / (ms * 1e-3) / 1e12, "frac_of_tensor_peak": flops / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"]})
     tb.taq_poll_device_status()
     best = results[-1]
+    kvl = tb.taq_kv_layout_of(desc1)
     line = {"metric": "TAQ multi-checkpoint serving, requests/s on the N=4096 x C=320 layer", "value": best["requests_per_s"], "unit": "requests/s", "n_gpus": 1,
             "steps": 16, "warmup": 8, "ms_per_step": best["ms_per_batch"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f16",
             "data": "synthetic",
             "config": {"workload": "config5: 64 synthetic checkpoints resident (packed W4 g128), each request routed to a random checkpoint with its own weights, K~/V~ and trigger span (1-3 tokens)",
                        "launch": "one kernel per batch (grid.z = request), batches rotate over 64 resident request slots (168 MB of activations)",
-                       "packed_bytes_per_checkpoint_all_16_layers": per_ckpt_all_layers, "fp16_bytes_per_checkpoint_all_16_layers": int(per_ckpt_all_layers / 4.25 * 16)},
-            "sweep": results, "clocks": sampler.stop(), "gpu_launches": 16}
+                       "packed_bytes_per_checkpoint_all_16_layers": per_ckpt_all_layers, "fp16_bytes_per_checkpoint_all_16_layers": int(per_ckpt_all_layers / 4.25 * 16),
+                       "kv_bytes_per_prompt_this_layer": kvl.block_bytes,
+                       "kv_bytes_per_prompt_this_layer_without_operand_images": kvl.block_bytes - kvl.operand_head_bytes * H},
+            "sweep": results, "clocks": sampler.stop(), "gpu_launches": 16,
+            "roofline": {"bound": "tensor", "achieved": best["TFLOP/s"], "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": best["frac_of_tensor_peak"],
+                         "traffic": None, "peak_source": peaks["source"]}}
     print(json.dumps(line), flush=True)
 
 
@@ -285,8 +393,8 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=10.0, help="CPU time to spend on the cpu_baseline sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--n-query", type=int, default=0, help="override N (profiling on a smaller case)")
-    ap.add_argument("--workload", default="config2", choices=["config2", "config3", "config5"],
-                    help="config2 (default) is the headline line; config3 / config5 print the other measured configurations")
+    ap.add_argument("--workload", default="config2", choices=["config1", "config2", "config3", "config4", "config5"],
+                    help="config2 (default) is the headline line; the others print the other measured configurations (config4: one line per SDXL layer)")
     args = ap.parse_args()
     if args.workload != "config2":
         run_other_workload(args)
@@ -387,12 +495,11 @@ def main():
     barrier()
     sampler = ClockSampler(local_rank)
     sampler.start()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    g_steps.replay()
-    e1.record()
+    # The graph of exactly K steps is replayed until about 0.4 s of device time have been timed, every replay between its
+    # own pair of CUDA events; the reported step time is the median replay divided by K (minimum and maximum beside it).
+    rep = time_replays(torch, g_steps)
     barrier()
-    ms_total = e0.elapsed_time(e1)
+    ms_total = rep["median"]
 
     # A step is one launch (the whole layer pass in one kernel), so the step time is that kernel's launch duration.  For
     # comparison the stand-alone entry points (fused to_q + attention, and to_q / attention / to_out as separate kernels)
@@ -491,7 +598,7 @@ def main():
     e2e_ms = f0.elapsed_time(f1)
     tb.taq_poll_device_status()
 
-    ms_total, e2e_ms = max_over_ranks([ms_total, e2e_ms], dist, "cuda")
+    ms_total, e2e_ms, ms_min, ms_max = max_over_ranks([ms_total, e2e_ms, rep["min"], rep["max"]], dist, "cuda")
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
@@ -506,9 +613,9 @@ def main():
     qbytes = M * C_ * (1 if shape.q_bits == 8 else 2) + (M * H * 4 if shape.q_bits == 8 else 0)
     img_bytes = tb.taq_kv_layout_of(desc).operand_head_bytes * H * B
     kernels = [
-        {"name": "qattn_c320_kernel<.,true>: the whole layer pass in one kernel (taq_layer_forward)", "ms": ms_per_step, "in_step": True,
-         "bytes": 2 * M * C_ * 2 + 2 * wbytes + img_bytes, "flops": 4 * M * C_ * C_ + 4 * M * T * C_, "traffic": TRAFFIC.get("layer")},
-        {"name": "qattn_c320_kernel<.,false>: to_q + Q_a + attention, stand-alone (taq_query_attention)", "ms": stage_ms["qattn"], "in_step": False,
+        {"name": "layer_c320_kernel<.,true>: the whole layer pass in one kernel (taq_layer_forward)", "ms": ms_per_step, "in_step": True,
+         "bytes": 2 * M * C_ * 2 + 2 * wbytes + img_bytes, "flops": 4 * M * C_ * C_ + 4 * M * T * C_, "traffic": measured_traffic("layer_c320_kernel")},
+        {"name": "layer_c320_kernel<.,false>: to_q + Q_a + attention, stand-alone (taq_query_attention)", "ms": stage_ms["qattn"], "in_step": False,
          "bytes": 2 * M * C_ * 2 + wbytes + img_bytes, "flops": 2 * M * C_ * C_ + 4 * M * T * C_, "traffic": None},
         {"name": "linear_sm100_kernel<160>: to_out dequant-GEMM, stand-alone (taq_quantized_linear)", "ms": stage_ms["to_out"], "in_step": False,
          "bytes": 2 * M * C_ * 2 + wbytes, "flops": 2 * M * C_ * C_, "traffic": None},
@@ -532,11 +639,15 @@ def main():
                 "flops_per_launch": dom["flops"], "bytes_per_launch": dom["bytes"], "ms_per_launch": dom["ms"],
                 "hbm": {"achieved_GBps": dom["GB/s"], "peak_GBps": peaks["hbm_gbs"], "frac": dom["GB/s"] / peaks["hbm_gbs"]},
                 "stages": [{"name": k["name"], "in_step": k["in_step"], "ms": round(k["ms"], 5), "GB/s": round(k["GB/s"], 1), "TFLOP/s": round(k["TFLOP/s"], 2)} for k in kernels]}
+    sm_mhz = clocks.get("sm_mhz") or 0.0
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f16",
             "data": "synthetic",
+            "timing": {"replays": rep["replays"], "ms_per_step_median": ms_per_step, "ms_per_step_min": ms_min / args.steps, "ms_per_step_max": ms_max / args.steps,
+                       "us_x_sm_mhz": ms_per_step * 1e3 * sm_mhz,
+                       "note": "each replay is one CUDA graph of exactly `steps` steps between its own pair of CUDA events; value = median replay"},
             "config": {"workload": WORKLOAD if not args.n_query else WORKLOAD + f" (N overridden to {N})", "kv_projection": "once per prompt, outside the step",
-                       "launch": "the K timed steps are one CUDA graph (one kernel launch per step: the whole layer pass)",
+                       "launch": "the K timed steps are one CUDA graph (one kernel launch per step: the whole layer pass), replayed until 0.4 s are timed",
                        "l2_policy": f"inputs larger than L2: ring of {n_sets} buffer sets ({n_sets * set_bytes / 1e6:.0f} MB of activations, L2 {l2 / 1e6:.0f} MB)",
                        "replicas": world},
             "clocks": clocks,
