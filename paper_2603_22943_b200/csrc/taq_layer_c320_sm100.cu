@@ -6,24 +6,26 @@
 // cluster and exchange their halves of O through distributed shared memory.  Warps: 0 producer (TMA / bulk copies),
 // 1 MMA issuer, 2..17 workers.  A worker thread is (row r, head hi) from start to end:
 //   phase 1  Q = X Wq^T for the CTA's 160 channels: workers expand the packed 4-bit codes to fp16-integer operand tiles
-//            (ring of three), one TMEM accumulator per scale group, folded into registers with the group's scales;
+//            (all five K blocks, before X has arrived), one TMEM accumulator per scale group, folded into registers with
+//            the group's scales;
 //   phase 2  the thread quantizes its 40 values (one head of one row) into the head's Q~ operand tile; the row scale
 //            stays in a register;
 //   phase 3  all four heads at once: four S accumulators (4 x 80 columns) and four O accumulators (4 x 48) fill the 512
 //            TMEM columns.  The thread that quantized (r, hi) also owns that row's 80 scores: maximum, exponentials, sum
 //            and Eq. 3 need no exchange between threads.  P (fp16 integers in units of 1/255, trigger columns fp16)
 //            overwrites the head's Q~ tile (keys 0..63) plus a 32-byte-swizzled tail tile (keys 64..79);
-//   phase 4  to_out for the CTA's 160 output channels over all 320 channels of O.  Each CTA writes its heads' O as
-//            32-channel operand tiles and sends them to its partner; the K steps over its own tiles run while the
-//            partner's are in flight (rank 0 walks the K blocks upwards, rank 1 downwards, so each begins with its own
-//            channels and every scale group still has its own accumulator).  The Wout tiles are expanded during phase
-//            3 into the dead K~ buffers, later into the dead V~^T buffers.  Y leaves as one TMA tensor store per head
-//            group of 40 channels.
-// Shared memory is reused: X tile -> Q~ / P tiles -> O tiles -> Y staging; weight ring -> V~^T tiles -> weight ring.
+//   phase 4  to_out for the CTA's 160 output channels over all 320 channels of O.  Each head's O goes, as soon as its own
+//            PV product is complete, into 32-channel operand tiles placed where only probability tiles of heads already
+//            finished lie; every tile is sent to the partner CTA as soon as it is complete.  The K steps over the CTA's
+//            own tiles run while the partner's are in flight (each CTA begins with its own channels; every scale group
+//            still has its own accumulator).  The Wout tiles are expanded during phase 3 into the dead K~ buffers, later
+//            into the dead V~^T buffers.  Y leaves as one TMA tensor store per head group of 40 channels.
+// Shared memory is reused: X tile -> Q~ / P tiles -> O tiles -> Y staging; weight tiles -> K~ and V~^T tiles -> weight ring.
 #include "taq_ptx.cuh"
 #include "taq_sm100.cuh"
 #include "taq_sm100_parts.cuh"
 #include "taq_prof.cuh"
+#include <type_traits>
 
 TAQ_PROF_DEFINE(layer)
 
@@ -68,15 +70,24 @@ static_assert(HG * K_BYTES == 2 * B_TILE, "the K~ tiles are exactly two ring sta
 static_assert(HG * Y_STAGE <= NKB * A_TILE, "Y staging fits into the X tile");
 static_assert(NQ * MAX_GROUPS * 4 <= SCALE_BYTES, "scale table");
 
-constexpr int NS1 = 3, NS4 = 4;                 // ring stages of phase 1 and of phase 4
-__device__ __forceinline__ int stage4_offset(int s) { return s < 2 ? OFF_K + s * B_TILE : OFF_R1 + (s - 2) * B_TILE; }
+constexpr int NS4 = 4;                          // ring stages of phase 4
+constexpr int NEXP = NWORK - NWORK / HG;        // worker threads that expand the Wout tiles: the warps of heads 0..2
+// Phase 1 keeps all five expanded Wq tiles: three in region 1, two where the K~ tiles arrive afterwards.
+__device__ __forceinline__ int stage1_offset(int kb) { return kb < 3 ? OFF_R1 + kb * B_TILE : OFF_K + (kb - 3) * B_TILE; }
+__host__ __device__ constexpr int stage4_offset(int s) { return s < 2 ? OFF_K + s * B_TILE : OFF_R1 + (s - 2) * B_TILE; }
+// O tiles of phase 4 inside region 0.  A CTA's own tile lt (0..4, 32 channels each) is written by heads lt - 1 and lt and
+// lies in the probability tile of head max(lt - 1, 0), dead by then (PV products complete in head order); the partner's
+// five tiles arrive, once every PV product of this CTA is complete, in the second halves of the other probability tiles
+// and in the tail tiles.
+__host__ __device__ constexpr int own_tile_offset(int lt) { return OFF_R0 + (lt < 2 ? lt * O_TILE : (lt - 1) * A_TILE); }
+__host__ __device__ constexpr int peer_tile_offset(int lt) { return OFF_R0 + (lt < 3 ? (lt + 1) * A_TILE + O_TILE : HG * A_TILE + (lt - 3) * O_TILE); }
 
 struct Misc {
     uint64_t a_full[NKB], w_full, w2_full, kc_full, vt_full;
-    uint64_t b1_full[NS1], b1_empty[NS1], b4_full[NS4], b4_empty[NS4];
+    uint64_t b1_full[NKB], b4_full[NKB], b4_empty[NS4], tile_done[N_OTILE / 2];       // b4_full: one per Wout tile of the walk
     uint64_t acc_full[MAX_GROUPS];
     uint64_t q_all, s_full[HG], p_full[HG], o_full[HG];
-    uint64_t o_own, o_all, peer_ready, peer_got, drain;
+    uint64_t o_all, peer_ready, peer_got, drain;
     uint32_t tmem_base;
     volatile int abort_flag;
 };
@@ -98,6 +109,25 @@ struct LayerArgs {
     long long wait_cycles;      // limit of every device-side wait
     int* status;
 };
+
+// The same by the first NT worker threads only (phase 4: the warps of the last head, whose probabilities are the last to
+// be complete, take no part, so that the tiles do not wait for them).
+template <int NT>
+__device__ __forceinline__ void expand_block_by(const unsigned char* raw, int kb, unsigned char* b_tile, int t) {
+    constexpr int NCH = (NQ * 8 + NT - 1) / NT;
+    uint32_t pw[NCH];
+#pragma unroll
+    for (int i = 0; i < NCH; ++i) {
+        const int id = t + NT * i;
+        pw[i] = 0;
+        if (id < NQ * 8) pw[i] = *reinterpret_cast<const uint32_t*>(raw + (id >> 3) * (KIN / 2) + kb * (BK / 2) + (id & 7) * 4);
+    }
+#pragma unroll
+    for (int i = 0; i < NCH; ++i) {
+        const int id = t + NT * i;
+        if (id < NQ * 8) *reinterpret_cast<uint4*>(b_tile + ptx::sw128_offset(id >> 3, id & 7)) = codes_w4_to_half(pw[i]);
+    }
+}
 
 // Expands one 64-wide K block of the packed 4-bit codes at OFF_RAW into a tile of fp16 integers (all worker threads).
 __device__ __forceinline__ void expand_block(const unsigned char* raw, int kb, unsigned char* b_tile, int wt) {
@@ -122,7 +152,10 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
 
 // The softmax of one thread's row over all TP keys: raw scores u (integer dot products) -> e_j = 2^(u_j f_j sq - m)
 // with the row's own maximum m (log2 units); returns their sum.  Keys at or beyond T get weight exactly 0.
-template <bool TAIL_ONLY>
+// The softmax of one thread's row over all TP keys: raw scores u (integer dot products) -> e_j = 2^(u_j f_j sq - m)
+// with the row's own maximum m (log2 units); returns their sum.  Keys at or beyond T get weight exactly 0; only keys from
+// TAIL_FROM on can be such keys (the launcher picks TAIL_FROM <= T).
+template <int TAIL_FROM>
 __device__ __forceinline__ float softmax_row(const uint32_t (&u)[TP], float (&e)[TP], const float* factor, float sq, int T, float& msq_out) {
     float m4[4] = {-1e30f, -1e30f, -1e30f, -1e30f};          // finite floor
 #pragma unroll
@@ -133,7 +166,7 @@ __device__ __forceinline__ float softmax_row(const uint32_t (&u)[TP], float (&e)
         for (int i = 0; i < 8; ++i) {
             const int j = 8 * j8 + i;
             e[j] = __uint_as_float(u[j]) * f[i];
-            if (j >= 64 || !TAIL_ONLY) { if (j >= T) e[j] = -INFINITY; }
+            if (j >= TAIL_FROM) { if (j >= T) e[j] = -INFINITY; }
         }
 #pragma unroll
         for (int i = 0; i < 4; ++i) m4[i] = max3(m4[i], e[8 * j8 + i], e[8 * j8 + 4 + i]);
@@ -144,7 +177,7 @@ __device__ __forceinline__ float softmax_row(const uint32_t (&u)[TP], float (&e)
 #pragma unroll
     for (int j = 0; j < TP; ++j) {
         float arg = fmaf(e[j], sq, -msq);
-        if (j >= 64 || !TAIL_ONLY) { if (j >= T) arg = -INFINITY; }      // also when sq = 0
+        if (j >= TAIL_FROM) { if (j >= T) arg = -INFINITY; }      // also when sq = 0
         e[j] = ex2_approx(arg);
     }
     float sum4[4] = {0.f, 0.f, 0.f, 0.f};
@@ -178,26 +211,57 @@ __device__ __forceinline__ void write_p_row(const float (&e)[TP], float k, unsig
 
 // Eq. 3, trigger columns: the probability stays fp16, fp16(e_j k).  A row has at most a few of them, at positions only
 // known at run time, so they are not carried through the unrolled code above: e_j is computed once more from the score
-// in TMEM with the same instructions (hence the same value) and the two bytes of the code are overwritten.  The loop
-// is warp-uniform (`trig` is the same for all rows of a head).
+// in TMEM with the same instructions (hence the same value) and the two bytes of the code are overwritten.  Up to four
+// columns are fetched per round trip to TMEM.  The loop is warp-uniform (`trig` is the same for all rows of a head).
 __device__ __forceinline__ void trigger_columns(const uint32_t (&trig)[3], uint32_t t_s, const float* factor, float sq, float msq, float k,
                                                 unsigned char* p_tile, unsigned char* p_tail, int r) {
 #pragma unroll 1
     for (int w = 0; w < 3; ++w) {
         uint32_t bits = trig[w];
         while (bits) {
-            const int j = w * 32 + __ffs(bits) - 1;
-            bits &= bits - 1;
-            if (j >= TP) break;
-            const float t = __uint_as_float(ptx::tmem_ld1_wait(t_s + j)) * factor[j];
-            const float ej = ex2_approx(fmaf(t, sq, -msq));
-            unsigned char* dst = j < 64 ? p_tile + ptx::sw128_offset(r, j >> 3) : p_tail + ptx::sw32_offset(r, (j - 64) >> 3);
-            *reinterpret_cast<__half*>(dst + (j & 7) * 2) = __float2half_rn(ej * k);
+            int jj[4];
+            uint32_t v[4];
+            int n = 0;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                jj[i] = 0;
+                if (bits) {
+                    const int j = w * 32 + __ffs(bits) - 1;
+                    bits &= bits - 1;
+                    if (j < TP) { jj[i] = j; n = i + 1; }
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                if (i < n) v[i] = ptx::tmem_ld1(t_s + jj[i]);
+            ptx::tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                if (i < n) {
+                    const int j = jj[i];
+                    asm volatile("" : "+r"(v[i]));
+                    const float t = __uint_as_float(v[i]) * factor[j];
+                    const float ej = ex2_approx(fmaf(t, sq, -msq));
+                    unsigned char* dst = j < 64 ? p_tile + ptx::sw128_offset(r, j >> 3) : p_tail + ptx::sw32_offset(r, (j - 64) >> 3);
+                    *reinterpret_cast<__half*>(dst + (j & 7) * 2) = __float2half_rn(ej * k);
+                }
         }
     }
 }
 
-template <bool TAIL_ONLY, bool FUSE_OUT>
+// The walk of phase 4 over the five 64-wide K blocks of O: each CTA starts with the channels of its own heads.
+//   rank 0: blocks 0, 1, first half of 2 | second half of 2, 3, 4        rank 1: second half of 2, 3, 4 | first half of 2, 1, 0
+// Step i of six: K block, which 32-channel halves, and (walk_tile) the order in which the Wout tiles are needed.
+__host__ __device__ constexpr int walk_block(int rank, int i) { return rank ? (i < 3 ? 2 + i : 5 - i) : (i < 3 ? i : i - 1); }
+__host__ __device__ constexpr int walk_halves(int rank, int i) { return i == 2 - 2 * rank ? (rank ? 2 : 1) : i == 3 ? (rank ? 1 : 2) : 3; }     // bit 0: first half, bit 1: second half
+__host__ __device__ constexpr int walk_tile(int rank, int n) { return rank ? (n < 3 ? 2 + n : 4 - n) : n; }            // n-th Wout tile to expand
+// Ring stage of a K block's Wout tile: the first four tiles of the walk take stages 0..3, the fifth reuses the stage of a
+// tile whose last use comes early (rank 0: block 0, stage 0; rank 1: block 3, stage 1).
+__host__ __device__ constexpr int walk_stage(int rank, int kb) { return rank ? (kb >= 2 ? kb - 2 : kb == 1 ? 3 : 1) : (kb < 4 ? kb : 0); }
+__host__ __device__ constexpr int walk_reuse_stage(int rank) { return rank ? 1 : 0; }
+__host__ __device__ constexpr int walk_order(int rank, int kb) { return rank ? (kb >= 2 ? kb - 2 : 4 - kb) : kb; }        // inverse of walk_tile
+
+template <int TAIL_FROM, bool FUSE_OUT>
 __global__ void __launch_bounds__(NTHREADS, 1) layer_c320_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_y, const LayerArgs a) {
     extern __shared__ unsigned char smem_dyn[];
     unsigned char* smem = smem_dyn + ((1024u - (ptx::smem_u32(smem_dyn) & 1023u)) & 1023u);   // 1024-byte aligned
@@ -218,13 +282,13 @@ __global__ void __launch_bounds__(NTHREADS, 1) layer_c320_kernel(const __grid_co
     TAQ_PROF_INIT
     if (tid == 0) { TAQ_PROF(0); TAQ_GPROF(30); }
     if (tid == 0) {
-        for (int i = 0; i < NKB; ++i) ptx::mbar_init(&misc->a_full[i], 1);
+        for (int i = 0; i < NKB; ++i) { ptx::mbar_init(&misc->a_full[i], 1); ptx::mbar_init(&misc->b1_full[i], NWORK / 32); }
         ptx::mbar_init(&misc->w_full, 1);
         ptx::mbar_init(&misc->w2_full, 1);
         ptx::mbar_init(&misc->kc_full, 1);
         ptx::mbar_init(&misc->vt_full, 1);
-        for (int i = 0; i < NS1; ++i) { ptx::mbar_init(&misc->b1_full[i], NWORK / 32); ptx::mbar_init(&misc->b1_empty[i], 1); }
-        for (int i = 0; i < NS4; ++i) { ptx::mbar_init(&misc->b4_full[i], NWORK / 32); ptx::mbar_init(&misc->b4_empty[i], 1); }
+        for (int i = 0; i < NKB; ++i) ptx::mbar_init(&misc->b4_full[i], NEXP / 32);
+        for (int i = 0; i < NS4; ++i) ptx::mbar_init(&misc->b4_empty[i], 1);
         for (int i = 0; i < MAX_GROUPS; ++i) ptx::mbar_init(&misc->acc_full[i], 1);
         ptx::mbar_init(&misc->q_all, NWORK / 32);
         for (int i = 0; i < HG; ++i) {
@@ -232,7 +296,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) layer_c320_kernel(const __grid_co
             ptx::mbar_init(&misc->p_full[i], NWORK / 32 / HG);     // the four warps of the head
             ptx::mbar_init(&misc->o_full[i], 1);
         }
-        ptx::mbar_init(&misc->o_own, NWORK / 32);
+        for (int lt = 0; lt < N_OTILE / 2; ++lt)                   // the warps of the one or two heads that write the tile
+            ptx::mbar_init(&misc->tile_done[lt], (lt == 0 || lt == HG ? 1 : 2) * (NWORK / 32 / HG));
         ptx::mbar_init(&misc->o_all, 1);
         ptx::mbar_init(&misc->peer_ready, 1);
         ptx::mbar_init(&misc->peer_got, 1);
@@ -249,7 +314,10 @@ __global__ void __launch_bounds__(NTHREADS, 1) layer_c320_kernel(const __grid_co
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = misc->tmem_base;
     ptx::pdl_trigger();
-    if (FUSE_OUT) ptx::cluster_sync_all();                   // the partner's barriers exist before anything arrives on them
+    // The partner's barriers must exist before anything arrives on them.  Every thread arrives at the cluster barrier
+    // here and waits on it much later, right before its warp's first operation on the partner's shared memory (or at
+    // the end), so that the barrier's latency stays off the start of the kernel.
+    if (FUSE_OUT) ptx::cluster_arrive();
     const uint32_t peer = FUSE_OUT ? (ptx::cluster_ctarank() ^ 1u) : 0u;
 
     const taq_kv_layout KL = kv_layout(H, T, D, a.max_trigger);
@@ -273,74 +341,84 @@ __global__ void __launch_bounds__(NTHREADS, 1) layer_c320_kernel(const __grid_co
             }
             const uint8_t* blk = a.reqs ? (const uint8_t*)a.reqs[zb].kv : (const uint8_t*)a.kv + (size_t)zb * KL.block_bytes;
             const uint8_t* img = blk + KL.off_operands + (size_t)h_begin * KL.operand_head_bytes;
-            ptx::mbar_arrive_expect_tx(&misc->kc_full, HG * (K_BYTES + kOperandConstBytes));
-            for (int hi = 0; hi < HG; ++hi) {
-                ptx::bulk_load(smem + OFF_K + hi * K_BYTES, img + (size_t)hi * KL.operand_head_bytes, K_BYTES, &misc->kc_full);
-                ptx::bulk_load(smem + OFF_CST + hi * kOperandConstBytes, img + (size_t)hi * KL.operand_head_bytes + K_BYTES + VT_BYTES, kOperandConstBytes, &misc->kc_full);
-            }
-            // Phase 1 over (every MMA complete, hence every Wq tile expanded): the ring becomes the V~^T tiles and the packed
-            // Wout rows of this CTA's output channels replace the packed Wq rows.
+            // Phase 1 over (every MMA complete, hence every Wq tile read): the weight tiles become the K~ and V~^T tiles and
+            // the packed Wout rows of this CTA's output channels replace the packed Wq rows.
             bool ok = ptx::mbar_wait(&misc->acc_full[n_groups - 1], 0, WL) && !misc->abort_flag;
-            bool vt_issued = false, w2_issued = false;
             if (ok) {
+                ptx::mbar_arrive_expect_tx(&misc->kc_full, HG * (K_BYTES + kOperandConstBytes));
+                for (int hi = 0; hi < HG; ++hi) {
+                    ptx::bulk_load(smem + OFF_K + hi * K_BYTES, img + (size_t)hi * KL.operand_head_bytes, K_BYTES, &misc->kc_full);
+                    ptx::bulk_load(smem + OFF_CST + hi * kOperandConstBytes, img + (size_t)hi * KL.operand_head_bytes + K_BYTES + VT_BYTES, kOperandConstBytes, &misc->kc_full);
+                }
                 ptx::mbar_arrive_expect_tx(&misc->vt_full, HG * VT_BYTES);
                 for (int hi = 0; hi < HG; ++hi)
                     ptx::bulk_load(smem + OFF_R1 + hi * VT_BYTES, img + (size_t)hi * KL.operand_head_bytes + K_BYTES, VT_BYTES, &misc->vt_full);
-                vt_issued = true;
                 if (FUSE_OUT) {
                     const uint8_t* blob2 = (const uint8_t*)(a.reqs ? a.reqs[zb].Wout : a.wout);
                     ptx::mbar_arrive_expect_tx(&misc->w2_full, RAW_BYTES + scale_bytes + NQ * 4);
                     ptx::bulk_load(smem + OFF_RAW, blob2 + L.off_codes + (size_t)col0 * L.row_bytes, RAW_BYTES, &misc->w2_full);
                     ptx::bulk_load(smem + OFF_SC, blob2 + L.off_scales + (size_t)col0 * n_groups * 4, scale_bytes, &misc->w2_full);
                     ptx::bulk_load(smem + OFF_BIAS, blob2 + L.off_bias + (size_t)col0 * 4, NQ * 4, &misc->w2_full);
-                    w2_issued = true;
-                }
-            }
-            if (FUSE_OUT && ok) {
-                // this CTA's five O tiles go to the partner once every worker warp has stored its part and the partner has
-                // announced that its probability tiles are dead; the copy completes on the partner's o_all barrier
-                ok = ptx::mbar_wait(&misc->peer_ready, 0, WL) && ptx::mbar_wait(&misc->o_own, 0, WL) && !misc->abort_flag;
-                if (ok) {
-                    unsigned char* mine = smem + OFF_R0 + rank * (N_OTILE / 2) * O_TILE;
-                    ptx::bulk_copy_to_cta(ptx::map_to_cta(ptx::smem_u32(mine), peer), mine, (uint32_t)((N_OTILE / 2) * O_TILE),
-                                          ptx::map_to_cta(ptx::smem_u32(&misc->o_all), peer));
-                    TAQ_PROF(57);
                 }
             }
             if (!ok) give_up();
-            if (misc->abort_flag) {   // give copies that are still in flight a bounded chance to land before the CTA exits
-                (void)ptx::mbar_wait(&misc->w_full, 0, WL);
+        }
+        if (FUSE_OUT) {
+            __syncwarp();
+            ptx::cluster_wait();                              // the partner's barriers exist
+            if (lane == 0 && !misc->abort_flag) {
+                // Every PV product of this CTA is complete when the last one is: its probability tiles may receive the
+                // partner's O.  Then this CTA's five O tiles go to the partner, each as soon as the heads that write it
+                // have stored their parts and the partner has announced the same about its probability tiles; the copies
+                // complete on the partner's o_all barrier.
+                bool ok = ptx::mbar_wait(&misc->o_full[HG - 1], 0, WL) && !misc->abort_flag;
+                if (ok) ptx::mbar_arrive_cluster_relaxed(ptx::map_to_cta(ptx::smem_u32(&misc->peer_ready), peer));
+                ok = ok && ptx::mbar_wait(&misc->peer_ready, 0, WL);
+                for (int lt = 0; lt < N_OTILE / 2 && ok; ++lt) {
+                    ok = ptx::mbar_wait(&misc->tile_done[lt], 0, WL) && !misc->abort_flag;
+                    if (!ok) break;
+                    unsigned char* mine = smem + own_tile_offset(lt);
+                    ptx::bulk_copy_to_cta(ptx::map_to_cta(ptx::smem_u32(smem + peer_tile_offset(lt)), peer), mine, (uint32_t)O_TILE,
+                                          ptx::map_to_cta(ptx::smem_u32(&misc->o_all), peer));
+                    if (lt == 0) TAQ_PROF(57);
+                }
+                if (!ok) give_up();
+            }
+        }
+        if (lane == 0 && misc->abort_flag) {   // give copies that are still in flight a bounded chance to land before the CTA exits
+            (void)ptx::mbar_wait(&misc->w_full, 0, WL);
+            for (int kb = 0; kb < NKB; ++kb) (void)ptx::mbar_wait(&misc->a_full[kb], 0, WL);
+            // (the image and Wout copies are issued only after phase 1 succeeded; when they were, these waits end with them)
+            if (ptx::mbar_try_wait(&misc->acc_full[n_groups - 1], 0)) {
                 (void)ptx::mbar_wait(&misc->kc_full, 0, WL);
-                for (int kb = 0; kb < NKB; ++kb) (void)ptx::mbar_wait(&misc->a_full[kb], 0, WL);
-                if (vt_issued) (void)ptx::mbar_wait(&misc->vt_full, 0, WL);
-                if (w2_issued) (void)ptx::mbar_wait(&misc->w2_full, 0, WL);
+                (void)ptx::mbar_wait(&misc->vt_full, 0, WL);
+                if (FUSE_OUT) (void)ptx::mbar_wait(&misc->w2_full, 0, WL);
             }
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         // All 32 lanes walk the control flow (waits, loop state and descriptor words stay warp-uniform); one elected lane
-        // issues the MMAs and commits.
+        // issues the MMAs and commits.  Its waits are bounded but do not poll the abort flag: the path between two MMAs is
+        // kept as short as possible.
         const bool leader = ptx::elect_one();
         bool ok = true;
-        auto wait = [&](uint64_t* bar, uint32_t parity) -> bool { return __all_sync(0xffffffffu, ptx::mbar_wait(bar, parity, WL) && !misc->abort_flag) != 0; };
+        auto wait = [&](uint64_t* bar, uint32_t parity) -> bool { return __all_sync(0xffffffffu, ptx::mbar_wait(bar, parity, WL)) != 0; };
         constexpr uint32_t idesc = ptx::idesc_f16_m128(NQ);
         constexpr uint32_t HI128 = ptx::kDescHiSw128, HI64 = ptx::kDescHiSw64, HI32 = ptx::kDescHiSw32;
         const uint32_t r0_lo = ptx::desc_lo(ptx::smem_u32(smem + OFF_R0)), r1_lo = ptx::desc_lo(ptx::smem_u32(smem + OFF_R1));
         const uint32_t pb_lo = ptx::desc_lo(ptx::smem_u32(smem + OFF_PB)), k_lo = ptx::desc_lo(ptx::smem_u32(smem + OFF_K));
-        {   // phase 1: one accumulation pass per scale group
+        {   // phase 1: one accumulation pass per scale group; every weight tile was expanded before X arrived
             int kb = 0;
             for (int g = 0; g < n_groups && ok; ++g) {
                 const int kb_end = min(NKB, kb + kb_per_group);
                 for (bool first = true; kb < kb_end && ok; ++kb) {
-                    const int s = kb % NS1;
-                    if (!wait(&misc->a_full[kb], 0) || !wait(&misc->b1_full[s], (uint32_t)(kb / NS1))) { ok = false; break; }
+                    if (!wait(&misc->b1_full[kb], 0) || !wait(&misc->a_full[kb], 0)) { ok = false; break; }
                     if (leader) {
                         TAQ_PROF(2 + kb);
-                        const uint32_t a_lo = r0_lo + kb * (A_TILE >> 4), b_lo = r1_lo + s * (B_TILE >> 4);
+                        const uint32_t a_lo = r0_lo + kb * (A_TILE >> 4), b_lo = ptx::desc_lo(ptx::smem_u32(smem + stage1_offset(kb)));
 #pragma unroll
                         for (int k = 0; k < BK / 16; ++k)
                             ptx::mma_f16_ss(tmem_base + TMEM_ACC + g * NQ, ptx::desc_join(HI128, a_lo + 2 * k), ptx::desc_join(HI128, b_lo + 2 * k), idesc, !(first && k == 0));
-                        ptx::mma_commit(&misc->b1_empty[s]);
                         if (kb + 1 == kb_end) ptx::mma_commit(&misc->acc_full[g]);
                     }
                     first = false;
@@ -349,7 +427,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) layer_c320_kernel(const __grid_co
         }
         // phase 3: the Q~ tiles of all four heads are in place once every worker warp has arrived (their reads of the
         // phase-1 accumulators, whose columns S and O reuse, are ordered before that arrival)
-        ok = ok && wait(&misc->q_all, 0) && wait(&misc->kc_full, 0);
+        ok = ok && wait(&misc->kc_full, 0) && wait(&misc->q_all, 0);
         ptx::tc_fence_after_sync();
         if (ok && leader) {
             TAQ_PROF(10);
@@ -376,50 +454,69 @@ __global__ void __launch_bounds__(NTHREADS, 1) layer_c320_kernel(const __grid_co
                 ptx::mma_commit(&misc->o_full[hi]);
             }
         }
-        if (FUSE_OUT && ok) {
-            // every PV product is complete when the last one is: this CTA's probability tiles may receive the partner's O
-            ok = wait(&misc->o_full[HG - 1], 0);
-            if (ok && leader) ptx::mbar_arrive_cluster_relaxed(ptx::map_to_cta(ptx::smem_u32(&misc->peer_ready), peer));
-            // phase 4: Y = O Wout^T for this CTA's 160 output channels.  Block i of the walk is K block i (rank 0) or
-            // 4 - i (rank 1); inside a block the CTA's own 32 channels come first.  Everything up to the first half of the
-            // third block reads this CTA's own O tiles, the rest the partner's.
-            ok = ok && wait(&misc->o_own, 0);
-            ptx::tc_fence_after_sync();                  // the workers' loads of the O accumulators
-            uint32_t started = 0;
-            int blocks_done[MAX_GROUPS] = {0, 0, 0};
-            for (int i = 0; i < NKB && ok; ++i) {
-                const int kb = rank ? NKB - 1 - i : i;
-                const int g = kb / kb_per_group;
-                const int s = i % NS4;
-                if (!wait(&misc->b4_full[s], (uint32_t)(i / NS4))) { ok = false; break; }
-                for (int hf = 0; hf < 2 && ok; ++hf) {
-                    const int half = rank ? 1 - hf : hf;             // which 32 channels of the block
-                    if (i == NKB / 2 && hf == 1) {
-                        ok = wait(&misc->o_all, 0);
-                        // the partner's copy has landed: it may leave without waiting for this CTA any longer
+        if (FUSE_OUT) {
+            ptx::cluster_wait();                          // the partner's barriers exist (peer_got below)
+            // phase 4: Y = O Wout^T for this CTA's 160 output channels, in six steps (see walk_block): three over this CTA's
+            // own O tiles, each as soon as the heads that write its tiles have stored them, then three over the partner's.
+            // The accumulators reuse the columns of S (all read long ago) and, for the third scale group, of O: both
+            // CTAs reach that group only after waiting for all five of their own tiles, i.e. for every head's reads of O.
+            // The walk is unrolled per rank so that tile addresses, stages and parities are constants: between two MMAs
+            // this warp, which shares its scheduler with four worker warps, should have as few instructions as possible.
+            auto phase4 = [&](auto rank_c) {
+                constexpr int R = decltype(rank_c)::value;
+                uint32_t first_mask = 0, last_mask = 0, seen = 0;       // bit i: walk step i begins / completes a scale group
+#pragma unroll
+                for (int i = 0; i < 6; ++i) {
+                    const int g = walk_block(R, i) / kb_per_group;
+                    if (!((seen >> g) & 1u)) first_mask |= 1u << i;
+                    seen |= 1u << g;
+                }
+                seen = 0;
+#pragma unroll
+                for (int i = 5; i >= 0; --i) {
+                    const int g = walk_block(R, i) / kb_per_group;
+                    if (!((seen >> g) & 1u)) last_mask |= 1u << i;
+                    seen |= 1u << g;
+                }
+                // this CTA's own five O tiles: every head has stored its part (and read its O accumulator)
+#pragma unroll
+                for (int lt = 0; lt < N_OTILE / 2; ++lt) ok = ok && wait(&misc->tile_done[lt], 0);
+                ptx::tc_fence_after_sync();
+#pragma unroll
+                for (int i = 0; i < 6; ++i) {
+                    const int kb = walk_block(R, i), halves = walk_halves(R, i), st = walk_stage(R, kb);
+                    const int g = kb / kb_per_group;
+                    if (i == 3) {
+                        ok = ok && wait(&misc->o_all, 0);
+                        // the partner's copies have landed: it may leave without waiting for this CTA any longer
                         if (ok && leader) ptx::mbar_arrive_cluster_relaxed(ptx::map_to_cta(ptx::smem_u32(&misc->peer_got), peer));
                         if (leader) TAQ_PROF(38);
-                        if (!ok) break;
+                    } else {
+                        // (block 2 returns at step 3 with the tile it already has)
+                        ok = ok && wait(&misc->b4_full[walk_order(R, kb)], 0);
                     }
-                    if (leader) {
-                        if (hf == 0) TAQ_PROF(40 + i);
-                        const uint32_t o_lo = r0_lo + (2 * kb + half) * (O_TILE >> 4);
-                        const uint32_t b_lo = ptx::desc_lo(ptx::smem_u32(smem + stage4_offset(s))) + 4 * half;
+                    if (ok && leader) {
+                        TAQ_PROF(40 + i);
+                        const uint32_t b_lo = ptx::desc_lo(ptx::smem_u32(smem + stage4_offset(st)));
+                        bool acc = !((first_mask >> i) & 1u);
 #pragma unroll
-                        for (int k = 0; k < 2; ++k)
-                            ptx::mma_f16_ss(tmem_base + TMEM_ACC + g * NQ, ptx::desc_join(HI64, o_lo + 2 * k), ptx::desc_join(HI128, b_lo + 2 * k), idesc,
-                                            ((started >> g) & 1u) != 0 || k != 0);
+                        for (int hf = 0; hf < 2; ++hf) {
+                            if (!((halves >> hf) & 1)) continue;
+                            const int t = 2 * kb + hf;                      // O tile (32 channels) of this half
+                            const int off = (t / (N_OTILE / 2)) == R ? own_tile_offset(t % (N_OTILE / 2)) : peer_tile_offset(t % (N_OTILE / 2));
+                            const uint32_t o_lo = ptx::desc_lo(ptx::smem_u32(smem + off));
+#pragma unroll
+                            for (int k = 0; k < 2; ++k) {
+                                ptx::mma_f16_ss(tmem_base + TMEM_ACC + g * NQ, ptx::desc_join(HI64, o_lo + 2 * k), ptx::desc_join(HI128, b_lo + 4 * hf + 2 * k), idesc, acc);
+                                acc = true;
+                            }
+                        }
+                        if (st == walk_reuse_stage(R) && kb != walk_tile(R, NKB - 1)) ptx::mma_commit(&misc->b4_empty[st]);
+                        if ((last_mask >> i) & 1u) ptx::mma_commit(&misc->acc_full[g]);
                     }
-                    started |= 1u << g;
                 }
-                if (!ok) break;
-                ++blocks_done[g];
-                if (leader) {
-                    ptx::mma_commit(&misc->b4_empty[s]);
-                    const int g_blocks = min(NKB, (g + 1) * kb_per_group) - g * kb_per_group;
-                    if (blocks_done[g] == g_blocks) ptx::mma_commit(&misc->acc_full[g]);
-                }
-            }
+            };
+            if (rank == 0) phase4(std::integral_constant<int, 0>{}); else phase4(std::integral_constant<int, 1>{});
         }
         if (!ok) {
             if (leader) {
@@ -480,12 +577,10 @@ __global__ void __launch_bounds__(NTHREADS, 1) layer_c320_kernel(const __grid_co
             ptx::tc_fence_before_sync();
         };
 
-        // ---- phase 1: expand the five Wq tiles (the first three before X has arrived), then fold ----
+        // ---- phase 1: expand all five Wq tiles (before X has arrived), then fold ----
         for (int kb = 0; kb < NKB; ++kb) {
-            const int s = kb % NS1;
-            if (kb >= NS1 && ok) ok = ptx::mbar_wait(&misc->b1_empty[s], 0, WL) && !misc->abort_flag;
-            if (ok) expand_block(raw, kb, smem + OFF_R1 + s * B_TILE, wt);
-            tile_built(&misc->b1_full[s]);
+            if (ok) expand_block(raw, kb, smem + stage1_offset(kb), wt);
+            tile_built(&misc->b1_full[kb]);
         }
         fold_groups(0, false);
         if (!ok) give_up();
@@ -498,7 +593,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) layer_c320_kernel(const __grid_co
         {
             float amax = 0.f;
 #pragma unroll
-            for (int c = 0; c < D; ++c) amax = fmaxf(amax, fabsf(y[c]));
+            for (int c = 0; c < D; c += 2) amax = max3(amax, fabsf(y[c]), fabsf(y[c + 1]));
             unsigned char* q_tile = smem + OFF_R0 + hi * A_TILE;
             if (a.q_bits == 8) {
                 const float sc = quant_scale(amax, 127.f);
@@ -542,8 +637,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) layer_c320_kernel(const __grid_co
             ptx::tc_fence_after_sync();
             float e[TP];
             uint32_t u[TP];
+            const uint32_t t_s = tmem_base + TMEM_S + hi * TP + lane_addr;
             {
-                const uint32_t t_s = tmem_base + TMEM_S + hi * TP + lane_addr;
                 uint32_t (&u8)[TP / 8][8] = *reinterpret_cast<uint32_t (*)[TP / 8][8]>(&u);
 #pragma unroll
                 for (int i = 0; i < TP / 8; ++i) ptx::tmem_ld8(t_s + i * 8, u8[i]);
@@ -551,37 +646,33 @@ __global__ void __launch_bounds__(NTHREADS, 1) layer_c320_kernel(const __grid_co
 #pragma unroll
                 for (int i = 1; i < TP / 8; ++i) ptx::reg_fence8(u8[i]);
             }
-            if (lane == 0 && hi == 0) TAQ_PROF(60 + q4);       // S in registers
             const OperandConsts* cst = reinterpret_cast<const OperandConsts*>(smem + OFF_CST + hi * kOperandConstBytes);
             float msq;
-            const float l = softmax_row<TAIL_ONLY>(u, e, cst->logit_factor, sq, T, msq);
-            if (lane == 0 && hi == 0) TAQ_PROF(64 + q4);       // exponentials done
-            if (lane == 0 && q4 == 0) TAQ_PROF(20 + hi);       // exponentials done
+            const float l = softmax_row<TAIL_FROM>(u, e, cst->logit_factor, sq, T, msq);
             const float k255 = __fdividef(pmax, l);
             const uint32_t trig[3] = {cst->trig_bits[0], cst->trig_bits[1], cst->trig_bits[2]};
             write_p_row(e, k255, smem + OFF_R0 + hi * A_TILE, smem + OFF_PB + hi * PB_TILE, r);
-            trigger_columns(trig, tmem_base + TMEM_S + hi * TP + lane_addr, cst->logit_factor, sq, msq, k255, smem + OFF_R0 + hi * A_TILE, smem + OFF_PB + hi * PB_TILE, r);
-            if (lane == 0 && hi == 0) TAQ_PROF(68 + q4);       // P stored
+            trigger_columns(trig, t_s, cst->logit_factor, sq, msq, k255, smem + OFF_R0 + hi * A_TILE, smem + OFF_PB + hi * PB_TILE, r);
         }
         ptx::tc_fence_before_sync();
         tile_built(&misc->p_full[hi]);
         if (lane == 0 && q4 == 0) TAQ_PROF(24 + hi);           // P written
 
         if (FUSE_OUT) {
-            // Wout tiles of the first two blocks of the walk go into the K~ buffers, dead once every S product is complete.
+            // The first Wout tile of the walk goes into a K~ buffer (dead once every S product is complete) while this
+            // head's PV product runs; the second follows after the head's O has been stored.  The warps of the last head,
+            // whose probabilities are the last to be complete, take no part in the expansion.
             ok = ok && ptx::mbar_wait(&misc->s_full[HG - 1], 0, WL) && ptx::mbar_wait(&misc->w2_full, 0, WL) && !misc->abort_flag;
             for (int i = wt; i < NQ * n_groups; i += NWORK) scales_t[(i % n_groups) * NQ + i / n_groups] = wscales[i];     // (last read in phase 1)
-            for (int i = 0; i < 2; ++i) {
-                if (ok) expand_block(raw, rank ? NKB - 1 - i : i, smem + stage4_offset(i), wt);
-                tile_built(&misc->b4_full[i]);
+            if (wt < NEXP) {
+                if (ok) expand_block_by<NEXP>(raw, walk_tile(rank, 0), smem + stage4_offset(0), wt);
+                tile_built(&misc->b4_full[0]);
             }
             if (wt == 0) TAQ_PROF(34);
         }
 
-        // ---- O of (row, head): the accumulator in units of 1 / pmax -> fp16 ----
-        // Every PV product is complete when the last one is; only then are the other heads' probability tiles, which the O
-        // tiles overlap, dead.
-        ok = ok && ptx::mbar_wait(&misc->o_full[FUSE_OUT ? HG - 1 : hi], 0, WL) && !misc->abort_flag;
+        // ---- O of (row, head): the accumulator in units of 1 / pmax -> fp16, as soon as this head's PV product is complete ----
+        ok = ok && ptx::mbar_wait(&misc->o_full[hi], 0, WL) && !misc->abort_flag;
         if (ok) {
             ptx::tc_fence_after_sync();
             const float inv = 1.0f / pmax;
@@ -600,8 +691,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) layer_c320_kernel(const __grid_co
                 for (int e2 = 0; e2 < 8; ++e2) f[e2] = __uint_as_float(v[i][e2]) * inv;
                 const uint4 o8 = pack8(f);
                 if (FUSE_OUT) {           // 8 channels of O as one chunk of the to_out operand tiles
-                    const int cg = (h_begin + hi) * D + i * 8;       // channel of O (0..319)
-                    *reinterpret_cast<uint4*>(smem + OFF_R0 + (cg >> 5) * O_TILE + ptx::sw64_offset(r, (cg & 31) >> 3)) = o8;
+                    const int c = hi * D + i * 8;                    // channel among this CTA's 160
+                    *reinterpret_cast<uint4*>(smem + own_tile_offset(c >> 5) + ptx::sw64_offset(r, (c & 31) >> 3)) = o8;
                 } else if (valid) {
                     *reinterpret_cast<uint4*>(orow + i * 8) = o8;
                 }
@@ -610,14 +701,21 @@ __global__ void __launch_bounds__(NTHREADS, 1) layer_c320_kernel(const __grid_co
         ptx::tc_fence_before_sync();
 
         if (FUSE_OUT) {
-            tile_built(&misc->o_own);
+            ptx::fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) { ptx::mbar_arrive(&misc->tile_done[hi]); ptx::mbar_arrive(&misc->tile_done[hi + 1]); }      // head hi writes tiles hi and hi + 1
             if (wt == 0) TAQ_PROF(32);
-            // ---- phase 4: the remaining Wout tiles (the V~^T buffers are dead: every PV product is complete), then fold ----
-            for (int i = 2; i < NKB; ++i) {
-                const int s = i % NS4;
-                if (i >= NS4 && ok) ok = ptx::mbar_wait(&misc->b4_empty[s], 0, WL) && !misc->abort_flag;
-                if (ok) expand_block(raw, rank ? NKB - 1 - i : i, smem + stage4_offset(s), wt);
-                tile_built(&misc->b4_full[s]);
+            // ---- phase 4: the remaining Wout tiles (the V~^T buffers are dead once every PV product is complete), then fold ----
+            if (wt < NEXP) {
+                if (ok) expand_block_by<NEXP>(raw, walk_tile(rank, 1), smem + stage4_offset(1), wt);
+                tile_built(&misc->b4_full[1]);
+                ok = ok && ptx::mbar_wait(&misc->o_full[HG - 1], 0, WL) && !misc->abort_flag;
+                for (int i = 2; i < NKB; ++i) {
+                    const int s = i < NS4 ? i : walk_reuse_stage(rank);
+                    if (i >= NS4 && ok) ok = ptx::mbar_wait(&misc->b4_empty[s], 0, WL) && !misc->abort_flag;
+                    if (ok) expand_block_by<NEXP>(raw, walk_tile(rank, i), smem + stage4_offset(s), wt);
+                    tile_built(&misc->b4_full[i]);
+                }
             }
             if (wt == 0) TAQ_PROF(35);
             asm volatile("bar.sync 1, 512;" ::: "memory");       // the transposed scale table is complete
@@ -647,6 +745,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) layer_c320_kernel(const __grid_co
                 ptx::bulk_store_wait_read();                     // shared memory is given back only after the store has read it
             }
             if (wt == 0) { TAQ_PROF(37); TAQ_GPROF(27); }
+            ptx::cluster_wait();
         } else if (!ok) {
             give_up();
         }
@@ -714,7 +813,8 @@ static cudaError_t launch_c320(const taq_layer_desc& d, const __half* x, const v
     a.wait_cycles = g_wait_cycles;
     a.status = status;
     dim3 grid((d.n_query + ROWS - 1) / ROWS, d.heads / HG, n_z);
-    const bool tail = d.n_ctx > 64, fuse_out = y != nullptr;
+    const int tail = d.n_ctx > 72 ? 72 : d.n_ctx > 64 ? 64 : 0;     // first key that can lie beyond the context (the kernel masks from there on)
+    const bool fuse_out = y != nullptr;
     CUtensorMap tmap_y = tmap;                        // (unused by the variant that stores O)
     if (fuse_out) {
         const cuuint32_t ybox[3] = {D, ROWS, 1};      // one head group: 40 channels = 80 bytes per row, dense in shared memory
@@ -723,7 +823,8 @@ static cudaError_t launch_c320(const taq_layer_desc& d, const __half* x, const v
         if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
     }
     void (*kern)(const CUtensorMap, const CUtensorMap, const LayerArgs) =
-        fuse_out ? (tail ? layer_c320_kernel<true, true> : layer_c320_kernel<false, true>) : (tail ? layer_c320_kernel<true, false> : layer_c320_kernel<false, false>);
+        fuse_out ? (tail == 72 ? layer_c320_kernel<72, true> : tail == 64 ? layer_c320_kernel<64, true> : layer_c320_kernel<0, true>)
+                 : (tail == 72 ? layer_c320_kernel<72, false> : tail == 64 ? layer_c320_kernel<64, false> : layer_c320_kernel<0, false>);
     // (the attribute belongs to the current device's copy of the function: set on every launch, it is cheap)
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TOTAL);
     if (e != cudaSuccess) return e;

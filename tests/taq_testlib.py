@@ -7,9 +7,26 @@ from oracle import taq_oracle as orc
 from paper_2603_22943_b200 import binding as tb
 from paper_2603_22943_b200 import synth
 
+import json
+import os
+
 # Layer-output tolerances of the parity contract (fp16 outputs against the fp64 contract-mode oracle).
 TOL_MAX_ABS = 2e-2
 TOL_REL_L2 = 1e-3
+# A query row in which the fp32 accumulation of the GPU and the fp64 one of the oracle round one Q (or, with integer
+# activations, O) code to different sides of a tie is compared end to end as well, but it is not the same computation any
+# more: one code step of a row of d values moves that row's logits, and the softmax amplifies it.  Such rows must be few,
+# and their error stays under a bound of its own.
+TOL_MAX_ABS_TIE_ROWS = 6e-2
+MAX_TIE_ROW_FRACTION = {0: 0.02, 8: 0.25}          # by a_bits
+
+
+def _log_parity(record):
+    """Appends one line per layer comparison to the file named by TAQ_PARITY_LOG (the figures quoted in the design notes)."""
+    path = os.environ.get("TAQ_PARITY_LOG")
+    if path:
+        with open(path, "a") as f:
+            f.write(json.dumps(record) + "\n")
 
 
 def dev(a: np.ndarray) -> torch.Tensor:
@@ -189,11 +206,12 @@ def check_layer(shape: synth.LayerShape, data, y_gpu, parts, rows=None, a_bits=0
         xc, xs = orc.quantize_rows(X.astype(np.float32), 127)
         assert np.array_equal(g["X_codes"], xc) and np.array_equal(g["X_scales"], xs), "X codes / scales"
     # (1)
-    nt = np.array([j for j in range(shape.n_ctx) if not data["mask"][0, j]], dtype=np.int64)
-    same_mask = bool((data["mask"] == data["mask"][0]).all())
-    if same_mask and len(nt):
-        for nm in ("K", "V"):
-            assert_codes_agree(g[nm + "_codes"][:, :, nt], kv_o[nm + "_codes"][:, :, nt], kv_o[nm][:, :, nt], kv_o[nm + "_scales"][:, :, nt], nm + " codes")
+    for b in range(data["mask"].shape[0]):                   # per sequence: every request may have its own mask
+        nt = np.array([j for j in range(shape.n_ctx) if not data["mask"][b, j]], dtype=np.int64)
+        if len(nt):
+            for nm in ("K", "V"):
+                assert_codes_agree(g[nm + "_codes"][b:b + 1][:, :, nt], kv_o[nm + "_codes"][b:b + 1][:, :, nt], kv_o[nm][b:b + 1][:, :, nt],
+                                   kv_o[nm + "_scales"][b:b + 1][:, :, nt], f"{nm} codes of sequence {b}")
     flipped_rows = np.zeros(X.shape[:2], dtype=bool)
     if shape.q_bits == 8:
         assert_codes_agree(g["Q_codes"], q_o["Q_codes"], q_o["Q"], q_o["Q_scales"], "Q codes")
@@ -213,7 +231,16 @@ def check_layer(shape: synth.LayerShape, data, y_gpu, parts, rows=None, a_bits=0
     # (3)
     max_abs, rel = errors(y, Y_o)
     assert rel <= TOL_REL_L2, f"{shape.name}: end-to-end rel-L2 {rel:.3e}"
-    if (~flipped_rows).any():
-        ma = float(np.max(np.abs(y.astype(np.float64) - Y_o)[~flipped_rows]))
-        assert ma <= TOL_MAX_ABS, f"{shape.name}: end-to-end max-abs {ma:.3e} on rows whose Q codes agree"
-    return {"same_decisions": same, "end_to_end": (max_abs, rel), "rows_with_q_flip": int(flipped_rows.sum()), "rows": int(flipped_rows.size)}
+    err = np.abs(y.astype(np.float64) - Y_o).max(axis=-1)                            # [B,n]: per query row
+    ma_same = float(err[~flipped_rows].max()) if (~flipped_rows).any() else 0.0
+    ma_tie = float(err[flipped_rows].max()) if flipped_rows.any() else 0.0
+    n_tie, n_rows = int(flipped_rows.sum()), int(flipped_rows.size)
+    rec = {"shape": shape.name, "a_bits": a_bits, "rows": n_rows, "rows_set_aside": n_tie, "max_abs_all_rows": max_abs, "max_abs_rows_with_equal_codes": ma_same,
+           "max_abs_rows_with_a_tie": ma_tie, "rel_l2": rel, "rel_l2_same_decisions": same[1], "max_abs_same_decisions": same[0]}
+    _log_parity(rec)
+    print(f"parity {shape.name}: max-abs over all {n_rows} rows {max_abs:.3e}, rel-L2 {rel:.3e}; {n_tie} rows set aside (max-abs there {ma_tie:.3e})")
+    assert ma_same <= TOL_MAX_ABS, f"{shape.name}: end-to-end max-abs {ma_same:.3e} on rows whose codes agree"
+    assert n_tie <= MAX_TIE_ROW_FRACTION[a_bits] * n_rows + 1, f"{shape.name}: {n_tie} of {n_rows} rows have a code on the other side of a tie"
+    assert ma_tie <= TOL_MAX_ABS_TIE_ROWS, f"{shape.name}: end-to-end max-abs {ma_tie:.3e} on rows with a code on the other side of a tie"
+    return {"same_decisions": same, "end_to_end": (max_abs, rel), "rows_with_q_flip": n_tie, "rows": n_rows, "max_abs_all_rows": max_abs,
+            "max_abs_tie_rows": ma_tie}

@@ -56,6 +56,51 @@ def test_quantize_rows_many_random_values():
     _check_rows(x)
 
 
+@pytest.mark.parametrize("part", range(10))
+def test_quantize_rows_1e8_values(part):
+    """The kernel multiplies by a reciprocal and falls back to the division of the definition only where the two could
+    round differently; that shortcut is allowed only if the codes stay bit-exact on a large sample.  Ten parts of 1.05e7
+    fp32 values each (1.05e8 in all): Gaussian rows of the widths the layers use, heavy tails, and rows built to sit on
+    rounding boundaries (values (k + 1/2) s +- one ulp for the row's own scale s)."""
+    r = np.random.default_rng(1000 + part)
+    rows, cols = 1 << 16, 160
+    if part < 4:
+        x = (r.standard_normal((rows, cols)) * r.uniform(1e-3, 50.0, (rows, 1))).astype(np.float32)
+    elif part < 6:
+        x = r.standard_cauchy((rows, cols)).astype(np.float32)
+    elif part < 8:                                           # values at and next to the rounding boundaries of the row's own grid
+        amax = r.uniform(0.5, 200.0, (rows, 1)).astype(np.float32)
+        s = (amax / np.float32(127.0)).astype(np.float32)
+        k = r.integers(-126, 126, (rows, cols)).astype(np.float32)
+        x = ((k + np.float32(0.5)) * s).astype(np.float32)
+        x = np.nextafter(x, np.where(r.integers(0, 3, x.shape) == 0, -np.inf, np.where(r.integers(0, 2, x.shape) == 0, np.inf, x)).astype(np.float32))
+        x[:, 0] = amax[:, 0]
+    else:                                                    # fp16-valued data (as the layer inputs are), where exact ties are common
+        x = (r.standard_normal((rows, cols)) * r.uniform(0.1, 30.0, (rows, 1))).astype(np.float16).astype(np.float32)
+    _check_rows(x)
+
+
+@pytest.mark.parametrize("part", range(4))
+def test_quantize_rows_f16_every_finite_value_for_1024_row_maxima(part):
+    """The per-token quantizer of fp16 data, exhaustively: every finite fp16 value as an element of a row, for 1024
+    different row maxima (random ones, powers of two, the largest and smallest fp16 numbers).  Elements larger than the
+    row's maximum are replaced by it, so that the maximum is what it is meant to be."""
+    allv = np.arange(0, 1 << 16, dtype=np.uint16).view(np.float16)
+    allv = allv[np.isfinite(allv)]                           # 63488 values (both zeros, subnormals included)
+    assert allv.size == 63488 and allv.size % 8 == 0
+    r = np.random.default_rng(77 + part)
+    rows = 256
+    m = np.abs((r.standard_normal(rows) * r.uniform(1e-3, 1e3, rows)).astype(np.float16))
+    m[:8] = np.array([65504, 6.1e-5, 5.96e-8, 1.0, 127.0, 63.5, 0.5, 2.0 ** -14], dtype=np.float16)[:8] if part == 0 else m[:8]
+    m = np.where(m == 0, np.float16(1.0), m)
+    x = np.where(np.abs(allv)[None, :] <= m[:, None], allv[None, :], m[:, None]).astype(np.float16)
+    codes, scales = tb.taq_quantize_rows_f16(dev(x))
+    want_c, want_s = orc.quantize_rows(x.astype(np.float32), 127)
+    assert np.array_equal(scales.cpu().numpy(), want_s)
+    got = codes.cpu().numpy()
+    assert np.array_equal(got, want_c.astype(np.int8)), f"{int((got != want_c).sum())} codes differ"
+
+
 @pytest.mark.parametrize("n_out,k_in,bits,group", [
     (320, 320, 4, 128),      # config 2 to_q / to_out: ragged last group of 64
     (320, 768, 4, 128),      # config 2 to_k / to_v
