@@ -20,6 +20,7 @@
 #include "taq_sm100.cuh"
 #include "taq_sm100_parts.cuh"
 #include "taq_prof.cuh"
+#include <type_traits>
 
 TAQ_PROF_DEFINE(linear)
 
@@ -32,6 +33,7 @@ using namespace parts;
 constexpr int BM = 128;
 constexpr int BK = 64;                     // fp16 elements per 128-byte operand row; the int8 variant has 2 BK
 constexpr int MAX_STAGE = 6;
+constexpr int MAX_PREBUILT = 12;           // k-blocks per CTA whose expanded weight tiles may all be resident at once
 constexpr int NWORK = 256;                  // worker threads: two per accumulator row
 constexpr int NTHREADS = 64 + NWORK;
 constexpr int A_TILE_BYTES = BM * BK * 2;   // 16 KB
@@ -49,7 +51,7 @@ struct Tile {
 
 struct Bars {
     uint64_t full_a[MAX_STAGE];
-    uint64_t full_b[MAX_STAGE];
+    uint64_t full_b[MAX_PREBUILT];
     uint64_t empty[MAX_STAGE];
     uint64_t w_full;
     uint64_t acc_full[2];
@@ -62,25 +64,31 @@ struct Bars {
 // Shared-memory plan of one launch (host and device agree through these numbers).
 struct Plan {
     int raw_bytes, scale_bytes, bias_bytes;   // BN rows of codes / scales / bias
+    int stage_bytes;                          // one ring stage: the activation tile, plus the weight tile unless prebuilt
+    int off_ball;                             // prebuilt: the CTA's expanded weight tiles, one per k-block
     int off_raw, off_scales, off_scales_t, off_bias, off_xchg, off_bars, total;
 };
 
+// prebuilt = number of k-blocks of the CTA when all of its expanded weight tiles are resident at once (0: the tiles go
+// through the ring with the activations).
 template <int BN>
-__host__ __device__ inline Plan make_plan(int k_in, int bits, int group, int nstage, int mode) {
+__host__ __device__ inline Plan make_plan(int k_in, int bits, int group, int nstage, int mode, int prebuilt = 0) {
     const WeightLayout L = weight_layout(BN, k_in, bits, group);
     Plan p;
+    p.stage_bytes = prebuilt ? A_TILE_BYTES : Tile<BN>::STAGE_BYTES;
+    p.off_ball = nstage * p.stage_bytes;
     // codes of the BN channels over the whole fan-in; mode 1: none (the codes are the B operand); mode 2: one 64-byte slice
     // per channel and ring stage
     p.raw_bytes = mode == 1 ? 0 : mode == 2 ? nstage * BN * BK : (int)(L.row_bytes * BN);
     p.scale_bytes = BN * L.n_groups * 4;
     p.bias_bytes = BN * 4;
-    p.off_raw = nstage * Tile<BN>::STAGE_BYTES;
+    p.off_raw = p.off_ball + prebuilt * Tile<BN>::B_TILE_BYTES;
     p.off_scales = p.off_raw + (p.raw_bytes + 127) / 128 * 128;
     p.off_scales_t = p.off_scales + (p.scale_bytes + 127) / 128 * 128;        // [n_groups][BN]
     p.off_bias = p.off_scales_t + (p.scale_bytes + 127) / 128 * 128;
     p.off_xchg = p.off_bias + (p.bias_bytes + 127) / 128 * 128;              // float [2][128]
     p.off_bars = p.off_xchg + 1024;
-    p.total = p.off_bars + 256 + 1024;        // barriers + slack to align the base to 1024
+    p.total = p.off_bars + 512 + 1024;        // barriers + slack to align the base to 1024
     return p;
 }
 
@@ -92,13 +100,14 @@ __host__ __device__ inline Plan make_plan(int k_in, int bits, int group, int nst
 // they exchange folded fp32 partial sums through bulk copies between the two shared memories, the first CTA adding and
 // storing rows 0..63 of the tile, the second rows 64..127.
 template <int BN, bool I8, bool SPLIT>
-__global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w, const LinearArgs a, const int nstage) {
+__global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w, const LinearArgs a, const int nstage, const int prebuilt) {
     using TL = Tile<BN>;
     constexpr int BKE = I8 ? 2 * BK : BK;             // elements per K block
     constexpr int HC = TL::HC;
     extern __shared__ unsigned char smem_dyn[];
     unsigned char* smem = smem_dyn + ((1024u - (ptx::smem_u32(smem_dyn) & 1023u)) & 1023u);   // 1024-byte aligned, still provably shared
-    const Plan P = make_plan<BN>(a.k_in, a.bits, a.group, nstage, a.w_direct);
+    const Plan P = make_plan<BN>(a.k_in, a.bits, a.group, nstage, a.w_direct, prebuilt);
+    static_assert(sizeof(Bars) <= 512, "barrier block");
     Bars* bars = reinterpret_cast<Bars*>(smem + P.off_bars);
     constexpr uint32_t TMEM_COLS = TL::TMEM_COLS;
 
@@ -125,9 +134,9 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
     if (tid == 0) {
         for (int s = 0; s < MAX_STAGE; ++s) {
             ptx::mbar_init(&bars->full_a[s], 1);
-            ptx::mbar_init(&bars->full_b[s], NWORK / 32);    // one arrival per worker warp
             ptx::mbar_init(&bars->empty[s], 1);
         }
+        for (int s = 0; s < MAX_PREBUILT; ++s) ptx::mbar_init(&bars->full_b[s], NWORK / 32);    // one arrival per worker warp
         ptx::mbar_init(&bars->w_full, 1);
         for (int i = 0; i < 2; ++i) {
             ptx::mbar_init(&bars->acc_full[i], 1);
@@ -167,8 +176,8 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
                 if (kb - kb_begin >= nstage && !ptx::mbar_wait(&bars->empty[s], ph ^ 1)) { raise_status(a.status, TAQ_ERR_TIMEOUT); bars->abort_flag = 1; }
                 if (bars->abort_flag) break;
                 ptx::mbar_arrive_expect_tx(&bars->full_a[s], A_TILE_BYTES + (a.w_direct == 1 ? BN * 128 : a.w_direct == 2 ? BN * BK : 0));
-                ptx::tma_load_3d(smem + s * TL::STAGE_BYTES, &tmap_x, &bars->full_a[s], kb * BKE, row0, z);
-                if (a.w_direct == 1) ptx::tma_load_3d(smem + s * TL::STAGE_BYTES + A_TILE_BYTES, &tmap_w, &bars->full_a[s], kb * BKE, col0, 0);
+                ptx::tma_load_3d(smem + s * P.stage_bytes, &tmap_x, &bars->full_a[s], kb * BKE, row0, z);
+                if (a.w_direct == 1) ptx::tma_load_3d(smem + s * P.stage_bytes + A_TILE_BYTES, &tmap_w, &bars->full_a[s], kb * BKE, col0, 0);
                 if (a.w_direct == 2) ptx::tma_load_3d(smem + P.off_raw + s * (BN * BK), &tmap_w, &bars->full_a[s], kb * BK, col0, 0);
                 issued = kb - kb_begin + 1;
                 if (++s == nstage) { s = 0; ph ^= 1; }
@@ -199,10 +208,12 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
             }
             const int kb_end = min(kb_stop, kb + kb_per_group);
             for (bool first = true; kb < kb_end && ok; ++kb) {
-                if (!wait(&bars->full_a[s], ph) || (a.w_direct != 1 && !wait(&bars->full_b[s], ph))) { ok = false; break; }
+                // (prebuilt: every weight tile has its own barrier, complete long before its activations arrive)
+                if ((a.w_direct != 1 && !wait(&bars->full_b[prebuilt ? kb - kb_begin : s], prebuilt ? 0u : ph)) || !wait(&bars->full_a[s], ph)) { ok = false; break; }
                 if (leader) {
                     if (kb < 20) TAQ_PROF(40 + kb);
-                    const uint32_t a_lo = lo0 + s * (TL::STAGE_BYTES >> 4), b_lo = a_lo + (A_TILE_BYTES >> 4);
+                    const uint32_t a_lo = lo0 + s * (P.stage_bytes >> 4);
+                    const uint32_t b_lo = prebuilt ? lo0 + ((P.off_ball + (kb - kb_begin) * TL::B_TILE_BYTES) >> 4) : a_lo + (A_TILE_BYTES >> 4);
 #pragma unroll
                     for (int k = 0; k < 4; ++k) {            // four 32-byte K slices per 128-byte operand row
                         if (I8) ptx::mma_i8_ss(tmem_base + buf * BN, ptx::desc_join(HI, a_lo + 2 * k), ptx::desc_join(HI, b_lo + 2 * k), idesc, !(first && k == 0));
@@ -289,10 +300,10 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
         auto build_group = [&](int g) -> bool {
             const int kb_end = min(kb_stop, kb + kb_per_group);
             for (; kb < kb_end; ++kb) {
-                if (kb - kb_begin >= nstage && !ptx::mbar_wait(&bars->empty[s], ph ^ 1)) return false;
+                if (!prebuilt && kb - kb_begin >= nstage && !ptx::mbar_wait(&bars->empty[s], ph ^ 1)) return false;
                 if (bars->abort_flag) return false;
                 if (a.w_direct == 2 && !ptx::mbar_wait(&bars->full_a[s], ph)) return false;    // this k-block's slice of the codes has arrived
-                unsigned char* b_tile = smem + s * TL::STAGE_BYTES + A_TILE_BYTES;
+                unsigned char* b_tile = prebuilt ? smem + P.off_ball + (kb - kb_begin) * TL::B_TILE_BYTES : smem + s * P.stage_bytes + A_TILE_BYTES;
                 // 16-byte chunks of the fp16 tile: 8 per weight row; this thread owns chunk c of rows n0, n0 + 32, ...
                 constexpr int NCH = (BN * 8 + NWORK - 1) / NWORK;
                 const int n0 = wt >> 3, c = wt & 7;
@@ -340,18 +351,23 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
                 }
                 ptx::fence_proxy_async_smem();            // make the generic-proxy writes visible to the tensor core
                 __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(&bars->full_b[s]);
+                if (lane == 0) ptx::mbar_arrive(&bars->full_b[prebuilt ? kb - kb_begin : s]);
                 if (wt == 0 && kb < 20) TAQ_PROF(60 + kb);
                 if (++s == nstage) { s = 0; ph ^= 1; }
             }
             return true;
         };
 
-        for (int g = g_begin; g < g_end && ok; ++g) {
-            ok = a.w_direct == 1 ? true : build_group(g);
-            if (ok && g > g_begin) ok = fold_group(g - 1);
+        if (prebuilt) {            // every weight tile first (nothing to wait for), then the folds as the groups complete
+            for (int g = g_begin; g < g_end && ok; ++g) ok = build_group(g);
+            for (int g = g_begin; g < g_end && ok; ++g) ok = fold_group(g);
+        } else {
+            for (int g = g_begin; g < g_end && ok; ++g) {
+                ok = a.w_direct == 1 ? true : build_group(g);
+                if (ok && g > g_begin) ok = fold_group(g - 1);
+            }
+            if (ok) ok = fold_group(g_end - 1);
         }
-        if (ok) ok = fold_group(g_end - 1);
         if (!ok) { raise_status(a.status, TAQ_ERR_TIMEOUT); bars->abort_flag = 1; }
         asm volatile("bar.sync 1, 256;" ::: "memory");       // every worker gets here; the decision below is uniform
         ok = !bars->abort_flag;
@@ -632,17 +648,53 @@ int pick_bn(const LinearArgs& a) {
     return 0;
 }
 
+// How a launch is laid out: ring depth, whether two CTAs share a tile (split of the K loop), and whether every CTA keeps
+// all of its expanded weight tiles resident (`prebuilt` = its number of k-blocks, else 0).
+struct Choice { int ns, prebuilt; bool split; };
+
+template <int BN>
+Choice choose(const LinearArgs& a, int n_z) {
+    const bool i8 = a.xq != nullptr;
+    const int mode = weight_mode<BN>(a);
+    Choice c{pick_nstage<BN>(a), 0, false};
+    const WeightLayout Lw = weight_layout(a.n_out, a.k_in, a.bits, a.group);
+    const int bke = i8 ? 2 * BK : BK;
+    const int n_kb = (a.k_in + bke - 1) / bke;
+    const long long tiles = ((a.rows + BM - 1) / BM) * (a.n_out / BN) * (long long)n_z;
+    const int staging = epilogue_staging_bytes<BN>(a);
+    const int part = NWORK * (BN * 2 + 16);          // fp32 partial sums in transit between the two CTAs of a split tile
+    // few tiles and a long K loop: two CTAs per tile, each with half of the scale groups (or of the k-blocks of a single
+    // group: not for integer activations, where a group's sum stays one exact int32 accumulation)
+    const bool want_split = (Lw.n_groups >= 2 || !i8) && tiles <= 74 * Tile<BN>::CTAS_PER_SM && n_kb >= 6;
+    c.split = want_split && (long long)c.ns * Tile<BN>::STAGE_BYTES >= part;
+    // One wave at one CTA per SM, codes staged once, fp16 activations: expand every weight tile of the CTA before the
+    // activations arrive (under the previous kernel's tail when the weights are known early), so that the K loop waits
+    // for the TMA loads only.
+    if (mode == 0 && !i8 && tiles <= 148) {
+        for (int with_split = (want_split && 2 * tiles <= 148) ? 1 : 0; with_split >= 0; --with_split) {
+            int n_cta = n_kb;
+            if (with_split) {
+                if (Lw.n_groups == 1) n_cta = n_kb - n_kb / 2;
+                else { const int kbg = Lw.group_len / bke, lo = (Lw.n_groups / 2) * kbg; n_cta = lo > n_kb - lo ? lo : n_kb - lo; }
+            }
+            const int ns = n_cta < 3 ? 2 : 3;
+            const Plan P = make_plan<BN>(a.k_in, a.bits, a.group, ns, 0, n_cta);
+            if (n_cta <= MAX_PREBUILT && P.total <= SMEM_LIMIT && P.off_raw >= staging && (!with_split || P.off_raw >= part)) {
+                c.ns = ns; c.prebuilt = n_cta; c.split = with_split != 0;
+                break;
+            }
+        }
+    }
+    return c;
+}
+
 template <int BN>
 cudaError_t launch_bn(const CUtensorMap& tmap, EncodeTiledFn enc, LinearArgs a, int n_z, cudaStream_t stream) {
     const bool i8 = a.xq != nullptr;
-    const int ns = pick_nstage<BN>(a);
-    const WeightLayout Lw = weight_layout(a.n_out, a.k_in, a.bits, a.group);
-    const int bke = i8 ? 2 * BK : BK;
-    const long long tiles = ((a.rows + BM - 1) / BM) * (a.n_out / BN) * (long long)n_z;
-    // few tiles and a long K loop: two CTAs per tile, each with half of the scale groups (or of the k-blocks of a single
-    // group: not for integer activations, where a group's sum stays one exact int32 accumulation)
-    const bool split = (Lw.n_groups >= 2 || !i8) && tiles <= 74 * Tile<BN>::CTAS_PER_SM && (a.k_in + bke - 1) / bke >= 6 && (long long)ns * Tile<BN>::STAGE_BYTES >= 256LL * (BN * 2 + 16);
-    void (*kern)(const CUtensorMap, const CUtensorMap, const LinearArgs, const int) =
+    const Choice ch = choose<BN>(a, n_z);
+    const int ns = ch.ns;
+    const bool split = ch.split;
+    void (*kern)(const CUtensorMap, const CUtensorMap, const LinearArgs, const int, const int) =
         split ? (i8 ? linear_sm100_kernel<BN, true, true> : linear_sm100_kernel<BN, false, true>)
               : (i8 ? linear_sm100_kernel<BN, true, false> : linear_sm100_kernel<BN, false, false>);
     a.w_direct = weight_mode<BN>(a);
@@ -660,10 +712,10 @@ cudaError_t launch_bn(const CUtensorMap& tmap, EncodeTiledFn enc, LinearArgs a, 
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT);
         if (e != cudaSuccess) return e;
     }
-    const Plan P = make_plan<BN>(a.k_in, a.bits, a.group, ns, a.w_direct);
+    const Plan P = make_plan<BN>(a.k_in, a.bits, a.group, ns, a.w_direct, ch.prebuilt);
     dim3 grid((unsigned)((a.rows + BM - 1) / BM) * (split ? 2u : 1u), a.n_out / BN, n_z);
-    if (split) return launch_pdl_cluster(kern, grid, dim3(2, 1, 1), dim3(NTHREADS), (size_t)P.total, stream, tmap, tmap_w, a, ns);
-    return launch_pdl(kern, grid, dim3(NTHREADS), (size_t)P.total, stream, tmap, tmap_w, a, ns);
+    if (split) return launch_pdl_cluster(kern, grid, dim3(2, 1, 1), dim3(NTHREADS), (size_t)P.total, stream, tmap, tmap_w, a, ns, ch.prebuilt);
+    return launch_pdl(kern, grid, dim3(NTHREADS), (size_t)P.total, stream, tmap, tmap_w, a, ns, ch.prebuilt);
 }
 
 }  // namespace
@@ -698,16 +750,24 @@ void linear_plan_of(const LinearArgs& a, int out[10]) {
     if (!ok) return;
     const int bn = pick_bn(a);
     if (bn == 0) return;
-    const int ns = nstage_for(a, bn);
-    if (ns < 2) return;
+    if (nstage_for(a, bn) < 2) return;
     Plan P;
-    int stage_bytes = 0, staging = 0, mode = 0;
+    int ring = 0, staging = 0, mode = 0, ns = 0;
+    auto fill = [&](auto bn_c) {
+        constexpr int B = decltype(bn_c)::value;
+        const Choice c = choose<B>(a, 1);
+        mode = weight_mode<B>(a); ns = c.ns;
+        P = make_plan<B>(a.k_in, a.bits, a.group, c.ns, mode, c.prebuilt);
+        ring = P.off_raw;                          // ring stages (and resident weight tiles): what the epilogue may reuse
+        staging = epilogue_staging_bytes<B>(a);
+        if (c.split && staging < NWORK * (B * 2 + 16)) staging = NWORK * (B * 2 + 16);
+    };
     switch (bn) {
-        case 64: mode = weight_mode<64>(a); P = make_plan<64>(a.k_in, a.bits, a.group, ns, mode); stage_bytes = Tile<64>::STAGE_BYTES; staging = epilogue_staging_bytes<64>(a); break;
-        case 80: mode = weight_mode<80>(a); P = make_plan<80>(a.k_in, a.bits, a.group, ns, mode); stage_bytes = Tile<80>::STAGE_BYTES; staging = epilogue_staging_bytes<80>(a); break;
-        default: mode = weight_mode<160>(a); P = make_plan<160>(a.k_in, a.bits, a.group, ns, mode); stage_bytes = Tile<160>::STAGE_BYTES; staging = epilogue_staging_bytes<160>(a); break;
+        case 64: fill(std::integral_constant<int, 64>{}); break;
+        case 80: fill(std::integral_constant<int, 80>{}); break;
+        default: fill(std::integral_constant<int, 160>{}); break;
     }
-    out[0] = bn; out[1] = ns; out[2] = mode; out[3] = ns * stage_bytes; out[4] = staging;
+    out[0] = bn; out[1] = ns; out[2] = mode; out[3] = ring; out[4] = staging;
     out[5] = P.off_raw; out[6] = P.off_bias; out[7] = P.off_bars; out[8] = P.total;
 }
 
