@@ -19,15 +19,25 @@ UNIT = {"byte": 1.0, "Kbyte": 1e3, "Mbyte": 1e6, "Gbyte": 1e9}
 
 
 def dram_bytes_per_launch(csv_path: str, kernel_regex: str):
-    rows = list(csv.reader(open(csv_path)))
-    hdr, units, data = rows[0], rows[1], rows[2:]
+    """Accepts both CSV forms ncu writes: the raw page of a report (one row per launch, one column per metric) and the
+    log of a ``--metrics ... --csv`` run (one row per launch and metric)."""
+    rows = [r for r in csv.reader(open(csv_path)) if len(r) > 5]
+    hdr = next(r for r in rows if "Kernel Name" in r)
     col = {h: i for i, h in enumerate(hdr)}
-    name_col = col["Kernel Name"]
-    rd, wr = col["dram__bytes_read.sum"], col["dram__bytes_write.sum"]
-    vals = []
-    for r in data:
-        if re.search(kernel_regex, r[name_col]):
-            vals.append(float(r[rd]) * UNIT[units[rd]] + float(r[wr]) * UNIT[units[wr]])
+    data = rows[rows.index(hdr) + 1:]
+    per_launch = {}
+    if "Metric Name" in col:
+        for r in data:
+            if r[col["Metric Name"]] in ("dram__bytes_read.sum", "dram__bytes_write.sum") and re.search(kernel_regex, r[col["Kernel Name"]]):
+                v = float(r[col["Metric Value"]].replace(",", "")) * UNIT[r[col["Metric Unit"]]]
+                per_launch[r[col["ID"]]] = per_launch.get(r[col["ID"]], 0.0) + v
+    else:
+        units = data[0]
+        rd, wr = col["dram__bytes_read.sum"], col["dram__bytes_write.sum"]
+        for r in data[1:]:
+            if re.search(kernel_regex, r[col["Kernel Name"]]):
+                per_launch[r[col["ID"]]] = float(r[rd]) * UNIT[units[rd]] + float(r[wr]) * UNIT[units[wr]]
+    vals = list(per_launch.values())
     if not vals:
         raise SystemExit(f"no launch matches {kernel_regex!r}")
     return sum(vals) / len(vals), len(vals)
