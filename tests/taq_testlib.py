@@ -18,7 +18,7 @@ TOL_REL_L2 = 1e-3
 # more: one code step of a row of d values moves that row's logits, and the softmax amplifies it.  Such rows must be few,
 # and their error stays under a bound of its own.
 TOL_MAX_ABS_TIE_ROWS = 6e-2
-MAX_TIE_ROW_FRACTION = {0: 0.02, 8: 0.25}          # by a_bits
+MAX_TIE_ROW_FRACTION = {0: 0.02, 8: 0.05}          # by a_bits (measured: at most 0.8 % and 2.8 %)
 
 
 def _log_parity(record):

@@ -114,7 +114,7 @@ def test_layer_forward_a8_matches_the_oracle(shape):
     y = y.cpu().numpy()
     assert np.isfinite(y).all()
     res = tl.check_layer(shape, data, y, {"desc": desc, "packed": P, "kv": kv, "mask": mask}, a_bits=8)
-    assert res["rows_with_q_flip"] <= 0.25 * res["rows"], res         # the end-to-end max-abs check kept most rows
+    assert res["rows_with_q_flip"] <= 0.05 * res["rows"] + 1, res   # (measured: at most 2.8 % of the rows)
     # the integer path is a different quantized network from the fp16-activation one, not a copy of it
     y16 = tl.gpu_layer(shape, data)
     assert tl.errors(y, y16)[1] > 1e-3, res
