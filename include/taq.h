@@ -264,6 +264,12 @@ taq_status taq_kv_set_prob_mask(const taq_layer_desc* desc, void* kv_packed_dev,
  * e.g. the K~/V~ blocks of all layers for one prompt; a multiple of 128, arena 128-byte aligned), never touches
  * the device and is safe to call from several host threads.  Entries in use by requests in flight are pinned;
  * a miss takes a free entry or evicts the least recently used unpinned one.
+ * Ordering is the caller's: the cache knows nothing of the GPU work.  A hit only says that the key was handed out
+ * before; the caller that got the miss must have ENQUEUED the fill (taq_kv_project_batched) before anyone acts on a
+ * hit for the same key, and the consumer must be ordered after that fill on the device (same stream, or an event).
+ * Likewise an entry is released only when the GPU work that reads it has been enqueued on a stream that later users
+ * of the (possibly evicted and refilled) entry are ordered behind.  One admission thread that acquires, fills and then
+ * publishes requests to the workers satisfies both.
  * -------------------------------------------------------------------------------------------------------- */
 typedef struct taq_kv_cache taq_kv_cache;
 typedef struct { int64_t capacity, used, hits, misses, evictions; } taq_kv_cache_stats;
