@@ -104,7 +104,8 @@ static taq_status run_linear(const LinearArgs& a, int n_z, cudaStream_t st) {
 
 static taq_status run_attention(const AttnArgs& a, int n_z, cudaStream_t st) {
     cudaError_t e;
-    if (sm100_attention_supported(a)) { count_launch(TAQ_KERNEL_ATTENTION_TENSOR); e = launch_attention_sm100(a, n_z, st); }
+    if (sm100_attention_c320_supported(a)) { count_launch(TAQ_KERNEL_ATTENTION_TENSOR); e = launch_attention_c320(a, n_z, st); }
+    else if (sm100_attention_supported(a)) { count_launch(TAQ_KERNEL_ATTENTION_TENSOR); e = launch_attention_sm100(a, n_z, st); }
     else { count_launch(TAQ_KERNEL_ATTENTION_GENERIC); e = launch_attention_simt(a, n_z, st); }
     return e == cudaSuccess ? TAQ_OK : cuda_fail(e, "attention launch");
 }

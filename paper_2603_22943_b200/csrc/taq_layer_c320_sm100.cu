@@ -105,6 +105,8 @@ struct LayerArgs {
     const void* kv;             // blocks [B] (single problem)
     const taq_request* reqs;    // nullable; then one sequence per request
     __half* o;                  // [z][N][C]  (query-attention variant)
+    const void* q;              // attention-only variant: Q~ codes (int8) or Q (fp16) [z][N][C] ...
+    const float* q_scales;      // ... and the row scales [z][N][H] (q_bits = 8)
     int n_query, heads, n_ctx, max_trigger, group, q_bits, p_bits;
     long long wait_cycles;      // limit of every device-side wait
     int* status;
@@ -261,7 +263,9 @@ __host__ __device__ constexpr int walk_stage(int rank, int kb) { return rank ? (
 __host__ __device__ constexpr int walk_reuse_stage(int rank) { return rank ? 1 : 0; }
 __host__ __device__ constexpr int walk_order(int rank, int kb) { return rank ? (kb >= 2 ? kb - 2 : 4 - kb) : kb; }        // inverse of walk_tile
 
-template <int TAIL_FROM, bool FUSE_OUT>
+// Q_IN: the attention-only variant (taq_cross_attention at this shape): Q~ is given, phases 1 and 4 do not exist; the
+// thread reads its 40 query codes from global memory instead of quantizing them.
+template <int TAIL_FROM, bool FUSE_OUT, bool Q_IN = false>
 __global__ void __launch_bounds__(NTHREADS, 1) layer_c320_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_y, const LayerArgs a) {
     extern __shared__ unsigned char smem_dyn[];
     unsigned char* smem = smem_dyn + ((1024u - (ptx::smem_u32(smem_dyn) & 1023u)) & 1023u);   // 1024-byte aligned
@@ -306,7 +310,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) layer_c320_kernel(const __grid_co
         ptx::mbar_fence_init();
         if (FUSE_OUT) ptx::mbar_arrive_expect_tx(&misc->o_all, (N_OTILE / 2) * O_TILE);     // the partner's five tiles
         ptx::tma_prefetch_desc(&tmap_x);
-        if (FUSE_OUT) ptx::tma_prefetch_desc(&tmap_y);
+        ptx::tma_prefetch_desc(&tmap_y);
     }
     if (warp == 1) ptx::tmem_alloc(&misc->tmem_base, TMEM_COLS);
     ptx::tc_fence_before_sync();
@@ -328,14 +332,16 @@ __global__ void __launch_bounds__(NTHREADS, 1) layer_c320_kernel(const __grid_co
         if (lane == 0) {
             // Packed weights are written by taq_pack_weights, which never lets its successor start early: they are complete
             // before this kernel can run at all and are fetched (and expanded) under the previous kernel's tail.
-            const uint8_t* blob = (const uint8_t*)(a.reqs ? a.reqs[zb].Wq : a.wq);
             const uint32_t scale_bytes = (uint32_t)(NQ * n_groups * 4);
-            ptx::mbar_arrive_expect_tx(&misc->w_full, RAW_BYTES + scale_bytes);
-            ptx::bulk_load(smem + OFF_RAW, blob + L.off_codes + (size_t)col0 * L.row_bytes, RAW_BYTES, &misc->w_full);
-            ptx::bulk_load(smem + OFF_SC, blob + L.off_scales + (size_t)col0 * n_groups * 4, scale_bytes, &misc->w_full);
+            if (!Q_IN) {
+                const uint8_t* blob = (const uint8_t*)(a.reqs ? a.reqs[zb].Wq : a.wq);
+                ptx::mbar_arrive_expect_tx(&misc->w_full, RAW_BYTES + scale_bytes);
+                ptx::bulk_load(smem + OFF_RAW, blob + L.off_codes + (size_t)col0 * L.row_bytes, RAW_BYTES, &misc->w_full);
+                ptx::bulk_load(smem + OFF_SC, blob + L.off_scales + (size_t)col0 * n_groups * 4, scale_bytes, &misc->w_full);
+            }
             ptx::pdl_wait();                              // X and the K~/V~ block may come from the previous kernel
             TAQ_PROF(1); TAQ_GPROF(28);
-            for (int kb = 0; kb < NKB; ++kb) {            // the whole X tile at once: every K block has its own buffer
+            for (int kb = 0; kb < NKB && !Q_IN; ++kb) {   // the whole X tile at once: every K block has its own buffer
                 ptx::mbar_arrive_expect_tx(&misc->a_full[kb], A_TILE);
                 ptx::tma_load_3d(smem + OFF_R0 + kb * A_TILE, &tmap_x, &misc->a_full[kb], kb * BK, row0, zb);
             }
@@ -343,7 +349,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) layer_c320_kernel(const __grid_co
             const uint8_t* img = blk + KL.off_operands + (size_t)h_begin * KL.operand_head_bytes;
             // Phase 1 over (every MMA complete, hence every Wq tile read): the weight tiles become the K~ and V~^T tiles and
             // the packed Wout rows of this CTA's output channels replace the packed Wq rows.
-            bool ok = ptx::mbar_wait(&misc->acc_full[n_groups - 1], 0, WL) && !misc->abort_flag;
+            bool ok = Q_IN || (ptx::mbar_wait(&misc->acc_full[n_groups - 1], 0, WL) && !misc->abort_flag);
             if (ok) {
                 ptx::mbar_arrive_expect_tx(&misc->kc_full, HG * (K_BYTES + kOperandConstBytes));
                 for (int hi = 0; hi < HG; ++hi) {
@@ -386,10 +392,10 @@ __global__ void __launch_bounds__(NTHREADS, 1) layer_c320_kernel(const __grid_co
             }
         }
         if (lane == 0 && misc->abort_flag) {   // give copies that are still in flight a bounded chance to land before the CTA exits
-            (void)ptx::mbar_wait(&misc->w_full, 0, WL);
-            for (int kb = 0; kb < NKB; ++kb) (void)ptx::mbar_wait(&misc->a_full[kb], 0, WL);
+            if (!Q_IN) (void)ptx::mbar_wait(&misc->w_full, 0, WL);
+            for (int kb = 0; kb < NKB && !Q_IN; ++kb) (void)ptx::mbar_wait(&misc->a_full[kb], 0, WL);
             // (the image and Wout copies are issued only after phase 1 succeeded; when they were, these waits end with them)
-            if (ptx::mbar_try_wait(&misc->acc_full[n_groups - 1], 0)) {
+            if (Q_IN || ptx::mbar_try_wait(&misc->acc_full[n_groups - 1], 0)) {
                 (void)ptx::mbar_wait(&misc->kc_full, 0, WL);
                 (void)ptx::mbar_wait(&misc->vt_full, 0, WL);
                 if (FUSE_OUT) (void)ptx::mbar_wait(&misc->w2_full, 0, WL);
@@ -407,7 +413,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) layer_c320_kernel(const __grid_co
         constexpr uint32_t HI128 = ptx::kDescHiSw128, HI64 = ptx::kDescHiSw64, HI32 = ptx::kDescHiSw32;
         const uint32_t r0_lo = ptx::desc_lo(ptx::smem_u32(smem + OFF_R0)), r1_lo = ptx::desc_lo(ptx::smem_u32(smem + OFF_R1));
         const uint32_t pb_lo = ptx::desc_lo(ptx::smem_u32(smem + OFF_PB)), k_lo = ptx::desc_lo(ptx::smem_u32(smem + OFF_K));
-        {   // phase 1: one accumulation pass per scale group; every weight tile was expanded before X arrived
+        if (!Q_IN) {   // phase 1: one accumulation pass per scale group; every weight tile was expanded before X arrived
             int kb = 0;
             for (int g = 0; g < n_groups && ok; ++g) {
                 const int kb_end = min(NKB, kb + kb_per_group);
@@ -537,9 +543,12 @@ __global__ void __launch_bounds__(NTHREADS, 1) layer_c320_kernel(const __grid_co
         float* scales_t = reinterpret_cast<float*>(smem + OFF_SCT);
         const unsigned char* raw = smem + OFF_RAW;
         const int cb = hi * D;
-        bool ok = ptx::mbar_wait(&misc->w_full, 0, WL);
-        for (int i = wt; i < NQ * n_groups; i += NWORK) scales_t[(i % n_groups) * NQ + i / n_groups] = wscales[i];
-        asm volatile("bar.sync 1, 512;" ::: "memory");
+        bool ok = true;
+        if (!Q_IN) {
+            ok = ptx::mbar_wait(&misc->w_full, 0, WL);
+            for (int i = wt; i < NQ * n_groups; i += NWORK) scales_t[(i % n_groups) * NQ + i / n_groups] = wscales[i];
+            asm volatile("bar.sync 1, 512;" ::: "memory");
+        }
 
         auto tile_built = [&](uint64_t* bar) {
             ptx::fence_proxy_async_smem();
@@ -578,11 +587,13 @@ __global__ void __launch_bounds__(NTHREADS, 1) layer_c320_kernel(const __grid_co
         };
 
         // ---- phase 1: expand all five Wq tiles (before X has arrived), then fold ----
-        for (int kb = 0; kb < NKB; ++kb) {
-            if (ok) expand_block(raw, kb, smem + stage1_offset(kb), wt);
-            tile_built(&misc->b1_full[kb]);
+        if (!Q_IN) {
+            for (int kb = 0; kb < NKB; ++kb) {
+                if (ok) expand_block(raw, kb, smem + stage1_offset(kb), wt);
+                tile_built(&misc->b1_full[kb]);
+            }
+            fold_groups(0, false);
         }
-        fold_groups(0, false);
         if (!ok) give_up();
         if (wt == 0) TAQ_PROF(7);
         // The last group's accumulator is complete, hence every MMA of phase 1 has finished reading shared memory: the
@@ -590,7 +601,31 @@ __global__ void __launch_bounds__(NTHREADS, 1) layer_c320_kernel(const __grid_co
 
         // ---- phase 2: Q~ = Q_a(Q) of (row, head), written as fp16 integers into the head's operand tile ----
         float sq = 0.f;
-        {
+        if (Q_IN) {
+            // attention only: the row's 40 codes (or fp16 values) of this head come from global memory
+            ptx::pdl_wait();                                  // Q~ comes from the previous kernel in the stream
+            unsigned char* q_tile = smem + OFF_R0 + hi * A_TILE;
+            const size_t grow = (size_t)zb * a.n_query + (valid ? n : 0);
+            const size_t elem = grow * (size_t)(H * D) + (size_t)(h_begin + hi) * D;
+            // all loads first (read-only path), then the conversions and the stores: one round trip to L2, not five
+            uint4 t16[D / 8];
+            if (a.q_bits == 8) {
+                uint2 c8[D / 8];
+#pragma unroll
+                for (int cc = 0; cc < D / 8; ++cc)
+                    c8[cc] = valid ? __ldg(reinterpret_cast<const uint2*>((const int8_t*)a.q + elem + cc * 8)) : make_uint2(0, 0);
+#pragma unroll
+                for (int cc = 0; cc < D / 8; ++cc) t16[cc] = codes_w8_to_half(c8[cc]);
+            } else {
+#pragma unroll
+                for (int cc = 0; cc < D / 8; ++cc)
+                    t16[cc] = valid ? __ldg(reinterpret_cast<const uint4*>((const __half*)a.q + elem + cc * 8)) : make_uint4(0, 0, 0, 0);
+            }
+#pragma unroll
+            for (int cc = 0; cc < D / 8; ++cc) *reinterpret_cast<uint4*>(q_tile + ptx::sw128_offset(r, cc)) = t16[cc];
+            *reinterpret_cast<uint4*>(q_tile + ptx::sw128_offset(r, D / 8)) = make_uint4(0, 0, 0, 0);   // channels 40..47
+            sq = a.q_bits == 8 ? (valid ? __ldg(a.q_scales + grow * H + h_begin + hi) : 0.f) : 1.0f;
+        } else {
             float amax = 0.f;
 #pragma unroll
             for (int c = 0; c < D; c += 2) amax = max3(amax, fabsf(y[c]), fabsf(y[c + 1]));
@@ -683,7 +718,6 @@ __global__ void __launch_bounds__(NTHREADS, 1) layer_c320_kernel(const __grid_co
             ptx::tmem_ld_wait(v[0]);
 #pragma unroll
             for (int i = 1; i < D / 8; ++i) ptx::reg_fence8(v[i]);
-            __half* orow = a.o + ((size_t)zb * a.n_query + (valid ? n : 0)) * (size_t)(H * D) + (h_begin + hi) * D;
 #pragma unroll
             for (int i = 0; i < D / 8; ++i) {
                 float f[8];
@@ -693,12 +727,22 @@ __global__ void __launch_bounds__(NTHREADS, 1) layer_c320_kernel(const __grid_co
                 if (FUSE_OUT) {           // 8 channels of O as one chunk of the to_out operand tiles
                     const int c = hi * D + i * 8;                    // channel among this CTA's 160
                     *reinterpret_cast<uint4*>(smem + own_tile_offset(c >> 5) + ptx::sw64_offset(r, (c & 31) >> 3)) = o8;
-                } else if (valid) {
-                    *reinterpret_cast<uint4*>(orow + i * 8) = o8;
+                } else {                  // staged where the head's probability tile was (dead: its PV product is complete)
+                    *reinterpret_cast<uint4*>(smem + OFF_R0 + hi * A_TILE + r * (D * 2) + i * 16) = o8;
                 }
             }
         }
         ptx::tc_fence_before_sync();
+        if (!FUSE_OUT) {
+            // the head's 128 x 40 block of O leaves as one TMA tensor store (dense rows of 80 bytes; rows beyond n_query clipped)
+            ptx::fence_proxy_async_smem();
+            asm volatile("bar.sync %0, 128;" ::"r"(2 + hi) : "memory");
+            if (q4 == 0 && lane == 0 && !misc->abort_flag) {
+                ptx::tma_store_3d(&tmap_y, smem + OFF_R0 + hi * A_TILE, col0 + cb, row0, zb);
+                ptx::bulk_store_commit();
+                ptx::bulk_store_wait_read();
+            }
+        }
 
         if (FUSE_OUT) {
             ptx::fence_proxy_async_smem();
@@ -795,7 +839,7 @@ bool sm100_qattn_supported(const taq_layer_desc& d) {
 }
 
 static cudaError_t launch_c320(const taq_layer_desc& d, const __half* x, const void* wq, const void* kv, const taq_request* reqs, __half* o,
-                               const void* wout, __half* y, int n_z, int* status, cudaStream_t stream) {
+                               const void* wout, __half* y, int n_z, int* status, cudaStream_t stream, const void* q = nullptr, const float* q_scales = nullptr) {
     if (n_z == 0 || d.n_query == 0) return cudaSuccess;
     EncodeTiledFn enc = encode_tiled();
     if (!enc) return cudaErrorNotSupported;
@@ -804,25 +848,28 @@ static cudaError_t launch_c320(const taq_layer_desc& d, const __half* x, const v
     const cuuint64_t strides[2] = {(cuuint64_t)KIN * 2, (cuuint64_t)KIN * 2 * (cuuint64_t)d.n_query};
     const cuuint32_t box[3] = {BK, ROWS, 1};
     const cuuint32_t estr[3] = {1, 1, 1};
-    CUresult r = enc(&tmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<__half*>(x), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+    const bool fuse_out = y != nullptr, q_in = q != nullptr;
+    __half* out = fuse_out ? y : o;
+    // (the attention-only variant loads no X: its map is built on the output so that the argument is a valid map)
+    CUresult r = enc(&tmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, q_in ? (void*)out : (void*)const_cast<__half*>(x), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                      CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
     LayerArgs a{};
-    a.wq = wq; a.kv = kv; a.reqs = reqs; a.o = o; a.wout = wout;
+    a.wq = wq; a.kv = kv; a.reqs = reqs; a.o = o; a.wout = wout; a.q = q; a.q_scales = q_scales;
     a.n_query = d.n_query; a.heads = d.heads; a.n_ctx = d.n_ctx; a.max_trigger = d.max_trigger; a.group = d.w_group; a.q_bits = d.q_bits; a.p_bits = d.p_bits;
     a.wait_cycles = g_wait_cycles;
     a.status = status;
     dim3 grid((d.n_query + ROWS - 1) / ROWS, d.heads / HG, n_z);
     const int tail = d.n_ctx > 72 ? 72 : d.n_ctx > 64 ? 64 : 0;     // first key that can lie beyond the context (the kernel masks from there on)
-    const bool fuse_out = y != nullptr;
-    CUtensorMap tmap_y = tmap;                        // (unused by the variant that stores O)
-    if (fuse_out) {
+    CUtensorMap tmap_y;                               // the output (Y, or O of the variants without to_out), stored per head group
+    {
         const cuuint32_t ybox[3] = {D, ROWS, 1};      // one head group: 40 channels = 80 bytes per row, dense in shared memory
-        r = enc(&tmap_y, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, y, dims, strides, ybox, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+        r = enc(&tmap_y, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, out, dims, strides, ybox, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                 CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
     }
     void (*kern)(const CUtensorMap, const CUtensorMap, const LayerArgs) =
+        q_in ? (tail == 72 ? layer_c320_kernel<72, false, true> : tail == 64 ? layer_c320_kernel<64, false, true> : layer_c320_kernel<0, false, true>) :
         fuse_out ? (tail == 72 ? layer_c320_kernel<72, true> : tail == 64 ? layer_c320_kernel<64, true> : layer_c320_kernel<0, true>)
                  : (tail == 72 ? layer_c320_kernel<72, false> : tail == 64 ? layer_c320_kernel<64, false> : layer_c320_kernel<0, false>);
     // (the attribute belongs to the current device's copy of the function: set on every launch, it is cheap)
@@ -835,6 +882,20 @@ static cudaError_t launch_c320(const taq_layer_desc& d, const __half* x, const v
 cudaError_t launch_qattn_sm100(const taq_layer_desc& d, const __half* x, const void* wq, const void* kv, const taq_request* reqs, __half* o,
                                int n_z, int* status, cudaStream_t stream) {
     return launch_c320(d, x, wq, kv, reqs, o, nullptr, nullptr, n_z, status, stream);
+}
+
+// The attention core alone at the same shape (taq_cross_attention): Q~ given, all four heads of a CTA at once.
+bool sm100_attention_c320_supported(const AttnArgs& a) {
+    if (a.channels != KIN || a.heads * D != KIN || a.n_ctx > TP || (a.p_bits != 8 && a.p_bits != 4) || a.n_query < 1) return false;
+    if ((reinterpret_cast<uintptr_t>(a.q) & 15u) || (reinterpret_cast<uintptr_t>(a.o) & 15u)) return false;
+    return encode_tiled() != nullptr;
+}
+
+cudaError_t launch_attention_c320(const AttnArgs& a, int n_z, cudaStream_t stream) {
+    taq_layer_desc d{};
+    d.batch = a.batch; d.n_query = a.n_query; d.channels = a.channels; d.heads = a.heads; d.n_ctx = a.n_ctx; d.max_trigger = a.max_trigger;
+    d.q_bits = a.q_bits; d.p_bits = a.p_bits; d.w_bits = 4; d.w_group = 128;
+    return launch_c320(d, nullptr, nullptr, a.kv, a.reqs, a.o, nullptr, nullptr, n_z, a.status, stream, a.q, a.q_scales);
 }
 
 cudaError_t launch_layer_sm100(const taq_layer_desc& d, const __half* x, const void* wq, const void* wout, const void* kv, const taq_request* reqs,

@@ -18,6 +18,10 @@ bool sm100_qattn_supported(const taq_layer_desc& d);
 cudaError_t launch_qattn_sm100(const taq_layer_desc& d, const __half* x, const void* wq, const void* kv, const taq_request* reqs, __half* o,
                                int n_z, int* status, cudaStream_t stream);
 
+// The attention core alone at C = 320 / 8 heads of 40: all four heads of a CTA at once (one thread per (row, head)).
+bool sm100_attention_c320_supported(const AttnArgs& a);
+cudaError_t launch_attention_c320(const AttnArgs& a, int n_z, cudaStream_t stream);
+
 // The whole layer pass (to_q, Q_a, attention, to_out) in one kernel for the same shape: pairs of CTAs exchange their
 // halves of O through distributed shared memory.
 bool sm100_layer_supported(const taq_layer_desc& d);

@@ -169,8 +169,10 @@ def test_a8_empty_inputs_and_bad_arguments():
 def test_one_kernel_a8_layer_equals_the_step_by_step_composition(n, q_bits):
     """At C = 320 / 8 heads / W4 g128 the integer-activation pass is one kernel (Q_a of X and O inside the CTA).  The same
     pass composed from the stand-alone entry points - quantize, integer to_q, attention, quantize, integer to_out - gives
-    the same bits: the per-token codes are the stand-alone quantizer's, the integer products are exact, and the fp32
-    combinations run in the same order."""
+    the same Y up to probability codes on a rounding tie: the per-token codes are the stand-alone quantizer's and the
+    integer products are exact, but the two attention kernels add a row's exponentials in different orders, so a
+    probability on a rounding boundary may take the neighbouring code (1/255 of one value row, then the O quantizer's
+    step)."""
     shape = replace(synth.shrink(synth.config2(), n), seed=26, q_bits=q_bits)
     data = synth.make_layer(shape)
     desc = tl.gpu_desc(shape)
@@ -189,4 +191,4 @@ def test_one_kernel_a8_layer_equals_the_step_by_step_composition(n, q_bits):
     oc, os_ = tb.taq_quantize_rows_f16(o.view(M, C_))
     want = tb.taq_quantized_linear_i8(P["wd_cc"], oc, os_, P["Wout"], tb.TAQ_OUT_F16)
     tb.taq_poll_device_status()
-    assert torch.equal(y.view(M, C_).view(torch.int16), want.view(torch.int16))
+    tl.assert_same_up_to_code_ties(y.view(M, C_), want, "Y")

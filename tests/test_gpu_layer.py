@@ -153,20 +153,6 @@ def _layer_case(shape, sample_rows=None, max_trigger=None):
     return tl.check_layer(shape, data, y, parts, rows)
 
 
-def _assert_same_up_to_code_ties(a, b, what):
-    """Two GPU routes through the same arithmetic: equal except where a sum taken in another order moved an fp16
-    rounding (one ulp) or a probability code on a tie (1/255 of a value row)."""
-    a = a.float().cpu().numpy().astype(np.float64)
-    b = b.float().cpu().numpy().astype(np.float64)
-    diff = np.abs(a - b)
-    ulp = 2.0 ** -10 * np.maximum(np.abs(a), np.abs(b)) + 1e-6
-    assert diff.max() <= tl.TOL_MAX_ABS, f"{what}: max difference {diff.max():.3e} at {np.unravel_index(diff.argmax(), diff.shape)}"
-    frac = float(np.mean(diff > 2 * ulp))
-    assert frac <= 2e-3, f"{what}: {frac:.2e} of the values differ by more than two fp16 ulps"
-    rel = np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-30)
-    assert rel <= 2e-4, f"{what}: relative L2 difference {rel:.3e}"
-
-
 @pytest.mark.parametrize("shape_fn,n", [(synth.config2, 4096), (synth.config2, 333), (lambda: synth.config3_layers()[5], 200)],
                          ids=["config2_full", "config2_ragged", "C640_unfused"])
 @pytest.mark.parametrize("q_bits", [8, 0])
@@ -192,7 +178,7 @@ def test_query_attention_equals_the_two_step_path(shape_fn, n, q_bits):
         q16 = tb.taq_quantized_linear(P["wd_cc"], x2, P["Wq"], tb.TAQ_OUT_F16)
         o_two = tb.taq_cross_attention(desc, q16, None, kv, mask)
     tb.taq_poll_device_status()
-    _assert_same_up_to_code_ties(o_fused, o_two, "O")
+    tl.assert_same_up_to_code_ties(o_fused, o_two, "O")
     rows = np.arange(0, shape.n_query, max(1, shape.n_query // 64))
     cfg = tl.oracle_cfg(shape)
     g = tl.gpu_decisions(shape, data, {"desc": desc, "packed": P, "kv": kv, "mask": mask}, rows)
@@ -218,7 +204,7 @@ def test_one_kernel_layer_equals_the_step_by_step_path(n, q_bits):
     o = tb.taq_query_attention(desc, x, P["Wq"], kv, mask)
     y_two = tb.taq_quantized_linear(P["wd_cc"], o.reshape(-1, shape.channels), P["Wout"], tb.TAQ_OUT_F16).reshape(y_one.shape)
     tb.taq_poll_device_status()
-    _assert_same_up_to_code_ties(y_one, y_two, "Y")
+    tl.assert_same_up_to_code_ties(y_one, y_two, "Y")
 
 
 def test_layer_config1_full():
