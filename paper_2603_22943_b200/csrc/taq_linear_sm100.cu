@@ -34,6 +34,7 @@ constexpr int BM = 128;
 constexpr int BK = 64;                     // fp16 elements per 128-byte operand row; the int8 variant has 2 BK
 constexpr int MAX_STAGE = 6;
 constexpr int MAX_PREBUILT = 12;           // k-blocks per CTA whose expanded weight tiles may all be resident at once
+constexpr int MAX_ACC = 8;                  // TMEM accumulators (scale groups in flight) per CTA
 constexpr int NWORK = 256;                  // worker threads: two per accumulator row
 constexpr int NTHREADS = 64 + NWORK;
 constexpr int A_TILE_BYTES = BM * BK * 2;   // 16 KB
@@ -54,8 +55,8 @@ struct Bars {
     uint64_t full_b[MAX_PREBUILT];
     uint64_t empty[MAX_STAGE];
     uint64_t w_full;
-    uint64_t acc_full[2];
-    uint64_t acc_free[2];
+    uint64_t acc_full[MAX_ACC];
+    uint64_t acc_free[MAX_ACC];
     uint64_t part_full[8], part_got[8], peer_ready;   // K loop split over a CTA pair: hand-over of the second CTA's partial sums
     uint32_t tmem_base;
     volatile int abort_flag;
@@ -100,7 +101,7 @@ __host__ __device__ inline Plan make_plan(int k_in, int bits, int group, int nst
 // they exchange folded fp32 partial sums through bulk copies between the two shared memories, the first CTA adding and
 // storing rows 0..63 of the tile, the second rows 64..127.
 template <int BN, bool I8, bool SPLIT>
-__global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w, const LinearArgs a, const int nstage, const int prebuilt) {
+__global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_y, const LinearArgs a, const int nstage, const int prebuilt) {
     using TL = Tile<BN>;
     constexpr int BKE = I8 ? 2 * BK : BK;             // elements per K block
     constexpr int HC = TL::HC;
@@ -109,7 +110,6 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
     const Plan P = make_plan<BN>(a.k_in, a.bits, a.group, nstage, a.w_direct, prebuilt);
     static_assert(sizeof(Bars) <= 512, "barrier block");
     Bars* bars = reinterpret_cast<Bars*>(smem + P.off_bars);
-    constexpr uint32_t TMEM_COLS = TL::TMEM_COLS;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int z = blockIdx.z;
@@ -127,6 +127,12 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
     const int g_begin = SPLIT && !split_kb && rank ? n_groups / 2 : 0, g_end = SPLIT && !split_kb && !rank ? n_groups / 2 : n_groups;
     const int kb_begin = split_kb ? (rank ? n_kb / 2 : 0) : g_begin * kb_per_group;
     const int kb_stop = split_kb ? (rank ? n_kb : n_kb / 2) : min(n_kb, g_end * kb_per_group);
+    // Accumulators: two (the workers fold one while the tensor core fills the other), or, when the weight tiles are all
+    // built before the first fold (prebuilt), one per scale group of the CTA as far as TMEM holds them, so that no MMA
+    // waits for a fold.
+    const int n_acc = prebuilt ? max(1, min(min(g_end - g_begin, 512 / BN), MAX_ACC)) : 2;
+    uint32_t tmem_cols = TL::TMEM_COLS;
+    if (prebuilt) for (tmem_cols = 32; tmem_cols < (uint32_t)(n_acc * BN); tmem_cols *= 2) {}
     constexpr uint32_t PART_ROW = (uint32_t)BN * 2u + 16u;           // a thread's fp32 partial sums (BN / 2 columns), padded against bank conflicts
 
     TAQ_PROF_INIT
@@ -138,7 +144,7 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
         }
         for (int s = 0; s < MAX_PREBUILT; ++s) ptx::mbar_init(&bars->full_b[s], NWORK / 32);    // one arrival per worker warp
         ptx::mbar_init(&bars->w_full, 1);
-        for (int i = 0; i < 2; ++i) {
+        for (int i = 0; i < MAX_ACC; ++i) {
             ptx::mbar_init(&bars->acc_full[i], 1);
             ptx::mbar_init(&bars->acc_free[i], NWORK / 32);
         }
@@ -151,7 +157,7 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
                 if (((i & 3) >> 1) == rank) ptx::mbar_arrive_expect_tx(&bars->part_full[i], 32u * PART_ROW);
         ptx::tma_prefetch_desc(&tmap_x);
     }
-    if (warp == 1) ptx::tmem_alloc(&bars->tmem_base, TMEM_COLS);
+    if (warp == 1) ptx::tmem_alloc(&bars->tmem_base, tmem_cols);
     ptx::tc_fence_before_sync();
     __syncthreads();
     ptx::tc_fence_after_sync();
@@ -201,9 +207,9 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
         bool ok = true;
         for (int g = g_begin; g < g_end && ok; ++g) {
             const int gl = g - g_begin;
-            const int buf = gl & 1;
-            if (gl >= 2) {                                  // the workers have emptied this accumulator
-                if (!wait(&bars->acc_free[buf], ((gl >> 1) - 1) & 1)) { ok = false; break; }
+            const int buf = gl % n_acc;
+            if (gl >= n_acc) {                              // the workers have emptied this accumulator
+                if (!wait(&bars->acc_free[buf], (gl / n_acc - 1) & 1)) { ok = false; break; }
                 ptx::tc_fence_after_sync();
             }
             const int kb_end = min(kb_stop, kb + kb_per_group);
@@ -229,8 +235,7 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
         if (!ok && leader) {
             raise_status(a.status, TAQ_ERR_TIMEOUT);
             bars->abort_flag = 1;
-            ptx::mma_commit(&bars->acc_full[0]);        // wake the workers; they see the abort flag
-            ptx::mma_commit(&bars->acc_full[1]);
+            for (int i = 0; i < n_acc; ++i) ptx::mma_commit(&bars->acc_full[i]);        // wake the workers; they see the abort flag
         }
     } else {
         // ---------------- workers (warps 2..9) ----------------
@@ -260,8 +265,8 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
 
         // y += scale[g] * accumulator of group g (this thread's HC columns of its row)
         auto fold_group = [&](int g) -> bool {
-            const int buf = (g - g_begin) & 1;
-            if (!ptx::mbar_wait(&bars->acc_full[buf], ((g - g_begin) >> 1) & 1) || bars->abort_flag) return false;
+            const int buf = (g - g_begin) % n_acc;
+            if (!ptx::mbar_wait(&bars->acc_full[buf], ((g - g_begin) / n_acc) & 1) || bars->abort_flag) return false;
             ptx::tc_fence_after_sync();
             const float* sg = scales_t + g * BN + cb;
 #pragma unroll
@@ -358,8 +363,43 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
             return true;
         };
 
+        // prebuilt (fp16 activations, codes staged): two tiles per pass, all loads before the conversions and the stores, one
+        // proxy fence for both
+        auto build_pair = [&](int kb0, int ntile) {
+            constexpr int NCH = (BN * 8 + NWORK - 1) / NWORK;
+            const int n0 = wt >> 3, c = wt & 7;
+            uint2 pw[2][NCH];
+#pragma unroll
+            for (int t = 0; t < 2; ++t)
+#pragma unroll
+                for (int i = 0; i < NCH; ++i) {
+                    const int n = n0 + (NWORK / 8) * i;
+                    pw[t][i] = make_uint2(0, 0);
+                    if (t < ntile && ((BN * 8) % NWORK == 0 || n < BN)) {
+                        if (a.bits == 4) pw[t][i].x = *reinterpret_cast<const uint32_t*>(raw + n * row_bytes + (kb0 + t) * (BK / 2) + c * 4);
+                        else pw[t][i] = *reinterpret_cast<const uint2*>(raw + n * row_bytes + (kb0 + t) * BK + c * 8);
+                    }
+                }
+#pragma unroll
+            for (int t = 0; t < 2; ++t) {
+                unsigned char* b_tile = smem + P.off_ball + (kb0 + t - kb_begin) * TL::B_TILE_BYTES;
+#pragma unroll
+                for (int i = 0; i < NCH; ++i) {
+                    const int n = n0 + (NWORK / 8) * i;
+                    if (t < ntile && ((BN * 8) % NWORK == 0 || n < BN))
+                        *reinterpret_cast<uint4*>(b_tile + ptx::sw128_offset(n, c)) = a.bits == 4 ? codes_w4_to_half(pw[t][i].x) : codes_w8_to_half(pw[t][i]);
+                }
+            }
+            ptx::fence_proxy_async_smem();
+            __syncwarp();
+            if (lane < ntile) ptx::mbar_arrive(&bars->full_b[kb0 + lane - kb_begin]);
+            if (wt == 0 && kb0 < 20) TAQ_PROF(60 + kb0);
+        };
+
         if (prebuilt) {            // every weight tile first (nothing to wait for), then the folds as the groups complete
-            for (int g = g_begin; g < g_end && ok; ++g) ok = build_group(g);
+            if (!I8)
+                for (int k2 = kb_begin; k2 < kb_stop && !bars->abort_flag; k2 += 2) build_pair(k2, min(2, kb_stop - k2));
+            ok = !bars->abort_flag;
             for (int g = g_begin; g < g_end && ok; ++g) ok = fold_group(g);
         } else {
             for (int g = g_begin; g < g_end && ok; ++g) {
@@ -427,14 +467,23 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
         }
 
         // ---------------- epilogue on this thread's HC columns ----------------
+        // Dense outputs (fp16, fp32, int8 codes) are staged in shared memory as the plain [128][BN] tile (the ring is free
+        // now) and leave by one TMA store per 32 rows, issued as soon as the two warps that own those rows have written
+        // them; the tensor map clips rows beyond the matrix.
+        const bool stores_rows = !SPLIT || (((warp - 2) & 3) >> 1) == rank;
+        auto store_quarter = [&](int esz) {
+            ptx::fence_proxy_async_smem();
+            asm volatile("bar.sync %0, 64;" ::"r"(3 + q) : "memory");
+            if (half == 0 && lane == 0 && stores_rows && (long long)row0 + q * 32 < a.rows) {
+                ptx::tma_store_3d(&tmap_y, smem + (size_t)q * 32 * BN * esz, col0, row0 + q * 32, z);
+                ptx::bulk_store_commit();
+                ptx::bulk_store_wait_read();
+            }
+        };
         if (ok) {
             if (a.epi == EPI_F16 || a.epi == EPI_F32) {
-                // The thread's HC outputs are one contiguous piece of its row: stage them in shared memory (the ring
-                // is free now; pieces are padded by 16 bytes against bank conflicts) and hand the piece to the copy
-                // engine, instead of 16-byte stores scattered over 128 rows per warp.
                 const int esz = a.epi == EPI_F16 ? 2 : 4;
-                unsigned char* seg = smem + (size_t)(half * 128 + r) * (HC * esz + 16);
-                const size_t o = ((size_t)z * a.rows + row) * a.n_out + col0 + cb;
+                unsigned char* seg = smem + ((size_t)r * BN + cb) * esz;
 #pragma unroll
                 for (int c = 0; c < HC; c += 8) {
                     float f[8];
@@ -447,12 +496,7 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
                         *reinterpret_cast<float4*>(seg + c * 4 + 16) = make_float4(f[4], f[5], f[6], f[7]);
                     }
                 }
-                ptx::fence_proxy_async_smem();
-                if (row < a.rows) {
-                    ptx::bulk_store((unsigned char*)a.y + o * esz, seg, HC * esz);
-                    ptx::bulk_store_commit();
-                    ptx::bulk_store_wait_read();
-                }
+                store_quarter(esz);
             } else {
                 // Per-(row, head) symmetric int8.  A thread's columns are either whole heads (HC a multiple of d) or half
                 // of the tile's single head (d = BN); in the second case the row's two threads exchange their absmax.
@@ -496,25 +540,11 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
                     const bool owner = whole_heads || half == 0;      // writes the head's scale
                     if (a.epi == EPI_Q8_HEAD) {
                         // Q~ = Q_a(Q), Eq. 2 third line
-                        int8_t* dst = (int8_t*)a.y + ((size_t)z * a.rows + row) * a.n_out + col0 + cb;
-                        if (HC % 16 == 0) {       // the codes of the thread's piece leave through shared memory in one bulk store
-                            unsigned char* seg = smem + (size_t)(half * 128 + r) * (HC + 16);
+                        unsigned char* seg = smem + (size_t)r * BN + cb;
 #pragma unroll
-                            for (int c = 0; c < HC; c += 8)
-                                if (c >= hc && c < hc + dd) *reinterpret_cast<uint2*>(seg + c) = quant8(y + c, rs);
-                            if (hc + dd >= HC) {  // last head of the piece
-                                ptx::fence_proxy_async_smem();
-                                if (row < a.rows) {
-                                    ptx::bulk_store(dst, seg, HC);
-                                    ptx::bulk_store_commit();
-                                    ptx::bulk_store_wait_read();
-                                }
-                            }
-                        } else if (row < a.rows) {
-#pragma unroll
-                            for (int c = 0; c < HC; c += 8)
-                                if (c >= hc && c < hc + dd) *reinterpret_cast<uint2*>(dst + c) = quant8(y + c, rs);
-                        }
+                        for (int c = 0; c < HC; c += 8)
+                            if (c >= hc && c < hc + dd) *reinterpret_cast<uint2*>(seg + c) = quant8(y + c, rs);
+                        if (hc + dd >= HC) store_quarter(1);  // last head of the piece
                         if (row < a.rows && owner) a.scales[((size_t)z * a.rows + row) * a.heads + h] = s;
                     } else if (row < a.rows) {
                         // Eq. 2 for K or V: rows of ordinary tokens -> int8 codes + scale, rows of trigger tokens -> fp16
@@ -559,7 +589,7 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
     if (tid == 0) { TAQ_PROF(9); TAQ_GPROF(29); }
     if (warp == 1) {
         ptx::tc_fence_after_sync();
-        ptx::tmem_dealloc(tmem_base, TMEM_COLS);
+        ptx::tmem_dealloc(tmem_base, tmem_cols);
     }
 }
 
@@ -590,14 +620,12 @@ int weight_mode(const LinearArgs& a) {
     return make_plan<BN>(a.k_in, a.bits, a.group, 2, 0).total > SMEM_LIMIT ? (a.reqs ? 0 : 2) : 0;
 }
 
-// Bytes of the ring that the epilogue reuses to stage a tile's output before the bulk stores: every one of the 256 worker
-// threads owns one piece of HC elements plus 16 bytes of padding.
+// Bytes of the ring that the epilogue reuses to stage a tile's output before the TMA stores: the dense [128][BN] tile.
 template <int BN>
 int epilogue_staging_bytes(const LinearArgs& a) {
-    constexpr int HC = Tile<BN>::HC;
-    if (a.epi == EPI_F16) return NWORK * (HC * 2 + 16);
-    if (a.epi == EPI_F32) return NWORK * (HC * 4 + 16);
-    if (a.epi == EPI_Q8_HEAD && HC % 16 == 0) return NWORK * (HC + 16);
+    if (a.epi == EPI_F16) return BM * BN * 2;
+    if (a.epi == EPI_F32) return BM * BN * 4;
+    if (a.epi == EPI_Q8_HEAD) return BM * BN;
     return 0;
 }
 
@@ -677,12 +705,17 @@ Choice choose(const LinearArgs& a, int n_z) {
                 if (Lw.n_groups == 1) n_cta = n_kb - n_kb / 2;
                 else { const int kbg = Lw.group_len / bke, lo = (Lw.n_groups / 2) * kbg; n_cta = lo > n_kb - lo ? lo : n_kb - lo; }
             }
-            const int ns = n_cta < 3 ? 2 : 3;
-            const Plan P = make_plan<BN>(a.k_in, a.bits, a.group, ns, 0, n_cta);
-            if (n_cta <= MAX_PREBUILT && P.total <= SMEM_LIMIT && P.off_raw >= staging && (!with_split || P.off_raw >= part)) {
-                c.ns = ns; c.prebuilt = n_cta; c.split = with_split != 0;
-                break;
+            // the activation ring as deep as shared memory allows: with the weight tiles resident the K loop's pace is
+            // the latency of the activation loads divided by the loads in flight
+            bool found = false;
+            for (int ns = n_cta < MAX_STAGE ? (n_cta < 2 ? 2 : n_cta) : MAX_STAGE; ns >= (n_cta < 3 ? 2 : 3) && !found; --ns) {
+                const Plan P = make_plan<BN>(a.k_in, a.bits, a.group, ns, 0, n_cta);
+                if (n_cta <= MAX_PREBUILT && P.total <= SMEM_LIMIT && P.off_raw >= staging && (!with_split || P.off_raw >= part)) {
+                    c.ns = ns; c.prebuilt = n_cta; c.split = with_split != 0;
+                    found = true;
+                }
             }
+            if (found) break;
         }
     }
     return c;
@@ -694,7 +727,7 @@ cudaError_t launch_bn(const CUtensorMap& tmap, EncodeTiledFn enc, LinearArgs a, 
     const Choice ch = choose<BN>(a, n_z);
     const int ns = ch.ns;
     const bool split = ch.split;
-    void (*kern)(const CUtensorMap, const CUtensorMap, const LinearArgs, const int, const int) =
+    void (*kern)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const LinearArgs, const int, const int) =
         split ? (i8 ? linear_sm100_kernel<BN, true, true> : linear_sm100_kernel<BN, false, true>)
               : (i8 ? linear_sm100_kernel<BN, true, false> : linear_sm100_kernel<BN, false, false>);
     a.w_direct = weight_mode<BN>(a);
@@ -703,9 +736,19 @@ cudaError_t launch_bn(const CUtensorMap& tmap, EncodeTiledFn enc, LinearArgs a, 
         const WeightLayout L = weight_layout(a.n_out, a.k_in, a.bits, a.group);
         const cuuint64_t dims[3] = {(cuuint64_t)a.k_in, (cuuint64_t)a.n_out, 1};
         const cuuint64_t strides[2] = {(cuuint64_t)L.row_bytes, (cuuint64_t)L.row_bytes * (cuuint64_t)a.n_out};
-        const cuuint32_t box[3] = {a.w_direct == 1 ? 2 * BK : BK, BN, 1}, estr[3] = {1, 1, 1};    // mode 2: plain rows of 64 codes
+        const cuuint32_t box[3] = {(cuuint32_t)(a.w_direct == 1 ? 2 * BK : BK), BN, 1}, estr[3] = {1, 1, 1};    // mode 2: plain rows of 64 codes
         CUresult r = enc(&tmap_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, (void*)((const uint8_t*)a.w + L.off_codes), dims, strides, box, estr,
                          CU_TENSOR_MAP_INTERLEAVE_NONE, a.w_direct == 1 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+    }
+    CUtensorMap tmap_y = tmap;                        // (unused by the K~/V~ epilogue, which scatters into the cache block)
+    if (a.epi == EPI_F16 || a.epi == EPI_F32 || a.epi == EPI_Q8_HEAD) {   // the output matrix [n_z][rows][n_out] in boxes of 32 rows x BN
+        const cuuint64_t esz = a.epi == EPI_F16 ? 2 : a.epi == EPI_F32 ? 4 : 1;
+        const cuuint64_t dims[3] = {(cuuint64_t)a.n_out, (cuuint64_t)a.rows, (cuuint64_t)n_z};
+        const cuuint64_t strides[2] = {(cuuint64_t)a.n_out * esz, (cuuint64_t)a.n_out * esz * (cuuint64_t)a.rows};
+        const cuuint32_t box[3] = {BN, 32, 1}, estr[3] = {1, 1, 1};
+        CUresult r = enc(&tmap_y, a.epi == EPI_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : a.epi == EPI_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_UINT8,
+                         3, a.y, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
     }
     {   // (the attribute belongs to the current device's copy of the function: set on every launch, it is cheap)
@@ -714,8 +757,8 @@ cudaError_t launch_bn(const CUtensorMap& tmap, EncodeTiledFn enc, LinearArgs a, 
     }
     const Plan P = make_plan<BN>(a.k_in, a.bits, a.group, ns, a.w_direct, ch.prebuilt);
     dim3 grid((unsigned)((a.rows + BM - 1) / BM) * (split ? 2u : 1u), a.n_out / BN, n_z);
-    if (split) return launch_pdl_cluster(kern, grid, dim3(2, 1, 1), dim3(NTHREADS), (size_t)P.total, stream, tmap, tmap_w, a, ns, ch.prebuilt);
-    return launch_pdl(kern, grid, dim3(NTHREADS), (size_t)P.total, stream, tmap, tmap_w, a, ns, ch.prebuilt);
+    if (split) return launch_pdl_cluster(kern, grid, dim3(2, 1, 1), dim3(NTHREADS), (size_t)P.total, stream, tmap, tmap_w, tmap_y, a, ns, ch.prebuilt);
+    return launch_pdl(kern, grid, dim3(NTHREADS), (size_t)P.total, stream, tmap, tmap_w, tmap_y, a, ns, ch.prebuilt);
 }
 
 }  // namespace
@@ -730,6 +773,7 @@ bool sm100_linear_supported(const LinearArgs& a) {
         if (a.group != 0 && a.group % BK) return false;
         if (reinterpret_cast<uintptr_t>(a.x) & 15u) return false;
     }
+    if (a.epi != EPI_KV && (reinterpret_cast<uintptr_t>(a.y) & 15u)) return false;   // the output leaves by TMA stores
     if (a.rows < 1 || a.rows > (1LL << 31) - 1) return false;
     const int bn = pick_bn(a);
     if (bn == 0) return false;

@@ -154,7 +154,7 @@ def test_linear_plan_keeps_every_region_inside_shared_memory(L):
     assert seen > 1000
     # the case that used to overflow: a 160-wide fp32 tile over a fan-in of 128 (two K blocks)
     plan = tb.taq_linear_plan(tb.weight_desc(320, 128, 4, 128), 8192, tb.TAQ_OUT_F32)
-    assert plan["bn"] == 160 and plan["staging_bytes"] == 256 * (80 * 4 + 16) and plan["ring_bytes"] >= plan["staging_bytes"]
+    assert plan["bn"] == 160 and plan["staging_bytes"] == 128 * 160 * 4 and plan["ring_bytes"] >= plan["staging_bytes"]
 
 
 def test_dispatch_counters_start_at_zero_and_reset(L):
