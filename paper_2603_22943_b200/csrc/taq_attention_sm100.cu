@@ -41,7 +41,13 @@ struct Cfg {
     static constexpr int OFF_KV = 0;
     static constexpr int OFF_Q = OFF_KV + KVBUF * HEAD_BYTES;
     static constexpr int OFF_P = OFF_Q + KBQ * A_BLOCK;
-    static constexpr int OFF_MISC = OFF_P + 2 * A_BLOCK;
+    // One image buffer (wide heads): the next head's K~ loads as soon as this head's S is complete and its V~^T as soon
+    // as this head's PV is, each with a barrier of its own; the constants of a head then live in a rotating slot of their
+    // own (three slots: the softmax of head h - 1 may still read its slot when the constants of head h + 1 arrive).
+    static constexpr bool SPLIT_KV = KVBUF == 1;
+    static constexpr int CST_SLOT = 384;
+    static constexpr int OFF_CST = OFF_P + 2 * A_BLOCK;
+    static constexpr int OFF_MISC = OFF_CST + (SPLIT_KV ? 3 * CST_SLOT : 0);
     static constexpr int TOTAL = OFF_MISC + 4096 + 128 + 1024;   // misc block + slack for 1024-byte alignment
     static constexpr uint32_t TMEM_S = 0, TMEM_O = 2 * TP;
     static constexpr uint32_t TMEM_COLS = (2 * TP + OBUF * DP) <= 256 ? 256 : 512;
@@ -57,6 +63,7 @@ struct Misc {
     float2 xchg[2][2][ROWS];     // [head parity][half][row]: (max, sum) of a thread's half of the softmax
 };
 static_assert(sizeof(Misc) <= 4096 + 128, "misc block");
+static_assert(sizeof(OperandConsts) % 16 == 0 && sizeof(OperandConsts) <= 384, "constants slot");
 
 // Half of the query codes (or fp16 values) of one row and head, held in registers between the global load and
 // the store into the operand tile: the row's two threads take the lower and the upper half of the 16-byte chunks.
@@ -137,6 +144,28 @@ __global__ void __launch_bounds__(ATT_THREADS, Cfg<D>::CTAS_PER_SM) attention_sm
             const uint8_t* blk = a.reqs ? (const uint8_t*)a.reqs[zb].kv : (const uint8_t*)a.kv + (size_t)b * KL.block_bytes;
             const uint8_t* img = blk + KL.off_operands + (size_t)h_begin * KL.operand_head_bytes;
             int issued = 0;
+            if (C::SPLIT_KV) {
+                // kv_full[0]: K~ and the constants of a head; kv_full[1]: its V~^T
+                int issued_v = 0;
+                for (int hi = 0; hi < HG; ++hi) {
+                    if (hi >= 1 && !ptx::mbar_wait(&misc->s_full[(hi - 1) & 1], ((hi - 1) >> 1) & 1)) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; }
+                    if (misc->abort_flag) break;
+                    const uint8_t* src = img + (size_t)hi * KL.operand_head_bytes;
+                    ptx::mbar_arrive_expect_tx(&misc->kv_full[0], C::K_BYTES + (uint32_t)sizeof(OperandConsts));
+                    ptx::bulk_load(smem + C::OFF_KV, src, C::K_BYTES, &misc->kv_full[0]);
+                    ptx::bulk_load(smem + C::OFF_CST + (hi % 3) * C::CST_SLOT, src + C::K_BYTES + C::VT_BYTES, (uint32_t)sizeof(OperandConsts), &misc->kv_full[0]);
+                    issued = hi + 1;
+                    if (hi >= 1 && !ptx::mbar_wait(&misc->kv_free[0], (hi - 1) & 1)) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; }
+                    if (misc->abort_flag) break;
+                    ptx::mbar_arrive_expect_tx(&misc->kv_full[1], C::VT_BYTES);
+                    ptx::bulk_load(smem + C::OFF_KV + C::K_BYTES, src + C::K_BYTES, C::VT_BYTES, &misc->kv_full[1]);
+                    issued_v = hi + 1;
+                }
+                if (misc->abort_flag) {   // let copies that were issued land before the CTA goes away
+                    if (issued) (void)ptx::mbar_wait(&misc->kv_full[0], (issued - 1) & 1);
+                    if (issued_v) (void)ptx::mbar_wait(&misc->kv_full[1], (issued_v - 1) & 1);
+                }
+            } else {
             for (int hi = 0; hi < HG; ++hi) {
                 const int buf = hi % C::KVBUF;
                 if (hi >= C::KVBUF && !ptx::mbar_wait(&misc->kv_free[buf], ((hi / C::KVBUF) - 1) & 1)) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; }
@@ -147,6 +176,7 @@ __global__ void __launch_bounds__(ATT_THREADS, Cfg<D>::CTAS_PER_SM) attention_sm
             }
             if (misc->abort_flag) {   // let copies that were issued land before the CTA goes away
                 for (int hi = issued > C::KVBUF ? issued - C::KVBUF : 0; hi < issued; ++hi) (void)ptx::mbar_wait(&misc->kv_full[hi % C::KVBUF], (hi / C::KVBUF) & 1);
+            }
             }
         }
     } else if (warp == MMA_WARP) {
@@ -159,7 +189,7 @@ __global__ void __launch_bounds__(ATT_THREADS, Cfg<D>::CTAS_PER_SM) attention_sm
         const uint32_t kv_lo0 = ptx::desc_lo(ptx::smem_u32(smem + C::OFF_KV));
         auto issue_s = [&](int hi) -> bool {
             const int buf = hi % C::KVBUF;
-            if (!wait(&misc->kv_full[buf], (hi / C::KVBUF) & 1) || !wait(&misc->q_full, hi & 1)) return false;
+            if (!wait(&misc->kv_full[buf], C::SPLIT_KV ? (hi & 1) : (hi / C::KVBUF) & 1) || !wait(&misc->q_full, hi & 1)) return false;
             ptx::tc_fence_after_sync();
             if (leader) {
                 const uint32_t k_lo = kv_lo0 + buf * (C::HEAD_BYTES >> 4);
@@ -173,6 +203,7 @@ __global__ void __launch_bounds__(ATT_THREADS, Cfg<D>::CTAS_PER_SM) attention_sm
         };
         auto issue_pv = [&](int hi) -> bool {
             const int buf = hi % C::KVBUF;
+            if (C::SPLIT_KV && !wait(&misc->kv_full[1], hi & 1)) return false;
             if (!wait(&misc->p_full, hi & 1)) return false;
             ptx::tc_fence_after_sync();
             if (leader) {
@@ -191,9 +222,13 @@ __global__ void __launch_bounds__(ATT_THREADS, Cfg<D>::CTAS_PER_SM) attention_sm
             if (C::KVBUF == 2) {          // S of the next head first: it runs under this head's softmax
                 if (hi + 1 < HG) ok = issue_s(hi + 1);
                 if (ok) ok = issue_pv(hi);
-            } else {                      // one K~/V~ buffer: the next head's image lands only after this PV
-                ok = issue_pv(hi);
-                if (ok && hi + 1 < HG) ok = issue_s(hi + 1);
+            } else {
+                // one image buffer: the next head's K~ arrives some time after this head's S; its S goes first if K~
+                // and Q~ are there already (it then runs under this head's softmax), else after this head's PV
+                const bool early = hi + 1 < HG && __all_sync(0xffffffffu, ptx::mbar_try_wait(&misc->kv_full[0], (hi + 1) & 1) && ptx::mbar_try_wait(&misc->q_full, (hi + 1) & 1)) != 0;
+                if (early) ok = issue_s(hi + 1);
+                if (ok) ok = issue_pv(hi);
+                if (ok && !early && hi + 1 < HG) ok = issue_s(hi + 1);
             }
         }
         if (!ok) {                        // wait (bounded) for whatever was issued before TMEM is given back
@@ -284,7 +319,8 @@ __global__ void __launch_bounds__(ATT_THREADS, Cfg<D>::CTAS_PER_SM) attention_sm
             if (more) stage_q(qr);              // S of this head is complete, so the Q~ tile is free again
 
             // ---- this thread's half of the softmax; the row's two threads then exchange (max, sum) ----
-            const OperandConsts* cst = reinterpret_cast<const OperandConsts*>(smem + C::OFF_KV + (hi % C::KVBUF) * C::HEAD_BYTES + C::K_BYTES + C::VT_BYTES);
+            const OperandConsts* cst = C::SPLIT_KV ? reinterpret_cast<const OperandConsts*>(smem + C::OFF_CST + (hi % 3) * C::CST_SLOT)
+                                                   : reinterpret_cast<const OperandConsts*>(smem + C::OFF_KV + (hi % C::KVBUF) * C::HEAD_BYTES + C::K_BYTES + C::VT_BYTES);
             float e[HK];
             float m_loc, l_loc;
             softmax_half<TAIL_ONLY>(u, cst->logit_factor + key0, sq, T, key0, e, m_loc, l_loc);
@@ -346,11 +382,9 @@ int pick_heads_per_cta(const AttnArgs& a, int n_z) {
 template <int D, bool Q8, bool TAIL_ONLY>
 cudaError_t launch_k(const AttnArgs& a, int n_z, cudaStream_t stream) {
     using C = Cfg<D>;
-    static bool configured = false;
-    if (!configured) {
+    {   // (the attribute belongs to the current device's copy of the function: set on every launch, it is cheap)
         cudaError_t e = cudaFuncSetAttribute(attention_sm100_kernel<D, Q8, TAIL_ONLY>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::TOTAL);
         if (e != cudaSuccess) return e;
-        configured = true;
     }
     const int hg = pick_heads_per_cta<D>(a, n_z);
     dim3 grid((a.n_query + ROWS - 1) / ROWS, a.heads / hg, n_z);
