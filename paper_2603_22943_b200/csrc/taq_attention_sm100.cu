@@ -11,11 +11,15 @@
 //   warp 9     one thread fetches each head's K~/V~ operand image (written once per prompt by the K/V projection)
 //              with a single bulk copy, one head ahead.
 // Two CTAs share an SM for head widths up to 80, so one CTA's loads overlap the other's arithmetic.
+#include "taq_prof.cuh"
 #include "taq_ptx.cuh"
 #include "taq_sm100.cuh"
 #include "taq_sm100_parts.cuh"
+#include <cstring>
 
 namespace taq {
+
+TAQ_PROF_DEFINE(attention)
 
 namespace {
 
@@ -47,7 +51,16 @@ struct Cfg {
     static constexpr bool SPLIT_KV = KVBUF == 1;
     static constexpr int CST_SLOT = 384;
     static constexpr int OFF_CST = OFF_P + 2 * A_BLOCK;
-    static constexpr int OFF_MISC = OFF_CST + (SPLIT_KV ? 3 * CST_SLOT : 0);
+    // Wide heads move Q~ and O by TMA through one staging buffer (a row's codes or outputs of one head are 80 to 320
+    // bytes at a stride of the whole channel width: per-thread global accesses of that shape keep the load/store
+    // unit busy for longer than the arithmetic takes).  The buffer holds the next head's raw Q~ tile until it has been
+    // expanded into the operand tile, then the previous head's O tile until the store has read it; int8 codes get a
+    // second, smaller buffer, so that their load never waits for the store.
+    static constexpr bool TMA_IO = D >= 80;
+    static constexpr int OFF_U = OFF_CST + (SPLIT_KV ? 3 * CST_SLOT : 0);
+    static constexpr int UO_BYTES = ROWS * D * 2;                  // an O tile, or a raw fp16 Q tile
+    static constexpr int U_BYTES = TMA_IO ? UO_BYTES + ROWS * D : 0; // + a raw int8 Q~ tile, which then has a buffer of its own
+    static constexpr int OFF_MISC = OFF_U + U_BYTES;
     static constexpr int TOTAL = OFF_MISC + 4096 + 128 + 1024;   // misc block + slack for 1024-byte alignment
     static constexpr uint32_t TMEM_S = 0, TMEM_O = 2 * TP;
     static constexpr uint32_t TMEM_COLS = (2 * TP + OBUF * DP) <= 256 ? 256 : 512;
@@ -57,7 +70,7 @@ struct Cfg {
 };
 
 struct Misc {
-    uint64_t kv_full[2], kv_free[2], q_full, s_full[2], p_full, o_full[2], drain;
+    uint64_t kv_full[2], kv_free[2], q_full, s_full[2], p_full, o_full[2], drain, qraw_full;
     uint32_t tmem_base;
     volatile int abort_flag;
     float2 xchg[2][2][ROWS];     // [head parity][half][row]: (max, sum) of a thread's half of the softmax
@@ -100,7 +113,7 @@ struct QRegs {
 };
 
 template <int D, bool Q8, bool TAIL_ONLY>
-__global__ void __launch_bounds__(ATT_THREADS, Cfg<D>::CTAS_PER_SM) attention_sm100_kernel(const AttnArgs a, const int heads_per_cta) {
+__global__ void __launch_bounds__(ATT_THREADS, Cfg<D>::CTAS_PER_SM) attention_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_o, const AttnArgs a, const int heads_per_cta) {
     using C = Cfg<D>;
     constexpr int DP = C::DP;
     extern __shared__ unsigned char smem_dyn[];
@@ -115,6 +128,8 @@ __global__ void __launch_bounds__(ATT_THREADS, Cfg<D>::CTAS_PER_SM) attention_sm
     const int h_begin = blockIdx.y * heads_per_cta;
     const int HG = heads_per_cta;
 
+    TAQ_PROF_INIT
+    if (tid == 0) { TAQ_PROF(0); TAQ_GPROF(126); }
     if (tid == 0) {
         for (int i = 0; i < 2; ++i) {
             ptx::mbar_init(&misc->kv_full[i], 1);
@@ -125,6 +140,7 @@ __global__ void __launch_bounds__(ATT_THREADS, Cfg<D>::CTAS_PER_SM) attention_sm
         ptx::mbar_init(&misc->q_full, ROW_WARPS);      // one arrival per row warp
         ptx::mbar_init(&misc->p_full, ROW_WARPS);
         ptx::mbar_init(&misc->drain, 1);
+        ptx::mbar_init(&misc->qraw_full, 1);
         misc->abort_flag = 0;
         ptx::mbar_fence_init();
     }
@@ -192,6 +208,7 @@ __global__ void __launch_bounds__(ATT_THREADS, Cfg<D>::CTAS_PER_SM) attention_sm
             if (!wait(&misc->kv_full[buf], C::SPLIT_KV ? (hi & 1) : (hi / C::KVBUF) & 1) || !wait(&misc->q_full, hi & 1)) return false;
             ptx::tc_fence_after_sync();
             if (leader) {
+                if (hi < 8) TAQ_PROF(80 + hi);
                 const uint32_t k_lo = kv_lo0 + buf * (C::HEAD_BYTES >> 4);
 #pragma unroll
                 for (int ks = 0; ks < DP / 16; ++ks)
@@ -207,6 +224,7 @@ __global__ void __launch_bounds__(ATT_THREADS, Cfg<D>::CTAS_PER_SM) attention_sm
             if (!wait(&misc->p_full, hi & 1)) return false;
             ptx::tc_fence_after_sync();
             if (leader) {
+                if (hi < 8) TAQ_PROF(96 + hi);
                 const uint32_t vt_lo = kv_lo0 + ((buf * C::HEAD_BYTES + C::K_BYTES) >> 4);
 #pragma unroll
                 for (int ks = 0; ks < TP / 16; ++ks)
@@ -254,7 +272,170 @@ __global__ void __launch_bounds__(ATT_THREADS, Cfg<D>::CTAS_PER_SM) attention_sm
         constexpr int OC = DP / 2;                       // O columns per thread
         bool alive = true;
         ptx::pdl_wait();                                 // Q~ comes from the previous kernel in the stream
+        if (tid == 0) TAQ_PROF(1);
 
+        if constexpr (C::TMA_IO) {
+            // ---- Q~ in and O out by TMA through the staging buffer U ----
+            // Every warp walks every barrier of the loop, whatever happened to its waits: a warp whose wait ran out
+            // skips the work, never a barrier.
+            unsigned char* U = smem + C::OFF_U;
+            constexpr bool SEPQ = Q8;                        // the raw Q~ tile has its own buffer
+            unsigned char* UQ = SEPQ ? U + C::UO_BYTES : U;
+            constexpr int QESZ = Q8 ? 1 : 2;
+            constexpr uint32_t QRAW_BYTES = (uint32_t)(ROWS * D * QESZ);
+            auto all256 = [&]() { asm volatile("bar.sync 5, 256;" ::: "memory"); };
+            auto load_q = [&](int hi) {          // one thread: raw Q~ tile of head hi (rows beyond n_query read as zero)
+                ptx::mbar_arrive_expect_tx(&misc->qraw_full, QRAW_BYTES);
+                ptx::tma_load_3d(UQ, &tmap_q, &misc->qraw_full, (h_begin + hi) * D, row0, zb);
+            };
+            // raw tile of head hi -> fp16 operand tile.  The 16-byte chunks of the tile are dealt out in linear order (thread t
+            // takes chunks t, t + 256, ...): consecutive lanes read consecutive words of the raw tile and write the eight
+            // chunk slots of a swizzled operand row, both free of bank conflicts.
+            auto stage_q_u = [&](int hi) {
+                static_assert(D % 8 == 0 && (ROWS * (D / 8)) % 256 == 0, "chunks per thread");
+                constexpr int CPR = D / 8;                   // chunks per row
+                alive = alive && __all_sync(0xffffffffu, ptx::mbar_wait(&misc->qraw_full, hi & 1) && !misc->abort_flag);
+                if (alive) {
+                    uint4 t16[ROWS * CPR / 256];
+#pragma unroll
+                    for (int i = 0; i < ROWS * CPR / 256; ++i) {
+                        const int j = tid + 256 * i;
+                        if (Q8) t16[i] = codes_w8_to_half(*reinterpret_cast<const uint2*>(UQ + (size_t)j * 8));
+                        else t16[i] = *reinterpret_cast<const uint4*>(UQ + (size_t)j * 16);
+                    }
+#pragma unroll
+                    for (int i = 0; i < ROWS * CPR / 256; ++i) {
+                        const int j = tid + 256 * i;
+                        const int row = j / CPR, cc = j - row * CPR;
+                        *reinterpret_cast<uint4*>(smem + C::OFF_Q + (cc >> 3) * C::A_BLOCK + ptx::sw128_offset(row, cc & 7)) = t16[i];
+                    }
+                    ptx::fence_proxy_async_smem();
+                }
+                __syncwarp();
+                if (alive && lane == 0) ptx::mbar_arrive(&misc->q_full);
+            };
+            // this thread's half of O of head hi: acc / 255 -> fp16 into U (the dense [128][D] tile)
+            auto stage_o_u = [&](int hi) {
+                const uint32_t t_o = tmem_base + C::TMEM_O + (hi % C::OBUF) * DP + half * OC + lane_addr;
+                uint32_t v[OC / 8][8];
+#pragma unroll
+                for (int i = 0; i < OC / 8; ++i) ptx::tmem_ld8(t_o + i * 8, v[i]);
+                ptx::tmem_ld_wait(v[0]);
+#pragma unroll
+                for (int i = 1; i < OC / 8; ++i) ptx::reg_fence8(v[i]);
+#pragma unroll
+                for (int i = 0; i < OC / 8; ++i) {
+                    if (half * OC + i * 8 < D) {
+                        uint32_t pk[4];
+#pragma unroll
+                        for (int e2 = 0; e2 < 4; ++e2) {
+                            __half2 hv = __floats2half2_rn(__uint_as_float(v[i][2 * e2]) * inv255, __uint_as_float(v[i][2 * e2 + 1]) * inv255);
+                            pk[e2] = *reinterpret_cast<uint32_t*>(&hv);
+                        }
+                        *reinterpret_cast<uint4*>(U + ((size_t)r * D + half * OC + i * 8) * 2) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    }
+                }
+                ptx::tc_fence_before_sync();
+                ptx::fence_proxy_async_smem();
+            };
+            auto send_o = [&](int hi) {          // one thread, after the barrier that follows stage_o_u
+                ptx::tma_store_3d(&tmap_o, U, (h_begin + hi) * D, row0, zb);
+                ptx::bulk_store_commit();
+            };
+
+            if (tid == 0) load_q(0);
+            float sq = 1.0f, sq_next = 1.0f;
+            if (Q8) sq = valid ? __ldg(a.q_scales + grow * H + h_begin) : 0.f;
+            stage_q_u(0);
+            all256();                                        // U has been read by everybody
+            if (tid == 0 && HG > 1) load_q(1);
+
+            for (int hi = 0; hi < HG; ++hi) {
+                const uint32_t ph = hi & 1;
+                const bool more = hi + 1 < HG;
+                if (Q8 && more) sq_next = valid ? __ldg(a.q_scales + grow * H + h_begin + hi + 1) : 0.f;
+                alive = alive && __all_sync(0xffffffffu, ptx::mbar_wait(&misc->s_full[ph], (hi >> 1) & 1) && !misc->abort_flag);
+                if (tid == 0 && hi < 8) TAQ_PROF(16 + hi);
+                float e[HK];
+                float k255 = 0.f;
+                unsigned long long trig = 0;
+                if (alive) {
+                    ptx::tc_fence_after_sync();
+                    uint32_t u[HK];
+                    {
+                        const uint32_t t_s = tmem_base + C::TMEM_S + ph * TP + key0 + lane_addr;
+                        uint32_t (&u8)[HK / 8][8] = *reinterpret_cast<uint32_t (*)[HK / 8][8]>(&u);
+#pragma unroll
+                        for (int i = 0; i < HK / 8; ++i) ptx::tmem_ld8(t_s + i * 8, u8[i]);
+                        ptx::tmem_ld_wait(u8[0]);
+#pragma unroll
+                        for (int i = 1; i < HK / 8; ++i) ptx::reg_fence8(u8[i]);
+                    }
+                    ptx::tc_fence_before_sync();
+                    const OperandConsts* cst = C::SPLIT_KV ? reinterpret_cast<const OperandConsts*>(smem + C::OFF_CST + (hi % 3) * C::CST_SLOT)
+                                                           : reinterpret_cast<const OperandConsts*>(smem + C::OFF_KV + (hi % C::KVBUF) * C::HEAD_BYTES + C::K_BYTES + C::VT_BYTES);
+                    float m_loc, l_loc;
+                    softmax_half<TAIL_ONLY>(u, cst->logit_factor + key0, sq, T, key0, e, m_loc, l_loc);
+                    trig = half == 0 ? ((unsigned long long)cst->trig_bits[0] | ((unsigned long long)(cst->trig_bits[1] & 0xFFu) << 32))
+                                     : ((unsigned long long)(cst->trig_bits[1] >> 8) | ((unsigned long long)cst->trig_bits[2] << 24));
+                    misc->xchg[ph][half][r] = make_float2(m_loc, l_loc);
+                    asm volatile("bar.sync %0, 64;" ::"r"(1 + q4) : "memory");
+                    const float2 other = misc->xchg[ph][half ^ 1][r];
+                    const float m_all = fmaxf(m_loc, other.x);
+                    const float c_self = ex2_approx(m_loc - m_all), c_other = ex2_approx(other.x - m_all);
+                    k255 = __fdividef(pmax * c_self, fmaf(l_loc, c_self, other.y * c_other));
+                } else {
+                    asm volatile("bar.sync %0, 64;" ::"r"(1 + q4) : "memory");
+                }
+                // S of this head is complete, so the Q~ operand tile is free: expand the next head's codes, which have had
+                // the softmax to arrive
+                if (tid == 128 && hi < 8) TAQ_PROF(104 + hi);
+                if (more) stage_q_u(hi + 1);
+                if (tid == 0 && hi < 8) TAQ_PROF(32 + hi);
+                if (tid == 128 && hi < 8) TAQ_PROF(112 + hi);
+                if (SEPQ && tid == 0) ptx::bulk_store_wait_read();      // (the store of the head before last: long done)
+                all256();                                    // the raw tile has been read by everybody, U by the store
+                if (SEPQ && tid == 0 && hi + 2 < HG && alive) load_q(hi + 2);
+                if (hi > 0) {                                // O of the previous head: TMEM -> U -> global (TMA store)
+                    alive = alive && __all_sync(0xffffffffu, ptx::mbar_wait(&misc->o_full[(hi - 1) % C::OBUF], ((hi - 1) / C::OBUF) & 1) && !misc->abort_flag);
+                    if (alive) {
+                        ptx::tc_fence_after_sync();
+                        stage_o_u(hi - 1);
+                    }
+                    all256();
+                    if (tid == 0 && alive) send_o(hi - 1);
+                }
+                if (tid == 0 && hi < 8) TAQ_PROF(48 + hi);
+                if (alive) {
+                    write_p_half(e, k255, trig, smem + C::OFF_P, C::A_BLOCK, r, half * (HK / 8));
+                    ptx::fence_proxy_async_smem();
+                    ptx::tc_fence_before_sync();
+                }
+                __syncwarp();
+                if (alive && lane == 0) ptx::mbar_arrive(&misc->p_full);
+                if (tid == 0 && hi < 8) TAQ_PROF(64 + hi);
+                if (!SEPQ && tid == 0) {                     // shared buffer: once the store has read it, the raw tile of the head after next may land
+                    ptx::bulk_store_wait_read();
+                    if (hi + 2 < HG && alive) load_q(hi + 2);
+                }
+                sq = sq_next;
+            }
+            alive = alive && __all_sync(0xffffffffu, ptx::mbar_wait(&misc->o_full[(HG - 1) % C::OBUF], ((HG - 1) / C::OBUF) & 1) && !misc->abort_flag);
+            if (SEPQ) {                                      // the store of the head before must have read U
+                if (tid == 0) ptx::bulk_store_wait_read();
+                all256();
+            }
+            if (alive) {
+                ptx::tc_fence_after_sync();
+                stage_o_u(HG - 1);
+            }
+            all256();
+            if (tid == 0) {
+                if (alive) send_o(HG - 1);
+                ptx::bulk_store_wait_read();
+            }
+            if (!alive) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; }
+        } else {
         auto store_o = [&](int hi) {        // this thread's half of O of head hi: acc / 255 -> fp16
             __half* orow = a.o + grow * Cch + (h_begin + hi) * D + half * OC;
             const uint32_t t_o = tmem_base + C::TMEM_O + (hi % C::OBUF) * DP + half * OC + lane_addr;
@@ -304,6 +485,7 @@ __global__ void __launch_bounds__(ATT_THREADS, Cfg<D>::CTAS_PER_SM) attention_sm
             }
             alive = __all_sync(0xffffffffu, ptx::mbar_wait(&misc->s_full[ph], (hi >> 1) & 1) && !misc->abort_flag);
             if (!alive) break;
+            if (tid == 0 && hi < 8) TAQ_PROF(16 + hi);
             ptx::tc_fence_after_sync();
             uint32_t u[HK];
             {
@@ -316,7 +498,6 @@ __global__ void __launch_bounds__(ATT_THREADS, Cfg<D>::CTAS_PER_SM) attention_sm
                 for (int i = 1; i < HK / 8; ++i) ptx::reg_fence8(u8[i]);
             }
             ptx::tc_fence_before_sync();
-            if (more) stage_q(qr);              // S of this head is complete, so the Q~ tile is free again
 
             // ---- this thread's half of the softmax; the row's two threads then exchange (max, sum) ----
             const OperandConsts* cst = C::SPLIT_KV ? reinterpret_cast<const OperandConsts*>(smem + C::OFF_CST + (hi % 3) * C::CST_SLOT)
@@ -333,6 +514,10 @@ __global__ void __launch_bounds__(ATT_THREADS, Cfg<D>::CTAS_PER_SM) attention_sm
             const float c_self = ex2_approx(m_loc - m_all), c_other = ex2_approx(other.x - m_all);
             const float k255 = __fdividef(pmax * c_self, fmaf(l_loc, c_self, other.y * c_other));
 
+            // S of this head is complete, so the Q~ tile is free again; the next head's codes, asked for at the top of this
+            // iteration, have had the softmax to arrive
+            if (more) stage_q(qr);
+            if (tid == 0 && hi < 8) TAQ_PROF(32 + hi);
             // the P tile is free once the previous head's PV has completed
             if (hi > 0) {
                 alive = __all_sync(0xffffffffu, ptx::mbar_wait(&misc->o_full[(hi - 1) % C::OBUF], ((hi - 1) / C::OBUF) & 1) && !misc->abort_flag);
@@ -340,11 +525,13 @@ __global__ void __launch_bounds__(ATT_THREADS, Cfg<D>::CTAS_PER_SM) attention_sm
                 ptx::tc_fence_after_sync();
                 if (C::OBUF == 1) store_o(hi - 1);   // one O accumulator: empty it before the next PV may start
             }
+            if (tid == 0 && hi < 8) TAQ_PROF(48 + hi);
             write_p_half(e, k255, trig, smem + C::OFF_P, C::A_BLOCK, r, half * (HK / 8));
             ptx::fence_proxy_async_smem();
             ptx::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(&misc->p_full);
+            if (tid == 0 && hi < 8) TAQ_PROF(64 + hi);
 
             if (hi > 0 && C::OBUF == 2) store_o(hi - 1);    // under this head's PV
             sq = sq_next;
@@ -357,14 +544,32 @@ __global__ void __launch_bounds__(ATT_THREADS, Cfg<D>::CTAS_PER_SM) attention_sm
             }
         }
         if (!alive) { raise_status(a.status, TAQ_ERR_TIMEOUT); misc->abort_flag = 1; }
+        }
     }
 
+    if (tid == 0) TAQ_PROF(9);
     ptx::tc_fence_before_sync();
     __syncthreads();
+    if (tid == 0) TAQ_GPROF(127);
     if (warp == MMA_WARP) {
         ptx::tc_fence_after_sync();
         ptx::tmem_dealloc(tmem_base, C::TMEM_COLS);
     }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn3() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess && qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
 }
 
 template <int D>
@@ -388,7 +593,23 @@ cudaError_t launch_k(const AttnArgs& a, int n_z, cudaStream_t stream) {
     }
     const int hg = pick_heads_per_cta<D>(a, n_z);
     dim3 grid((a.n_query + ROWS - 1) / ROWS, a.heads / hg, n_z);
-    return launch_pdl(attention_sm100_kernel<D, Q8, TAIL_ONLY>, grid, dim3(ATT_THREADS), (size_t)C::TOTAL, stream, a, hg);
+    CUtensorMap tmap_q, tmap_o;
+    memset(&tmap_q, 0, sizeof(tmap_q));
+    memset(&tmap_o, 0, sizeof(tmap_o));
+    if (C::TMA_IO) {      // Q~ and O as [n_z][n_query][channels] in boxes of 128 rows x one head
+        EncodeTiledFn enc = encode_tiled_fn3();
+        if (!enc) return cudaErrorNotSupported;
+        const cuuint64_t qesz = Q8 ? 1 : 2;
+        const cuuint64_t dims[3] = {(cuuint64_t)a.channels, (cuuint64_t)a.n_query, (cuuint64_t)n_z};
+        const cuuint64_t qstr[2] = {(cuuint64_t)a.channels * qesz, (cuuint64_t)a.channels * qesz * (cuuint64_t)a.n_query};
+        const cuuint64_t ostr[2] = {(cuuint64_t)a.channels * 2, (cuuint64_t)a.channels * 2 * (cuuint64_t)a.n_query};
+        const cuuint32_t box[3] = {(cuuint32_t)D, ROWS, 1}, estr[3] = {1, 1, 1};
+        if (enc(&tmap_q, Q8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<void*>(a.q), dims, qstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) return cudaErrorInvalidValue;
+        if (enc(&tmap_o, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, (void*)a.o, dims, ostr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) return cudaErrorInvalidValue;
+    }
+    return launch_pdl(attention_sm100_kernel<D, Q8, TAIL_ONLY>, grid, dim3(ATT_THREADS), (size_t)C::TOTAL, stream, tmap_q, tmap_o, a, hg);
 }
 
 template <int D>
