@@ -9,8 +9,10 @@
 //              their partial maximum and sum once per head), epilogue of the previous head;
 //   warp 8     one thread issues the MMAs: S of head h+1 is in flight while the rows are in the softmax of head h;
 //   warp 9     one thread fetches each head's K~/V~ operand image (written once per prompt by the K/V projection)
-//              with a single bulk copy, one head ahead.
-// Two CTAs share an SM for head widths up to 80, so one CTA's loads overlap the other's arithmetic.
+//              by bulk copies, one head ahead: the whole image into the second buffer (head widths up to 64), or,
+//              with a single buffer, K~ as soon as this head's S is complete and V~^T as soon as its PV is.
+// Head widths up to 64: two CTAs share an SM, and the row threads read Q~ and write O themselves.  Head widths 80 and
+// 160: one CTA per SM; Q~ tiles arrive and O tiles leave by TMA through a staging buffer.
 #include "taq_prof.cuh"
 #include "taq_ptx.cuh"
 #include "taq_sm100.cuh"
