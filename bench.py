@@ -285,7 +285,8 @@ def _workload_line(metric, workload, layers, ms, rep, per_step, steps, n_sets, p
 def run_other_workload(args):
     """The other measured configurations (not the headline line): `config1`, the SD-1.5 lowest-resolution layer (W8);
     `config3`, one SD-1.5 UNet step of all 16 cross-attention layers; `config4`, the two SDXL-shaped layers (one line
-    each); `config5`, the multi-checkpoint serving sweep on the 64x64 layer.  One GPU."""
+    each); `config5`, the multi-checkpoint serving sweep on the 64x64 layer; `attention`, taq_cross_attention alone at
+    three launches of many CTAs (one line each, HBM roofline).  One GPU."""
     import torch
     from paper_2603_22943_b200 import binding as tb
     from paper_2603_22943_b200 import synth
@@ -296,6 +297,60 @@ def run_other_workload(args):
     l2 = torch.cuda.get_device_properties(0).L2_cache_size
     sampler = ClockSampler(0)
     sampler.start()
+    if args.workload == "attention":
+        # taq_cross_attention alone at launches of many CTAs: Q~ codes and scales in, O out (the HBM-bound stage)
+        lines = []
+        for B, N, C_, H, Dc in ((64, 256, 1280, 8, 768), (16, 1024, 640, 8, 768), (32, 4096, 320, 8, 768)):
+            T = 77
+            desc = tb.layer_desc(B, N, C_, H, T, Dc, 4, 128, q_bits=8, max_trigger=2)
+            r = np.random.default_rng(7)
+            wd = tb.weight_desc(C_, Dc, 4, 128)
+            Wk = tb.taq_pack_weights(wd, dev((r.standard_normal((C_, Dc)) / np.sqrt(Dc)).astype(np.float32)))
+            Wv = tb.taq_pack_weights(wd, dev((r.standard_normal((C_, Dc)) / np.sqrt(Dc)).astype(np.float32)))
+            m = np.zeros((B, T), np.uint8)
+            m[:, 4:6] = 1
+            mask = dev(m)
+            kv = tb.taq_kv_project(desc, dev(r.standard_normal((B, T, Dc)).astype(np.float16)), Wk, Wv, mask)
+            img = tb.taq_kv_layout_of(desc).operand_head_bytes * H * B
+            nbytes = B * N * (C_ + 4 * H) + B * N * C_ * 2 + img          # Q~ codes + scales, O, operand images
+            n_sets = max(3, int(np.ceil(2.2 * l2 / nbytes)))
+            sets = [(torch.randint(-127, 128, (B * N, C_), dtype=torch.int8, device="cuda"), torch.rand((B * N, H), device="cuda") * 0.05,
+                     torch.empty((B, N, C_), dtype=torch.float16, device="cuda")) for _ in range(n_sets)]
+
+            def step(i, sets=sets, desc=desc, kv=kv, mask=mask, n_sets=n_sets):
+                q, qs, o = sets[i % n_sets]
+                tb.taq_cross_attention(desc, q, qs, kv, mask, o)
+
+            steps = max(n_sets, 12)
+            for i in range(8):
+                step(i)
+            torch.cuda.synchronize()
+            tb.taq_dispatch_reset()
+            step(0)
+            torch.cuda.synchronize()
+            counts = tb.taq_dispatch_counts()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=torch.cuda.Stream()):
+                for i in range(steps):
+                    step(i)
+            rep = time_replays(torch, g, min_total_ms=200.0)
+            ms = rep["median"] / steps
+            gbs = nbytes / (ms * 1e-3) / 1e9
+            lines.append({"metric": "TAQ attention queries/s (taq_cross_attention alone)", "value": B * N / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": steps,
+                          "warmup": 8, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f16", "data": "synthetic",
+                          "config": {"workload": f"attention: B={B} N={N} C={C_} H={H} d={C_ // H} T=77, int8 Q~ per (row, head), trigger {{4,5}}",
+                                     "l2_policy": f"ring of {n_sets} buffer sets ({n_sets * nbytes / 1e6:.0f} MB)"},
+                          "timing": {"replays": rep["replays"], "ms_per_step_min": rep["min"] / steps, "ms_per_step_max": rep["max"] / steps},
+                          "kernel_launches_per_step": counts, "gpu_launches": steps,
+                          "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
+                                       "traffic": None, "bytes_per_launch": nbytes, "peak_source": peaks["source"]}})
+            del sets
+        tb.taq_poll_device_status()
+        clocks = sampler.stop()
+        for line in lines:
+            line["clocks"] = clocks
+            print(json.dumps(line), flush=True)
+        return
     if args.workload in ("config1", "config3", "config4"):
         if args.workload == "config1":
             cases = [("TAQ cross-attn queries/s per layer", "config1: SD-1.5 8x8 cross-attn layer, B=1 N=64 C=1280 H=8 d=160 T=77 Dc=768, W8 per-channel, trigger {5}",
@@ -393,8 +448,8 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=10.0, help="CPU time to spend on the cpu_baseline sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--n-query", type=int, default=0, help="override N (profiling on a smaller case)")
-    ap.add_argument("--workload", default="config2", choices=["config1", "config2", "config3", "config4", "config5"],
-                    help="config2 (default) is the headline line; the others print the other measured configurations (config4: one line per SDXL layer)")
+    ap.add_argument("--workload", default="config2", choices=["config1", "config2", "config3", "config4", "config5", "attention"],
+                    help="config2 (default) is the headline line; the others print the other measured configurations (config4: one line per SDXL layer; attention: one line per shape)")
     args = ap.parse_args()
     if args.workload != "config2":
         run_other_workload(args)
@@ -621,7 +676,7 @@ def main():
          "bytes": 2 * M * C_ * 2 + wbytes, "flops": 2 * M * C_ * C_, "traffic": None},
         {"name": "linear_sm100_kernel<160>: to_q dequant-GEMM + Q_a epilogue, stand-alone (taq_quantized_linear)", "ms": stage_ms["to_q"], "in_step": False,
          "bytes": M * C_ * 2 + qbytes + wbytes, "flops": 2 * M * C_ * C_, "traffic": None},
-        {"name": "attention_sm100_kernel<40>: attention, stand-alone (taq_cross_attention)", "ms": stage_ms["attn"], "in_step": False,
+        {"name": "layer_c320_kernel<.,false,Q given>: attention, stand-alone (taq_cross_attention)", "ms": stage_ms["attn"], "in_step": False,
          "bytes": qbytes + M * C_ * 2 + img_bytes, "flops": 4 * M * T * C_, "traffic": None},
         {"name": "qattn_c320_kernel<.,true,int8>: integer-activation layer pass in one kernel, Q_a(X) and Q_a(O) inside the CTA (taq_layer_forward_a8)", "ms": stage_ms["layer_a8"],
          "in_step": False, "bytes": 2 * M * C_ * 2 + 2 * wbytes + img_bytes, "flops": 4 * M * C_ * C_ + 4 * M * T * C_, "traffic": None},
