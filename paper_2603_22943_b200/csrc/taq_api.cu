@@ -104,7 +104,10 @@ static taq_status run_linear(const LinearArgs& a, int n_z, cudaStream_t st) {
 
 static taq_status run_attention(const AttnArgs& a, int n_z, cudaStream_t st) {
     cudaError_t e;
-    if (sm100_attention_c320_supported(a)) { count_launch(TAQ_KERNEL_ATTENTION_TENSOR); e = launch_attention_c320(a, n_z, st); }
+    // C = 320 / 8 heads: up to one wave of CTAs the head-parallel kernel (four heads of a row tile at once) is the shorter
+    // chain; beyond that the per-head kernel, which keeps two CTAs on an SM, has the higher throughput.
+    const long long c320_ctas = (long long)((a.n_query + 127) / 128) * 2 * n_z;
+    if (c320_ctas <= 148 && sm100_attention_c320_supported(a)) { count_launch(TAQ_KERNEL_ATTENTION_TENSOR); e = launch_attention_c320(a, n_z, st); }
     else if (sm100_attention_supported(a)) { count_launch(TAQ_KERNEL_ATTENTION_TENSOR); e = launch_attention_sm100(a, n_z, st); }
     else { count_launch(TAQ_KERNEL_ATTENTION_GENERIC); e = launch_attention_simt(a, n_z, st); }
     return e == cudaSuccess ? TAQ_OK : cuda_fail(e, "attention launch");
