@@ -144,6 +144,8 @@ struct LinearArgs {
                                 // k-block by TMA, expanded by the workers; 0: all codes staged once
     int early_weights;          // the previous kernel in the stream is known not to write the weights: fetch and expand
                                 // them before waiting for it
+    int head_pair;              // (set by the launcher) EPI_Q8_HEAD with heads twice as wide as the tile: the two CTAs whose
+                                // tiles make up a head exchange their rows' absmax through the cluster
     int* status;
 };
 

@@ -58,6 +58,7 @@ struct Bars {
     uint64_t acc_full[MAX_ACC];
     uint64_t acc_free[MAX_ACC];
     uint64_t part_full[8], part_got[8], peer_ready;   // K loop split over a CTA pair: hand-over of the second CTA's partial sums
+    uint64_t pair_full[4], pair_got[4];               // head split over two column tiles: the rows' absmax from / to the other tile's CTA
     uint32_t tmem_base;
     volatile int abort_flag;
 };
@@ -88,8 +89,8 @@ __host__ __device__ inline Plan make_plan(int k_in, int bits, int group, int nst
     p.off_scales_t = p.off_scales + (p.scale_bytes + 127) / 128 * 128;        // [n_groups][BN]
     p.off_bias = p.off_scales_t + (p.scale_bytes + 127) / 128 * 128;
     p.off_xchg = p.off_bias + (p.bias_bytes + 127) / 128 * 128;              // float [2][128]
-    p.off_bars = p.off_xchg + 1024;
-    p.total = p.off_bars + 512 + 1024;        // barriers + slack to align the base to 1024
+    p.off_bars = p.off_xchg + 2048;           // float [2][128] exchange between a row's two threads, [128] out and [128] in for the head pair
+    p.total = p.off_bars + 1024 + 1024;       // barriers + slack to align the base to 1024
     return p;
 }
 
@@ -108,7 +109,7 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
     extern __shared__ unsigned char smem_dyn[];
     unsigned char* smem = smem_dyn + ((1024u - (ptx::smem_u32(smem_dyn) & 1023u)) & 1023u);   // 1024-byte aligned, still provably shared
     const Plan P = make_plan<BN>(a.k_in, a.bits, a.group, nstage, a.w_direct, prebuilt);
-    static_assert(sizeof(Bars) <= 512, "barrier block");
+    static_assert(sizeof(Bars) <= 1024, "barrier block");
     Bars* bars = reinterpret_cast<Bars*>(smem + P.off_bars);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -150,11 +151,15 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
         }
         for (int i = 0; i < 8; ++i) { ptx::mbar_init(&bars->part_full[i], 1); ptx::mbar_init(&bars->part_got[i], 1); }
         ptx::mbar_init(&bars->peer_ready, 1);
+        for (int i = 0; i < 4; ++i) { ptx::mbar_init(&bars->pair_full[i], 1); ptx::mbar_init(&bars->pair_got[i], 1); }
         bars->abort_flag = 0;
         ptx::mbar_fence_init();
         if (SPLIT)                                          // the worker warps whose rows this CTA finishes receive a piece each
             for (int i = 0; i < 8; ++i)
                 if (((i & 3) >> 1) == rank) ptx::mbar_arrive_expect_tx(&bars->part_full[i], 32u * PART_ROW);
+        if (SPLIT && a.head_pair)                           // the TMEM lane quarters whose rows this CTA finishes: (q + 2) & 3 of worker warp q
+            for (int ww = 0; ww < 4; ++ww)
+                if ((ww >> 1) == rank) ptx::mbar_arrive_expect_tx(&bars->pair_full[(ww + 2) & 3], 128u);
         ptx::tma_prefetch_desc(&tmap_x);
     }
     if (warp == 1) ptx::tmem_alloc(&bars->tmem_base, tmem_cols);
@@ -420,7 +425,7 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
             // memories, one barrier per warp) or receives the partner's piece and adds it, so both directions of the
             // exchange run at once and each CTA stores half of the tile.
             const int ww = wt >> 5, wl = wt & 31;
-            const uint32_t peer = (uint32_t)rank ^ 1u;
+            const uint32_t peer = ptx::cluster_ctarank() ^ 1u;   // (clusters are two CTAs along x, times two along y for a head pair)
             const bool keep = ((ww & 3) >> 1) == rank;
             unsigned char* warp_part = smem + (size_t)ww * 32 * PART_ROW;
             float* piece = reinterpret_cast<float*>(warp_part + (size_t)wl * PART_ROW);
@@ -534,6 +539,30 @@ __global__ void __launch_bounds__(NTHREADS, Tile<BN>::CTAS_PER_SM) linear_sm100_
                         xchg[half * 128 + r] = amax;
                         asm volatile("bar.sync 2, 256;" ::: "memory");
                         amax = fmaxf(amax, xchg[(half ^ 1) * 128 + r]);
+                        if (SPLIT && a.head_pair && stores_rows) {
+                            // The head's other 80 channels belong to the CTA next to this one along y (same rows, same
+                            // half of the K loop): each sends its rows' absmax over (one 128-byte copy between the shared
+                            // memories per 32 rows), waits for the other's, and confirms, so that the source outlives the copy.
+                            float* out = xchg + 256, * in = xchg + 384;
+                            const uint32_t other = ptx::cluster_ctarank() ^ 2u;
+                            bool got = true;
+                            if (half == 0) {
+                                out[r] = amax;
+                                ptx::fence_proxy_async_smem();
+                                __syncwarp();
+                                if (lane == 0)
+                                    ptx::bulk_copy_to_cta(ptx::map_to_cta(ptx::smem_u32(in + q * 32), other), out + q * 32, 128u,
+                                                          ptx::map_to_cta(ptx::smem_u32(&bars->pair_full[q]), other));
+                            }
+                            got = ptx::mbar_wait(&bars->pair_full[q], 0);
+                            if (got) amax = fmaxf(amax, in[r]);
+                            asm volatile("bar.sync %0, 64;" ::"r"(7 + q) : "memory");      // both warps of the quarter have read the piece
+                            if (half == 0 && lane == 0) {
+                                ptx::mbar_arrive_cluster_relaxed(ptx::map_to_cta(ptx::smem_u32(&bars->pair_got[q]), other));
+                                got = ptx::mbar_wait(&bars->pair_got[q], 0) && got;
+                            }
+                            if (!got) { raise_status(a.status, TAQ_ERR_TIMEOUT); bars->abort_flag = 1; }
+                        }
                     }
                     const float s = quant_scale(amax, a.epi == EPI_KV && a.kv_qmax ? (float)a.kv_qmax : 127.f);
                     const float rs = s > 0.f ? __frcp_rn(s) : 0.f;
@@ -658,7 +687,12 @@ int nstage_for(const LinearArgs& a, int bn) {
     return 0;
 }
 
-int pick_bn(const LinearArgs& a) {
+// EPI_Q8_HEAD with heads of 160 channels: instead of one 160-wide tile per head (whose expanded weight tiles do not fit
+// resident) two 80-wide tiles whose CTAs exchange the rows' absmax, when that launch is one wave of split tiles with
+// resident weight tiles (clusters of 2 x 2: halves of the K loop along x, halves of the head along y).
+bool head_pair_mode(const LinearArgs& a, int n_z);
+
+int pick_bn(const LinearArgs& a, int n_z = 1) {
     // Every column tile re-reads the activation rows, so tiles are as wide as the row count allows while the grid
     // still covers most of the SMs; a width whose ring and staging do not fit shared memory is passed over.
     const long long row_tiles = (a.rows + BM - 1) / BM;
@@ -667,6 +701,7 @@ int pick_bn(const LinearArgs& a) {
         const int d = a.n_out / a.heads;
         if (d == 40 && a.heads % 4 == 0 && row_tiles * (a.n_out / 160) >= 96 && fits(160)) return 160;   // two heads per worker thread
         if (d == 40 && a.heads % 2 == 0) return fits(80) ? 80 : 0;     // one head per worker thread
+        if (d == 160 && a.epi == EPI_Q8_HEAD && head_pair_mode(a, n_z)) return 80;
         if (d == 64 || d == 80 || d == 160) return fits(d) ? d : 0;   // one head per tile, split between the row's two threads
         return 0;
     }
@@ -721,6 +756,13 @@ Choice choose(const LinearArgs& a, int n_z) {
     return c;
 }
 
+bool head_pair_mode(const LinearArgs& a, int n_z) {
+    if (a.epi != EPI_Q8_HEAD || a.heads <= 0 || a.n_out != a.heads * 160 || a.xq || a.reqs) return false;
+    if (nstage_for(a, 80) < 2) return false;
+    const Choice c = choose<80>(a, n_z);
+    return c.split && c.prebuilt > 0;
+}
+
 template <int BN>
 cudaError_t launch_bn(const CUtensorMap& tmap, EncodeTiledFn enc, LinearArgs a, int n_z, cudaStream_t stream) {
     const bool i8 = a.xq != nullptr;
@@ -731,6 +773,8 @@ cudaError_t launch_bn(const CUtensorMap& tmap, EncodeTiledFn enc, LinearArgs a, 
         split ? (i8 ? linear_sm100_kernel<BN, true, true> : linear_sm100_kernel<BN, false, true>)
               : (i8 ? linear_sm100_kernel<BN, true, false> : linear_sm100_kernel<BN, false, false>);
     a.w_direct = weight_mode<BN>(a);
+    a.head_pair = (BN == 80 && a.epi == EPI_Q8_HEAD && a.n_out == a.heads * 160) ? 1 : 0;
+    if (a.head_pair && !(split && ch.prebuilt)) return cudaErrorNotSupported;
     CUtensorMap tmap_w = tmap;                        // (unused unless w_direct)
     if (a.w_direct) {                                 // the codes section of the blob as an int8 matrix [n_out][k_in]
         const WeightLayout L = weight_layout(a.n_out, a.k_in, a.bits, a.group);
@@ -757,7 +801,7 @@ cudaError_t launch_bn(const CUtensorMap& tmap, EncodeTiledFn enc, LinearArgs a, 
     }
     const Plan P = make_plan<BN>(a.k_in, a.bits, a.group, ns, a.w_direct, ch.prebuilt);
     dim3 grid((unsigned)((a.rows + BM - 1) / BM) * (split ? 2u : 1u), a.n_out / BN, n_z);
-    if (split) return launch_pdl_cluster(kern, grid, dim3(2, 1, 1), dim3(NTHREADS), (size_t)P.total, stream, tmap, tmap_w, tmap_y, a, ns, ch.prebuilt);
+    if (split) return launch_pdl_cluster(kern, grid, dim3(2, a.head_pair ? 2 : 1, 1), dim3(NTHREADS), (size_t)P.total, stream, tmap, tmap_w, tmap_y, a, ns, ch.prebuilt);
     return launch_pdl(kern, grid, dim3(NTHREADS), (size_t)P.total, stream, tmap, tmap_w, tmap_y, a, ns, ch.prebuilt);
 }
 
@@ -830,7 +874,7 @@ cudaError_t launch_linear_sm100(const LinearArgs& a, int n_z, cudaStream_t strea
                      i8 ? (void*)const_cast<int8_t*>(a.xq) : (void*)const_cast<__half*>(a.x), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                      CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
-    switch (pick_bn(a)) {
+    switch (pick_bn(a, n_z)) {
         case 64: return launch_bn<64>(tmap, enc, a, n_z, stream);
         case 80: return launch_bn<80>(tmap, enc, a, n_z, stream);
         case 160: return launch_bn<160>(tmap, enc, a, n_z, stream);
