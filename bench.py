@@ -343,7 +343,8 @@ def run_other_workload(args):
                           "timing": {"replays": rep["replays"], "ms_per_step_min": rep["min"] / steps, "ms_per_step_max": rep["max"] / steps},
                           "kernel_launches_per_step": counts, "gpu_launches": steps,
                           "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
-                                       "traffic": None, "bytes_per_launch": nbytes, "peak_source": peaks["source"]}})
+                                       "traffic": measured_traffic(f"attention_sm100_kernel_d{C_ // H}_b{B}"), "bytes_per_launch": nbytes,
+                                       "peak_source": peaks["source"]}})
             del sets
         tb.taq_poll_device_status()
         clocks = sampler.stop()
