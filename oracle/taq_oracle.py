@@ -23,6 +23,10 @@ fixed by the benchmark configuration: symmetric, dynamic, round-to-nearest-even;
 The quantizer itself is evaluated in IEEE binary32 (numpy float32, no fused multiply-add), because
 integer codes are compared bit for bit; everything else is float64.
 
+Logarithmic quantizer (``p_log``): Table 4 of the paper has "Logarithmic" rows and the text never defines that
+quantizer.  ``quantize_prob_log`` is this reading's definition (power-of-two codes, see its docstring): PARITY
+UNPINNED - its tests check it against closed forms of that definition, not against anything the paper fixes.
+
 Integer activations (``a_bits = 8``): the paper's W/A bit-widths (Table 1, "W/A" column) and its BOPs
 accounting count activation bits for every layer, which read literally means that the inputs of the four
 projections - the hidden states X, the text context and the attention output O - are quantized too.  With
@@ -129,6 +133,19 @@ def quantize_prob(A: np.ndarray, bits: int = 8) -> Tuple[np.ndarray, np.ndarray]
     return code, p_hat.astype(F64)
 
 
+def quantize_prob_log(A: np.ndarray, bits: int = 8) -> Tuple[np.ndarray, np.ndarray]:
+    """Logarithmic quantizer of attention probabilities (the "Logarithmic" rows of Table 4).  The paper names it and
+    never defines it; the reading taken here is the usual power-of-two code for softmax outputs:
+    code = clamp(rint(-log2 p), 0, 2^bits - 1) taken in float32, p^ = 2^-code (p = 0 takes the last code).
+    PARITY UNPINNED: the definition is this reading's, not the paper's.  Returns (codes int32, p^ float64)."""
+    cmax = 2 ** bits - 1
+    p = np.asarray(A, dtype=F32)
+    with np.errstate(divide="ignore"):
+        x = (-np.log2(p)).astype(F32)
+    code = np.where(p > 0, np.clip(np.rint(x), 0, cmax), cmax).astype(np.int32)
+    return code, np.ldexp(F64(1.0), -code)
+
+
 def f16_round(x: np.ndarray) -> np.ndarray:
     """Round to nearest-even fp16, returned as float64."""
     return np.asarray(x).astype(np.float16).astype(F64)
@@ -147,6 +164,7 @@ class TaqConfig:
     kv_bits: int = 8         # 8 / 4 = non-trigger K/V rows int8 / 4-bit (qmax 7); 0 = no K/V quantization at all
     p_bits: int = 8          # 8 / 4 = non-trigger probabilities uint8 / 4-bit (15 levels); 0 = no probability quantization
     a_bits: int = 0          # 8 = inputs of the projections (X, ctx, O) int8 per token; 0 = left in fp16
+    p_log: bool = False      # non-trigger probabilities through the logarithmic quantizer (p_bits levels) instead of the linear one
     contract: bool = True    # fp16 storage roundings on (contract) or off (ideal)
 
 
@@ -240,9 +258,16 @@ def taq_attention(Q_tilde: np.ndarray, K_tilde: np.ndarray, V_tilde: np.ndarray,
     if cfg.p_bits not in (0, 4, 8):
         raise ValueError("p_bits must be 0, 4 or 8")
     pmax = float(2 ** cfg.p_bits - 1) if cfg.p_bits else 255.0
+    if cfg.p_log and cfg.p_bits:
+        pmax = 256.0                                              # power-of-two codes sit on a power-of-two unit
     kept = f16_round(A * pmax) / pmax if cfg.contract else A
     if cfg.p_bits == 0:
         A_hat = np.where(M, kept, A)
+    elif cfg.p_log:
+        _, Aq = quantize_prob_log(A, cfg.p_bits)
+        if cfg.contract:
+            Aq = f16_round(Aq * pmax) / pmax                      # fp16 operand: codes beyond 32 flush to zero
+        A_hat = np.where(M, kept, Aq)
     else:
         _, Aq = quantize_prob(A, cfg.p_bits)
         A_hat = np.where(M, kept, Aq)                             # Eq. 3

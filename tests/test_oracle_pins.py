@@ -128,8 +128,41 @@ def check_prob_quantizer(o):
     np.testing.assert_allclose(Ah, code / 255.0, rtol=0, atol=1e-7)
 
 
+def check_log_prob_quantizer(o):
+    """The logarithmic reading (power-of-two codes; the paper does not define it, so these are closed forms of the
+    reading, not of the paper): exact powers of two are fixed points, the decision boundary between codes k and k + 1
+    is 2^-(k + 1/2), the last code absorbs everything below, and inside a layer the trigger columns bypass it."""
+    p = np.array([1.0, 0.5, 0.25, 2.0 ** -7, 2.0 ** -15, 2.0 ** -40, 0.0])
+    c8, h8 = o.quantize_prob_log(p, 8)
+    assert c8.tolist() == [0, 1, 2, 7, 15, 40, 255] and h8[:6].tolist() == p[:6].tolist()
+    c4, h4 = o.quantize_prob_log(p, 4)
+    assert c4.tolist() == [0, 1, 2, 7, 15, 15, 15] and h4[-1] == 2.0 ** -15
+    for k in range(6):                                            # just above / below the boundary 2^-(k + 1/2)
+        b = 2.0 ** -(k + 0.5)
+        c, _ = o.quantize_prob_log(np.array([b * 1.001, b * 0.999]), 8)
+        assert c.tolist() == [k, k + 1]
+    A = _rng(9).dirichlet(np.ones(77), size=300)
+    c, Ah = o.quantize_prob_log(A, 8)
+    assert np.all(Ah / A <= 2 ** 0.5 * (1 + 1e-6)) and np.all(Ah / A >= 2 ** -0.5 * (1 - 1e-6))   # within half an octave
+    assert np.all(np.log2(Ah) == -c)
+    # inside the layer: ordinary columns take the power-of-two value, trigger columns the fp16 probability
+    X, ctx, Wq, Wk, Wv, Wo, bo = _tiny_layer(12)
+    mask = np.zeros((2, 7), np.uint8)
+    mask[:, 2] = 1
+    cfg = o.TaqConfig(heads=2, w_bits=0, q_bits=0, kv_bits=0, p_bits=8, p_log=True, contract=False)
+    q = o.taq_q(X, Wq, cfg)
+    kv = o.taq_kv(ctx, Wk, Wv, mask, cfg)
+    _, A0, Ahat = o.taq_attention(q["Q_tilde"], kv["K_tilde"], kv["V_tilde"], mask, cfg, return_probs=True)
+    np.testing.assert_array_equal(Ahat[..., 2], A0[..., 2])
+    rest = np.delete(Ahat, 2, axis=-1)
+    assert np.all(np.log2(rest) == np.rint(np.log2(rest)))
+    want = np.exp2(-np.clip(np.rint(-np.log2(np.delete(A0, 2, axis=-1).astype(np.float32))), 0, 255))
+    np.testing.assert_array_equal(rest, want)
+
+
 @pytest.mark.parametrize("check", [check_quantizer_hand_values, check_quantizer_exact_rational,
-                                   check_quantizer_idempotent_and_pow2, check_weight_quantizer, check_prob_quantizer])
+                                   check_quantizer_idempotent_and_pow2, check_weight_quantizer, check_prob_quantizer,
+                                   check_log_prob_quantizer])
 def test_quantizers(check):
     check(orc)
 
@@ -668,6 +701,10 @@ MUTATIONS = {
     "contract_q16_not_rounded": [("Qt = f16_round(Q) if cfg.contract else Q", "Qt = Q")],
     "contract_trigger_rows_not_rounded": [("kept = f16_round(Z) if cfg.contract else Z", "kept = Z")],
     "contract_y_not_rounded": [("    return f16_round(Y) if cfg.contract else Y", "    return Y")],
+    "log_code_floor_instead_of_rint": [("code = np.where(p > 0, np.clip(np.rint(x), 0, cmax), cmax)", "code = np.where(p > 0, np.clip(np.floor(x), 0, cmax), cmax)")],
+    "log_code_not_clamped": [("code = np.where(p > 0, np.clip(np.rint(x), 0, cmax), cmax)", "code = np.where(p > 0, np.rint(x), cmax)")],
+    "log_base_e": [("x = (-np.log2(p)).astype(F32)", "x = (-np.log(p)).astype(F32)")],
+    "log_mask_ignored": [("        A_hat = np.where(M, kept, Aq)\n    else:", "        A_hat = Aq\n    else:")],
     "heads_interleaved": [("return x.reshape(B, L, heads, d).transpose(0, 2, 1, 3)", "return x.reshape(B, L, d, heads).transpose(0, 3, 1, 2)")],
 }
 
@@ -678,7 +715,7 @@ ALL_CHECKS = None
 def test_unmutated_copy_passes_every_pin():
     m = _mutant(text=[])
     for c in [check_quantizer_hand_values, check_quantizer_exact_rational, check_quantizer_idempotent_and_pow2,
-              check_weight_quantizer, check_prob_quantizer] + LAYER_CHECKS:
+              check_weight_quantizer, check_prob_quantizer, check_log_prob_quantizer] + LAYER_CHECKS:
         c(m)
 
 
@@ -686,7 +723,7 @@ def test_unmutated_copy_passes_every_pin():
 def test_planted_mistake_is_caught(name):
     m = _mutant(text=MUTATIONS[name])
     checks = [check_quantizer_hand_values, check_quantizer_exact_rational, check_quantizer_idempotent_and_pow2,
-              check_weight_quantizer, check_prob_quantizer] + LAYER_CHECKS
+              check_weight_quantizer, check_prob_quantizer, check_log_prob_quantizer] + LAYER_CHECKS
     caught = []
     for c in checks:
         try:
