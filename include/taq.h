@@ -107,6 +107,10 @@ typedef struct {
                              of Table 1; stored one code per byte) */
     int32_t p_bits;       /* 8: ordinary probabilities uint8, code = rint(255 p); 4: 16 levels, code = rint(15 p) */
     int32_t max_trigger;  /* capacity of fp16 trigger rows per sequence, 0..n_ctx */
+    int32_t p_log;        /* 0: the linear probability quantizer above.  1: the logarithmic quantizer of Table 4's
+                             "Logarithmic" rows, which the paper names and does not define; the reading taken:
+                             code = clamp(rint(-log2 p), 0, 2^p_bits - 1), p^ = 2^-code, trigger columns fp16 as before.
+                             Layers with p_log = 1 run as separate launches (projection, attention, projection). */
 } taq_layer_desc;
 
 /* Mixed-precision K~/V~ of Eq. 2, one block per sequence, blocks back to back.  Offsets inside a block: */

@@ -45,7 +45,7 @@ class WeightDesc(C.Structure):
 
 class LayerDesc(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("batch", "n_query", "channels", "heads", "n_ctx", "ctx_dim", "w_bits",
-                                          "w_group", "q_bits", "kv_bits", "p_bits", "max_trigger")]
+                                          "w_group", "q_bits", "kv_bits", "p_bits", "max_trigger", "p_log")]
 
     @property
     def d_head(self) -> int:
@@ -167,8 +167,8 @@ def weight_desc(n_out: int, k_in: int, bits: int, group: int) -> WeightDesc:
 
 
 def layer_desc(batch, n_query, channels, heads, n_ctx, ctx_dim, w_bits, w_group, q_bits=8, kv_bits=8, p_bits=8,
-               max_trigger=8) -> LayerDesc:
-    return LayerDesc(batch, n_query, channels, heads, n_ctx, ctx_dim, w_bits, w_group, q_bits, kv_bits, p_bits, max_trigger)
+               max_trigger=8, p_log=0) -> LayerDesc:
+    return LayerDesc(batch, n_query, channels, heads, n_ctx, ctx_dim, w_bits, w_group, q_bits, kv_bits, p_bits, max_trigger, p_log)
 
 
 # ------------------------------------------------------------------------------------------------

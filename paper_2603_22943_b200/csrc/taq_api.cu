@@ -67,6 +67,7 @@ static taq_status check_layer_desc(const taq_layer_desc* d) {
     if (d->q_bits != 0 && d->q_bits != 8) return fail(TAQ_ERR_INVALID_ARG, "q_bits must be 0 or 8, got %d", d->q_bits);
     if (d->kv_bits != 8 && d->kv_bits != 4) return fail(TAQ_ERR_UNSUPPORTED, "kv_bits must be 8 or 4, got %d", d->kv_bits);
     if (d->p_bits != 8 && d->p_bits != 4) return fail(TAQ_ERR_UNSUPPORTED, "p_bits must be 8 or 4, got %d", d->p_bits);
+    if (d->p_log != 0 && d->p_log != 1) return fail(TAQ_ERR_INVALID_ARG, "p_log must be 0 or 1, got %d", d->p_log);
     if (d->max_trigger < 0 || d->max_trigger > d->n_ctx) return fail(TAQ_ERR_SHAPE, "max_trigger must be in [0,n_ctx], got %d", d->max_trigger);
     if ((long long)d->batch * d->n_query > (1LL << 31) - 1) return fail(TAQ_ERR_SHAPE, "batch * n_query too large");
     taq_weight_desc w{d->channels, d->channels, d->w_bits, d->w_group};
@@ -302,7 +303,7 @@ taq_status taq_quantized_linear(const taq_weight_desc* d, const void* x_f16_dev,
 static AttnArgs attn_args(const taq_layer_desc* d, int* status) {
     AttnArgs a{};
     a.batch = d->batch; a.n_query = d->n_query; a.channels = d->channels; a.heads = d->heads; a.n_ctx = d->n_ctx;
-    a.max_trigger = d->max_trigger; a.q_bits = d->q_bits; a.p_bits = d->p_bits;
+    a.max_trigger = d->max_trigger; a.q_bits = d->q_bits; a.p_bits = d->p_bits; a.p_log = d->p_log;
     a.status = status;
     return a;
 }

@@ -108,8 +108,13 @@ __global__ void __launch_bounds__(ATT_WARPS * 32) attention_simt_kernel(const At
             if (j < T) {
                 const float pj = __fdiv_rn(s[u], sum);
                 float ph;
-                const float pmax = a.p_bits == 4 ? 15.0f : 255.0f;                                  // levels of the code: 2^bits - 1
+                const float pmax = a.p_log ? 256.0f : a.p_bits == 4 ? 15.0f : 255.0f;             // the unit of the stored probabilities is 1 / pmax
                 if (msk[j] || a.p_bits == 0) ph = __fdiv_rn(__half2float(__float2half_rn(__fmul_rn(pj, pmax))), pmax);     // Eq. 3, trigger column: fp16 in units of 1/pmax
+                else if (a.p_log) {                                                                  // logarithmic code: p^ = 2^-clamp(rint(-log2 p))
+                    const float cmax = a.p_bits == 4 ? 15.0f : 255.0f;
+                    const float code = pj > 0.f ? fminf(fmaxf(rintf(-log2f(pj)), 0.f), cmax) : cmax;
+                    ph = code <= 32.f ? exp2f(-code) : 0.f;                                          // (an fp16 operand in units of 1/256)
+                }
                 else ph = __fdiv_rn(rintf(__fmul_rn(pj, pmax)), pmax);                               // Eq. 3, integer code / pmax
                 p[j] = ph;
             }

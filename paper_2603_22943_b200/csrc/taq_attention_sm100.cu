@@ -268,7 +268,8 @@ __global__ void __launch_bounds__(ATT_THREADS, Cfg<D>::CTAS_PER_SM) attention_sm
         const size_t grow = (size_t)zb * a.n_query + (valid ? n : 0);
         const uint32_t lane_addr = (uint32_t)(q4 * 32) << 16;
         const int key0 = half * HK;
-        const float pmax = a.p_bits == 4 ? 15.0f : 255.0f;     // probabilities are held in units of 1 / pmax (uint8 or 4-bit codes)
+        const float cmax = a.p_bits == 4 ? 15.0f : 255.0f;     // last code
+        const float pmax = a.p_log ? 256.0f : cmax;            // probabilities are held in units of 1 / pmax (linear codes: 1 / last code)
         const float inv255 = 1.0f / pmax;
         constexpr int CH2 = QRegs<D, Q8>::CH2;
         constexpr int OC = DP / 2;                       // O columns per thread
@@ -409,7 +410,8 @@ __global__ void __launch_bounds__(ATT_THREADS, Cfg<D>::CTAS_PER_SM) attention_sm
                 }
                 if (tid == 0 && hi < 8) TAQ_PROF(48 + hi);
                 if (alive) {
-                    write_p_half(e, k255, trig, smem + C::OFF_P, C::A_BLOCK, r, half * (HK / 8));
+                    if (a.p_log) write_p_half_log(e, k255, cmax, trig, smem + C::OFF_P, C::A_BLOCK, r, half * (HK / 8));
+                    else write_p_half(e, k255, trig, smem + C::OFF_P, C::A_BLOCK, r, half * (HK / 8));
                     ptx::fence_proxy_async_smem();
                     ptx::tc_fence_before_sync();
                 }
@@ -528,7 +530,8 @@ __global__ void __launch_bounds__(ATT_THREADS, Cfg<D>::CTAS_PER_SM) attention_sm
                 if (C::OBUF == 1) store_o(hi - 1);   // one O accumulator: empty it before the next PV may start
             }
             if (tid == 0 && hi < 8) TAQ_PROF(48 + hi);
-            write_p_half(e, k255, trig, smem + C::OFF_P, C::A_BLOCK, r, half * (HK / 8));
+            if (a.p_log) write_p_half_log(e, k255, cmax, trig, smem + C::OFF_P, C::A_BLOCK, r, half * (HK / 8));
+            else write_p_half(e, k255, trig, smem + C::OFF_P, C::A_BLOCK, r, half * (HK / 8));
             ptx::fence_proxy_async_smem();
             ptx::tc_fence_before_sync();
             __syncwarp();

@@ -158,6 +158,7 @@ struct AttnArgs {
     __half* o;                  // [z][B][N][C]
     int batch, n_query, channels, heads, n_ctx, max_trigger;
     int q_bits, p_bits;
+    int p_log;                  // 1: logarithmic probability codes (p^ = 2^-code) instead of the linear ones
     int early_kv;               // the previous kernel in the stream is known not to write the K~/V~ blocks
     int* status;
 };

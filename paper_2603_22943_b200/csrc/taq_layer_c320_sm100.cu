@@ -833,7 +833,7 @@ bool sm100_qattn_supported(const taq_layer_desc& d) {
     if (d.channels != KIN || d.heads * D != KIN) return false;
     if (d.w_bits != 4) return false;
     if (d.w_group != 0 && (d.w_group % BK || (KIN + d.w_group - 1) / d.w_group > MAX_GROUPS)) return false;
-    if (d.n_ctx > TP || (d.p_bits != 8 && d.p_bits != 4)) return false;
+    if (d.n_ctx > TP || (d.p_bits != 8 && d.p_bits != 4) || d.p_log) return false;   // (logarithmic codes: the stand-alone attention kernel)
     if (d.n_query < 1) return false;
     return encode_tiled() != nullptr;
 }
@@ -886,7 +886,7 @@ cudaError_t launch_qattn_sm100(const taq_layer_desc& d, const __half* x, const v
 
 // The attention core alone at the same shape (taq_cross_attention): Q~ given, all four heads of a CTA at once.
 bool sm100_attention_c320_supported(const AttnArgs& a) {
-    if (a.channels != KIN || a.heads * D != KIN || a.n_ctx > TP || (a.p_bits != 8 && a.p_bits != 4) || a.n_query < 1) return false;
+    if (a.channels != KIN || a.heads * D != KIN || a.n_ctx > TP || (a.p_bits != 8 && a.p_bits != 4) || a.p_log || a.n_query < 1) return false;
     if ((reinterpret_cast<uintptr_t>(a.q) & 15u) || (reinterpret_cast<uintptr_t>(a.o) & 15u)) return false;
     return encode_tiled() != nullptr;
 }

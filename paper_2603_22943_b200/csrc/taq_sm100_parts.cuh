@@ -136,6 +136,32 @@ __device__ __forceinline__ void write_p_half(const float (&e)[HK], float k255, u
     }
 }
 
+// The logarithmic reading of the probability quantizer: t = e_j * k is 256 p; ordinary columns take
+// code = clamp(rint(-log2 p), 0, cmax) = clamp(rint(8 - log2 t), 0, cmax) and are stored as the fp16 value 2^(8 - code)
+// (units of 1/256; exact down to the smallest fp16 subnormal at code 32, zero beyond); trigger columns are fp16(t).
+__device__ __forceinline__ uint32_t log_code_to_half_bits(float t, float cmax) {
+    const float x = 8.0f - __log2f(t);                      // t = 0 -> +inf -> the last code
+    const int c = (int)fminf(fmaxf(rintf(x), 0.f), cmax);
+    return c <= 22 ? (uint32_t)(23 - c) << 10 : (c <= 32 ? 1u << (32 - c) : 0u);
+}
+__device__ __forceinline__ void write_p_half_log(const float (&e)[HK], float k256, float cmax, unsigned long long trig, unsigned char* p_tile, int a_block, int r, int chunk0) {
+#pragma unroll
+    for (int g = 0; g < HK / 8; ++g) {
+        const uint32_t bits = (uint32_t)(trig >> (8 * g)) & 0xFFu;
+        uint32_t pk[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int j = g * 8 + 2 * i;
+            const float t0 = e[j] * k256, t1 = e[j + 1] * k256;
+            uint32_t h0 = log_code_to_half_bits(t0, cmax), h1 = log_code_to_half_bits(t1, cmax);
+            if ((bits >> (2 * i)) & 1u) h0 = __half_as_ushort(__float2half_rn(t0));
+            if ((bits >> (2 * i + 1)) & 1u) h1 = __half_as_ushort(__float2half_rn(t1));
+            pk[i] = h0 | (h1 << 16);
+        }
+        const int chunk = chunk0 + g;
+        *reinterpret_cast<uint4*>(p_tile + (chunk >> 3) * a_block + ptx::sw128_offset(r, chunk & 7)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+    }
+}
 
 }  // namespace parts
 }  // namespace taq

@@ -39,6 +39,7 @@ class LayerShape:
     q_bits: int = 8      # 8: Q is quantized (Eq. 2, third line); 0: Q stays unquantized
     kv_bits: int = 8     # 8 or 4: width of the ordinary K/V rows (Table 1 lists 8 and 4)
     p_bits: int = 8      # 8 or 4: width of the ordinary attention probabilities
+    p_log: int = 0       # 1: those probabilities through the logarithmic quantizer (power-of-two codes)
     seed: int = 0
     name: str = ""
 

@@ -48,7 +48,7 @@ def assert_layer_close(got, want, what=""):
 
 def oracle_cfg(shape: synth.LayerShape, contract=True, a_bits=0) -> orc.TaqConfig:
     return orc.TaqConfig(heads=shape.heads, w_bits=shape.w_bits, w_group=shape.w_group, q_bits=shape.q_bits, kv_bits=shape.kv_bits,
-                         p_bits=shape.p_bits, contract=contract, a_bits=a_bits)
+                         p_bits=shape.p_bits, contract=contract, a_bits=a_bits, p_log=bool(shape.p_log))
 
 
 def oracle_layer(shape: synth.LayerShape, data, contract=True, rows=None):
@@ -62,7 +62,7 @@ def gpu_desc(shape: synth.LayerShape, max_trigger=None, batch=None, n_query=None
     mt = max(1, len(shape.trigger)) if max_trigger is None else max_trigger
     return tb.layer_desc(shape.batch if batch is None else batch, shape.n_query if n_query is None else n_query,
                          shape.channels, shape.heads, shape.n_ctx, shape.ctx_dim, shape.w_bits, shape.w_group,
-                         q_bits=shape.q_bits, kv_bits=shape.kv_bits, p_bits=shape.p_bits, max_trigger=mt)
+                         q_bits=shape.q_bits, kv_bits=shape.kv_bits, p_bits=shape.p_bits, max_trigger=mt, p_log=shape.p_log)
 
 
 def pack_layer_weights(shape: synth.LayerShape, data):
