@@ -157,6 +157,16 @@ def test_linear_plan_keeps_every_region_inside_shared_memory(L):
     assert plan["bn"] == 160 and plan["staging_bytes"] == 128 * 160 * 4 and plan["ring_bytes"] >= plan["staging_bytes"]
 
 
+def test_linear_plan_of_heads_of_160_channels(L):
+    """Per-head Q_a over heads of 160 channels: up to one wave of split tiles the projection runs on 80-wide tiles (two
+    per head, resident weight tiles); beyond that on one 160-wide tile per head."""
+    wd = tb.weight_desc(1280, 1280, 4, 128)
+    assert tb.taq_linear_plan(wd, 512, tb.TAQ_OUT_INT8_HEAD_ROWS, heads=8)["bn"] == 80
+    assert tb.taq_linear_plan(wd, 64, tb.TAQ_OUT_INT8_HEAD_ROWS, heads=8)["bn"] == 80
+    assert tb.taq_linear_plan(wd, 1300, tb.TAQ_OUT_INT8_HEAD_ROWS, heads=8)["bn"] == 160
+    assert tb.taq_linear_plan(tb.weight_desc(1280, 1280, 8, 0), 64, tb.TAQ_OUT_INT8_HEAD_ROWS, heads=8)["bn"] == 160   # W8: codes too large to stage
+
+
 def test_dispatch_counters_start_at_zero_and_reset(L):
     tb.taq_dispatch_reset()
     assert set(tb.taq_dispatch_counts().values()) == {0}

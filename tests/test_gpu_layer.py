@@ -83,6 +83,9 @@ def test_kv_project_trigger_capacity_overflow_raises_device_status():
     (1000, 640, 640, 4, 128, 10),     # SDXL d=64
     (513, 1280, 1280, 4, 128, 20),
     (130, 640, 640, 4, 128, 8),       # d=80
+    (512, 1280, 1280, 4, 128, 8),     # d=160: a head over two 80-wide tiles, absmax exchanged through the cluster
+    (130, 1280, 1280, 4, 128, 8),     # the same, ragged row tile
+    (1300, 1280, 1280, 4, 128, 8),    # d=160 beyond one wave: one 160-wide tile per head
     (5, 16, 8, 4, 0, 2), (1, 64, 64, 8, 0, 1), (77, 96, 72, 4, 0, 4),
 ])
 def test_quantized_linear(rows, n_out, k_in, bits, group, heads):
